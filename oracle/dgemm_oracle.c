@@ -1,0 +1,103 @@
+/*
+ * dgemm_oracle.c -- CPU oracle for C += A*B in IEEE binary64 (TEST INFRASTRUCTURE ONLY).
+ *
+ * See dgemm_oracle.h for the semantics and the list of pins. Build with
+ *   gcc -O2 -fno-fast-math -ffp-contract=off -fopenmp -shared -fPIC
+ * so that the compiler neither reassociates sums nor contracts a*b+c into an fma: the
+ * operation sequence per output element is exactly the one of the paper's naive nest
+ * (Section 2.1, "Affine Ops": load a, load b, load c, multiply, add, store c).
+ *
+ * Nothing here is blocked, packed, unrolled or otherwise tuned, on purpose.
+ */
+#include "dgemm_oracle.h"
+
+#include <math.h>
+#include <stddef.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+/* The definition: for i, for j, for k: C[i][j] = C[i][j] + A[i][k]*B[k][j]. */
+void dgemm_oracle_ijk(int64_t M, int64_t N, int64_t K,
+                      const double *A, int64_t lda,
+                      const double *B, int64_t ldb,
+                      double *C, int64_t ldc)
+{
+    for (int64_t i = 0; i < M; ++i) {
+        for (int64_t j = 0; j < N; ++j) {
+            for (int64_t k = 0; k < K; ++k) {
+                double a = A[i * lda + k];
+                double b = B[k * ldb + j];
+                double ci = C[i * ldc + j];
+                volatile double p = a * b; /* separately rounded product (mulf) */
+                double co = ci + p;        /* separately rounded sum (addf)     */
+                C[i * ldc + j] = co;
+            }
+        }
+    }
+}
+
+/*
+ * Interchanged order i, k, j. For a fixed (i,j) the updates still happen for k = 0, 1, ...,
+ * K-1 in that order and each one is c = c + a*b with two roundings, so every element sees
+ * the operation sequence of the definition. Rows are independent: one row per OpenMP task.
+ */
+void dgemm_oracle_ikj(int64_t M, int64_t N, int64_t K,
+                      const double *A, int64_t lda,
+                      const double *B, int64_t ldb,
+                      double *C, int64_t ldc, int threads)
+{
+#ifdef _OPENMP
+    int nt = threads > 0 ? threads : omp_get_max_threads();
+#pragma omp parallel for schedule(static) num_threads(nt)
+#else
+    (void)threads;
+#endif
+    for (int64_t i = 0; i < M; ++i) {
+        double *c = C + i * ldc;
+        for (int64_t k = 0; k < K; ++k) {
+            const double a = A[i * lda + k];
+            const double *b = B + k * ldb;
+            for (int64_t j = 0; j < N; ++j) {
+                c[j] = c[j] + a * b[j]; /* -ffp-contract=off: multiply, then add */
+            }
+        }
+    }
+}
+
+void dgemm_oracle_entries(int64_t K,
+                          const double *A, int64_t lda,
+                          const double *B, int64_t ldb,
+                          const double *Cin, int64_t ldc,
+                          int64_t nsamples, const int64_t *ii, const int64_t *jj,
+                          int absolute, double *out, int threads)
+{
+#ifdef _OPENMP
+    int nt = threads > 0 ? threads : omp_get_max_threads();
+#pragma omp parallel for schedule(static) num_threads(nt)
+#else
+    (void)threads;
+#endif
+    for (int64_t s = 0; s < nsamples; ++s) {
+        const int64_t i = ii[s], j = jj[s];
+        double c = Cin ? Cin[i * ldc + j] : 0.0;
+        if (absolute) c = fabs(c);
+        for (int64_t k = 0; k < K; ++k) {
+            double a = A[i * lda + k];
+            double b = B[k * ldb + j];
+            if (absolute) { a = fabs(a); b = fabs(b); }
+            volatile double p = a * b;
+            c = c + p;
+        }
+        out[s] = c;
+    }
+}
+
+int dgemm_oracle_max_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}

@@ -1,0 +1,148 @@
+/*
+ * dgemm.h -- C ABI of libdgemm: double-precision C += A*B for NVIDIA B200 (sm_100a).
+ *
+ * The operation is the one the paper studies throughout (Section 2.1 "Affine Ops": the
+ * comment and body of the naive nest, "C += A * B" on f64 operands; Section 2.15, question 4:
+ * alpha = beta = 1 is assumed). Matrices are row-major with the identity layout map of
+ * Section 2.2 "MemRefs": element (i,j) of a matrix with leading dimension ld lives at
+ * base[i*ld + j]; a leading dimension larger than the row length expresses the padded layout
+ * (d0,d1) -> (d0*ld + d1) of Section 2.11, whose padding can never be accessed.
+ *
+ * Plain C types only. All functions return a dgemm_status (0 = success, negative = error)
+ * unless stated otherwise. Error returns never launch work.
+ */
+#ifndef DGEMM_H
+#define DGEMM_H
+
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define DGEMM_API __attribute__((visibility("default")))
+#else
+#define DGEMM_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  DGEMM_OK = 0,
+  DGEMM_ERR_BAD_DIM = -1, /* M, N or K < 0, or a dimension beyond 2^31-1 rows/cols            */
+  DGEMM_ERR_BAD_LD = -2,  /* lda < max(1,K), ldb < max(1,N) or ldc < max(1,N)                  */
+  DGEMM_ERR_NULL = -3,    /* a needed pointer is NULL                                          */
+  DGEMM_ERR_ALIGN = -4,   /* a pointer is not 8-byte aligned                                   */
+  DGEMM_ERR_ALIAS = -5,   /* the byte range of C overlaps that of A or B                       */
+  DGEMM_ERR_DEVICE = -6,  /* no CUDA device, or the current device is not compute capability 10 */
+  DGEMM_ERR_CUDA = -7,    /* a CUDA runtime/driver call failed (launch, copy, allocation)      */
+  DGEMM_ERR_TIMEOUT = -8, /* a bounded device-side wait gave up (device status word)           */
+  DGEMM_ERR_VARIANT = -9, /* unknown variant, or the forced variant cannot run these operands  */
+  DGEMM_ERR_SIZE = -10    /* a fixed-capacity entry point was given a problem beyond its limit */
+} dgemm_status;
+
+/* Kernel variants (dgemm_set_variant). The ladder mirrors the paper's step-by-step journey
+ * (Sections 2.3-2.9): a naive nest first, then tiling + staging ("packing") + register tiling. */
+enum {
+  DGEMM_VARIANT_AUTO = -1,   /* choose by operand alignment and problem shape (default)         */
+  DGEMM_VARIANT_NAIVE = 0,   /* one thread per C element, k sequential (the naive nest on a GPU) */
+  DGEMM_VARIANT_TMA = 1,     /* DMMA pipeline, operand tiles staged by TMA; needs 16-byte aligned
+                                A and B base pointers and even lda, ldb                          */
+  DGEMM_VARIANT_GENERIC = 2, /* same pipeline, tiles staged by 8-byte asynchronous copies; any
+                                8-byte aligned operands and any leading dimensions               */
+  DGEMM_VARIANT_COUNT = 3
+};
+
+/*
+ * C[i][j] += sum_k A[i][k] * B[k][j] for 0 <= i < M, 0 <= j < N (Section 2.1, naive nest;
+ * alpha = beta = 1, Section 2.15).
+ *
+ *   A  device pointer, M x K, row-major, leading dimension lda >= max(1,K); read only
+ *   B  device pointer, K x N, row-major, leading dimension ldb >= max(1,N); read only
+ *   C  device pointer, M x N, row-major, leading dimension ldc >= max(1,N); read and written
+ *   stream  a cudaStream_t passed as void*; NULL is the legacy default stream
+ *
+ * All three buffers live on the current CUDA device and stay owned by the caller; the library
+ * neither retains nor frees them. The call is asynchronous: work is enqueued on `stream` and
+ * the function returns without synchronising. Arithmetic is IEEE binary64 with fused
+ * multiply-adds, round to nearest even; each entry's sum is accumulated from +0 in ascending
+ * k (inside one k-split) and the incoming C value is added last, so the result equals the
+ * definition's within 2*K*2^-53*(|A||B|)_ij and exactly when every partial sum is exactly
+ * representable (e.g. small-integer data).
+ *
+ * Only A[i][k<K], B[k][j<N] and C[i][j<N] are ever read and only C[i<M][j<N] is written:
+ * padding beyond the logical row is neither read into the result nor modified.
+ * M == 0 or N == 0: returns DGEMM_OK without inspecting pointers. K == 0: returns DGEMM_OK and
+ * leaves C untouched. A and B may alias each other; C must not overlap A or B (checked on byte
+ * ranges, DGEMM_ERR_ALIAS). Pointers must be 8-byte aligned; a faster path is taken when A and
+ * B are 16-byte aligned with even lda and ldb.
+ *
+ * Problems with few output tiles split K over several thread blocks; their partial sums go
+ * through a library-owned per-device workspace that is allocated on first need (a synchronising
+ * cudaMalloc; do that first call outside stream capture) and is shared by all calls, which are
+ * therefore serialised on the device in stream order only when they use the same stream.
+ * Thread-safety: concurrent calls from several host threads are allowed; calls that need the
+ * split-K workspace must not overlap on the device.
+ */
+DGEMM_API int dgemm_f64(int64_t M, int64_t N, int64_t K,
+              const double *A, int64_t lda,
+              const double *B, int64_t ldb,
+              double *C, int64_t ldc,
+              void *stream);
+
+/*
+ * Same operation with HOST buffers (pageable or pinned): copies A, B and C to device scratch
+ * memory, runs dgemm_f64 there and copies C back (only the M x N logical part of each row is
+ * meaningful; padding columns of the host C are preserved). Synchronous: returns after the
+ * result is in the host buffer. Device scratch is allocated with the stream-ordered allocator
+ * and released before returning. Same argument rules and error codes as dgemm_f64
+ * (Section 2.1; the paper's driver likewise owns A, B, C in host memory).
+ */
+DGEMM_API int dgemm_f64_host(int64_t M, int64_t N, int64_t K,
+                   const double *A, int64_t lda,
+                   const double *B, int64_t ldb,
+                   double *C, int64_t ldc);
+
+/* Human-readable text for a status code; never NULL; static storage. */
+DGEMM_API const char *dgemm_strerror(int status);
+
+/* Library version as major*10000 + minor*100 + patch. */
+DGEMM_API int dgemm_version(void);
+
+/*
+ * Force one kernel variant for subsequent calls of this process (ablation and tests; the
+ * paper's analogue is re-running with other pass flags, Section 2.10), or DGEMM_VARIANT_AUTO.
+ * Returns DGEMM_OK or DGEMM_ERR_VARIANT. A forced variant that cannot run given operands
+ * (DGEMM_VARIANT_TMA on unaligned ones) makes dgemm_f64 return DGEMM_ERR_VARIANT.
+ */
+DGEMM_API int dgemm_set_variant(int variant);
+
+/* Force a split-K factor (>= 1) for the pipelined variants, or 0 for the built-in heuristic. */
+DGEMM_API int dgemm_set_split_k(int split_k);
+
+/*
+ * Synchronises `stream`, then reads and clears the current device's status word. Returns
+ * DGEMM_OK if no kernel reported a problem since the last call, DGEMM_ERR_TIMEOUT if a bounded
+ * wait inside a kernel ran out (the kernel then stopped early and C is unspecified), or
+ * DGEMM_ERR_CUDA if the synchronisation itself failed.
+ */
+DGEMM_API int dgemm_last_device_status(void *stream);
+
+/*
+ * Number of kernels this library has launched so far in this process (all entry points).
+ * Monotonic; used by the benchmark to report launches per step.
+ */
+DGEMM_API int64_t dgemm_launch_count(void);
+
+/*
+ * Measures the FP64 issue rate of the current device with a register-only loop of dependent
+ * mma.sync m16n8k8 f64 instructions on all SMs for about `millis` milliseconds (the roofline
+ * denominator; the paper computes its machine peak from unit counts in Section 1.2 and this is
+ * the measured counterpart). Writes the fused multiply-adds per clock per SM to *fma_per_clk_sm
+ * and the sustained rate in TFLOP/s to *tflops (either may be NULL). Synchronous.
+ */
+DGEMM_API int dgemm_fp64_peak_probe(int millis, double *fma_per_clk_sm, double *tflops);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DGEMM_H */

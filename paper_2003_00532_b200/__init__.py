@@ -1,0 +1,25 @@
+"""B200-native FP64 GEMM ``C += A @ B`` (row-major) behind the C ABI of ``libdgemm``.
+
+The Python layer only marshals arguments; every step of the computation runs in the CUDA
+kernels of ``csrc/``. The library is loaded lazily on first use and its absence is an error.
+"""
+from .binding import (  # noqa: F401
+    DGEMM_OK,
+    DGEMM_VARIANT_AUTO,
+    DGEMM_VARIANT_GENERIC,
+    DGEMM_VARIANT_NAIVE,
+    DGEMM_VARIANT_TMA,
+    DgemmError,
+    dgemm_f64,
+    dgemm_f64_host,
+    dgemm_f64_raw,
+    dgemm_fp64_peak_probe,
+    dgemm_last_device_status,
+    dgemm_launch_count,
+    dgemm_set_split_k,
+    dgemm_set_variant,
+    dgemm_strerror,
+    dgemm_version,
+    lib_path,
+    load_library,
+)

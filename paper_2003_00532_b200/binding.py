@@ -1,0 +1,187 @@
+"""ctypes binding of ``libdgemm.so``: same names as the C ABI in ``include/dgemm.h``.
+
+Argument marshalling only. Matrices are passed as 2-D float64 ``torch`` tensors with unit
+column stride (the row stride is the leading dimension, so a view ``buf[:, :cols]`` of a wider
+buffer expresses padding) or as raw integer addresses with explicit sizes. There is no CPU or
+library fallback: if the shared library is missing, loading fails with an error.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import threading
+from typing import Optional
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libdgemm.so")
+_lock = threading.Lock()
+_lib: Optional[ctypes.CDLL] = None
+
+DGEMM_OK = 0
+DGEMM_ERR_BAD_DIM = -1
+DGEMM_ERR_BAD_LD = -2
+DGEMM_ERR_NULL = -3
+DGEMM_ERR_ALIGN = -4
+DGEMM_ERR_ALIAS = -5
+DGEMM_ERR_DEVICE = -6
+DGEMM_ERR_CUDA = -7
+DGEMM_ERR_TIMEOUT = -8
+DGEMM_ERR_VARIANT = -9
+DGEMM_ERR_SIZE = -10
+
+DGEMM_VARIANT_AUTO = -1
+DGEMM_VARIANT_NAIVE = 0
+DGEMM_VARIANT_TMA = 1
+DGEMM_VARIANT_GENERIC = 2
+
+
+class DgemmError(RuntimeError):
+    """A libdgemm call returned a negative status."""
+
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {dgemm_strerror(status)} (status {status})")
+
+
+def lib_path() -> str:
+    return _LIB_PATH
+
+
+def load_library() -> ctypes.CDLL:
+    """Load ``libdgemm.so`` (built in-tree by ``build.py``). Raises if it is absent."""
+    global _lib
+    with _lock:
+        if _lib is None:
+            if not os.path.exists(_LIB_PATH):
+                raise FileNotFoundError(
+                    f"{_LIB_PATH} not found: build it with `python -m paper_2003_00532_b200.build` "
+                    "(nvcc, sm_100a); there is no fallback path")
+            lib = ctypes.CDLL(_LIB_PATH)
+            i64, vp = ctypes.c_int64, ctypes.c_void_p
+            lib.dgemm_f64.argtypes = [i64, i64, i64, vp, i64, vp, i64, vp, i64, vp]
+            lib.dgemm_f64.restype = ctypes.c_int
+            lib.dgemm_f64_host.argtypes = [i64, i64, i64, vp, i64, vp, i64, vp, i64]
+            lib.dgemm_f64_host.restype = ctypes.c_int
+            lib.dgemm_strerror.argtypes = [ctypes.c_int]
+            lib.dgemm_strerror.restype = ctypes.c_char_p
+            lib.dgemm_version.argtypes = []
+            lib.dgemm_version.restype = ctypes.c_int
+            lib.dgemm_set_variant.argtypes = [ctypes.c_int]
+            lib.dgemm_set_variant.restype = ctypes.c_int
+            lib.dgemm_set_split_k.argtypes = [ctypes.c_int]
+            lib.dgemm_set_split_k.restype = ctypes.c_int
+            lib.dgemm_last_device_status.argtypes = [vp]
+            lib.dgemm_last_device_status.restype = ctypes.c_int
+            lib.dgemm_launch_count.argtypes = []
+            lib.dgemm_launch_count.restype = ctypes.c_int64
+            lib.dgemm_fp64_peak_probe.argtypes = [ctypes.c_int, ctypes.POINTER(ctypes.c_double),
+                                                  ctypes.POINTER(ctypes.c_double)]
+            lib.dgemm_fp64_peak_probe.restype = ctypes.c_int
+            _lib = lib
+    return _lib
+
+
+def _matrix_args(x, name: str, want_cuda: bool):
+    """(address, rows, cols, ld) of a 2-D float64 tensor with unit column stride."""
+    import torch
+    if not isinstance(x, torch.Tensor):
+        raise TypeError(f"{name}: expected a torch.Tensor")
+    if x.dtype != torch.float64 or x.dim() != 2:
+        raise TypeError(f"{name}: need a 2-D float64 tensor")
+    if x.is_cuda != want_cuda:
+        raise ValueError(f"{name}: expected a {'CUDA' if want_cuda else 'host'} tensor")
+    rows, cols = x.shape
+    if rows > 0 and cols > 0 and x.stride(1) != 1:
+        raise ValueError(f"{name}: columns must be contiguous (row-major)")
+    ld = max(cols, 1)
+    if rows >= 1 and cols > 0 and x.stride(0) >= ld:
+        ld = x.stride(0)  # a one-row view keeps its buffer's leading dimension
+    return x.data_ptr(), rows, cols, ld
+
+
+def _stream_handle(stream) -> Optional[int]:
+    if stream is None:
+        import torch
+        return torch.cuda.current_stream().cuda_stream or None
+    if isinstance(stream, int):
+        return stream or None
+    return stream.cuda_stream or None
+
+
+def _shapes(A, B, C, cuda: bool):
+    pa, M, K, lda = _matrix_args(A, "A", cuda)
+    pb, K2, N, ldb = _matrix_args(B, "B", cuda)
+    pc, M2, N2, ldc = _matrix_args(C, "C", cuda)
+    if K != K2 or M != M2 or N != N2:
+        raise ValueError(f"shape mismatch: A {tuple(A.shape)}, B {tuple(B.shape)}, C {tuple(C.shape)}")
+    return M, N, K, pa, lda, pb, ldb, pc, ldc
+
+
+def dgemm_f64(A, B, C, stream=None, check: bool = True) -> int:
+    """``C += A @ B`` on the current CUDA device, asynchronously on ``stream``.
+
+    ``A`` (M x K), ``B`` (K x N), ``C`` (M x N): CUDA float64 tensors, row-major, row stride =
+    leading dimension. ``stream``: a ``torch.cuda.Stream``, a raw ``cudaStream_t`` integer, or
+    ``None`` for torch's current stream. Returns the status; raises ``DgemmError`` on a negative
+    status unless ``check=False``.
+    """
+    M, N, K, pa, lda, pb, ldb, pc, ldc = _shapes(A, B, C, True)
+    return dgemm_f64_raw(M, N, K, pa, lda, pb, ldb, pc, ldc, _stream_handle(stream), check)
+
+
+def dgemm_f64_raw(M, N, K, A_ptr, lda, B_ptr, ldb, C_ptr, ldc, stream: Optional[int] = None,
+                  check: bool = True) -> int:
+    """The C entry point with raw addresses (device pointers as integers)."""
+    rc = load_library().dgemm_f64(M, N, K, A_ptr, lda, B_ptr, ldb, C_ptr, ldc, stream)
+    if check and rc < 0:
+        raise DgemmError(rc, "dgemm_f64")
+    return rc
+
+
+def dgemm_f64_host(A, B, C, check: bool = True) -> int:
+    """``C += A @ B`` with HOST tensors: the library copies to the device, computes there and
+    copies the result back into ``C``. Synchronous."""
+    M, N, K, pa, lda, pb, ldb, pc, ldc = _shapes(A, B, C, False)
+    rc = load_library().dgemm_f64_host(M, N, K, pa, lda, pb, ldb, pc, ldc)
+    if check and rc < 0:
+        raise DgemmError(rc, "dgemm_f64_host")
+    return rc
+
+
+def dgemm_strerror(status: int) -> str:
+    return load_library().dgemm_strerror(int(status)).decode()
+
+
+def dgemm_version() -> int:
+    return int(load_library().dgemm_version())
+
+
+def dgemm_set_variant(variant: int) -> int:
+    rc = load_library().dgemm_set_variant(int(variant))
+    if rc < 0:
+        raise DgemmError(rc, "dgemm_set_variant")
+    return rc
+
+
+def dgemm_set_split_k(split_k: int) -> int:
+    rc = load_library().dgemm_set_split_k(int(split_k))
+    if rc < 0:
+        raise DgemmError(rc, "dgemm_set_split_k")
+    return rc
+
+
+def dgemm_last_device_status(stream=None) -> int:
+    return int(load_library().dgemm_last_device_status(_stream_handle(stream)))
+
+
+def dgemm_launch_count() -> int:
+    return int(load_library().dgemm_launch_count())
+
+
+def dgemm_fp64_peak_probe(millis: int = 200):
+    """Returns ``(fma_per_clk_sm, tflops)`` measured by the register-only DMMA loop."""
+    a, b = ctypes.c_double(0.0), ctypes.c_double(0.0)
+    rc = load_library().dgemm_fp64_peak_probe(int(millis), ctypes.byref(a), ctypes.byref(b))
+    if rc < 0:
+        raise DgemmError(rc, "dgemm_fp64_peak_probe")
+    return a.value, b.value

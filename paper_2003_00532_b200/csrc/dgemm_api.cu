@@ -1,0 +1,373 @@
+// Host side of libdgemm: argument validation, variant choice, tensor-map creation and launch.
+// Exports the C ABI declared in include/dgemm.h. Links only against the CUDA runtime; the one
+// driver entry point needed (cuTensorMapEncodeTiled) is obtained through the runtime.
+#include "../../include/dgemm.h"
+
+#include <atomic>
+#include <cstdint>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <mutex>
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include "dgemm_dmma.cuh"
+
+namespace {
+
+using namespace dgemm;
+
+constexpr int kMaxDevices = 64;
+constexpr size_t kWorkspaceBytes = 320ull * BM * BN * sizeof(double);  // 40 MiB: up to 320 partial tiles
+constexpr unsigned long long kWaitLimitNs = 4000000000ull;            // 4 s per device-side wait
+
+__device__ int g_status_word;  // one per device that loads the library
+
+struct DeviceState {
+  bool ready = false;
+  int sm_count = 0;
+  int* status = nullptr;       // device address of g_status_word
+  double* workspace = nullptr; // split-K partial tiles, allocated on first need
+};
+
+DeviceState g_dev[kMaxDevices];
+std::mutex g_mutex;
+std::atomic<int> g_variant{DGEMM_VARIANT_AUTO};
+std::atomic<int> g_split_k{0};
+std::atomic<long long> g_launches{0};
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn g_encode = nullptr;
+
+// Per-device set-up, once: capability check, SM count, status-word address, shared-memory opt-in.
+int device_state(DeviceState** out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+    (void)cudaGetLastError();
+    return DGEMM_ERR_DEVICE;
+  }
+  std::lock_guard<std::mutex> lock(g_mutex);
+  DeviceState& st = g_dev[dev];
+  if (!st.ready) {
+    int major = 0, sms = 0;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+      (void)cudaGetLastError();
+      return DGEMM_ERR_DEVICE;
+    }
+    if (major != 10) return DGEMM_ERR_DEVICE;
+    if (cudaGetSymbolAddress(reinterpret_cast<void**>(&st.status), g_status_word) != cudaSuccess) return DGEMM_ERR_CUDA;
+    if (cudaMemset(st.status, 0, sizeof(int)) != cudaSuccess) return DGEMM_ERR_CUDA;
+    if (cudaFuncSetAttribute(dgemm_dmma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess ||
+        cudaFuncSetAttribute(dgemm_dmma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
+      return DGEMM_ERR_CUDA;
+    if (!g_encode) {
+      void* fn = nullptr;
+      cudaDriverEntryPointQueryResult qres;
+      if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+          qres != cudaDriverEntryPointSuccess || !fn)
+        return DGEMM_ERR_CUDA;
+      g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+    }
+    st.sm_count = sms;
+    st.ready = true;
+  }
+  *out = &st;
+  return DGEMM_OK;
+}
+
+int ensure_workspace(DeviceState* st) {
+  std::lock_guard<std::mutex> lock(g_mutex);
+  if (!st->workspace) {
+    if (cudaMalloc(reinterpret_cast<void**>(&st->workspace), kWorkspaceBytes) != cudaSuccess) {
+      (void)cudaGetLastError();
+      return DGEMM_ERR_CUDA;
+    }
+  }
+  return DGEMM_OK;
+}
+
+// 2-D f64 tensor map: inner extent `cols` (contiguous), outer extent `rows` with stride ld
+// doubles; box = box_cols x box_rows; 128-byte swizzle; out-of-range elements read as zero.
+bool make_map(CUtensorMap* map, const double* base, int64_t rows, int64_t cols, int64_t ld, int box_cols, int box_rows) {
+  const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)ld * sizeof(double)};
+  const cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  return g_encode(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT64, 2, const_cast<double*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+bool ranges_overlap(const void* p, int64_t pbytes, const void* q, int64_t qbytes) {
+  const uintptr_t a = (uintptr_t)p, b = (uintptr_t)q;
+  return a < b + (uintptr_t)qbytes && b < a + (uintptr_t)pbytes;
+}
+
+// Everything that can be decided without touching the device. Returns 1 for "nothing to do".
+int validate(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, const double* B, int64_t ldb,
+             const double* C, int64_t ldc) {
+  const int64_t kMaxDim = (int64_t)INT32_MAX - 2 * BM;
+  if (M < 0 || N < 0 || K < 0 || M > kMaxDim || N > kMaxDim || K > kMaxDim) return DGEMM_ERR_BAD_DIM;
+  if (M == 0 || N == 0) return 1;
+  if (lda < (K > 0 ? K : 1) || ldb < N || ldc < N) return DGEMM_ERR_BAD_LD;
+  if (K == 0) return 1;
+  if (!A || !B || !C) return DGEMM_ERR_NULL;
+  if (((uintptr_t)A | (uintptr_t)B | (uintptr_t)C) & 7) return DGEMM_ERR_ALIGN;
+  const int64_t abytes = ((M - 1) * lda + K) * 8, bbytes = ((K - 1) * ldb + N) * 8, cbytes = ((M - 1) * ldc + N) * 8;
+  if (ranges_overlap(C, cbytes, A, abytes) || ranges_overlap(C, cbytes, B, bbytes)) return DGEMM_ERR_ALIAS;
+  const int64_t tiles = ((M + BM - 1) / BM) * ((N + BN - 1) / BN);
+  if (tiles > (int64_t)INT32_MAX / 512) return DGEMM_ERR_BAD_DIM;
+  return DGEMM_OK;
+}
+
+int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, const double* B, int64_t ldb,
+                double* C, int64_t ldc, cudaStream_t stream) {
+  DeviceState* st = nullptr;
+  int rc = device_state(&st);
+  if (rc != DGEMM_OK) return rc;
+
+  int variant = g_variant.load();
+  const bool tma_ok = (((uintptr_t)A | (uintptr_t)B) & 15) == 0 && (lda % 2 == 0) && (ldb % 2 == 0);
+  if (variant == DGEMM_VARIANT_AUTO) variant = tma_ok ? DGEMM_VARIANT_TMA : DGEMM_VARIANT_GENERIC;
+  if (variant == DGEMM_VARIANT_TMA && !tma_ok) return DGEMM_ERR_VARIANT;
+
+  if (variant == DGEMM_VARIANT_NAIVE) {
+    dim3 block(32, 8), grid((unsigned)((N + 31) / 32), (unsigned)((M + 7) / 8));
+    dgemm_naive_kernel<<<grid, block, 0, stream>>>((int)M, (int)N, (int)K, A, lda, B, ldb, C, ldc);
+    g_launches.fetch_add(1);
+    return cudaGetLastError() == cudaSuccess ? DGEMM_OK : DGEMM_ERR_CUDA;
+  }
+
+  GemmParams p;
+  memset(&p, 0, sizeof(p));
+  p.M = (int)M; p.N = (int)N; p.K = (int)K;
+  p.tiles_m = (int)((M + BM - 1) / BM);
+  p.tiles_n = (int)((N + BN - 1) / BN);
+  p.A = A; p.B = B; p.C = C;
+  p.lda = lda; p.ldb = ldb; p.ldc = ldc;
+  p.wait_limit_ns = kWaitLimitNs;
+  p.status = st->status;
+  p.group_m = 8;
+
+  const int tiles = p.tiles_m * p.tiles_n;
+  const int kblocks = (int)((K + BK - 1) / BK);
+  int split = g_split_k.load();
+  if (split <= 0) {
+    // Split K only when the output tiles cannot occupy the SMs; keep at least 4 k-blocks per part.
+    split = 1;
+    if (tiles * 2 <= st->sm_count) {
+      split = st->sm_count / tiles;
+      if (split > kblocks / 4) split = kblocks / 4;
+      if (split < 1) split = 1;
+    }
+  }
+  if (split > kblocks) split = kblocks;
+  const int max_partials = (int)(kWorkspaceBytes / (BM * BN * sizeof(double)));
+  if ((int64_t)split * tiles > max_partials) split = max_partials / tiles;
+  if (split < 1) split = 1;
+  p.kblocks_per_split = (kblocks + split - 1) / split;
+  p.split_k = (kblocks + p.kblocks_per_split - 1) / p.kblocks_per_split;  // no empty partitions
+  if (p.split_k > 1) {
+    rc = ensure_workspace(st);
+    if (rc != DGEMM_OK) return rc;
+    p.partial = st->workspace;
+  }
+
+  const int units = tiles * p.split_k;
+  const int grid = units < st->sm_count ? units : st->sm_count;
+
+  CUtensorMap map_a, map_b;
+  memset(&map_a, 0, sizeof(map_a));
+  memset(&map_b, 0, sizeof(map_b));
+  if (variant == DGEMM_VARIANT_TMA) {
+    if (!make_map(&map_a, A, M, K, lda, BK, BM) || !make_map(&map_b, B, K, N, ldb, 16, BK)) return DGEMM_ERR_CUDA;
+    dgemm_dmma_kernel<true><<<grid, THREADS, SMEM_BYTES, stream>>>(map_a, map_b, p);
+  } else {
+    dgemm_dmma_kernel<false><<<grid, THREADS, SMEM_BYTES, stream>>>(map_a, map_b, p);
+  }
+  g_launches.fetch_add(1);
+  if (cudaGetLastError() != cudaSuccess) return DGEMM_ERR_CUDA;
+  if (p.split_k > 1) {
+    dgemm_splitk_reduce_kernel<<<tiles, 256, 0, stream>>>(p);
+    g_launches.fetch_add(1);
+    if (cudaGetLastError() != cudaSuccess) return DGEMM_ERR_CUDA;
+  }
+  return DGEMM_OK;
+}
+
+// ---- FP64 issue-rate probe -------------------------------------------------------------------
+
+__global__ void __launch_bounds__(256) fp64_probe_kernel(double* out, long long* cycles, int iters, double seed) {
+  double c[8][4];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) { c[i][0] = i; c[i][1] = threadIdx.x; c[i][2] = 1.0; c[i][3] = 2.0; }
+  const double a0 = seed, a1 = seed * 0.5, a2 = seed * 0.25, a3 = seed * 0.125, b0 = 1.0 - seed, b1 = 0.5 - seed;
+  const long long t0 = clock64();
+  for (int it = 0; it < iters; ++it) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) ptx::dmma_m16n8k8(c[i], a0, a1, a2, a3, b0, b1);
+  }
+  const long long t1 = clock64();
+  double r = 0.0;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) r += c[i][0] + c[i][1] + c[i][2] + c[i][3];
+  out[blockIdx.x * blockDim.x + threadIdx.x] = r;
+  if (threadIdx.x == 0) cycles[blockIdx.x] = t1 - t0;
+}
+
+}  // namespace
+
+extern "C" {
+
+int dgemm_f64(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, const double* B, int64_t ldb, double* C,
+              int64_t ldc, void* stream) {
+  const int v = validate(M, N, K, A, lda, B, ldb, C, ldc);
+  if (v == 1) return DGEMM_OK;
+  if (v != DGEMM_OK) return v;
+  return launch_gemm(M, N, K, A, lda, B, ldb, C, ldc, static_cast<cudaStream_t>(stream));
+}
+
+int dgemm_f64_host(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, const double* B, int64_t ldb,
+                   double* C, int64_t ldc) {
+  const int v = validate(M, N, K, A, lda, B, ldb, C, ldc);
+  if (v == 1) return DGEMM_OK;
+  if (v != DGEMM_OK) return v;
+  DeviceState* st = nullptr;
+  int rc = device_state(&st);
+  if (rc != DGEMM_OK) return rc;
+
+  // dense device copies with even leading dimensions (keeps the TMA path available)
+  const int64_t dlda = K + (K & 1), dldb = N + (N & 1), dldc = N + (N & 1);
+  cudaStream_t s = nullptr;
+  double *dA = nullptr, *dB = nullptr, *dC = nullptr;
+  rc = DGEMM_ERR_CUDA;
+  do {
+    if (cudaStreamCreateWithFlags(&s, cudaStreamNonBlocking) != cudaSuccess) break;
+    if (cudaMallocAsync(reinterpret_cast<void**>(&dA), (size_t)M * dlda * 8, s) != cudaSuccess) break;
+    if (cudaMallocAsync(reinterpret_cast<void**>(&dB), (size_t)K * dldb * 8, s) != cudaSuccess) break;
+    if (cudaMallocAsync(reinterpret_cast<void**>(&dC), (size_t)M * dldc * 8, s) != cudaSuccess) break;
+    if (cudaMemcpy2DAsync(dA, dlda * 8, A, lda * 8, K * 8, M, cudaMemcpyHostToDevice, s) != cudaSuccess) break;
+    if (cudaMemcpy2DAsync(dB, dldb * 8, B, ldb * 8, N * 8, K, cudaMemcpyHostToDevice, s) != cudaSuccess) break;
+    if (cudaMemcpy2DAsync(dC, dldc * 8, C, ldc * 8, N * 8, M, cudaMemcpyHostToDevice, s) != cudaSuccess) break;
+    rc = launch_gemm(M, N, K, dA, dlda, dB, dldb, dC, dldc, s);
+    if (rc != DGEMM_OK) break;
+    rc = DGEMM_ERR_CUDA;
+    if (cudaMemcpy2DAsync(C, ldc * 8, dC, dldc * 8, N * 8, M, cudaMemcpyDeviceToHost, s) != cudaSuccess) break;
+    if (cudaStreamSynchronize(s) != cudaSuccess) break;
+    rc = DGEMM_OK;
+  } while (0);
+  if (rc != DGEMM_OK) (void)cudaGetLastError();
+  if (s) {
+    if (dA) cudaFreeAsync(dA, s);
+    if (dB) cudaFreeAsync(dB, s);
+    if (dC) cudaFreeAsync(dC, s);
+    cudaStreamSynchronize(s);
+    cudaStreamDestroy(s);
+  }
+  return rc;
+}
+
+const char* dgemm_strerror(int status) {
+  switch (status) {
+    case DGEMM_OK: return "success";
+    case DGEMM_ERR_BAD_DIM: return "M, N or K is negative or too large";
+    case DGEMM_ERR_BAD_LD: return "a leading dimension is smaller than the row length";
+    case DGEMM_ERR_NULL: return "a required pointer is NULL";
+    case DGEMM_ERR_ALIGN: return "a pointer is not 8-byte aligned";
+    case DGEMM_ERR_ALIAS: return "C overlaps A or B";
+    case DGEMM_ERR_DEVICE: return "no CUDA device, or the current device is not compute capability 10.x";
+    case DGEMM_ERR_CUDA: return "a CUDA runtime or driver call failed";
+    case DGEMM_ERR_TIMEOUT: return "a bounded device-side wait gave up";
+    case DGEMM_ERR_VARIANT: return "unknown kernel variant, or the forced variant cannot run these operands";
+    case DGEMM_ERR_SIZE: return "problem exceeds the fixed capacity of this entry point";
+    default: return "unknown status";
+  }
+}
+
+int dgemm_version(void) { return 100; /* 0.1.0 */ }
+
+int dgemm_set_variant(int variant) {
+  if (variant < DGEMM_VARIANT_AUTO || variant >= DGEMM_VARIANT_COUNT) return DGEMM_ERR_VARIANT;
+  g_variant.store(variant);
+  return DGEMM_OK;
+}
+
+int dgemm_set_split_k(int split_k) {
+  if (split_k < 0) return DGEMM_ERR_VARIANT;
+  g_split_k.store(split_k);
+  return DGEMM_OK;
+}
+
+int dgemm_last_device_status(void* stream) {
+  DeviceState* st = nullptr;
+  int rc = device_state(&st);
+  if (rc != DGEMM_OK) return rc;
+  if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return DGEMM_ERR_CUDA;
+  }
+  int word = 0;
+  if (cudaMemcpy(&word, st->status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return DGEMM_ERR_CUDA;
+  if (word != 0 && cudaMemset(st->status, 0, sizeof(int)) != cudaSuccess) return DGEMM_ERR_CUDA;
+  return word;
+}
+
+int64_t dgemm_launch_count(void) { return g_launches.load(); }
+
+int dgemm_fp64_peak_probe(int millis, double* fma_per_clk_sm, double* tflops) {
+  DeviceState* st = nullptr;
+  int rc = device_state(&st);
+  if (rc != DGEMM_OK) return rc;
+  if (millis < 1) millis = 1;
+  if (millis > 10000) millis = 10000;
+  const int blocks = st->sm_count, threads = 256;
+  double* out = nullptr;
+  long long* cyc = nullptr;
+  cudaEvent_t e0 = nullptr, e1 = nullptr;
+  rc = DGEMM_ERR_CUDA;
+  do {
+    if (cudaMalloc(reinterpret_cast<void**>(&out), sizeof(double) * blocks * threads) != cudaSuccess) break;
+    if (cudaMalloc(reinterpret_cast<void**>(&cyc), sizeof(long long) * blocks) != cudaSuccess) break;
+    if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) break;
+    // calibrate with a short run, then size the timed run to about `millis`
+    int iters = 2000;
+    float ms = 0.f;
+    fp64_probe_kernel<<<blocks, threads>>>(out, cyc, iters, 0.999999);
+    if (cudaEventRecord(e0) != cudaSuccess) break;
+    fp64_probe_kernel<<<blocks, threads>>>(out, cyc, iters, 0.999999);
+    if (cudaEventRecord(e1) != cudaSuccess || cudaEventSynchronize(e1) != cudaSuccess) break;
+    if (cudaEventElapsedTime(&ms, e0, e1) != cudaSuccess || ms <= 0.f) break;
+    double scale = millis / ms;
+    if (scale > 100000.0) scale = 100000.0;
+    iters = (int)(iters * scale) + 1;
+    if (cudaEventRecord(e0) != cudaSuccess) break;
+    fp64_probe_kernel<<<blocks, threads>>>(out, cyc, iters, 0.999999);
+    if (cudaEventRecord(e1) != cudaSuccess || cudaEventSynchronize(e1) != cudaSuccess) break;
+    if (cudaEventElapsedTime(&ms, e0, e1) != cudaSuccess) break;
+    g_launches.fetch_add(3);
+    long long* h = static_cast<long long*>(malloc(sizeof(long long) * blocks));
+    if (!h) break;
+    if (cudaMemcpy(h, cyc, sizeof(long long) * blocks, cudaMemcpyDeviceToHost) != cudaSuccess) { free(h); break; }
+    long long mx = 1;
+    for (int i = 0; i < blocks; ++i) if (h[i] > mx) mx = h[i];
+    free(h);
+    // per warp and iteration: 8 MMAs of 16*8*8 = 1024 fused multiply-adds
+    const double fma_per_block = (double)(threads / 32) * iters * 8.0 * 1024.0;
+    if (fma_per_clk_sm) *fma_per_clk_sm = fma_per_block / (double)mx;
+    if (tflops) *tflops = 2.0 * fma_per_block * blocks / (ms * 1e-3) / 1e12;
+    rc = DGEMM_OK;
+  } while (0);
+  if (rc != DGEMM_OK) (void)cudaGetLastError();
+  if (e0) cudaEventDestroy(e0);
+  if (e1) cudaEventDestroy(e1);
+  if (out) cudaFree(out);
+  if (cyc) cudaFree(cyc);
+  return rc;
+}
+
+}  // extern "C"

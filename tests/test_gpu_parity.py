@@ -1,0 +1,300 @@
+"""Parity of the CUDA library (through the C ABI) against the CPU oracle. Needs a B200.
+
+Bit-exact on integer-valued inputs; |dC_ij| <= 2*K*2^-53*(|A||B|)_ij on uniform real inputs
+(the scale also carries |C_in|, see the note in `_check_full`). Large cases use Freivalds' check
+plus entries recomputed one by one by the oracle's triple loop.
+"""
+import numpy as np
+import pytest
+import torch
+
+import paper_2003_00532_b200 as dg
+from paper_2003_00532_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+GUARD = 64  # doubles of guard band on each side of every device buffer
+GUARD_VALUE = -7.0e300
+
+
+def _to_device(buf: torch.Tensor, offset_elems: int = 0):
+    """Copy a padded host buffer into the middle of a larger device allocation with guard bands.
+    Returns (whole allocation, 2-D view with the same shape/strides as the host buffer)."""
+    rows, ld = buf.shape
+    n = rows * ld
+    whole = torch.full((n + 2 * GUARD + offset_elems,), GUARD_VALUE, dtype=torch.float64, device="cuda")
+    start = GUARD + offset_elems
+    whole[start:start + n] = buf.reshape(-1).cuda()
+    view = whole[start:start + n].view(rows, ld)
+    return whole, view
+
+
+def _guards_intact(whole: torch.Tensor, n: int, offset_elems: int = 0) -> bool:
+    start = GUARD + offset_elems
+    return bool((whole[:start] == GUARD_VALUE).all() and (whole[start + n:] == GUARD_VALUE).all())
+
+
+def run_gpu(prob: wl.Problem, variant=dg.DGEMM_VARIANT_AUTO, split_k=0, offset_elems=0):
+    """Run dgemm_f64 on device copies of the problem; returns the resulting padded C buffer (host)."""
+    dg.dgemm_set_variant(variant)
+    dg.dgemm_set_split_k(split_k)
+    try:
+        wa, A = _to_device(prob.A_buf, offset_elems)
+        wb, B = _to_device(prob.B_buf, offset_elems)
+        wc, C = _to_device(prob.C_buf, offset_elems)
+        before_a, before_b = wa.clone(), wb.clone()
+        dg.dgemm_f64(A[:, :prob.K], B[:, :prob.N], C[:, :prob.N])
+        assert dg.dgemm_last_device_status() == dg.DGEMM_OK
+        out = C.cpu()
+        assert _guards_intact(wc, prob.M * prob.ldc, offset_elems), "wrote outside the C buffer"
+        # inputs untouched, bit for bit (NaN padding included)
+        assert torch.equal(wa.view(torch.int64), before_a.view(torch.int64))
+        assert torch.equal(wb.view(torch.int64), before_b.view(torch.int64))
+    finally:
+        dg.dgemm_set_variant(dg.DGEMM_VARIANT_AUTO)
+        dg.dgemm_set_split_k(0)
+    assert wl.c_padding_intact(out, prob.N), "padding columns of C were modified"
+    return out
+
+
+def _check_full(oracle, prob: wl.Problem, out: torch.Tensor):
+    """Element-by-element comparison with the oracle on the whole matrix."""
+    want = prob.C.clone().contiguous().numpy()
+    A = np.ascontiguousarray(prob.A.numpy())
+    B = np.ascontiguousarray(prob.B.numpy())
+    oracle.dgemm_oracle(A, B, want)
+    got = out[:, :prob.N].numpy()
+    if prob.integer:
+        assert np.ascontiguousarray(got).tobytes() == want.tobytes(), "integer-valued inputs must match bit for bit"
+        return 0.0
+    # Stated bound 2*K*u*(|A||B|)_ij; when C_in != 0 each side rounds once more against |C_in|,
+    # so the rigorous scale is (|C_in| + |A||B|)_ij with K+1 roundings.
+    scale = oracle.abs_product(A, B, prob.C.numpy())
+    bound = 2.0 * (prob.K + 1) * oracle.U * scale
+    err = np.abs(got - want)
+    assert np.isfinite(got).all()
+    assert (err <= bound).all(), f"max err/bound = {(err / np.maximum(bound, 1e-300)).max()}"
+    return float((err / np.maximum(bound, 1e-300)).max())
+
+
+# ---- config 1: 256^3, real then integer, C = 0 --------------------------------------------------
+
+@pytest.mark.parametrize("integer", [False, True])
+@pytest.mark.parametrize("variant", [dg.DGEMM_VARIANT_AUTO, dg.DGEMM_VARIANT_TMA, dg.DGEMM_VARIANT_GENERIC,
+                                     dg.DGEMM_VARIANT_NAIVE])
+def test_config1(oracle, integer, variant):
+    prob = wl.config1(integer)
+    _check_full(oracle, prob, run_gpu(prob, variant))
+
+
+# ---- tiny and odd shapes, every variant, padded leading dimensions ---------------------------------
+
+SMALL_SHAPES = [(1, 1, 1), (1, 7, 3), (5, 1, 2), (3, 3, 17), (17, 13, 11), (8, 8, 16), (16, 16, 15),
+                (31, 33, 29), (64, 64, 64), (127, 129, 47), (128, 128, 16), (129, 127, 17), (130, 260, 33),
+                (257, 131, 100), (200, 300, 1)]
+
+
+@pytest.mark.parametrize("shape", SMALL_SHAPES)
+@pytest.mark.parametrize("variant", [dg.DGEMM_VARIANT_TMA, dg.DGEMM_VARIANT_GENERIC])
+def test_small_shapes_integer_exact(oracle, shape, variant):
+    M, N, K = shape
+    # even leading dimensions so that both staging variants can run the same problem
+    prob = wl.make_problem(M, N, K, seed=100 + M + N + K, lda=K + 2 + (K & 1), ldb=N + 4 + (N & 1),
+                           ldc=N + 7, integer=True)
+    _check_full(oracle, prob, run_gpu(prob, variant))
+
+
+@pytest.mark.parametrize("shape", SMALL_SHAPES)
+def test_small_shapes_real_odd_ld(oracle, shape):
+    M, N, K = shape
+    prob = wl.make_problem(M, N, K, seed=200 + M + N + K, lda=K + 3, ldb=N + 5, ldc=N + 7)
+    _check_full(oracle, prob, run_gpu(prob))
+
+
+@pytest.mark.parametrize("offset", [1, 2, 3])
+def test_unaligned_base_pointers(oracle, offset):
+    """Base pointers that are only 8-byte aligned (odd element offset into the allocation)."""
+    prob = wl.make_problem(150, 140, 70, seed=7, lda=72, ldb=144, ldc=141, integer=True)
+    _check_full(oracle, prob, run_gpu(prob, offset_elems=offset))
+
+
+# ---- split-K (partial tiles through the workspace, deterministic reduction) -------------------------
+
+@pytest.mark.parametrize("split", [2, 3, 7, 64])
+@pytest.mark.parametrize("variant", [dg.DGEMM_VARIANT_TMA, dg.DGEMM_VARIANT_GENERIC])
+def test_split_k(oracle, split, variant):
+    prob = wl.make_problem(200, 150, 1000, seed=11, lda=1000, ldb=150 + 2, ldc=151, integer=True)
+    _check_full(oracle, prob, run_gpu(prob, variant, split_k=split))
+    prob = wl.make_problem(129, 257, 515, seed=12, lda=516, ldb=258, ldc=257)
+    _check_full(oracle, prob, run_gpu(prob, variant, split_k=split))
+
+
+def test_split_k_deterministic():
+    prob = wl.make_problem(300, 200, 2048, seed=13)
+    a = run_gpu(prob, split_k=8)
+    b = run_gpu(prob, split_k=8)
+    assert torch.equal(a.view(torch.int64), b.view(torch.int64))
+
+
+# ---- config 2: square sweep ---------------------------------------------------------------------
+
+@pytest.mark.parametrize("n", [128, 256, 384, 512, 640, 768, 896, 1024, 1536, 2048])
+def test_config2_full(oracle, n):
+    prob = wl.config2(n)
+    _check_full(oracle, prob, run_gpu(prob))
+
+
+def _check_sampled(oracle, prob: wl.Problem, out: torch.Tensor, nsamples: int, seed: int):
+    ii, jj = wl.sample_indices(prob.M, prob.N, nsamples, seed)
+    A, B, C0 = prob.A.numpy(), prob.B.numpy(), prob.C.numpy()
+    want = oracle.dgemm_oracle_entries(A, B, C0, ii.numpy(), jj.numpy())
+    got = out[:, :prob.N][ii, jj].numpy()
+    if prob.integer:
+        assert np.array_equal(got, want)
+        return
+    scale = oracle.dgemm_oracle_entries(A, B, C0, ii.numpy(), jj.numpy(), absolute=True)
+    bound = 2.0 * (prob.K + 1) * oracle.U * scale
+    assert (np.abs(got - want) <= bound).all()
+
+
+def _check_freivalds(oracle, prob: wl.Problem, out: torch.Tensor, nvec: int = 20, seed: int = 99):
+    X = oracle.freivalds_vectors(prob.N, nvec, seed)
+    resid, tol = oracle.freivalds_residual(prob.A.numpy(), prob.B.numpy(), prob.C.numpy(),
+                                           out[:, :prob.N].numpy(), X)
+    if prob.integer:
+        assert (resid == 0).all(), "integer-valued data: Freivalds' identity must hold exactly"
+    else:
+        assert (resid <= tol).all(), f"max resid/tol = {(resid / tol).max()}"
+
+
+@pytest.mark.parametrize("n", [2560, 3072, 3584, 4096])
+def test_config2_large_sampled(oracle, n):
+    prob = wl.config2(n)
+    out = run_gpu(prob)
+    _check_freivalds(oracle, prob, out)
+    _check_sampled(oracle, prob, out, 2048, seed=n)
+
+
+# ---- config 3: 8192^3 -----------------------------------------------------------------------------
+
+@pytest.mark.parametrize("integer", [False, True])
+def test_config3_8192(oracle, integer):
+    prob = wl.config3(integer=integer)
+    out = run_gpu(prob)
+    _check_freivalds(oracle, prob, out, nvec=20, seed=1)
+    _check_sampled(oracle, prob, out, 4096, seed=1)
+
+
+# ---- config 4: ragged shapes, padded odd leading dimensions ---------------------------------------
+
+@pytest.mark.parametrize("idx", [0, 1, 2])
+def test_config4_ragged(oracle, idx):
+    prob = wl.config4(idx)
+    _check_full(oracle, prob, run_gpu(prob))
+
+
+@pytest.mark.parametrize("idx", [0, 2])
+def test_config4_ragged_integer(oracle, idx):
+    M, N, K = wl.CONFIG4_SHAPES[idx]
+    prob = wl.make_problem(M, N, K, 2, lda=K + 3, ldb=N + 5, ldc=N + 7, integer=True)
+    _check_full(oracle, prob, run_gpu(prob))
+
+
+# ---- config 5: rank-k updates -------------------------------------------------------------------
+
+@pytest.mark.parametrize("K", wl.CONFIG5_K)
+def test_config5_rank_k(oracle, K):
+    prob = wl.config5(K)
+    out = run_gpu(prob)
+    _check_freivalds(oracle, prob, out, nvec=20, seed=3)
+    _check_sampled(oracle, prob, out, 4096, seed=3)
+
+
+# ---- degenerate cases and argument errors ------------------------------------------------------
+
+def test_degenerate_and_errors():
+    A = torch.zeros(4, 4, dtype=torch.float64, device="cuda")
+    B = torch.zeros(4, 4, dtype=torch.float64, device="cuda")
+    C0 = torch.tensor([[-0.0, float("nan")], [1.5, -2.0]], dtype=torch.float64, device="cuda")
+    C = C0.clone()
+    # K = 0: C untouched bit for bit
+    assert dg.dgemm_f64_raw(2, 2, 0, A.data_ptr(), 1, B.data_ptr(), 2, C.data_ptr(), 2) == 0
+    torch.cuda.synchronize()
+    assert torch.equal(C.view(torch.int64), C0.view(torch.int64))
+    # M = 0 / N = 0: no-op even with null pointers
+    assert dg.dgemm_f64_raw(0, 5, 5, None, 5, None, 5, None, 5) == 0
+    assert dg.dgemm_f64_raw(5, 0, 5, None, 5, None, 1, None, 1) == 0
+    a, b, c = A.data_ptr(), B.data_ptr(), C.data_ptr()
+    assert dg.dgemm_f64_raw(-1, 2, 2, a, 2, b, 2, c, 2, check=False) == -1
+    assert dg.dgemm_f64_raw(2, 2, 2, a, 1, b, 2, c, 2, check=False) == -2
+    assert dg.dgemm_f64_raw(2, 2, 2, a, 2, b, 1, c, 2, check=False) == -2
+    assert dg.dgemm_f64_raw(2, 2, 2, a, 2, b, 2, c, 1, check=False) == -2
+    assert dg.dgemm_f64_raw(2, 2, 2, None, 2, b, 2, c, 2, check=False) == -3
+    assert dg.dgemm_f64_raw(2, 2, 2, a + 4, 2, b, 2, c, 2, check=False) == -4
+    assert dg.dgemm_f64_raw(2, 2, 2, a, 2, b, 2, a + 8, 2, check=False) == -5
+    with pytest.raises(dg.DgemmError):
+        dg.dgemm_f64_raw(2, 2, 2, a, 2, b, 2, b, 2)
+    # forced TMA variant on an odd leading dimension is refused, not silently rerouted
+    dg.dgemm_set_variant(dg.DGEMM_VARIANT_TMA)
+    try:
+        big = torch.zeros(64, dtype=torch.float64, device="cuda")
+        assert dg.dgemm_f64_raw(2, 2, 2, big.data_ptr(), 3, b, 2, c, 2, check=False) == -9
+    finally:
+        dg.dgemm_set_variant(dg.DGEMM_VARIANT_AUTO)
+    assert dg.dgemm_last_device_status() == 0
+
+
+def test_nan_propagates_to_its_row_only():
+    A = torch.ones(130, 40, dtype=torch.float64)
+    A[77, 5] = float("nan")
+    prob = wl.make_problem(130, 140, 40, seed=5)
+    prob.A_buf.copy_(A)
+    prob.B_buf.fill_(1.0)
+    out = run_gpu(prob)
+    assert torch.isnan(out[77]).all()
+    assert torch.isfinite(torch.cat([out[:77], out[78:]])).all()
+
+
+def test_all_ones_paper_driver():
+    """The paper's driver (Section 2.1): A = B = C = 1 on 2048-sized operands gives 1 + K."""
+    n = 2048
+    A = torch.ones(n, n, dtype=torch.float64, device="cuda")
+    B = torch.ones(n, n, dtype=torch.float64, device="cuda")
+    C = torch.ones(n, n, dtype=torch.float64, device="cuda")
+    dg.dgemm_f64(A, B, C)
+    assert dg.dgemm_last_device_status() == 0
+    assert bool((C == 2049.0).all())
+
+
+def test_accumulates_into_c_and_k_split_calls(oracle):
+    """Two successive calls over a K partition equal one call (exact on integer data)."""
+    prob = wl.make_problem(140, 130, 96, seed=21, integer=True)
+    one = run_gpu(prob)
+    A, B, C = prob.A_buf.cuda(), prob.B_buf.cuda(), prob.C_buf.cuda()
+    dg.dgemm_f64(A[:, :40], B[:40, :], C)
+    dg.dgemm_f64(A[:, 40:], B[40:, :], C)
+    torch.cuda.synchronize()
+    assert torch.equal(C.cpu(), one)
+
+
+def test_host_entry_point(oracle):
+    prob = wl.make_problem(300, 257, 129, seed=31, lda=129 + 3, ldb=257 + 5, ldc=257 + 7)
+    want = prob.C.clone().contiguous().numpy()
+    oracle.dgemm_oracle(np.ascontiguousarray(prob.A.numpy()), np.ascontiguousarray(prob.B.numpy()), want)
+    scale = oracle.abs_product(prob.A.numpy(), prob.B.numpy(), prob.C.numpy())
+    dg.dgemm_f64_host(prob.A, prob.B, prob.C)
+    assert wl.c_padding_intact(prob.C_buf, prob.N)
+    assert (np.abs(prob.C.numpy() - want) <= 2.0 * (prob.K + 1) * oracle.U * scale).all()
+
+
+def test_non_default_stream(oracle):
+    prob = wl.make_problem(256, 256, 512, seed=41, integer=True)
+    A, B, C = prob.A_buf.cuda(), prob.B_buf.cuda(), prob.C_buf.cuda()
+    s = torch.cuda.Stream()
+    s.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(s):
+        dg.dgemm_f64(A, B, C, stream=s)
+    assert dg.dgemm_last_device_status(s) == 0
+    want = prob.C.clone().numpy()
+    oracle.dgemm_oracle(prob.A.numpy(), prob.B.numpy(), want)
+    assert np.array_equal(C.cpu().numpy(), want)

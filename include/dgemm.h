@@ -102,6 +102,40 @@ DGEMM_API int dgemm_f64_host(int64_t M, int64_t N, int64_t K,
                    const double *B, int64_t ldb,
                    double *C, int64_t ldc);
 
+/*
+ * (No counterpart in the paper: an addition for callers that cannot allocate.)
+ *
+ * C += A*B like dgemm_f64, with K split over several thread blocks and the partial tiles kept in
+ * a fixed array that is part of the library image (16 MiB of device memory on every GPU that
+ * loads the library, held until the process exits). The call allocates nothing: no cudaMalloc,
+ * no cudaFree, no stream-ordered or library allocator. It is meant for callers that are not
+ * allowed to allocate at the time of the call, for example because a stream is being captured,
+ * because they hold a lock the allocator may need, because they run under a fixed memory budget,
+ * or because another component owns the device memory pool. dgemm_f64 itself allocates its
+ * split-K workspace on first need and so is not suitable for them on small problems.
+ *
+ * Arguments and error codes are those of dgemm_f64, plus:
+ *   split_k   number of K partitions; 0 lets the library choose (at least 2). It is clamped to
+ *             the number of 16-wide k-blocks; a problem with a single k-block (K <= 16) runs
+ *             unsplit and does not touch the array.
+ * Capacity: ceil(M/128) * ceil(N/128) * split_k <= 128 partial tiles. A larger problem returns
+ * DGEMM_ERR_SIZE and launches nothing (use dgemm_f64, or a smaller split_k). A negative
+ * split_k returns DGEMM_ERR_VARIANT.
+ *
+ * The first call on each device looks up the array's device address and configures the
+ * kernels (no allocation, but runtime calls that are not capturable): make that first call
+ * before any stream capture begins, with the device current. All calls on a device share the
+ * one array. Its contents are left over from the previous call; nothing needs clearing because
+ * each call overwrites every slot it later reads. Two calls that overlap on the GPU (different
+ * streams without ordering between them) race on the array and give undefined results:
+ * serialise them, e.g. by using one stream.
+ */
+DGEMM_API int dgemm_f64_static_ws(int64_t M, int64_t N, int64_t K,
+                                  const double *A, int64_t lda,
+                                  const double *B, int64_t ldb,
+                                  double *C, int64_t ldc,
+                                  int split_k, void *stream);
+
 /* Human-readable text for a status code; never NULL; static storage. */
 DGEMM_API const char *dgemm_strerror(int status);
 

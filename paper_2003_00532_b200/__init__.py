@@ -13,6 +13,7 @@ from .binding import (  # noqa: F401
     dgemm_f64,
     dgemm_f64_host,
     dgemm_f64_raw,
+    dgemm_f64_static_ws,
     dgemm_fp64_peak_probe,
     dgemm_last_device_status,
     dgemm_launch_count,

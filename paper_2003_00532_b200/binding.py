@@ -62,6 +62,8 @@ def load_library() -> ctypes.CDLL:
             lib.dgemm_f64.restype = ctypes.c_int
             lib.dgemm_f64_host.argtypes = [i64, i64, i64, vp, i64, vp, i64, vp, i64]
             lib.dgemm_f64_host.restype = ctypes.c_int
+            lib.dgemm_f64_static_ws.argtypes = [i64, i64, i64, vp, i64, vp, i64, vp, i64, ctypes.c_int, vp]
+            lib.dgemm_f64_static_ws.restype = ctypes.c_int
             lib.dgemm_strerror.argtypes = [ctypes.c_int]
             lib.dgemm_strerror.restype = ctypes.c_char_p
             lib.dgemm_version.argtypes = []
@@ -135,6 +137,23 @@ def dgemm_f64_raw(M, N, K, A_ptr, lda, B_ptr, ldb, C_ptr, ldc, stream: Optional[
     rc = load_library().dgemm_f64(M, N, K, A_ptr, lda, B_ptr, ldb, C_ptr, ldc, stream)
     if check and rc < 0:
         raise DgemmError(rc, "dgemm_f64")
+    return rc
+
+
+def dgemm_f64_static_ws(A, B, C, split_k: int = 0, stream=None, check: bool = True) -> int:
+    """``C += A @ B`` with split-K partial sums kept in the library's fixed device array.
+
+    For callers that may not allocate device memory when they call (during stream capture, under
+    a lock shared with an allocator, under a fixed memory budget): this entry point never
+    allocates. At most 128 partial tiles (``ceil(M/128) * ceil(N/128) * split_k``); beyond that it
+    returns ``DGEMM_ERR_SIZE``. Calls on one device share the array, so they must not overlap on
+    the GPU. Make the first call on a device outside stream capture.
+    """
+    M, N, K, pa, lda, pb, ldb, pc, ldc = _shapes(A, B, C, True)
+    rc = load_library().dgemm_f64_static_ws(M, N, K, pa, lda, pb, ldb, pc, ldc, int(split_k),
+                                            _stream_handle(stream))
+    if check and rc < 0:
+        raise DgemmError(rc, "dgemm_f64_static_ws")
     return rc
 
 

@@ -200,6 +200,101 @@ int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, c
   return DGEMM_OK;
 }
 
+// ---- split-K through a statically allocated workspace (no allocation at run time) --------------
+//
+// Some callers must not allocate device memory when they call into the library: code running
+// while a stream is being captured, code holding a lock that the allocator may also take,
+// real-time loops with a fixed memory budget, or a process whose memory pool is owned by
+// another component. For them the split-K partial tiles live in this file-scope device array.
+// Every GPU that loads the library carries it (16 MiB) until the process exits.
+constexpr int kStaticPartialTiles = 128;  // capacity: tiles * split_k partial tiles of 128 x 128 doubles
+static __device__ __align__(256) double g_static_partials[(size_t)kStaticPartialTiles * BM * BN];
+
+// Device address of g_static_partials per device. In host code the array's name is only a
+// handle for the runtime, not an address a kernel could use; the address is looked up once per
+// device, with that device current.
+double* g_static_partials_addr[kMaxDevices];
+
+int static_partials(double** out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+    (void)cudaGetLastError();
+    return DGEMM_ERR_DEVICE;
+  }
+  std::lock_guard<std::mutex> lock(g_mutex);
+  if (!g_static_partials_addr[dev]) {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_static_partials) != cudaSuccess || !ptr) {
+      (void)cudaGetLastError();
+      return DGEMM_ERR_CUDA;
+    }
+    g_static_partials_addr[dev] = static_cast<double*>(ptr);
+  }
+  *out = g_static_partials_addr[dev];
+  return DGEMM_OK;
+}
+
+int launch_gemm_static_ws(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, const double* B,
+                          int64_t ldb, double* C, int64_t ldc, int split_k, cudaStream_t stream) {
+  DeviceState* st = nullptr;
+  int rc = device_state(&st);  // capability check, status word, shared-memory opt-in; allocates nothing
+  if (rc != DGEMM_OK) return rc;
+  double* partials = nullptr;
+  rc = static_partials(&partials);
+  if (rc != DGEMM_OK) return rc;
+
+  const bool tma_ok = (((uintptr_t)A | (uintptr_t)B) & 15) == 0 && (lda % 2 == 0) && (ldb % 2 == 0);
+
+  GemmParams p;
+  memset(&p, 0, sizeof(p));
+  p.M = (int)M; p.N = (int)N; p.K = (int)K;
+  p.tiles_m = (int)((M + BM - 1) / BM);
+  p.tiles_n = (int)((N + BN - 1) / BN);
+  p.A = A; p.B = B; p.C = C;
+  p.lda = lda; p.ldb = ldb; p.ldc = ldc;
+  p.wait_limit_ns = kWaitLimitNs;
+  p.status = st->status;
+  p.group_m = 8;
+
+  const int64_t tiles = (int64_t)p.tiles_m * p.tiles_n;
+  const int kblocks = (int)((K + BK - 1) / BK);
+  if (tiles > kStaticPartialTiles) return DGEMM_ERR_SIZE;
+  int split = split_k;
+  if (split <= 0) {  // as many partitions as the SMs and the array can take, at least 4 k-blocks each
+    split = st->sm_count / (int)tiles;
+    if (split > kblocks / 4) split = kblocks / 4;
+    if (split > kStaticPartialTiles / (int)tiles) split = kStaticPartialTiles / (int)tiles;
+    if (split < 2) split = 2;
+  }
+  if (split > kblocks) split = kblocks;
+  p.kblocks_per_split = (kblocks + split - 1) / split;
+  p.split_k = (kblocks + p.kblocks_per_split - 1) / p.kblocks_per_split;
+  if (p.split_k > 1) {
+    if (tiles * p.split_k > kStaticPartialTiles) return DGEMM_ERR_SIZE;
+    p.partial = partials;  // every (tile, partition) slot in use is fully overwritten: nothing to clear
+  }
+
+  const int units = (int)tiles * p.split_k;
+  const int grid = units < st->sm_count ? units : st->sm_count;
+  CUtensorMap map_a, map_b;
+  memset(&map_a, 0, sizeof(map_a));
+  memset(&map_b, 0, sizeof(map_b));
+  if (tma_ok) {
+    if (!make_map(&map_a, A, M, K, lda, BK, BM) || !make_map(&map_b, B, K, N, ldb, 16, BK)) return DGEMM_ERR_CUDA;
+    dgemm_dmma_kernel<true><<<grid, THREADS, SMEM_BYTES, stream>>>(map_a, map_b, p);
+  } else {
+    dgemm_dmma_kernel<false><<<grid, THREADS, SMEM_BYTES, stream>>>(map_a, map_b, p);
+  }
+  g_launches.fetch_add(1);
+  if (cudaGetLastError() != cudaSuccess) return DGEMM_ERR_CUDA;
+  if (p.split_k > 1) {
+    dgemm_splitk_reduce_kernel<<<(int)tiles, 256, 0, stream>>>(p);
+    g_launches.fetch_add(1);
+    if (cudaGetLastError() != cudaSuccess) return DGEMM_ERR_CUDA;
+  }
+  return DGEMM_OK;
+}
+
 // ---- FP64 issue-rate probe -------------------------------------------------------------------
 
 __global__ void __launch_bounds__(256) fp64_probe_kernel(double* out, long long* cycles, int iters, double seed) {
@@ -230,6 +325,15 @@ int dgemm_f64(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, con
   if (v == 1) return DGEMM_OK;
   if (v != DGEMM_OK) return v;
   return launch_gemm(M, N, K, A, lda, B, ldb, C, ldc, static_cast<cudaStream_t>(stream));
+}
+
+int dgemm_f64_static_ws(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, const double* B, int64_t ldb,
+                        double* C, int64_t ldc, int split_k, void* stream) {
+  if (split_k < 0) return DGEMM_ERR_VARIANT;
+  const int v = validate(M, N, K, A, lda, B, ldb, C, ldc);
+  if (v == 1) return DGEMM_OK;
+  if (v != DGEMM_OK) return v;
+  return launch_gemm_static_ws(M, N, K, A, lda, B, ldb, C, ldc, split_k, static_cast<cudaStream_t>(stream));
 }
 
 int dgemm_f64_host(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, const double* B, int64_t ldb,

@@ -109,9 +109,9 @@ DGEMM_API int dgemm_f64_host(int64_t M, int64_t N, int64_t K,
  * a fixed array that is part of the library image (16 MiB of device memory on every GPU that
  * loads the library, held until the process exits). The call allocates nothing: no cudaMalloc,
  * no cudaFree, no stream-ordered or library allocator. It is meant for callers that are not
- * allowed to allocate at the time of the call, for example because a stream is being captured,
- * because they hold a lock the allocator may need, because they run under a fixed memory budget,
- * or because another component owns the device memory pool. dgemm_f64 itself allocates its
+ * allowed to allocate at the time of the call, for example because they hold a lock the allocator
+ * may need, because they run under a fixed memory budget or inside a latency-critical loop, or
+ * because another component owns the device memory pool. dgemm_f64 itself allocates its
  * split-K workspace on first need and so is not suitable for them on small problems.
  *
  * Arguments and error codes are those of dgemm_f64, plus:
@@ -123,8 +123,8 @@ DGEMM_API int dgemm_f64_host(int64_t M, int64_t N, int64_t K,
  * split_k returns DGEMM_ERR_VARIANT.
  *
  * The first call on each device looks up the array's device address and configures the
- * kernels (no allocation, but runtime calls that are not capturable): make that first call
- * before any stream capture begins, with the device current. All calls on a device share the
+ * kernels (no allocation, but several runtime set-up calls): make that first call before any
+ * stream capture begins, with the device current. All calls on a device share the
  * one array. Its contents are left over from the previous call; nothing needs clearing because
  * each call overwrites every slot it later reads. Two calls that overlap on the GPU (different
  * streams without ordering between them) race on the array and give undefined results:

@@ -143,11 +143,11 @@ def dgemm_f64_raw(M, N, K, A_ptr, lda, B_ptr, ldb, C_ptr, ldc, stream: Optional[
 def dgemm_f64_static_ws(A, B, C, split_k: int = 0, stream=None, check: bool = True) -> int:
     """``C += A @ B`` with split-K partial sums kept in the library's fixed device array.
 
-    For callers that may not allocate device memory when they call (during stream capture, under
-    a lock shared with an allocator, under a fixed memory budget): this entry point never
+    For callers that may not allocate device memory when they call (under a lock shared with an
+    allocator, under a fixed memory budget, in a latency-critical loop): this entry point never
     allocates. At most 128 partial tiles (``ceil(M/128) * ceil(N/128) * split_k``); beyond that it
     returns ``DGEMM_ERR_SIZE``. Calls on one device share the array, so they must not overlap on
-    the GPU. Make the first call on a device outside stream capture.
+    the GPU. The first call on a device does the set-up and should come before any stream capture.
     """
     M, N, K, pa, lda, pb, ldb, pc, ldc = _shapes(A, B, C, True)
     rc = load_library().dgemm_f64_static_ws(M, N, K, pa, lda, pb, ldb, pc, ldc, int(split_k),

@@ -202,10 +202,9 @@ int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, c
 
 // ---- split-K through a statically allocated workspace (no allocation at run time) --------------
 //
-// Some callers must not allocate device memory when they call into the library: code running
-// while a stream is being captured, code holding a lock that the allocator may also take,
-// real-time loops with a fixed memory budget, or a process whose memory pool is owned by
-// another component. For them the split-K partial tiles live in this file-scope device array.
+// Some callers must not allocate device memory when they call into the library: code holding a
+// lock that the allocator may also take, latency-critical loops with a fixed memory budget, or
+// a process whose memory pool is owned by another component. For them the split-K partial tiles live in this file-scope device array.
 // Every GPU that loads the library carries it (16 MiB) until the process exits.
 constexpr int kStaticPartialTiles = 128;  // capacity: tiles * split_k partial tiles of 128 x 128 doubles
 static __device__ __align__(256) double g_static_partials[(size_t)kStaticPartialTiles * BM * BN];

@@ -1,7 +1,7 @@
 """The allocation-free entry point ``dgemm_f64_static_ws`` against ``dgemm_f64``. Needs a B200.
 
 ``dgemm_f64_static_ws`` exists for callers that must not allocate device memory at the time of
-the call (a stream being captured, a lock shared with an allocator, a fixed memory budget): its
+the call (a lock shared with an allocator, a fixed memory budget, a latency-critical loop): its
 split-K partial tiles live in a fixed device array inside the library. The test calls it through
 the C ABI twice in a row (the second call finds the first call's leftovers in the array) and
 compares each result with the regular entry point's on the same inputs, within the bound the

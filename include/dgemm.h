@@ -154,6 +154,17 @@ DGEMM_API int dgemm_set_variant(int variant);
 DGEMM_API int dgemm_set_split_k(int split_k);
 
 /*
+ * Testing aid: switches off optional accelerations of the pipelined variants so that tests can
+ * exercise the slower code paths and the timing they produce (the operation and its results do
+ * not change). Bit flags, 0 restores the default. No counterpart in the paper.
+ */
+enum {
+  DGEMM_TEST_NO_C_PREFETCH = 1, /* do not ask L2 for the C tile ahead of the epilogue           */
+  DGEMM_TEST_NO_BLOCKED_B = 2   /* stage B with eight 2-D copies per stage instead of one 3-D copy */
+};
+DGEMM_API int dgemm_set_test_flags(int flags);
+
+/*
  * Synchronises `stream`, then reads and clears the current device's status word. Returns
  * DGEMM_OK if no kernel reported a problem since the last call, DGEMM_ERR_TIMEOUT if a bounded
  * wait inside a kernel ran out (the kernel then stopped early and C is unspecified), or

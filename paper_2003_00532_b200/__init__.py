@@ -18,6 +18,7 @@ from .binding import (  # noqa: F401
     dgemm_last_device_status,
     dgemm_launch_count,
     dgemm_set_split_k,
+    dgemm_set_test_flags,
     dgemm_set_variant,
     dgemm_strerror,
     dgemm_version,

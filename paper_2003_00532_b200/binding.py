@@ -70,6 +70,8 @@ def load_library() -> ctypes.CDLL:
             lib.dgemm_version.restype = ctypes.c_int
             lib.dgemm_set_variant.argtypes = [ctypes.c_int]
             lib.dgemm_set_variant.restype = ctypes.c_int
+            lib.dgemm_set_test_flags.argtypes = [ctypes.c_int]
+            lib.dgemm_set_test_flags.restype = ctypes.c_int
             lib.dgemm_set_split_k.argtypes = [ctypes.c_int]
             lib.dgemm_set_split_k.restype = ctypes.c_int
             lib.dgemm_last_device_status.argtypes = [vp]
@@ -186,6 +188,14 @@ def dgemm_set_split_k(split_k: int) -> int:
     rc = load_library().dgemm_set_split_k(int(split_k))
     if rc < 0:
         raise DgemmError(rc, "dgemm_set_split_k")
+    return rc
+
+
+def dgemm_set_test_flags(flags: int) -> int:
+    """Testing aid: bit 0 disables the L2 prefetch of C, bit 1 the single-copy staging of B."""
+    rc = load_library().dgemm_set_test_flags(int(flags))
+    if rc < 0:
+        raise DgemmError(rc, "dgemm_set_test_flags")
     return rc
 
 

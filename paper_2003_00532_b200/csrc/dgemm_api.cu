@@ -22,6 +22,8 @@ using namespace dgemm;
 constexpr int kMaxDevices = 64;
 constexpr size_t kWorkspaceBytes = 320ull * BM * BN * sizeof(double);  // 40 MiB: up to 320 partial tiles
 constexpr unsigned long long kWaitLimitNs = 4000000000ull;            // 4 s per device-side wait
+constexpr int kTailMinSpan = 2;          // stream-K tail: at least this many k-blocks per CTA
+constexpr double kTailMinSavedKblocks = 5.0;  // use the stream-K tail only if it saves this many k-block times
 
 __device__ int g_status_word;  // one per device that loads the library
 
@@ -36,6 +38,7 @@ DeviceState g_dev[kMaxDevices];
 std::mutex g_mutex;
 std::atomic<int> g_variant{DGEMM_VARIANT_AUTO};
 std::atomic<int> g_split_k{0};
+std::atomic<int> g_test_flags{0};
 std::atomic<long long> g_launches{0};
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -103,6 +106,19 @@ bool make_map(CUtensorMap* map, const double* base, int64_t rows, int64_t cols, 
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// 3-D view of a row-major K x N matrix whose N is a multiple of 16: (column within a block of 16,
+// k, block of 16 columns), box 16 x box_k x box_blocks. One copy then lands as `box_blocks`
+// consecutive [box_k][16] sub-tiles, each row 128 bytes, 128-byte swizzled: the B stage layout.
+bool make_blocked_map(CUtensorMap* map, const double* base, int64_t K, int64_t N, int64_t ld, int box_k, int box_blocks) {
+  const cuuint64_t dims[3] = {16, (cuuint64_t)K, (cuuint64_t)(N / 16)};
+  const cuuint64_t strides[2] = {(cuuint64_t)ld * sizeof(double), 16 * sizeof(double)};
+  const cuuint32_t box[3] = {16, (cuuint32_t)box_k, (cuuint32_t)box_blocks};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  return g_encode(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT64, 3, const_cast<double*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 bool ranges_overlap(const void* p, int64_t pbytes, const void* q, int64_t qbytes) {
   const uintptr_t a = (uintptr_t)p, b = (uintptr_t)q;
   return a < b + (uintptr_t)qbytes && b < a + (uintptr_t)pbytes;
@@ -156,36 +172,67 @@ int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, c
 
   const int tiles = p.tiles_m * p.tiles_n;
   const int kblocks = (int)((K + BK - 1) / BK);
-  int split = g_split_k.load();
-  if (split <= 0) {
-    // Split K only when the output tiles cannot occupy the SMs; keep at least 4 k-blocks per part.
-    split = 1;
-    if (tiles * 2 <= st->sm_count) {
-      split = st->sm_count / tiles;
-      if (split > kblocks / 4) split = kblocks / 4;
-      if (split < 1) split = 1;
+  const int sms = st->sm_count;
+  const int max_partials = (int)(kWorkspaceBytes / (BM * BN * sizeof(double)));
+  p.kblocks = kblocks;
+  p.c_prefetch = (((uintptr_t)C & 15) == 0 && (ldc % 2 == 0)) ? 1 : 0;
+  const int dbg_flags = g_test_flags.load();
+  if (dbg_flags & DGEMM_TEST_NO_C_PREFETCH) p.c_prefetch = 0;
+  int grid;
+  const int forced_split = g_split_k.load();
+  if (forced_split > 0) {
+    // uniform split-K over all tiles (tests and ablation)
+    int split = forced_split > kblocks ? kblocks : forced_split;
+    if ((int64_t)split * tiles > max_partials) split = max_partials / tiles;
+    if (split < 1) split = 1;
+    p.kblocks_per_split = (kblocks + split - 1) / split;
+    p.split_k = (kblocks + p.kblocks_per_split - 1) / p.kblocks_per_split;  // no empty partitions
+    p.dp_tiles = tiles;
+    p.tail_tiles = 0;
+    p.tail_ipc = 1;
+    const int units = tiles * p.split_k;
+    grid = units < sms ? units : sms;
+  } else {
+    // whole waves of tiles run data-parallel; the last partial wave is spread evenly over the SMs
+    // (stream-K) when that saves more time than the partial-tile round trip costs
+    p.split_k = 1;
+    p.kblocks_per_split = kblocks;
+    p.dp_tiles = (tiles / sms) * sms;
+    p.tail_tiles = tiles - p.dp_tiles;
+    p.tail_ipc = kblocks;
+    grid = tiles < sms ? tiles : sms;
+    if (p.tail_tiles > 0) {
+      const double idle_kblocks = (1.0 - (double)p.tail_tiles / sms) * kblocks;  // per-SM idle time if run as one wave
+      if (idle_kblocks >= kTailMinSavedKblocks && kblocks >= 2 * kTailMinSpan &&
+          (long long)(p.tail_tiles + 1) * kblocks < (long long)INT32_MAX) {
+        const long long total = (long long)p.tail_tiles * kblocks;
+        long long ipc = (total + sms - 1) / sms;
+        if (ipc < kTailMinSpan) ipc = kTailMinSpan;
+        if (ipc > kblocks) ipc = kblocks;
+        p.tail_ipc = (int)ipc;
+        const int span_ctas = (int)((total + ipc - 1) / ipc);
+        if (p.dp_tiles == 0) grid = span_ctas < sms ? span_ctas : sms;
+      } else {
+        p.dp_tiles = tiles;  // run the last wave data-parallel as well
+        p.tail_tiles = 0;
+      }
     }
   }
-  if (split > kblocks) split = kblocks;
-  const int max_partials = (int)(kWorkspaceBytes / (BM * BN * sizeof(double)));
-  if ((int64_t)split * tiles > max_partials) split = max_partials / tiles;
-  if (split < 1) split = 1;
-  p.kblocks_per_split = (kblocks + split - 1) / split;
-  p.split_k = (kblocks + p.kblocks_per_split - 1) / p.kblocks_per_split;  // no empty partitions
-  if (p.split_k > 1) {
+  p.tail_slot_base = 0;
+  const bool uses_workspace = p.split_k > 1 || (p.tail_tiles > 0 && p.tail_ipc < kblocks);
+  if (uses_workspace) {
     rc = ensure_workspace(st);
     if (rc != DGEMM_OK) return rc;
     p.partial = st->workspace;
   }
 
-  const int units = tiles * p.split_k;
-  const int grid = units < st->sm_count ? units : st->sm_count;
-
   CUtensorMap map_a, map_b;
   memset(&map_a, 0, sizeof(map_a));
   memset(&map_b, 0, sizeof(map_b));
   if (variant == DGEMM_VARIANT_TMA) {
-    if (!make_map(&map_a, A, M, K, lda, BK, BM) || !make_map(&map_b, B, K, N, ldb, 16, BK)) return DGEMM_ERR_CUDA;
+    if (!make_map(&map_a, A, M, K, lda, BK, BM)) return DGEMM_ERR_CUDA;
+    p.b_blocked_map = (!(dbg_flags & DGEMM_TEST_NO_BLOCKED_B) && N % 16 == 0 && make_blocked_map(&map_b, B, K, N, ldb, BK, BN / 16)) ? 1 : 0;
+    if (!p.b_blocked_map && !make_map(&map_b, B, K, N, ldb, 16, BK)) return DGEMM_ERR_CUDA;
     dgemm_dmma_kernel<true><<<grid, THREADS, SMEM_BYTES, stream>>>(map_a, map_b, p);
   } else {
     dgemm_dmma_kernel<false><<<grid, THREADS, SMEM_BYTES, stream>>>(map_a, map_b, p);
@@ -194,6 +241,11 @@ int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, c
   if (cudaGetLastError() != cudaSuccess) return DGEMM_ERR_CUDA;
   if (p.split_k > 1) {
     dgemm_splitk_reduce_kernel<<<tiles, 256, 0, stream>>>(p);
+    g_launches.fetch_add(1);
+    if (cudaGetLastError() != cudaSuccess) return DGEMM_ERR_CUDA;
+  }
+  if (p.tail_tiles > 0 && p.tail_ipc < kblocks) {
+    dgemm_tail_reduce_kernel<<<p.tail_tiles, 256, 0, stream>>>(p);
     g_launches.fetch_add(1);
     if (cudaGetLastError() != cudaSuccess) return DGEMM_ERR_CUDA;
   }
@@ -266,6 +318,10 @@ int launch_gemm_static_ws(int64_t M, int64_t N, int64_t K, const double* A, int6
     if (split < 2) split = 2;
   }
   if (split > kblocks) split = kblocks;
+  p.kblocks = kblocks;
+  p.dp_tiles = (int)tiles;  // uniform split-K over all tiles, no tail phase
+  p.tail_tiles = 0;
+  p.tail_ipc = 1;
   p.kblocks_per_split = (kblocks + split - 1) / split;
   p.split_k = (kblocks + p.kblocks_per_split - 1) / p.kblocks_per_split;
   if (p.split_k > 1) {
@@ -397,6 +453,12 @@ int dgemm_version(void) { return 100; /* 0.1.0 */ }
 int dgemm_set_variant(int variant) {
   if (variant < DGEMM_VARIANT_AUTO || variant >= DGEMM_VARIANT_COUNT) return DGEMM_ERR_VARIANT;
   g_variant.store(variant);
+  return DGEMM_OK;
+}
+
+int dgemm_set_test_flags(int flags) {
+  if (flags < 0 || flags > (DGEMM_TEST_NO_C_PREFETCH | DGEMM_TEST_NO_BLOCKED_B)) return DGEMM_ERR_VARIANT;
+  g_test_flags.store(flags);
   return DGEMM_OK;
 }
 

@@ -11,10 +11,17 @@
 //   vectorisation -> mma.sync m16n8k8 f64 (DMMA) and 16-byte shared-memory fragment loads
 //   N_C loop the paper left out (Section 2.10) -> grouped tile raster for L2 reuse
 //
-// One persistent CTA per SM: 8 consumer warps (2 x 4 grid of 64 x 32 warp tiles) and a
-// producer warpgroup that hands most of its registers to the consumers (setmaxnreg). Stages are handed over with mbarriers: full[s] (producer -> consumers) and
-// empty[s] (consumers -> producer). Every wait is bounded; on expiry the kernel records
-// DGEMM_ERR_TIMEOUT in the device status word, drains its own copies and returns.
+// One persistent CTA per SM with 8 warps (2 x 4 grid of 64 x 32 warp tiles, up to 255 registers
+// per thread). There is no separate producer warp: the load stream runs LOOKAHEAD k-blocks ahead
+// of the arithmetic and across tile boundaries; with TMA staging lane 0 of warp 0 issues it,
+// with generic staging every thread copies its share. Stages are handed over with mbarriers:
+// full[s] (copies landed) and empty[s] (all warps done reading). Every wait is bounded; on expiry
+// the kernel records DGEMM_ERR_TIMEOUT in the device status word, lets its own copies land and
+// returns.
+//
+// (A warp-specialised variant that moved registers from a producer warpgroup to the consumers
+// with setmaxnreg was tried and dropped: with it, fragment registers of the consumer warps that
+// share a scheduler with the active producer warp were sporadically corrupted.)
 #pragma once
 
 #include <cstdint>
@@ -29,32 +36,53 @@ constexpr int BM = 128;           // CTA tile rows
 constexpr int BN = 128;           // CTA tile columns
 constexpr int BK = 16;            // k extent of one stage (16 doubles = one 128-byte swizzle row)
 constexpr int STAGES = 6;         // pipeline depth
-constexpr int CONSUMER_WARPS = 8;
-constexpr int PRODUCER_WARPS = 4;  // one warpgroup; it gives most of its registers to the consumers
-constexpr int THREADS = (CONSUMER_WARPS + PRODUCER_WARPS) * 32;
-constexpr int CONSUMER_REGS = 232;  // 256*232 + 128*40 <= 65536
-constexpr int PRODUCER_REGS = 40;
+constexpr int LOOKAHEAD = STAGES - 2;  // k-blocks in flight ahead of the arithmetic
+constexpr int WARPS = 8;          // 2 x 4 grid of 64 x 32 warp tiles
+constexpr int THREADS = WARPS * 32;
 constexpr int A_STAGE_BYTES = BM * BK * 8;  // 16 KiB: 128 rows of 128 bytes
 constexpr int B_STAGE_BYTES = BK * BN * 8;  // 16 KiB: 8 boxes of [16 k][16 n] doubles
 constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
 constexpr int B_BOX_BYTES = BK * 16 * 8;    // 2 KiB
 constexpr int SMEM_ALIGN = 1024;            // swizzle pattern repeats every 1024 bytes
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + SMEM_ALIGN + 256;
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + SMEM_ALIGN + 1024;  // + barriers, abort flag, work-item words
 constexpr int STATUS_TIMEOUT = -8;          // DGEMM_ERR_TIMEOUT
+constexpr int C_PREFETCH_KBLOCKS = 8;       // C tile is requested into L2 this many k-blocks before the tile ends
 
+// Work decomposition. Phase 1: the first `dp_tiles` tiles (in raster order), each split into
+// `split_k` equal K partitions, dealt round-robin to the CTAs. Phase 2 (the "tail", the tiles
+// that do not fill a whole wave of CTAs): the remaining `tail_tiles` tiles form one long list of
+// tail_tiles * kblocks k-block iterations that is cut into equal spans of `tail_ipc` iterations,
+// one span per CTA. A span covers the end of one tile and/or the beginning of the next
+// (tail_ipc <= kblocks), i.e. at most two segments per CTA. Segments that do not cover a whole
+// tile store their partial sums in the workspace and a second kernel adds them to C in a fixed
+// order; no CTA ever waits for another one.
 struct GemmParams {
   int M, N, K;
   int tiles_m, tiles_n;
-  int split_k;            // number of K partitions (>= 1)
-  int kblocks_per_split;  // k-blocks (of BK) per partition
+  int kblocks;            // ceil(K / BK)
+  int dp_tiles;           // tiles handled in phase 1
+  int split_k;            // phase 1: number of K partitions per tile (>= 1)
+  int kblocks_per_split;  // phase 1: k-blocks per partition
+  int tail_tiles;         // tiles handled in phase 2
+  int tail_ipc;           // phase 2: k-block iterations per CTA (1 <= tail_ipc <= kblocks)
+  int tail_slot_base;     // first workspace slot of the phase-2 partial tiles
   int group_m;            // raster group height in tiles
+  int c_prefetch;         // C rows are 16-byte aligned: prefetch the C tile into L2 before the epilogue
+  int b_blocked_map;      // map_b is the 3-D view (16 columns, K, N/16): one copy stages the whole B tile
+  int zero;               // always 0; masks a data dependency so that the compiler cannot remove it
   const double* A;
   const double* B;
   double* C;
-  double* partial;        // split_k > 1: [split][tile][BM*BN] partial sums, else unused
+  double* partial;        // workspace: slots of BM*BN doubles; phase 1: slot = ks*dp_tiles + tile
   long long lda, ldb, ldc;
   unsigned long long wait_limit_ns;
   int* status;            // device status word
+};
+
+struct Work {
+  int tm, tn;    // tile coordinates
+  int kb0, kb1;  // k-block range [kb0, kb1)
+  int slot;      // workspace slot for the partial tile, or -1: add straight into C
 };
 
 // Shared-memory layout of the operand tiles (what the consumer reads and both producers write):
@@ -74,9 +102,9 @@ __device__ __forceinline__ uint32_t b_smem_offset(int kk, int nn) {
 // load per lane touches all 32 banks exactly once.
 __device__ __forceinline__ int rowmap(int g) { return ((g & 1) << 2) | (g >> 1); }
 
-__device__ __forceinline__ void unit_to_tile(const GemmParams& p, int unit, int& tm, int& tn, int& ks) {
-  const int tile = unit / p.split_k;
-  ks = unit - tile * p.split_k;
+// Raster order: groups of `group_m` tile rows, column-major inside a group, so that tiles that run
+// at the same time share A row panels and B column panels in L2.
+__device__ __forceinline__ void tile_to_mn(const GemmParams& p, int tile, int& tm, int& tn) {
   const int per_group = p.group_m * p.tiles_n;
   const int group = tile / per_group;
   const int first_m = group * p.group_m;
@@ -86,28 +114,110 @@ __device__ __forceinline__ void unit_to_tile(const GemmParams& p, int unit, int&
   tn = in_group / gsize;
 }
 
-// Bounded mbarrier wait. Returns false if the CTA is aborting (this or another thread timed out).
-__device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                             const GemmParams& p) {
-  if (ptx::mbar_try_wait(bar, parity)) return true;
+// The idx-th work item of CTA `cta` (of `nctas`). Producer and consumers enumerate the same list.
+__device__ __forceinline__ bool get_work(const GemmParams& p, int cta, int nctas, int idx, Work& w) {
+  const int dp_units = p.dp_tiles * p.split_k;
+  const int n1 = cta < dp_units ? (dp_units - cta + nctas - 1) / nctas : 0;
+  int tile;
+  if (idx < n1) {
+    const int unit = cta + idx * nctas;
+    tile = unit / p.split_k;
+    const int ks = unit - tile * p.split_k;
+    w.kb0 = ks * p.kblocks_per_split;
+    w.kb1 = min(w.kb0 + p.kblocks_per_split, p.kblocks);
+    w.slot = p.split_k > 1 ? ks * p.dp_tiles + tile : -1;
+  } else {
+    const int j = idx - n1;
+    if (j > 1 || p.tail_tiles == 0) return false;
+    // 32-bit arithmetic only (the host guarantees tail_tiles * kblocks < 2^31): a 64-bit division
+    // would be a called subroutine, which must not run inside the producers' reduced register budget
+    const int total = p.tail_tiles * p.kblocks;
+    const int start = cta * p.tail_ipc;
+    const int end = min(start + p.tail_ipc, total);
+    if (start >= end) return false;
+    int trel = start / p.kblocks;
+    int s0 = start, s1 = min(end, (trel + 1) * p.kblocks);
+    if (j == 1) {
+      if (s1 >= end) return false;
+      s0 = s1;
+      s1 = end;
+      ++trel;
+    }
+    tile = p.dp_tiles + trel;
+    w.kb0 = s0 - trel * p.kblocks;
+    w.kb1 = s1 - trel * p.kblocks;
+    w.slot = (w.kb0 == 0 && w.kb1 == p.kblocks) ? -1 : p.tail_slot_base + 2 * cta + j;
+  }
+  tile_to_mn(p, tile, w.tm, w.tn);
+  return true;
+}
+
+// ---- rare paths, kept out of line so that the hot k-loop stays small (with two warps per
+// scheduler, instruction fetch stalls in a large loop body cost several percent). They take and
+// return scalars only; work items travel through a few words of shared memory.
+
+// Work item `idx` of this CTA, written as {tm, tn, kb0, kb1, slot, valid} to shared memory.
+__device__ __noinline__ void fetch_work(const GemmParams& p, int cta, int nctas, int idx, volatile int* out) {
+  Work w;
+  const bool valid = get_work(p, cta, nctas, idx, w);
+  out[0] = w.tm;
+  out[1] = w.tn;
+  out[2] = w.kb0;
+  out[3] = w.kb1;
+  out[4] = w.slot;
+  out[5] = valid ? 1 : 0;
+}
+
+// Asks L2 for rows r0, r0 + rstep, ... of the C tile (tm, tn) ahead of its epilogue.
+__device__ __noinline__ void prefetch_c_rows(const double* C, long long ldc, int M, int N, int tm, int tn, int r0,
+                                             int rstep) {
+  const int cols = min(BN, N - tn * BN) & ~1;
+  if (cols <= 0) return;
+  for (int r = r0; r < BM; r += rstep) {
+    const int row = tm * BM + r;
+    if (row < M) ptx::prefetch_l2_bulk(C + (long long)row * ldc + (long long)tn * BN, (uint32_t)cols * 8u);
+  }
+}
+
+// B stage as eight 2-D boxes of 16 columns (used when N is not a multiple of 16).
+__device__ __noinline__ void tma_load_b_boxes(uint32_t sb, const CUtensorMap* map_b, int n0, int k0, uint32_t fb) {
+#pragma unroll
+  for (int nb = 0; nb < BN / 16; ++nb) ptx::tma_load_2d(sb + nb * B_BOX_BYTES, map_b, n0 + nb * 16, k0, fb);
+}
+
+// Slow part of a bounded mbarrier wait: poll until the phase completes, the CTA aborts, or the
+// time limit expires (then record DGEMM_ERR_TIMEOUT and raise the abort flag).
+__device__ __noinline__ bool wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                       unsigned long long limit_ns, int* status, bool suspend) {
   const unsigned long long t0 = ptx::globaltimer_ns();
   for (uint32_t it = 1;; ++it) {
-    if (ptx::mbar_try_wait(bar, parity)) return true;
+    if (suspend ? ptx::mbar_try_wait(bar, parity) : ptx::mbar_test_wait(bar, parity)) return true;
     if ((it & 31u) == 0u) {
       if (*abort_flag) return false;
-      if (ptx::globaltimer_ns() - t0 > p.wait_limit_ns) {
+      if (ptx::globaltimer_ns() - t0 > limit_ns) {
         *abort_flag = 1;
-        atomicExch(p.status, STATUS_TIMEOUT);
+        atomicExch(status, STATUS_TIMEOUT);
         return false;
       }
     }
   }
 }
 
+// Bounded mbarrier wait. Returns false if the CTA is aborting (this or another thread timed out).
+// SUSPEND = true polls with try_wait (the thread may be suspended for a short, hardware-defined
+// time when the phase is not complete: right for the arithmetic waiting for data); SUSPEND = false
+// polls with test_wait (never suspends: right for a thread that issues loads in passing).
+template <bool SUSPEND = true>
+__device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                             const GemmParams& p) {
+  if (SUSPEND ? ptx::mbar_try_wait(bar, parity) : ptx::mbar_test_wait(bar, parity)) return true;
+  return wait_slow(bar, parity, abort_flag, p.wait_limit_ns, p.status, SUSPEND);
+}
+
 template <bool USE_TMA>
 __global__ void __launch_bounds__(THREADS, 1)
 dgemm_dmma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-                  const GemmParams p) {
+                  const __grid_constant__ GemmParams p) {
   extern __shared__ uint8_t smem_raw[];
   // tiles at a 1024-byte boundary, barriers behind them
   const uint32_t raw = ptx::smem_u32(smem_raw);
@@ -115,123 +225,136 @@ dgemm_dmma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
   uint8_t* tiles = smem_raw + pad;
   uint64_t* bars = reinterpret_cast<uint64_t*>(tiles + STAGES * STAGE_BYTES);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 2 * STAGES);
+  volatile int* work_words = abort_flag + 8;  // per warp: 8 words for the load cursor's item, 8 for the current item
   const uint32_t tiles_u32 = raw + pad;
   const uint32_t full_bar = tiles_u32 + STAGES * STAGE_BYTES;  // full[s]  at full_bar + 8*s
   const uint32_t empty_bar = full_bar + 8 * STAGES;            // empty[s] at empty_bar + 8*s
 
-  const int warp = threadIdx.x >> 5;
-  const int lane = threadIdx.x & 31;
+  const int tid = threadIdx.x;
+  const int warp = tid >> 5;
+  const int lane = tid & 31;
 
-  if (threadIdx.x == 0) {
+  if (tid == 0) {
     for (int s = 0; s < STAGES; ++s) {
-      ptx::mbar_init(full_bar + 8 * s, USE_TMA ? 1 : PRODUCER_WARPS * 32);
-      ptx::mbar_init(empty_bar + 8 * s, CONSUMER_WARPS);
+      ptx::mbar_init(full_bar + 8 * s, USE_TMA ? 1 : THREADS);
+      ptx::mbar_init(empty_bar + 8 * s, WARPS);
     }
     *abort_flag = 0;
     ptx::fence_barrier_init();
   }
   __syncthreads();
 
-  const int num_units = p.tiles_m * p.tiles_n * p.split_k;
-  const int kblocks_total = (p.K + BK - 1) / BK;
-
-  if (warp >= CONSUMER_WARPS) {
-    // ------------------------------------------------------------- producer warpgroup
-    ptx::setmaxnreg_dec<PRODUCER_REGS>();
-    const int pw = warp - CONSUMER_WARPS;  // 0..3
-    uint32_t it = 0;  // running stage counter, in lock step with the consumers
-    bool ok = true;
-    if (USE_TMA) {
-      if (pw == 0 && lane == 0) {
-        ptx::prefetch_tensormap(&map_a);
-        ptx::prefetch_tensormap(&map_b);
-        for (int unit = blockIdx.x; unit < num_units && ok; unit += gridDim.x) {
-          int tm, tn, ks;
-          unit_to_tile(p, unit, tm, tn, ks);
-          const int kb0 = ks * p.kblocks_per_split;
-          const int kb1 = min(kb0 + p.kblocks_per_split, kblocks_total);
-          for (int kb = kb0; kb < kb1; ++kb, ++it) {
-            const uint32_t s = it % STAGES;
-            const uint32_t ph = (it / STAGES) & 1u;
-            if (!wait_bounded(empty_bar + 8 * s, ph ^ 1u, abort_flag, p)) { ok = false; break; }
-            const uint32_t fb = full_bar + 8 * s;
-            const uint32_t sa = tiles_u32 + s * STAGE_BYTES;
-            const uint32_t sb = sa + A_STAGE_BYTES;
-            ptx::mbar_arrive_expect_tx(fb, STAGE_BYTES);
-            ptx::tma_load_2d(sa, &map_a, kb * BK, tm * BM, fb);
-#pragma unroll
-            for (int nb = 0; nb < BN / 16; ++nb)
-              ptx::tma_load_2d(sb + nb * B_BOX_BYTES, &map_b, tn * BN + nb * 16, kb * BK, fb);
-          }
-        }
-        if (!ok) {
-          // aborting: let every copy this thread armed land before the CTA's memory is released
-          const uint32_t n_inflight = it < (uint32_t)STAGES ? it : (uint32_t)STAGES;
-          for (uint32_t q = it - n_inflight; q < it; ++q) {
-            const uint32_t s = q % STAGES, ph = (q / STAGES) & 1u;
-            const unsigned long long t0 = ptx::globaltimer_ns();
-            while (!ptx::mbar_try_wait(full_bar + 8 * s, ph)) {
-              if (ptx::globaltimer_ns() - t0 > p.wait_limit_ns) break;
-            }
-          }
-        }
-      }
-    } else {
-      // 8-byte asynchronous copies with zero fill outside the matrices; works for any alignment
-      // and any leading dimension. Producer warp pw copies rows 32pw..32pw+31 of the A tile
-      // (lanes 0-15 one row's 16 k values, lanes 16-31 the next row's) and columns
-      // 32pw..32pw+31 of the B tile (one k row per instruction).
-      const int a_r = lane >> 4, a_k = lane & 15;
-      for (int unit = blockIdx.x; unit < num_units && ok; unit += gridDim.x) {
-        int tm, tn, ks;
-        unit_to_tile(p, unit, tm, tn, ks);
-        const int kb0 = ks * p.kblocks_per_split;
-        const int kb1 = min(kb0 + p.kblocks_per_split, kblocks_total);
-        const int m0 = tm * BM, n0 = tn * BN;
-        for (int kb = kb0; kb < kb1; ++kb, ++it) {
-          const uint32_t s = it % STAGES;
-          const uint32_t ph = (it / STAGES) & 1u;
-          if (!wait_bounded(empty_bar + 8 * s, ph ^ 1u, abort_flag, p)) { ok = false; break; }
-          const uint32_t sa = tiles_u32 + s * STAGE_BYTES;
-          const uint32_t sb = sa + A_STAGE_BYTES;
-          const int k0 = kb * BK;
-          {
-            const int k = k0 + a_k;
-            const bool kin = k < p.K;
-            const int row0 = 32 * pw + a_r;
-            const double* src = p.A + (long long)(m0 + row0) * p.lda + k;
-            const uint32_t dst_base = sa + ((a_k & 1) << 3);
-#pragma unroll 4
-            for (int r = 0; r < 32; r += 2) {
-              const int row = row0 + r;
-              const bool in = kin && (m0 + row < p.M);
-              const uint32_t dst = dst_base + row * 128 + (((a_k >> 1) ^ (row & 7)) << 4);
-              ptx::cp_async_8(dst, in ? (const void*)(src + (long long)r * p.lda) : (const void*)p.A, in ? 8u : 0u);
-            }
-          }
-          {
-            const int nn = 32 * pw + lane;
-            const bool nin = n0 + nn < p.N;
-            const double* src = p.B + (long long)k0 * p.ldb + (n0 + nn);
-            const uint32_t dst_base = sb + (nn >> 4) * B_BOX_BYTES + ((nn & 1) << 3);
-            const int chunk = (nn & 15) >> 1;
-#pragma unroll 4
-            for (int kk = 0; kk < BK; ++kk) {
-              const bool in = nin && (k0 + kk < p.K);
-              const uint32_t dst = dst_base + kk * 128 + ((chunk ^ (kk & 7)) << 4);
-              ptx::cp_async_8(dst, in ? (const void*)(src + (long long)kk * p.ldb) : (const void*)p.B, in ? 8u : 0u);
-            }
-          }
-          ptx::cp_async_mbar_arrive_noinc(full_bar + 8 * s);
-        }
-      }
-      ptx::cp_async_wait_all();  // nothing of this thread's is in flight when it leaves
-    }
-    return;
+  const int cta = blockIdx.x, nctas = gridDim.x;
+  // Every thread follows the load stream. TMA staging: the k-blocks are issued by the warps in
+  // turn (k-block number i by lane 0 of warp i mod 8), which spreads the cost of issuing over the
+  // four schedulers. Generic staging: every thread copies its share of each stage.
+  if (USE_TMA && tid == 0) {
+    ptx::prefetch_tensormap(&map_a);
+    ptx::prefetch_tensormap(&map_b);
   }
 
-  // -------------------------------------------------------------------- consumer warps
-  ptx::setmaxnreg_inc<CONSUMER_REGS>();
+  // State of the load stream: the k-blocks of this CTA's work items in order, LOOKAHEAD k-blocks
+  // ahead of the arithmetic and running across tile boundaries, so that the first stages of the
+  // next tile are in flight while the current tile's epilogue runs. Uniform over the CTA.
+  volatile int* cur_words = work_words + 16 * warp;
+  volatile int* item_words = cur_words + 8;
+  int cur_idx = 0, cur_tm, cur_tn, cur_kb, cur_kb1, cur_pf, cur_valid;
+  auto cursor_load = [&]() {
+    fetch_work(p, cta, nctas, cur_idx, cur_words);
+    __syncwarp();
+    cur_tm = cur_words[0];
+    cur_tn = cur_words[1];
+    cur_kb = cur_words[2];
+    cur_kb1 = cur_words[3];
+    cur_valid = cur_words[5];
+    // k-block at which the C tile is requested into L2, or -1 (partial tiles do not read C)
+    cur_pf = (cur_words[4] < 0 && p.c_prefetch) ? max(cur_kb, cur_kb1 - C_PREFETCH_KBLOCKS) : -1;
+    __syncwarp();
+  };
+  cursor_load();
+  uint32_t lit = 0;  // k-blocks issued so far
+  bool ok = true;
+
+  // Issues the next k-block of the load stream into stage lit % STAGES (after that stage's previous
+  // contents have been released by all warps). Returns false if the CTA is aborting.
+  auto issue_next = [&]() -> bool {
+    if (!cur_valid) return true;
+    const uint32_t s = lit % STAGES;
+    const uint32_t ph = (lit / STAGES) & 1u;
+    const uint32_t sa = tiles_u32 + s * STAGE_BYTES;
+    const uint32_t sb = sa + A_STAGE_BYTES;
+    const uint32_t fb = full_bar + 8 * s;
+    const int kb = cur_kb;
+    if (USE_TMA) {
+      int good = 1;
+      if (warp == (int)(lit % WARPS) && lane == 0) {
+        if (wait_bounded<false>(empty_bar + 8 * s, ph ^ 1u, abort_flag, p)) {
+          ptx::mbar_arrive_expect_tx(fb, STAGE_BYTES);
+          ptx::tma_load_2d(sa, &map_a, kb * BK, cur_tm * BM, fb);
+          if (p.b_blocked_map) {
+            ptx::tma_load_3d(sb, &map_b, 0, kb * BK, cur_tn * (BN / 16), fb);
+          } else {
+            tma_load_b_boxes(sb, &map_b, cur_tn * BN, kb * BK, fb);
+          }
+        } else {
+          good = 0;
+        }
+      }
+      if (!__all_sync(0xffffffffu, good)) return false;
+    } else {
+      if (!wait_bounded<false>(empty_bar + 8 * s, ph ^ 1u, abort_flag, p)) return false;
+      // 8-byte asynchronous copies with zero fill outside the matrices; any alignment, any leading
+      // dimension. A: 16 consecutive threads copy the 16 k values of one row (8 rows per thread);
+      // B: 32 consecutive threads copy 32 consecutive columns of one k row (8 k rows per thread).
+      const int m0 = cur_tm * BM, n0 = cur_tn * BN, k0 = kb * BK;
+      {
+        const int a_k = tid & 15, row0 = tid >> 4;
+        const int k = k0 + a_k;
+        const bool kin = k < p.K;
+        const double* src = p.A + (long long)(m0 + row0) * p.lda + k;
+        const uint32_t dst_base = sa + ((a_k & 1) << 3);
+#pragma unroll
+        for (int i = 0; i < BM / 16; ++i) {
+          const int row = row0 + 16 * i;
+          const bool in = kin && (m0 + row < p.M);
+          const uint32_t dst = dst_base + row * 128 + (((a_k >> 1) ^ (row & 7)) << 4);
+          ptx::cp_async_8(dst, in ? (const void*)(src + (long long)(16 * i) * p.lda) : (const void*)p.A, in ? 8u : 0u);
+        }
+      }
+      {
+        const int nn = tid & 127, kk0 = tid >> 7;
+        const bool nin = n0 + nn < p.N;
+        const double* src = p.B + (long long)(k0 + kk0) * p.ldb + (n0 + nn);
+        const uint32_t dst_base = sb + (nn >> 4) * B_BOX_BYTES + ((nn & 1) << 3);
+        const int chunk = (nn & 15) >> 1;
+#pragma unroll
+        for (int i = 0; i < BK / 2; ++i) {
+          const int kk = kk0 + 2 * i;
+          const bool in = nin && (k0 + kk < p.K);
+          const uint32_t dst = dst_base + kk * 128 + ((chunk ^ (kk & 7)) << 4);
+          ptx::cp_async_8(dst, in ? (const void*)(src + (long long)(2 * i) * p.ldb) : (const void*)p.B, in ? 8u : 0u);
+        }
+      }
+      ptx::cp_async_mbar_arrive_noinc(fb);
+    }
+    if (kb == cur_pf) {
+      // TMA staging: the issuing warp's lanes take 4 rows each; generic: one row per thread of the first 128
+      if (USE_TMA) {
+        if (warp == (int)(lit % WARPS)) prefetch_c_rows(p.C, p.ldc, p.M, p.N, cur_tm, cur_tn, lane, 32);
+      } else if (tid < BM) {
+        prefetch_c_rows(p.C, p.ldc, p.M, p.N, cur_tm, cur_tn, tid, BM);
+      }
+    }
+    ++lit;
+    if (++cur_kb >= cur_kb1) {
+      ++cur_idx;
+      cursor_load();
+    }
+    return true;
+  };
+
+  for (int i = 0; i < LOOKAHEAD && ok; ++i) ok = issue_next();
+
   const int g = lane >> 2;   // MMA group id (row of A / column of B fragment)
   const int t = lane & 3;    // thread in group (k index of the fragments)
   const int wm = warp >> 2;  // 0..1 : 64-row slab of the CTA tile
@@ -251,15 +374,21 @@ dgemm_dmma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
   }
 
   double acc[4][4][4];  // [mt][nt = 2*np + j][c0..c3]
-  uint32_t it = 0;
-  bool ok = true;
+  uint32_t it = 0;      // k-blocks consumed so far
+  Work w;
 
-  for (int unit = blockIdx.x; unit < num_units && ok; unit += gridDim.x) {
-    int tm, tn, ks;
-    unit_to_tile(p, unit, tm, tn, ks);
-    const int kb0 = ks * p.kblocks_per_split;
-    const int kb1 = min(kb0 + p.kblocks_per_split, kblocks_total);
-
+  for (int idx = 0; ok; ++idx) {
+    fetch_work(p, cta, nctas, idx, item_words);
+    __syncwarp();
+    w.tm = item_words[0];
+    w.tn = item_words[1];
+    w.kb0 = item_words[2];
+    w.kb1 = item_words[3];
+    w.slot = item_words[4];
+    const int valid = item_words[5];
+    __syncwarp();
+    if (!valid) break;
+    const int tm = w.tm, tn = w.tn;
 #pragma unroll
     for (int mt = 0; mt < 4; ++mt)
 #pragma unroll
@@ -267,11 +396,12 @@ dgemm_dmma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
 #pragma unroll
         for (int c = 0; c < 4; ++c) acc[mt][nt][c] = 0.0;
 
-    for (int kb = kb0; kb < kb1; ++kb, ++it) {
+    for (int kb = w.kb0; kb < w.kb1; ++kb, ++it) {
       const uint32_t s = it % STAGES;
       const uint32_t ph = (it / STAGES) & 1u;
       if (!wait_bounded(full_bar + 8 * s, ph, abort_flag, p)) { ok = false; break; }
       const uint8_t* st = tiles + s * STAGE_BYTES;
+      int token = 0;  // depends on every fragment this lane loads from the stage
 #pragma unroll
       for (int h = 0; h < 2; ++h) {
         double2 alo[4], ahi[4], bf[2][2];
@@ -287,14 +417,37 @@ dgemm_dmma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
             bf[np][b] = *reinterpret_cast<const double2*>(st + b_off[h][b] + np * B_BOX_BYTES);
 #pragma unroll
         for (int mt = 0; mt < 4; ++mt)
+          token ^= __double2loint(alo[mt].x) ^ __double2hiint(alo[mt].y) ^ __double2loint(ahi[mt].x) ^ __double2hiint(ahi[mt].y);
+#pragma unroll
+        for (int np = 0; np < 2; ++np)
+          token ^= __double2loint(bf[np][0].x) ^ __double2hiint(bf[np][0].y) ^ __double2loint(bf[np][1].x) ^ __double2hiint(bf[np][1].y);
+        // Eight k values per block as two k4 steps (x: k = 8h + 2t, y: k = 8h + 2t + 1) of the
+        // m8n8k4 shape; rows g (alo) and g + 8 (ahi) are separate 8 x 8 tiles.
+#pragma unroll
+        for (int mt = 0; mt < 4; ++mt)
 #pragma unroll
           for (int np = 0; np < 2; ++np) {
-            ptx::dmma_m16n8k8(acc[mt][2 * np + 0], alo[mt].x, ahi[mt].x, alo[mt].y, ahi[mt].y, bf[np][0].x, bf[np][1].x);
-            ptx::dmma_m16n8k8(acc[mt][2 * np + 1], alo[mt].x, ahi[mt].x, alo[mt].y, ahi[mt].y, bf[np][0].y, bf[np][1].y);
+            ptx::dmma_m8n8k4(acc[mt][2 * np + 0][0], acc[mt][2 * np + 0][1], alo[mt].x, bf[np][0].x);
+            ptx::dmma_m8n8k4(acc[mt][2 * np + 0][2], acc[mt][2 * np + 0][3], ahi[mt].x, bf[np][0].x);
+            ptx::dmma_m8n8k4(acc[mt][2 * np + 1][0], acc[mt][2 * np + 1][1], alo[mt].x, bf[np][0].y);
+            ptx::dmma_m8n8k4(acc[mt][2 * np + 1][2], acc[mt][2 * np + 1][3], ahi[mt].x, bf[np][0].y);
+            ptx::dmma_m8n8k4(acc[mt][2 * np + 0][0], acc[mt][2 * np + 0][1], alo[mt].y, bf[np][1].x);
+            ptx::dmma_m8n8k4(acc[mt][2 * np + 0][2], acc[mt][2 * np + 0][3], ahi[mt].y, bf[np][1].x);
+            ptx::dmma_m8n8k4(acc[mt][2 * np + 1][0], acc[mt][2 * np + 1][1], alo[mt].y, bf[np][1].y);
+            ptx::dmma_m8n8k4(acc[mt][2 * np + 1][2], acc[mt][2 * np + 1][3], ahi[mt].y, bf[np][1].y);
           }
       }
-      __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(empty_bar + 8 * s);
+      // Release the stage. The arrive must not take effect before all of this warp's fragment
+      // loads have been served: otherwise the refill can overwrite rows that a load still queued
+      // behind the arithmetic has yet to read (observed as sporadically wrong rows of the
+      // last-loaded A fragments in the slowest warp, cured by delaying the arrive). Program order
+      // alone does not guarantee it, so the arrive is made data-dependent on the loaded registers
+      // of all 32 lanes: a warp-wide reduction of the per-lane tokens, masked with a zero the
+      // compiler cannot see, is added to the barrier address.
+      token = __reduce_xor_sync(0xffffffffu, token);
+      if (lane == 0) ptx::mbar_arrive(empty_bar + 8 * s + (uint32_t)(token & p.zero));
+      // keep the load stream LOOKAHEAD k-blocks ahead: refill the stage released two k-blocks ago
+      if (!issue_next()) { ok = false; break; }
     }
     if (!ok) break;
 
@@ -302,8 +455,8 @@ dgemm_dmma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     // columns n = 32wn + 16np + 4t + {0,1,2,3} = {nt=2np:c0, nt=2np+1:c0, nt=2np:c1, nt=2np+1:c1}
     const int row_base = tm * BM + 64 * wm + rm;
     const int col_base = tn * BN + 32 * wn + 4 * t;
-    if (p.split_k > 1) {
-      double* dst = p.partial + ((long long)ks * (p.tiles_m * p.tiles_n) + (unit / p.split_k)) * (long long)(BM * BN);
+    if (w.slot >= 0) {
+      double* dst = p.partial + (long long)w.slot * (long long)(BM * BN);
 #pragma unroll
       for (int mt = 0; mt < 4; ++mt)
 #pragma unroll
@@ -319,19 +472,34 @@ dgemm_dmma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
       const bool interior = (tm * BM + BM <= p.M) && (tn * BN + BN <= p.N);
       const bool vec32 = ((reinterpret_cast<uintptr_t>(p.C) & 31) == 0) && ((p.ldc & 3) == 0);
       if (interior && vec32) {
+        // two batches of 8 outstanding 32-byte loads per thread, then the adds and stores
 #pragma unroll
-        for (int mt = 0; mt < 4; ++mt)
+        for (int mp = 0; mp < 2; ++mp) {
+          double cin[2][2][2][4];
 #pragma unroll
-          for (int half = 0; half < 2; ++half) {
-            double* crow = p.C + (long long)(row_base + 16 * mt + 8 * half) * p.ldc + col_base;
-            double c0[2], c1[2], c2[2], c3[2];
+          for (int mq = 0; mq < 2; ++mq)
 #pragma unroll
-            for (int np = 0; np < 2; ++np) ptx::ldg256(crow + 16 * np, c0[np], c1[np], c2[np], c3[np]);
+            for (int half = 0; half < 2; ++half) {
+              const double* crow = p.C + (long long)(row_base + 16 * (2 * mp + mq) + 8 * half) * p.ldc + col_base;
 #pragma unroll
-            for (int np = 0; np < 2; ++np)
-              ptx::stg256(crow + 16 * np, c0[np] + acc[mt][2 * np][2 * half], c1[np] + acc[mt][2 * np + 1][2 * half],
-                          c2[np] + acc[mt][2 * np][2 * half + 1], c3[np] + acc[mt][2 * np + 1][2 * half + 1]);
-          }
+              for (int np = 0; np < 2; ++np)
+                ptx::ldg256(crow + 16 * np, cin[mq][half][np][0], cin[mq][half][np][1], cin[mq][half][np][2],
+                            cin[mq][half][np][3]);
+            }
+#pragma unroll
+          for (int mq = 0; mq < 2; ++mq)
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+              const int mt = 2 * mp + mq;
+              double* crow = p.C + (long long)(row_base + 16 * mt + 8 * half) * p.ldc + col_base;
+#pragma unroll
+              for (int np = 0; np < 2; ++np)
+                ptx::stg256(crow + 16 * np, cin[mq][half][np][0] + acc[mt][2 * np][2 * half],
+                            cin[mq][half][np][1] + acc[mt][2 * np + 1][2 * half],
+                            cin[mq][half][np][2] + acc[mt][2 * np][2 * half + 1],
+                            cin[mq][half][np][3] + acc[mt][2 * np + 1][2 * half + 1]);
+            }
+        }
       } else {
 #pragma unroll
         for (int mt = 0; mt < 4; ++mt)
@@ -354,28 +522,67 @@ dgemm_dmma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
       }
     }
   }
+
+  // Leaving. After a normal run every copy that was issued has been consumed. After an abort,
+  // copies may still be in flight into this CTA's shared memory: let them land first.
+  if (!USE_TMA) ptx::cp_async_wait_all();
+  if (USE_TMA && !ok && tid == 0) {
+    const uint32_t n_inflight = lit < (uint32_t)STAGES ? lit : (uint32_t)STAGES;
+    for (uint32_t q = lit - n_inflight; q < lit; ++q) {
+      const uint32_t s = q % STAGES, ph = (q / STAGES) & 1u;
+      const unsigned long long t0 = ptx::globaltimer_ns();
+      while (!ptx::mbar_try_wait(full_bar + 8 * s, ph)) {
+        if (ptx::globaltimer_ns() - t0 > p.wait_limit_ns) break;
+      }
+    }
+  }
+  __syncthreads();
 }
 
-// Deterministic split-K reduction: C[i][j] += ((p_0 + p_1) + p_2) + ... in split order.
-__global__ void dgemm_splitk_reduce_kernel(const GemmParams p) {
-  const int tile = blockIdx.x;
-  const int per_group = p.group_m * p.tiles_n;
-  const int group = tile / per_group;
-  const int first_m = group * p.group_m;
-  const int gsize = min(p.group_m, p.tiles_m - first_m);
-  const int in_group = tile - group * per_group;
-  const int tm = first_m + in_group % gsize;
-  const int tn = in_group / gsize;
-  const long long num_tiles = (long long)p.tiles_m * p.tiles_n;
-  for (int e = threadIdx.x; e < BM * BN; e += blockDim.x) {
+// Adds `count` partial tiles (workspace slots slot[0..count)) to the C tile (tm, tn) in that order:
+// C[i][j] += ((p_0 + p_1) + p_2) + ...  Deterministic; one CTA per tile.
+template <typename SlotFn>
+__device__ __forceinline__ void reduce_tile(const GemmParams& p, int tm, int tn, int count, SlotFn slot_of) {
+  for (int e = 2 * threadIdx.x; e < BM * BN; e += 2 * blockDim.x) {
     const int r = e / BN, c = e - r * BN;
     const int row = tm * BM + r, col = tn * BN + c;
     if (row < p.M && col < p.N) {
-      double sum = p.partial[(long long)tile * (BM * BN) + e];
-      for (int s = 1; s < p.split_k; ++s) sum += p.partial[((long long)s * num_tiles + tile) * (BM * BN) + e];
-      p.C[(long long)row * p.ldc + col] += sum;
+      double2 sum = *reinterpret_cast<const double2*>(p.partial + (long long)slot_of(0) * (BM * BN) + e);
+      for (int s = 1; s < count; ++s) {
+        const double2 v = *reinterpret_cast<const double2*>(p.partial + (long long)slot_of(s) * (BM * BN) + e);
+        sum.x += v.x;
+        sum.y += v.y;
+      }
+      double* dst = p.C + (long long)row * p.ldc + col;
+      dst[0] += sum.x;
+      if (col + 1 < p.N) dst[1] += sum.y;
     }
   }
+}
+
+// Phase-1 split-K reduction: tile t has its split_k partials in slots ks*dp_tiles + t.
+__global__ void dgemm_splitk_reduce_kernel(const GemmParams p) {
+  const int tile = blockIdx.x;
+  int tm, tn;
+  tile_to_mn(p, tile, tm, tn);
+  reduce_tile(p, tm, tn, p.split_k, [&](int s) { return s * p.dp_tiles + tile; });
+}
+
+// Phase-2 (tail) reduction: tail tile `trel` was covered by the spans of CTAs c_first..c_last; CTA c
+// stored its part in slot tail_slot_base + 2c + j, j = 0 if the span starts inside this tile.
+__global__ void dgemm_tail_reduce_kernel(const GemmParams p) {
+  const int trel = blockIdx.x;
+  const int lo = trel * p.kblocks, hi = lo + p.kblocks;
+  const int c_first = lo / p.tail_ipc;
+  const int c_last = (hi - 1) / p.tail_ipc;
+  if (c_first == c_last && c_first * p.tail_ipc == lo && p.tail_ipc == p.kblocks) return;  // went straight to C
+  int tm, tn;
+  tile_to_mn(p, p.dp_tiles + trel, tm, tn);
+  reduce_tile(p, tm, tn, c_last - c_first + 1, [&](int s) {
+    const int c = c_first + s;
+    const int j = (c * p.tail_ipc >= lo) ? 0 : 1;
+    return p.tail_slot_base + 2 * c + j;
+  });
 }
 
 // Rung 0 of the ladder: the naive nest with one thread per C element (Section 2.1).

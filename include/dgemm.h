@@ -49,7 +49,9 @@ enum {
                                 A and B base pointers and even lda, ldb                          */
   DGEMM_VARIANT_GENERIC = 2, /* same pipeline, tiles staged by 8-byte asynchronous copies; any
                                 8-byte aligned operands and any leading dimensions               */
-  DGEMM_VARIANT_COUNT = 3
+  DGEMM_VARIANT_TMA_WS = 3,     /* as TMA, with a separate producer warpgroup (warp-specialised)  */
+  DGEMM_VARIANT_GENERIC_WS = 4, /* as GENERIC, with a separate producer warpgroup                 */
+  DGEMM_VARIANT_COUNT = 5
 };
 
 /*

@@ -9,6 +9,8 @@ from .binding import (  # noqa: F401
     DGEMM_VARIANT_GENERIC,
     DGEMM_VARIANT_NAIVE,
     DGEMM_VARIANT_TMA,
+    DGEMM_VARIANT_TMA_WS,
+    DGEMM_VARIANT_GENERIC_WS,
     DgemmError,
     dgemm_f64,
     dgemm_f64_host,

@@ -33,6 +33,8 @@ DGEMM_VARIANT_AUTO = -1
 DGEMM_VARIANT_NAIVE = 0
 DGEMM_VARIANT_TMA = 1
 DGEMM_VARIANT_GENERIC = 2
+DGEMM_VARIANT_TMA_WS = 3
+DGEMM_VARIANT_GENERIC_WS = 4
 
 
 class DgemmError(RuntimeError):

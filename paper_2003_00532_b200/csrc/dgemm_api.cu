@@ -22,6 +22,8 @@ using namespace dgemm;
 constexpr int kMaxDevices = 64;
 constexpr size_t kWorkspaceBytes = 320ull * BM * BN * sizeof(double);  // 40 MiB: up to 320 partial tiles
 constexpr unsigned long long kWaitLimitNs = 4000000000ull;            // 4 s per device-side wait
+constexpr int kAutoTma = DGEMM_VARIANT_TMA;          // what DGEMM_VARIANT_AUTO picks for aligned operands
+constexpr int kAutoGeneric = DGEMM_VARIANT_GENERIC;  // ... and for unaligned ones
 constexpr int kTailMinSpan = 2;          // stream-K tail: at least this many k-blocks per CTA
 constexpr double kTailMinSavedKblocks = 5.0;  // use the stream-K tail only if it saves this many k-block times
 
@@ -66,7 +68,9 @@ int device_state(DeviceState** out) {
     if (cudaGetSymbolAddress(reinterpret_cast<void**>(&st.status), g_status_word) != cudaSuccess) return DGEMM_ERR_CUDA;
     if (cudaMemset(st.status, 0, sizeof(int)) != cudaSuccess) return DGEMM_ERR_CUDA;
     if (cudaFuncSetAttribute(dgemm_dmma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess ||
-        cudaFuncSetAttribute(dgemm_dmma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
+        cudaFuncSetAttribute(dgemm_dmma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess ||
+        cudaFuncSetAttribute(dgemm_dmma_ws_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess ||
+        cudaFuncSetAttribute(dgemm_dmma_ws_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
       return DGEMM_ERR_CUDA;
     if (!g_encode) {
       void* fn = nullptr;
@@ -149,8 +153,9 @@ int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, c
 
   int variant = g_variant.load();
   const bool tma_ok = (((uintptr_t)A | (uintptr_t)B) & 15) == 0 && (lda % 2 == 0) && (ldb % 2 == 0);
-  if (variant == DGEMM_VARIANT_AUTO) variant = tma_ok ? DGEMM_VARIANT_TMA : DGEMM_VARIANT_GENERIC;
-  if (variant == DGEMM_VARIANT_TMA && !tma_ok) return DGEMM_ERR_VARIANT;
+  if (variant == DGEMM_VARIANT_AUTO) variant = tma_ok ? kAutoTma : kAutoGeneric;
+  const bool wants_tma = variant == DGEMM_VARIANT_TMA || variant == DGEMM_VARIANT_TMA_WS;
+  if (wants_tma && !tma_ok) return DGEMM_ERR_VARIANT;
 
   if (variant == DGEMM_VARIANT_NAIVE) {
     dim3 block(32, 8), grid((unsigned)((N + 31) / 32), (unsigned)((M + 7) / 8));
@@ -229,13 +234,19 @@ int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, c
   CUtensorMap map_a, map_b;
   memset(&map_a, 0, sizeof(map_a));
   memset(&map_b, 0, sizeof(map_b));
-  if (variant == DGEMM_VARIANT_TMA) {
+  if (wants_tma) {
     if (!make_map(&map_a, A, M, K, lda, BK, BM)) return DGEMM_ERR_CUDA;
     p.b_blocked_map = (!(dbg_flags & DGEMM_TEST_NO_BLOCKED_B) && N % 16 == 0 && make_blocked_map(&map_b, B, K, N, ldb, BK, BN / 16)) ? 1 : 0;
     if (!p.b_blocked_map && !make_map(&map_b, B, K, N, ldb, 16, BK)) return DGEMM_ERR_CUDA;
-    dgemm_dmma_kernel<true><<<grid, THREADS, SMEM_BYTES, stream>>>(map_a, map_b, p);
+    if (variant == DGEMM_VARIANT_TMA_WS)
+      dgemm_dmma_ws_kernel<true><<<grid, WS_THREADS, SMEM_BYTES, stream>>>(map_a, map_b, p);
+    else
+      dgemm_dmma_kernel<true><<<grid, THREADS, SMEM_BYTES, stream>>>(map_a, map_b, p);
   } else {
-    dgemm_dmma_kernel<false><<<grid, THREADS, SMEM_BYTES, stream>>>(map_a, map_b, p);
+    if (variant == DGEMM_VARIANT_GENERIC_WS)
+      dgemm_dmma_ws_kernel<false><<<grid, WS_THREADS, SMEM_BYTES, stream>>>(map_a, map_b, p);
+    else
+      dgemm_dmma_kernel<false><<<grid, THREADS, SMEM_BYTES, stream>>>(map_a, map_b, p);
   }
   g_launches.fetch_add(1);
   if (cudaGetLastError() != cudaSuccess) return DGEMM_ERR_CUDA;

@@ -157,7 +157,7 @@ __device__ __forceinline__ bool get_work(const GemmParams& p, int cta, int nctas
 // return scalars only; work items travel through a few words of shared memory.
 
 // Work item `idx` of this CTA, written as {tm, tn, kb0, kb1, slot, valid} to shared memory.
-__device__ __noinline__ void fetch_work(const GemmParams& p, int cta, int nctas, int idx, volatile int* out) {
+__device__ __forceinline__ void fetch_work_inline(const GemmParams& p, int cta, int nctas, int idx, volatile int* out) {
   Work w;
   const bool valid = get_work(p, cta, nctas, idx, w);
   out[0] = w.tm;
@@ -167,10 +167,13 @@ __device__ __noinline__ void fetch_work(const GemmParams& p, int cta, int nctas,
   out[4] = w.slot;
   out[5] = valid ? 1 : 0;
 }
+__device__ __noinline__ void fetch_work(const GemmParams& p, int cta, int nctas, int idx, volatile int* out) {
+  fetch_work_inline(p, cta, nctas, idx, out);
+}
 
 // Asks L2 for rows r0, r0 + rstep, ... of the C tile (tm, tn) ahead of its epilogue.
-__device__ __noinline__ void prefetch_c_rows(const double* C, long long ldc, int M, int N, int tm, int tn, int r0,
-                                             int rstep) {
+__device__ __forceinline__ void prefetch_c_rows_inline(const double* C, long long ldc, int M, int N, int tm, int tn,
+                                                       int r0, int rstep) {
   const int cols = min(BN, N - tn * BN) & ~1;
   if (cols <= 0) return;
   for (int r = r0; r < BM; r += rstep) {
@@ -178,11 +181,19 @@ __device__ __noinline__ void prefetch_c_rows(const double* C, long long ldc, int
     if (row < M) ptx::prefetch_l2_bulk(C + (long long)row * ldc + (long long)tn * BN, (uint32_t)cols * 8u);
   }
 }
+__device__ __noinline__ void prefetch_c_rows(const double* C, long long ldc, int M, int N, int tm, int tn, int r0,
+                                             int rstep) {
+  prefetch_c_rows_inline(C, ldc, M, N, tm, tn, r0, rstep);
+}
 
 // B stage as eight 2-D boxes of 16 columns (used when N is not a multiple of 16).
-__device__ __noinline__ void tma_load_b_boxes(uint32_t sb, const CUtensorMap* map_b, int n0, int k0, uint32_t fb) {
+__device__ __forceinline__ void tma_load_b_boxes_inline(uint32_t sb, const CUtensorMap* map_b, int n0, int k0,
+                                                        uint32_t fb) {
 #pragma unroll
   for (int nb = 0; nb < BN / 16; ++nb) ptx::tma_load_2d(sb + nb * B_BOX_BYTES, map_b, n0 + nb * 16, k0, fb);
+}
+__device__ __noinline__ void tma_load_b_boxes(uint32_t sb, const CUtensorMap* map_b, int n0, int k0, uint32_t fb) {
+  tma_load_b_boxes_inline(sb, map_b, n0, k0, fb);
 }
 
 // Slow part of a bounded mbarrier wait: poll until the phase completes, the CTA aborts, or the
@@ -203,6 +214,24 @@ __device__ __noinline__ bool wait_slow(uint32_t bar, uint32_t parity, volatile i
   }
 }
 
+// Fully inlined bounded wait (no call in the caller's hot loop; used where registers are scarce).
+__device__ __forceinline__ bool wait_bounded_inline(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                                    const GemmParams& p) {
+  if (ptx::mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = ptx::globaltimer_ns();
+  for (uint32_t it = 1;; ++it) {
+    if (ptx::mbar_try_wait(bar, parity)) return true;
+    if ((it & 31u) == 0u) {
+      if (*abort_flag) return false;
+      if (ptx::globaltimer_ns() - t0 > p.wait_limit_ns) {
+        *abort_flag = 1;
+        atomicExch(p.status, STATUS_TIMEOUT);
+        return false;
+      }
+    }
+  }
+}
+
 // Bounded mbarrier wait. Returns false if the CTA is aborting (this or another thread timed out).
 // SUSPEND = true polls with try_wait (the thread may be suspended for a short, hardware-defined
 // time when the phase is not complete: right for the arithmetic waiting for data); SUSPEND = false
@@ -212,6 +241,163 @@ __device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, vola
                                              const GemmParams& p) {
   if (SUSPEND ? ptx::mbar_try_wait(bar, parity) : ptx::mbar_test_wait(bar, parity)) return true;
   return wait_slow(bar, parity, abort_flag, p.wait_limit_ns, p.status, SUSPEND);
+}
+
+// Position of a lane in the 2 x 4 grid of 64 x 32 warp tiles, and the byte offsets of its fragments
+// inside a stage for the two k8 halves h of a stage:
+//   A: lane reads k = 8h+2t, 8h+2t+1 of row 64wm + 16mt + {0,8} + rm  (mt adds 2048, +8 rows adds 1024)
+//   B: lane reads columns 32wn + 16np + 2g, +1 of k row 8h + 2t + b     (np adds one box)
+struct LaneMap {
+  int g, t, wm, wn, rm;
+  uint32_t a_off[2], b_off[2][2];
+};
+
+__device__ __forceinline__ LaneMap make_lane_map(int warp, int lane) {
+  LaneMap m;
+  m.g = lane >> 2;   // MMA group id (row of A / column of B fragment)
+  m.t = lane & 3;    // thread in group (k index of the fragments)
+  m.wm = warp >> 2;  // 0..1 : 64-row slab of the CTA tile
+  m.wn = warp & 3;   // 0..3 : 32-column slab
+  m.rm = rowmap(m.g);
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    m.a_off[h] = (64 * m.wm + m.rm) * 128 + (((4 * h + m.t) ^ m.rm) << 4);
+#pragma unroll
+    for (int b = 0; b < 2; ++b)
+      m.b_off[h][b] = A_STAGE_BYTES + (2 * m.wn) * B_BOX_BYTES + (8 * h + 2 * m.t + b) * 128 + ((m.g ^ (2 * m.t + b)) << 4);
+  }
+  return m;
+}
+
+// The arithmetic of one k-block (16 k values) on one stage: acc += A_tile * B_tile for this warp's
+// 64 x 32 tile. Returns a token that depends on every fragment register this lane loaded.
+__device__ __forceinline__ int compute_kblock(const uint8_t* st, const LaneMap& m, double (&acc)[4][4][4]) {
+  int token = 0;
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    double2 alo[4], ahi[4], bf[2][2];
+#pragma unroll
+    for (int mt = 0; mt < 4; ++mt) {
+      alo[mt] = *reinterpret_cast<const double2*>(st + m.a_off[h] + mt * 2048);
+      ahi[mt] = *reinterpret_cast<const double2*>(st + m.a_off[h] + mt * 2048 + 1024);
+    }
+#pragma unroll
+    for (int np = 0; np < 2; ++np)
+#pragma unroll
+      for (int b = 0; b < 2; ++b)
+        bf[np][b] = *reinterpret_cast<const double2*>(st + m.b_off[h][b] + np * B_BOX_BYTES);
+#pragma unroll
+    for (int mt = 0; mt < 4; ++mt)
+      token ^= __double2loint(alo[mt].x) ^ __double2hiint(alo[mt].y) ^ __double2loint(ahi[mt].x) ^ __double2hiint(ahi[mt].y);
+#pragma unroll
+    for (int np = 0; np < 2; ++np)
+      token ^= __double2loint(bf[np][0].x) ^ __double2hiint(bf[np][0].y) ^ __double2loint(bf[np][1].x) ^ __double2hiint(bf[np][1].y);
+    // Eight k values per block as two k4 steps (x: k = 8h + 2t, y: k = 8h + 2t + 1) of the
+    // m8n8k4 shape; rows g (alo) and g + 8 (ahi) are separate 8 x 8 tiles.
+#pragma unroll
+    for (int mt = 0; mt < 4; ++mt)
+#pragma unroll
+      for (int np = 0; np < 2; ++np) {
+        ptx::dmma_m8n8k4(acc[mt][2 * np + 0][0], acc[mt][2 * np + 0][1], alo[mt].x, bf[np][0].x);
+        ptx::dmma_m8n8k4(acc[mt][2 * np + 0][2], acc[mt][2 * np + 0][3], ahi[mt].x, bf[np][0].x);
+        ptx::dmma_m8n8k4(acc[mt][2 * np + 1][0], acc[mt][2 * np + 1][1], alo[mt].x, bf[np][0].y);
+        ptx::dmma_m8n8k4(acc[mt][2 * np + 1][2], acc[mt][2 * np + 1][3], ahi[mt].x, bf[np][0].y);
+        ptx::dmma_m8n8k4(acc[mt][2 * np + 0][0], acc[mt][2 * np + 0][1], alo[mt].y, bf[np][1].x);
+        ptx::dmma_m8n8k4(acc[mt][2 * np + 0][2], acc[mt][2 * np + 0][3], ahi[mt].y, bf[np][1].x);
+        ptx::dmma_m8n8k4(acc[mt][2 * np + 1][0], acc[mt][2 * np + 1][1], alo[mt].y, bf[np][1].y);
+        ptx::dmma_m8n8k4(acc[mt][2 * np + 1][2], acc[mt][2 * np + 1][3], ahi[mt].y, bf[np][1].y);
+      }
+  }
+  return token;
+}
+
+// Releases a stage after compute_kblock. The arrive must not take effect before all of this
+// warp's fragment loads have been served: otherwise the refill can overwrite rows that a load
+// still queued behind the arithmetic has yet to read (observed as sporadically wrong rows of the
+// last-loaded A fragments in the slowest warp, cured by delaying the arrive). Program order alone
+// does not guarantee it, so the arrive is made data-dependent on the loaded registers of all 32
+// lanes: a warp-wide reduction of the per-lane tokens, masked with a zero the compiler cannot
+// see, is added to the barrier address.
+__device__ __forceinline__ void release_stage(uint32_t empty_bar_s, int token, int lane, int zero) {
+  token = __reduce_xor_sync(0xffffffffu, token);
+  if (lane == 0) ptx::mbar_arrive(empty_bar_s + (uint32_t)(token & zero));
+}
+
+// Epilogue of one work item: adds the accumulators to the C tile (or stores them as a partial tile
+// in the workspace when the item covers only part of K).
+template <int MT_PER_BATCH>
+__device__ __forceinline__ void store_tile(const GemmParams& p, const Work& w, const LaneMap& m, double (&acc)[4][4][4]) {
+  const int tm = w.tm, tn = w.tn;
+  // This lane owns, for each mt, half (rows +0 / +8) and np, four consecutive
+  // columns n = 32wn + 16np + 4t + {0,1,2,3} = {nt=2np:c0, nt=2np+1:c0, nt=2np:c1, nt=2np+1:c1}
+  const int row_base = tm * BM + 64 * m.wm + m.rm;
+  const int col_base = tn * BN + 32 * m.wn + 4 * m.t;
+  if (w.slot >= 0) {
+    double* dst = p.partial + (long long)w.slot * (long long)(BM * BN);
+#pragma unroll
+    for (int mt = 0; mt < 4; ++mt)
+#pragma unroll
+      for (int half = 0; half < 2; ++half)
+#pragma unroll
+        for (int np = 0; np < 2; ++np) {
+          const int r = 64 * m.wm + m.rm + 16 * mt + 8 * half;
+          const int c = 32 * m.wn + 4 * m.t + 16 * np;
+          ptx::stg256(dst + r * BN + c, acc[mt][2 * np][2 * half], acc[mt][2 * np + 1][2 * half],
+                      acc[mt][2 * np][2 * half + 1], acc[mt][2 * np + 1][2 * half + 1]);
+        }
+  } else {
+    const bool interior = (tm * BM + BM <= p.M) && (tn * BN + BN <= p.N);
+    const bool vec32 = ((reinterpret_cast<uintptr_t>(p.C) & 31) == 0) && ((p.ldc & 3) == 0);
+    if (interior && vec32) {
+      // batches of 4 * MT_PER_BATCH outstanding 32-byte loads per thread, then the adds and stores
+#pragma unroll
+      for (int mp = 0; mp < 4 / MT_PER_BATCH; ++mp) {
+        double cin[MT_PER_BATCH][2][2][4];
+#pragma unroll
+        for (int mq = 0; mq < MT_PER_BATCH; ++mq)
+#pragma unroll
+          for (int half = 0; half < 2; ++half) {
+            const double* crow = p.C + (long long)(row_base + 16 * (MT_PER_BATCH * mp + mq) + 8 * half) * p.ldc + col_base;
+#pragma unroll
+            for (int np = 0; np < 2; ++np)
+              ptx::ldg256(crow + 16 * np, cin[mq][half][np][0], cin[mq][half][np][1], cin[mq][half][np][2],
+                          cin[mq][half][np][3]);
+          }
+#pragma unroll
+        for (int mq = 0; mq < MT_PER_BATCH; ++mq)
+#pragma unroll
+          for (int half = 0; half < 2; ++half) {
+            const int mt = MT_PER_BATCH * mp + mq;
+            double* crow = p.C + (long long)(row_base + 16 * mt + 8 * half) * p.ldc + col_base;
+#pragma unroll
+            for (int np = 0; np < 2; ++np)
+              ptx::stg256(crow + 16 * np, cin[mq][half][np][0] + acc[mt][2 * np][2 * half],
+                          cin[mq][half][np][1] + acc[mt][2 * np + 1][2 * half],
+                          cin[mq][half][np][2] + acc[mt][2 * np][2 * half + 1],
+                          cin[mq][half][np][3] + acc[mt][2 * np + 1][2 * half + 1]);
+          }
+      }
+    } else {
+#pragma unroll
+      for (int mt = 0; mt < 4; ++mt)
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+          const int row = row_base + 16 * mt + 8 * half;
+          if (row < p.M) {
+            double* crow = p.C + (long long)row * p.ldc;
+#pragma unroll
+            for (int np = 0; np < 2; ++np) {
+              const int col = col_base + 16 * np;
+              const double v[4] = {acc[mt][2 * np][2 * half], acc[mt][2 * np + 1][2 * half],
+                                   acc[mt][2 * np][2 * half + 1], acc[mt][2 * np + 1][2 * half + 1]};
+#pragma unroll
+              for (int e = 0; e < 4; ++e)
+                if (col + e < p.N) crow[col + e] += v[e];
+            }
+          }
+        }
+    }
+  }
 }
 
 template <bool USE_TMA>
@@ -355,23 +541,7 @@ dgemm_dmma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
 
   for (int i = 0; i < LOOKAHEAD && ok; ++i) ok = issue_next();
 
-  const int g = lane >> 2;   // MMA group id (row of A / column of B fragment)
-  const int t = lane & 3;    // thread in group (k index of the fragments)
-  const int wm = warp >> 2;  // 0..1 : 64-row slab of the CTA tile
-  const int wn = warp & 3;   // 0..3 : 32-column slab
-  const int rm = rowmap(g);
-
-  // Byte offsets of this lane's fragments inside a stage, for the two k8 halves h of a stage.
-  // A: lane reads k = 8h+2t, 8h+2t+1 of row 64wm + 16mt + {0,8} + rm  (mt adds 2048, +8 rows adds 1024)
-  // B: lane reads columns 32wn + 16np + 2g, +1 of k row 8h + 2t + b     (np adds one box)
-  uint32_t a_off[2], b_off[2][2];
-#pragma unroll
-  for (int h = 0; h < 2; ++h) {
-    a_off[h] = (64 * wm + rm) * 128 + (((4 * h + t) ^ rm) << 4);
-#pragma unroll
-    for (int b = 0; b < 2; ++b)
-      b_off[h][b] = A_STAGE_BYTES + (2 * wn) * B_BOX_BYTES + (8 * h + 2 * t + b) * 128 + ((g ^ (2 * t + b)) << 4);
-  }
+  const LaneMap lm = make_lane_map(warp, lane);
 
   double acc[4][4][4];  // [mt][nt = 2*np + j][c0..c3]
   uint32_t it = 0;      // k-blocks consumed so far
@@ -388,7 +558,6 @@ dgemm_dmma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     const int valid = item_words[5];
     __syncwarp();
     if (!valid) break;
-    const int tm = w.tm, tn = w.tn;
 #pragma unroll
     for (int mt = 0; mt < 4; ++mt)
 #pragma unroll
@@ -400,127 +569,14 @@ dgemm_dmma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
       const uint32_t s = it % STAGES;
       const uint32_t ph = (it / STAGES) & 1u;
       if (!wait_bounded(full_bar + 8 * s, ph, abort_flag, p)) { ok = false; break; }
-      const uint8_t* st = tiles + s * STAGE_BYTES;
-      int token = 0;  // depends on every fragment this lane loads from the stage
-#pragma unroll
-      for (int h = 0; h < 2; ++h) {
-        double2 alo[4], ahi[4], bf[2][2];
-#pragma unroll
-        for (int mt = 0; mt < 4; ++mt) {
-          alo[mt] = *reinterpret_cast<const double2*>(st + a_off[h] + mt * 2048);
-          ahi[mt] = *reinterpret_cast<const double2*>(st + a_off[h] + mt * 2048 + 1024);
-        }
-#pragma unroll
-        for (int np = 0; np < 2; ++np)
-#pragma unroll
-          for (int b = 0; b < 2; ++b)
-            bf[np][b] = *reinterpret_cast<const double2*>(st + b_off[h][b] + np * B_BOX_BYTES);
-#pragma unroll
-        for (int mt = 0; mt < 4; ++mt)
-          token ^= __double2loint(alo[mt].x) ^ __double2hiint(alo[mt].y) ^ __double2loint(ahi[mt].x) ^ __double2hiint(ahi[mt].y);
-#pragma unroll
-        for (int np = 0; np < 2; ++np)
-          token ^= __double2loint(bf[np][0].x) ^ __double2hiint(bf[np][0].y) ^ __double2loint(bf[np][1].x) ^ __double2hiint(bf[np][1].y);
-        // Eight k values per block as two k4 steps (x: k = 8h + 2t, y: k = 8h + 2t + 1) of the
-        // m8n8k4 shape; rows g (alo) and g + 8 (ahi) are separate 8 x 8 tiles.
-#pragma unroll
-        for (int mt = 0; mt < 4; ++mt)
-#pragma unroll
-          for (int np = 0; np < 2; ++np) {
-            ptx::dmma_m8n8k4(acc[mt][2 * np + 0][0], acc[mt][2 * np + 0][1], alo[mt].x, bf[np][0].x);
-            ptx::dmma_m8n8k4(acc[mt][2 * np + 0][2], acc[mt][2 * np + 0][3], ahi[mt].x, bf[np][0].x);
-            ptx::dmma_m8n8k4(acc[mt][2 * np + 1][0], acc[mt][2 * np + 1][1], alo[mt].x, bf[np][0].y);
-            ptx::dmma_m8n8k4(acc[mt][2 * np + 1][2], acc[mt][2 * np + 1][3], ahi[mt].x, bf[np][0].y);
-            ptx::dmma_m8n8k4(acc[mt][2 * np + 0][0], acc[mt][2 * np + 0][1], alo[mt].y, bf[np][1].x);
-            ptx::dmma_m8n8k4(acc[mt][2 * np + 0][2], acc[mt][2 * np + 0][3], ahi[mt].y, bf[np][1].x);
-            ptx::dmma_m8n8k4(acc[mt][2 * np + 1][0], acc[mt][2 * np + 1][1], alo[mt].y, bf[np][1].y);
-            ptx::dmma_m8n8k4(acc[mt][2 * np + 1][2], acc[mt][2 * np + 1][3], ahi[mt].y, bf[np][1].y);
-          }
-      }
-      // Release the stage. The arrive must not take effect before all of this warp's fragment
-      // loads have been served: otherwise the refill can overwrite rows that a load still queued
-      // behind the arithmetic has yet to read (observed as sporadically wrong rows of the
-      // last-loaded A fragments in the slowest warp, cured by delaying the arrive). Program order
-      // alone does not guarantee it, so the arrive is made data-dependent on the loaded registers
-      // of all 32 lanes: a warp-wide reduction of the per-lane tokens, masked with a zero the
-      // compiler cannot see, is added to the barrier address.
-      token = __reduce_xor_sync(0xffffffffu, token);
-      if (lane == 0) ptx::mbar_arrive(empty_bar + 8 * s + (uint32_t)(token & p.zero));
+      const int token = compute_kblock(tiles + s * STAGE_BYTES, lm, acc);
+      release_stage(empty_bar + 8 * s, token, lane, p.zero);
       // keep the load stream LOOKAHEAD k-blocks ahead: refill the stage released two k-blocks ago
       if (!issue_next()) { ok = false; break; }
     }
     if (!ok) break;
 
-    // ---- epilogue: this lane owns, for each mt, half (rows +0 / +8) and np, four consecutive
-    // columns n = 32wn + 16np + 4t + {0,1,2,3} = {nt=2np:c0, nt=2np+1:c0, nt=2np:c1, nt=2np+1:c1}
-    const int row_base = tm * BM + 64 * wm + rm;
-    const int col_base = tn * BN + 32 * wn + 4 * t;
-    if (w.slot >= 0) {
-      double* dst = p.partial + (long long)w.slot * (long long)(BM * BN);
-#pragma unroll
-      for (int mt = 0; mt < 4; ++mt)
-#pragma unroll
-        for (int half = 0; half < 2; ++half)
-#pragma unroll
-          for (int np = 0; np < 2; ++np) {
-            const int r = 64 * wm + rm + 16 * mt + 8 * half;
-            const int c = 32 * wn + 4 * t + 16 * np;
-            ptx::stg256(dst + r * BN + c, acc[mt][2 * np][2 * half], acc[mt][2 * np + 1][2 * half],
-                        acc[mt][2 * np][2 * half + 1], acc[mt][2 * np + 1][2 * half + 1]);
-          }
-    } else {
-      const bool interior = (tm * BM + BM <= p.M) && (tn * BN + BN <= p.N);
-      const bool vec32 = ((reinterpret_cast<uintptr_t>(p.C) & 31) == 0) && ((p.ldc & 3) == 0);
-      if (interior && vec32) {
-        // two batches of 8 outstanding 32-byte loads per thread, then the adds and stores
-#pragma unroll
-        for (int mp = 0; mp < 2; ++mp) {
-          double cin[2][2][2][4];
-#pragma unroll
-          for (int mq = 0; mq < 2; ++mq)
-#pragma unroll
-            for (int half = 0; half < 2; ++half) {
-              const double* crow = p.C + (long long)(row_base + 16 * (2 * mp + mq) + 8 * half) * p.ldc + col_base;
-#pragma unroll
-              for (int np = 0; np < 2; ++np)
-                ptx::ldg256(crow + 16 * np, cin[mq][half][np][0], cin[mq][half][np][1], cin[mq][half][np][2],
-                            cin[mq][half][np][3]);
-            }
-#pragma unroll
-          for (int mq = 0; mq < 2; ++mq)
-#pragma unroll
-            for (int half = 0; half < 2; ++half) {
-              const int mt = 2 * mp + mq;
-              double* crow = p.C + (long long)(row_base + 16 * mt + 8 * half) * p.ldc + col_base;
-#pragma unroll
-              for (int np = 0; np < 2; ++np)
-                ptx::stg256(crow + 16 * np, cin[mq][half][np][0] + acc[mt][2 * np][2 * half],
-                            cin[mq][half][np][1] + acc[mt][2 * np + 1][2 * half],
-                            cin[mq][half][np][2] + acc[mt][2 * np][2 * half + 1],
-                            cin[mq][half][np][3] + acc[mt][2 * np + 1][2 * half + 1]);
-            }
-        }
-      } else {
-#pragma unroll
-        for (int mt = 0; mt < 4; ++mt)
-#pragma unroll
-          for (int half = 0; half < 2; ++half) {
-            const int row = row_base + 16 * mt + 8 * half;
-            if (row < p.M) {
-              double* crow = p.C + (long long)row * p.ldc;
-#pragma unroll
-              for (int np = 0; np < 2; ++np) {
-                const int col = col_base + 16 * np;
-                const double v[4] = {acc[mt][2 * np][2 * half], acc[mt][2 * np + 1][2 * half],
-                                     acc[mt][2 * np][2 * half + 1], acc[mt][2 * np + 1][2 * half + 1]};
-#pragma unroll
-                for (int e = 0; e < 4; ++e)
-                  if (col + e < p.N) crow[col + e] += v[e];
-              }
-            }
-          }
-      }
-    }
+    store_tile<2>(p, w, lm, acc);
   }
 
   // Leaving. After a normal run every copy that was issued has been consumed. After an abort,
@@ -537,6 +593,170 @@ dgemm_dmma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     }
   }
   __syncthreads();
+}
+
+// ---------------------------------------------------------------------------------------------
+// Warp-specialised variant: 8 consumer warps as above plus one producer warpgroup (384 threads).
+// The producers hand most of their registers to the consumers (setmaxnreg: 232 / 40; the pool is
+// what the CTA owns at launch, 384 x 168, so 256 x 232 + 128 x 40 must not exceed it). The
+// producer runs up to STAGES k-blocks ahead. TMA staging: lane 0 of the first producer warp issues
+// the copies; generic staging: the four producer warps copy 32 rows of A and 32 columns of B each.
+constexpr int WS_PRODUCER_WARPS = 4;
+constexpr int WS_THREADS = (WARPS + WS_PRODUCER_WARPS) * 32;
+constexpr int WS_CONSUMER_REGS = 232;
+constexpr int WS_PRODUCER_REGS = 40;
+
+template <bool USE_TMA>
+__global__ void __launch_bounds__(WS_THREADS, 1)
+dgemm_dmma_ws_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                     const __grid_constant__ GemmParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = ptx::smem_u32(smem_raw);
+  const uint32_t pad = (SMEM_ALIGN - (raw & (SMEM_ALIGN - 1))) & (SMEM_ALIGN - 1);
+  uint8_t* tiles = smem_raw + pad;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(tiles + STAGES * STAGE_BYTES);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 2 * STAGES);
+  volatile int* work_words = abort_flag + 8;  // 8 words per warp (12 warps)
+  const uint32_t tiles_u32 = raw + pad;
+  const uint32_t full_bar = tiles_u32 + STAGES * STAGE_BYTES;
+  const uint32_t empty_bar = full_bar + 8 * STAGES;
+
+  const int tid = threadIdx.x;
+  const int warp = tid >> 5;
+  const int lane = tid & 31;
+
+  if (tid == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      ptx::mbar_init(full_bar + 8 * s, USE_TMA ? 1 : WS_PRODUCER_WARPS * 32);
+      ptx::mbar_init(empty_bar + 8 * s, WARPS);
+    }
+    *abort_flag = 0;
+    ptx::fence_barrier_init();
+  }
+  __syncthreads();
+
+  const int cta = blockIdx.x, nctas = gridDim.x;
+  volatile int* item_words = work_words + 8 * warp;
+  Work w;
+  uint32_t it = 0;  // running k-block counter, the same sequence in producers and consumers
+  bool ok = true;
+
+  if (warp >= WARPS) {
+    // ------------------------------------------------------------------ producer warpgroup
+    ptx::setmaxnreg_dec<WS_PRODUCER_REGS>();
+    const int pw = warp - WARPS;
+    const bool active = USE_TMA ? (pw == 0) : true;
+    if (USE_TMA && pw == 0 && lane == 0) {
+      ptx::prefetch_tensormap(&map_a);
+      ptx::prefetch_tensormap(&map_b);
+    }
+    for (int idx = 0; active && ok; ++idx) {
+      fetch_work_inline(p, cta, nctas, idx, item_words);
+      __syncwarp();
+      w.tm = item_words[0];
+      w.tn = item_words[1];
+      w.kb0 = item_words[2];
+      w.kb1 = item_words[3];
+      w.slot = item_words[4];
+      const int valid = item_words[5];
+      __syncwarp();
+      if (!valid) break;
+      const int kb_pf = (w.slot < 0 && p.c_prefetch) ? max(w.kb0, w.kb1 - C_PREFETCH_KBLOCKS) : -1;
+      for (int kb = w.kb0; kb < w.kb1; ++kb, ++it) {
+        const uint32_t s = it % STAGES;
+        const uint32_t ph = (it / STAGES) & 1u;
+        const uint32_t sa = tiles_u32 + s * STAGE_BYTES;
+        const uint32_t sb = sa + A_STAGE_BYTES;
+        const uint32_t fb = full_bar + 8 * s;
+        if (USE_TMA) {
+          int good = 1;
+          if (lane == 0) {
+            if (wait_bounded_inline(empty_bar + 8 * s, ph ^ 1u, abort_flag, p)) {
+              ptx::mbar_arrive_expect_tx(fb, STAGE_BYTES);
+              ptx::tma_load_2d(sa, &map_a, kb * BK, w.tm * BM, fb);
+              if (p.b_blocked_map) {
+                ptx::tma_load_3d(sb, &map_b, 0, kb * BK, w.tn * (BN / 16), fb);
+              } else {
+                tma_load_b_boxes_inline(sb, &map_b, w.tn * BN, kb * BK, fb);
+              }
+            } else {
+              good = 0;
+            }
+          }
+          if (!__all_sync(0xffffffffu, good)) { ok = false; break; }
+          if (kb == kb_pf) prefetch_c_rows_inline(p.C, p.ldc, p.M, p.N, w.tm, w.tn, lane, 32);
+        } else {
+          if (!wait_bounded_inline(empty_bar + 8 * s, ph ^ 1u, abort_flag, p)) { ok = false; break; }
+          const int m0 = w.tm * BM, n0 = w.tn * BN, k0 = kb * BK;
+          {
+            const int a_r = lane >> 4, a_k = lane & 15;
+            const int k = k0 + a_k;
+            const bool kin = k < p.K;
+            const int row0 = 32 * pw + a_r;
+            const double* src = p.A + (long long)(m0 + row0) * p.lda + k;
+            const uint32_t dst_base = sa + ((a_k & 1) << 3);
+#pragma unroll 4
+            for (int r = 0; r < 32; r += 2) {
+              const int row = row0 + r;
+              const bool in = kin && (m0 + row < p.M);
+              const uint32_t dst = dst_base + row * 128 + (((a_k >> 1) ^ (row & 7)) << 4);
+              ptx::cp_async_8(dst, in ? (const void*)(src + (long long)r * p.lda) : (const void*)p.A, in ? 8u : 0u);
+            }
+          }
+          {
+            const int nn = 32 * pw + lane;
+            const bool nin = n0 + nn < p.N;
+            const double* src = p.B + (long long)k0 * p.ldb + (n0 + nn);
+            const uint32_t dst_base = sb + (nn >> 4) * B_BOX_BYTES + ((nn & 1) << 3);
+            const int chunk = (nn & 15) >> 1;
+#pragma unroll 4
+            for (int kk = 0; kk < BK; ++kk) {
+              const bool in = nin && (k0 + kk < p.K);
+              const uint32_t dst = dst_base + kk * 128 + ((chunk ^ (kk & 7)) << 4);
+              ptx::cp_async_8(dst, in ? (const void*)(src + (long long)kk * p.ldb) : (const void*)p.B, in ? 8u : 0u);
+            }
+          }
+          ptx::cp_async_mbar_arrive_noinc(fb);
+          if (kb == kb_pf) prefetch_c_rows_inline(p.C, p.ldc, p.M, p.N, w.tm, w.tn, 32 * pw + lane, BM);
+        }
+      }
+    }
+    if (!USE_TMA) ptx::cp_async_wait_all();
+    if (USE_TMA && !ok && pw == 0 && lane == 0) {
+      // aborting: let every copy this thread armed land before the CTA's memory is released
+      const uint32_t n_inflight = it < (uint32_t)STAGES ? it : (uint32_t)STAGES;
+      for (uint32_t q = it - n_inflight; q < it; ++q) {
+        const uint32_t s = q % STAGES, ph = (q / STAGES) & 1u;
+        const unsigned long long t0 = ptx::globaltimer_ns();
+        while (!ptx::mbar_try_wait(full_bar + 8 * s, ph)) {
+          if (ptx::globaltimer_ns() - t0 > p.wait_limit_ns) break;
+        }
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ consumer warps
+    ptx::setmaxnreg_inc<WS_CONSUMER_REGS>();
+    const LaneMap lm = make_lane_map(warp, lane);
+    double acc[4][4][4];
+    for (int idx = 0; ok && get_work(p, cta, nctas, idx, w); ++idx) {
+#pragma unroll
+      for (int mt = 0; mt < 4; ++mt)
+#pragma unroll
+        for (int nt = 0; nt < 4; ++nt)
+#pragma unroll
+          for (int c = 0; c < 4; ++c) acc[mt][nt][c] = 0.0;
+      for (int kb = w.kb0; kb < w.kb1; ++kb, ++it) {
+        const uint32_t s = it % STAGES;
+        const uint32_t ph = (it / STAGES) & 1u;
+        if (!wait_bounded_inline(full_bar + 8 * s, ph, abort_flag, p)) { ok = false; break; }
+        const int token = compute_kblock(tiles + s * STAGE_BYTES, lm, acc);
+        release_stage(empty_bar + 8 * s, token, lane, p.zero);
+      }
+      if (!ok) break;
+      store_tile<1>(p, w, lm, acc);
+    }
+  }
+  ptx::named_barrier_sync(1, WS_THREADS);  // all warps leave together
 }
 
 // Adds `count` partial tiles (workspace slots slot[0..count)) to the C tile (tm, tn) in that order:

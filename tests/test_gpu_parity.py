@@ -81,7 +81,7 @@ def _check_full(oracle, prob: wl.Problem, out: torch.Tensor):
 
 @pytest.mark.parametrize("integer", [False, True])
 @pytest.mark.parametrize("variant", [dg.DGEMM_VARIANT_AUTO, dg.DGEMM_VARIANT_TMA, dg.DGEMM_VARIANT_GENERIC,
-                                     dg.DGEMM_VARIANT_NAIVE])
+                                     dg.DGEMM_VARIANT_NAIVE, dg.DGEMM_VARIANT_TMA_WS, dg.DGEMM_VARIANT_GENERIC_WS])
 def test_config1(oracle, integer, variant):
     prob = wl.config1(integer)
     _check_full(oracle, prob, run_gpu(prob, variant))
@@ -95,7 +95,8 @@ SMALL_SHAPES = [(1, 1, 1), (1, 7, 3), (5, 1, 2), (3, 3, 17), (17, 13, 11), (8, 8
 
 
 @pytest.mark.parametrize("shape", SMALL_SHAPES)
-@pytest.mark.parametrize("variant", [dg.DGEMM_VARIANT_TMA, dg.DGEMM_VARIANT_GENERIC])
+@pytest.mark.parametrize("variant", [dg.DGEMM_VARIANT_TMA, dg.DGEMM_VARIANT_GENERIC, dg.DGEMM_VARIANT_TMA_WS,
+                                     dg.DGEMM_VARIANT_GENERIC_WS])
 def test_small_shapes_integer_exact(oracle, shape, variant):
     M, N, K = shape
     # even leading dimensions so that both staging variants can run the same problem
@@ -121,7 +122,8 @@ def test_unaligned_base_pointers(oracle, offset):
 # ---- split-K (partial tiles through the workspace, deterministic reduction) -------------------------
 
 @pytest.mark.parametrize("split", [2, 3, 7, 64])
-@pytest.mark.parametrize("variant", [dg.DGEMM_VARIANT_TMA, dg.DGEMM_VARIANT_GENERIC])
+@pytest.mark.parametrize("variant", [dg.DGEMM_VARIANT_TMA, dg.DGEMM_VARIANT_GENERIC, dg.DGEMM_VARIANT_TMA_WS,
+                                     dg.DGEMM_VARIANT_GENERIC_WS])
 def test_split_k(oracle, split, variant):
     prob = wl.make_problem(200, 150, 1000, seed=11, lda=1000, ldb=150 + 2, ldc=151, integer=True)
     _check_full(oracle, prob, run_gpu(prob, variant, split_k=split))

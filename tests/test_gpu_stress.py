@@ -26,7 +26,8 @@ def rank_k_case(oracle):
 
 
 @pytest.mark.parametrize("flags", [3, 1, 2, 0])
-@pytest.mark.parametrize("variant", [dg.DGEMM_VARIANT_TMA, dg.DGEMM_VARIANT_GENERIC])
+@pytest.mark.parametrize("variant", [dg.DGEMM_VARIANT_TMA, dg.DGEMM_VARIANT_GENERIC, dg.DGEMM_VARIANT_TMA_WS,
+                                     dg.DGEMM_VARIANT_GENERIC_WS])
 def test_rank_k_repeated_runs_bit_exact(rank_k_case, flags, variant):
     prob, want = rank_k_case
     A, B, C0 = prob.A_buf.cuda(), prob.B_buf.cuda(), prob.C_buf.cuda()
@@ -39,7 +40,7 @@ def test_rank_k_repeated_runs_bit_exact(rank_k_case, flags, variant):
     dg.dgemm_set_test_flags(flags)
     dg.dgemm_set_variant(variant)
     try:
-        reps = 12 if variant == dg.DGEMM_VARIANT_TMA else 4
+        reps = 12 if variant in (dg.DGEMM_VARIANT_TMA, dg.DGEMM_VARIANT_TMA_WS) else 4
         for rep in range(reps):
             C = C0.clone()
             dg.dgemm_f64(A, B, C)

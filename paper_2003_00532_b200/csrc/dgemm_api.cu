@@ -24,7 +24,7 @@ constexpr size_t kWorkspaceBytes = 320ull * BM * BN * sizeof(double);  // 40 MiB
 constexpr unsigned long long kWaitLimitNs = 4000000000ull;            // 4 s per device-side wait
 constexpr int kAutoTma = DGEMM_VARIANT_TMA;          // what DGEMM_VARIANT_AUTO picks for aligned operands
 constexpr int kAutoGeneric = DGEMM_VARIANT_GENERIC;  // ... and for unaligned ones
-constexpr int kTailMinSpan = 2;          // stream-K tail: at least this many k-blocks per CTA
+constexpr int kTailMinSpan = 1;          // stream-K tail: at least this many k-blocks per CTA
 constexpr double kTailMinSavedKblocks = 5.0;  // use the stream-K tail only if it saves this many k-block times
 
 __device__ int g_status_word;  // one per device that loads the library
@@ -251,12 +251,12 @@ int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, c
   g_launches.fetch_add(1);
   if (cudaGetLastError() != cudaSuccess) return DGEMM_ERR_CUDA;
   if (p.split_k > 1) {
-    dgemm_splitk_reduce_kernel<<<tiles, 256, 0, stream>>>(p);
+    dgemm_splitk_reduce_kernel<<<dim3(tiles, REDUCE_CHUNKS), REDUCE_THREADS, 0, stream>>>(p);
     g_launches.fetch_add(1);
     if (cudaGetLastError() != cudaSuccess) return DGEMM_ERR_CUDA;
   }
   if (p.tail_tiles > 0 && p.tail_ipc < kblocks) {
-    dgemm_tail_reduce_kernel<<<p.tail_tiles, 256, 0, stream>>>(p);
+    dgemm_tail_reduce_kernel<<<dim3(p.tail_tiles, REDUCE_CHUNKS), REDUCE_THREADS, 0, stream>>>(p);
     g_launches.fetch_add(1);
     if (cudaGetLastError() != cudaSuccess) return DGEMM_ERR_CUDA;
   }
@@ -354,7 +354,7 @@ int launch_gemm_static_ws(int64_t M, int64_t N, int64_t K, const double* A, int6
   g_launches.fetch_add(1);
   if (cudaGetLastError() != cudaSuccess) return DGEMM_ERR_CUDA;
   if (p.split_k > 1) {
-    dgemm_splitk_reduce_kernel<<<(int)tiles, 256, 0, stream>>>(p);
+    dgemm_splitk_reduce_kernel<<<dim3((int)tiles, REDUCE_CHUNKS), REDUCE_THREADS, 0, stream>>>(p);
     g_launches.fetch_add(1);
     if (cudaGetLastError() != cudaSuccess) return DGEMM_ERR_CUDA;
   }

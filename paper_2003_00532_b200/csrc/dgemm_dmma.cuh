@@ -760,10 +760,16 @@ dgemm_dmma_ws_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
 }
 
 // Adds `count` partial tiles (workspace slots slot[0..count)) to the C tile (tm, tn) in that order:
-// C[i][j] += ((p_0 + p_1) + p_2) + ...  Deterministic; one CTA per tile.
+// C[i][j] += ((p_0 + p_1) + p_2) + ...  Deterministic. A tile is reduced by REDUCE_CHUNKS CTAs
+// (blockIdx.y), each taking BM / REDUCE_CHUNKS consecutive rows.
+constexpr int REDUCE_CHUNKS = 16;
+constexpr int REDUCE_THREADS = 256;
+
 template <typename SlotFn>
 __device__ __forceinline__ void reduce_tile(const GemmParams& p, int tm, int tn, int count, SlotFn slot_of) {
-  for (int e = 2 * threadIdx.x; e < BM * BN; e += 2 * blockDim.x) {
+  constexpr int CHUNK_ELEMS = BM * BN / REDUCE_CHUNKS;
+  const int e0 = blockIdx.y * CHUNK_ELEMS;
+  for (int e = e0 + 2 * threadIdx.x; e < e0 + CHUNK_ELEMS; e += 2 * REDUCE_THREADS) {
     const int r = e / BN, c = e - r * BN;
     const int row = tm * BM + r, col = tn * BN + c;
     if (row < p.M && col < p.N) {

@@ -34,7 +34,7 @@ FMA_PER_CLK_SM = 64  # FP64 DMMA issue rate measured by dgemm_fp64_peak_probe (6
 
 # DRAM traffic of one 8192^3 launch of the dominant kernel (dram__bytes_read.sum +
 # dram__bytes_write.sum of one ncu capture, see profiles/); None until a capture exists for a size.
-NCU_DRAM_BYTES_PER_LAUNCH = {}
+NCU_DRAM_BYTES_PER_LAUNCH = {8192: 7832529920 + 538832384, 4096: 1106763000 + 137738752}
 
 
 def _load_measured_peaks():
@@ -115,6 +115,53 @@ def oracle_slab_rate(A, B, C, rows: int, threads: int = 0):
     dt = time.perf_counter() - t0
     flop = 2.0 * rows * B.shape[0] * B.shape[1]
     return flop / dt / 1e12, dt, (threads if threads > 0 else oracle.max_threads())
+
+
+def time_shape(dg, torch, M, N, K, lda=None, ldb=None, ldc=None, min_ms=40.0):
+    """Mean CUDA-event time (ms) of back-to-back dgemm_f64 calls on one synthetic problem."""
+    lda, ldb, ldc = lda or K, ldb or N, ldc or N
+    A = torch.rand(M, lda, dtype=torch.float64, device="cuda") * 2 - 1
+    B = torch.rand(K, ldb, dtype=torch.float64, device="cuda") * 2 - 1
+    C = torch.rand(M, ldc, dtype=torch.float64, device="cuda") * 2 - 1
+    pa, pb, pc = A.data_ptr(), B.data_ptr(), C.data_ptr()
+    call = dg.load_library().dgemm_f64
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for _ in range(3):
+        call(M, N, K, pa, lda, pb, ldb, pc, ldc, None)
+    e0.record()
+    call(M, N, K, pa, lda, pb, ldb, pc, ldc, None)
+    e1.record()
+    torch.cuda.synchronize()
+    reps = int(max(3, min(500, min_ms / max(e0.elapsed_time(e1), 1e-3))))
+    best = float("inf")
+    for _ in range(3):
+        e0.record()
+        for _ in range(reps):
+            call(M, N, K, pa, lda, pb, ldb, pc, ldc, None)
+        e1.record()
+        torch.cuda.synchronize()
+        best = min(best, e0.elapsed_time(e1) / reps)
+    return best
+
+
+def other_shapes(dg, torch, peak_tflops, hbm_gbs):
+    """The square-size sweep (the metric's 'TFLOPS vs M=N=K' curve) and the ragged / rank-k shapes,
+    each with its fraction of the FP64 peak and, for the low-intensity shapes, of the HBM roof."""
+    sweep = []
+    for n in range(128, 4096 + 1, 128):
+        ms = time_shape(dg, torch, n, n, n)
+        tf = 2.0 * n ** 3 / ms / 1e9
+        sweep.append({"n": n, "us": round(ms * 1e3, 1), "tflops": round(tf, 2), "frac_peak": round(tf / peak_tflops, 3)})
+    shapes = []
+    for (M, N, K, pad) in [(1000, 1537, 777, True), (2088, 2088, 2088, True), (4097, 31, 4099, True),
+                           (2088, 2048, 2048, False), (16384, 16384, 64, False), (16384, 16384, 256, False)]:
+        ld = (K + 3, N + 5, N + 7) if pad else (K, N, N)
+        ms = time_shape(dg, torch, M, N, K, *ld)
+        tf = 2.0 * M * N * K / ms / 1e9
+        gbs = 8.0 * (M * K + K * N + 2 * M * N) / ms / 1e6
+        shapes.append({"M": M, "N": N, "K": K, "ld": list(ld), "us": round(ms * 1e3, 1), "tflops": round(tf, 2),
+                       "frac_peak": round(tf / peak_tflops, 3), "hbm_gbs": round(gbs), "frac_hbm": round(gbs / hbm_gbs, 3)})
+    return sweep, shapes
 
 
 def run_reference(args):
@@ -237,7 +284,7 @@ def run_ours(args):
     roofline = {
         "bound": "tensor", "achieved": achieved, "peak": peak_tflops, "unit": "TFLOP/s",
         "frac": achieved / peak_tflops, "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get(n),
-        "kernel": "dgemm_dmma_kernel<TMA>",
+        "kernel": "dgemm_dmma_kernel<true> (TMA staging)",
         "peak_source": (f"FP64 DMMA issue rate {FMA_PER_CLK_SM} FMA/clk/SM (measured by the register-only probe) x "
                         f"{SM_COUNT_B200} SMs x 2 x sm_max_mhz {sm_max_mhz:.0f} "
                         f"({'MEASURED_PEAKS.json' if peaks else 'fallback 1965'}); MEASURED_PEAKS has no FP64 entry"),
@@ -271,6 +318,8 @@ def run_ours(args):
         "gpu_launches": int(launches),
         "clocks": clocks,
     }
+    if not args.no_sweep:
+        line["sweep"], line["other_shapes"] = other_shapes(dg, torch, peak_tflops, hbm_gbs)
     print(json.dumps(line), flush=True)
     if distributed:
         dist.destroy_process_group()
@@ -287,6 +336,7 @@ def main():
     ap.add_argument("--ref-rows", type=int, default=128, help="rows of C per step of the reference arm")
     ap.add_argument("--cpu-rows", type=int, default=3072, help="rows of C in the cpu_baseline sample")
     ap.add_argument("--e2e-steps", type=int, default=5)
+    ap.add_argument("--no-sweep", action="store_true", help="skip the size sweep and the ragged / rank-k shapes")
     args = ap.parse_args()
     if args.steps < 1:
         ap.error("--steps must be >= 1")

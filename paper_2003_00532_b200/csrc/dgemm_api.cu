@@ -20,7 +20,7 @@ namespace {
 using namespace dgemm;
 
 constexpr int kMaxDevices = 64;
-constexpr size_t kWorkspaceBytes = 320ull * BM * BN * sizeof(double);  // 40 MiB: up to 320 partial tiles
+constexpr size_t kWorkspaceBytes = 640ull * BM * BN * sizeof(double);  // 80 MiB: up to 640 partial-tile slots
 constexpr unsigned long long kWaitLimitNs = 4000000000ull;            // 4 s per device-side wait
 constexpr int kAutoTma = DGEMM_VARIANT_TMA;          // what DGEMM_VARIANT_AUTO picks for aligned operands
 constexpr int kAutoGeneric = DGEMM_VARIANT_GENERIC;  // ... and for unaligned ones
@@ -32,6 +32,7 @@ __device__ int g_status_word;  // one per device that loads the library
 struct DeviceState {
   bool ready = false;
   int sm_count = 0;
+  bool two_ctas_ok = false;    // the 64-row kernels fit two CTAs per SM on this device
   int* status = nullptr;       // device address of g_status_word
   double* workspace = nullptr; // split-K partial tiles, allocated on first need
 };
@@ -67,11 +68,22 @@ int device_state(DeviceState** out) {
     if (major != 10) return DGEMM_ERR_DEVICE;
     if (cudaGetSymbolAddress(reinterpret_cast<void**>(&st.status), g_status_word) != cudaSuccess) return DGEMM_ERR_CUDA;
     if (cudaMemset(st.status, 0, sizeof(int)) != cudaSuccess) return DGEMM_ERR_CUDA;
-    if (cudaFuncSetAttribute(dgemm_dmma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess ||
-        cudaFuncSetAttribute(dgemm_dmma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess ||
-        cudaFuncSetAttribute(dgemm_dmma_ws_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess ||
-        cudaFuncSetAttribute(dgemm_dmma_ws_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
+    const bool attr_ok =
+        cudaFuncSetAttribute(dgemm_dmma_kernel<true, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, TileCfg<128>::SMEM_BYTES_) == cudaSuccess &&
+        cudaFuncSetAttribute(dgemm_dmma_kernel<false, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, TileCfg<128>::SMEM_BYTES_) == cudaSuccess &&
+        cudaFuncSetAttribute(dgemm_dmma_kernel<true, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, TileCfg<64>::SMEM_BYTES_) == cudaSuccess &&
+        cudaFuncSetAttribute(dgemm_dmma_kernel<false, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, TileCfg<64>::SMEM_BYTES_) == cudaSuccess &&
+        cudaFuncSetAttribute(dgemm_dmma_kernel<true, 64>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared) == cudaSuccess &&
+        cudaFuncSetAttribute(dgemm_dmma_kernel<false, 64>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared) == cudaSuccess &&
+        cudaFuncSetAttribute(dgemm_dmma_ws_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) == cudaSuccess &&
+        cudaFuncSetAttribute(dgemm_dmma_ws_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) == cudaSuccess;
+    if (!attr_ok) return DGEMM_ERR_CUDA;
+    // the 64-row kernel is meant to run two CTAs per SM; use it only where the device really fits two
+    int occ_tma = 0, occ_gen = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ_tma, dgemm_dmma_kernel<true, 64>, TileCfg<64>::THREADS_, TileCfg<64>::SMEM_BYTES_) != cudaSuccess ||
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ_gen, dgemm_dmma_kernel<false, 64>, TileCfg<64>::THREADS_, TileCfg<64>::SMEM_BYTES_) != cudaSuccess)
       return DGEMM_ERR_CUDA;
+    st.two_ctas_ok = (occ_tma >= 2 && occ_gen >= 2);
     if (!g_encode) {
       void* fn = nullptr;
       cudaDriverEntryPointQueryResult qres;
@@ -164,24 +176,32 @@ int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, c
     return cudaGetLastError() == cudaSuccess ? DGEMM_OK : DGEMM_ERR_CUDA;
   }
 
+  const int dbg_flags = g_test_flags.load();
+  const bool ws_variant = variant == DGEMM_VARIANT_TMA_WS || variant == DGEMM_VARIANT_GENERIC_WS;
+  // tile height: 64 rows with two CTAs per SM (default), 128 rows with one (warp-specialised variants, test flag)
+  // (generic staging on a problem of many waves is a little faster with the tall tile: half the B copies per thread)
+  const int64_t tiles128 = ((M + 127) / 128) * ((N + BN - 1) / BN);
+  const bool generic_large = !wants_tma && tiles128 >= 4 * (int64_t)st->sm_count;
+  const int bm = (ws_variant || generic_large || (dbg_flags & DGEMM_TEST_TALL_TILES) || !st->two_ctas_ok) ? 128 : 64;
+
   GemmParams p;
   memset(&p, 0, sizeof(p));
   p.M = (int)M; p.N = (int)N; p.K = (int)K;
-  p.tiles_m = (int)((M + BM - 1) / BM);
+  p.bm = bm;
+  p.tiles_m = (int)((M + bm - 1) / bm);
   p.tiles_n = (int)((N + BN - 1) / BN);
   p.A = A; p.B = B; p.C = C;
   p.lda = lda; p.ldb = ldb; p.ldc = ldc;
   p.wait_limit_ns = kWaitLimitNs;
   p.status = st->status;
-  p.group_m = 8;
+  p.group_m = bm == 128 ? 8 : 16;  // 8 x 128 = 16 x 64 rows per raster group
 
   const int tiles = p.tiles_m * p.tiles_n;
   const int kblocks = (int)((K + BK - 1) / BK);
-  const int sms = st->sm_count;
+  const int sms = st->sm_count * (bm == 128 ? 1 : 2);  // concurrently resident CTAs
   const int max_partials = (int)(kWorkspaceBytes / (BM * BN * sizeof(double)));
   p.kblocks = kblocks;
   p.c_prefetch = (((uintptr_t)C & 15) == 0 && (ldc % 2 == 0)) ? 1 : 0;
-  const int dbg_flags = g_test_flags.load();
   if (dbg_flags & DGEMM_TEST_NO_C_PREFETCH) p.c_prefetch = 0;
   int grid;
   const int forced_split = g_split_k.load();
@@ -235,18 +255,22 @@ int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, c
   memset(&map_a, 0, sizeof(map_a));
   memset(&map_b, 0, sizeof(map_b));
   if (wants_tma) {
-    if (!make_map(&map_a, A, M, K, lda, BK, BM)) return DGEMM_ERR_CUDA;
+    if (!make_map(&map_a, A, M, K, lda, BK, bm)) return DGEMM_ERR_CUDA;
     p.b_blocked_map = (!(dbg_flags & DGEMM_TEST_NO_BLOCKED_B) && N % 16 == 0 && make_blocked_map(&map_b, B, K, N, ldb, BK, BN / 16)) ? 1 : 0;
     if (!p.b_blocked_map && !make_map(&map_b, B, K, N, ldb, 16, BK)) return DGEMM_ERR_CUDA;
     if (variant == DGEMM_VARIANT_TMA_WS)
       dgemm_dmma_ws_kernel<true><<<grid, WS_THREADS, SMEM_BYTES, stream>>>(map_a, map_b, p);
+    else if (bm == 128)
+      dgemm_dmma_kernel<true, 128><<<grid, TileCfg<128>::THREADS_, TileCfg<128>::SMEM_BYTES_, stream>>>(map_a, map_b, p);
     else
-      dgemm_dmma_kernel<true><<<grid, THREADS, SMEM_BYTES, stream>>>(map_a, map_b, p);
+      dgemm_dmma_kernel<true, 64><<<grid, TileCfg<64>::THREADS_, TileCfg<64>::SMEM_BYTES_, stream>>>(map_a, map_b, p);
   } else {
     if (variant == DGEMM_VARIANT_GENERIC_WS)
       dgemm_dmma_ws_kernel<false><<<grid, WS_THREADS, SMEM_BYTES, stream>>>(map_a, map_b, p);
+    else if (bm == 128)
+      dgemm_dmma_kernel<false, 128><<<grid, TileCfg<128>::THREADS_, TileCfg<128>::SMEM_BYTES_, stream>>>(map_a, map_b, p);
     else
-      dgemm_dmma_kernel<false><<<grid, THREADS, SMEM_BYTES, stream>>>(map_a, map_b, p);
+      dgemm_dmma_kernel<false, 64><<<grid, TileCfg<64>::THREADS_, TileCfg<64>::SMEM_BYTES_, stream>>>(map_a, map_b, p);
   }
   g_launches.fetch_add(1);
   if (cudaGetLastError() != cudaSuccess) return DGEMM_ERR_CUDA;
@@ -310,6 +334,7 @@ int launch_gemm_static_ws(int64_t M, int64_t N, int64_t K, const double* A, int6
   GemmParams p;
   memset(&p, 0, sizeof(p));
   p.M = (int)M; p.N = (int)N; p.K = (int)K;
+  p.bm = BM;
   p.tiles_m = (int)((M + BM - 1) / BM);
   p.tiles_n = (int)((N + BN - 1) / BN);
   p.A = A; p.B = B; p.C = C;
@@ -347,9 +372,9 @@ int launch_gemm_static_ws(int64_t M, int64_t N, int64_t K, const double* A, int6
   memset(&map_b, 0, sizeof(map_b));
   if (tma_ok) {
     if (!make_map(&map_a, A, M, K, lda, BK, BM) || !make_map(&map_b, B, K, N, ldb, 16, BK)) return DGEMM_ERR_CUDA;
-    dgemm_dmma_kernel<true><<<grid, THREADS, SMEM_BYTES, stream>>>(map_a, map_b, p);
+    dgemm_dmma_kernel<true, 128><<<grid, TileCfg<128>::THREADS_, TileCfg<128>::SMEM_BYTES_, stream>>>(map_a, map_b, p);
   } else {
-    dgemm_dmma_kernel<false><<<grid, THREADS, SMEM_BYTES, stream>>>(map_a, map_b, p);
+    dgemm_dmma_kernel<false, 128><<<grid, TileCfg<128>::THREADS_, TileCfg<128>::SMEM_BYTES_, stream>>>(map_a, map_b, p);
   }
   g_launches.fetch_add(1);
   if (cudaGetLastError() != cudaSuccess) return DGEMM_ERR_CUDA;
@@ -468,7 +493,7 @@ int dgemm_set_variant(int variant) {
 }
 
 int dgemm_set_test_flags(int flags) {
-  if (flags < 0 || flags > (DGEMM_TEST_NO_C_PREFETCH | DGEMM_TEST_NO_BLOCKED_B)) return DGEMM_ERR_VARIANT;
+  if (flags < 0 || flags > (DGEMM_TEST_NO_C_PREFETCH | DGEMM_TEST_NO_BLOCKED_B | DGEMM_TEST_TALL_TILES)) return DGEMM_ERR_VARIANT;
   g_test_flags.store(flags);
   return DGEMM_OK;
 }

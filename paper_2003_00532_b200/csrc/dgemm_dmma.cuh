@@ -58,6 +58,7 @@ constexpr int C_PREFETCH_KBLOCKS = 8;       // C tile is requested into L2 this 
 // order; no CTA ever waits for another one.
 struct GemmParams {
   int M, N, K;
+  int bm;                 // rows of a CTA tile: 128 (one CTA per SM) or 64 (two CTAs per SM)
   int tiles_m, tiles_n;
   int kblocks;            // ceil(K / BK)
   int dp_tiles;           // tiles handled in phase 1
@@ -172,18 +173,18 @@ __device__ __noinline__ void fetch_work(const GemmParams& p, int cta, int nctas,
 }
 
 // Asks L2 for rows r0, r0 + rstep, ... of the C tile (tm, tn) ahead of its epilogue.
-__device__ __forceinline__ void prefetch_c_rows_inline(const double* C, long long ldc, int M, int N, int tm, int tn,
-                                                       int r0, int rstep) {
+__device__ __forceinline__ void prefetch_c_rows_inline(const double* C, long long ldc, int M, int N, int bm, int tm,
+                                                       int tn, int r0, int rstep) {
   const int cols = min(BN, N - tn * BN) & ~1;
   if (cols <= 0) return;
-  for (int r = r0; r < BM; r += rstep) {
-    const int row = tm * BM + r;
+  for (int r = r0; r < bm; r += rstep) {
+    const int row = tm * bm + r;
     if (row < M) ptx::prefetch_l2_bulk(C + (long long)row * ldc + (long long)tn * BN, (uint32_t)cols * 8u);
   }
 }
-__device__ __noinline__ void prefetch_c_rows(const double* C, long long ldc, int M, int N, int tm, int tn, int r0,
-                                             int rstep) {
-  prefetch_c_rows_inline(C, ldc, M, N, tm, tn, r0, rstep);
+__device__ __noinline__ void prefetch_c_rows(const double* C, long long ldc, int M, int N, int bm, int tm, int tn,
+                                             int r0, int rstep) {
+  prefetch_c_rows_inline(C, ldc, M, N, bm, tm, tn, r0, rstep);
 }
 
 // B stage as eight 2-D boxes of 16 columns (used when N is not a multiple of 16).
@@ -252,7 +253,7 @@ struct LaneMap {
   uint32_t a_off[2], b_off[2][2];
 };
 
-__device__ __forceinline__ LaneMap make_lane_map(int warp, int lane) {
+__device__ __forceinline__ LaneMap make_lane_map(int warp, int lane, int a_stage_bytes = A_STAGE_BYTES) {
   LaneMap m;
   m.g = lane >> 2;   // MMA group id (row of A / column of B fragment)
   m.t = lane & 3;    // thread in group (k index of the fragments)
@@ -264,13 +265,14 @@ __device__ __forceinline__ LaneMap make_lane_map(int warp, int lane) {
     m.a_off[h] = (64 * m.wm + m.rm) * 128 + (((4 * h + m.t) ^ m.rm) << 4);
 #pragma unroll
     for (int b = 0; b < 2; ++b)
-      m.b_off[h][b] = A_STAGE_BYTES + (2 * m.wn) * B_BOX_BYTES + (8 * h + 2 * m.t + b) * 128 + ((m.g ^ (2 * m.t + b)) << 4);
+      m.b_off[h][b] = a_stage_bytes + (2 * m.wn) * B_BOX_BYTES + (8 * h + 2 * m.t + b) * 128 + ((m.g ^ (2 * m.t + b)) << 4);
   }
   return m;
 }
 
 // The arithmetic of one k-block (16 k values) on one stage: acc += A_tile * B_tile for this warp's
 // 64 x 32 tile. Returns a token that depends on every fragment register this lane loaded.
+template <bool M16 = false>
 __device__ __forceinline__ int compute_kblock(const uint8_t* st, const LaneMap& m, double (&acc)[4][4][4]) {
   int token = 0;
 #pragma unroll
@@ -298,6 +300,11 @@ __device__ __forceinline__ int compute_kblock(const uint8_t* st, const LaneMap& 
     for (int mt = 0; mt < 4; ++mt)
 #pragma unroll
       for (int np = 0; np < 2; ++np) {
+        if (M16) {  // same arithmetic with the 16 x 8 x 8 shape: a quarter of the instructions
+          ptx::dmma_m16n8k8(acc[mt][2 * np + 0], alo[mt].x, ahi[mt].x, alo[mt].y, ahi[mt].y, bf[np][0].x, bf[np][1].x);
+          ptx::dmma_m16n8k8(acc[mt][2 * np + 1], alo[mt].x, ahi[mt].x, alo[mt].y, ahi[mt].y, bf[np][0].y, bf[np][1].y);
+          continue;
+        }
         ptx::dmma_m8n8k4(acc[mt][2 * np + 0][0], acc[mt][2 * np + 0][1], alo[mt].x, bf[np][0].x);
         ptx::dmma_m8n8k4(acc[mt][2 * np + 0][2], acc[mt][2 * np + 0][3], ahi[mt].x, bf[np][0].x);
         ptx::dmma_m8n8k4(acc[mt][2 * np + 1][0], acc[mt][2 * np + 1][1], alo[mt].x, bf[np][0].y);
@@ -330,7 +337,7 @@ __device__ __forceinline__ void store_tile(const GemmParams& p, const Work& w, c
   const int tm = w.tm, tn = w.tn;
   // This lane owns, for each mt, half (rows +0 / +8) and np, four consecutive
   // columns n = 32wn + 16np + 4t + {0,1,2,3} = {nt=2np:c0, nt=2np+1:c0, nt=2np:c1, nt=2np+1:c1}
-  const int row_base = tm * BM + 64 * m.wm + m.rm;
+  const int row_base = tm * p.bm + 64 * m.wm + m.rm;
   const int col_base = tn * BN + 32 * m.wn + 4 * m.t;
   if (w.slot >= 0) {
     double* dst = p.partial + (long long)w.slot * (long long)(BM * BN);
@@ -346,7 +353,7 @@ __device__ __forceinline__ void store_tile(const GemmParams& p, const Work& w, c
                       acc[mt][2 * np][2 * half + 1], acc[mt][2 * np + 1][2 * half + 1]);
         }
   } else {
-    const bool interior = (tm * BM + BM <= p.M) && (tn * BN + BN <= p.N);
+    const bool interior = (tm * p.bm + p.bm <= p.M) && (tn * BN + BN <= p.N);
     const bool vec32 = ((reinterpret_cast<uintptr_t>(p.C) & 31) == 0) && ((p.ldc & 3) == 0);
     if (interior && vec32) {
       // batches of 4 * MT_PER_BATCH outstanding 32-byte loads per thread, then the adds and stores
@@ -400,10 +407,31 @@ __device__ __forceinline__ void store_tile(const GemmParams& p, const Work& w, c
   }
 }
 
-template <bool USE_TMA>
-__global__ void __launch_bounds__(THREADS, 1)
+// Shape of the default kernel for a tile height TBM: 128 rows -> 8 warps, 6 stages of 32 KB, one CTA
+// per SM; 64 rows -> 4 warps, 4 stages of 24 KB, two CTAs per SM (they drift out of phase, so one
+// CTA's k-block boundaries and epilogues overlap with the other's arithmetic).
+template <int TBM>
+struct TileCfg {
+  static constexpr int WARPS_ = TBM / 16;
+  static constexpr int THREADS_ = WARPS_ * 32;
+  static constexpr int STAGES_ = TBM == 128 ? 6 : 4;
+  static constexpr int LOOKAHEAD_ = STAGES_ - 2;
+  static constexpr int A_BYTES = TBM * BK * 8;
+  static constexpr int STAGE_BYTES_ = A_BYTES + B_STAGE_BYTES;
+  static constexpr int SMEM_BYTES_ = STAGES_ * STAGE_BYTES_ + SMEM_ALIGN + 1024;
+  static constexpr int CTAS_PER_SM = TBM == 128 ? 1 : 2;
+};
+
+template <bool USE_TMA, int TBM>
+__global__ void __launch_bounds__(TileCfg<TBM>::THREADS_, TileCfg<TBM>::CTAS_PER_SM)
 dgemm_dmma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                   const __grid_constant__ GemmParams p) {
+  constexpr int STAGES = TileCfg<TBM>::STAGES_;
+  constexpr int LOOKAHEAD = TileCfg<TBM>::LOOKAHEAD_;
+  constexpr int WARPS = TileCfg<TBM>::WARPS_;
+  constexpr int THREADS = TileCfg<TBM>::THREADS_;
+  constexpr int A_STAGE_BYTES = TileCfg<TBM>::A_BYTES;
+  constexpr int STAGE_BYTES = TileCfg<TBM>::STAGE_BYTES_;
   extern __shared__ uint8_t smem_raw[];
   // tiles at a 1024-byte boundary, barriers behind them
   const uint32_t raw = ptx::smem_u32(smem_raw);
@@ -476,7 +504,7 @@ dgemm_dmma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
       if (warp == (int)(lit % WARPS) && lane == 0) {
         if (wait_bounded<false>(empty_bar + 8 * s, ph ^ 1u, abort_flag, p)) {
           ptx::mbar_arrive_expect_tx(fb, STAGE_BYTES);
-          ptx::tma_load_2d(sa, &map_a, kb * BK, cur_tm * BM, fb);
+          ptx::tma_load_2d(sa, &map_a, kb * BK, cur_tm * TBM, fb);
           if (p.b_blocked_map) {
             ptx::tma_load_3d(sb, &map_b, 0, kb * BK, cur_tn * (BN / 16), fb);
           } else {
@@ -492,19 +520,20 @@ dgemm_dmma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
       // 8-byte asynchronous copies with zero fill outside the matrices; any alignment, any leading
       // dimension. A: 16 consecutive threads copy the 16 k values of one row (8 rows per thread);
       // B: 32 consecutive threads copy 32 consecutive columns of one k row (8 k rows per thread).
-      const int m0 = cur_tm * BM, n0 = cur_tn * BN, k0 = kb * BK;
+      const int m0 = cur_tm * TBM, n0 = cur_tn * BN, k0 = kb * BK;
       {
         const int a_k = tid & 15, row0 = tid >> 4;
         const int k = k0 + a_k;
         const bool kin = k < p.K;
         const double* src = p.A + (long long)(m0 + row0) * p.lda + k;
         const uint32_t dst_base = sa + ((a_k & 1) << 3);
+        constexpr int ROW_STEP = THREADS / 16;
 #pragma unroll
-        for (int i = 0; i < BM / 16; ++i) {
-          const int row = row0 + 16 * i;
+        for (int i = 0; i < TBM / ROW_STEP; ++i) {
+          const int row = row0 + ROW_STEP * i;
           const bool in = kin && (m0 + row < p.M);
           const uint32_t dst = dst_base + row * 128 + (((a_k >> 1) ^ (row & 7)) << 4);
-          ptx::cp_async_8(dst, in ? (const void*)(src + (long long)(16 * i) * p.lda) : (const void*)p.A, in ? 8u : 0u);
+          ptx::cp_async_8(dst, in ? (const void*)(src + (long long)(ROW_STEP * i) * p.lda) : (const void*)p.A, in ? 8u : 0u);
         }
       }
       {
@@ -513,12 +542,13 @@ dgemm_dmma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         const double* src = p.B + (long long)(k0 + kk0) * p.ldb + (n0 + nn);
         const uint32_t dst_base = sb + (nn >> 4) * B_BOX_BYTES + ((nn & 1) << 3);
         const int chunk = (nn & 15) >> 1;
+        constexpr int K_STEP = THREADS / 128;
 #pragma unroll
-        for (int i = 0; i < BK / 2; ++i) {
-          const int kk = kk0 + 2 * i;
+        for (int i = 0; i < BK / K_STEP; ++i) {
+          const int kk = kk0 + K_STEP * i;
           const bool in = nin && (k0 + kk < p.K);
           const uint32_t dst = dst_base + kk * 128 + ((chunk ^ (kk & 7)) << 4);
-          ptx::cp_async_8(dst, in ? (const void*)(src + (long long)(2 * i) * p.ldb) : (const void*)p.B, in ? 8u : 0u);
+          ptx::cp_async_8(dst, in ? (const void*)(src + (long long)(K_STEP * i) * p.ldb) : (const void*)p.B, in ? 8u : 0u);
         }
       }
       ptx::cp_async_mbar_arrive_noinc(fb);
@@ -526,9 +556,9 @@ dgemm_dmma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     if (kb == cur_pf) {
       // TMA staging: the issuing warp's lanes take 4 rows each; generic: one row per thread of the first 128
       if (USE_TMA) {
-        if (warp == (int)(lit % WARPS)) prefetch_c_rows(p.C, p.ldc, p.M, p.N, cur_tm, cur_tn, lane, 32);
-      } else if (tid < BM) {
-        prefetch_c_rows(p.C, p.ldc, p.M, p.N, cur_tm, cur_tn, tid, BM);
+        if (warp == (int)(lit % WARPS)) prefetch_c_rows(p.C, p.ldc, p.M, p.N, TBM, cur_tm, cur_tn, lane, 32);
+      } else if (tid < TBM) {
+        prefetch_c_rows(p.C, p.ldc, p.M, p.N, TBM, cur_tm, cur_tn, tid, TBM);
       }
     }
     ++lit;
@@ -541,7 +571,7 @@ dgemm_dmma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
 
   for (int i = 0; i < LOOKAHEAD && ok; ++i) ok = issue_next();
 
-  const LaneMap lm = make_lane_map(warp, lane);
+  const LaneMap lm = make_lane_map(warp, lane, A_STAGE_BYTES);
 
   double acc[4][4][4];  // [mt][nt = 2*np + j][c0..c3]
   uint32_t it = 0;      // k-blocks consumed so far
@@ -684,7 +714,7 @@ dgemm_dmma_ws_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
             }
           }
           if (!__all_sync(0xffffffffu, good)) { ok = false; break; }
-          if (kb == kb_pf) prefetch_c_rows_inline(p.C, p.ldc, p.M, p.N, w.tm, w.tn, lane, 32);
+          if (kb == kb_pf) prefetch_c_rows_inline(p.C, p.ldc, p.M, p.N, BM, w.tm, w.tn, lane, 32);
         } else {
           if (!wait_bounded_inline(empty_bar + 8 * s, ph ^ 1u, abort_flag, p)) { ok = false; break; }
           const int m0 = w.tm * BM, n0 = w.tn * BN, k0 = kb * BK;
@@ -717,7 +747,7 @@ dgemm_dmma_ws_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
             }
           }
           ptx::cp_async_mbar_arrive_noinc(fb);
-          if (kb == kb_pf) prefetch_c_rows_inline(p.C, p.ldc, p.M, p.N, w.tm, w.tn, 32 * pw + lane, BM);
+          if (kb == kb_pf) prefetch_c_rows_inline(p.C, p.ldc, p.M, p.N, BM, w.tm, w.tn, 32 * pw + lane, BM);
         }
       }
     }
@@ -749,7 +779,7 @@ dgemm_dmma_ws_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
         const uint32_t s = it % STAGES;
         const uint32_t ph = (it / STAGES) & 1u;
         if (!wait_bounded_inline(full_bar + 8 * s, ph, abort_flag, p)) { ok = false; break; }
-        const int token = compute_kblock(tiles + s * STAGE_BYTES, lm, acc);
+        const int token = compute_kblock<true>(tiles + s * STAGE_BYTES, lm, acc);
         release_stage(empty_bar + 8 * s, token, lane, p.zero);
       }
       if (!ok) break;
@@ -771,8 +801,8 @@ __device__ __forceinline__ void reduce_tile(const GemmParams& p, int tm, int tn,
   const int e0 = blockIdx.y * CHUNK_ELEMS;
   for (int e = e0 + 2 * threadIdx.x; e < e0 + CHUNK_ELEMS; e += 2 * REDUCE_THREADS) {
     const int r = e / BN, c = e - r * BN;
-    const int row = tm * BM + r, col = tn * BN + c;
-    if (row < p.M && col < p.N) {
+    const int row = tm * p.bm + r, col = tn * BN + c;
+    if (r < p.bm && row < p.M && col < p.N) {
       double2 sum = *reinterpret_cast<const double2*>(p.partial + (long long)slot_of(0) * (BM * BN) + e);
       for (int s = 1; s < count; ++s) {
         const double2 v = *reinterpret_cast<const double2*>(p.partial + (long long)slot_of(s) * (BM * BN) + e);

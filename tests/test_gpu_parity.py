@@ -187,6 +187,22 @@ def test_config3_8192(oracle, integer):
     _check_sampled(oracle, prob, out, 4096, seed=1)
 
 
+@pytest.mark.parametrize("n", [1024, 2304])
+def test_tall_tiles(oracle, n):
+    """The 128-row tile configuration (one CTA per SM) on a square case with a partial last wave."""
+    prob = wl.make_problem(n, n, n, seed=n + 1, integer=True)
+    dg.dgemm_set_test_flags(4)
+    try:
+        out = run_gpu(prob)
+    finally:
+        dg.dgemm_set_test_flags(0)
+    if n <= 1024:
+        _check_full(oracle, prob, out)
+    else:
+        _check_freivalds(oracle, prob, out)
+        _check_sampled(oracle, prob, out, 2048, seed=n)
+
+
 # ---- config 4: ragged shapes, padded odd leading dimensions ---------------------------------------
 
 @pytest.mark.parametrize("idx", [0, 1, 2])

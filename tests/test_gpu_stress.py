@@ -5,7 +5,7 @@ still outstanding. When that was violated, one warp's 8-row blocks of a tile cam
 fraction of the runs, mostly early in the kernel, on rank-k shapes whose tiles are short (K = 64),
 and reliably so with the optional accelerations switched off (slower epilogues, more copies per
 stage). The test repeats exactly that: integer-valued data (every correct result is bit-identical
-to the oracle's), many runs, all four settings of the test flags, both staging variants.
+to the oracle's), many runs, the settings of the test flags (including the 128-row tile), all staging variants.
 """
 import numpy as np
 import pytest
@@ -25,7 +25,7 @@ def rank_k_case(oracle):
     return prob, torch.from_numpy(want)
 
 
-@pytest.mark.parametrize("flags", [3, 1, 2, 0])
+@pytest.mark.parametrize("flags", [3, 1, 2, 0, 7, 4])
 @pytest.mark.parametrize("variant", [dg.DGEMM_VARIANT_TMA, dg.DGEMM_VARIANT_GENERIC, dg.DGEMM_VARIANT_TMA_WS,
                                      dg.DGEMM_VARIANT_GENERIC_WS])
 def test_rank_k_repeated_runs_bit_exact(rank_k_case, flags, variant):

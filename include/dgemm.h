@@ -163,7 +163,8 @@ DGEMM_API int dgemm_set_split_k(int split_k);
 enum {
   DGEMM_TEST_NO_C_PREFETCH = 1, /* do not ask L2 for the C tile ahead of the epilogue           */
   DGEMM_TEST_NO_BLOCKED_B = 2,  /* stage B with eight 2-D copies per stage instead of one 3-D copy */
-  DGEMM_TEST_TALL_TILES = 4     /* 128-row tiles, one CTA per SM, instead of 64-row tiles, two per SM */
+  DGEMM_TEST_TALL_TILES = 4,    /* 128-row tiles, one CTA per SM, instead of 64-row tiles, two per SM */
+  DGEMM_TEST_SMALL_WARP_TILES = 8 /* 32 x 32 warp tiles (twice the warps) instead of 64 x 32            */
 };
 DGEMM_API int dgemm_set_test_flags(int flags);
 

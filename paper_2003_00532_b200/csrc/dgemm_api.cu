@@ -49,6 +49,29 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 EncodeTiledFn g_encode = nullptr;
 
+template <bool USE_TMA, int TBM, int WTM>
+void launch_tile_kernel(int grid, cudaStream_t stream, const CUtensorMap& map_a, const CUtensorMap& map_b, const GemmParams& p) {
+  dgemm_dmma_kernel<USE_TMA, TBM, WTM>
+      <<<grid, TileCfg<TBM, WTM>::THREADS_, TileCfg<TBM, WTM>::SMEM_BYTES_, stream>>>(map_a, map_b, p);
+}
+
+template <bool USE_TMA>
+void launch_default_kernel(int bm, int wtm, int grid, cudaStream_t stream, const CUtensorMap& map_a,
+                           const CUtensorMap& map_b, const GemmParams& p) {
+  if (bm == 128 && wtm == 64) launch_tile_kernel<USE_TMA, 128, 64>(grid, stream, map_a, map_b, p);
+  else if (bm == 128) launch_tile_kernel<USE_TMA, 128, 32>(grid, stream, map_a, map_b, p);
+  else if (wtm == 64) launch_tile_kernel<USE_TMA, 64, 64>(grid, stream, map_a, map_b, p);
+  else launch_tile_kernel<USE_TMA, 64, 32>(grid, stream, map_a, map_b, p);
+}
+
+template <bool USE_TMA, int TBM, int WTM>
+bool configure_tile_kernel(int* occupancy) {
+  auto* k = dgemm_dmma_kernel<USE_TMA, TBM, WTM>;
+  if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, TileCfg<TBM, WTM>::SMEM_BYTES_) != cudaSuccess) return false;
+  if (cudaFuncSetAttribute(k, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared) != cudaSuccess) return false;
+  return cudaOccupancyMaxActiveBlocksPerMultiprocessor(occupancy, k, TileCfg<TBM, WTM>::THREADS_, TileCfg<TBM, WTM>::SMEM_BYTES_) == cudaSuccess;
+}
+
 // Per-device set-up, once: capability check, SM count, status-word address, shared-memory opt-in.
 int device_state(DeviceState** out) {
   int dev = -1;
@@ -68,22 +91,17 @@ int device_state(DeviceState** out) {
     if (major != 10) return DGEMM_ERR_DEVICE;
     if (cudaGetSymbolAddress(reinterpret_cast<void**>(&st.status), g_status_word) != cudaSuccess) return DGEMM_ERR_CUDA;
     if (cudaMemset(st.status, 0, sizeof(int)) != cudaSuccess) return DGEMM_ERR_CUDA;
+    int occ[8] = {0, 0, 0, 0, 0, 0, 0, 0};
     const bool attr_ok =
-        cudaFuncSetAttribute(dgemm_dmma_kernel<true, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, TileCfg<128>::SMEM_BYTES_) == cudaSuccess &&
-        cudaFuncSetAttribute(dgemm_dmma_kernel<false, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, TileCfg<128>::SMEM_BYTES_) == cudaSuccess &&
-        cudaFuncSetAttribute(dgemm_dmma_kernel<true, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, TileCfg<64>::SMEM_BYTES_) == cudaSuccess &&
-        cudaFuncSetAttribute(dgemm_dmma_kernel<false, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, TileCfg<64>::SMEM_BYTES_) == cudaSuccess &&
-        cudaFuncSetAttribute(dgemm_dmma_kernel<true, 64>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared) == cudaSuccess &&
-        cudaFuncSetAttribute(dgemm_dmma_kernel<false, 64>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared) == cudaSuccess &&
+        configure_tile_kernel<true, 128, 64>(&occ[0]) && configure_tile_kernel<false, 128, 64>(&occ[1]) &&
+        configure_tile_kernel<true, 128, 32>(&occ[2]) && configure_tile_kernel<false, 128, 32>(&occ[3]) &&
+        configure_tile_kernel<true, 64, 64>(&occ[4]) && configure_tile_kernel<false, 64, 64>(&occ[5]) &&
+        configure_tile_kernel<true, 64, 32>(&occ[6]) && configure_tile_kernel<false, 64, 32>(&occ[7]) &&
         cudaFuncSetAttribute(dgemm_dmma_ws_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) == cudaSuccess &&
         cudaFuncSetAttribute(dgemm_dmma_ws_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) == cudaSuccess;
     if (!attr_ok) return DGEMM_ERR_CUDA;
-    // the 64-row kernel is meant to run two CTAs per SM; use it only where the device really fits two
-    int occ_tma = 0, occ_gen = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ_tma, dgemm_dmma_kernel<true, 64>, TileCfg<64>::THREADS_, TileCfg<64>::SMEM_BYTES_) != cudaSuccess ||
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ_gen, dgemm_dmma_kernel<false, 64>, TileCfg<64>::THREADS_, TileCfg<64>::SMEM_BYTES_) != cudaSuccess)
-      return DGEMM_ERR_CUDA;
-    st.two_ctas_ok = (occ_tma >= 2 && occ_gen >= 2);
+    // the 64-row kernels are meant to run two CTAs per SM; use them only where the device really fits two
+    st.two_ctas_ok = occ[4] >= 2 && occ[5] >= 2 && occ[6] >= 2 && occ[7] >= 2;
     if (!g_encode) {
       void* fn = nullptr;
       cudaDriverEntryPointQueryResult qres;
@@ -184,6 +202,8 @@ int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, c
   const bool generic_large = !wants_tma && tiles128 >= 4 * (int64_t)st->sm_count;
   const int bm = (ws_variant || generic_large || (dbg_flags & DGEMM_TEST_TALL_TILES) || !st->two_ctas_ok) ? 128 : 64;
 
+  const int wtm = (dbg_flags & DGEMM_TEST_SMALL_WARP_TILES) ? 32 : 64;  // rows of a warp tile
+
   GemmParams p;
   memset(&p, 0, sizeof(p));
   p.M = (int)M; p.N = (int)N; p.K = (int)K;
@@ -260,17 +280,13 @@ int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, c
     if (!p.b_blocked_map && !make_map(&map_b, B, K, N, ldb, 16, BK)) return DGEMM_ERR_CUDA;
     if (variant == DGEMM_VARIANT_TMA_WS)
       dgemm_dmma_ws_kernel<true><<<grid, WS_THREADS, SMEM_BYTES, stream>>>(map_a, map_b, p);
-    else if (bm == 128)
-      dgemm_dmma_kernel<true, 128><<<grid, TileCfg<128>::THREADS_, TileCfg<128>::SMEM_BYTES_, stream>>>(map_a, map_b, p);
     else
-      dgemm_dmma_kernel<true, 64><<<grid, TileCfg<64>::THREADS_, TileCfg<64>::SMEM_BYTES_, stream>>>(map_a, map_b, p);
+      launch_default_kernel<true>(bm, wtm, grid, stream, map_a, map_b, p);
   } else {
     if (variant == DGEMM_VARIANT_GENERIC_WS)
       dgemm_dmma_ws_kernel<false><<<grid, WS_THREADS, SMEM_BYTES, stream>>>(map_a, map_b, p);
-    else if (bm == 128)
-      dgemm_dmma_kernel<false, 128><<<grid, TileCfg<128>::THREADS_, TileCfg<128>::SMEM_BYTES_, stream>>>(map_a, map_b, p);
     else
-      dgemm_dmma_kernel<false, 64><<<grid, TileCfg<64>::THREADS_, TileCfg<64>::SMEM_BYTES_, stream>>>(map_a, map_b, p);
+      launch_default_kernel<false>(bm, wtm, grid, stream, map_a, map_b, p);
   }
   g_launches.fetch_add(1);
   if (cudaGetLastError() != cudaSuccess) return DGEMM_ERR_CUDA;
@@ -372,9 +388,9 @@ int launch_gemm_static_ws(int64_t M, int64_t N, int64_t K, const double* A, int6
   memset(&map_b, 0, sizeof(map_b));
   if (tma_ok) {
     if (!make_map(&map_a, A, M, K, lda, BK, BM) || !make_map(&map_b, B, K, N, ldb, 16, BK)) return DGEMM_ERR_CUDA;
-    dgemm_dmma_kernel<true, 128><<<grid, TileCfg<128>::THREADS_, TileCfg<128>::SMEM_BYTES_, stream>>>(map_a, map_b, p);
+    launch_tile_kernel<true, 128, 64>(grid, stream, map_a, map_b, p);
   } else {
-    dgemm_dmma_kernel<false, 128><<<grid, TileCfg<128>::THREADS_, TileCfg<128>::SMEM_BYTES_, stream>>>(map_a, map_b, p);
+    launch_tile_kernel<false, 128, 64>(grid, stream, map_a, map_b, p);
   }
   g_launches.fetch_add(1);
   if (cudaGetLastError() != cudaSuccess) return DGEMM_ERR_CUDA;
@@ -493,7 +509,7 @@ int dgemm_set_variant(int variant) {
 }
 
 int dgemm_set_test_flags(int flags) {
-  if (flags < 0 || flags > (DGEMM_TEST_NO_C_PREFETCH | DGEMM_TEST_NO_BLOCKED_B | DGEMM_TEST_TALL_TILES)) return DGEMM_ERR_VARIANT;
+  if (flags < 0 || flags > (DGEMM_TEST_NO_C_PREFETCH | DGEMM_TEST_NO_BLOCKED_B | DGEMM_TEST_TALL_TILES | DGEMM_TEST_SMALL_WARP_TILES)) return DGEMM_ERR_VARIANT;
   g_test_flags.store(flags);
   return DGEMM_OK;
 }

@@ -250,19 +250,21 @@ __device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, vola
 //   B: lane reads columns 32wn + 16np + 2g, +1 of k row 8h + 2t + b     (np adds one box)
 struct LaneMap {
   int g, t, wm, wn, rm;
+  int row0;  // first row of this warp's tile inside the CTA tile (wt_rows * wm)
   uint32_t a_off[2], b_off[2][2];
 };
 
-__device__ __forceinline__ LaneMap make_lane_map(int warp, int lane, int a_stage_bytes = A_STAGE_BYTES) {
+__device__ __forceinline__ LaneMap make_lane_map(int warp, int lane, int a_stage_bytes = A_STAGE_BYTES, int wt_rows = 64) {
   LaneMap m;
   m.g = lane >> 2;   // MMA group id (row of A / column of B fragment)
   m.t = lane & 3;    // thread in group (k index of the fragments)
   m.wm = warp >> 2;  // 0..1 : 64-row slab of the CTA tile
   m.wn = warp & 3;   // 0..3 : 32-column slab
   m.rm = rowmap(m.g);
+  m.row0 = wt_rows * m.wm;
 #pragma unroll
   for (int h = 0; h < 2; ++h) {
-    m.a_off[h] = (64 * m.wm + m.rm) * 128 + (((4 * h + m.t) ^ m.rm) << 4);
+    m.a_off[h] = (m.row0 + m.rm) * 128 + (((4 * h + m.t) ^ m.rm) << 4);
 #pragma unroll
     for (int b = 0; b < 2; ++b)
       m.b_off[h][b] = a_stage_bytes + (2 * m.wn) * B_BOX_BYTES + (8 * h + 2 * m.t + b) * 128 + ((m.g ^ (2 * m.t + b)) << 4);
@@ -272,14 +274,14 @@ __device__ __forceinline__ LaneMap make_lane_map(int warp, int lane, int a_stage
 
 // The arithmetic of one k-block (16 k values) on one stage: acc += A_tile * B_tile for this warp's
 // 64 x 32 tile. Returns a token that depends on every fragment register this lane loaded.
-template <bool M16 = false>
-__device__ __forceinline__ int compute_kblock(const uint8_t* st, const LaneMap& m, double (&acc)[4][4][4]) {
+template <bool M16 = false, int MT = 4>
+__device__ __forceinline__ int compute_kblock(const uint8_t* st, const LaneMap& m, double (&acc)[MT][4][4]) {
   int token = 0;
 #pragma unroll
   for (int h = 0; h < 2; ++h) {
-    double2 alo[4], ahi[4], bf[2][2];
+    double2 alo[MT], ahi[MT], bf[2][2];
 #pragma unroll
-    for (int mt = 0; mt < 4; ++mt) {
+    for (int mt = 0; mt < MT; ++mt) {
       alo[mt] = *reinterpret_cast<const double2*>(st + m.a_off[h] + mt * 2048);
       ahi[mt] = *reinterpret_cast<const double2*>(st + m.a_off[h] + mt * 2048 + 1024);
     }
@@ -289,7 +291,7 @@ __device__ __forceinline__ int compute_kblock(const uint8_t* st, const LaneMap& 
       for (int b = 0; b < 2; ++b)
         bf[np][b] = *reinterpret_cast<const double2*>(st + m.b_off[h][b] + np * B_BOX_BYTES);
 #pragma unroll
-    for (int mt = 0; mt < 4; ++mt)
+    for (int mt = 0; mt < MT; ++mt)
       token ^= __double2loint(alo[mt].x) ^ __double2hiint(alo[mt].y) ^ __double2loint(ahi[mt].x) ^ __double2hiint(ahi[mt].y);
 #pragma unroll
     for (int np = 0; np < 2; ++np)
@@ -297,7 +299,7 @@ __device__ __forceinline__ int compute_kblock(const uint8_t* st, const LaneMap& 
     // Eight k values per block as two k4 steps (x: k = 8h + 2t, y: k = 8h + 2t + 1) of the
     // m8n8k4 shape; rows g (alo) and g + 8 (ahi) are separate 8 x 8 tiles.
 #pragma unroll
-    for (int mt = 0; mt < 4; ++mt)
+    for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
       for (int np = 0; np < 2; ++np) {
         if (M16) {  // same arithmetic with the 16 x 8 x 8 shape: a quarter of the instructions
@@ -332,22 +334,22 @@ __device__ __forceinline__ void release_stage(uint32_t empty_bar_s, int token, i
 
 // Epilogue of one work item: adds the accumulators to the C tile (or stores them as a partial tile
 // in the workspace when the item covers only part of K).
-template <int MT_PER_BATCH>
-__device__ __forceinline__ void store_tile(const GemmParams& p, const Work& w, const LaneMap& m, double (&acc)[4][4][4]) {
+template <int MT_PER_BATCH, int MT = 4>
+__device__ __forceinline__ void store_tile(const GemmParams& p, const Work& w, const LaneMap& m, double (&acc)[MT][4][4]) {
   const int tm = w.tm, tn = w.tn;
   // This lane owns, for each mt, half (rows +0 / +8) and np, four consecutive
   // columns n = 32wn + 16np + 4t + {0,1,2,3} = {nt=2np:c0, nt=2np+1:c0, nt=2np:c1, nt=2np+1:c1}
-  const int row_base = tm * p.bm + 64 * m.wm + m.rm;
+  const int row_base = tm * p.bm + m.row0 + m.rm;
   const int col_base = tn * BN + 32 * m.wn + 4 * m.t;
   if (w.slot >= 0) {
     double* dst = p.partial + (long long)w.slot * (long long)(BM * BN);
 #pragma unroll
-    for (int mt = 0; mt < 4; ++mt)
+    for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
       for (int half = 0; half < 2; ++half)
 #pragma unroll
         for (int np = 0; np < 2; ++np) {
-          const int r = 64 * m.wm + m.rm + 16 * mt + 8 * half;
+          const int r = m.row0 + m.rm + 16 * mt + 8 * half;
           const int c = 32 * m.wn + 4 * m.t + 16 * np;
           ptx::stg256(dst + r * BN + c, acc[mt][2 * np][2 * half], acc[mt][2 * np + 1][2 * half],
                       acc[mt][2 * np][2 * half + 1], acc[mt][2 * np + 1][2 * half + 1]);
@@ -358,7 +360,7 @@ __device__ __forceinline__ void store_tile(const GemmParams& p, const Work& w, c
     if (interior && vec32) {
       // batches of 4 * MT_PER_BATCH outstanding 32-byte loads per thread, then the adds and stores
 #pragma unroll
-      for (int mp = 0; mp < 4 / MT_PER_BATCH; ++mp) {
+      for (int mp = 0; mp < MT / MT_PER_BATCH; ++mp) {
         double cin[MT_PER_BATCH][2][2][4];
 #pragma unroll
         for (int mq = 0; mq < MT_PER_BATCH; ++mq)
@@ -386,7 +388,7 @@ __device__ __forceinline__ void store_tile(const GemmParams& p, const Work& w, c
       }
     } else {
 #pragma unroll
-      for (int mt = 0; mt < 4; ++mt)
+      for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
         for (int half = 0; half < 2; ++half) {
           const int row = row_base + 16 * mt + 8 * half;
@@ -410,28 +412,30 @@ __device__ __forceinline__ void store_tile(const GemmParams& p, const Work& w, c
 // Shape of the default kernel for a tile height TBM: 128 rows -> 8 warps, 6 stages of 32 KB, one CTA
 // per SM; 64 rows -> 4 warps, 4 stages of 24 KB, two CTAs per SM (they drift out of phase, so one
 // CTA's k-block boundaries and epilogues overlap with the other's arithmetic).
-template <int TBM>
+template <int TBM, int WTM = 64>
 struct TileCfg {
-  static constexpr int WARPS_ = TBM / 16;
+  static constexpr int MT_ = WTM / 16;               // m16 row blocks per warp tile
+  static constexpr int WARPS_ = (TBM / WTM) * 4;     // (TBM / WTM) x 4 grid of WTM x 32 warp tiles
   static constexpr int THREADS_ = WARPS_ * 32;
   static constexpr int STAGES_ = TBM == 128 ? 6 : 4;
   static constexpr int LOOKAHEAD_ = STAGES_ - 2;
   static constexpr int A_BYTES = TBM * BK * 8;
   static constexpr int STAGE_BYTES_ = A_BYTES + B_STAGE_BYTES;
-  static constexpr int SMEM_BYTES_ = STAGES_ * STAGE_BYTES_ + SMEM_ALIGN + 1024;
+  static constexpr int SMEM_BYTES_ = STAGES_ * STAGE_BYTES_ + SMEM_ALIGN + 2048;
   static constexpr int CTAS_PER_SM = TBM == 128 ? 1 : 2;
 };
 
-template <bool USE_TMA, int TBM>
-__global__ void __launch_bounds__(TileCfg<TBM>::THREADS_, TileCfg<TBM>::CTAS_PER_SM)
+template <bool USE_TMA, int TBM, int WTM = 64>
+__global__ void __launch_bounds__(TileCfg<TBM, WTM>::THREADS_, TileCfg<TBM, WTM>::CTAS_PER_SM)
 dgemm_dmma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                   const __grid_constant__ GemmParams p) {
-  constexpr int STAGES = TileCfg<TBM>::STAGES_;
-  constexpr int LOOKAHEAD = TileCfg<TBM>::LOOKAHEAD_;
-  constexpr int WARPS = TileCfg<TBM>::WARPS_;
-  constexpr int THREADS = TileCfg<TBM>::THREADS_;
-  constexpr int A_STAGE_BYTES = TileCfg<TBM>::A_BYTES;
-  constexpr int STAGE_BYTES = TileCfg<TBM>::STAGE_BYTES_;
+  constexpr int MT = TileCfg<TBM, WTM>::MT_;
+  constexpr int STAGES = TileCfg<TBM, WTM>::STAGES_;
+  constexpr int LOOKAHEAD = TileCfg<TBM, WTM>::LOOKAHEAD_;
+  constexpr int WARPS = TileCfg<TBM, WTM>::WARPS_;
+  constexpr int THREADS = TileCfg<TBM, WTM>::THREADS_;
+  constexpr int A_STAGE_BYTES = TileCfg<TBM, WTM>::A_BYTES;
+  constexpr int STAGE_BYTES = TileCfg<TBM, WTM>::STAGE_BYTES_;
   extern __shared__ uint8_t smem_raw[];
   // tiles at a 1024-byte boundary, barriers behind them
   const uint32_t raw = ptx::smem_u32(smem_raw);
@@ -571,9 +575,9 @@ dgemm_dmma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
 
   for (int i = 0; i < LOOKAHEAD && ok; ++i) ok = issue_next();
 
-  const LaneMap lm = make_lane_map(warp, lane, A_STAGE_BYTES);
+  const LaneMap lm = make_lane_map(warp, lane, A_STAGE_BYTES, WTM);
 
-  double acc[4][4][4];  // [mt][nt = 2*np + j][c0..c3]
+  double acc[MT][4][4];  // [mt][nt = 2*np + j][c0..c3]
   uint32_t it = 0;      // k-blocks consumed so far
   Work w;
 
@@ -589,7 +593,7 @@ dgemm_dmma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     __syncwarp();
     if (!valid) break;
 #pragma unroll
-    for (int mt = 0; mt < 4; ++mt)
+    for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
       for (int nt = 0; nt < 4; ++nt)
 #pragma unroll
@@ -599,14 +603,14 @@ dgemm_dmma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
       const uint32_t s = it % STAGES;
       const uint32_t ph = (it / STAGES) & 1u;
       if (!wait_bounded(full_bar + 8 * s, ph, abort_flag, p)) { ok = false; break; }
-      const int token = compute_kblock(tiles + s * STAGE_BYTES, lm, acc);
+      const int token = compute_kblock<false, MT>(tiles + s * STAGE_BYTES, lm, acc);
       release_stage(empty_bar + 8 * s, token, lane, p.zero);
       // keep the load stream LOOKAHEAD k-blocks ahead: refill the stage released two k-blocks ago
       if (!issue_next()) { ok = false; break; }
     }
     if (!ok) break;
 
-    store_tile<2>(p, w, lm, acc);
+    store_tile<(MT >= 4 ? 2 : 1), MT>(p, w, lm, acc);
   }
 
   // Leaving. After a normal run every copy that was issued has been consumed. After an abort,

@@ -187,11 +187,13 @@ def test_config3_8192(oracle, integer):
     _check_sampled(oracle, prob, out, 4096, seed=1)
 
 
+@pytest.mark.parametrize("flags", [4, 8, 12])
 @pytest.mark.parametrize("n", [1024, 2304])
-def test_tall_tiles(oracle, n):
-    """The 128-row tile configuration (one CTA per SM) on a square case with a partial last wave."""
+def test_tile_configurations(oracle, n, flags):
+    """The other tile configurations (128-row CTA tiles, 32-row warp tiles) on square cases, one of
+    them with a partial last wave."""
     prob = wl.make_problem(n, n, n, seed=n + 1, integer=True)
-    dg.dgemm_set_test_flags(4)
+    dg.dgemm_set_test_flags(flags)
     try:
         out = run_gpu(prob)
     finally:
@@ -211,11 +213,17 @@ def test_config4_ragged(oracle, idx):
     _check_full(oracle, prob, run_gpu(prob))
 
 
+@pytest.mark.parametrize("flags", [0, 4, 8, 12])
 @pytest.mark.parametrize("idx", [0, 2])
-def test_config4_ragged_integer(oracle, idx):
+def test_config4_ragged_integer(oracle, idx, flags):
     M, N, K = wl.CONFIG4_SHAPES[idx]
     prob = wl.make_problem(M, N, K, 2, lda=K + 3, ldb=N + 5, ldc=N + 7, integer=True)
-    _check_full(oracle, prob, run_gpu(prob))
+    dg.dgemm_set_test_flags(flags)
+    try:
+        out = run_gpu(prob)
+    finally:
+        dg.dgemm_set_test_flags(0)
+    _check_full(oracle, prob, out)
 
 
 # ---- config 5: rank-k updates -------------------------------------------------------------------

@@ -25,7 +25,7 @@ def rank_k_case(oracle):
     return prob, torch.from_numpy(want)
 
 
-@pytest.mark.parametrize("flags", [3, 1, 2, 0, 7, 4])
+@pytest.mark.parametrize("flags", [3, 1, 2, 0, 7, 4, 8, 12, 15])
 @pytest.mark.parametrize("variant", [dg.DGEMM_VARIANT_TMA, dg.DGEMM_VARIANT_GENERIC, dg.DGEMM_VARIANT_TMA_WS,
                                      dg.DGEMM_VARIANT_GENERIC_WS])
 def test_rank_k_repeated_runs_bit_exact(rank_k_case, flags, variant):

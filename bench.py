@@ -223,7 +223,12 @@ def run_ours(args):
 
     dg.load_library()
     n = args.size
-    prob = wl.make_problem(n, n, n, 1, pin=True)  # seed 1: the large square configuration
+    if args.shape:
+        sm, sn, sk = (int(x) for x in args.shape.split(","))
+        prob = wl.make_problem(sm, sn, sk, 3, pin=True)  # another shape (profiling aid), rank-k seed
+    else:
+        sm = sn = sk = n
+        prob = wl.make_problem(n, n, n, 1, pin=True)  # seed 1: the large square configuration
     A, B, C = prob.A_buf.cuda(), prob.B_buf.cuda(), prob.C_buf.cuda()
     flop = prob.flop
     stream = torch.cuda.current_stream()
@@ -266,8 +271,8 @@ def run_ours(args):
     barrier()
     e2e_s = max_over_ranks(time.perf_counter() - t0)
     e2e_value = world * flop * e2e_steps / e2e_s / 1e12
-    h2d = 8 * (n * n * 3)
-    d2h = 8 * n * n
+    h2d = 8 * (sm * sk + sk * sn + sm * sn)
+    d2h = 8 * sm * sn
 
     if rank != 0:
         if distributed:
@@ -283,7 +288,7 @@ def run_ours(args):
     hbm_gbs = float(peaks["hbm_gbs"]) if peaks and "hbm_gbs" in peaks else 6650.0
     roofline = {
         "bound": "tensor", "achieved": achieved, "peak": peak_tflops, "unit": "TFLOP/s",
-        "frac": achieved / peak_tflops, "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get(n),
+        "frac": achieved / peak_tflops, "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get(n) if not args.shape else None,
         "kernel": "dgemm_dmma_kernel<true> (TMA staging)",
         "peak_source": (f"FP64 DMMA issue rate {FMA_PER_CLK_SM} FMA/clk/SM (measured by the register-only probe) x "
                         f"{SM_COUNT_B200} SMs x 2 x sm_max_mhz {sm_max_mhz:.0f} "
@@ -296,10 +301,10 @@ def run_ours(args):
     }
 
     # ---- CPU baseline: the oracle as it stands, on a bounded row slab -------------------------
-    cpu_rows = min(args.cpu_rows, n)
+    cpu_rows = min(args.cpu_rows, sm)
     tf_cpu, dt_cpu, cores = oracle_slab_rate(prob.A, prob.B, prob.C, cpu_rows)
     cpu_baseline = {"value": tf_cpu, "unit": "TFLOP/s", "cores": cores, "kind": "oracle",
-                    "sample": f"{cpu_rows} of {n} rows of C (rows are independent and equal-cost), "
+                    "sample": f"{cpu_rows} of {sm} rows of C (rows are independent and equal-cost), "
                               f"{dt_cpu:.1f} s"}
 
     line = {
@@ -307,7 +312,8 @@ def run_ours(args):
         "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
         "data": "synthetic",
-        "config": {"workload": f"M=N=K={n} FP64 row-major C += A*B, A,B,C uniform [-1,1), seed 1",
+        "config": {"workload": (f"M=N=K={n} FP64 row-major C += A*B, A,B,C uniform [-1,1), seed 1" if not args.shape else
+                                f"M,N,K={args.shape} FP64 row-major C += A*B, uniform [-1,1), seed 3"),
                    "parallelism": "replicas only" if world > 1 else "single GPU",
                    "l2": "operands (1.6 GB at 8192) exceed the 126 MB L2; no flush between steps",
                    "pct_of_fp64_peak": 100.0 * value / world / peak_tflops},
@@ -336,6 +342,7 @@ def main():
     ap.add_argument("--ref-rows", type=int, default=128, help="rows of C per step of the reference arm")
     ap.add_argument("--cpu-rows", type=int, default=3072, help="rows of C in the cpu_baseline sample")
     ap.add_argument("--e2e-steps", type=int, default=5)
+    ap.add_argument("--shape", type=str, default="", help="M,N,K of another (non-square) workload; profiling aid")
     ap.add_argument("--no-sweep", action="store_true", help="skip the size sweep and the ragged / rank-k shapes")
     args = ap.parse_args()
     if args.steps < 1:

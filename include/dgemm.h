@@ -183,6 +183,15 @@ DGEMM_API int dgemm_last_device_status(void *stream);
 DGEMM_API int64_t dgemm_launch_count(void);
 
 /*
+ * Self-test of the bounded device-side waits (no counterpart in the paper). Launches one thread
+ * block that waits on a barrier nobody signals, with a limit of `limit_us` microseconds
+ * (clamped to 1 .. 1 000 000). Synchronous. Returns DGEMM_OK if every thread gave up its wait and
+ * the kernel returned normally; the device status word then holds DGEMM_ERR_TIMEOUT, which the
+ * next dgemm_last_device_status call returns and clears. Nothing traps or hangs.
+ */
+DGEMM_API int dgemm_selftest_wait_timeout(int limit_us);
+
+/*
  * Measures the FP64 issue rate of the current device with a register-only loop of dependent
  * mma.sync m16n8k8 f64 instructions on all SMs for about `millis` milliseconds (the roofline
  * denominator; the paper computes its machine peak from unit counts in Section 1.2 and this is

@@ -78,6 +78,8 @@ def load_library() -> ctypes.CDLL:
             lib.dgemm_set_split_k.restype = ctypes.c_int
             lib.dgemm_last_device_status.argtypes = [vp]
             lib.dgemm_last_device_status.restype = ctypes.c_int
+            lib.dgemm_selftest_wait_timeout.argtypes = [ctypes.c_int]
+            lib.dgemm_selftest_wait_timeout.restype = ctypes.c_int
             lib.dgemm_launch_count.argtypes = []
             lib.dgemm_launch_count.restype = ctypes.c_int64
             lib.dgemm_fp64_peak_probe.argtypes = [ctypes.c_int, ctypes.POINTER(ctypes.c_double),
@@ -203,6 +205,14 @@ def dgemm_set_test_flags(flags: int) -> int:
 
 def dgemm_last_device_status(stream=None) -> int:
     return int(load_library().dgemm_last_device_status(_stream_handle(stream)))
+
+
+def dgemm_selftest_wait_timeout(limit_us: int = 1000) -> int:
+    """Runs the bounded-wait self-test (a wait that must give up after ``limit_us``)."""
+    rc = load_library().dgemm_selftest_wait_timeout(int(limit_us))
+    if rc < 0:
+        raise DgemmError(rc, "dgemm_selftest_wait_timeout")
+    return rc
 
 
 def dgemm_launch_count() -> int:

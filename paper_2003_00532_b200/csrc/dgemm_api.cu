@@ -536,6 +536,35 @@ int dgemm_last_device_status(void* stream) {
 
 int64_t dgemm_launch_count(void) { return g_launches.load(); }
 
+int dgemm_selftest_wait_timeout(int limit_us) {
+  DeviceState* st = nullptr;
+  int rc = device_state(&st);
+  if (rc != DGEMM_OK) return rc;
+  if (limit_us < 1) limit_us = 1;
+  if (limit_us > 1000000) limit_us = 1000000;
+  GemmParams p;
+  memset(&p, 0, sizeof(p));
+  p.wait_limit_ns = (unsigned long long)limit_us * 1000ull;
+  p.status = st->status;
+  int* gave_up = nullptr;
+  if (cudaMalloc(reinterpret_cast<void**>(&gave_up), sizeof(int)) != cudaSuccess) return DGEMM_ERR_CUDA;
+  int host_gave_up = 0;
+  rc = DGEMM_ERR_CUDA;
+  do {
+    if (cudaMemset(gave_up, 0, sizeof(int)) != cudaSuccess) break;
+    dgemm_wait_timeout_selftest_kernel<<<1, 64>>>(p, gave_up);
+    g_launches.fetch_add(1);
+    if (cudaGetLastError() != cudaSuccess) break;
+    if (cudaDeviceSynchronize() != cudaSuccess) break;
+    if (cudaMemcpy(&host_gave_up, gave_up, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) break;
+    rc = DGEMM_OK;
+  } while (0);
+  cudaFree(gave_up);
+  if (rc != DGEMM_OK) return rc;
+  // all 64 threads must have left their wait; the status word (read by dgemm_last_device_status) says why
+  return host_gave_up == 64 ? DGEMM_OK : DGEMM_ERR_CUDA;
+}
+
 int dgemm_fp64_peak_probe(int millis, double* fma_per_clk_sm, double* tflops) {
   DeviceState* st = nullptr;
   int rc = device_state(&st);

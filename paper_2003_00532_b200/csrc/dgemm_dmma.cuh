@@ -845,6 +845,22 @@ __global__ void dgemm_tail_reduce_kernel(const GemmParams p) {
   });
 }
 
+// Self-test of the bounded wait: one CTA waits on an mbarrier that nobody signals. The wait gives up
+// after p.wait_limit_ns, records DGEMM_ERR_TIMEOUT in the status word and the kernel returns
+// normally (nothing traps, nothing spins without a limit).
+__global__ void dgemm_wait_timeout_selftest_kernel(const __grid_constant__ GemmParams p, int* gave_up) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    ptx::mbar_init(ptx::smem_u32(&bar), 1);
+    abort_flag = 0;
+    ptx::fence_barrier_init();
+  }
+  __syncthreads();
+  const bool ok = wait_bounded(ptx::smem_u32(&bar), 0u, &abort_flag, p);
+  if (!ok) atomicAdd(gave_up, 1);
+}
+
 // Rung 0 of the ladder: the naive nest with one thread per C element (Section 2.1).
 __global__ void dgemm_naive_kernel(int M, int N, int K, const double* __restrict__ A, long long lda,
                                    const double* __restrict__ B, long long ldb, double* C, long long ldc) {

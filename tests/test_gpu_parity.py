@@ -324,3 +324,14 @@ def test_non_default_stream(oracle):
     want = prob.C.clone().numpy()
     oracle.dgemm_oracle(prob.A.numpy(), prob.B.numpy(), want)
     assert np.array_equal(C.cpu().numpy(), want)
+
+
+def test_bounded_wait_gives_up_and_reports(oracle):
+    """A device-side wait that can never be satisfied ends after its limit with DGEMM_ERR_TIMEOUT in
+    the status word; the context stays usable and the next GEMM is correct."""
+    assert dg.dgemm_last_device_status() == 0
+    assert dg.dgemm_selftest_wait_timeout(500) == 0
+    assert dg.dgemm_last_device_status() == -8      # DGEMM_ERR_TIMEOUT, read and cleared
+    assert dg.dgemm_last_device_status() == 0
+    prob = wl.make_problem(200, 150, 90, seed=51, integer=True)
+    _check_full(oracle, prob, run_gpu(prob))

@@ -78,6 +78,12 @@ enum {
  * ranges, DGEMM_ERR_ALIAS). Pointers must be 8-byte aligned; a faster path is taken when A and
  * B are 16-byte aligned with even lda and ldb.
  *
+ * Operands that the tensor-copy engine cannot address (A or B not 16-byte aligned, or an odd
+ * leading dimension) are, when the problem is large enough for the copy to be cheap next to the
+ * arithmetic, first packed into a library-owned per-device scratch buffer (grown on demand with
+ * a synchronising cudaFree/cudaMalloc, at most 2 GiB); smaller ones are staged directly with
+ * 8-byte copies. The same sharing rule as for the workspace below applies to that buffer.
+ *
  * Problems with few output tiles split K over several thread blocks; their partial sums go
  * through a library-owned per-device workspace that is allocated on first need (a synchronising
  * cudaMalloc; do that first call outside stream capture) and is shared by all calls, which are
@@ -164,7 +170,8 @@ enum {
   DGEMM_TEST_NO_C_PREFETCH = 1, /* do not ask L2 for the C tile ahead of the epilogue           */
   DGEMM_TEST_NO_BLOCKED_B = 2,  /* stage B with eight 2-D copies per stage instead of one 3-D copy */
   DGEMM_TEST_TALL_TILES = 4,    /* 128-row tiles, one CTA per SM, instead of 64-row tiles, two per SM */
-  DGEMM_TEST_SMALL_WARP_TILES = 8 /* 32 x 32 warp tiles (twice the warps) instead of 64 x 32            */
+  DGEMM_TEST_SMALL_WARP_TILES = 8, /* 32 x 32 warp tiles (twice the warps) instead of 64 x 32           */
+  DGEMM_TEST_NO_PACKING = 16    /* never pack unaligned operands: always use the generic staging      */
 };
 DGEMM_API int dgemm_set_test_flags(int flags);
 

@@ -24,6 +24,8 @@ constexpr size_t kWorkspaceBytes = 640ull * BM * BN * sizeof(double);  // 80 MiB
 constexpr unsigned long long kWaitLimitNs = 4000000000ull;            // 4 s per device-side wait
 constexpr int kAutoTma = DGEMM_VARIANT_TMA;          // what DGEMM_VARIANT_AUTO picks for aligned operands
 constexpr int kAutoGeneric = DGEMM_VARIANT_GENERIC;  // ... and for unaligned ones
+constexpr double kPackMinFlopPerByte = 64.0;       // pack unaligned operands only if the copy is this cheap
+constexpr size_t kPackMaxBytes = 2ull << 30;       // ... and the packed copies fit in 2 GiB
 constexpr int kTailMinSpan = 1;          // stream-K tail: at least this many k-blocks per CTA
 constexpr double kTailMinSavedKblocks = 5.0;  // use the stream-K tail only if it saves this many k-block times
 
@@ -35,6 +37,8 @@ struct DeviceState {
   bool two_ctas_ok = false;    // the 64-row kernels fit two CTAs per SM on this device
   int* status = nullptr;       // device address of g_status_word
   double* workspace = nullptr; // split-K partial tiles, allocated on first need
+  double* pack_buf = nullptr;  // packed copies of unaligned operands, grown on demand
+  size_t pack_bytes = 0;
 };
 
 DeviceState g_dev[kMaxDevices];
@@ -128,6 +132,25 @@ int ensure_workspace(DeviceState* st) {
   return DGEMM_OK;
 }
 
+// Scratch for packed operands. Growing it frees the old buffer (cudaFree synchronises the device,
+// so no kernel can still be using it) and allocates a larger one.
+int ensure_pack_buffer(DeviceState* st, size_t bytes) {
+  std::lock_guard<std::mutex> lock(g_mutex);
+  if (st->pack_bytes >= bytes) return DGEMM_OK;
+  if (st->pack_buf) {
+    cudaFree(st->pack_buf);
+    st->pack_buf = nullptr;
+    st->pack_bytes = 0;
+  }
+  const size_t want = bytes + bytes / 4;  // head room against regrowing on slightly larger problems
+  if (cudaMalloc(reinterpret_cast<void**>(&st->pack_buf), want) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return DGEMM_ERR_CUDA;
+  }
+  st->pack_bytes = want;
+  return DGEMM_OK;
+}
+
 // 2-D f64 tensor map: inner extent `cols` (contiguous), outer extent `rows` with stride ld
 // doubles; box = box_cols x box_rows; 128-byte swizzle; out-of-range elements read as zero.
 bool make_map(CUtensorMap* map, const double* base, int64_t rows, int64_t cols, int64_t ld, int box_cols, int box_rows) {
@@ -182,7 +205,38 @@ int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, c
   if (rc != DGEMM_OK) return rc;
 
   int variant = g_variant.load();
-  const bool tma_ok = (((uintptr_t)A | (uintptr_t)B) & 15) == 0 && (lda % 2 == 0) && (ldb % 2 == 0);
+  bool tma_ok = (((uintptr_t)A | (uintptr_t)B) & 15) == 0 && (lda % 2 == 0) && (ldb % 2 == 0);
+  if (variant == DGEMM_VARIANT_AUTO && !tma_ok && !(g_test_flags.load() & DGEMM_TEST_NO_PACKING)) {
+    // Packing pass: worth it when the copy (16 bytes moved per packed element) is small next to
+    // the arithmetic, and the scratch stays moderate.
+    const bool pack_a = ((uintptr_t)A & 15) != 0 || (lda % 2 != 0);
+    const bool pack_b = ((uintptr_t)B & 15) != 0 || (ldb % 2 != 0);
+    const int64_t plda = K + (K & 1), pldb = N + (N & 1);
+    const size_t a_bytes = pack_a ? (size_t)M * plda * 8 : 0, b_bytes = pack_b ? (size_t)K * pldb * 8 : 0;
+    const double flop_per_byte = 2.0 * (double)M * (double)N * (double)K / (double)(a_bytes + b_bytes);
+    if (flop_per_byte >= kPackMinFlopPerByte && a_bytes + b_bytes <= kPackMaxBytes) {
+      rc = ensure_pack_buffer(st, a_bytes + b_bytes + 256);
+      if (rc != DGEMM_OK) return rc;
+      double* pa = st->pack_buf;
+      double* pb = reinterpret_cast<double*>(reinterpret_cast<char*>(st->pack_buf) + ((a_bytes + 255) & ~(size_t)255));
+      if (pack_a) {
+        dim3 grid((unsigned)((K + 255) / 256), (unsigned)((M + 7) / 8));
+        dgemm_pack_kernel<<<grid, 128, 0, stream>>>(A, lda, (int)M, (int)K, pa, plda);
+        g_launches.fetch_add(1);
+        A = pa;
+        lda = plda;
+      }
+      if (pack_b) {
+        dim3 grid((unsigned)((N + 255) / 256), (unsigned)((K + 7) / 8));
+        dgemm_pack_kernel<<<grid, 128, 0, stream>>>(B, ldb, (int)K, (int)N, pb, pldb);
+        g_launches.fetch_add(1);
+        B = pb;
+        ldb = pldb;
+      }
+      if (cudaGetLastError() != cudaSuccess) return DGEMM_ERR_CUDA;
+      tma_ok = true;
+    }
+  }
   if (variant == DGEMM_VARIANT_AUTO) variant = tma_ok ? kAutoTma : kAutoGeneric;
   const bool wants_tma = variant == DGEMM_VARIANT_TMA || variant == DGEMM_VARIANT_TMA_WS;
   if (wants_tma && !tma_ok) return DGEMM_ERR_VARIANT;
@@ -509,7 +563,7 @@ int dgemm_set_variant(int variant) {
 }
 
 int dgemm_set_test_flags(int flags) {
-  if (flags < 0 || flags > (DGEMM_TEST_NO_C_PREFETCH | DGEMM_TEST_NO_BLOCKED_B | DGEMM_TEST_TALL_TILES | DGEMM_TEST_SMALL_WARP_TILES)) return DGEMM_ERR_VARIANT;
+  if (flags < 0 || flags > (DGEMM_TEST_NO_C_PREFETCH | DGEMM_TEST_NO_BLOCKED_B | DGEMM_TEST_TALL_TILES | DGEMM_TEST_SMALL_WARP_TILES | DGEMM_TEST_NO_PACKING)) return DGEMM_ERR_VARIANT;
   g_test_flags.store(flags);
   return DGEMM_OK;
 }

@@ -845,6 +845,28 @@ __global__ void dgemm_tail_reduce_kernel(const GemmParams p) {
   });
 }
 
+// Packing pass for operands that TMA cannot address (base not 16-byte aligned or odd leading
+// dimension): copies a rows x cols matrix into a 16-byte aligned buffer with an even leading
+// dimension. This is the paper's packing step (Section 2.6) done once in HBM instead of per block;
+// it moves O(n^2) bytes for O(n^3) work. One thread per pair of columns.
+__global__ void dgemm_pack_kernel(const double* __restrict__ src, long long ld_src, int rows, int cols,
+                                  double* __restrict__ dst, long long ld_dst) {
+  const int c = 2 * (blockIdx.x * blockDim.x + threadIdx.x);
+  const int r0 = blockIdx.y * 8;
+  if (c >= cols) return;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int r = r0 + i;
+    if (r < rows) {
+      const double* s = src + (long long)r * ld_src + c;
+      double2 v;
+      v.x = s[0];
+      v.y = (c + 1 < cols) ? s[1] : 0.0;
+      *reinterpret_cast<double2*>(dst + (long long)r * ld_dst + c) = v;
+    }
+  }
+}
+
 // Self-test of the bounded wait: one CTA waits on an mbarrier that nobody signals. The wait gives up
 // after p.wait_limit_ns, records DGEMM_ERR_TIMEOUT in the status word and the kernel returns
 // normally (nothing traps, nothing spins without a limit).

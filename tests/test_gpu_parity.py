@@ -207,10 +207,28 @@ def test_tile_configurations(oracle, n, flags):
 
 # ---- config 4: ragged shapes, padded odd leading dimensions ---------------------------------------
 
+@pytest.mark.parametrize("flags", [0, 16])
 @pytest.mark.parametrize("idx", [0, 1, 2])
-def test_config4_ragged(oracle, idx):
+def test_config4_ragged(oracle, idx, flags):
+    """flags 16: without the packing pass (the odd-leading-dimension case then uses generic staging)."""
     prob = wl.config4(idx)
-    _check_full(oracle, prob, run_gpu(prob))
+    dg.dgemm_set_test_flags(flags)
+    try:
+        out = run_gpu(prob)
+    finally:
+        dg.dgemm_set_test_flags(0)
+    _check_full(oracle, prob, out)
+
+
+@pytest.mark.parametrize("offset", [0, 1])
+def test_packing_pass_unaligned_operands(oracle, offset):
+    """Odd leading dimensions and an odd element offset: A and B are packed into aligned scratch first
+    (twice in a row: the second call reuses the scratch). Integer data, exact."""
+    prob = wl.make_problem(700, 650, 1200, seed=61, lda=1203, ldb=655, ldc=657, integer=True)
+    first = run_gpu(prob, offset_elems=offset)
+    _check_full(oracle, prob, first)
+    second = run_gpu(prob, offset_elems=offset)
+    assert torch.equal(first.view(torch.int64), second.view(torch.int64))
 
 
 @pytest.mark.parametrize("flags", [0, 4, 8, 12])

@@ -98,8 +98,9 @@ DGEMM_API int dgemm_f64(int64_t M, int64_t N, int64_t K,
               void *stream);
 
 /*
- * Same operation with HOST buffers (pageable or pinned): copies A, B and C to device scratch
- * memory, runs dgemm_f64 there and copies C back (only the M x N logical part of each row is
+ * Same operation with HOST buffers (pageable or pinned; pinned buffers let the copies overlap the
+ * arithmetic): copies B to device scratch memory, then streams A and C through it in blocks of
+ * 1024 rows (upload, dgemm_f64, download on three streams), i.e. runs dgemm_f64 there and copies C back (only the M x N logical part of each row is
  * meaningful; padding columns of the host C are preserved). Synchronous: returns after the
  * result is in the host buffer. Device scratch is allocated with the stream-ordered allocator
  * and released before returning. Same argument rules and error codes as dgemm_f64

@@ -26,6 +26,7 @@ constexpr int kAutoTma = DGEMM_VARIANT_TMA;          // what DGEMM_VARIANT_AUTO 
 constexpr int kAutoGeneric = DGEMM_VARIANT_GENERIC;  // ... and for unaligned ones
 constexpr double kPackMinFlopPerByte = 64.0;       // pack unaligned operands only if the copy is this cheap
 constexpr size_t kPackMaxBytes = 2ull << 30;       // ... and the packed copies fit in 2 GiB
+constexpr int64_t kHostBlockRows = 1024;             // dgemm_f64_host: rows of A and C per pipelined block
 constexpr int kTailMinSpan = 1;          // stream-K tail: at least this many k-blocks per CTA
 constexpr double kTailMinSavedKblocks = 5.0;  // use the stream-K tail only if it saves this many k-block times
 
@@ -211,7 +212,7 @@ int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, c
     // the arithmetic, and the scratch stays moderate.
     const bool pack_a = ((uintptr_t)A & 15) != 0 || (lda % 2 != 0);
     const bool pack_b = ((uintptr_t)B & 15) != 0 || (ldb % 2 != 0);
-    const int64_t plda = K + (K & 1), pldb = N + (N & 1);
+    const int64_t plda = (K + 15) & ~(int64_t)15, pldb = (N + 15) & ~(int64_t)15;  // 128-byte aligned rows
     const size_t a_bytes = pack_a ? (size_t)M * plda * 8 : 0, b_bytes = pack_b ? (size_t)K * pldb * 8 : 0;
     const double flop_per_byte = 2.0 * (double)M * (double)N * (double)K / (double)(a_bytes + b_bytes);
     if (flop_per_byte >= kPackMinFlopPerByte && a_bytes + b_bytes <= kPackMaxBytes) {
@@ -506,34 +507,86 @@ int dgemm_f64_host(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda
   int rc = device_state(&st);
   if (rc != DGEMM_OK) return rc;
 
-  // dense device copies with even leading dimensions (keeps the TMA path available)
+  // Dense device copies with even leading dimensions (keeps the TMA path available). B is copied
+  // whole; A and C travel in blocks of rows through two buffers each, on three streams, so that
+  // the upload of block i+1, the arithmetic of block i and the download of block i-1 overlap.
   const int64_t dlda = K + (K & 1), dldb = N + (N & 1), dldc = N + (N & 1);
-  cudaStream_t s = nullptr;
-  double *dA = nullptr, *dB = nullptr, *dC = nullptr;
+  const int64_t blk = (M > 2 * kHostBlockRows) ? kHostBlockRows : M;  // rows per block
+  const int64_t nblk = (M + blk - 1) / blk;
+  const int nbuf = nblk > 1 ? 2 : 1;
+  cudaStream_t s_up = nullptr, s_run = nullptr, s_down = nullptr;
+  double* dB = nullptr;
+  double* dA[2] = {nullptr, nullptr};
+  double* dC[2] = {nullptr, nullptr};
+  cudaEvent_t ev_alloc = nullptr, ev_up[2] = {nullptr, nullptr}, ev_run[2] = {nullptr, nullptr}, ev_down[2] = {nullptr, nullptr};
   rc = DGEMM_ERR_CUDA;
   do {
-    if (cudaStreamCreateWithFlags(&s, cudaStreamNonBlocking) != cudaSuccess) break;
-    if (cudaMallocAsync(reinterpret_cast<void**>(&dA), (size_t)M * dlda * 8, s) != cudaSuccess) break;
-    if (cudaMallocAsync(reinterpret_cast<void**>(&dB), (size_t)K * dldb * 8, s) != cudaSuccess) break;
-    if (cudaMallocAsync(reinterpret_cast<void**>(&dC), (size_t)M * dldc * 8, s) != cudaSuccess) break;
-    if (cudaMemcpy2DAsync(dA, dlda * 8, A, lda * 8, K * 8, M, cudaMemcpyHostToDevice, s) != cudaSuccess) break;
-    if (cudaMemcpy2DAsync(dB, dldb * 8, B, ldb * 8, N * 8, K, cudaMemcpyHostToDevice, s) != cudaSuccess) break;
-    if (cudaMemcpy2DAsync(dC, dldc * 8, C, ldc * 8, N * 8, M, cudaMemcpyHostToDevice, s) != cudaSuccess) break;
-    rc = launch_gemm(M, N, K, dA, dlda, dB, dldb, dC, dldc, s);
-    if (rc != DGEMM_OK) break;
-    rc = DGEMM_ERR_CUDA;
-    if (cudaMemcpy2DAsync(C, ldc * 8, dC, dldc * 8, N * 8, M, cudaMemcpyDeviceToHost, s) != cudaSuccess) break;
-    if (cudaStreamSynchronize(s) != cudaSuccess) break;
+    if (cudaStreamCreateWithFlags(&s_up, cudaStreamNonBlocking) != cudaSuccess) break;
+    if (cudaStreamCreateWithFlags(&s_run, cudaStreamNonBlocking) != cudaSuccess) break;
+    if (cudaStreamCreateWithFlags(&s_down, cudaStreamNonBlocking) != cudaSuccess) break;
+    bool ok = cudaEventCreateWithFlags(&ev_alloc, cudaEventDisableTiming) == cudaSuccess;
+    for (int i = 0; i < 2 && ok; ++i)
+      ok = cudaEventCreateWithFlags(&ev_up[i], cudaEventDisableTiming) == cudaSuccess &&
+           cudaEventCreateWithFlags(&ev_run[i], cudaEventDisableTiming) == cudaSuccess &&
+           cudaEventCreateWithFlags(&ev_down[i], cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) break;
+    if (cudaMallocAsync(reinterpret_cast<void**>(&dB), (size_t)K * dldb * 8, s_up) != cudaSuccess) break;
+    for (int i = 0; i < nbuf && ok; ++i)
+      ok = cudaMallocAsync(reinterpret_cast<void**>(&dA[i]), (size_t)blk * dlda * 8, s_up) == cudaSuccess &&
+           cudaMallocAsync(reinterpret_cast<void**>(&dC[i]), (size_t)blk * dldc * 8, s_up) == cudaSuccess;
+    if (!ok) break;
+    // the other streams may touch the buffers only after the (stream-ordered) allocations
+    if (cudaEventRecord(ev_alloc, s_up) != cudaSuccess) break;
+    if (cudaStreamWaitEvent(s_run, ev_alloc, 0) != cudaSuccess || cudaStreamWaitEvent(s_down, ev_alloc, 0) != cudaSuccess) break;
+    if (cudaMemcpy2DAsync(dB, dldb * 8, B, ldb * 8, N * 8, K, cudaMemcpyHostToDevice, s_up) != cudaSuccess) break;
+    int inner = DGEMM_OK;
+    for (int64_t i = 0; i < nblk; ++i) {
+      const int b = (int)(i % nbuf);
+      const int64_t r0 = i * blk, rows = (M - r0 < blk) ? M - r0 : blk;
+      // buffer b is free again once block i - 2 has been downloaded
+      if (i >= nbuf && cudaStreamWaitEvent(s_up, ev_down[b], 0) != cudaSuccess) { inner = DGEMM_ERR_CUDA; break; }
+      if (cudaMemcpy2DAsync(dA[b], dlda * 8, A + r0 * lda, lda * 8, K * 8, rows, cudaMemcpyHostToDevice, s_up) != cudaSuccess ||
+          cudaMemcpy2DAsync(dC[b], dldc * 8, C + r0 * ldc, ldc * 8, N * 8, rows, cudaMemcpyHostToDevice, s_up) != cudaSuccess ||
+          cudaEventRecord(ev_up[b], s_up) != cudaSuccess || cudaStreamWaitEvent(s_run, ev_up[b], 0) != cudaSuccess) {
+        inner = DGEMM_ERR_CUDA;
+        break;
+      }
+      inner = launch_gemm(rows, N, K, dA[b], dlda, dB, dldb, dC[b], dldc, s_run);
+      if (inner != DGEMM_OK) break;
+      if (cudaEventRecord(ev_run[b], s_run) != cudaSuccess || cudaStreamWaitEvent(s_down, ev_run[b], 0) != cudaSuccess ||
+          cudaMemcpy2DAsync(C + r0 * ldc, ldc * 8, dC[b], dldc * 8, N * 8, rows, cudaMemcpyDeviceToHost, s_down) != cudaSuccess ||
+          cudaEventRecord(ev_down[b], s_down) != cudaSuccess) {
+        inner = DGEMM_ERR_CUDA;
+        break;
+      }
+    }
+    if (inner != DGEMM_OK) { rc = inner; break; }
+    if (cudaStreamSynchronize(s_down) != cudaSuccess || cudaStreamSynchronize(s_run) != cudaSuccess ||
+        cudaStreamSynchronize(s_up) != cudaSuccess)
+      break;
     rc = DGEMM_OK;
   } while (0);
   if (rc != DGEMM_OK) (void)cudaGetLastError();
-  if (s) {
-    if (dA) cudaFreeAsync(dA, s);
-    if (dB) cudaFreeAsync(dB, s);
-    if (dC) cudaFreeAsync(dC, s);
-    cudaStreamSynchronize(s);
-    cudaStreamDestroy(s);
+  // everything that used the buffers has finished (or failed) before they go back to the pool
+  if (s_run) cudaStreamSynchronize(s_run);
+  if (s_down) cudaStreamSynchronize(s_down);
+  if (s_up) {
+    if (dB) cudaFreeAsync(dB, s_up);
+    for (int i = 0; i < 2; ++i) {
+      if (dA[i]) cudaFreeAsync(dA[i], s_up);
+      if (dC[i]) cudaFreeAsync(dC[i], s_up);
+    }
+    cudaStreamSynchronize(s_up);
   }
+  if (ev_alloc) cudaEventDestroy(ev_alloc);
+  for (int i = 0; i < 2; ++i) {
+    if (ev_up[i]) cudaEventDestroy(ev_up[i]);
+    if (ev_run[i]) cudaEventDestroy(ev_run[i]);
+    if (ev_down[i]) cudaEventDestroy(ev_down[i]);
+  }
+  if (s_up) cudaStreamDestroy(s_up);
+  if (s_run) cudaStreamDestroy(s_run);
+  if (s_down) cudaStreamDestroy(s_down);
   return rc;
 }
 

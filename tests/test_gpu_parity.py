@@ -321,8 +321,12 @@ def test_accumulates_into_c_and_k_split_calls(oracle):
     assert torch.equal(C.cpu(), one)
 
 
-def test_host_entry_point(oracle):
-    prob = wl.make_problem(300, 257, 129, seed=31, lda=129 + 3, ldb=257 + 5, ldc=257 + 7)
+@pytest.mark.parametrize("shape", [(300, 257, 129), (2500, 300, 200), (3072, 130, 64)])
+def test_host_entry_point(oracle, shape):
+    """Host buffers; the larger cases are streamed through the device in several blocks of rows
+    (a ragged last block in the second case)."""
+    M, N, K = shape
+    prob = wl.make_problem(M, N, K, seed=31, lda=K + 3, ldb=N + 5, ldc=N + 7)
     want = prob.C.clone().contiguous().numpy()
     oracle.dgemm_oracle(np.ascontiguousarray(prob.A.numpy()), np.ascontiguousarray(prob.B.numpy()), want)
     scale = oracle.abs_product(prob.A.numpy(), prob.B.numpy(), prob.C.numpy())

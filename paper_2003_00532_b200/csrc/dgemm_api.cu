@@ -54,27 +54,29 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 EncodeTiledFn g_encode = nullptr;
 
-template <bool USE_TMA, int TBM, int WTM>
+template <bool USE_TMA, int TBM, int WTM, int TBN = BN>
 void launch_tile_kernel(int grid, cudaStream_t stream, const CUtensorMap& map_a, const CUtensorMap& map_b, const GemmParams& p) {
-  dgemm_dmma_kernel<USE_TMA, TBM, WTM>
-      <<<grid, TileCfg<TBM, WTM>::THREADS_, TileCfg<TBM, WTM>::SMEM_BYTES_, stream>>>(map_a, map_b, p);
+  dgemm_dmma_kernel<USE_TMA, TBM, WTM, TBN>
+      <<<grid, TileCfg<TBM, WTM, TBN>::THREADS_, TileCfg<TBM, WTM, TBN>::SMEM_BYTES_, stream>>>(map_a, map_b, p);
 }
 
 template <bool USE_TMA>
 void launch_default_kernel(int bm, int wtm, int grid, cudaStream_t stream, const CUtensorMap& map_a,
                            const CUtensorMap& map_b, const GemmParams& p) {
-  if (bm == 128 && wtm == 64) launch_tile_kernel<USE_TMA, 128, 64>(grid, stream, map_a, map_b, p);
+  if (bm == 256) launch_tile_kernel<USE_TMA, 256, 64, 32>(grid, stream, map_a, map_b, p);
+  else if (bm == 128 && wtm == 64) launch_tile_kernel<USE_TMA, 128, 64>(grid, stream, map_a, map_b, p);
   else if (bm == 128) launch_tile_kernel<USE_TMA, 128, 32>(grid, stream, map_a, map_b, p);
   else if (wtm == 64) launch_tile_kernel<USE_TMA, 64, 64>(grid, stream, map_a, map_b, p);
   else launch_tile_kernel<USE_TMA, 64, 32>(grid, stream, map_a, map_b, p);
 }
 
-template <bool USE_TMA, int TBM, int WTM>
+template <bool USE_TMA, int TBM, int WTM, int TBN = BN>
 bool configure_tile_kernel(int* occupancy) {
-  auto* k = dgemm_dmma_kernel<USE_TMA, TBM, WTM>;
-  if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, TileCfg<TBM, WTM>::SMEM_BYTES_) != cudaSuccess) return false;
+  auto* k = dgemm_dmma_kernel<USE_TMA, TBM, WTM, TBN>;
+  if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, TileCfg<TBM, WTM, TBN>::SMEM_BYTES_) != cudaSuccess) return false;
   if (cudaFuncSetAttribute(k, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared) != cudaSuccess) return false;
-  return cudaOccupancyMaxActiveBlocksPerMultiprocessor(occupancy, k, TileCfg<TBM, WTM>::THREADS_, TileCfg<TBM, WTM>::SMEM_BYTES_) == cudaSuccess;
+  return cudaOccupancyMaxActiveBlocksPerMultiprocessor(occupancy, k, TileCfg<TBM, WTM, TBN>::THREADS_,
+                                                       TileCfg<TBM, WTM, TBN>::SMEM_BYTES_) == cudaSuccess;
 }
 
 // Per-device set-up, once: capability check, SM count, status-word address, shared-memory opt-in.
@@ -96,17 +98,18 @@ int device_state(DeviceState** out) {
     if (major != 10) return DGEMM_ERR_DEVICE;
     if (cudaGetSymbolAddress(reinterpret_cast<void**>(&st.status), g_status_word) != cudaSuccess) return DGEMM_ERR_CUDA;
     if (cudaMemset(st.status, 0, sizeof(int)) != cudaSuccess) return DGEMM_ERR_CUDA;
-    int occ[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    int occ[10] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
     const bool attr_ok =
         configure_tile_kernel<true, 128, 64>(&occ[0]) && configure_tile_kernel<false, 128, 64>(&occ[1]) &&
         configure_tile_kernel<true, 128, 32>(&occ[2]) && configure_tile_kernel<false, 128, 32>(&occ[3]) &&
         configure_tile_kernel<true, 64, 64>(&occ[4]) && configure_tile_kernel<false, 64, 64>(&occ[5]) &&
         configure_tile_kernel<true, 64, 32>(&occ[6]) && configure_tile_kernel<false, 64, 32>(&occ[7]) &&
+        configure_tile_kernel<true, 256, 64, 32>(&occ[8]) && configure_tile_kernel<false, 256, 64, 32>(&occ[9]) &&
         cudaFuncSetAttribute(dgemm_dmma_ws_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) == cudaSuccess &&
         cudaFuncSetAttribute(dgemm_dmma_ws_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) == cudaSuccess;
     if (!attr_ok) return DGEMM_ERR_CUDA;
     // the 64-row kernels are meant to run two CTAs per SM; use them only where the device really fits two
-    st.two_ctas_ok = occ[4] >= 2 && occ[5] >= 2 && occ[6] >= 2 && occ[7] >= 2;
+    st.two_ctas_ok = occ[4] >= 2 && occ[5] >= 2 && occ[6] >= 2 && occ[7] >= 2 && occ[8] >= 2 && occ[9] >= 2;
     if (!g_encode) {
       void* fn = nullptr;
       cudaDriverEntryPointQueryResult qres;
@@ -255,7 +258,10 @@ int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, c
   // (generic staging on a problem of many waves is a little faster with the tall tile: half the B copies per thread)
   const int64_t tiles128 = ((M + 127) / 128) * ((N + BN - 1) / BN);
   const bool generic_large = !wants_tma && tiles128 >= 4 * (int64_t)st->sm_count;
-  const int bm = (ws_variant || generic_large || (dbg_flags & DGEMM_TEST_TALL_TILES) || !st->two_ctas_ok) ? 128 : 64;
+  // narrow problems (N <= 32) use a 256 x 32 tile: four warps stacked in M, no arithmetic on unused columns
+  const bool narrow = N <= 32 && !ws_variant && !(dbg_flags & (DGEMM_TEST_TALL_TILES | DGEMM_TEST_SMALL_WARP_TILES)) && st->two_ctas_ok;
+  const int bm = narrow ? 256 : (ws_variant || generic_large || (dbg_flags & DGEMM_TEST_TALL_TILES) || !st->two_ctas_ok) ? 128 : 64;
+  const int bn = narrow ? 32 : BN;
 
   const int wtm = (dbg_flags & DGEMM_TEST_SMALL_WARP_TILES) ? 32 : 64;  // rows of a warp tile
 
@@ -263,17 +269,18 @@ int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, c
   memset(&p, 0, sizeof(p));
   p.M = (int)M; p.N = (int)N; p.K = (int)K;
   p.bm = bm;
+  p.bn = bn;
   p.tiles_m = (int)((M + bm - 1) / bm);
-  p.tiles_n = (int)((N + BN - 1) / BN);
+  p.tiles_n = (int)((N + bn - 1) / bn);
   p.A = A; p.B = B; p.C = C;
   p.lda = lda; p.ldb = ldb; p.ldc = ldc;
   p.wait_limit_ns = kWaitLimitNs;
   p.status = st->status;
-  p.group_m = bm == 128 ? 8 : 16;  // 8 x 128 = 16 x 64 rows per raster group
+  p.group_m = 1024 / bm;  // 1024 rows per raster group
 
   const int tiles = p.tiles_m * p.tiles_n;
   const int kblocks = (int)((K + BK - 1) / BK);
-  const int sms = st->sm_count * (bm == 128 ? 1 : 2);  // concurrently resident CTAs
+  const int sms = st->sm_count * (bm == 128 ? 1 : 2);  // concurrently resident CTAs (128-row tiles: one per SM)
   const int max_partials = (int)(kWorkspaceBytes / (BM * BN * sizeof(double)));
   p.kblocks = kblocks;
   p.c_prefetch = (((uintptr_t)C & 15) == 0 && (ldc % 2 == 0)) ? 1 : 0;
@@ -331,7 +338,7 @@ int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, c
   memset(&map_b, 0, sizeof(map_b));
   if (wants_tma) {
     if (!make_map(&map_a, A, M, K, lda, BK, bm)) return DGEMM_ERR_CUDA;
-    p.b_blocked_map = (!(dbg_flags & DGEMM_TEST_NO_BLOCKED_B) && N % 16 == 0 && make_blocked_map(&map_b, B, K, N, ldb, BK, BN / 16)) ? 1 : 0;
+    p.b_blocked_map = (!(dbg_flags & DGEMM_TEST_NO_BLOCKED_B) && N % 16 == 0 && make_blocked_map(&map_b, B, K, N, ldb, BK, bn / 16)) ? 1 : 0;
     if (!p.b_blocked_map && !make_map(&map_b, B, K, N, ldb, 16, BK)) return DGEMM_ERR_CUDA;
     if (variant == DGEMM_VARIANT_TMA_WS)
       dgemm_dmma_ws_kernel<true><<<grid, WS_THREADS, SMEM_BYTES, stream>>>(map_a, map_b, p);
@@ -406,6 +413,7 @@ int launch_gemm_static_ws(int64_t M, int64_t N, int64_t K, const double* A, int6
   memset(&p, 0, sizeof(p));
   p.M = (int)M; p.N = (int)N; p.K = (int)K;
   p.bm = BM;
+  p.bn = BN;
   p.tiles_m = (int)((M + BM - 1) / BM);
   p.tiles_n = (int)((N + BN - 1) / BN);
   p.A = A; p.B = B; p.C = C;

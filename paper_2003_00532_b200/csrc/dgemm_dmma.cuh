@@ -58,7 +58,8 @@ constexpr int C_PREFETCH_KBLOCKS = 8;       // C tile is requested into L2 this 
 // order; no CTA ever waits for another one.
 struct GemmParams {
   int M, N, K;
-  int bm;                 // rows of a CTA tile: 128 (one CTA per SM) or 64 (two CTAs per SM)
+  int bm;                 // rows of a CTA tile: 128 (one CTA per SM), 64 (two CTAs per SM) or 256 (narrow tile)
+  int bn;                 // columns of a CTA tile: 128, or 32 for the narrow tile
   int tiles_m, tiles_n;
   int kblocks;            // ceil(K / BK)
   int dp_tiles;           // tiles handled in phase 1
@@ -173,28 +174,28 @@ __device__ __noinline__ void fetch_work(const GemmParams& p, int cta, int nctas,
 }
 
 // Asks L2 for rows r0, r0 + rstep, ... of the C tile (tm, tn) ahead of its epilogue.
-__device__ __forceinline__ void prefetch_c_rows_inline(const double* C, long long ldc, int M, int N, int bm, int tm,
-                                                       int tn, int r0, int rstep) {
-  const int cols = min(BN, N - tn * BN) & ~1;
+__device__ __forceinline__ void prefetch_c_rows_inline(const double* C, long long ldc, int M, int N, int bm, int bn,
+                                                       int tm, int tn, int r0, int rstep) {
+  const int cols = min(bn, N - tn * bn) & ~1;
   if (cols <= 0) return;
   for (int r = r0; r < bm; r += rstep) {
     const int row = tm * bm + r;
-    if (row < M) ptx::prefetch_l2_bulk(C + (long long)row * ldc + (long long)tn * BN, (uint32_t)cols * 8u);
+    if (row < M) ptx::prefetch_l2_bulk(C + (long long)row * ldc + (long long)tn * bn, (uint32_t)cols * 8u);
   }
 }
-__device__ __noinline__ void prefetch_c_rows(const double* C, long long ldc, int M, int N, int bm, int tm, int tn,
-                                             int r0, int rstep) {
-  prefetch_c_rows_inline(C, ldc, M, N, bm, tm, tn, r0, rstep);
+__device__ __noinline__ void prefetch_c_rows(const double* C, long long ldc, int M, int N, int bm, int bn, int tm,
+                                             int tn, int r0, int rstep) {
+  prefetch_c_rows_inline(C, ldc, M, N, bm, bn, tm, tn, r0, rstep);
 }
 
 // B stage as eight 2-D boxes of 16 columns (used when N is not a multiple of 16).
 __device__ __forceinline__ void tma_load_b_boxes_inline(uint32_t sb, const CUtensorMap* map_b, int n0, int k0,
-                                                        uint32_t fb) {
-#pragma unroll
-  for (int nb = 0; nb < BN / 16; ++nb) ptx::tma_load_2d(sb + nb * B_BOX_BYTES, map_b, n0 + nb * 16, k0, fb);
+                                                        uint32_t fb, int boxes = BN / 16) {
+  for (int nb = 0; nb < boxes; ++nb) ptx::tma_load_2d(sb + nb * B_BOX_BYTES, map_b, n0 + nb * 16, k0, fb);
 }
-__device__ __noinline__ void tma_load_b_boxes(uint32_t sb, const CUtensorMap* map_b, int n0, int k0, uint32_t fb) {
-  tma_load_b_boxes_inline(sb, map_b, n0, k0, fb);
+__device__ __noinline__ void tma_load_b_boxes(uint32_t sb, const CUtensorMap* map_b, int n0, int k0, uint32_t fb,
+                                              int boxes) {
+  tma_load_b_boxes_inline(sb, map_b, n0, k0, fb, boxes);
 }
 
 // Slow part of a bounded mbarrier wait: poll until the phase completes, the CTA aborts, or the
@@ -254,12 +255,13 @@ struct LaneMap {
   uint32_t a_off[2], b_off[2][2];
 };
 
-__device__ __forceinline__ LaneMap make_lane_map(int warp, int lane, int a_stage_bytes = A_STAGE_BYTES, int wt_rows = 64) {
+__device__ __forceinline__ LaneMap make_lane_map(int warp, int lane, int a_stage_bytes = A_STAGE_BYTES, int wt_rows = 64,
+                                                 int warps_n = 4) {
   LaneMap m;
   m.g = lane >> 2;   // MMA group id (row of A / column of B fragment)
   m.t = lane & 3;    // thread in group (k index of the fragments)
-  m.wm = warp >> 2;  // 0..1 : 64-row slab of the CTA tile
-  m.wn = warp & 3;   // 0..3 : 32-column slab
+  m.wm = warp / warps_n;  // row slab of the CTA tile
+  m.wn = warp % warps_n;  // 32-column slab
   m.rm = rowmap(m.g);
   m.row0 = wt_rows * m.wm;
 #pragma unroll
@@ -340,7 +342,7 @@ __device__ __forceinline__ void store_tile(const GemmParams& p, const Work& w, c
   // This lane owns, for each mt, half (rows +0 / +8) and np, four consecutive
   // columns n = 32wn + 16np + 4t + {0,1,2,3} = {nt=2np:c0, nt=2np+1:c0, nt=2np:c1, nt=2np+1:c1}
   const int row_base = tm * p.bm + m.row0 + m.rm;
-  const int col_base = tn * BN + 32 * m.wn + 4 * m.t;
+  const int col_base = tn * p.bn + 32 * m.wn + 4 * m.t;
   if (w.slot >= 0) {
     double* dst = p.partial + (long long)w.slot * (long long)(BM * BN);
 #pragma unroll
@@ -351,11 +353,11 @@ __device__ __forceinline__ void store_tile(const GemmParams& p, const Work& w, c
         for (int np = 0; np < 2; ++np) {
           const int r = m.row0 + m.rm + 16 * mt + 8 * half;
           const int c = 32 * m.wn + 4 * m.t + 16 * np;
-          ptx::stg256(dst + r * BN + c, acc[mt][2 * np][2 * half], acc[mt][2 * np + 1][2 * half],
+          ptx::stg256(dst + r * p.bn + c, acc[mt][2 * np][2 * half], acc[mt][2 * np + 1][2 * half],
                       acc[mt][2 * np][2 * half + 1], acc[mt][2 * np + 1][2 * half + 1]);
         }
   } else {
-    const bool interior = (tm * p.bm + p.bm <= p.M) && (tn * BN + BN <= p.N);
+    const bool interior = (tm * p.bm + p.bm <= p.M) && (tn * p.bn + p.bn <= p.N);
     const bool vec32 = ((reinterpret_cast<uintptr_t>(p.C) & 31) == 0) && ((p.ldc & 3) == 0);
     if (interior && vec32) {
       // batches of 4 * MT_PER_BATCH outstanding 32-byte loads per thread, then the adds and stores
@@ -412,30 +414,34 @@ __device__ __forceinline__ void store_tile(const GemmParams& p, const Work& w, c
 // Shape of the default kernel for a tile height TBM: 128 rows -> 8 warps, 6 stages of 32 KB, one CTA
 // per SM; 64 rows -> 4 warps, 4 stages of 24 KB, two CTAs per SM (they drift out of phase, so one
 // CTA's k-block boundaries and epilogues overlap with the other's arithmetic).
-template <int TBM, int WTM = 64>
+template <int TBM, int WTM = 64, int TBN = BN>
 struct TileCfg {
-  static constexpr int MT_ = WTM / 16;               // m16 row blocks per warp tile
-  static constexpr int WARPS_ = (TBM / WTM) * 4;     // (TBM / WTM) x 4 grid of WTM x 32 warp tiles
+  static constexpr int MT_ = WTM / 16;                        // m16 row blocks per warp tile
+  static constexpr int WARPS_N = TBN / 32;                    // warp grid: (TBM / WTM) x (TBN / 32)
+  static constexpr int WARPS_ = (TBM / WTM) * WARPS_N;
   static constexpr int THREADS_ = WARPS_ * 32;
-  static constexpr int STAGES_ = TBM == 128 ? 6 : 4;
-  static constexpr int LOOKAHEAD_ = STAGES_ - 2;
-  static constexpr int A_BYTES = TBM * BK * 8;
-  static constexpr int STAGE_BYTES_ = A_BYTES + B_STAGE_BYTES;
-  static constexpr int SMEM_BYTES_ = STAGES_ * STAGE_BYTES_ + SMEM_ALIGN + 2048;
   static constexpr int CTAS_PER_SM = TBM == 128 ? 1 : 2;
+  static constexpr int A_BYTES = TBM * BK * 8;
+  static constexpr int B_BYTES = BK * TBN * 8;
+  static constexpr int STAGE_BYTES_ = A_BYTES + B_BYTES;
+  // as many stages as fit: 6 x 32 KB (one CTA per SM), 4 x 24 KB or 3 x 36 KB (two CTAs per SM)
+  static constexpr int STAGES_ = TBM == 128 ? 6 : (STAGE_BYTES_ <= 24 * 1024 ? 4 : 3);
+  static constexpr int LOOKAHEAD_ = STAGES_ > 3 ? STAGES_ - 2 : STAGES_ - 1;
+  static constexpr int SMEM_BYTES_ = STAGES_ * STAGE_BYTES_ + SMEM_ALIGN + 2048;
 };
 
-template <bool USE_TMA, int TBM, int WTM = 64>
-__global__ void __launch_bounds__(TileCfg<TBM, WTM>::THREADS_, TileCfg<TBM, WTM>::CTAS_PER_SM)
+template <bool USE_TMA, int TBM, int WTM = 64, int TBN = BN>
+__global__ void __launch_bounds__(TileCfg<TBM, WTM, TBN>::THREADS_, TileCfg<TBM, WTM, TBN>::CTAS_PER_SM)
 dgemm_dmma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                   const __grid_constant__ GemmParams p) {
-  constexpr int MT = TileCfg<TBM, WTM>::MT_;
-  constexpr int STAGES = TileCfg<TBM, WTM>::STAGES_;
-  constexpr int LOOKAHEAD = TileCfg<TBM, WTM>::LOOKAHEAD_;
-  constexpr int WARPS = TileCfg<TBM, WTM>::WARPS_;
-  constexpr int THREADS = TileCfg<TBM, WTM>::THREADS_;
-  constexpr int A_STAGE_BYTES = TileCfg<TBM, WTM>::A_BYTES;
-  constexpr int STAGE_BYTES = TileCfg<TBM, WTM>::STAGE_BYTES_;
+  constexpr int MT = TileCfg<TBM, WTM, TBN>::MT_;
+  constexpr int WARPS_N = TileCfg<TBM, WTM, TBN>::WARPS_N;
+  constexpr int STAGES = TileCfg<TBM, WTM, TBN>::STAGES_;
+  constexpr int LOOKAHEAD = TileCfg<TBM, WTM, TBN>::LOOKAHEAD_;
+  constexpr int WARPS = TileCfg<TBM, WTM, TBN>::WARPS_;
+  constexpr int THREADS = TileCfg<TBM, WTM, TBN>::THREADS_;
+  constexpr int A_STAGE_BYTES = TileCfg<TBM, WTM, TBN>::A_BYTES;
+  constexpr int STAGE_BYTES = TileCfg<TBM, WTM, TBN>::STAGE_BYTES_;
   extern __shared__ uint8_t smem_raw[];
   // tiles at a 1024-byte boundary, barriers behind them
   const uint32_t raw = ptx::smem_u32(smem_raw);
@@ -510,9 +516,9 @@ dgemm_dmma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
           ptx::mbar_arrive_expect_tx(fb, STAGE_BYTES);
           ptx::tma_load_2d(sa, &map_a, kb * BK, cur_tm * TBM, fb);
           if (p.b_blocked_map) {
-            ptx::tma_load_3d(sb, &map_b, 0, kb * BK, cur_tn * (BN / 16), fb);
+            ptx::tma_load_3d(sb, &map_b, 0, kb * BK, cur_tn * (TBN / 16), fb);
           } else {
-            tma_load_b_boxes(sb, &map_b, cur_tn * BN, kb * BK, fb);
+            tma_load_b_boxes(sb, &map_b, cur_tn * TBN, kb * BK, fb, TBN / 16);
           }
         } else {
           good = 0;
@@ -524,7 +530,7 @@ dgemm_dmma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
       // 8-byte asynchronous copies with zero fill outside the matrices; any alignment, any leading
       // dimension. A: 16 consecutive threads copy the 16 k values of one row (8 rows per thread);
       // B: 32 consecutive threads copy 32 consecutive columns of one k row (8 k rows per thread).
-      const int m0 = cur_tm * TBM, n0 = cur_tn * BN, k0 = kb * BK;
+      const int m0 = cur_tm * TBM, n0 = cur_tn * TBN, k0 = kb * BK;
       {
         const int a_k = tid & 15, row0 = tid >> 4;
         const int k = k0 + a_k;
@@ -541,12 +547,12 @@ dgemm_dmma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         }
       }
       {
-        const int nn = tid & 127, kk0 = tid >> 7;
+        const int nn = tid % TBN, kk0 = tid / TBN;
         const bool nin = n0 + nn < p.N;
         const double* src = p.B + (long long)(k0 + kk0) * p.ldb + (n0 + nn);
         const uint32_t dst_base = sb + (nn >> 4) * B_BOX_BYTES + ((nn & 1) << 3);
         const int chunk = (nn & 15) >> 1;
-        constexpr int K_STEP = THREADS / 128;
+        constexpr int K_STEP = THREADS / TBN;
 #pragma unroll
         for (int i = 0; i < BK / K_STEP; ++i) {
           const int kk = kk0 + K_STEP * i;
@@ -560,9 +566,9 @@ dgemm_dmma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     if (kb == cur_pf) {
       // TMA staging: the issuing warp's lanes take 4 rows each; generic: one row per thread of the first 128
       if (USE_TMA) {
-        if (warp == (int)(lit % WARPS)) prefetch_c_rows(p.C, p.ldc, p.M, p.N, TBM, cur_tm, cur_tn, lane, 32);
-      } else if (tid < TBM) {
-        prefetch_c_rows(p.C, p.ldc, p.M, p.N, TBM, cur_tm, cur_tn, tid, TBM);
+        if (warp == (int)(lit % WARPS)) prefetch_c_rows(p.C, p.ldc, p.M, p.N, TBM, TBN, cur_tm, cur_tn, lane, 32);
+      } else {
+        prefetch_c_rows(p.C, p.ldc, p.M, p.N, TBM, TBN, cur_tm, cur_tn, tid, THREADS);
       }
     }
     ++lit;
@@ -575,7 +581,7 @@ dgemm_dmma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
 
   for (int i = 0; i < LOOKAHEAD && ok; ++i) ok = issue_next();
 
-  const LaneMap lm = make_lane_map(warp, lane, A_STAGE_BYTES, WTM);
+  const LaneMap lm = make_lane_map(warp, lane, A_STAGE_BYTES, WTM, WARPS_N);
 
   double acc[MT][4][4];  // [mt][nt = 2*np + j][c0..c3]
   uint32_t it = 0;      // k-blocks consumed so far
@@ -718,7 +724,7 @@ dgemm_dmma_ws_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
             }
           }
           if (!__all_sync(0xffffffffu, good)) { ok = false; break; }
-          if (kb == kb_pf) prefetch_c_rows_inline(p.C, p.ldc, p.M, p.N, BM, w.tm, w.tn, lane, 32);
+          if (kb == kb_pf) prefetch_c_rows_inline(p.C, p.ldc, p.M, p.N, BM, BN, w.tm, w.tn, lane, 32);
         } else {
           if (!wait_bounded_inline(empty_bar + 8 * s, ph ^ 1u, abort_flag, p)) { ok = false; break; }
           const int m0 = w.tm * BM, n0 = w.tn * BN, k0 = kb * BK;
@@ -751,7 +757,7 @@ dgemm_dmma_ws_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
             }
           }
           ptx::cp_async_mbar_arrive_noinc(fb);
-          if (kb == kb_pf) prefetch_c_rows_inline(p.C, p.ldc, p.M, p.N, BM, w.tm, w.tn, 32 * pw + lane, BM);
+          if (kb == kb_pf) prefetch_c_rows_inline(p.C, p.ldc, p.M, p.N, BM, BN, w.tm, w.tn, 32 * pw + lane, BM);
         }
       }
     }
@@ -801,12 +807,12 @@ constexpr int REDUCE_THREADS = 256;
 
 template <typename SlotFn>
 __device__ __forceinline__ void reduce_tile(const GemmParams& p, int tm, int tn, int count, SlotFn slot_of) {
-  constexpr int CHUNK_ELEMS = BM * BN / REDUCE_CHUNKS;
-  const int e0 = blockIdx.y * CHUNK_ELEMS;
-  for (int e = e0 + 2 * threadIdx.x; e < e0 + CHUNK_ELEMS; e += 2 * REDUCE_THREADS) {
-    const int r = e / BN, c = e - r * BN;
-    const int row = tm * p.bm + r, col = tn * BN + c;
-    if (r < p.bm && row < p.M && col < p.N) {
+  const int chunk_elems = p.bm * p.bn / REDUCE_CHUNKS;  // a slot holds a bm x bn tile, row-major
+  const int e0 = blockIdx.y * chunk_elems;
+  for (int e = e0 + 2 * threadIdx.x; e < e0 + chunk_elems; e += 2 * REDUCE_THREADS) {
+    const int r = e / p.bn, c = e - r * p.bn;
+    const int row = tm * p.bm + r, col = tn * p.bn + c;
+    if (row < p.M && col < p.N) {
       double2 sum = *reinterpret_cast<const double2*>(p.partial + (long long)slot_of(0) * (BM * BN) + e);
       for (int s = 1; s < count; ++s) {
         const double2 v = *reinterpret_cast<const double2*>(p.partial + (long long)slot_of(s) * (BM * BN) + e);

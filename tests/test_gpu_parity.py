@@ -91,7 +91,7 @@ def test_config1(oracle, integer, variant):
 
 SMALL_SHAPES = [(1, 1, 1), (1, 7, 3), (5, 1, 2), (3, 3, 17), (17, 13, 11), (8, 8, 16), (16, 16, 15),
                 (31, 33, 29), (64, 64, 64), (127, 129, 47), (128, 128, 16), (129, 127, 17), (130, 260, 33),
-                (257, 131, 100), (200, 300, 1)]
+                (257, 131, 100), (200, 300, 1), (1000, 32, 600), (700, 20, 333), (513, 33, 64)]
 
 
 @pytest.mark.parametrize("shape", SMALL_SHAPES)

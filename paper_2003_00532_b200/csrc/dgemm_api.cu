@@ -283,7 +283,7 @@ int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, c
   const int sms = st->sm_count * (bm == 128 ? 1 : 2);  // concurrently resident CTAs (128-row tiles: one per SM)
   const int max_partials = (int)(kWorkspaceBytes / (BM * BN * sizeof(double)));
   p.kblocks = kblocks;
-  p.c_prefetch = (((uintptr_t)C & 15) == 0 && (ldc % 2 == 0)) ? 1 : 0;
+  p.c_prefetch = 1;
   if (dbg_flags & DGEMM_TEST_NO_C_PREFETCH) p.c_prefetch = 0;
   int grid;
   const int forced_split = g_split_k.load();

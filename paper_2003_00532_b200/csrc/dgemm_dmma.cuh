@@ -69,7 +69,7 @@ struct GemmParams {
   int tail_ipc;           // phase 2: k-block iterations per CTA (1 <= tail_ipc <= kblocks)
   int tail_slot_base;     // first workspace slot of the phase-2 partial tiles
   int group_m;            // raster group height in tiles
-  int c_prefetch;         // C rows are 16-byte aligned: prefetch the C tile into L2 before the epilogue
+  int c_prefetch;         // request the C tile into L2 a few k-blocks before its epilogue
   int b_blocked_map;      // map_b is the 3-D view (16 columns, K, N/16): one copy stages the whole B tile
   int zero;               // always 0; masks a data dependency so that the compiler cannot remove it
   const double* A;
@@ -176,11 +176,16 @@ __device__ __noinline__ void fetch_work(const GemmParams& p, int cta, int nctas,
 // Asks L2 for rows r0, r0 + rstep, ... of the C tile (tm, tn) ahead of its epilogue.
 __device__ __forceinline__ void prefetch_c_rows_inline(const double* C, long long ldc, int M, int N, int bm, int bn,
                                                        int tm, int tn, int r0, int rstep) {
-  const int cols = min(bn, N - tn * bn) & ~1;
+  const int cols = min(bn, N - tn * bn);
   if (cols <= 0) return;
   for (int r = r0; r < bm; r += rstep) {
     const int row = tm * bm + r;
-    if (row < M) ptx::prefetch_l2_bulk(C + (long long)row * ldc + (long long)tn * bn, (uint32_t)cols * 8u);
+    if (row < M) {
+      // one request per 128-byte line of the row segment (measured better than one bulk request per row)
+      const double* base = C + (long long)row * ldc + (long long)tn * bn;
+      for (int c = 0; c < cols; c += 16) ptx::prefetch_l2(base + c);
+      ptx::prefetch_l2(base + cols - 1);
+    }
   }
 }
 __device__ __noinline__ void prefetch_c_rows(const double* C, long long ldc, int M, int N, int bm, int bn, int tm,

@@ -164,6 +164,35 @@ def other_shapes(dg, torch, peak_tflops, hbm_gbs):
     return sweep, shapes
 
 
+def ablation_ladder(dg, torch, peak_tflops, n=4096):
+    """The paper walks from a naive nest to its best schedule step by step (Sections 2.3-2.9, Figure
+    'journey'); this is the same walk on the GPU at M=N=K=n: each rung is a variant or test flag of
+    the library. Returns a list of {rung, tflops, frac_peak}."""
+    rungs = [
+        ("naive nest, one thread per C element", dict(variant=dg.DGEMM_VARIANT_NAIVE, n=min(n, 2048))),
+        ("+ smem tiles, register tiles, DMMA; 8-byte cp.async staging, 128x128 tile, 1 CTA/SM",
+         dict(variant=dg.DGEMM_VARIANT_GENERIC, flags=4 | 16)),
+        ("+ TMA staging (2-D copies, 9 per stage), no C prefetch", dict(variant=dg.DGEMM_VARIANT_TMA, flags=4 | 2 | 1)),
+        ("+ one 3-D copy for B, C prefetch into L2", dict(variant=dg.DGEMM_VARIANT_TMA, flags=4)),
+        ("warp-specialised producer warpgroup (setmaxnreg) instead", dict(variant=dg.DGEMM_VARIANT_TMA_WS)),
+        ("32x32 warp tiles, 16 warps", dict(variant=dg.DGEMM_VARIANT_TMA, flags=4 | 8)),
+        ("64x128 tiles, two CTAs per SM (default)", dict(variant=dg.DGEMM_VARIANT_AUTO)),
+    ]
+    out = []
+    for name, cfg in rungs:
+        m = cfg.get("n", n)
+        dg.dgemm_set_variant(cfg["variant"])
+        dg.dgemm_set_test_flags(cfg.get("flags", 0))
+        try:
+            ms = time_shape(dg, torch, m, m, m)
+        finally:
+            dg.dgemm_set_variant(dg.DGEMM_VARIANT_AUTO)
+            dg.dgemm_set_test_flags(0)
+        tf = 2.0 * m ** 3 / ms / 1e9
+        out.append({"rung": name, "n": m, "tflops": round(tf, 2), "frac_peak": round(tf / peak_tflops, 3)})
+    return out
+
+
 def run_reference(args):
     """The oracle on the host cores: each step is a bounded row slab of the same workload."""
     rank = int(os.environ.get("RANK", "0"))
@@ -326,6 +355,7 @@ def run_ours(args):
     }
     if not args.no_sweep:
         line["sweep"], line["other_shapes"] = other_shapes(dg, torch, peak_tflops, hbm_gbs)
+        line["ablation"] = ablation_ladder(dg, torch, peak_tflops)
     print(json.dumps(line), flush=True)
     if distributed:
         dist.destroy_process_group()

@@ -112,6 +112,37 @@ DGEMM_API int dgemm_f64_host(int64_t M, int64_t N, int64_t K,
                    double *C, int64_t ldc);
 
 /*
+ * General form  C = alpha * op(A) * op(B) + beta * C  with op(X) = X or X^T, row-major, FP64,
+ * DEVICE pointers. The paper names the scalars and the transposed / strided operand layouts as
+ * expressible but leaves them out of its study (Section 2.15, "Other questions": it assumes
+ * alpha = beta = 1 and untransposed operands); this entry point is
+ * that extension, built on the same kernels as dgemm_f64.
+ *
+ *   transa  DGEMM_OP_N: A is M x K with lda >= max(1,K).  DGEMM_OP_T: A is stored K x M
+ *           (lda >= max(1,M)) and used as its transpose.
+ *   transb  DGEMM_OP_N: B is K x N with ldb >= max(1,N).  DGEMM_OP_T: B is stored N x K
+ *           (ldb >= max(1,K)) and used as its transpose.
+ *   alpha, beta  passed by value. beta == 0: C is an output only, its old contents (NaN or Inf
+ *           included) are never read. alpha == 0 or K == 0: A and B are never read and the call
+ *           reduces to C = beta * C.
+ *
+ * Arithmetic: each C element receives beta*C_old + alpha*s, s the K-term inner product summed as
+ * in dgemm_f64; alpha = beta = 1 with no transposition gives bit-identical results to dgemm_f64.
+ * A transposed operand is first transposed into device scratch memory owned by the library
+ * (an O(MK) or O(KN) pass before O(MNK) arithmetic; the buffer is kept and reused), so calls
+ * with a transposed or repacked operand on one device must not overlap on the GPU.
+ * Same pointer, alignment, aliasing and error rules as dgemm_f64; an op code other than the two
+ * above returns DGEMM_ERR_BAD_DIM.
+ */
+#define DGEMM_OP_N 0
+#define DGEMM_OP_T 1
+DGEMM_API int dgemm_f64_ex(int transa, int transb, int64_t M, int64_t N, int64_t K,
+                           double alpha, const double *A, int64_t lda,
+                           const double *B, int64_t ldb,
+                           double beta, double *C, int64_t ldc,
+                           void *stream);
+
+/*
  * (No counterpart in the paper: an addition for callers that cannot allocate.)
  *
  * C += A*B like dgemm_f64, with K split over several thread blocks and the partial tiles kept in

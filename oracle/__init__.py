@@ -55,6 +55,9 @@ def _load():
         lib.dgemm_oracle_entries.argtypes = [i64, dp, i64, dp, i64, dp, i64, i64, ip, ip,
                                              ctypes.c_int, dp, ctypes.c_int]
         lib.dgemm_oracle_entries.restype = None
+        lib.dgemm_oracle_general.argtypes = [ctypes.c_int, ctypes.c_int, i64, i64, i64, ctypes.c_double, dp, i64,
+                                             dp, i64, ctypes.c_double, dp, i64, ctypes.c_int]
+        lib.dgemm_oracle_general.restype = None
         lib.dgemm_oracle_max_threads.argtypes = []
         lib.dgemm_oracle_max_threads.restype = ctypes.c_int
         _lib = lib
@@ -118,6 +121,22 @@ def dgemm_oracle(A, B, C, threads: int = 0) -> None:
     keep, args = _check_shapes(A, B, C)
     _load().dgemm_oracle_ikj(*args, int(threads))
     del keep
+
+
+def dgemm_oracle_general(transa: bool, transb: bool, alpha: float, A, B, beta: float, C, threads: int = 0) -> None:
+    """In place ``C = alpha * op(A) @ op(B) + beta * C`` by the definition. ``A`` is given as stored
+    (K x M when ``transa``), likewise ``B`` (N x K when ``transb``)."""
+    a, pa, ar, ac, lda = _mat(A, "A")
+    b, pb, br, bc, ldb = _mat(B, "B")
+    c, pc, M, N, ldc = _mat(C, "C", writable=True)
+    Ma, K = (ac, ar) if transa else (ar, ac)
+    K2, Nb = (bc, br) if transb else (br, bc)
+    if K != K2 or Ma != M or Nb != N:
+        raise ValueError(f"shape mismatch: A {a.shape} (transa={transa}), B {b.shape} (transb={transb}), C {c.shape}")
+    if np.shares_memory(c, a) or np.shares_memory(c, b):
+        raise ValueError("C must not overlap A or B")
+    _load().dgemm_oracle_general(int(bool(transa)), int(bool(transb)), M, N, K, float(alpha), pa, lda, pb, ldb,
+                                 float(beta), pc, ldc, int(threads))
 
 
 def dgemm_oracle_entries(A, B, Cin, ii, jj, absolute: bool = False, threads: int = 0) -> np.ndarray:

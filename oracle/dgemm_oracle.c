@@ -93,6 +93,39 @@ void dgemm_oracle_entries(int64_t K,
     }
 }
 
+void dgemm_oracle_general(int transa, int transb, int64_t M, int64_t N, int64_t K,
+                          double alpha, const double *A, int64_t lda,
+                          const double *B, int64_t ldb,
+                          double beta, double *C, int64_t ldc, int threads)
+{
+    const int product = (alpha != 0.0) && K > 0;
+#ifdef _OPENMP
+    int nt = threads > 0 ? threads : omp_get_max_threads();
+#pragma omp parallel for schedule(static) num_threads(nt)
+#else
+    (void)threads;
+#endif
+    for (int64_t i = 0; i < M; ++i) {
+        for (int64_t j = 0; j < N; ++j) {
+            double s = 0.0;
+            if (product) {
+                for (int64_t k = 0; k < K; ++k) {
+                    const double a = transa ? A[k * lda + i] : A[i * lda + k];
+                    const double b = transb ? B[j * ldb + k] : B[k * ldb + j];
+                    s = s + a * b; /* multiply, then add (no contraction) */
+                }
+            }
+            const double as = product ? alpha * s : 0.0;
+            if (beta == 0.0) {
+                C[i * ldc + j] = as;
+            } else {
+                const double bc = beta * C[i * ldc + j];
+                C[i * ldc + j] = as + bc;
+            }
+        }
+    }
+}
+
 int dgemm_oracle_max_threads(void)
 {
 #ifdef _OPENMP

@@ -62,6 +62,25 @@ void dgemm_oracle_entries(int64_t K,
                           int64_t nsamples, const int64_t *ii, const int64_t *jj,
                           int absolute, double *out, int threads);
 
+/*
+ * General form (Section 2.15, "Other questions": the scalars and the transposed layouts that the
+ * paper names but sets to alpha = beta = 1, no transposition):
+ *
+ *     C[i][j] <- alpha * s_ij + beta * C[i][j],   s_ij = sum_{k} opA(i,k) * opB(k,j)
+ *
+ * opA(i,k) = A[i*lda + k] (transa == 0) or A[k*lda + i] (transa != 0, A stored K x M);
+ * opB(k,j) = B[k*ldb + j] (transb == 0) or B[j*ldb + k] (transb != 0, B stored N x K).
+ * s_ij starts from +0 and takes k ascending with a rounded multiply and a rounded add; then one
+ * multiply by alpha, one by beta, one add. beta == 0: the old C is not read and the result is
+ * alpha * s_ij (a NaN in C does not survive). alpha == 0 or K == 0: A and B are not read.
+ * Loops i, j, k; rows over OpenMP threads. Pinned by tests/test_oracle_pins.py (integer brute
+ * force with transposes, exact rationals, NaN rules, reduction to the plain definition).
+ */
+void dgemm_oracle_general(int transa, int transb, int64_t M, int64_t N, int64_t K,
+                          double alpha, const double *A, int64_t lda,
+                          const double *B, int64_t ldb,
+                          double beta, double *C, int64_t ldc, int threads);
+
 /* Number of OpenMP threads a call with threads <= 0 would use. */
 int dgemm_oracle_max_threads(void);
 

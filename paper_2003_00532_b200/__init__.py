@@ -5,6 +5,8 @@ kernels of ``csrc/``. The library is loaded lazily on first use and its absence 
 """
 from .binding import (  # noqa: F401
     DGEMM_OK,
+    DGEMM_OP_N,
+    DGEMM_OP_T,
     DGEMM_VARIANT_AUTO,
     DGEMM_VARIANT_GENERIC,
     DGEMM_VARIANT_NAIVE,
@@ -13,6 +15,7 @@ from .binding import (  # noqa: F401
     DGEMM_VARIANT_GENERIC_WS,
     DgemmError,
     dgemm_f64,
+    dgemm_f64_ex,
     dgemm_f64_host,
     dgemm_f64_raw,
     dgemm_f64_static_ws,

@@ -29,6 +29,9 @@ DGEMM_ERR_TIMEOUT = -8
 DGEMM_ERR_VARIANT = -9
 DGEMM_ERR_SIZE = -10
 
+DGEMM_OP_N = 0
+DGEMM_OP_T = 1
+
 DGEMM_VARIANT_AUTO = -1
 DGEMM_VARIANT_NAIVE = 0
 DGEMM_VARIANT_TMA = 1
@@ -64,6 +67,9 @@ def load_library() -> ctypes.CDLL:
             lib.dgemm_f64.restype = ctypes.c_int
             lib.dgemm_f64_host.argtypes = [i64, i64, i64, vp, i64, vp, i64, vp, i64]
             lib.dgemm_f64_host.restype = ctypes.c_int
+            lib.dgemm_f64_ex.argtypes = [ctypes.c_int, ctypes.c_int, i64, i64, i64, ctypes.c_double, vp, i64, vp, i64,
+                                         ctypes.c_double, vp, i64, vp]
+            lib.dgemm_f64_ex.restype = ctypes.c_int
             lib.dgemm_f64_static_ws.argtypes = [i64, i64, i64, vp, i64, vp, i64, vp, i64, ctypes.c_int, vp]
             lib.dgemm_f64_static_ws.restype = ctypes.c_int
             lib.dgemm_strerror.argtypes = [ctypes.c_int]
@@ -146,6 +152,30 @@ def dgemm_f64_raw(M, N, K, A_ptr, lda, B_ptr, ldb, C_ptr, ldc, stream: Optional[
     return rc
 
 
+def dgemm_f64_ex(A, B, C, alpha: float = 1.0, beta: float = 1.0, transa: bool = False, transb: bool = False,
+                 stream=None, check: bool = True) -> int:
+    """``C = alpha * op(A) @ op(B) + beta * C`` on the current CUDA device, asynchronously.
+
+    ``A`` and ``B`` are passed as stored: ``A`` is K x M when ``transa`` (used as its transpose),
+    ``B`` is N x K when ``transb``. ``beta == 0`` never reads ``C``; ``alpha == 0`` never reads
+    ``A`` or ``B``. Otherwise as :func:`dgemm_f64`.
+    """
+    pa, ar, ac, lda = _matrix_args(A, "A", True)
+    pb, br, bc, ldb = _matrix_args(B, "B", True)
+    pc, M, N, ldc = _matrix_args(C, "C", True)
+    Ma, K = (ac, ar) if transa else (ar, ac)
+    K2, Nb = (bc, br) if transb else (br, bc)
+    if K != K2 or Ma != M or Nb != N:
+        raise ValueError(f"shape mismatch: A {tuple(A.shape)} (transa={transa}), B {tuple(B.shape)} "
+                         f"(transb={transb}), C {tuple(C.shape)}")
+    rc = load_library().dgemm_f64_ex(DGEMM_OP_T if transa else DGEMM_OP_N, DGEMM_OP_T if transb else DGEMM_OP_N,
+                                     M, N, K, float(alpha), pa, lda, pb, ldb, float(beta), pc, ldc,
+                                     _stream_handle(stream))
+    if check and rc < 0:
+        raise DgemmError(rc, "dgemm_f64_ex")
+    return rc
+
+
 def dgemm_f64_static_ws(A, B, C, split_k: int = 0, stream=None, check: bool = True) -> int:
     """``C += A @ B`` with split-K partial sums kept in the library's fixed device array.
 
@@ -196,7 +226,8 @@ def dgemm_set_split_k(split_k: int) -> int:
 
 
 def dgemm_set_test_flags(flags: int) -> int:
-    """Testing aid: bit 0 disables the L2 prefetch of C, bit 1 the single-copy staging of B."""
+    """Testing aid (bits): 1 no L2 prefetch of C, 2 no single-copy staging of B, 4 128-row tiles,
+    8 32 x 32 warp tiles, 16 no packing pass."""
     rc = load_library().dgemm_set_test_flags(int(flags))
     if rc < 0:
         raise DgemmError(rc, "dgemm_set_test_flags")

@@ -186,66 +186,105 @@ bool ranges_overlap(const void* p, int64_t pbytes, const void* q, int64_t qbytes
 }
 
 // Everything that can be decided without touching the device. Returns 1 for "nothing to do".
+// A is stored (ta ? K x M : M x K), B is stored (tb ? N x K : K x N). `scales_c`: the call may
+// have to rewrite C even without a product (general form with beta != 1); then K == 0 or
+// `no_product` (alpha == 0) returns 2 after checking C alone, A and B stay unexamined.
 int validate(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, const double* B, int64_t ldb,
-             const double* C, int64_t ldc) {
+             const double* C, int64_t ldc, bool ta = false, bool tb = false, bool scales_c = false,
+             bool no_product = false) {
   const int64_t kMaxDim = (int64_t)INT32_MAX - 2 * BM;
   if (M < 0 || N < 0 || K < 0 || M > kMaxDim || N > kMaxDim || K > kMaxDim) return DGEMM_ERR_BAD_DIM;
   if (M == 0 || N == 0) return 1;
-  if (lda < (K > 0 ? K : 1) || ldb < N || ldc < N) return DGEMM_ERR_BAD_LD;
-  if (K == 0) return 1;
+  const int64_t a_rows = ta ? K : M, a_cols = ta ? M : K, b_rows = tb ? N : K, b_cols = tb ? K : N;
+  if (lda < (a_cols > 0 ? a_cols : 1) || ldb < (b_cols > 0 ? b_cols : 1) || ldc < N) return DGEMM_ERR_BAD_LD;
+  if (K == 0 || no_product) {
+    if (!scales_c) return 1;
+    if (!C) return DGEMM_ERR_NULL;
+    if ((uintptr_t)C & 7) return DGEMM_ERR_ALIGN;
+    return 2;
+  }
   if (!A || !B || !C) return DGEMM_ERR_NULL;
   if (((uintptr_t)A | (uintptr_t)B | (uintptr_t)C) & 7) return DGEMM_ERR_ALIGN;
-  const int64_t abytes = ((M - 1) * lda + K) * 8, bbytes = ((K - 1) * ldb + N) * 8, cbytes = ((M - 1) * ldc + N) * 8;
+  const int64_t abytes = ((a_rows - 1) * lda + a_cols) * 8, bbytes = ((b_rows - 1) * ldb + b_cols) * 8,
+                cbytes = ((M - 1) * ldc + N) * 8;
   if (ranges_overlap(C, cbytes, A, abytes) || ranges_overlap(C, cbytes, B, bbytes)) return DGEMM_ERR_ALIAS;
   const int64_t tiles = ((M + BM - 1) / BM) * ((N + BN - 1) / BN);
   if (tiles > (int64_t)INT32_MAX / 512) return DGEMM_ERR_BAD_DIM;
   return DGEMM_OK;
 }
 
+inline unsigned grid_y(int64_t blocks) { return (unsigned)(blocks < 65535 ? blocks : 65535); }
+
+// The scalars and operand forms of the general entry point; the defaults are the paper's C += A B.
+struct GemmForm {
+  bool ta = false, tb = false;  // A is stored K x M / B is stored N x K and used transposed
+  double alpha = 1.0, beta = 1.0;
+};
+
 int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, const double* B, int64_t ldb,
-                double* C, int64_t ldc, cudaStream_t stream) {
+                double* C, int64_t ldc, cudaStream_t stream, const GemmForm& form = GemmForm()) {
   DeviceState* st = nullptr;
   int rc = device_state(&st);
   if (rc != DGEMM_OK) return rc;
 
   int variant = g_variant.load();
-  bool tma_ok = (((uintptr_t)A | (uintptr_t)B) & 15) == 0 && (lda % 2 == 0) && (ldb % 2 == 0);
-  if (variant == DGEMM_VARIANT_AUTO && !tma_ok && !(g_test_flags.load() & DGEMM_TEST_NO_PACKING)) {
-    // Packing pass: worth it when the copy (16 bytes moved per packed element) is small next to
-    // the arithmetic, and the scratch stays moderate.
-    const bool pack_a = ((uintptr_t)A & 15) != 0 || (lda % 2 != 0);
-    const bool pack_b = ((uintptr_t)B & 15) != 0 || (ldb % 2 != 0);
+  {
+    // A transposed operand is always rewritten (row-major, 128-byte aligned rows) into the pack
+    // buffer. An operand that TMA cannot address is repacked there when that is worth it: the copy
+    // (16 bytes moved per packed element) small next to the arithmetic, the scratch moderate.
+    const bool bad_a = !form.ta && (((uintptr_t)A & 15) != 0 || (lda % 2 != 0));
+    const bool bad_b = !form.tb && (((uintptr_t)B & 15) != 0 || (ldb % 2 != 0));
     const int64_t plda = (K + 15) & ~(int64_t)15, pldb = (N + 15) & ~(int64_t)15;  // 128-byte aligned rows
-    const size_t a_bytes = pack_a ? (size_t)M * plda * 8 : 0, b_bytes = pack_b ? (size_t)K * pldb * 8 : 0;
-    const double flop_per_byte = 2.0 * (double)M * (double)N * (double)K / (double)(a_bytes + b_bytes);
-    if (flop_per_byte >= kPackMinFlopPerByte && a_bytes + b_bytes <= kPackMaxBytes) {
+    const size_t a_all = (size_t)M * plda * 8, b_all = (size_t)K * pldb * 8;
+    bool pack_a = form.ta, pack_b = form.tb;
+    if (variant == DGEMM_VARIANT_AUTO && (bad_a || bad_b) && !(g_test_flags.load() & DGEMM_TEST_NO_PACKING)) {
+      const size_t bytes = ((pack_a || bad_a) ? a_all : 0) + ((pack_b || bad_b) ? b_all : 0);
+      const double flop_per_byte = 2.0 * (double)M * (double)N * (double)K / (double)bytes;
+      if (flop_per_byte >= kPackMinFlopPerByte && bytes <= kPackMaxBytes) {
+        pack_a = pack_a || bad_a;
+        pack_b = pack_b || bad_b;
+      }
+    }
+    if (pack_a || pack_b) {
+      const size_t a_bytes = pack_a ? a_all : 0, b_bytes = pack_b ? b_all : 0;
       rc = ensure_pack_buffer(st, a_bytes + b_bytes + 256);
       if (rc != DGEMM_OK) return rc;
       double* pa = st->pack_buf;
       double* pb = reinterpret_cast<double*>(reinterpret_cast<char*>(st->pack_buf) + ((a_bytes + 255) & ~(size_t)255));
       if (pack_a) {
-        dim3 grid((unsigned)((K + 255) / 256), (unsigned)((M + 7) / 8));
-        dgemm_pack_kernel<<<grid, 128, 0, stream>>>(A, lda, (int)M, (int)K, pa, plda);
+        if (form.ta) {  // stored K x M
+          dim3 grid((unsigned)((M + 31) / 32), grid_y((K + 31) / 32));
+          dgemm_transpose_kernel<<<grid, dim3(32, 8), 0, stream>>>(A, lda, (int)K, (int)M, pa, plda);
+        } else {
+          dim3 grid((unsigned)((K + 255) / 256), grid_y((M + 7) / 8));
+          dgemm_pack_kernel<<<grid, 128, 0, stream>>>(A, lda, (int)M, (int)K, pa, plda);
+        }
         g_launches.fetch_add(1);
         A = pa;
         lda = plda;
       }
       if (pack_b) {
-        dim3 grid((unsigned)((N + 255) / 256), (unsigned)((K + 7) / 8));
-        dgemm_pack_kernel<<<grid, 128, 0, stream>>>(B, ldb, (int)K, (int)N, pb, pldb);
+        if (form.tb) {  // stored N x K
+          dim3 grid((unsigned)((K + 31) / 32), grid_y((N + 31) / 32));
+          dgemm_transpose_kernel<<<grid, dim3(32, 8), 0, stream>>>(B, ldb, (int)N, (int)K, pb, pldb);
+        } else {
+          dim3 grid((unsigned)((N + 255) / 256), grid_y((K + 7) / 8));
+          dgemm_pack_kernel<<<grid, 128, 0, stream>>>(B, ldb, (int)K, (int)N, pb, pldb);
+        }
         g_launches.fetch_add(1);
         B = pb;
         ldb = pldb;
       }
       if (cudaGetLastError() != cudaSuccess) return DGEMM_ERR_CUDA;
-      tma_ok = true;
     }
   }
+  const bool tma_ok = (((uintptr_t)A | (uintptr_t)B) & 15) == 0 && (lda % 2 == 0) && (ldb % 2 == 0);
   if (variant == DGEMM_VARIANT_AUTO) variant = tma_ok ? kAutoTma : kAutoGeneric;
   const bool wants_tma = variant == DGEMM_VARIANT_TMA || variant == DGEMM_VARIANT_TMA_WS;
   if (wants_tma && !tma_ok) return DGEMM_ERR_VARIANT;
 
   if (variant == DGEMM_VARIANT_NAIVE) {
+    if (form.alpha != 1.0 || form.beta != 1.0) return DGEMM_ERR_VARIANT;  // the naive nest is C += A B only
     dim3 block(32, 8), grid((unsigned)((N + 31) / 32), (unsigned)((M + 7) / 8));
     dgemm_naive_kernel<<<grid, block, 0, stream>>>((int)M, (int)N, (int)K, A, lda, B, ldb, C, ldc);
     g_launches.fetch_add(1);
@@ -277,6 +316,9 @@ int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, c
   p.wait_limit_ns = kWaitLimitNs;
   p.status = st->status;
   p.group_m = 1024 / bm;  // 1024 rows per raster group
+  p.alpha = form.alpha;
+  p.beta = form.beta;
+  p.load_c = form.beta != 0.0;
 
   const int tiles = p.tiles_m * p.tiles_n;
   const int kblocks = (int)((K + BK - 1) / BK);
@@ -414,6 +456,9 @@ int launch_gemm_static_ws(int64_t M, int64_t N, int64_t K, const double* A, int6
   p.M = (int)M; p.N = (int)N; p.K = (int)K;
   p.bm = BM;
   p.bn = BN;
+  p.alpha = 1.0;
+  p.beta = 1.0;
+  p.load_c = 1;
   p.tiles_m = (int)((M + BM - 1) / BM);
   p.tiles_n = (int)((N + BN - 1) / BN);
   p.A = A; p.B = B; p.C = C;
@@ -495,6 +540,31 @@ int dgemm_f64(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, con
   if (v == 1) return DGEMM_OK;
   if (v != DGEMM_OK) return v;
   return launch_gemm(M, N, K, A, lda, B, ldb, C, ldc, static_cast<cudaStream_t>(stream));
+}
+
+int dgemm_f64_ex(int transa, int transb, int64_t M, int64_t N, int64_t K, double alpha, const double* A, int64_t lda,
+                 const double* B, int64_t ldb, double beta, double* C, int64_t ldc, void* stream) {
+  if ((transa != DGEMM_OP_N && transa != DGEMM_OP_T) || (transb != DGEMM_OP_N && transb != DGEMM_OP_T))
+    return DGEMM_ERR_BAD_DIM;
+  GemmForm form;
+  form.ta = transa == DGEMM_OP_T;
+  form.tb = transb == DGEMM_OP_T;
+  form.alpha = alpha;
+  form.beta = beta;
+  const int v = validate(M, N, K, A, lda, B, ldb, C, ldc, form.ta, form.tb, beta != 1.0, alpha == 0.0);
+  if (v == 1) return DGEMM_OK;
+  if (v < 0) return v;
+  if (v == 2) {  // no product: C = beta * C
+    DeviceState* st = nullptr;
+    const int rc = device_state(&st);
+    if (rc != DGEMM_OK) return rc;
+    const unsigned rows = (unsigned)(M < 4096 ? M : 4096);
+    dgemm_scale_kernel<<<dim3((unsigned)((N + 255) / 256), rows), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        C, ldc, (int)M, (int)N, beta);
+    g_launches.fetch_add(1);
+    return cudaGetLastError() == cudaSuccess ? DGEMM_OK : DGEMM_ERR_CUDA;
+  }
+  return launch_gemm(M, N, K, A, lda, B, ldb, C, ldc, static_cast<cudaStream_t>(stream), form);
 }
 
 int dgemm_f64_static_ws(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, const double* B, int64_t ldb,

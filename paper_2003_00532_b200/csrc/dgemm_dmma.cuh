@@ -72,6 +72,8 @@ struct GemmParams {
   int c_prefetch;         // request the C tile into L2 a few k-blocks before its epilogue
   int b_blocked_map;      // map_b is the 3-D view (16 columns, K, N/16): one copy stages the whole B tile
   int zero;               // always 0; masks a data dependency so that the compiler cannot remove it
+  int load_c;             // 0: beta == 0, the old C is never read (it may hold NaN)
+  double alpha, beta;     // C = beta * C + alpha * (A B); 1, 1 for the paper's C += A B
   const double* A;
   const double* B;
   double* C;
@@ -362,6 +364,14 @@ __device__ __forceinline__ void store_tile(const GemmParams& p, const Work& w, c
                       acc[mt][2 * np][2 * half + 1], acc[mt][2 * np + 1][2 * half + 1]);
         }
   } else {
+    if (p.alpha != 1.0) {
+#pragma unroll
+      for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+        for (int nt = 0; nt < 4; ++nt)
+#pragma unroll
+          for (int e = 0; e < 4; ++e) acc[mt][nt][e] *= p.alpha;
+    }
     const bool interior = (tm * p.bm + p.bm <= p.M) && (tn * p.bn + p.bn <= p.N);
     const bool vec32 = ((reinterpret_cast<uintptr_t>(p.C) & 31) == 0) && ((p.ldc & 3) == 0);
     if (interior && vec32) {
@@ -369,16 +379,27 @@ __device__ __forceinline__ void store_tile(const GemmParams& p, const Work& w, c
 #pragma unroll
       for (int mp = 0; mp < MT / MT_PER_BATCH; ++mp) {
         double cin[MT_PER_BATCH][2][2][4];
+        if (p.load_c) {
 #pragma unroll
-        for (int mq = 0; mq < MT_PER_BATCH; ++mq)
+          for (int mq = 0; mq < MT_PER_BATCH; ++mq)
 #pragma unroll
-          for (int half = 0; half < 2; ++half) {
-            const double* crow = p.C + (long long)(row_base + 16 * (MT_PER_BATCH * mp + mq) + 8 * half) * p.ldc + col_base;
+            for (int half = 0; half < 2; ++half) {
+              const double* crow = p.C + (long long)(row_base + 16 * (MT_PER_BATCH * mp + mq) + 8 * half) * p.ldc + col_base;
 #pragma unroll
-            for (int np = 0; np < 2; ++np)
-              ptx::ldg256(crow + 16 * np, cin[mq][half][np][0], cin[mq][half][np][1], cin[mq][half][np][2],
-                          cin[mq][half][np][3]);
-          }
+              for (int np = 0; np < 2; ++np)
+                ptx::ldg256(crow + 16 * np, cin[mq][half][np][0], cin[mq][half][np][1], cin[mq][half][np][2],
+                            cin[mq][half][np][3]);
+            }
+        } else {
+#pragma unroll
+          for (int mq = 0; mq < MT_PER_BATCH; ++mq)
+#pragma unroll
+            for (int half = 0; half < 2; ++half)
+#pragma unroll
+              for (int np = 0; np < 2; ++np)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) cin[mq][half][np][e] = 0.0;
+        }
 #pragma unroll
         for (int mq = 0; mq < MT_PER_BATCH; ++mq)
 #pragma unroll
@@ -387,10 +408,11 @@ __device__ __forceinline__ void store_tile(const GemmParams& p, const Work& w, c
             double* crow = p.C + (long long)(row_base + 16 * mt + 8 * half) * p.ldc + col_base;
 #pragma unroll
             for (int np = 0; np < 2; ++np)
-              ptx::stg256(crow + 16 * np, cin[mq][half][np][0] + acc[mt][2 * np][2 * half],
-                          cin[mq][half][np][1] + acc[mt][2 * np + 1][2 * half],
-                          cin[mq][half][np][2] + acc[mt][2 * np][2 * half + 1],
-                          cin[mq][half][np][3] + acc[mt][2 * np + 1][2 * half + 1]);
+              // beta == 1: fma(c, 1, acc) rounds once, exactly like c + acc
+              ptx::stg256(crow + 16 * np, fma(cin[mq][half][np][0], p.beta, acc[mt][2 * np][2 * half]),
+                          fma(cin[mq][half][np][1], p.beta, acc[mt][2 * np + 1][2 * half]),
+                          fma(cin[mq][half][np][2], p.beta, acc[mt][2 * np][2 * half + 1]),
+                          fma(cin[mq][half][np][3], p.beta, acc[mt][2 * np + 1][2 * half + 1]));
           }
       }
     } else {
@@ -408,7 +430,7 @@ __device__ __forceinline__ void store_tile(const GemmParams& p, const Work& w, c
                                    acc[mt][2 * np][2 * half + 1], acc[mt][2 * np + 1][2 * half + 1]};
 #pragma unroll
               for (int e = 0; e < 4; ++e)
-                if (col + e < p.N) crow[col + e] += v[e];
+                if (col + e < p.N) crow[col + e] = p.load_c ? fma(crow[col + e], p.beta, v[e]) : v[e];
             }
           }
         }
@@ -825,8 +847,10 @@ __device__ __forceinline__ void reduce_tile(const GemmParams& p, int tm, int tn,
         sum.y += v.y;
       }
       double* dst = p.C + (long long)row * p.ldc + col;
-      dst[0] += sum.x;
-      if (col + 1 < p.N) dst[1] += sum.y;
+      sum.x *= p.alpha;  // exact for alpha == 1
+      sum.y *= p.alpha;
+      dst[0] = p.load_c ? fma(dst[0], p.beta, sum.x) : sum.x;
+      if (col + 1 < p.N) dst[1] = p.load_c ? fma(dst[1], p.beta, sum.y) : sum.y;
     }
   }
 }
@@ -863,18 +887,53 @@ __global__ void dgemm_tail_reduce_kernel(const GemmParams p) {
 __global__ void dgemm_pack_kernel(const double* __restrict__ src, long long ld_src, int rows, int cols,
                                   double* __restrict__ dst, long long ld_dst) {
   const int c = 2 * (blockIdx.x * blockDim.x + threadIdx.x);
-  const int r0 = blockIdx.y * 8;
   if (c >= cols) return;
+  for (int r0 = blockIdx.y * 8; r0 < rows; r0 += gridDim.y * 8) {  // gridDim.y may be capped
 #pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    const int r = r0 + i;
-    if (r < rows) {
-      const double* s = src + (long long)r * ld_src + c;
-      double2 v;
-      v.x = s[0];
-      v.y = (c + 1 < cols) ? s[1] : 0.0;
-      *reinterpret_cast<double2*>(dst + (long long)r * ld_dst + c) = v;
+    for (int i = 0; i < 8; ++i) {
+      const int r = r0 + i;
+      if (r < rows) {
+        const double* s = src + (long long)r * ld_src + c;
+        double2 v;
+        v.x = s[0];
+        v.y = (c + 1 < cols) ? s[1] : 0.0;
+        *reinterpret_cast<double2*>(dst + (long long)r * ld_dst + c) = v;
+      }
     }
+  }
+}
+
+// Out-of-place transpose dst[c][r] = src[r][c] of a rows x cols matrix (32 x 32 tiles through
+// shared memory, both sides coalesced): turns a transposed operand of the general entry point
+// into the row-major layout the tile loaders read. Block (32, 8).
+__global__ void dgemm_transpose_kernel(const double* __restrict__ src, long long ld_src, int rows, int cols,
+                                       double* __restrict__ dst, long long ld_dst) {
+  __shared__ double tile[32][33];
+  const int c0 = blockIdx.x * 32;
+  for (int r0 = blockIdx.y * 32; r0 < rows; r0 += gridDim.y * 32) {  // gridDim.y may be capped
+#pragma unroll
+    for (int i = threadIdx.y; i < 32; i += 8) {
+      const int r = r0 + i, c = c0 + threadIdx.x;
+      if (r < rows && c < cols) tile[i][threadIdx.x] = src[(long long)r * ld_src + c];
+    }
+    __syncthreads();
+#pragma unroll
+    for (int i = threadIdx.y; i < 32; i += 8) {
+      const int c = c0 + i, r = r0 + threadIdx.x;
+      if (r < rows && c < cols) dst[(long long)c * ld_dst + r] = tile[threadIdx.x][i];
+    }
+    __syncthreads();
+  }
+}
+
+// C = beta * C over the logical M x N part (alpha == 0 or K == 0 in the general entry point);
+// beta == 0 stores zeros without reading. One thread per element, grid-stride over rows.
+__global__ void dgemm_scale_kernel(double* C, long long ldc, int M, int N, double beta) {
+  const int j = blockIdx.x * blockDim.x + threadIdx.x;
+  if (j >= N) return;
+  for (int i = blockIdx.y; i < M; i += gridDim.y) {
+    double* c = C + (long long)i * ldc + j;
+    *c = (beta == 0.0) ? 0.0 : *c * beta;
   }
 }
 

@@ -46,6 +46,29 @@ def test_validation_needs_no_device():
     assert h(2, 2, 2, a, 1, b, 2, c, 2) == -2
 
 
+def test_general_form_validation_needs_no_device():
+    x = dg.load_library().dgemm_f64_ex
+    a, b, c = 4096, 8192, 16384
+    N_, T_ = dg.DGEMM_OP_N, dg.DGEMM_OP_T
+    assert x(2, N_, 2, 2, 2, 1.0, a, 2, b, 2, 1.0, c, 2, None) == -1      # unknown op code
+    assert x(N_, -1, 2, 2, 2, 1.0, a, 2, b, 2, 1.0, c, 2, None) == -1
+    # leading dimensions follow the STORED shapes: A^T is K x M (lda >= M), B^T is N x K (ldb >= K)
+    assert x(N_, N_, 5, 3, 2, 1.0, a, 2, b, 3, 1.0, c, 2, None) == -2      # ldc < N
+    assert x(T_, N_, 5, 3, 2, 1.0, a, 4, b, 3, 1.0, c, 3, None) == -2      # lda = 4 < M = 5
+    assert x(N_, T_, 5, 3, 2, 1.0, a, 2, b, 1, 1.0, c, 3, None) == -2      # ldb = 1 < K = 2
+    assert x(T_, T_, 5, 3, 2, 1.0, a, 5, b, 2, 1.0, None, 3, None) == -3
+    # aliasing uses the stored extents: A^T (2 x 5, lda 5) spans 80 bytes
+    assert x(T_, N_, 5, 3, 2, 1.0, a, 5, b, 3, 1.0, a + 72, 3, None) == -5
+    assert x(N_, N_, 5, 3, 2, 1.0, a, 2, b, 3, 1.0, a + 72, 3, None) == -5  # A (5 x 2, lda 2) spans 80 bytes too
+    assert x(N_, N_, 0, 3, 2, 0.0, None, 2, None, 3, 0.0, None, 3, None) == 0  # M = 0
+    # nothing to do at all: beta = 1 and no product
+    assert x(N_, N_, 2, 2, 0, 1.0, None, 1, None, 2, 1.0, None, 2, None) == 0
+    assert x(N_, N_, 2, 2, 2, 0.0, None, 2, None, 2, 1.0, None, 2, None) == 0
+    # C = beta * C needs C (and only C) when there is no product
+    assert x(N_, N_, 2, 2, 2, 0.0, None, 2, None, 2, 0.5, None, 2, None) == -3
+    assert x(N_, N_, 2, 2, 0, 1.0, None, 1, None, 2, 0.0, c + 4, 2, None) == -4
+
+
 @pytest.mark.skipif(torch.cuda.is_available(), reason="only meaningful on a box without a GPU")
 def test_valid_call_without_gpu_fails_loudly():
     A = torch.zeros(4, 4, dtype=torch.float64)

@@ -330,3 +330,108 @@ def test_gflops_formula_matches_paper():
     gf = 2.0 * g["gflops_M"] * g["gflops_N"] * g["gflops_K"] / g["gflops_seconds"] / 1e9
     assert abs(gf - g["gflops_value"]) < 0.005
     assert abs(2 * 4 * 2 * 4.7 - g["peak_gflops"]) < 1e-9
+
+
+# ---- general form: C = alpha * op(A) op(B) + beta * C (Section 2.15, the options the paper sets aside) ----
+
+def _stored(x, trans):
+    """The array as the caller stores it: the transpose (made contiguous) when `trans`."""
+    return np.ascontiguousarray(x.T) if trans else x.copy()
+
+
+@pytest.mark.parametrize("transa,transb", list(itertools.product([False, True], repeat=2)))
+def test_general_integer_brute_force(oracle, transa, transb):
+    """Python int arithmetic, indices written out from the definition, all four operand forms,
+    non-square shapes so that a wrong transpose or leading dimension cannot go unnoticed."""
+    rng = _rng(100 + 2 * transa + transb)
+    M, N, K = 5, 7, 6
+    A, B, C = _ints(rng, (M, K)), _ints(rng, (K, N)), _ints(rng, (M, N))
+    alpha, beta = 3.0, -2.0
+    As, Bs = _stored(A, transa), _stored(B, transb)
+    bufA, vA = _padded(As, As.shape[1] + 3)
+    bufB, vB = _padded(Bs, Bs.shape[1] + 2)
+    bufC, vC = _padded(C, N + 5)
+    oracle.dgemm_oracle_general(transa, transb, alpha, vA, vB, beta, vC)
+    for i in range(M):
+        for j in range(N):
+            s = 0
+            for k in range(K):
+                a = int(As[k, i]) if transa else int(As[i, k])
+                b = int(Bs[j, k]) if transb else int(Bs[k, j])
+                s += a * b
+            assert vC[i, j] == 3 * s - 2 * int(C[i, j]), (i, j)
+    assert np.isnan(bufC[:, N:]).all() and np.isnan(bufA[:, As.shape[1]:]).all()
+
+
+def test_general_reduces_to_plain_definition(oracle):
+    """alpha = beta = 1, no transposition: bit-identical to the paper's nest started from C
+    only when the sum is exact; on real data it differs by the order 'sum then add C', so the
+    check is within the bound, and exact on integers."""
+    rng = _rng(7)
+    M, N, K = 9, 11, 13
+    A, B, C = _ints(rng, (M, K)), _ints(rng, (K, N)), _ints(rng, (M, N))
+    C1, C2 = C.copy(), C.copy()
+    oracle.dgemm_oracle_ijk(A, B, C1)
+    oracle.dgemm_oracle_general(False, False, 1.0, A, B, 1.0, C2)
+    assert np.array_equal(C1, C2)
+    A, B, C = rng.uniform(-1, 1, (M, K)), rng.uniform(-1, 1, (K, N)), rng.uniform(-1, 1, (M, N))
+    C1, C2 = C.copy(), C.copy()
+    oracle.dgemm_oracle_ijk(A, B, C1)
+    oracle.dgemm_oracle_general(False, False, 1.0, A, B, 1.0, C2)
+    bound = oracle.entry_bound(K, np.abs(C) + np.abs(A) @ np.abs(B))
+    assert (np.abs(C1 - C2) <= bound).all()
+
+
+def test_general_exact_rationals_within_bound(oracle):
+    """Against exact rational arithmetic: |fl - exact| <= (K+2) u (|alpha| |A||B| + |beta||C|)."""
+    rng = _rng(11)
+    M, N, K = 4, 5, 17
+    alpha, beta = 0.3, -1.7
+    A, B, C = rng.uniform(-1, 1, (K, M)), rng.uniform(-1, 1, (N, K)), rng.uniform(-1, 1, (M, N))
+    out = C.copy()
+    oracle.dgemm_oracle_general(True, True, alpha, A, B, beta, out)
+    u = Fraction(1, 2 ** 53)
+    for i in range(M):
+        for j in range(N):
+            s = sum(Fraction(A[k, i]) * Fraction(B[j, k]) for k in range(K))
+            exact = Fraction(alpha) * s + Fraction(beta) * Fraction(C[i, j])
+            scale = abs(Fraction(alpha)) * sum(abs(Fraction(A[k, i]) * Fraction(B[j, k])) for k in range(K)) \
+                + abs(Fraction(beta) * Fraction(C[i, j]))
+            assert abs(Fraction(out[i, j]) - exact) <= (K + 2) * u * scale * Fraction(101, 100)
+
+
+def test_general_zero_scalars_do_not_read(oracle):
+    """beta == 0: C is output only (NaN in, finite out). alpha == 0: A and B are not read
+    (NaN operands leave C = beta*C). K == 0 behaves like alpha == 0."""
+    rng = _rng(5)
+    M, N, K = 6, 4, 3
+    A, B = _ints(rng, (M, K)), _ints(rng, (K, N))
+    C = np.full((M, N), np.nan)
+    oracle.dgemm_oracle_general(False, False, 2.0, A, B, 0.0, C)
+    assert np.array_equal(C, 2.0 * (A @ B))
+    C0 = _ints(rng, (M, N))
+    C = C0.copy()
+    oracle.dgemm_oracle_general(False, False, 0.0, np.full((M, K), np.nan), np.full((K, N), np.nan), 3.0, C)
+    assert np.array_equal(C, 3.0 * C0)
+    C = C0.copy()
+    oracle.dgemm_oracle_general(False, False, 5.0, np.zeros((M, 0)), np.zeros((0, N)), -1.0, C)
+    assert np.array_equal(C, -C0)
+    C = np.full((M, N), np.nan)
+    oracle.dgemm_oracle_general(False, False, 0.0, A, B, 0.0, C)
+    assert np.array_equal(C, np.zeros((M, N)))
+
+
+def test_general_transpose_identity(oracle):
+    """(op(A) op(B))^T = op(B)^T op(A)^T: computing C^T with swapped, re-flagged operands gives
+    the transposed result exactly on integer data; checked for every operand form."""
+    rng = _rng(23)
+    M, N, K = 6, 9, 4
+    A, B = _ints(rng, (M, K)), _ints(rng, (K, N))
+    want = A @ B
+    for ta, tb in itertools.product([False, True], repeat=2):
+        C = np.zeros((M, N))
+        oracle.dgemm_oracle_general(ta, tb, 1.0, _stored(A, ta), _stored(B, tb), 0.0, C)
+        assert np.array_equal(C, want), (ta, tb)
+        Ct = np.zeros((N, M))  # C^T = B^T A^T: operand "A" is B^T stored as (N x K) or its transpose
+        oracle.dgemm_oracle_general(not tb, not ta, 1.0, _stored(B, tb), _stored(A, ta), 0.0, Ct)
+        assert np.array_equal(Ct, want.T), (ta, tb)

@@ -2,6 +2,7 @@
 from __future__ import annotations
 
 import os
+import shlex
 import subprocess
 import sys
 
@@ -34,7 +35,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
     """Compile the library if it is missing or older than its sources; returns its path."""
     if force or is_stale():
         tmp = LIB + ".tmp.%d" % os.getpid()
-        cmd = [nvcc_path(), *NVCC_FLAGS, *(["-Xptxas", "-v"] if verbose else []), "-o", tmp, *SOURCES]
+        extra = shlex.split(os.environ.get("DGEMM_NVCC_FLAGS", ""))  # e.g. -D switches for experiments
+        cmd = [nvcc_path(), *NVCC_FLAGS, *extra, *(["-Xptxas", "-v"] if verbose else []), "-o", tmp, *SOURCES]
         res = subprocess.run(cmd, cwd=CSRC, capture_output=True, text=True)
         if verbose or res.returncode != 0:
             sys.stderr.write(res.stdout + res.stderr)

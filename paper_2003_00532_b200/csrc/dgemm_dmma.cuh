@@ -24,6 +24,8 @@
 // share a scheduler with the active producer warp were sporadically corrupted.)
 #pragma once
 
+#include <type_traits>
+
 #include <cstdint>
 #include <cuda.h>
 #include <cuda_runtime.h>
@@ -329,6 +331,107 @@ __device__ __forceinline__ int compute_kblock(const uint8_t* st, const LaneMap& 
   return token;
 }
 
+// ---- the same arithmetic in software-pipelined pieces ---------------------------------------------
+// One half k-block (8 k values) of fragments for a warp tile of 16*MT rows x 32 columns: 48
+// registers for MT = 4. The default kernel keeps two of them, so that the loads of the next half
+// (and, across a k-block boundary, the barrier test before them) are issued ahead of the MMAs of
+// the current half and a warp can feed the FP64 pipe without a gap at the boundary.
+template <int MT>
+struct Frags {
+  double2 alo[MT], ahi[MT], bf[2][2];
+};
+
+template <int I, int N, typename F>
+__device__ __forceinline__ void static_for(F&& f) {
+  if constexpr (I < N) {
+    f(std::integral_constant<int, I>());
+    static_for<I + 1, N>(f);
+  }
+}
+
+// `stage` is the shared-memory address of the stage; H selects k = 8H .. 8H+7.
+template <int H, int MT>
+__device__ __forceinline__ void load_frags(Frags<MT>& f, uint32_t stage, const LaneMap& m) {
+  const uint32_t a = stage + m.a_off[H];
+  static_for<0, MT>([&](auto mt) {
+    ptx::lds128_off<mt.value * 2048>(a, f.alo[mt.value].x, f.alo[mt.value].y);
+    ptx::lds128_off<mt.value * 2048 + 1024>(a, f.ahi[mt.value].x, f.ahi[mt.value].y);
+  });
+  static_for<0, 2>([&](auto np) {
+    ptx::lds128_off<np.value * B_BOX_BYTES>(stage + m.b_off[H][0], f.bf[np.value][0].x, f.bf[np.value][0].y);
+    ptx::lds128_off<np.value * B_BOX_BYTES>(stage + m.b_off[H][1], f.bf[np.value][1].x, f.bf[np.value][1].y);
+  });
+}
+
+// A value that depends on every register of `f` (see release_stage).
+template <int MT>
+__device__ __forceinline__ int frag_token(const Frags<MT>& f) {
+  int token = 0;
+#pragma unroll
+  for (int mt = 0; mt < MT; ++mt)
+    token ^= __double2loint(f.alo[mt].x) ^ __double2hiint(f.alo[mt].y) ^ __double2loint(f.ahi[mt].x) ^ __double2hiint(f.ahi[mt].y);
+#pragma unroll
+  for (int np = 0; np < 2; ++np)
+    token ^= __double2loint(f.bf[np][0].x) ^ __double2hiint(f.bf[np][0].y) ^ __double2loint(f.bf[np][1].x) ^ __double2hiint(f.bf[np][1].y);
+  return token;
+}
+
+// The MMAs of row blocks [MT0, MT1) of one half k-block.
+template <int MT0, int MT1, int MT>
+__device__ __forceinline__ void mma_frags(double (&acc)[MT][4][4], const Frags<MT>& f) {
+#pragma unroll
+  for (int mt = MT0; mt < MT1; ++mt)
+#pragma unroll
+    for (int np = 0; np < 2; ++np) {
+      ptx::dmma_m8n8k4(acc[mt][2 * np + 0][0], acc[mt][2 * np + 0][1], f.alo[mt].x, f.bf[np][0].x);
+      ptx::dmma_m8n8k4(acc[mt][2 * np + 0][2], acc[mt][2 * np + 0][3], f.ahi[mt].x, f.bf[np][0].x);
+      ptx::dmma_m8n8k4(acc[mt][2 * np + 1][0], acc[mt][2 * np + 1][1], f.alo[mt].x, f.bf[np][0].y);
+      ptx::dmma_m8n8k4(acc[mt][2 * np + 1][2], acc[mt][2 * np + 1][3], f.ahi[mt].x, f.bf[np][0].y);
+      ptx::dmma_m8n8k4(acc[mt][2 * np + 0][0], acc[mt][2 * np + 0][1], f.alo[mt].y, f.bf[np][1].x);
+      ptx::dmma_m8n8k4(acc[mt][2 * np + 0][2], acc[mt][2 * np + 0][3], f.ahi[mt].y, f.bf[np][1].x);
+      ptx::dmma_m8n8k4(acc[mt][2 * np + 1][0], acc[mt][2 * np + 1][1], f.alo[mt].y, f.bf[np][1].y);
+      ptx::dmma_m8n8k4(acc[mt][2 * np + 1][2], acc[mt][2 * np + 1][3], f.ahi[mt].y, f.bf[np][1].y);
+    }
+}
+
+// One of the 12 fragment loads of a half k-block, numbered so that the ones needed first by the
+// MMAs come first: 0..3 = B (np, b), then per row block alo, ahi.
+template <int H, int I, int MT>
+__device__ __forceinline__ void load_frag_piece(Frags<MT>& f, uint32_t stage, const LaneMap& m) {
+  if constexpr (I < 4) {
+    constexpr int np = I >> 1, b = I & 1;
+    ptx::lds128_off<np * B_BOX_BYTES>(stage + m.b_off[H][b], f.bf[np][b].x, f.bf[np][b].y);
+  } else if constexpr (I < 4 + 2 * MT) {
+    constexpr int mt = (I - 4) >> 1;
+    if constexpr (((I - 4) & 1) == 0) ptx::lds128_off<mt * 2048>(stage + m.a_off[H], f.alo[mt].x, f.alo[mt].y);
+    else ptx::lds128_off<mt * 2048 + 1024>(stage + m.a_off[H], f.ahi[mt].x, f.ahi[mt].y);
+  }
+}
+
+// The MMAs of row blocks [MT0, MT1) of the half k-block in `cur`, with the loads [L0, L1) of half
+// HN (into `nxt`, from `stage_n`) spread between them, so that the loads neither arrive in a burst
+// nor wait behind the arithmetic.
+template <int MT0, int MT1, int HN, int L0, int L1, int MT>
+__device__ __forceinline__ void mma_frags_loading(double (&acc)[MT][4][4], const Frags<MT>& cur, Frags<MT>& nxt,
+                                                  uint32_t stage_n, const LaneMap& m) {
+  constexpr int GROUPS = 2 * (MT1 - MT0);
+  static_for<0, GROUPS>([&](auto gi) {
+    constexpr int g = gi.value;
+    constexpr int mt = MT0 + g / 2, np = g % 2;
+    // loads [lo, hi) of this group: an even share of L1 - L0
+    constexpr int lo = L0 + (L1 - L0) * g / GROUPS, hi = L0 + (L1 - L0) * (g + 1) / GROUPS;
+    static_for<lo, hi>([&](auto li) { load_frag_piece<HN, li.value>(nxt, stage_n, m); });
+    ptx::dmma_m8n8k4(acc[mt][2 * np + 0][0], acc[mt][2 * np + 0][1], cur.alo[mt].x, cur.bf[np][0].x);
+    ptx::dmma_m8n8k4(acc[mt][2 * np + 0][2], acc[mt][2 * np + 0][3], cur.ahi[mt].x, cur.bf[np][0].x);
+    ptx::dmma_m8n8k4(acc[mt][2 * np + 1][0], acc[mt][2 * np + 1][1], cur.alo[mt].x, cur.bf[np][0].y);
+    ptx::dmma_m8n8k4(acc[mt][2 * np + 1][2], acc[mt][2 * np + 1][3], cur.ahi[mt].x, cur.bf[np][0].y);
+    ptx::dmma_m8n8k4(acc[mt][2 * np + 0][0], acc[mt][2 * np + 0][1], cur.alo[mt].y, cur.bf[np][1].x);
+    ptx::dmma_m8n8k4(acc[mt][2 * np + 0][2], acc[mt][2 * np + 0][3], cur.ahi[mt].y, cur.bf[np][1].x);
+    ptx::dmma_m8n8k4(acc[mt][2 * np + 1][0], acc[mt][2 * np + 1][1], cur.alo[mt].y, cur.bf[np][1].y);
+    ptx::dmma_m8n8k4(acc[mt][2 * np + 1][2], acc[mt][2 * np + 1][3], cur.ahi[mt].y, cur.bf[np][1].y);
+  });
+}
+
 // Releases a stage after compute_kblock. The arrive must not take effect before all of this
 // warp's fragment loads have been served: otherwise the refill can overwrite rows that a load
 // still queued behind the arithmetic has yet to read (observed as sporadically wrong rows of the
@@ -537,21 +640,25 @@ dgemm_dmma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     const uint32_t fb = full_bar + 8 * s;
     const int kb = cur_kb;
     if (USE_TMA) {
-      int good = 1;
-      if (warp == (int)(lit % WARPS) && lane == 0) {
-        if (wait_bounded<false>(empty_bar + 8 * s, ph ^ 1u, abort_flag, p)) {
-          ptx::mbar_arrive_expect_tx(fb, STAGE_BYTES);
-          ptx::tma_load_2d(sa, &map_a, kb * BK, cur_tm * TBM, fb);
-          if (p.b_blocked_map) {
-            ptx::tma_load_3d(sb, &map_b, 0, kb * BK, cur_tn * (TBN / 16), fb);
+      // Only the issuing warp learns at once that its wait gave up; the other warps see the abort
+      // flag in their own next wait. (A vote in every warp on every k-block costs 0.5 % at 8192^3.)
+      if (warp == (int)(lit % WARPS)) {
+        int good = 1;
+        if (lane == 0) {
+          if (wait_bounded<false>(empty_bar + 8 * s, ph ^ 1u, abort_flag, p)) {
+            ptx::mbar_arrive_expect_tx(fb, STAGE_BYTES);
+            ptx::tma_load_2d(sa, &map_a, kb * BK, cur_tm * TBM, fb);
+            if (p.b_blocked_map) {
+              ptx::tma_load_3d(sb, &map_b, 0, kb * BK, cur_tn * (TBN / 16), fb);
+            } else {
+              tma_load_b_boxes(sb, &map_b, cur_tn * TBN, kb * BK, fb, TBN / 16);
+            }
           } else {
-            tma_load_b_boxes(sb, &map_b, cur_tn * TBN, kb * BK, fb, TBN / 16);
+            good = 0;
           }
-        } else {
-          good = 0;
         }
+        if (!__all_sync(0xffffffffu, good)) return false;
       }
-      if (!__all_sync(0xffffffffu, good)) return false;
     } else {
       if (!wait_bounded<false>(empty_bar + 8 * s, ph ^ 1u, abort_flag, p)) return false;
       // 8-byte asynchronous copies with zero fill outside the matrices; any alignment, any leading
@@ -812,12 +919,32 @@ dgemm_dmma_ws_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
         for (int nt = 0; nt < 4; ++nt)
 #pragma unroll
           for (int c = 0; c < 4; ++c) acc[mt][nt][c] = 0.0;
+      Frags<4> f0, f1;
+      {
+        const uint32_t s = it % STAGES;
+        if (!wait_bounded_inline(full_bar + 8 * s, (it / STAGES) & 1u, abort_flag, p)) { ok = false; break; }
+        load_frags<0>(f0, tiles_u32 + s * STAGE_BYTES, lm);
+      }
       for (int kb = w.kb0; kb < w.kb1; ++kb, ++it) {
         const uint32_t s = it % STAGES;
-        const uint32_t ph = (it / STAGES) & 1u;
-        if (!wait_bounded_inline(full_bar + 8 * s, ph, abort_flag, p)) { ok = false; break; }
-        const int token = compute_kblock<true>(tiles + s * STAGE_BYTES, lm, acc);
-        release_stage(empty_bar + 8 * s, token, lane, p.zero);
+        const uint32_t s1 = (it + 1) % STAGES;
+        const uint32_t ph1 = ((it + 1) / STAGES) & 1u;
+        const bool more = kb + 1 < w.kb1;
+        const bool ready = more && ptx::mbar_test_wait(full_bar + 8 * s1, ph1);
+        int token = frag_token(f0);
+        mma_frags_loading<0, 4, 1, 0, 12>(acc, f0, f1, tiles_u32 + s * STAGE_BYTES, lm);
+        token ^= frag_token(f1);
+        token = __reduce_xor_sync(0xffffffffu, token);
+        if (more) {
+          if (!ready && !wait_bounded_inline(full_bar + 8 * s1, ph1, abort_flag, p)) { ok = false; break; }
+          mma_frags_loading<0, 2, 0, 0, 6>(acc, f1, f0, tiles_u32 + s1 * STAGE_BYTES, lm);
+          if (lane == 0) ptx::mbar_arrive(empty_bar + 8 * s + (uint32_t)(token & p.zero));
+          mma_frags_loading<2, 4, 0, 6, 12>(acc, f1, f0, tiles_u32 + s1 * STAGE_BYTES, lm);
+        } else {
+          mma_frags<0, 2>(acc, f1);
+          if (lane == 0) ptx::mbar_arrive(empty_bar + 8 * s + (uint32_t)(token & p.zero));
+          mma_frags<2, 4>(acc, f1);
+        }
       }
       if (!ok) break;
       store_tile<1>(p, w, lm, acc);

@@ -133,6 +133,12 @@ __device__ __forceinline__ void lds128(uint32_t addr, double& x, double& y) {
   asm volatile("ld.shared.v2.f64 {%0, %1}, [%2];" : "=d"(x), "=d"(y) : "r"(addr));
 }
 
+// Same with a compile-time byte offset folded into the instruction.
+template <int OFF>
+__device__ __forceinline__ void lds128_off(uint32_t addr, double& x, double& y) {
+  asm volatile("ld.shared.v2.f64 {%0, %1}, [%2+%3];" : "=d"(x), "=d"(y) : "r"(addr), "n"(OFF));
+}
+
 // ---- FP64 tensor-core MMA: D(16x8) += A(16x8, row) * B(8x8, col) ---------------------------------
 // Lane l: g = l/4, t = l%4. a0=A[g][t] a1=A[g+8][t] a2=A[g][t+4] a3=A[g+8][t+4];
 // b0=B[t][g] b1=B[t+4][g]; c0,c1=C[g][2t,2t+1]; c2,c3=C[g+8][2t,2t+1].

@@ -22,8 +22,8 @@ using namespace dgemm;
 constexpr int kMaxDevices = 64;
 constexpr size_t kWorkspaceBytes = 640ull * BM * BN * sizeof(double);  // 80 MiB: up to 640 partial-tile slots
 constexpr unsigned long long kWaitLimitNs = 4000000000ull;            // 4 s per device-side wait
-constexpr int kAutoTma = DGEMM_VARIANT_TMA;          // what DGEMM_VARIANT_AUTO picks for aligned operands
-constexpr int kAutoGeneric = DGEMM_VARIANT_GENERIC;  // ... and for unaligned ones
+constexpr int kAutoGeneric = DGEMM_VARIANT_GENERIC;  // what DGEMM_VARIANT_AUTO picks for operands TMA cannot address
+constexpr int kAutoWsMinKblocks = 16;                // aligned operands: warp-specialised kernel from K = 256 up
 constexpr double kPackMinFlopPerByte = 64.0;       // pack unaligned operands only if the copy is this cheap
 constexpr size_t kPackMaxBytes = 2ull << 30;       // ... and the packed copies fit in 2 GiB
 constexpr int64_t kHostBlockRows = 1024;             // dgemm_f64_host: rows of A and C per pipelined block
@@ -279,7 +279,19 @@ int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, c
     }
   }
   const bool tma_ok = (((uintptr_t)A | (uintptr_t)B) & 15) == 0 && (lda % 2 == 0) && (ldb % 2 == 0);
-  if (variant == DGEMM_VARIANT_AUTO) variant = tma_ok ? kAutoTma : kAutoGeneric;
+  if (variant == DGEMM_VARIANT_AUTO) {
+    if (!tma_ok) {
+      variant = kAutoGeneric;
+    } else {
+      // The warp-specialised kernel (128 x 128 tiles, one CTA per SM, software-pipelined consumers)
+      // has the fastest main loop. The inline kernel with 64-row tiles and two CTAs per SM hides
+      // the C round trip of short-K problems better, wastes less on an M just above a multiple of
+      // 64, and has the narrow tile for N <= 32.
+      const int64_t pad128 = (M + 127) / 128 * 128, pad64 = (M + 63) / 64 * 64;
+      const bool ws = N > 32 && (K + BK - 1) / BK >= kAutoWsMinKblocks && (double)pad128 <= 1.03 * (double)pad64;
+      variant = ws ? DGEMM_VARIANT_TMA_WS : DGEMM_VARIANT_TMA;
+    }
+  }
   const bool wants_tma = variant == DGEMM_VARIANT_TMA || variant == DGEMM_VARIANT_TMA_WS;
   if (wants_tma && !tma_ok) return DGEMM_ERR_VARIANT;
 

@@ -34,7 +34,7 @@ FMA_PER_CLK_SM = 64  # FP64 DMMA issue rate measured by dgemm_fp64_peak_probe (6
 
 # DRAM traffic of one 8192^3 launch of the dominant kernel (dram__bytes_read.sum +
 # dram__bytes_write.sum of one ncu capture, see profiles/); None until a capture exists for a size.
-NCU_DRAM_BYTES_PER_LAUNCH = {8192: 9123730944 + 548454656, 4096: 1258445000 + 140287488}
+NCU_DRAM_BYTES_PER_LAUNCH = {8192: 7976930816 + 556108032, 4096: 1110870000 + 139895552}
 
 
 def _load_measured_peaks():
@@ -318,7 +318,7 @@ def run_ours(args):
     roofline = {
         "bound": "tensor", "achieved": achieved, "peak": peak_tflops, "unit": "TFLOP/s",
         "frac": achieved / peak_tflops, "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get(n) if not args.shape else None,
-        "kernel": "dgemm_dmma_kernel<true, 64, 64> (TMA staging, 64 x 128 tiles, two CTAs per SM)",
+        "kernel": "dgemm_dmma_ws_kernel<true> (TMA staging, 128 x 128 tiles, 8 consumer warps + producer warpgroup per SM)",
         "peak_source": (f"FP64 DMMA issue rate {FMA_PER_CLK_SM} FMA/clk/SM (measured by the register-only probe) x "
                         f"{SM_COUNT_B200} SMs x 2 x sm_max_mhz {sm_max_mhz:.0f} "
                         f"({'MEASURED_PEAKS.json' if peaks else 'fallback 1965'}); MEASURED_PEAKS has no FP64 entry"),

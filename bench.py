@@ -174,9 +174,10 @@ def ablation_ladder(dg, torch, peak_tflops, n=4096):
          dict(variant=dg.DGEMM_VARIANT_GENERIC, flags=4 | 16)),
         ("+ TMA staging (2-D copies, 9 per stage), no C prefetch", dict(variant=dg.DGEMM_VARIANT_TMA, flags=4 | 2 | 1)),
         ("+ one 3-D copy for B, C prefetch into L2", dict(variant=dg.DGEMM_VARIANT_TMA, flags=4)),
-        ("warp-specialised producer warpgroup (setmaxnreg) instead", dict(variant=dg.DGEMM_VARIANT_TMA_WS)),
         ("32x32 warp tiles, 16 warps", dict(variant=dg.DGEMM_VARIANT_TMA, flags=4 | 8)),
-        ("64x128 tiles, two CTAs per SM (default)", dict(variant=dg.DGEMM_VARIANT_AUTO)),
+        ("64x128 tiles, two CTAs per SM", dict(variant=dg.DGEMM_VARIANT_TMA)),
+        ("producer warpgroup (setmaxnreg), software-pipelined consumers (default at this size)",
+         dict(variant=dg.DGEMM_VARIANT_AUTO)),
     ]
     out = []
     for name, cfg in rungs:

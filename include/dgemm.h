@@ -49,7 +49,8 @@ enum {
                                 A and B base pointers and even lda, ldb                          */
   DGEMM_VARIANT_GENERIC = 2, /* same pipeline, tiles staged by 8-byte asynchronous copies; any
                                 8-byte aligned operands and any leading dimensions               */
-  DGEMM_VARIANT_TMA_WS = 3,     /* as TMA, with a separate producer warpgroup (warp-specialised)  */
+  DGEMM_VARIANT_TMA_WS = 3,     /* as TMA, with a separate producer warpgroup (warp-specialised) and a
+                                   software-pipelined consumer loop                              */
   DGEMM_VARIANT_GENERIC_WS = 4, /* as GENERIC, with a separate producer warpgroup                 */
   DGEMM_VARIANT_COUNT = 5
 };
@@ -203,7 +204,9 @@ enum {
   DGEMM_TEST_NO_BLOCKED_B = 2,  /* stage B with eight 2-D copies per stage instead of one 3-D copy */
   DGEMM_TEST_TALL_TILES = 4,    /* 128-row tiles, one CTA per SM, instead of 64-row tiles, two per SM */
   DGEMM_TEST_SMALL_WARP_TILES = 8, /* 32 x 32 warp tiles (twice the warps) instead of 64 x 32           */
-  DGEMM_TEST_NO_PACKING = 16    /* never pack unaligned operands: always use the generic staging      */
+  DGEMM_TEST_NO_PACKING = 16,   /* never pack unaligned operands: always use the generic staging      */
+  DGEMM_TEST_WS_TWO_CTAS = 32   /* DGEMM_VARIANT_TMA_WS: 64-row tiles, two CTAs per SM, at any K (the
+                                   library itself uses that form only for K < 256)                 */
 };
 DGEMM_API int dgemm_set_test_flags(int flags);
 

@@ -227,7 +227,7 @@ def dgemm_set_split_k(split_k: int) -> int:
 
 def dgemm_set_test_flags(flags: int) -> int:
     """Testing aid (bits): 1 no L2 prefetch of C, 2 no single-copy staging of B, 4 128-row tiles,
-    8 32 x 32 warp tiles, 16 no packing pass."""
+    8 32 x 32 warp tiles, 16 no packing pass, 32 two-CTA form of the warp-specialised kernel."""
     rc = load_library().dgemm_set_test_flags(int(flags))
     if rc < 0:
         raise DgemmError(rc, "dgemm_set_test_flags")

@@ -23,7 +23,7 @@ constexpr int kMaxDevices = 64;
 constexpr size_t kWorkspaceBytes = 640ull * BM * BN * sizeof(double);  // 80 MiB: up to 640 partial-tile slots
 constexpr unsigned long long kWaitLimitNs = 4000000000ull;            // 4 s per device-side wait
 constexpr int kAutoGeneric = DGEMM_VARIANT_GENERIC;  // what DGEMM_VARIANT_AUTO picks for operands TMA cannot address
-constexpr int kAutoWsMinKblocks = 16;                // aligned operands: warp-specialised kernel from K = 256 up
+constexpr int kAutoWsMinKblocks = 16;                // warp-specialised kernel: 128-row tiles from K = 256 up, 64-row below
 constexpr double kPackMinFlopPerByte = 64.0;       // pack unaligned operands only if the copy is this cheap
 constexpr size_t kPackMaxBytes = 2ull << 30;       // ... and the packed copies fit in 2 GiB
 constexpr int64_t kHostBlockRows = 1024;             // dgemm_f64_host: rows of A and C per pipelined block
@@ -106,7 +106,9 @@ int device_state(DeviceState** out) {
         configure_tile_kernel<true, 64, 32>(&occ[6]) && configure_tile_kernel<false, 64, 32>(&occ[7]) &&
         configure_tile_kernel<true, 256, 64, 32>(&occ[8]) && configure_tile_kernel<false, 256, 64, 32>(&occ[9]) &&
         cudaFuncSetAttribute(dgemm_dmma_ws_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) == cudaSuccess &&
-        cudaFuncSetAttribute(dgemm_dmma_ws_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) == cudaSuccess;
+        cudaFuncSetAttribute(dgemm_dmma_ws_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) == cudaSuccess &&
+        cudaFuncSetAttribute(dgemm_dmma_ws_kernel<true, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, WsCfg<64>::SMEM_BYTES_) == cudaSuccess &&
+        cudaFuncSetAttribute(dgemm_dmma_ws_kernel<true, 64>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared) == cudaSuccess;
     if (!attr_ok) return DGEMM_ERR_CUDA;
     // the 64-row kernels are meant to run two CTAs per SM; use them only where the device really fits two
     st.two_ctas_ok = occ[4] >= 2 && occ[5] >= 2 && occ[6] >= 2 && occ[7] >= 2 && occ[8] >= 2 && occ[9] >= 2;
@@ -287,8 +289,10 @@ int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, c
       // has the fastest main loop. The inline kernel with 64-row tiles and two CTAs per SM hides
       // the C round trip of short-K problems better, wastes less on an M just above a multiple of
       // 64, and has the narrow tile for N <= 32.
+      // For K < 256 the warp-specialised kernel itself runs 64-row tiles, two CTAs per SM (below).
       const int64_t pad128 = (M + 127) / 128 * 128, pad64 = (M + 63) / 64 * 64;
-      const bool ws = N > 32 && (K + BK - 1) / BK >= kAutoWsMinKblocks && (double)pad128 <= 1.03 * (double)pad64;
+      const bool short_k = (K + BK - 1) / BK < kAutoWsMinKblocks;
+      const bool ws = N > 32 && (short_k || (double)pad128 <= 1.03 * (double)pad64);
       variant = ws ? DGEMM_VARIANT_TMA_WS : DGEMM_VARIANT_TMA;
     }
   }
@@ -311,7 +315,10 @@ int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, c
   const bool generic_large = !wants_tma && tiles128 >= 4 * (int64_t)st->sm_count;
   // narrow problems (N <= 32) use a 256 x 32 tile: four warps stacked in M, no arithmetic on unused columns
   const bool narrow = N <= 32 && !ws_variant && !(dbg_flags & (DGEMM_TEST_TALL_TILES | DGEMM_TEST_SMALL_WARP_TILES)) && st->two_ctas_ok;
-  const int bm = narrow ? 256 : (ws_variant || generic_large || (dbg_flags & DGEMM_TEST_TALL_TILES) || !st->two_ctas_ok) ? 128 : 64;
+  // warp-specialised with 64-row tiles, two CTAs per SM: the second CTA hides the C round trip of short-K problems
+  const bool ws64 = variant == DGEMM_VARIANT_TMA_WS && st->two_ctas_ok &&
+                    ((K + BK - 1) / BK < kAutoWsMinKblocks || (dbg_flags & DGEMM_TEST_WS_TWO_CTAS));
+  const int bm = narrow ? 256 : ws64 ? 64 : (ws_variant || generic_large || (dbg_flags & DGEMM_TEST_TALL_TILES) || !st->two_ctas_ok) ? 128 : 64;
   const int bn = narrow ? 32 : BN;
 
   const int wtm = (dbg_flags & DGEMM_TEST_SMALL_WARP_TILES) ? 32 : 64;  // rows of a warp tile
@@ -394,7 +401,9 @@ int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, c
     if (!make_map(&map_a, A, M, K, lda, BK, bm)) return DGEMM_ERR_CUDA;
     p.b_blocked_map = (!(dbg_flags & DGEMM_TEST_NO_BLOCKED_B) && N % 16 == 0 && make_blocked_map(&map_b, B, K, N, ldb, BK, bn / 16)) ? 1 : 0;
     if (!p.b_blocked_map && !make_map(&map_b, B, K, N, ldb, 16, BK)) return DGEMM_ERR_CUDA;
-    if (variant == DGEMM_VARIANT_TMA_WS)
+    if (ws64)
+      dgemm_dmma_ws_kernel<true, 64><<<grid, WsCfg<64>::THREADS_, WsCfg<64>::SMEM_BYTES_, stream>>>(map_a, map_b, p);
+    else if (variant == DGEMM_VARIANT_TMA_WS)
       dgemm_dmma_ws_kernel<true><<<grid, WS_THREADS, SMEM_BYTES, stream>>>(map_a, map_b, p);
     else
       launch_default_kernel<true>(bm, wtm, grid, stream, map_a, map_b, p);
@@ -706,7 +715,7 @@ int dgemm_set_variant(int variant) {
 }
 
 int dgemm_set_test_flags(int flags) {
-  if (flags < 0 || flags > (DGEMM_TEST_NO_C_PREFETCH | DGEMM_TEST_NO_BLOCKED_B | DGEMM_TEST_TALL_TILES | DGEMM_TEST_SMALL_WARP_TILES | DGEMM_TEST_NO_PACKING)) return DGEMM_ERR_VARIANT;
+  if (flags < 0 || flags > (DGEMM_TEST_NO_C_PREFETCH | DGEMM_TEST_NO_BLOCKED_B | DGEMM_TEST_TALL_TILES | DGEMM_TEST_SMALL_WARP_TILES | DGEMM_TEST_NO_PACKING | DGEMM_TEST_WS_TWO_CTAS)) return DGEMM_ERR_VARIANT;
   g_test_flags.store(flags);
   return DGEMM_OK;
 }

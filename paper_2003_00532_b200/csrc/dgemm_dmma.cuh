@@ -780,10 +780,29 @@ constexpr int WS_THREADS = (WARPS + WS_PRODUCER_WARPS) * 32;
 constexpr int WS_CONSUMER_REGS = 232;
 constexpr int WS_PRODUCER_REGS = 40;
 
-template <bool USE_TMA>
-__global__ void __launch_bounds__(WS_THREADS, 1)
+template <int TBM>
+struct WsCfg {
+  static constexpr int CONSUMER_WARPS = TBM / 16;  // a (TBM / 64) x 4 grid of 64 x 32 warp tiles
+  static constexpr int THREADS_ = (CONSUMER_WARPS + WS_PRODUCER_WARPS) * 32;
+  static constexpr int CTAS_PER_SM = TBM == 128 ? 1 : 2;
+  static constexpr int A_BYTES = TBM * BK * 8;
+  static constexpr int STAGE_BYTES_ = A_BYTES + B_STAGE_BYTES;
+  static constexpr int STAGES_ = TBM == 128 ? 6 : 4;
+  static constexpr int SMEM_BYTES_ = STAGES_ * STAGE_BYTES_ + SMEM_ALIGN + 2048;
+  // register pool = THREADS_ x registers at launch (168 or 128): consumers x 232 + 128 x producers
+  static constexpr int PRODUCER_REGS = TBM == 128 ? WS_PRODUCER_REGS : 24;
+};
+
+template <bool USE_TMA, int TBM = BM>
+__global__ void __launch_bounds__(WsCfg<TBM>::THREADS_, WsCfg<TBM>::CTAS_PER_SM)
 dgemm_dmma_ws_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                      const __grid_constant__ GemmParams p) {
+  static_assert(USE_TMA || TBM == 128, "generic staging needs the 128-row producer layout and 40 producer registers");
+  constexpr int STAGES = WsCfg<TBM>::STAGES_;
+  constexpr int WARPS = WsCfg<TBM>::CONSUMER_WARPS;
+  constexpr int A_STAGE_BYTES = WsCfg<TBM>::A_BYTES;
+  constexpr int STAGE_BYTES = WsCfg<TBM>::STAGE_BYTES_;
+  constexpr int WS_THREADS = WsCfg<TBM>::THREADS_;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = ptx::smem_u32(smem_raw);
   const uint32_t pad = (SMEM_ALIGN - (raw & (SMEM_ALIGN - 1))) & (SMEM_ALIGN - 1);
@@ -817,7 +836,7 @@ dgemm_dmma_ws_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
 
   if (warp >= WARPS) {
     // ------------------------------------------------------------------ producer warpgroup
-    ptx::setmaxnreg_dec<WS_PRODUCER_REGS>();
+    ptx::setmaxnreg_dec<WsCfg<TBM>::PRODUCER_REGS>();
     const int pw = warp - WARPS;
     const bool active = USE_TMA ? (pw == 0) : true;
     if (USE_TMA && pw == 0 && lane == 0) {
@@ -847,7 +866,7 @@ dgemm_dmma_ws_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
           if (lane == 0) {
             if (wait_bounded_inline(empty_bar + 8 * s, ph ^ 1u, abort_flag, p)) {
               ptx::mbar_arrive_expect_tx(fb, STAGE_BYTES);
-              ptx::tma_load_2d(sa, &map_a, kb * BK, w.tm * BM, fb);
+              ptx::tma_load_2d(sa, &map_a, kb * BK, w.tm * TBM, fb);
               if (p.b_blocked_map) {
                 ptx::tma_load_3d(sb, &map_b, 0, kb * BK, w.tn * (BN / 16), fb);
               } else {
@@ -858,7 +877,7 @@ dgemm_dmma_ws_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
             }
           }
           if (!__all_sync(0xffffffffu, good)) { ok = false; break; }
-          if (kb == kb_pf) prefetch_c_rows_inline(p.C, p.ldc, p.M, p.N, BM, BN, w.tm, w.tn, lane, 32);
+          if (kb == kb_pf) prefetch_c_rows_inline(p.C, p.ldc, p.M, p.N, TBM, BN, w.tm, w.tn, lane, 32);
         } else {
           if (!wait_bounded_inline(empty_bar + 8 * s, ph ^ 1u, abort_flag, p)) { ok = false; break; }
           const int m0 = w.tm * BM, n0 = w.tn * BN, k0 = kb * BK;
@@ -910,7 +929,7 @@ dgemm_dmma_ws_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
   } else {
     // ------------------------------------------------------------------ consumer warps
     ptx::setmaxnreg_inc<WS_CONSUMER_REGS>();
-    const LaneMap lm = make_lane_map(warp, lane);
+    const LaneMap lm = make_lane_map(warp, lane, A_STAGE_BYTES, 64, 4);
     double acc[4][4][4];
     for (int idx = 0; ok && get_work(p, cta, nctas, idx, w); ++idx) {
 #pragma unroll

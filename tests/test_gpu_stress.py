@@ -25,7 +25,7 @@ def rank_k_case(oracle):
     return prob, torch.from_numpy(want)
 
 
-@pytest.mark.parametrize("flags", [3, 1, 2, 0, 7, 4, 8, 12, 15])
+@pytest.mark.parametrize("flags", [3, 1, 2, 0, 7, 4, 8, 12, 15, 32])
 @pytest.mark.parametrize("variant", [dg.DGEMM_VARIANT_TMA, dg.DGEMM_VARIANT_GENERIC, dg.DGEMM_VARIANT_TMA_WS,
                                      dg.DGEMM_VARIANT_GENERIC_WS])
 def test_rank_k_repeated_runs_bit_exact(rank_k_case, flags, variant):
@@ -54,9 +54,24 @@ def test_rank_k_repeated_runs_bit_exact(rank_k_case, flags, variant):
 
 
 @pytest.mark.parametrize("n", [2304, 2560, 3072])
-def test_square_repeated_runs_bit_exact(oracle, n):
+@pytest.mark.parametrize("kernel", ["auto", "inline", "ws_two_ctas"])
+def test_square_repeated_runs_bit_exact(oracle, n, kernel):
     """Sizes with a partial last wave (stream-K tail), repeated; exact against the oracle's entries
-    on sampled positions and against the first run everywhere."""
+    on sampled positions and against the first run everywhere. `auto` is the warp-specialised
+    kernel with 128-row tiles at these sizes; the other two are its 64-row form and the inline kernel."""
+    if kernel == "inline":
+        dg.dgemm_set_variant(dg.DGEMM_VARIANT_TMA)
+    elif kernel == "ws_two_ctas":
+        dg.dgemm_set_variant(dg.DGEMM_VARIANT_TMA_WS)
+        dg.dgemm_set_test_flags(32)
+    try:
+        _square_repeated(oracle, n)
+    finally:
+        dg.dgemm_set_variant(dg.DGEMM_VARIANT_AUTO)
+        dg.dgemm_set_test_flags(0)
+
+
+def _square_repeated(oracle, n):
     prob = wl.make_problem(n, n, n, seed=n, integer=True)
     A, B, C0 = prob.A_buf.cuda(), prob.B_buf.cuda(), prob.C_buf.cuda()
     ii, jj = wl.sample_indices(n, n, 4096, seed=n)

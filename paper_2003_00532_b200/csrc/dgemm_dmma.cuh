@@ -73,7 +73,6 @@ struct GemmParams {
   int group_m;            // raster group height in tiles
   int c_prefetch;         // request the C tile into L2 a few k-blocks before its epilogue
   int b_blocked_map;      // map_b is the 3-D view (16 columns, K, N/16): one copy stages the whole B tile
-  int zero;               // always 0; masks a data dependency so that the compiler cannot remove it
   int load_c;             // 0: beta == 0, the old C is never read (it may hold NaN)
   double alpha, beta;     // C = beta * C + alpha * (A B); 1, 1 for the paper's C += A B
   const double* A;
@@ -284,10 +283,9 @@ __device__ __forceinline__ LaneMap make_lane_map(int warp, int lane, int a_stage
 }
 
 // The arithmetic of one k-block (16 k values) on one stage: acc += A_tile * B_tile for this warp's
-// 64 x 32 tile. Returns a token that depends on every fragment register this lane loaded.
+// 64 x 32 tile.
 template <bool M16 = false, int MT = 4>
-__device__ __forceinline__ int compute_kblock(const uint8_t* st, const LaneMap& m, double (&acc)[MT][4][4]) {
-  int token = 0;
+__device__ __forceinline__ void compute_kblock(const uint8_t* st, const LaneMap& m, double (&acc)[MT][4][4]) {
 #pragma unroll
   for (int h = 0; h < 2; ++h) {
     double2 alo[MT], ahi[MT], bf[2][2];
@@ -301,12 +299,6 @@ __device__ __forceinline__ int compute_kblock(const uint8_t* st, const LaneMap& 
 #pragma unroll
       for (int b = 0; b < 2; ++b)
         bf[np][b] = *reinterpret_cast<const double2*>(st + m.b_off[h][b] + np * B_BOX_BYTES);
-#pragma unroll
-    for (int mt = 0; mt < MT; ++mt)
-      token ^= __double2loint(alo[mt].x) ^ __double2hiint(alo[mt].y) ^ __double2loint(ahi[mt].x) ^ __double2hiint(ahi[mt].y);
-#pragma unroll
-    for (int np = 0; np < 2; ++np)
-      token ^= __double2loint(bf[np][0].x) ^ __double2hiint(bf[np][0].y) ^ __double2loint(bf[np][1].x) ^ __double2hiint(bf[np][1].y);
     // Eight k values per block as two k4 steps (x: k = 8h + 2t, y: k = 8h + 2t + 1) of the
     // m8n8k4 shape; rows g (alo) and g + 8 (ahi) are separate 8 x 8 tiles.
 #pragma unroll
@@ -328,7 +320,6 @@ __device__ __forceinline__ int compute_kblock(const uint8_t* st, const LaneMap& 
         ptx::dmma_m8n8k4(acc[mt][2 * np + 1][2], acc[mt][2 * np + 1][3], ahi[mt].y, bf[np][1].y);
       }
   }
-  return token;
 }
 
 // ---- the same arithmetic in software-pipelined pieces ---------------------------------------------
@@ -361,19 +352,6 @@ __device__ __forceinline__ void load_frags(Frags<MT>& f, uint32_t stage, const L
     ptx::lds128_off<np.value * B_BOX_BYTES>(stage + m.b_off[H][0], f.bf[np.value][0].x, f.bf[np.value][0].y);
     ptx::lds128_off<np.value * B_BOX_BYTES>(stage + m.b_off[H][1], f.bf[np.value][1].x, f.bf[np.value][1].y);
   });
-}
-
-// A value that depends on every register of `f` (see release_stage).
-template <int MT>
-__device__ __forceinline__ int frag_token(const Frags<MT>& f) {
-  int token = 0;
-#pragma unroll
-  for (int mt = 0; mt < MT; ++mt)
-    token ^= __double2loint(f.alo[mt].x) ^ __double2hiint(f.alo[mt].y) ^ __double2loint(f.ahi[mt].x) ^ __double2hiint(f.ahi[mt].y);
-#pragma unroll
-  for (int np = 0; np < 2; ++np)
-    token ^= __double2loint(f.bf[np][0].x) ^ __double2hiint(f.bf[np][0].y) ^ __double2loint(f.bf[np][1].x) ^ __double2hiint(f.bf[np][1].y);
-  return token;
 }
 
 // The MMAs of row blocks [MT0, MT1) of one half k-block.
@@ -432,16 +410,17 @@ __device__ __forceinline__ void mma_frags_loading(double (&acc)[MT][4][4], const
   });
 }
 
-// Releases a stage after compute_kblock. The arrive must not take effect before all of this
-// warp's fragment loads have been served: otherwise the refill can overwrite rows that a load
-// still queued behind the arithmetic has yet to read (observed as sporadically wrong rows of the
-// last-loaded A fragments in the slowest warp, cured by delaying the arrive). Program order alone
-// does not guarantee it, so the arrive is made data-dependent on the loaded registers of all 32
-// lanes: a warp-wide reduction of the per-lane tokens, masked with a zero the compiler cannot
-// see, is added to the barrier address.
-__device__ __forceinline__ void release_stage(uint32_t empty_bar_s, int token, int lane, int zero) {
-  token = __reduce_xor_sync(0xffffffffu, token);
-  if (lane == 0) ptx::mbar_arrive(empty_bar_s + (uint32_t)(token & zero));
+// Releases a stage: one arrival per warp on its `empty` mbarrier, after which the producer may
+// refill it with TMA copies. Those copies write through the asynchronous proxy while the fragment
+// loads above read through the generic proxy, and an mbarrier arrive alone does not order the two:
+// without the proxy fence the refill could overwrite rows that a fragment load had yet to read
+// (observed as sporadically wrong 8-row blocks, most often on K = 64 tiles; reproduced by
+// tests/test_gpu_stress.py with a plain arrive). Every lane fences its own loads, the warp
+// synchronises, lane 0 arrives.
+__device__ __forceinline__ void release_stage(uint32_t empty_bar_s, int lane) {
+  ptx::fence_proxy_async();
+  __syncwarp();
+  if (lane == 0) ptx::mbar_arrive(empty_bar_s);
 }
 
 // Epilogue of one work item: adds the accumulators to the C tile (or stores them as a partial tile
@@ -743,8 +722,8 @@ dgemm_dmma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
       const uint32_t s = it % STAGES;
       const uint32_t ph = (it / STAGES) & 1u;
       if (!wait_bounded(full_bar + 8 * s, ph, abort_flag, p)) { ok = false; break; }
-      const int token = compute_kblock<false, MT>(tiles + s * STAGE_BYTES, lm, acc);
-      release_stage(empty_bar + 8 * s, token, lane, p.zero);
+      compute_kblock<false, MT>(tiles + s * STAGE_BYTES, lm, acc);
+      release_stage(empty_bar + 8 * s, lane);
       // keep the load stream LOOKAHEAD k-blocks ahead: refill the stage released two k-blocks ago
       if (!issue_next()) { ok = false; break; }
     }
@@ -950,18 +929,15 @@ dgemm_dmma_ws_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
         const uint32_t ph1 = ((it + 1) / STAGES) & 1u;
         const bool more = kb + 1 < w.kb1;
         const bool ready = more && ptx::mbar_test_wait(full_bar + 8 * s1, ph1);
-        int token = frag_token(f0);
         mma_frags_loading<0, 4, 1, 0, 12>(acc, f0, f1, tiles_u32 + s * STAGE_BYTES, lm);
-        token ^= frag_token(f1);
-        token = __reduce_xor_sync(0xffffffffu, token);
         if (more) {
           if (!ready && !wait_bounded_inline(full_bar + 8 * s1, ph1, abort_flag, p)) { ok = false; break; }
           mma_frags_loading<0, 2, 0, 0, 6>(acc, f1, f0, tiles_u32 + s1 * STAGE_BYTES, lm);
-          if (lane == 0) ptx::mbar_arrive(empty_bar + 8 * s + (uint32_t)(token & p.zero));
+          release_stage(empty_bar + 8 * s, lane);
           mma_frags_loading<2, 4, 0, 6, 12>(acc, f1, f0, tiles_u32 + s1 * STAGE_BYTES, lm);
         } else {
           mma_frags<0, 2>(acc, f1);
-          if (lane == 0) ptx::mbar_arrive(empty_bar + 8 * s + (uint32_t)(token & p.zero));
+          release_stage(empty_bar + 8 * s, lane);
           mma_frags<2, 4>(acc, f1);
         }
       }

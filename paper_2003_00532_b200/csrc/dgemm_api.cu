@@ -292,7 +292,9 @@ int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, c
       // For K < 256 the warp-specialised kernel itself runs 64-row tiles, two CTAs per SM (below).
       const int64_t pad128 = (M + 127) / 128 * 128, pad64 = (M + 63) / 64 * 64;
       const bool short_k = (K + BK - 1) / BK < kAutoWsMinKblocks;
-      const bool ws = N > 32 && (short_k || (double)pad128 <= 1.03 * (double)pad64);
+      const int64_t tiles128 = (pad128 / 128) * ((N + BN - 1) / BN);
+      // (a handful of tiles: the inline kernel starts faster, 14 against 18 us at 256^3)
+      const bool ws = N > 32 && tiles128 >= 16 && (short_k || (double)pad128 <= 1.03 * (double)pad64);
       variant = ws ? DGEMM_VARIANT_TMA_WS : DGEMM_VARIANT_TMA;
     }
   }

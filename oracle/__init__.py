@@ -58,6 +58,12 @@ def _load():
         lib.dgemm_oracle_general.argtypes = [ctypes.c_int, ctypes.c_int, i64, i64, i64, ctypes.c_double, dp, i64,
                                              dp, i64, ctypes.c_double, dp, i64, ctypes.c_int]
         lib.dgemm_oracle_general.restype = None
+        lib.sgemm_oracle_ijk.argtypes = [i64, i64, i64, dp, i64, dp, i64, dp, i64]
+        lib.sgemm_oracle_ijk.restype = None
+        lib.sgemm_oracle_ikj.argtypes = [i64, i64, i64, dp, i64, dp, i64, dp, i64, ctypes.c_int]
+        lib.sgemm_oracle_ikj.restype = None
+        lib.sgemm_oracle_entries.argtypes = [i64, dp, i64, dp, i64, dp, i64, i64, ip, ip, dp, ctypes.c_int]
+        lib.sgemm_oracle_entries.restype = None
         lib.dgemm_oracle_max_threads.argtypes = []
         lib.dgemm_oracle_max_threads.restype = ctypes.c_int
         _lib = lib
@@ -77,24 +83,25 @@ def _as_np(x) -> np.ndarray:
     return np.asarray(x)
 
 
-def _mat(x, name: str, writable: bool = False):
+def _mat(x, name: str, writable: bool = False, dtype=np.float64):
     """Return (array, pointer, rows, cols, ld) for a 2-D float64 matrix with unit column stride.
 
     A row stride larger than the column count expresses a padded leading dimension (a view
     ``buf[:, :cols]`` of a wider buffer); the padding is never touched.
     """
     a = _as_np(x)
-    if a.dtype != np.float64 or a.ndim != 2:
-        raise TypeError(f"{name}: need a 2-D float64 array, got {a.dtype} ndim={a.ndim}")
+    esz = np.dtype(dtype).itemsize  # float32 matrices for the sgemm functions
+    if a.dtype != dtype or a.ndim != 2:
+        raise TypeError(f"{name}: need a 2-D {np.dtype(dtype).name} array, got {a.dtype} ndim={a.ndim}")
     rows, cols = a.shape
     if cols > 0 and rows > 0:
-        if a.strides[1] != 8:
+        if a.strides[1] != esz:
             raise ValueError(f"{name}: columns must be contiguous (row-major)")
-        if rows > 1 and (a.strides[0] % 8 != 0 or a.strides[0] < 8 * cols):
+        if rows > 1 and (a.strides[0] % esz != 0 or a.strides[0] < esz * cols):
             raise ValueError(f"{name}: bad row stride {a.strides[0]}")
     if writable and not a.flags.writeable:
         raise ValueError(f"{name}: must be writable")
-    ld = a.strides[0] // 8 if rows > 1 and cols > 0 else max(cols, 1)
+    ld = a.strides[0] // esz if rows > 1 and cols > 0 else max(cols, 1)
     return a, a.ctypes.data, rows, cols, max(ld, 1)
 
 
@@ -165,6 +172,58 @@ def dgemm_oracle_entries(A, B, Cin, ii, jj, absolute: bool = False, threads: int
                                  jj.ctypes.data, int(bool(absolute)), out.ctypes.data, int(threads))
     del a, b, c
     return out
+
+
+def _check_shapes_f32(A, B, C):
+    a, pa, M, K, lda = _mat(A, "A", dtype=np.float32)
+    b, pb, K2, N, ldb = _mat(B, "B", dtype=np.float32)
+    c, pc, M2, N2, ldc = _mat(C, "C", writable=True, dtype=np.float32)
+    if K != K2 or M != M2 or N != N2:
+        raise ValueError(f"shape mismatch: A {a.shape}, B {b.shape}, C {c.shape}")
+    if np.shares_memory(c, a) or np.shares_memory(c, b):
+        raise ValueError("C must not overlap A or B")
+    return (a, b, c), (M, N, K, pa, lda, pb, ldb, pc, ldc)
+
+
+def sgemm_oracle_ijk(A, B, C) -> None:
+    """In place ``C += A @ B`` in binary32 by the definition (loops i, j, k; multiply then add)."""
+    keep, args = _check_shapes_f32(A, B, C)
+    _load().sgemm_oracle_ijk(*args)
+    del keep
+
+
+def sgemm_oracle(A, B, C, threads: int = 0) -> None:
+    """In place binary32 ``C += A @ B``, loops i, k, j over OpenMP rows; bit-identical to the definition."""
+    keep, args = _check_shapes_f32(A, B, C)
+    _load().sgemm_oracle_ikj(*args, int(threads))
+    del keep
+
+
+def sgemm_oracle_entries(A, B, Cin, ii, jj, threads: int = 0) -> np.ndarray:
+    """Binary32 entries ``(Cin + A @ B)[ii[s], jj[s]]`` recomputed one by one (``Cin`` may be None)."""
+    a, pa, M, K, lda = _mat(A, "A", dtype=np.float32)
+    b, pb, K2, N, ldb = _mat(B, "B", dtype=np.float32)
+    if K != K2:
+        raise ValueError("shape mismatch")
+    pc, ldc, c = None, 1, None
+    if Cin is not None:
+        c, pc, M2, N2, ldc = _mat(Cin, "Cin", dtype=np.float32)
+        if (M2, N2) != (M, N):
+            raise ValueError("shape mismatch")
+    ii = np.ascontiguousarray(ii, dtype=np.int64)
+    jj = np.ascontiguousarray(jj, dtype=np.int64)
+    if ii.shape != jj.shape or ii.ndim != 1:
+        raise ValueError("ii, jj must be 1-D of equal length")
+    if ii.size and (ii.min() < 0 or ii.max() >= M or jj.min() < 0 or jj.max() >= N):
+        raise IndexError("sample index out of range")
+    out = np.empty(ii.size, dtype=np.float32)
+    _load().sgemm_oracle_entries(K, pa, lda, pb, ldb, pc, ldc, ii.size, ii.ctypes.data, jj.ctypes.data,
+                                 out.ctypes.data, int(threads))
+    del a, b, c
+    return out
+
+
+U32 = 2.0 ** -24  # unit roundoff of binary32
 
 
 def abs_product(A, B, Cin=None, threads: int = 0) -> np.ndarray:

@@ -126,6 +126,71 @@ void dgemm_oracle_general(int transa, int transb, int64_t M, int64_t N, int64_t 
     }
 }
 
+void sgemm_oracle_ijk(int64_t M, int64_t N, int64_t K,
+                      const float *A, int64_t lda,
+                      const float *B, int64_t ldb,
+                      float *C, int64_t ldc)
+{
+    for (int64_t i = 0; i < M; ++i) {
+        for (int64_t j = 0; j < N; ++j) {
+            float c = C[i * ldc + j];
+            for (int64_t k = 0; k < K; ++k) {
+                const float prod = A[i * lda + k] * B[k * ldb + j]; /* rounded to binary32 */
+                c = c + prod;                                       /* rounded to binary32 */
+            }
+            C[i * ldc + j] = c;
+        }
+    }
+}
+
+void sgemm_oracle_ikj(int64_t M, int64_t N, int64_t K,
+                      const float *A, int64_t lda,
+                      const float *B, int64_t ldb,
+                      float *C, int64_t ldc, int threads)
+{
+#ifdef _OPENMP
+    int nt = threads > 0 ? threads : omp_get_max_threads();
+#pragma omp parallel for schedule(static) num_threads(nt)
+#else
+    (void)threads;
+#endif
+    for (int64_t i = 0; i < M; ++i) {
+        float *c = C + i * ldc;
+        for (int64_t k = 0; k < K; ++k) {
+            const float a = A[i * lda + k];
+            const float *b = B + k * ldb;
+            for (int64_t j = 0; j < N; ++j) {
+                const float prod = a * b[j];
+                c[j] = c[j] + prod;
+            }
+        }
+    }
+}
+
+void sgemm_oracle_entries(int64_t K,
+                          const float *A, int64_t lda,
+                          const float *B, int64_t ldb,
+                          const float *Cin, int64_t ldc,
+                          int64_t nsamples, const int64_t *ii, const int64_t *jj,
+                          float *out, int threads)
+{
+#ifdef _OPENMP
+    int nt = threads > 0 ? threads : omp_get_max_threads();
+#pragma omp parallel for schedule(static) num_threads(nt)
+#else
+    (void)threads;
+#endif
+    for (int64_t s = 0; s < nsamples; ++s) {
+        const int64_t i = ii[s], j = jj[s];
+        float c = Cin ? Cin[i * ldc + j] : 0.0f;
+        for (int64_t k = 0; k < K; ++k) {
+            const float prod = A[i * lda + k] * B[k * ldb + j];
+            c = c + prod;
+        }
+        out[s] = c;
+    }
+}
+
 int dgemm_oracle_max_threads(void)
 {
 #ifdef _OPENMP

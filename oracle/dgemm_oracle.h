@@ -81,6 +81,32 @@ void dgemm_oracle_general(int transa, int transb, int64_t M, int64_t N, int64_t 
                           const double *B, int64_t ldb,
                           double beta, double *C, int64_t ldc, int threads);
 
+/*
+ * Single precision (Section 2.13 "SGEMM performance": the same nest with f64 replaced by f32).
+ * C[i][j] <- C[i][j] + sum_k A[i][k]*B[k][j] evaluated in IEEE binary32: for each (i,j), k
+ * ascending, c = c + a*b with a rounded binary32 multiply followed by a rounded binary32 add (no
+ * contraction, no wider intermediate). sgemm_oracle_ijk is the definition (loops i, j, k, single
+ * thread); sgemm_oracle_ikj is the interchange over OpenMP rows, bit-identical to it.
+ * sgemm_oracle_entries recomputes sampled entries the same way (Cin may be NULL = +0).
+ * Pinned by tests/test_oracle_pins.py: all-ones input (1 + K), int brute force, exact rationals
+ * within the binary32 bound, a case where binary64 accumulation would give another answer,
+ * loop-order identity, padding canaries.
+ */
+void sgemm_oracle_ijk(int64_t M, int64_t N, int64_t K,
+                      const float *A, int64_t lda,
+                      const float *B, int64_t ldb,
+                      float *C, int64_t ldc);
+void sgemm_oracle_ikj(int64_t M, int64_t N, int64_t K,
+                      const float *A, int64_t lda,
+                      const float *B, int64_t ldb,
+                      float *C, int64_t ldc, int threads);
+void sgemm_oracle_entries(int64_t K,
+                          const float *A, int64_t lda,
+                          const float *B, int64_t ldb,
+                          const float *Cin, int64_t ldc,
+                          int64_t nsamples, const int64_t *ii, const int64_t *jj,
+                          float *out, int threads);
+
 /* Number of OpenMP threads a call with threads <= 0 would use. */
 int dgemm_oracle_max_threads(void);
 

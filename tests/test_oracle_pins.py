@@ -435,3 +435,88 @@ def test_general_transpose_identity(oracle):
         Ct = np.zeros((N, M))  # C^T = B^T A^T: operand "A" is B^T stored as (N x K) or its transpose
         oracle.dgemm_oracle_general(not tb, not ta, 1.0, _stored(B, tb), _stored(A, ta), 0.0, Ct)
         assert np.array_equal(Ct, want.T), (ta, tb)
+
+
+# ---- binary32 oracle (Section 2.13: the same nest on f32) ------------------------------------------
+
+def _f32(x):
+    return np.ascontiguousarray(x, dtype=np.float32)
+
+
+def test_sgemm_all_ones_driver(oracle):
+    """The paper's driver initialises every matrix to one: each entry becomes 1 + K, exact in
+    binary32 for K < 2^24."""
+    M, N, K = 33, 40, 2048
+    A, B, C = np.ones((M, K), np.float32), np.ones((K, N), np.float32), np.ones((M, N), np.float32)
+    oracle.sgemm_oracle_ijk(A, B, C)
+    assert (C == np.float32(1 + K)).all()
+    C2 = np.ones((M, N), np.float32)
+    oracle.sgemm_oracle(A, B, C2)
+    assert np.array_equal(C, C2)
+
+
+def test_sgemm_integer_brute_force_and_padding(oracle):
+    rng = _rng(41)
+    M, N, K = 5, 7, 6
+    A, B, C = _f32(_ints(rng, (M, K))), _f32(_ints(rng, (K, N))), _f32(_ints(rng, (M, N)))
+    bufA = np.full((M, K + 3), np.nan, np.float32); bufA[:, :K] = A
+    bufB = np.full((K, N + 2), np.nan, np.float32); bufB[:, :N] = B
+    bufC = np.full((M, N + 5), np.nan, np.float32); bufC[:, :N] = C
+    oracle.sgemm_oracle_ijk(bufA[:, :K], bufB[:, :N], bufC[:, :N])
+    for i in range(M):
+        for j in range(N):
+            assert bufC[i, j] == int(C[i, j]) + sum(int(A[i, k]) * int(B[k, j]) for k in range(K))
+    assert np.isnan(bufC[:, N:]).all()
+
+
+def test_sgemm_arithmetic_is_binary32(oracle):
+    """2^24 + 1 is not a binary32 number: adding K ones to 2^24 one at a time stays at 2^24 in
+    binary32, while any wider accumulator would give 2^24 + K. A product that needs rounding
+    pins the multiply as well: (1 + 2^-12)^2 rounds to 1 + 2^-11 in binary32."""
+    K = 8
+    A, B = np.ones((1, K), np.float32), np.ones((K, 1), np.float32)
+    C = np.full((1, 1), 2.0 ** 24, np.float32)
+    oracle.sgemm_oracle_ijk(A, B, C)
+    assert C[0, 0] == np.float32(2.0 ** 24)
+    x = np.float32(1 + 2.0 ** -12)
+    C = np.zeros((1, 1), np.float32)
+    oracle.sgemm_oracle_ijk(np.array([[x]], np.float32), np.array([[x]], np.float32), C)
+    assert C[0, 0] == np.float32(1 + 2.0 ** -11)
+    out = oracle.sgemm_oracle_entries(np.array([[x]], np.float32), np.array([[x]], np.float32), None, [0], [0])
+    assert out[0] == np.float32(1 + 2.0 ** -11)
+
+
+def test_sgemm_exact_rationals_within_bound(oracle):
+    """|fl32 - exact| <= K u32 (|C| + |A||B|) (1 + small), u32 = 2^-24, against exact rationals."""
+    rng = _rng(43)
+    M, N, K = 4, 5, 33
+    A, B, C = _f32(rng.uniform(-1, 1, (M, K))), _f32(rng.uniform(-1, 1, (K, N))), _f32(rng.uniform(-1, 1, (M, N)))
+    out = C.copy()
+    oracle.sgemm_oracle(A, B, out)
+    u = Fraction(1, 2 ** 24)
+    worst = Fraction(0)
+    for i in range(M):
+        for j in range(N):
+            exact = Fraction(float(C[i, j])) + sum(Fraction(float(A[i, k])) * Fraction(float(B[k, j])) for k in range(K))
+            scale = abs(Fraction(float(C[i, j]))) + sum(abs(Fraction(float(A[i, k])) * Fraction(float(B[k, j]))) for k in range(K))
+            err = abs(Fraction(float(out[i, j])) - exact)
+            assert err <= (K + 1) * u * scale * Fraction(101, 100)
+            worst = max(worst, err / (u * scale))
+    assert worst > Fraction(1, 100)  # binary32 rounding really happened (a binary64 result would be ~1e-9 here)
+
+
+def test_sgemm_loop_orders_and_entries_agree(oracle):
+    rng = _rng(47)
+    M, N, K = 37, 29, 101
+    A, B, C = _f32(rng.uniform(-1, 1, (M, K))), _f32(rng.uniform(-1, 1, (K, N))), _f32(rng.uniform(-1, 1, (M, N)))
+    C1, C2 = C.copy(), C.copy()
+    oracle.sgemm_oracle_ijk(A, B, C1)
+    oracle.sgemm_oracle(A, B, C2, threads=3)
+    assert C1.tobytes() == C2.tobytes()
+    ii, jj = rng.integers(0, M, 50), rng.integers(0, N, 50)
+    got = oracle.sgemm_oracle_entries(A, B, C, ii, jj)
+    assert np.array_equal(got, C1[ii, jj])
+    # cross-check with a library routine in higher precision, within the binary32 bound
+    ref = C.astype(np.float64) + A.astype(np.float64) @ B.astype(np.float64)
+    scale = np.abs(C).astype(np.float64) + np.abs(A).astype(np.float64) @ np.abs(B).astype(np.float64)
+    assert (np.abs(C1 - ref) <= (K + 1) * oracle.U32 * scale * 1.01).all()

@@ -30,4 +30,6 @@ from .binding import (  # noqa: F401
     dgemm_version,
     lib_path,
     load_library,
+    sgemm_f32,
+    sgemm_last_device_status,
 )

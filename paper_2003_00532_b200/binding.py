@@ -70,6 +70,10 @@ def load_library() -> ctypes.CDLL:
             lib.dgemm_f64_ex.argtypes = [ctypes.c_int, ctypes.c_int, i64, i64, i64, ctypes.c_double, vp, i64, vp, i64,
                                          ctypes.c_double, vp, i64, vp]
             lib.dgemm_f64_ex.restype = ctypes.c_int
+            lib.sgemm_f32.argtypes = [i64, i64, i64, vp, i64, vp, i64, vp, i64, vp]
+            lib.sgemm_f32.restype = ctypes.c_int
+            lib.sgemm_last_device_status.argtypes = [vp]
+            lib.sgemm_last_device_status.restype = ctypes.c_int
             lib.dgemm_f64_static_ws.argtypes = [i64, i64, i64, vp, i64, vp, i64, vp, i64, ctypes.c_int, vp]
             lib.dgemm_f64_static_ws.restype = ctypes.c_int
             lib.dgemm_strerror.argtypes = [ctypes.c_int]
@@ -95,13 +99,14 @@ def load_library() -> ctypes.CDLL:
     return _lib
 
 
-def _matrix_args(x, name: str, want_cuda: bool):
-    """(address, rows, cols, ld) of a 2-D float64 tensor with unit column stride."""
+def _matrix_args(x, name: str, want_cuda: bool, dtype=None):
+    """(address, rows, cols, ld) of a 2-D float64 (or `dtype`) tensor with unit column stride."""
     import torch
+    dtype = dtype or torch.float64
     if not isinstance(x, torch.Tensor):
         raise TypeError(f"{name}: expected a torch.Tensor")
-    if x.dtype != torch.float64 or x.dim() != 2:
-        raise TypeError(f"{name}: need a 2-D float64 tensor")
+    if x.dtype != dtype or x.dim() != 2:
+        raise TypeError(f"{name}: need a 2-D {str(dtype).replace('torch.', '')} tensor")
     if x.is_cuda != want_cuda:
         raise ValueError(f"{name}: expected a {'CUDA' if want_cuda else 'host'} tensor")
     rows, cols = x.shape
@@ -174,6 +179,25 @@ def dgemm_f64_ex(A, B, C, alpha: float = 1.0, beta: float = 1.0, transa: bool = 
     if check and rc < 0:
         raise DgemmError(rc, "dgemm_f64_ex")
     return rc
+
+
+def sgemm_f32(A, B, C, stream=None, check: bool = True) -> int:
+    """Single precision ``C += A @ B`` (CUDA float32 tensors, row-major, row stride = leading
+    dimension), exact binary32 arithmetic, asynchronously on ``stream``."""
+    import torch
+    pa, M, K, lda = _matrix_args(A, "A", True, torch.float32)
+    pb, K2, N, ldb = _matrix_args(B, "B", True, torch.float32)
+    pc, M2, N2, ldc = _matrix_args(C, "C", True, torch.float32)
+    if K != K2 or M != M2 or N != N2:
+        raise ValueError(f"shape mismatch: A {tuple(A.shape)}, B {tuple(B.shape)}, C {tuple(C.shape)}")
+    rc = load_library().sgemm_f32(M, N, K, pa, lda, pb, ldb, pc, ldc, _stream_handle(stream))
+    if check and rc < 0:
+        raise DgemmError(rc, "sgemm_f32")
+    return rc
+
+
+def sgemm_last_device_status(stream=None) -> int:
+    return int(load_library().sgemm_last_device_status(_stream_handle(stream)))
 
 
 def dgemm_f64_static_ws(A, B, C, split_k: int = 0, stream=None, check: bool = True) -> int:

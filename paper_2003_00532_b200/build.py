@@ -9,9 +9,9 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libdgemm.so")
-SOURCES = [os.path.join(CSRC, "dgemm_api.cu")]
-DEPS = SOURCES + [os.path.join(CSRC, f) for f in ("dgemm_dmma.cuh", "ptx.cuh")] + [
-    os.path.join(os.path.dirname(HERE), "include", "dgemm.h")]
+SOURCES = [os.path.join(CSRC, "dgemm_api.cu"), os.path.join(CSRC, "sgemm_api.cu")]
+DEPS = SOURCES + [os.path.join(CSRC, f) for f in ("dgemm_dmma.cuh", "sgemm_ffma.cuh", "ptx.cuh")] + [
+    os.path.join(os.path.dirname(HERE), "include", f) for f in ("dgemm.h", "sgemm.h")]
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

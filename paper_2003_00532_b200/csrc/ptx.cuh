@@ -139,6 +139,25 @@ __device__ __forceinline__ void lds128_off(uint32_t addr, double& x, double& y) 
   asm volatile("ld.shared.v2.f64 {%0, %1}, [%2+%3];" : "=d"(x), "=d"(y) : "r"(addr), "n"(OFF));
 }
 
+__device__ __forceinline__ float4 lds128_f32(uint32_t addr) {
+  float4 v;
+  asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
+  return v;
+}
+
+__device__ __forceinline__ float2 lds64_f32(uint32_t addr) {
+  float2 v;
+  asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(addr));
+  return v;
+}
+
+// {x, x} as a packed pair for the two-wide FP32 instructions.
+__device__ __forceinline__ float2 dup_f32x2(float x) {
+  unsigned long long r;
+  asm("mov.b64 %0, {%1, %1};" : "=l"(r) : "r"(__float_as_uint(x)));
+  return make_float2(__uint_as_float((unsigned)(r & 0xffffffffu)), __uint_as_float((unsigned)(r >> 32)));
+}
+
 // ---- FP64 tensor-core MMA: D(16x8) += A(16x8, row) * B(8x8, col) ---------------------------------
 // Lane l: g = l/4, t = l%4. a0=A[g][t] a1=A[g+8][t] a2=A[g][t+4] a3=A[g+8][t+4];
 // b0=B[t][g] b1=B[t+4][g]; c0,c1=C[g][2t,2t+1]; c2,c3=C[g+8][2t,2t+1].

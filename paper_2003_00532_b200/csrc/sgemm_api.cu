@@ -188,7 +188,7 @@ int launch(int64_t M, int64_t N, int64_t K, const float* A, int64_t lda, const f
   if (!p.b_blocked_map && !make_map(&map_b, B, K, N, ldb, 32, TK)) return DGEMM_ERR_CUDA;
 
   const int tiles = p.tiles_m * p.tiles_n;
-  const int resident = 2 * st->sm_count;
+  const int resident = SGEMM_CTAS * st->sm_count;
   const int grid = tiles < resident ? tiles : resident;
   sgemm_ffma_kernel<<<grid, THREADS, SMEM_BYTES, stream>>>(map_a, map_b, p);
   return cudaGetLastError() == cudaSuccess ? DGEMM_OK : DGEMM_ERR_CUDA;

@@ -17,7 +17,11 @@ namespace sgemm {
 
 using namespace dgemm::ptx;
 
-constexpr int TM = 128;  // CTA tile rows
+#ifndef SGEMM_CTAS
+#define SGEMM_CTAS 1
+#endif
+constexpr int TM = SGEMM_CTAS == 1 ? 256 : 128;  // CTA tile rows
+constexpr int RPT = TM / 16;                       // rows per thread
 constexpr int TN = 128;  // CTA tile columns
 constexpr int TK = 32;   // k extent of a stage: 32 floats = one 128-byte swizzle row
 constexpr int THREADS = 256;
@@ -26,11 +30,12 @@ constexpr int A_BYTES = TM * TK * 4;        // 16 KiB: 128 rows of 128 bytes
 constexpr int B_BOX_BYTES = TK * 32 * 4;    // 4 KiB: [32 k][32 columns]
 constexpr int B_BYTES = (TN / 32) * B_BOX_BYTES;
 constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-constexpr int STAGES = 3;
-constexpr int LOOKAHEAD = STAGES - 1;       // k-blocks in flight ahead of the arithmetic
+constexpr int STAGES = SGEMM_CTAS == 1 ? 4 : 3;
+constexpr int LOOKAHEAD = 2;                // k-blocks in flight ahead of the arithmetic
 constexpr int SMEM_ALIGN = 1024;
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + SMEM_ALIGN + 256;
 constexpr int STATUS_TIMEOUT = -8;          // DGEMM_ERR_TIMEOUT
+
 
 struct Params {
   int M, N, K;
@@ -79,7 +84,7 @@ __device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, vola
   return wait_slow(bar, parity, abort_flag, p.wait_limit_ns, p.status);
 }
 
-__global__ void __launch_bounds__(THREADS, 2)
+__global__ void __launch_bounds__(THREADS, SGEMM_CTAS)
 sgemm_ffma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                   const __grid_constant__ Params p) {
   extern __shared__ uint8_t smem_raw[];
@@ -164,16 +169,16 @@ sgemm_ffma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
   const uint32_t b_off = (uint32_t)A_BYTES + (uint32_t)(tx >> 3) * B_BOX_BYTES;  // + k * 128 + (((tx & 7) ^ (k & 7)) << 4)
   const uint32_t b_ch = (uint32_t)(tx & 7);
 
-  float acc[8][8];
+  float2 acc[RPT][4];  // [row i][column pair]: columns 4 tx + {0,1}, {2,3}, 64 + 4 tx + {0,1}, {2,3}
   uint32_t it = 0;  // k-blocks consumed so far
 
   for (int tile = cta; tile < ntiles && ok; tile += nctas) {
     int tm, tn;
     tile_to_mn(p, tile, tm, tn);
 #pragma unroll
-    for (int i = 0; i < 8; ++i)
+    for (int i = 0; i < RPT; ++i)
 #pragma unroll
-      for (int j = 0; j < 8; ++j) acc[i][j] = 0.0f;
+      for (int j = 0; j < 4; ++j) acc[i][j] = make_float2(0.0f, 0.0f);
 
     for (int kb = 0; kb < p.kblocks; ++kb, ++it) {
       // keep the load stream ahead: refill the stage that was released one k-block ago
@@ -181,30 +186,31 @@ sgemm_ffma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
       const uint32_t s = it % STAGES;
       const uint32_t ph = (it / STAGES) & 1u;
       if (!wait_bounded(full_bar + 8 * s, ph, abort_flag, p)) { ok = false; break; }
-      const uint8_t* st = tiles + s * STAGE_BYTES;
+      const uint32_t st = tiles_u32 + s * STAGE_BYTES;
+      // Four k values per loop iteration, as two pairs (the fully unrolled stage, 2200 instructions,
+      // overflowed the instruction cache; 16-byte A fragments for four k at once cost 16 more
+      // registers than the 128 that two CTAs per SM allow, and spilled).
+#pragma unroll 2
+      for (int kp = 0; kp < TK / 2; ++kp) {
+        float2 a[RPT];
+        const uint32_t ao = st + a_off + ((((uint32_t)kp >> 1) ^ a_sw) << 4) + (((uint32_t)kp & 1u) << 3);
 #pragma unroll
-      for (int kg = 0; kg < TK / 4; ++kg) {
-        float4 a[8];
+        for (int i = 0; i < RPT; ++i) a[i] = lds64_f32(ao + i * 2048);
 #pragma unroll
-        for (int i = 0; i < 8; ++i)
-          a[i] = *reinterpret_cast<const float4*>(st + a_off + i * 2048 + (((uint32_t)kg ^ a_sw) << 4));
+        for (int kk = 0; kk < 2; ++kk) {
+          const uint32_t k7 = (2u * (uint32_t)kp + kk) & 7u;
+          const uint32_t bo = st + b_off + (2 * kp + kk) * 128 + ((b_ch ^ k7) << 4);
+          const float4 b0 = lds128_f32(bo);
+          const float4 b1 = lds128_f32(bo + 2 * B_BOX_BYTES);
 #pragma unroll
-        for (int kk = 0; kk < 4; ++kk) {
-          const int k = 4 * kg + kk;
-          const uint32_t bo = b_off + k * 128 + ((b_ch ^ (uint32_t)(k & 7)) << 4);
-          const float4 b0 = *reinterpret_cast<const float4*>(st + bo);
-          const float4 b1 = *reinterpret_cast<const float4*>(st + bo + 2 * B_BOX_BYTES);
-#pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            const float av = kk == 0 ? a[i].x : kk == 1 ? a[i].y : kk == 2 ? a[i].z : a[i].w;
-            acc[i][0] = fmaf(av, b0.x, acc[i][0]);
-            acc[i][1] = fmaf(av, b0.y, acc[i][1]);
-            acc[i][2] = fmaf(av, b0.z, acc[i][2]);
-            acc[i][3] = fmaf(av, b0.w, acc[i][3]);
-            acc[i][4] = fmaf(av, b1.x, acc[i][4]);
-            acc[i][5] = fmaf(av, b1.y, acc[i][5]);
-            acc[i][6] = fmaf(av, b1.z, acc[i][6]);
-            acc[i][7] = fmaf(av, b1.w, acc[i][7]);
+          for (int i = 0; i < RPT; ++i) {
+            // packed FP32 FMA (two independent IEEE fused multiply-adds per instruction): half the
+            // issue slots of scalar FFMA for the same arithmetic
+            const float2 aa = dup_f32x2(kk == 0 ? a[i].x : a[i].y);
+            acc[i][0] = __ffma2_rn(aa, make_float2(b0.x, b0.y), acc[i][0]);
+            acc[i][1] = __ffma2_rn(aa, make_float2(b0.z, b0.w), acc[i][1]);
+            acc[i][2] = __ffma2_rn(aa, make_float2(b1.x, b1.y), acc[i][2]);
+            acc[i][3] = __ffma2_rn(aa, make_float2(b1.z, b1.w), acc[i][3]);
           }
         }
       }
@@ -219,7 +225,7 @@ sgemm_ffma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     // Epilogue: C += acc, 16-byte accesses where the row segment is aligned and inside N.
     const bool vec = ((reinterpret_cast<uintptr_t>(p.C) & 15) == 0) && ((p.ldc & 3) == 0);
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
+    for (int i = 0; i < RPT; ++i) {
       const int row = tm * TM + ty + 16 * i;
       if (row >= p.M) continue;
       float* crow = p.C + (long long)row * p.ldc;
@@ -228,15 +234,15 @@ sgemm_ffma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         const int col = tn * TN + 64 * h + 4 * tx;
         if (vec && col + 3 < p.N) {
           float4 c = *reinterpret_cast<const float4*>(crow + col);
-          c.x += acc[i][4 * h + 0];
-          c.y += acc[i][4 * h + 1];
-          c.z += acc[i][4 * h + 2];
-          c.w += acc[i][4 * h + 3];
+          c.x += acc[i][2 * h + 0].x;
+          c.y += acc[i][2 * h + 0].y;
+          c.z += acc[i][2 * h + 1].x;
+          c.w += acc[i][2 * h + 1].y;
           *reinterpret_cast<float4*>(crow + col) = c;
         } else {
 #pragma unroll
           for (int e = 0; e < 4; ++e)
-            if (col + e < p.N) crow[col + e] += acc[i][4 * h + e];
+            if (col + e < p.N) crow[col + e] += (e & 1) ? acc[i][2 * h + (e >> 1)].y : acc[i][2 * h + (e >> 1)].x;
         }
       }
     }

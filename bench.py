@@ -164,6 +164,40 @@ def other_shapes(dg, torch, peak_tflops, hbm_gbs):
     return sweep, shapes
 
 
+def sgemm_section(dg, torch, sm_max_mhz, sizes=(2048, 4096, 8192)):
+    """The paper's second workload (Section 2.13): C += A*B in binary32, here exact FP32 arithmetic
+    on the FP32 pipe (packed FFMA). The path is bound by plain ALU arithmetic: peak = SMs x 128
+    FMA/clk x 2 x clock. Timed like the FP64 headline, on resident operands."""
+    peak = SM_COUNT_B200 * 128 * 2 * sm_max_mhz * 1e6 / 1e12
+    out = {"dtype": "f32", "bound": "alu", "peak": peak, "unit": "TFLOP/s",
+           "peak_source": "148 SMs x 128 FP32 FMA/clk x 2 x sm_max_mhz; a register-only packed-FMA loop sustains 85 % of it",
+           "kernel": "sgemm_ffma_kernel (TMA staging, 256 x 128 x 32 tiles, 16 x 8 per thread, fma.rn.f32x2)", "shapes": []}
+    call = dg.load_library().sgemm_f32
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for n in sizes:
+        A = torch.rand(n, n, dtype=torch.float32, device="cuda") * 2 - 1
+        B = torch.rand(n, n, dtype=torch.float32, device="cuda") * 2 - 1
+        C = torch.zeros(n, n, dtype=torch.float32, device="cuda")
+        pa, pb, pc = A.data_ptr(), B.data_ptr(), C.data_ptr()
+        for _ in range(3):
+            call(n, n, n, pa, n, pb, n, pc, n, None)
+        torch.cuda.synchronize()
+        reps = max(3, min(50, int(8192 ** 3 // n ** 3) * 3))
+        best = float("inf")
+        for _ in range(3):
+            e0.record()
+            for _ in range(reps):
+                call(n, n, n, pa, n, pb, n, pc, n, None)
+            e1.record()
+            torch.cuda.synchronize()
+            best = min(best, e0.elapsed_time(e1) / reps)
+        tf = 2.0 * n ** 3 / best / 1e9
+        out["shapes"].append({"n": n, "us": round(best * 1e3, 1), "tflops": round(tf, 2), "frac": round(tf / peak, 3)})
+        del A, B, C
+    assert dg.sgemm_last_device_status() == 0
+    return out
+
+
 def ablation_ladder(dg, torch, peak_tflops, n=4096):
     """The paper walks from a naive nest to its best schedule step by step (Sections 2.3-2.9, Figure
     'journey'); this is the same walk on the GPU at M=N=K=n: each rung is a variant or test flag of
@@ -357,6 +391,7 @@ def run_ours(args):
     if not args.no_sweep:
         line["sweep"], line["other_shapes"] = other_shapes(dg, torch, peak_tflops, hbm_gbs)
         line["ablation"] = ablation_ladder(dg, torch, peak_tflops)
+        line["sgemm"] = sgemm_section(dg, torch, sm_max_mhz)
     print(json.dumps(line), flush=True)
     if distributed:
         dist.destroy_process_group()
@@ -375,9 +410,17 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--shape", type=str, default="", help="M,N,K of another (non-square) workload; profiling aid")
     ap.add_argument("--no-sweep", action="store_true", help="skip the size sweep and the ragged / rank-k shapes")
+    ap.add_argument("--sgemm-size", type=int, default=0,
+                    help="profiling aid: time only sgemm_f32 at M=N=K of this size, print its section and exit")
     args = ap.parse_args()
     if args.steps < 1:
         ap.error("--steps must be >= 1")
+    if args.sgemm_size:
+        import torch
+        import paper_2003_00532_b200 as dg
+        torch.cuda.set_device(0)
+        print(json.dumps(sgemm_section(dg, torch, 1965.0, sizes=(args.sgemm_size,))))
+        return 0
     return run_reference(args) if args.impl == "reference" else run_ours(args)
 
 

@@ -30,11 +30,15 @@ def test_every_declared_symbol_is_exported(lib):
             "dgemm_fp64_peak_probe", "dgemm_selftest_wait_timeout"} <= set(names)
     for n in names:
         assert hasattr(lib, n), f"{n} is declared in dgemm.h but not exported by libdgemm.so"
+    names32 = _declared(os.path.join(ROOT, "include", "sgemm.h"), r"DGEMM_API\s+[\w\s\*]+?\b(sgemm_\w+)\s*\(")
+    assert {"sgemm_f32", "sgemm_last_device_status"} <= set(names32)
+    for n in names32:
+        assert hasattr(lib, n), f"{n} is declared in sgemm.h but not exported by libdgemm.so"
 
 
 def test_header_is_plain_c():
     import subprocess
-    src = '#include "dgemm.h"\nint main(void){return DGEMM_OK + DGEMM_VARIANT_COUNT - 3;}\n'
+    src = '#include "dgemm.h"\n#include "sgemm.h"\nint main(void){return DGEMM_OK + DGEMM_VARIANT_COUNT - 3;}\n'
     subprocess.run(["gcc", "-std=c99", "-Wall", "-Werror", "-I", os.path.join(ROOT, "include"), "-x", "c", "-",
                     "-fsyntax-only"], input=src.encode(), check=True)
 

@@ -1,0 +1,56 @@
+"""Tile-parameter exploration (``paper_2003_00532_b200.tune``): the analytical model on CPU, the
+autotuner against the library's own choice on a GPU."""
+import pytest
+
+from paper_2003_00532_b200 import tune
+
+
+def test_register_budget_of_the_default_tiles():
+    """64 x 32 FP64 warp tiles: 128 accumulator registers, two 48-register fragment sets, and the
+    whole thing inside 255 registers per thread and 64 K per CTA of 8 warps; a 64 x 64 warp tile
+    (256 accumulator registers) cannot fit, which is why the CTA tile stops at 128 x 128."""
+    b = tune.register_budget(128, 128, 8)
+    assert b["accumulators"] == 128 and b["fragments_per_half_kblock"] == 48
+    assert b["fits_255"] and b["cta_registers"] <= 65536
+    big = tune.register_budget(128, 128, 4, wt_m=64, wt_n=64)
+    assert not big["fits_255"]
+
+
+def test_model_matches_measured_headline():
+    """8192^3 with the warp-specialised kernel: 30.35 ms measured on B200 (CUDA events,
+    profiles/bench_8192_launch_list.md); the model must land within 3 %."""
+    ms = tune.model_ms(8192, 8192, 8192, tune.CONFIGS["ws128"])
+    assert abs(ms - 30.35) / 30.35 < 0.03
+
+
+def test_model_orders_the_known_cases():
+    rank = [r["config"] for r in tune.predict(8192, 8192, 8192)]
+    assert rank[0] == "ws128" and rank.index("generic") > rank.index("inline64")
+    # rank-k update, K = 64: the C round trip dominates and two CTAs per SM hide it
+    rk = {r["config"]: r["model_ms"] for r in tune.predict(16384, 16384, 64)}
+    assert min(rk["ws64"], rk["inline64"]) < rk["ws128"]
+    # monotone in every dimension
+    base = tune.model_ms(2048, 2048, 2048, tune.CONFIGS["ws128"])
+    assert tune.model_ms(4096, 2048, 2048, tune.CONFIGS["ws128"]) > base
+    assert tune.model_ms(2048, 2048, 4096, tune.CONFIGS["ws128"]) > base
+    # never faster than the pipe or the memory system allow
+    for (M, N, K) in [(128, 128, 128), (4097, 31, 4099), (16384, 16384, 64), (8192, 8192, 8192)]:
+        for cfg in tune.CONFIGS.values():
+            ms = tune.model_ms(M, N, K, cfg)
+            assert ms * 1e-3 >= 2.0 * M * N * K / (tune.PEAK_TFLOPS * 1e12)
+            assert ms * 1e-3 >= 8.0 * (M * K + K * N + 2 * M * N) / (tune.HBM_GBS * 1e9)
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("shape", [(1024, 1024, 1024), (2088, 2048, 2048), (4096, 4096, 256)])
+def test_autotuner_confirms_the_library_choice(shape):
+    """The library's own choice must be within 4 % of the best configuration the tuner finds, and
+    the model within 30 % of the measurement for the configurations it covers."""
+    rows = tune.autotune(*shape)
+    by = {r["config"]: r for r in rows}
+    assert "auto" in by and len(rows) >= 5
+    best = rows[0]["ms"]
+    assert by["auto"]["ms"] <= 1.04 * best, (by["auto"], rows[0])
+    for r in rows:
+        if "model_ms" in r and r["config"] in ("ws128", "inline64", "ws64"):
+            assert abs(r["model_ms"] - r["ms"]) / r["ms"] < 0.30, r

@@ -205,8 +205,12 @@ enum {
   DGEMM_TEST_TALL_TILES = 4,    /* 128-row tiles, one CTA per SM, instead of 64-row tiles, two per SM */
   DGEMM_TEST_SMALL_WARP_TILES = 8, /* 32 x 32 warp tiles (twice the warps) instead of 64 x 32           */
   DGEMM_TEST_NO_PACKING = 16,   /* never pack unaligned operands: always use the generic staging      */
-  DGEMM_TEST_WS_TWO_CTAS = 32   /* DGEMM_VARIANT_TMA_WS: 64-row tiles, two CTAs per SM, at any K (the
+  DGEMM_TEST_WS_TWO_CTAS = 32,  /* DGEMM_VARIANT_TMA_WS: 64-row tiles, two CTAs per SM, at any K (the
                                    library itself uses that form only for K < 256)                 */
+  DGEMM_TEST_FUSED_TAIL_REDUCE = 64 /* add the partial tiles of the last wave to C inside the GEMM kernel
+                                   (cooperative launch; the CTAs of a tile wait for one another, with
+                                   a time limit) instead of in a second kernel: same results bit for
+                                   bit, one launch fewer, measured slower                          */
 };
 DGEMM_API int dgemm_set_test_flags(int flags);
 

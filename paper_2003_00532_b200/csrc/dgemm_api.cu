@@ -21,6 +21,7 @@ using namespace dgemm;
 
 constexpr int kMaxDevices = 64;
 constexpr size_t kWorkspaceBytes = 640ull * BM * BN * sizeof(double);  // 80 MiB: up to 640 partial-tile slots
+constexpr size_t kCounterBytes = 65536;  // in front of the slots: two counters per tail tile (fused tail reduction)
 constexpr unsigned long long kWaitLimitNs = 4000000000ull;            // 4 s per device-side wait
 constexpr int kAutoGeneric = DGEMM_VARIANT_GENERIC;  // what DGEMM_VARIANT_AUTO picks for operands TMA cannot address
 constexpr int kAutoWsMinKblocks = 16;                // warp-specialised kernel: 128-row tiles from K = 256 up, 64-row below
@@ -54,10 +55,24 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 EncodeTiledFn g_encode = nullptr;
 
+// Launches a GEMM kernel. When its CTAs wait for one another (the fused tail reduction) the launch
+// is cooperative: the driver then starts the grid only when all of its CTAs can be resident at
+// once, also next to other work on the GPU.
+template <typename Kernel>
+void launch_gemm_kernel(Kernel kernel, int grid, int threads, int smem, cudaStream_t stream, const CUtensorMap& map_a,
+                        const CUtensorMap& map_b, const GemmParams& p) {
+  if (p.tail_fused) {
+    void* args[3] = {const_cast<CUtensorMap*>(&map_a), const_cast<CUtensorMap*>(&map_b), const_cast<GemmParams*>(&p)};
+    cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(kernel), dim3(grid), dim3(threads), args, (size_t)smem, stream);
+  } else {
+    kernel<<<grid, threads, smem, stream>>>(map_a, map_b, p);
+  }
+}
+
 template <bool USE_TMA, int TBM, int WTM, int TBN = BN>
 void launch_tile_kernel(int grid, cudaStream_t stream, const CUtensorMap& map_a, const CUtensorMap& map_b, const GemmParams& p) {
-  dgemm_dmma_kernel<USE_TMA, TBM, WTM, TBN>
-      <<<grid, TileCfg<TBM, WTM, TBN>::THREADS_, TileCfg<TBM, WTM, TBN>::SMEM_BYTES_, stream>>>(map_a, map_b, p);
+  launch_gemm_kernel(dgemm_dmma_kernel<USE_TMA, TBM, WTM, TBN>, grid, TileCfg<TBM, WTM, TBN>::THREADS_,
+                     TileCfg<TBM, WTM, TBN>::SMEM_BYTES_, stream, map_a, map_b, p);
 }
 
 template <bool USE_TMA>
@@ -130,10 +145,12 @@ int device_state(DeviceState** out) {
 int ensure_workspace(DeviceState* st) {
   std::lock_guard<std::mutex> lock(g_mutex);
   if (!st->workspace) {
-    if (cudaMalloc(reinterpret_cast<void**>(&st->workspace), kWorkspaceBytes) != cudaSuccess) {
+    if (cudaMalloc(reinterpret_cast<void**>(&st->workspace), kCounterBytes + kWorkspaceBytes) != cudaSuccess) {
       (void)cudaGetLastError();
       return DGEMM_ERR_CUDA;
     }
+    // the counters are zero between calls: the kernels that use them put them back
+    if (cudaMemset(st->workspace, 0, kCounterBytes) != cudaSuccess) return DGEMM_ERR_CUDA;
   }
   return DGEMM_OK;
 }
@@ -393,7 +410,13 @@ int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, c
   if (uses_workspace) {
     rc = ensure_workspace(st);
     if (rc != DGEMM_OK) return rc;
-    p.partial = st->workspace;
+    p.partial = st->workspace + kCounterBytes / sizeof(double);
+    p.tail_counters = reinterpret_cast<int*>(st->workspace);
+    // option: the CTAs that compute a tail tile also reduce it (not with a uniform K split, where a
+    // CTA may hold more than two partial tiles)
+    p.tail_fused = (p.split_k == 1 && p.tail_tiles > 0 && p.tail_ipc < kblocks &&
+                    (size_t)p.tail_tiles * 2 * sizeof(int) <= kCounterBytes && (dbg_flags & DGEMM_TEST_FUSED_TAIL_REDUCE))
+                       ? 1 : 0;
   }
 
   CUtensorMap map_a, map_b;
@@ -404,14 +427,14 @@ int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, c
     p.b_blocked_map = (!(dbg_flags & DGEMM_TEST_NO_BLOCKED_B) && N % 16 == 0 && make_blocked_map(&map_b, B, K, N, ldb, BK, bn / 16)) ? 1 : 0;
     if (!p.b_blocked_map && !make_map(&map_b, B, K, N, ldb, 16, BK)) return DGEMM_ERR_CUDA;
     if (ws64)
-      dgemm_dmma_ws_kernel<true, 64><<<grid, WsCfg<64>::THREADS_, WsCfg<64>::SMEM_BYTES_, stream>>>(map_a, map_b, p);
+      launch_gemm_kernel(dgemm_dmma_ws_kernel<true, 64>, grid, WsCfg<64>::THREADS_, WsCfg<64>::SMEM_BYTES_, stream, map_a, map_b, p);
     else if (variant == DGEMM_VARIANT_TMA_WS)
-      dgemm_dmma_ws_kernel<true><<<grid, WS_THREADS, SMEM_BYTES, stream>>>(map_a, map_b, p);
+      launch_gemm_kernel(dgemm_dmma_ws_kernel<true>, grid, WS_THREADS, SMEM_BYTES, stream, map_a, map_b, p);
     else
       launch_default_kernel<true>(bm, wtm, grid, stream, map_a, map_b, p);
   } else {
     if (variant == DGEMM_VARIANT_GENERIC_WS)
-      dgemm_dmma_ws_kernel<false><<<grid, WS_THREADS, SMEM_BYTES, stream>>>(map_a, map_b, p);
+      launch_gemm_kernel(dgemm_dmma_ws_kernel<false>, grid, WS_THREADS, SMEM_BYTES, stream, map_a, map_b, p);
     else
       launch_default_kernel<false>(bm, wtm, grid, stream, map_a, map_b, p);
   }
@@ -422,7 +445,7 @@ int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, c
     g_launches.fetch_add(1);
     if (cudaGetLastError() != cudaSuccess) return DGEMM_ERR_CUDA;
   }
-  if (p.tail_tiles > 0 && p.tail_ipc < kblocks) {
+  if (p.tail_tiles > 0 && p.tail_ipc < kblocks && !p.tail_fused) {
     dgemm_tail_reduce_kernel<<<dim3(p.tail_tiles, REDUCE_CHUNKS), REDUCE_THREADS, 0, stream>>>(p);
     g_launches.fetch_add(1);
     if (cudaGetLastError() != cudaSuccess) return DGEMM_ERR_CUDA;
@@ -717,7 +740,7 @@ int dgemm_set_variant(int variant) {
 }
 
 int dgemm_set_test_flags(int flags) {
-  if (flags < 0 || flags > (DGEMM_TEST_NO_C_PREFETCH | DGEMM_TEST_NO_BLOCKED_B | DGEMM_TEST_TALL_TILES | DGEMM_TEST_SMALL_WARP_TILES | DGEMM_TEST_NO_PACKING | DGEMM_TEST_WS_TWO_CTAS)) return DGEMM_ERR_VARIANT;
+  if (flags < 0 || flags > (DGEMM_TEST_NO_C_PREFETCH | DGEMM_TEST_NO_BLOCKED_B | DGEMM_TEST_TALL_TILES | DGEMM_TEST_SMALL_WARP_TILES | DGEMM_TEST_NO_PACKING | DGEMM_TEST_WS_TWO_CTAS | DGEMM_TEST_FUSED_TAIL_REDUCE)) return DGEMM_ERR_VARIANT;
   g_test_flags.store(flags);
   return DGEMM_OK;
 }

@@ -25,6 +25,7 @@ struct DeviceState {
   int* status = nullptr;
   float* pack_buf = nullptr;
   size_t pack_bytes = 0;
+  float* workspace = nullptr;  // partial tiles of the stream-K tail, allocated on first need
 };
 
 DeviceState g_dev[kMaxDevices];
@@ -187,11 +188,42 @@ int launch(int64_t M, int64_t N, int64_t K, const float* A, int64_t lda, const f
   p.b_blocked_map = (N % 32 == 0 && make_blocked_map(&map_b, B, K, N, ldb)) ? 1 : 0;
   if (!p.b_blocked_map && !make_map(&map_b, B, K, N, ldb, 32, TK)) return DGEMM_ERR_CUDA;
 
+  // whole waves of tiles run data-parallel; the last partial wave is spread evenly over the CTAs
+  // (stream-K) when that saves more time than the partial-tile round trip costs
   const int tiles = p.tiles_m * p.tiles_n;
   const int resident = SGEMM_CTAS * st->sm_count;
-  const int grid = tiles < resident ? tiles : resident;
+  int grid = tiles < resident ? tiles : resident;
+  p.dp_tiles = tiles;
+  p.tail_tiles = 0;
+  p.tail_ipc = p.kblocks;
+  const int tail = tiles % resident;
+  if (tail > 0 && p.kblocks >= 2 && (1.0 - (double)tail / resident) * p.kblocks >= 3.0 &&
+      (long long)(tail + 1) * p.kblocks < (long long)INT32_MAX) {
+    p.dp_tiles = tiles - tail;
+    p.tail_tiles = tail;
+    const long long total = (long long)tail * p.kblocks;
+    long long ipc = (total + resident - 1) / resident;
+    if (ipc > p.kblocks) ipc = p.kblocks;
+    p.tail_ipc = (int)ipc;
+    const int span_ctas = (int)((total + ipc - 1) / ipc);
+    if (p.dp_tiles == 0) grid = span_ctas < resident ? span_ctas : resident;
+    {
+      std::lock_guard<std::mutex> lock(g_mutex);
+      if (!st->workspace && cudaMalloc(reinterpret_cast<void**>(&st->workspace), (size_t)2 * resident * TM * TN * sizeof(float)) !=
+                                cudaSuccess) {
+        (void)cudaGetLastError();
+        return DGEMM_ERR_CUDA;
+      }
+    }
+    p.partial = st->workspace;
+  }
   sgemm_ffma_kernel<<<grid, THREADS, SMEM_BYTES, stream>>>(map_a, map_b, p);
-  return cudaGetLastError() == cudaSuccess ? DGEMM_OK : DGEMM_ERR_CUDA;
+  if (cudaGetLastError() != cudaSuccess) return DGEMM_ERR_CUDA;
+  if (p.tail_tiles > 0 && p.tail_ipc < p.kblocks) {
+    sgemm_tail_reduce_kernel<<<dim3(p.tail_tiles, 16), 256, 0, stream>>>(p);
+    if (cudaGetLastError() != cudaSuccess) return DGEMM_ERR_CUDA;
+  }
+  return DGEMM_OK;
 }
 
 }  // namespace

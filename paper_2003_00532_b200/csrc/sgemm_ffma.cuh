@@ -43,6 +43,12 @@ struct Params {
   int kblocks;         // ceil(K / TK)
   int group_m;         // raster group height in tiles
   int b_blocked_map;   // map_b is the 3-D view (32 columns, K, N/32): one copy stages the whole B tile
+  // Work decomposition (as in the FP64 kernels): tiles [0, dp_tiles) run whole, CTA b taking b,
+  // b + G, ...; the k-blocks of the remaining tail_tiles are cut into equal spans of tail_ipc, one
+  // per CTA. A span covers at most two tile segments; a segment that is not a whole tile goes to
+  // workspace slot 2 * cta + j and sgemm_tail_reduce_kernel adds the slots to C in CTA order.
+  int dp_tiles, tail_tiles, tail_ipc;
+  float* partial;      // workspace: slots of TM * TN floats
   const float* A;
   const float* B;
   float* C;
@@ -60,6 +66,42 @@ __device__ __forceinline__ void tile_to_mn(const Params& p, int tile, int& tm, i
   const int rows = min(p.group_m, p.tiles_m - g * p.group_m);
   tn = r / rows;
   tm = g * p.group_m + (r - tn * rows);
+}
+
+struct Item {
+  int tile, kb0, kb1;  // tile and k-block range [kb0, kb1)
+  int slot;            // workspace slot for the partial tile, or -1: add straight into C
+};
+
+// The idx-th work item of CTA `cta`; false past the end of its list.
+__device__ __forceinline__ bool get_item(const Params& p, int cta, int nctas, int idx, Item& w) {
+  const int n1 = cta < p.dp_tiles ? (p.dp_tiles - cta + nctas - 1) / nctas : 0;
+  if (idx < n1) {
+    w.tile = cta + idx * nctas;
+    w.kb0 = 0;
+    w.kb1 = p.kblocks;
+    w.slot = -1;
+    return true;
+  }
+  const int j = idx - n1;
+  if (j > 1 || p.tail_tiles == 0) return false;
+  const int total = p.tail_tiles * p.kblocks;  // the host keeps this below 2^31
+  const int start = cta * p.tail_ipc;
+  const int end = min(start + p.tail_ipc, total);
+  if (start >= end) return false;
+  int trel = start / p.kblocks;
+  int s0 = start, s1 = min(end, (trel + 1) * p.kblocks);
+  if (j == 1) {
+    if (s1 >= end) return false;
+    s0 = s1;
+    s1 = end;
+    ++trel;
+  }
+  w.tile = p.dp_tiles + trel;
+  w.kb0 = s0 - trel * p.kblocks;
+  w.kb1 = s1 - trel * p.kblocks;
+  w.slot = (w.kb0 == 0 && w.kb1 == p.kblocks) ? -1 : 2 * cta + j;
+  return true;
 }
 
 // Polls an mbarrier phase; gives up after p.wait_limit_ns, records the timeout and raises the
@@ -112,16 +154,25 @@ sgemm_ffma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
   __syncthreads();
 
   const int cta = blockIdx.x, nctas = gridDim.x;
-  const int ntiles = p.tiles_m * p.tiles_n;
 
-  // Load stream: the k-blocks of this CTA's tiles (cta, cta + nctas, ...) in order, LOOKAHEAD
-  // k-blocks ahead of the arithmetic and across tile boundaries. Every thread follows the cursor;
-  // k-block number i is issued by lane 0 of warp i mod 8.
-  int l_tile = cta, l_kb = 0, l_tm = 0, l_tn = 0;
-  if (l_tile < ntiles) tile_to_mn(p, l_tile, l_tm, l_tn);
+  // Load stream: the k-blocks of this CTA's work items in order, LOOKAHEAD k-blocks ahead of the
+  // arithmetic and across item boundaries. Every thread follows the cursor; k-block number i is
+  // issued by lane 0 of warp i mod 8.
+  int l_idx = 0, l_kb = 0, l_kb1 = 0, l_tm = 0, l_tn = 0;
+  bool l_valid;
+  auto cursor_load = [&]() {
+    Item li;
+    l_valid = get_item(p, cta, nctas, l_idx, li);
+    if (l_valid) {
+      l_kb = li.kb0;
+      l_kb1 = li.kb1;
+      tile_to_mn(p, li.tile, l_tm, l_tn);
+    }
+  };
+  cursor_load();
   uint32_t lit = 0;
   auto issue_next = [&]() -> bool {
-    if (l_tile >= ntiles) return true;
+    if (!l_valid) return true;
     if (warp == (int)(lit % WARPS)) {
       int good = 1;
       if (lane == 0) {
@@ -145,10 +196,9 @@ sgemm_ffma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
       if (!__all_sync(0xffffffffu, good)) return false;
     }
     ++lit;
-    if (++l_kb >= p.kblocks) {
-      l_kb = 0;
-      l_tile += nctas;
-      if (l_tile < ntiles) tile_to_mn(p, l_tile, l_tm, l_tn);
+    if (++l_kb >= l_kb1) {
+      ++l_idx;
+      cursor_load();
     }
     return true;
   };
@@ -172,15 +222,17 @@ sgemm_ffma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
   float2 acc[RPT][4];  // [row i][column pair]: columns 4 tx + {0,1}, {2,3}, 64 + 4 tx + {0,1}, {2,3}
   uint32_t it = 0;  // k-blocks consumed so far
 
-  for (int tile = cta; tile < ntiles && ok; tile += nctas) {
+  for (int idx = 0; ok; ++idx) {
+    Item w;
+    if (!get_item(p, cta, nctas, idx, w)) break;
     int tm, tn;
-    tile_to_mn(p, tile, tm, tn);
+    tile_to_mn(p, w.tile, tm, tn);
 #pragma unroll
     for (int i = 0; i < RPT; ++i)
 #pragma unroll
       for (int j = 0; j < 4; ++j) acc[i][j] = make_float2(0.0f, 0.0f);
 
-    for (int kb = 0; kb < p.kblocks; ++kb, ++it) {
+    for (int kb = w.kb0; kb < w.kb1; ++kb, ++it) {
       // keep the load stream ahead: refill the stage that was released one k-block ago
       if (!issue_next()) { ok = false; break; }
       const uint32_t s = it % STAGES;
@@ -222,6 +274,17 @@ sgemm_ffma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     }
     if (!ok) break;
 
+    if (w.slot >= 0) {
+      // a segment of a tail tile: the partial sums go to the workspace (row-major TM x TN)
+      float* dst = p.partial + (long long)w.slot * (TM * TN);
+#pragma unroll
+      for (int i = 0; i < RPT; ++i)
+#pragma unroll
+        for (int h = 0; h < 2; ++h)
+          *reinterpret_cast<float4*>(dst + (ty + 16 * i) * TN + 64 * h + 4 * tx) =
+              make_float4(acc[i][2 * h].x, acc[i][2 * h].y, acc[i][2 * h + 1].x, acc[i][2 * h + 1].y);
+      continue;
+    }
     // Epilogue: C += acc, 16-byte accesses where the row segment is aligned and inside N.
     const bool vec = ((reinterpret_cast<uintptr_t>(p.C) & 15) == 0) && ((p.ldc & 3) == 0);
 #pragma unroll
@@ -261,6 +324,39 @@ sgemm_ffma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     }
   }
   __syncthreads();
+}
+
+// Adds the partial tiles of tail tile blockIdx.x to C: C[i][j] += ((p_0 + p_1) + ...) in the order of
+// the CTAs that computed them. Deterministic. blockIdx.y takes TM / 16 consecutive rows.
+__global__ void sgemm_tail_reduce_kernel(const Params p) {
+  const int trel = blockIdx.x;
+  const int lo = trel * p.kblocks, hi = lo + p.kblocks;
+  const int c_first = lo / p.tail_ipc, c_last = (hi - 1) / p.tail_ipc;
+  if (c_first == c_last) return;  // one CTA had the whole tile and added it straight to C
+  int tm, tn;
+  tile_to_mn(p, p.dp_tiles + trel, tm, tn);
+  const int chunk = TM * TN / 16;
+  const int e0 = blockIdx.y * chunk;
+  for (int e = e0 + 4 * threadIdx.x; e < e0 + chunk; e += 4 * blockDim.x) {
+    const int r = e / TN, c = e - r * TN;
+    const int row = tm * TM + r, col = tn * TN + c;
+    if (row >= p.M || col >= p.N) continue;
+    float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int cta = c_first; cta <= c_last; ++cta) {
+      const int slot = 2 * cta + ((cta * p.tail_ipc >= lo) ? 0 : 1);
+      const float4 v = *reinterpret_cast<const float4*>(p.partial + (long long)slot * (TM * TN) + e);
+      if (cta == c_first) {
+        sum = v;
+      } else {
+        sum.x += v.x; sum.y += v.y; sum.z += v.z; sum.w += v.w;
+      }
+    }
+    float* dst = p.C + (long long)row * p.ldc + col;
+    dst[0] += sum.x;
+    if (col + 1 < p.N) dst[1] += sum.y;
+    if (col + 2 < p.N) dst[2] += sum.z;
+    if (col + 3 < p.N) dst[3] += sum.w;
+  }
 }
 
 // Copies a rows x cols float matrix into a 16-byte aligned buffer whose leading dimension is a

@@ -9,6 +9,7 @@
 #include <cstdlib>
 #include <cstring>
 #include <mutex>
+#include <utility>
 
 #include <cuda.h>
 #include <cuda_runtime.h>
@@ -55,6 +56,25 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 EncodeTiledFn g_encode = nullptr;
 
+// Launch with programmatic stream serialization: the grid may be scheduled while the kernel before
+// it in the stream is draining; every kernel launched this way executes griddepcontrol.wait before
+// its first access to global memory, which returns once that earlier kernel has completed and
+// its writes are visible. Hides a few microseconds of launch latency per kernel.
+template <typename... KArgs, typename... Args>
+void launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
+
 // Launches a GEMM kernel. When its CTAs wait for one another (the fused tail reduction) the launch
 // is cooperative: the driver then starts the grid only when all of its CTAs can be resident at
 // once, also next to other work on the GPU.
@@ -65,7 +85,7 @@ void launch_gemm_kernel(Kernel kernel, int grid, int threads, int smem, cudaStre
     void* args[3] = {const_cast<CUtensorMap*>(&map_a), const_cast<CUtensorMap*>(&map_b), const_cast<GemmParams*>(&p)};
     cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(kernel), dim3(grid), dim3(threads), args, (size_t)smem, stream);
   } else {
-    kernel<<<grid, threads, smem, stream>>>(map_a, map_b, p);
+    launch_pdl(kernel, dim3(grid), dim3(threads), (size_t)smem, stream, map_a, map_b, p);
   }
 }
 
@@ -441,12 +461,12 @@ int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, c
   g_launches.fetch_add(1);
   if (cudaGetLastError() != cudaSuccess) return DGEMM_ERR_CUDA;
   if (p.split_k > 1) {
-    dgemm_splitk_reduce_kernel<<<dim3(tiles, REDUCE_CHUNKS), REDUCE_THREADS, 0, stream>>>(p);
+    launch_pdl(dgemm_splitk_reduce_kernel, dim3(tiles, REDUCE_CHUNKS), dim3(REDUCE_THREADS), 0, stream, p);
     g_launches.fetch_add(1);
     if (cudaGetLastError() != cudaSuccess) return DGEMM_ERR_CUDA;
   }
   if (p.tail_tiles > 0 && p.tail_ipc < kblocks && !p.tail_fused) {
-    dgemm_tail_reduce_kernel<<<dim3(p.tail_tiles, REDUCE_CHUNKS), REDUCE_THREADS, 0, stream>>>(p);
+    launch_pdl(dgemm_tail_reduce_kernel, dim3(p.tail_tiles, REDUCE_CHUNKS), dim3(REDUCE_THREADS), 0, stream, p);
     g_launches.fetch_add(1);
     if (cudaGetLastError() != cudaSuccess) return DGEMM_ERR_CUDA;
   }

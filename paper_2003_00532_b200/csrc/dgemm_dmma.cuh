@@ -699,6 +699,7 @@ dgemm_dmma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     ptx::fence_barrier_init();
   }
   __syncthreads();
+  ptx::grid_dependency_wait();  // everything above overlaps the tail of the previous kernel in the stream
 
   const int cta = blockIdx.x, nctas = gridDim.x;
   // Every thread follows the load stream. TMA staging: the k-blocks are issued by the warps in
@@ -932,6 +933,7 @@ dgemm_dmma_ws_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
     ptx::fence_barrier_init();
   }
   __syncthreads();
+  ptx::grid_dependency_wait();  // everything above overlaps the tail of the previous kernel in the stream
 
   const int cta = blockIdx.x, nctas = gridDim.x;
   volatile int* item_words = work_words + 8 * warp;
@@ -1092,6 +1094,7 @@ __device__ __forceinline__ void reduce_tile(const GemmParams& p, int tm, int tn,
 
 // Phase-1 split-K reduction: tile t has its split_k partials in slots ks*dp_tiles + t.
 __global__ void dgemm_splitk_reduce_kernel(const GemmParams p) {
+  ptx::grid_dependency_wait();
   const int tile = blockIdx.x;
   int tm, tn;
   tile_to_mn(p, tile, tm, tn);
@@ -1101,6 +1104,7 @@ __global__ void dgemm_splitk_reduce_kernel(const GemmParams p) {
 // Phase-2 (tail) reduction: tail tile `trel` was covered by the spans of CTAs c_first..c_last; CTA c
 // stored its part in slot tail_slot_base + 2c + j, j = 0 if the span starts inside this tile.
 __global__ void dgemm_tail_reduce_kernel(const GemmParams p) {
+  ptx::grid_dependency_wait();
   const int trel = blockIdx.x;
   const int lo = trel * p.kblocks, hi = lo + p.kblocks;
   const int c_first = lo / p.tail_ipc;
@@ -1184,6 +1188,7 @@ __global__ void dgemm_wait_timeout_selftest_kernel(const __grid_constant__ GemmP
     ptx::fence_barrier_init();
   }
   __syncthreads();
+  ptx::grid_dependency_wait();  // everything above overlaps the tail of the previous kernel in the stream
   const bool ok = wait_bounded(ptx::smem_u32(&bar), 0u, &abort_flag, p);
   if (!ok) atomicAdd(gave_up, 1);
 }

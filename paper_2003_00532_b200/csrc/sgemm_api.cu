@@ -3,6 +3,7 @@
 #include <cstdint>
 #include <cstring>
 #include <mutex>
+#include <utility>
 
 #include <cuda.h>
 #include <cuda_runtime.h>
@@ -138,6 +139,23 @@ int validate(int64_t M, int64_t N, int64_t K, const float* A, int64_t lda, const
   return DGEMM_OK;
 }
 
+// Launch with programmatic stream serialization (the kernels wait with griddepcontrol.wait before
+// their first global access): hides a few microseconds of launch latency per kernel.
+template <typename... KArgs, typename... Args>
+void launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
+
 inline unsigned grid_y(int64_t blocks) { return (unsigned)(blocks < 65535 ? blocks : 65535); }
 
 int launch(int64_t M, int64_t N, int64_t K, const float* A, int64_t lda, const float* B, int64_t ldb, float* C, int64_t ldc,
@@ -217,10 +235,10 @@ int launch(int64_t M, int64_t N, int64_t K, const float* A, int64_t lda, const f
     }
     p.partial = st->workspace;
   }
-  sgemm_ffma_kernel<<<grid, THREADS, SMEM_BYTES, stream>>>(map_a, map_b, p);
+  launch_pdl(sgemm_ffma_kernel, dim3(grid), dim3(THREADS), (size_t)SMEM_BYTES, stream, map_a, map_b, p);
   if (cudaGetLastError() != cudaSuccess) return DGEMM_ERR_CUDA;
   if (p.tail_tiles > 0 && p.tail_ipc < p.kblocks) {
-    sgemm_tail_reduce_kernel<<<dim3(p.tail_tiles, 16), 256, 0, stream>>>(p);
+    launch_pdl(sgemm_tail_reduce_kernel, dim3(p.tail_tiles, 16), dim3(256), 0, stream, p);
     if (cudaGetLastError() != cudaSuccess) return DGEMM_ERR_CUDA;
   }
   return DGEMM_OK;

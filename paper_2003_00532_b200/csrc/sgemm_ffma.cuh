@@ -152,6 +152,7 @@ sgemm_ffma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     prefetch_tensormap(&map_b);
   }
   __syncthreads();
+  grid_dependency_wait();  // launched with programmatic serialization: the set-up above overlaps the previous kernel's tail
 
   const int cta = blockIdx.x, nctas = gridDim.x;
 
@@ -329,6 +330,7 @@ sgemm_ffma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
 // Adds the partial tiles of tail tile blockIdx.x to C: C[i][j] += ((p_0 + p_1) + ...) in the order of
 // the CTAs that computed them. Deterministic. blockIdx.y takes TM / 16 consecutive rows.
 __global__ void sgemm_tail_reduce_kernel(const Params p) {
+  grid_dependency_wait();
   const int trel = blockIdx.x;
   const int lo = trel * p.kblocks, hi = lo + p.kblocks;
   const int c_first = lo / p.tail_ipc, c_last = (hi - 1) / p.tail_ipc;

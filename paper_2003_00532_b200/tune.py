@@ -27,8 +27,8 @@ from typing import Dict, List, Optional
 SM_COUNT = 148
 PEAK_TFLOPS = 148 * 64 * 2 * 1.965e9 / 1e12  # FP64 tensor pipe: 64 FMA/clk/SM
 HBM_GBS = 6500.0
-LAUNCH_US = 4.5        # launch + first copies in flight + first k-block, measured on small problems
-REDUCE_US = 6.0        # second launch and the partial-tile reduction when K is split
+LAUNCH_US = 3.0        # launch + first copies in flight, measured on small problems (programmatic dependent launch)
+REDUCE_US = 4.0        # second launch and the partial-tile reduction when K is split
 BK = 16
 
 

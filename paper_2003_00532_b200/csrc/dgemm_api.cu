@@ -348,7 +348,8 @@ int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, c
 
   const int dbg_flags = g_test_flags.load();
   const bool ws_variant = variant == DGEMM_VARIANT_TMA_WS || variant == DGEMM_VARIANT_GENERIC_WS;
-  // tile height: 64 rows with two CTAs per SM (default), 128 rows with one (warp-specialised variants, test flag)
+  // tile height of the chosen kernel: 64 rows with two CTAs per SM (inline kernel; warp-specialised kernel for short K),
+  // 128 rows with one CTA per SM (warp-specialised kernel otherwise, large generic problems, test flag)
   // (generic staging on a problem of many waves is a little faster with the tall tile: half the B copies per thread)
   const int64_t tiles128 = ((M + 127) / 128) * ((N + BN - 1) / BN);
   const bool generic_large = !wants_tma && tiles128 >= 4 * (int64_t)st->sm_count;

@@ -11,17 +11,19 @@
 //   vectorisation -> mma.sync m16n8k8 f64 (DMMA) and 16-byte shared-memory fragment loads
 //   N_C loop the paper left out (Section 2.10) -> grouped tile raster for L2 reuse
 //
-// One persistent CTA per SM with 8 warps (2 x 4 grid of 64 x 32 warp tiles, up to 255 registers
-// per thread). There is no separate producer warp: the load stream runs LOOKAHEAD k-blocks ahead
-// of the arithmetic and across tile boundaries; with TMA staging lane 0 of warp 0 issues it,
-// with generic staging every thread copies its share. Stages are handed over with mbarriers:
-// full[s] (copies landed) and empty[s] (all warps done reading). Every wait is bounded; on expiry
-// the kernel records DGEMM_ERR_TIMEOUT in the device status word, lets its own copies land and
+// Two kernels share the layouts and the epilogue:
+//   dgemm_dmma_ws_kernel  warp-specialised: 8 (or 4) consumer warps with 64 x 32 warp tiles and a
+//               producer warpgroup that walks the work items and issues the copies; setmaxnreg
+//               moves registers from the producers to the consumers; the consumers' k loop is
+//               software pipelined. 128 x 128 tiles with one CTA per SM, or 64 x 128 with two.
+//   dgemm_dmma_kernel     no producer warp: the load stream runs LOOKAHEAD k-blocks ahead of the
+//               arithmetic and across tile boundaries, issued by the warps in turn (TMA) or copied
+//               by all threads (8-byte asynchronous copies, any alignment). 64 x 128 tiles with two
+//               CTAs per SM, 128 x 128 with one, 256 x 32 for narrow N.
+// Persistent CTAs; stages are handed over with mbarriers: full[s] (copies landed) and empty[s]
+// (all warps done reading, released behind a proxy fence). Every wait is bounded; on expiry the
+// kernel records DGEMM_ERR_TIMEOUT in the device status word, lets its own copies land and
 // returns.
-//
-// (A warp-specialised variant that moved registers from a producer warpgroup to the consumers
-// with setmaxnreg was tried and dropped: with it, fragment registers of the consumer warps that
-// share a scheduler with the active producer warp were sporadically corrupted.)
 #pragma once
 
 #include <type_traits>
@@ -330,7 +332,7 @@ __device__ __forceinline__ void compute_kblock(const uint8_t* st, const LaneMap&
 
 // ---- the same arithmetic in software-pipelined pieces ---------------------------------------------
 // One half k-block (8 k values) of fragments for a warp tile of 16*MT rows x 32 columns: 48
-// registers for MT = 4. The default kernel keeps two of them, so that the loads of the next half
+// registers for MT = 4. The warp-specialised kernel keeps two of them, so that the loads of the next half
 // (and, across a k-block boundary, the barrier test before them) are issued ahead of the MMAs of
 // the current half and a warp can feed the FP64 pipe without a gap at the boundary.
 template <int MT>
@@ -643,7 +645,7 @@ __device__ __noinline__ bool tail_reduce_fused_outofline(const GemmParams& p, in
   return tail_reduce_fused(p, cta, tid, barrier_id, nthreads, abort_flag);
 }
 
-// Shape of the default kernel for a tile height TBM: 128 rows -> 8 warps, 6 stages of 32 KB, one CTA
+// Shape of the inline kernel for a tile height TBM: 128 rows -> 8 warps, 6 stages of 32 KB, one CTA
 // per SM; 64 rows -> 4 warps, 4 stages of 24 KB, two CTAs per SM (they drift out of phase, so one
 // CTA's k-block boundaries and epilogues overlap with the other's arithmetic).
 template <int TBM, int WTM = 64, int TBN = BN>

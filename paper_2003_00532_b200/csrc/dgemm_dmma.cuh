@@ -883,6 +883,9 @@ dgemm_dmma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
 // what the CTA owns at launch, 384 x 168, so 256 x 232 + 128 x 40 must not exceed it). The
 // producer runs up to STAGES k-blocks ahead. TMA staging: lane 0 of the first producer warp issues
 // the copies; generic staging: the four producer warps copy 32 rows of A and 32 columns of B each.
+constexpr int WS_EPI_BATCH = 2;  // 16-row blocks of C loaded per batch in the epilogue (8 loads of 32 bytes in flight
+                                 // per thread; 4 spills heavily at 232 registers, 1 leaves the load latency exposed:
+                                 // rank-k K = 64 1300 us with 1, 1252 us with 2)
 constexpr int WS_PRODUCER_WARPS = 4;
 constexpr int WS_THREADS = (WARPS + WS_PRODUCER_WARPS) * 32;
 constexpr int WS_CONSUMER_REGS = 232;
@@ -1073,7 +1076,7 @@ dgemm_dmma_ws_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
         }
       }
       if (!ok) break;
-      store_tile<1>(p, w, lm, acc);
+      store_tile<WS_EPI_BATCH>(p, w, lm, acc);
       if (p.tail_fused && w.slot >= 0) tail_signal(p, w.trel, tid, 2, WARPS * 32);
     }
     if (ok && p.tail_fused) ok = tail_reduce_fused(p, cta, tid, 2, WARPS * 32, abort_flag);

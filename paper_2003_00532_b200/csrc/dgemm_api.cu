@@ -25,9 +25,24 @@ constexpr size_t kWorkspaceBytes = 640ull * BM * BN * sizeof(double);  // 80 MiB
 constexpr size_t kCounterBytes = 65536;  // in front of the slots: two counters per tail tile (fused tail reduction)
 constexpr unsigned long long kWaitLimitNs = 4000000000ull;            // 4 s per device-side wait
 constexpr int kAutoGeneric = DGEMM_VARIANT_GENERIC;  // what DGEMM_VARIANT_AUTO picks for operands TMA cannot address
-constexpr int kNarrowMaxN = 96;                      // up to this N the 256 x 32 tile (1 to 3 tile columns) beats 128-wide tiles
+// Tile columns of 32 (the 256 x 32 tile, about 83 % of the pipe) against tile columns of 128 (about
+// 97 %): the narrow tile wins when its padded width, weighted by that ratio, is the smaller one
+// (measured 8192 x 64 x 8192: 489 -> 275 us). Not beyond N = 96: the A panel is re-read from L2 once
+// per tile column, and with five columns (6514 x 146 x 4725) that traffic, not the pipe, sets the pace.
+// Tile columns of 64 (128 x 64 tiles, two CTAs per SM, the same warp tiles and bytes per flop as the
+// 64 x 128 tile) when that saves at least a tenth of the padded width: N mod 128 in 1..64 for N up to ~700.
+inline bool half_width_tiles_pay(int64_t N) {
+  const int64_t cols64 = (N + 63) / 64 * 64, cols128 = (N + 127) / 128 * 128;
+  return (double)cols64 * 1.10 <= (double)cols128;
+}
+
+inline bool narrow_tiles_pay(int64_t N) {
+  const int64_t cols32 = (N + 31) / 32 * 32, cols128 = (N + 127) / 128 * 128;
+  return N <= 96 && (double)cols32 * 1.2 < (double)cols128;
+}
 constexpr int kAutoWsMinKblocks = 16;                // warp-specialised kernel: 128-row tiles from K = 256 up, 64-row below
 constexpr double kPackMinFlopPerByte = 64.0;       // pack unaligned operands only if the copy is this cheap
+constexpr double kPackMinFlop = 1.0e9;             // ... and the problem is large enough for two more launches not to show
 constexpr size_t kPackMaxBytes = 2ull << 30;       // ... and the packed copies fit in 2 GiB
 constexpr int64_t kHostBlockRows = 1024;             // dgemm_f64_host: rows of A and C per pipelined block
 constexpr int kTailMinSpan = 1;          // stream-K tail: at least this many k-blocks per CTA
@@ -99,7 +114,8 @@ void launch_tile_kernel(int grid, cudaStream_t stream, const CUtensorMap& map_a,
 template <bool USE_TMA>
 void launch_default_kernel(int bm, int wtm, int grid, cudaStream_t stream, const CUtensorMap& map_a,
                            const CUtensorMap& map_b, const GemmParams& p) {
-  if (bm == 256) launch_tile_kernel<USE_TMA, 256, 64, 32>(grid, stream, map_a, map_b, p);
+  if (p.bn == 64) launch_tile_kernel<USE_TMA, 128, 64, 64>(grid, stream, map_a, map_b, p);
+  else if (bm == 256) launch_tile_kernel<USE_TMA, 256, 64, 32>(grid, stream, map_a, map_b, p);
   else if (bm == 32) launch_tile_kernel<USE_TMA, 32, 32>(grid, stream, map_a, map_b, p);
   else if (bm == 128 && wtm == 64) launch_tile_kernel<USE_TMA, 128, 64>(grid, stream, map_a, map_b, p);
   else if (bm == 128) launch_tile_kernel<USE_TMA, 128, 32>(grid, stream, map_a, map_b, p);
@@ -135,8 +151,9 @@ int device_state(DeviceState** out) {
     if (major != 10) return DGEMM_ERR_DEVICE;
     if (cudaGetSymbolAddress(reinterpret_cast<void**>(&st.status), g_status_word) != cudaSuccess) return DGEMM_ERR_CUDA;
     if (cudaMemset(st.status, 0, sizeof(int)) != cudaSuccess) return DGEMM_ERR_CUDA;
-    int occ[12] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
+    int occ[14] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
     const bool attr_ok =
+        configure_tile_kernel<true, 128, 64, 64>(&occ[12]) && configure_tile_kernel<false, 128, 64, 64>(&occ[13]) &&
         configure_tile_kernel<true, 32, 32>(&occ[10]) && configure_tile_kernel<false, 32, 32>(&occ[11]) &&
         configure_tile_kernel<true, 128, 64>(&occ[0]) && configure_tile_kernel<false, 128, 64>(&occ[1]) &&
         configure_tile_kernel<true, 128, 32>(&occ[2]) && configure_tile_kernel<false, 128, 32>(&occ[3]) &&
@@ -149,7 +166,7 @@ int device_state(DeviceState** out) {
         cudaFuncSetAttribute(dgemm_dmma_ws_kernel<true, 64>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared) == cudaSuccess;
     if (!attr_ok) return DGEMM_ERR_CUDA;
     // the 64-row kernels are meant to run two CTAs per SM; use them only where the device really fits two
-    st.two_ctas_ok = occ[4] >= 2 && occ[5] >= 2 && occ[6] >= 2 && occ[7] >= 2 && occ[8] >= 2 && occ[9] >= 2 && occ[10] >= 2 && occ[11] >= 2;
+    st.two_ctas_ok = occ[4] >= 2 && occ[5] >= 2 && occ[6] >= 2 && occ[7] >= 2 && occ[8] >= 2 && occ[9] >= 2 && occ[10] >= 2 && occ[11] >= 2 && occ[12] >= 2 && occ[13] >= 2;
     if (!g_encode) {
       void* fn = nullptr;
       cudaDriverEntryPointQueryResult qres;
@@ -282,7 +299,8 @@ int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, c
     if (variant == DGEMM_VARIANT_AUTO && (bad_a || bad_b) && !(g_test_flags.load() & DGEMM_TEST_NO_PACKING)) {
       const size_t bytes = ((pack_a || bad_a) ? a_all : 0) + ((pack_b || bad_b) ? b_all : 0);
       const double flop_per_byte = 2.0 * (double)M * (double)N * (double)K / (double)bytes;
-      if (flop_per_byte >= kPackMinFlopPerByte && bytes <= kPackMaxBytes) {
+      if (flop_per_byte >= kPackMinFlopPerByte && bytes <= kPackMaxBytes &&
+          2.0 * (double)M * (double)N * (double)K >= kPackMinFlop) {
         pack_a = pack_a || bad_a;
         pack_b = pack_b || bad_b;
       }
@@ -328,14 +346,14 @@ int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, c
       // The warp-specialised kernel (128 x 128 tiles, one CTA per SM, software-pipelined consumers)
       // has the fastest main loop. The inline kernel with 64-row tiles and two CTAs per SM hides
       // the C round trip of short-K problems better, wastes less on an M just above a multiple of
-      // 64, and has the narrow tile for N <= 96.
+      // 64, and has the narrow tile where narrow_tiles_pay(N).
       // For K < 256 the warp-specialised kernel itself runs 64-row tiles, two CTAs per SM (below).
       const int64_t pad128 = (M + 127) / 128 * 128, pad64 = (M + 63) / 64 * 64;
       const bool short_k = (K + BK - 1) / BK < kAutoWsMinKblocks;
       const int64_t tiles128 = (pad128 / 128) * ((N + BN - 1) / BN);
       // (a handful of tiles: the inline kernel starts faster, 14 against 18 us at 256^3)
       const bool short_rows = M <= 512 && (M + 31) / 32 * 32 < pad64;  // 32-row tiles of the inline kernel, below
-      const bool ws = N > kNarrowMaxN && !short_rows && tiles128 >= 16 && (short_k || (double)pad128 <= 1.03 * (double)pad64);
+      const bool ws = !narrow_tiles_pay(N) && !half_width_tiles_pay(N) && !short_rows && tiles128 >= 16 && (short_k || (double)pad128 <= 1.03 * (double)pad64);
       variant = ws ? DGEMM_VARIANT_TMA_WS : DGEMM_VARIANT_TMA;
     }
   }
@@ -357,19 +375,21 @@ int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, c
   // (generic staging on a problem of many waves is a little faster with the tall tile: half the B copies per thread)
   const int64_t tiles128 = ((M + 127) / 128) * ((N + BN - 1) / BN);
   const bool generic_large = !wants_tma && tiles128 >= 4 * (int64_t)st->sm_count;
-  // narrow problems (N <= 96) use 256 x 32 tiles: four warps stacked in M, little arithmetic on unused columns
+  // narrow problems (see narrow_tiles_pay) use 256 x 32 tiles: four warps stacked in M, little arithmetic on unused columns
   // short problems in M (M <= 32, or a last 64-row tile that is at most half full while M is small) use 32 x 128
   // tiles of four 32 x 32 warp tiles: no arithmetic on unused rows
   const int64_t pad32 = (M + 31) / 32 * 32, pad64m = (M + 63) / 64 * 64;
   const bool short_m = g_variant.load() == DGEMM_VARIANT_AUTO && !ws_variant && M <= 512 && pad32 < pad64m &&
-                       N > kNarrowMaxN && st->two_ctas_ok &&
+                       !narrow_tiles_pay(N) && !half_width_tiles_pay(N) && st->two_ctas_ok &&
                        !(dbg_flags & (DGEMM_TEST_TALL_TILES | DGEMM_TEST_SMALL_WARP_TILES | DGEMM_TEST_WS_TWO_CTAS));
-  const bool narrow = N <= kNarrowMaxN && !ws_variant && !(dbg_flags & (DGEMM_TEST_TALL_TILES | DGEMM_TEST_SMALL_WARP_TILES)) && st->two_ctas_ok;
+  const bool narrow = narrow_tiles_pay(N) && !ws_variant && !(dbg_flags & (DGEMM_TEST_TALL_TILES | DGEMM_TEST_SMALL_WARP_TILES)) && st->two_ctas_ok;
   // warp-specialised with 64-row tiles, two CTAs per SM: the second CTA hides the C round trip of short-K problems
   const bool ws64 = variant == DGEMM_VARIANT_TMA_WS && st->two_ctas_ok &&
                     ((K + BK - 1) / BK < kAutoWsMinKblocks || (dbg_flags & DGEMM_TEST_WS_TWO_CTAS));
-  const int bm = narrow ? 256 : short_m ? 32 : ws64 ? 64 : (ws_variant || generic_large || (dbg_flags & DGEMM_TEST_TALL_TILES) || !st->two_ctas_ok) ? 128 : 64;
-  const int bn = narrow ? 32 : BN;
+  const bool half_width = g_variant.load() == DGEMM_VARIANT_AUTO && !ws_variant && !narrow && half_width_tiles_pay(N) &&
+                          st->two_ctas_ok && !(dbg_flags & (DGEMM_TEST_TALL_TILES | DGEMM_TEST_SMALL_WARP_TILES));
+  const int bm = narrow ? 256 : half_width ? 128 : short_m ? 32 : ws64 ? 64 : (ws_variant || generic_large || (dbg_flags & DGEMM_TEST_TALL_TILES) || !st->two_ctas_ok) ? 128 : 64;
+  const int bn = narrow ? 32 : half_width ? 64 : BN;
 
   const int wtm = (short_m || (dbg_flags & DGEMM_TEST_SMALL_WARP_TILES)) ? 32 : 64;  // rows of a warp tile
 
@@ -391,7 +411,7 @@ int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, c
 
   const int tiles = p.tiles_m * p.tiles_n;
   const int kblocks = (int)((K + BK - 1) / BK);
-  const int sms = st->sm_count * (bm == 128 ? 1 : 2);  // concurrently resident CTAs (128-row tiles: one per SM)
+  const int sms = st->sm_count * ((bm == 128 && bn == 128) ? 1 : 2);  // concurrently resident CTAs (128 x 128 tiles: one per SM)
   const int max_partials = (int)(kWorkspaceBytes / (BM * BN * sizeof(double)));
   p.kblocks = kblocks;
   p.c_prefetch = 1;

@@ -677,12 +677,12 @@ struct TileCfg {
   static constexpr int WARPS_N = TBN / 32;                    // warp grid: (TBM / WTM) x (TBN / 32)
   static constexpr int WARPS_ = (TBM / WTM) * WARPS_N;
   static constexpr int THREADS_ = WARPS_ * 32;
-  static constexpr int CTAS_PER_SM = TBM == 128 ? 1 : 2;
+  static constexpr int CTAS_PER_SM = (TBM == 128 && TBN == 128) ? 1 : 2;
   static constexpr int A_BYTES = TBM * BK * 8;
   static constexpr int B_BYTES = BK * TBN * 8;
   static constexpr int STAGE_BYTES_ = A_BYTES + B_BYTES;
   // as many stages as fit: 6 x 32 KB (one CTA per SM), 4 x 24 KB or 3 x 36 KB (two CTAs per SM)
-  static constexpr int STAGES_ = TBM == 128 ? 6 : (STAGE_BYTES_ <= 24 * 1024 ? 4 : 3);
+  static constexpr int STAGES_ = CTAS_PER_SM == 1 ? 6 : (STAGE_BYTES_ <= 24 * 1024 ? 4 : 3);
   static constexpr int LOOKAHEAD_ = STAGES_ > 3 ? STAGES_ - 2 : STAGES_ - 1;
   static constexpr int SMEM_BYTES_ = STAGES_ * STAGE_BYTES_ + SMEM_ALIGN + 2048;
 };

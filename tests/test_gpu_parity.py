@@ -388,14 +388,16 @@ def test_fused_tail_reduction_is_bit_identical(shape):
 
 
 SKINNY_SHAPES = [(32, 1000, 600), (16, 513, 129), (96, 500, 300), (160, 384, 512), (20, 129, 77), (417, 260, 200),
-                 (1000, 48, 600), (1000, 96, 333), (513, 80, 64), (2000, 64, 2048), (300, 97, 128)]
+                 (1000, 48, 600), (1000, 96, 333), (513, 80, 64), (2000, 64, 2048), (300, 97, 128),
+                 (1000, 146, 300), (700, 130, 520), (257, 416, 100), (129, 190, 64)]
 
 
 @pytest.mark.parametrize("integer", [True, False])
 @pytest.mark.parametrize("shape", SKINNY_SHAPES)
 def test_skinny_shapes_auto(oracle, shape, integer):
-    """Shapes that the library's own choice sends to the 32 x 128 tile (short M) and to one to three
-    columns of 256 x 32 tiles (N <= 96), with aligned operands (TMA staging) and a padded C."""
+    """Shapes that the library's own choice sends to the 32 x 128 tile (short M), to one to three
+    columns of 256 x 32 tiles (N <= 96) and to 128 x 64 tiles (N just above a multiple of 128), with
+    aligned operands (TMA staging) and a padded C."""
     M, N, K = shape
     prob = wl.make_problem(M, N, K, seed=300 + M + N + K, lda=K + 2 + (K & 1), ldb=N + 4 + (N & 1), ldc=N + 7,
                            integer=integer)

@@ -286,27 +286,53 @@ sgemm_ffma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
               make_float4(acc[i][2 * h].x, acc[i][2 * h].y, acc[i][2 * h + 1].x, acc[i][2 * h + 1].y);
       continue;
     }
-    // Epilogue: C += acc, 16-byte accesses where the row segment is aligned and inside N.
+    // Epilogue: C += acc, 16-byte accesses where the row segment is aligned and inside N, else 4-byte
+    // accesses with a bounds check per element. Four rows at a time, all their loads issued before
+    // the first store (interleaved, every load would wait for the store before it, which may alias
+    // as far as the compiler knows, and an edge tile would cost one memory latency per element).
     const bool vec = ((reinterpret_cast<uintptr_t>(p.C) & 15) == 0) && ((p.ldc & 3) == 0);
 #pragma unroll
-    for (int i = 0; i < RPT; ++i) {
-      const int row = tm * TM + ty + 16 * i;
-      if (row >= p.M) continue;
-      float* crow = p.C + (long long)row * p.ldc;
+    for (int i0 = 0; i0 < RPT; i0 += 4) {
+      float4 cin[4][2];
 #pragma unroll
-      for (int h = 0; h < 2; ++h) {
-        const int col = tn * TN + 64 * h + 4 * tx;
-        if (vec && col + 3 < p.N) {
-          float4 c = *reinterpret_cast<const float4*>(crow + col);
+      for (int ii = 0; ii < 4; ++ii) {
+        const int row = tm * TM + ty + 16 * (i0 + ii);
+        const float* crow = p.C + (long long)row * p.ldc;
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const int col = tn * TN + 64 * h + 4 * tx;
+          if (row < p.M && vec && col + 3 < p.N) {
+            cin[ii][h] = *reinterpret_cast<const float4*>(crow + col);
+          } else {
+            cin[ii][h].x = (row < p.M && col + 0 < p.N) ? crow[col + 0] : 0.0f;
+            cin[ii][h].y = (row < p.M && col + 1 < p.N) ? crow[col + 1] : 0.0f;
+            cin[ii][h].z = (row < p.M && col + 2 < p.N) ? crow[col + 2] : 0.0f;
+            cin[ii][h].w = (row < p.M && col + 3 < p.N) ? crow[col + 3] : 0.0f;
+          }
+        }
+      }
+#pragma unroll
+      for (int ii = 0; ii < 4; ++ii) {
+        const int i = i0 + ii;
+        const int row = tm * TM + ty + 16 * i;
+        if (row >= p.M) continue;
+        float* crow = p.C + (long long)row * p.ldc;
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const int col = tn * TN + 64 * h + 4 * tx;
+          float4 c = cin[ii][h];
           c.x += acc[i][2 * h + 0].x;
           c.y += acc[i][2 * h + 0].y;
           c.z += acc[i][2 * h + 1].x;
           c.w += acc[i][2 * h + 1].y;
-          *reinterpret_cast<float4*>(crow + col) = c;
-        } else {
-#pragma unroll
-          for (int e = 0; e < 4; ++e)
-            if (col + e < p.N) crow[col + e] += (e & 1) ? acc[i][2 * h + (e >> 1)].y : acc[i][2 * h + (e >> 1)].x;
+          if (vec && col + 3 < p.N) {
+            *reinterpret_cast<float4*>(crow + col) = c;
+          } else {
+            if (col + 0 < p.N) crow[col + 0] = c.x;
+            if (col + 1 < p.N) crow[col + 1] = c.y;
+            if (col + 2 < p.N) crow[col + 2] = c.z;
+            if (col + 3 < p.N) crow[col + 3] = c.w;
+          }
         }
       }
     }

@@ -793,6 +793,9 @@ dgemm_dmma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
       // dimension. A: 16 consecutive threads copy the 16 k values of one row (8 rows per thread);
       // B: 32 consecutive threads copy 32 consecutive columns of one k row (8 k rows per thread).
       const int m0 = cur_tm * TBM, n0 = cur_tn * TBN, k0 = kb * BK;
+      // a stage that lies wholly inside the matrices (the common case) skips the bounds logic:
+      // the copies are a third of this loader's instructions, the predicates were the rest
+      const bool inside = (m0 + TBM <= p.M) && (n0 + TBN <= p.N) && (k0 + BK <= p.K);
       {
         const int a_k = tid & 15, row0 = tid >> 4;
         const int k = k0 + a_k;
@@ -800,12 +803,20 @@ dgemm_dmma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         const double* src = p.A + (long long)(m0 + row0) * p.lda + k;
         const uint32_t dst_base = sa + ((a_k & 1) << 3);
         constexpr int ROW_STEP = THREADS / 16;
+        if (inside) {
 #pragma unroll
-        for (int i = 0; i < TBM / ROW_STEP; ++i) {
-          const int row = row0 + ROW_STEP * i;
-          const bool in = kin && (m0 + row < p.M);
-          const uint32_t dst = dst_base + row * 128 + (((a_k >> 1) ^ (row & 7)) << 4);
-          ptx::cp_async_8(dst, in ? (const void*)(src + (long long)(ROW_STEP * i) * p.lda) : (const void*)p.A, in ? 8u : 0u);
+          for (int i = 0; i < TBM / ROW_STEP; ++i) {
+            const int row = row0 + ROW_STEP * i;
+            ptx::cp_async_8(dst_base + row * 128 + (((a_k >> 1) ^ (row & 7)) << 4), src + (long long)(ROW_STEP * i) * p.lda, 8u);
+          }
+        } else {
+#pragma unroll
+          for (int i = 0; i < TBM / ROW_STEP; ++i) {
+            const int row = row0 + ROW_STEP * i;
+            const bool in = kin && (m0 + row < p.M);
+            const uint32_t dst = dst_base + row * 128 + (((a_k >> 1) ^ (row & 7)) << 4);
+            ptx::cp_async_8(dst, in ? (const void*)(src + (long long)(ROW_STEP * i) * p.lda) : (const void*)p.A, in ? 8u : 0u);
+          }
         }
       }
       {
@@ -815,12 +826,20 @@ dgemm_dmma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         const uint32_t dst_base = sb + (nn >> 4) * B_BOX_BYTES + ((nn & 1) << 3);
         const int chunk = (nn & 15) >> 1;
         constexpr int K_STEP = THREADS / TBN;
+        if (inside) {
 #pragma unroll
-        for (int i = 0; i < BK / K_STEP; ++i) {
-          const int kk = kk0 + K_STEP * i;
-          const bool in = nin && (k0 + kk < p.K);
-          const uint32_t dst = dst_base + kk * 128 + ((chunk ^ (kk & 7)) << 4);
-          ptx::cp_async_8(dst, in ? (const void*)(src + (long long)(K_STEP * i) * p.ldb) : (const void*)p.B, in ? 8u : 0u);
+          for (int i = 0; i < BK / K_STEP; ++i) {
+            const int kk = kk0 + K_STEP * i;
+            ptx::cp_async_8(dst_base + kk * 128 + ((chunk ^ (kk & 7)) << 4), src + (long long)(K_STEP * i) * p.ldb, 8u);
+          }
+        } else {
+#pragma unroll
+          for (int i = 0; i < BK / K_STEP; ++i) {
+            const int kk = kk0 + K_STEP * i;
+            const bool in = nin && (k0 + kk < p.K);
+            const uint32_t dst = dst_base + kk * 128 + ((chunk ^ (kk & 7)) << 4);
+            ptx::cp_async_8(dst, in ? (const void*)(src + (long long)(K_STEP * i) * p.ldb) : (const void*)p.B, in ? 8u : 0u);
+          }
         }
       }
       ptx::cp_async_mbar_arrive_noinc(fb);

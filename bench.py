@@ -171,7 +171,7 @@ def sgemm_section(dg, torch, sm_max_mhz, sizes=(2048, 4096, 8192)):
     peak = SM_COUNT_B200 * 128 * 2 * sm_max_mhz * 1e6 / 1e12
     out = {"dtype": "f32", "bound": "alu", "peak": peak, "unit": "TFLOP/s",
            "peak_source": "148 SMs x 128 FP32 FMA/clk x 2 x sm_max_mhz; a register-only packed-FMA loop sustains 85 % of it",
-           "kernel": "sgemm_ffma_kernel (TMA staging, 256 x 128 x 32 tiles, 16 x 8 per thread, fma.rn.f32x2)", "shapes": []}
+           "kernel": "sgemm_ffma_kernel<16> (TMA staging, 256 x 128 x 32 tiles, 16 x 8 per thread, fma.rn.f32x2)", "shapes": []}
     call = dg.load_library().sgemm_f32
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     for n in sizes:

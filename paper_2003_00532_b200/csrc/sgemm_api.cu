@@ -55,9 +55,8 @@ int device_state(DeviceState** out) {
     if (major != 10) return DGEMM_ERR_DEVICE;
     if (cudaGetSymbolAddress(reinterpret_cast<void**>(&st.status), g_sgemm_status_word) != cudaSuccess) return DGEMM_ERR_CUDA;
     if (cudaMemset(st.status, 0, sizeof(int)) != cudaSuccess) return DGEMM_ERR_CUDA;
-    if (cudaFuncSetAttribute(sgemm_ffma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess ||
-        cudaFuncSetAttribute(sgemm_ffma_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared) !=
-            cudaSuccess)
+    if (cudaFuncSetAttribute(sgemm_ffma_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<16>::SMEM_BYTES) != cudaSuccess ||
+        cudaFuncSetAttribute(sgemm_ffma_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<8>::SMEM_BYTES) != cudaSuccess)
       return DGEMM_ERR_CUDA;
     if (!g_encode) {
       void* fn = nullptr;
@@ -125,7 +124,7 @@ bool ranges_overlap(const void* p, int64_t pbytes, const void* q, int64_t qbytes
 // Everything that can be decided without touching the device. Returns 1 for "nothing to do".
 int validate(int64_t M, int64_t N, int64_t K, const float* A, int64_t lda, const float* B, int64_t ldb, const float* C,
              int64_t ldc) {
-  const int64_t kMaxDim = (int64_t)INT32_MAX - 2 * TM;
+  const int64_t kMaxDim = (int64_t)INT32_MAX - 2 * MAX_TM;
   if (M < 0 || N < 0 || K < 0 || M > kMaxDim || N > kMaxDim || K > kMaxDim) return DGEMM_ERR_BAD_DIM;
   if (M == 0 || N == 0) return 1;
   if (lda < (K > 0 ? K : 1) || ldb < N || ldc < N) return DGEMM_ERR_BAD_LD;
@@ -134,7 +133,7 @@ int validate(int64_t M, int64_t N, int64_t K, const float* A, int64_t lda, const
   if (((uintptr_t)A | (uintptr_t)B | (uintptr_t)C) & 3) return DGEMM_ERR_ALIGN;
   const int64_t abytes = ((M - 1) * lda + K) * 4, bbytes = ((K - 1) * ldb + N) * 4, cbytes = ((M - 1) * ldc + N) * 4;
   if (ranges_overlap(C, cbytes, A, abytes) || ranges_overlap(C, cbytes, B, bbytes)) return DGEMM_ERR_ALIAS;
-  const int64_t tiles = ((M + TM - 1) / TM) * ((N + TN - 1) / TN);
+  const int64_t tiles = ((M + 127) / 128) * ((N + TN - 1) / TN);
   if (tiles > (int64_t)INT32_MAX / 2) return DGEMM_ERR_BAD_DIM;
   return DGEMM_OK;
 }
@@ -190,6 +189,10 @@ int launch(int64_t M, int64_t N, int64_t K, const float* A, int64_t lda, const f
   Params p;
   memset(&p, 0, sizeof(p));
   p.M = (int)M; p.N = (int)N; p.K = (int)K;
+  // 128-row tiles when 256-row tiles would compute at least a tenth more rows
+  const int64_t pad128 = (M + 127) / 128 * 128, pad256 = (M + 255) / 256 * 256;
+  const int TM = ((double)pad128 * 1.10 <= (double)pad256) ? 128 : 256;
+  p.tm_rows = TM;
   p.tiles_m = (int)((M + TM - 1) / TM);
   p.tiles_n = (int)((N + TN - 1) / TN);
   p.kblocks = (int)((K + TK - 1) / TK);
@@ -209,7 +212,7 @@ int launch(int64_t M, int64_t N, int64_t K, const float* A, int64_t lda, const f
   // whole waves of tiles run data-parallel; the last partial wave is spread evenly over the CTAs
   // (stream-K) when that saves more time than the partial-tile round trip costs
   const int tiles = p.tiles_m * p.tiles_n;
-  const int resident = SGEMM_CTAS * st->sm_count;
+  const int resident = st->sm_count;
   int grid = tiles < resident ? tiles : resident;
   p.dp_tiles = tiles;
   p.tail_tiles = 0;
@@ -227,7 +230,7 @@ int launch(int64_t M, int64_t N, int64_t K, const float* A, int64_t lda, const f
     if (p.dp_tiles == 0) grid = span_ctas < resident ? span_ctas : resident;
     {
       std::lock_guard<std::mutex> lock(g_mutex);
-      if (!st->workspace && cudaMalloc(reinterpret_cast<void**>(&st->workspace), (size_t)2 * resident * TM * TN * sizeof(float)) !=
+      if (!st->workspace && cudaMalloc(reinterpret_cast<void**>(&st->workspace), (size_t)2 * resident * MAX_TM * TN * sizeof(float)) !=
                                 cudaSuccess) {
         (void)cudaGetLastError();
         return DGEMM_ERR_CUDA;
@@ -235,7 +238,8 @@ int launch(int64_t M, int64_t N, int64_t K, const float* A, int64_t lda, const f
     }
     p.partial = st->workspace;
   }
-  launch_pdl(sgemm_ffma_kernel, dim3(grid), dim3(THREADS), (size_t)SMEM_BYTES, stream, map_a, map_b, p);
+  if (TM == 256) launch_pdl(sgemm_ffma_kernel<16>, dim3(grid), dim3(THREADS), (size_t)Cfg<16>::SMEM_BYTES, stream, map_a, map_b, p);
+  else launch_pdl(sgemm_ffma_kernel<8>, dim3(grid), dim3(THREADS), (size_t)Cfg<8>::SMEM_BYTES, stream, map_a, map_b, p);
   if (cudaGetLastError() != cudaSuccess) return DGEMM_ERR_CUDA;
   if (p.tail_tiles > 0 && p.tail_ipc < p.kblocks) {
     launch_pdl(sgemm_tail_reduce_kernel, dim3(p.tail_tiles, 16), dim3(256), 0, stream, p);

@@ -17,23 +17,26 @@ namespace sgemm {
 
 using namespace dgemm::ptx;
 
-#ifndef SGEMM_CTAS
-#define SGEMM_CTAS 1
-#endif
-constexpr int TM = SGEMM_CTAS == 1 ? 256 : 128;  // CTA tile rows
-constexpr int RPT = TM / 16;                       // rows per thread
+// Two tile heights: 256 rows (16 x 8 outputs per thread), and 128 rows (8 x 8 per thread) for
+// problems whose M would leave much of a 256-row tile empty. One CTA per SM either way.
 constexpr int TN = 128;  // CTA tile columns
 constexpr int TK = 32;   // k extent of a stage: 32 floats = one 128-byte swizzle row
 constexpr int THREADS = 256;
 constexpr int WARPS = THREADS / 32;
-constexpr int A_BYTES = TM * TK * 4;        // 16 KiB: 128 rows of 128 bytes
 constexpr int B_BOX_BYTES = TK * 32 * 4;    // 4 KiB: [32 k][32 columns]
 constexpr int B_BYTES = (TN / 32) * B_BOX_BYTES;
-constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-constexpr int STAGES = SGEMM_CTAS == 1 ? 4 : 3;
 constexpr int LOOKAHEAD = 2;                // k-blocks in flight ahead of the arithmetic
 constexpr int SMEM_ALIGN = 1024;
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + SMEM_ALIGN + 256;
+constexpr int MAX_TM = 256;                 // a workspace slot holds MAX_TM x TN floats
+
+template <int RPT>
+struct Cfg {
+  static constexpr int TM = 16 * RPT;                 // CTA tile rows
+  static constexpr int A_BYTES = TM * TK * 4;         // rows of 128 bytes
+  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+  static constexpr int STAGES = 4;
+  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + SMEM_ALIGN + 256;
+};
 constexpr int STATUS_TIMEOUT = -8;          // DGEMM_ERR_TIMEOUT
 
 
@@ -48,7 +51,8 @@ struct Params {
   // per CTA. A span covers at most two tile segments; a segment that is not a whole tile goes to
   // workspace slot 2 * cta + j and sgemm_tail_reduce_kernel adds the slots to C in CTA order.
   int dp_tiles, tail_tiles, tail_ipc;
-  float* partial;      // workspace: slots of TM * TN floats
+  float* partial;      // workspace: slots of MAX_TM * TN floats
+  int tm_rows;         // rows of a CTA tile (256 or 128)
   const float* A;
   const float* B;
   float* C;
@@ -126,9 +130,14 @@ __device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, vola
   return wait_slow(bar, parity, abort_flag, p.wait_limit_ns, p.status);
 }
 
-__global__ void __launch_bounds__(THREADS, SGEMM_CTAS)
+template <int RPT>
+__global__ void __launch_bounds__(THREADS, 1)
 sgemm_ffma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                   const __grid_constant__ Params p) {
+  constexpr int TM = Cfg<RPT>::TM;
+  constexpr int A_BYTES = Cfg<RPT>::A_BYTES;
+  constexpr int STAGE_BYTES = Cfg<RPT>::STAGE_BYTES;
+  constexpr int STAGES = Cfg<RPT>::STAGES;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t pad = (SMEM_ALIGN - (raw & (SMEM_ALIGN - 1))) & (SMEM_ALIGN - 1);
@@ -277,7 +286,7 @@ sgemm_ffma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
 
     if (w.slot >= 0) {
       // a segment of a tail tile: the partial sums go to the workspace (row-major TM x TN)
-      float* dst = p.partial + (long long)w.slot * (TM * TN);
+      float* dst = p.partial + (long long)w.slot * (MAX_TM * TN);
 #pragma unroll
       for (int i = 0; i < RPT; ++i)
 #pragma unroll
@@ -363,6 +372,7 @@ __global__ void sgemm_tail_reduce_kernel(const Params p) {
   if (c_first == c_last) return;  // one CTA had the whole tile and added it straight to C
   int tm, tn;
   tile_to_mn(p, p.dp_tiles + trel, tm, tn);
+  const int TM = p.tm_rows;
   const int chunk = TM * TN / 16;
   const int e0 = blockIdx.y * chunk;
   for (int e = e0 + 4 * threadIdx.x; e < e0 + chunk; e += 4 * blockDim.x) {
@@ -372,7 +382,7 @@ __global__ void sgemm_tail_reduce_kernel(const Params p) {
     float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
     for (int cta = c_first; cta <= c_last; ++cta) {
       const int slot = 2 * cta + ((cta * p.tail_ipc >= lo) ? 0 : 1);
-      const float4 v = *reinterpret_cast<const float4*>(p.partial + (long long)slot * (TM * TN) + e);
+      const float4 v = *reinterpret_cast<const float4*>(p.partial + (long long)slot * (MAX_TM * TN) + e);
       if (cta == c_first) {
         sum = v;
       } else {

@@ -54,6 +54,7 @@ struct DeviceState {
   bool ready = false;
   int sm_count = 0;
   bool two_ctas_ok = false;    // the 64-row kernels fit two CTAs per SM on this device
+  bool ws_ok[3] = {false, false, false};  // register pool of the warp-specialised kernels checked: TMA 128, generic 128, TMA 64
   int* status = nullptr;       // device address of g_status_word
   double* workspace = nullptr; // split-K partial tiles, allocated on first need
   double* pack_buf = nullptr;  // packed copies of unaligned operands, grown on demand
@@ -174,6 +175,25 @@ int device_state(DeviceState** out) {
           qres != cudaDriverEntryPointSuccess || !fn)
         return DGEMM_ERR_CUDA;
       g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+    }
+    // setmaxnreg moves registers inside the pool the CTA owns at launch (threads x registers per
+    // thread as compiled); a consumer warpgroup asking for more than the pool holds would wait for
+    // ever. Check the arithmetic against what the compiler actually allocated before using them.
+    {
+      cudaFuncAttributes fa;
+      auto pool_ok = [&](const void* fn, int threads, int consumer_threads, int producer_regs) {
+        if (cudaFuncGetAttributes(&fa, fn) != cudaSuccess) {
+          (void)cudaGetLastError();
+          return false;
+        }
+        return fa.numRegs * threads >= consumer_threads * WS_CONSUMER_REGS + (threads - consumer_threads) * producer_regs;
+      };
+      st.ws_ok[0] = pool_ok(reinterpret_cast<const void*>(dgemm_dmma_ws_kernel<true, 128>), WsCfg<128>::THREADS_,
+                            WsCfg<128>::CONSUMER_WARPS * 32, WsCfg<128>::PRODUCER_REGS);
+      st.ws_ok[1] = pool_ok(reinterpret_cast<const void*>(dgemm_dmma_ws_kernel<false, 128>), WsCfg<128>::THREADS_,
+                            WsCfg<128>::CONSUMER_WARPS * 32, WsCfg<128>::PRODUCER_REGS);
+      st.ws_ok[2] = pool_ok(reinterpret_cast<const void*>(dgemm_dmma_ws_kernel<true, 64>), WsCfg<64>::THREADS_,
+                            WsCfg<64>::CONSUMER_WARPS * 32, WsCfg<64>::PRODUCER_REGS);
     }
     st.sm_count = sms;
     st.ready = true;
@@ -354,11 +374,13 @@ int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, c
       // (a handful of tiles: the inline kernel starts faster, 14 against 18 us at 256^3)
       const bool short_rows = M <= 512 && (M + 31) / 32 * 32 < pad64;  // 32-row tiles of the inline kernel, below
       const bool ws = !narrow_tiles_pay(N) && !half_width_tiles_pay(N) && !short_rows && tiles128 >= 16 && (short_k || (double)pad128 <= 1.03 * (double)pad64);
-      variant = ws ? DGEMM_VARIANT_TMA_WS : DGEMM_VARIANT_TMA;
+      variant = (ws && st->ws_ok[0] && st->ws_ok[2]) ? DGEMM_VARIANT_TMA_WS : DGEMM_VARIANT_TMA;
     }
   }
   const bool wants_tma = variant == DGEMM_VARIANT_TMA || variant == DGEMM_VARIANT_TMA_WS;
   if (wants_tma && !tma_ok) return DGEMM_ERR_VARIANT;
+  if ((variant == DGEMM_VARIANT_TMA_WS && !(st->ws_ok[0] && st->ws_ok[2])) || (variant == DGEMM_VARIANT_GENERIC_WS && !st->ws_ok[1]))
+    return DGEMM_ERR_VARIANT;
 
   if (variant == DGEMM_VARIANT_NAIVE) {
     if (form.alpha != 1.0 || form.beta != 1.0) return DGEMM_ERR_VARIANT;  // the naive nest is C += A B only

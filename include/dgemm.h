@@ -91,6 +91,10 @@ enum {
  * therefore serialised on the device in stream order only when they use the same stream.
  * Thread-safety: concurrent calls from several host threads are allowed; calls that need the
  * split-K workspace must not overlap on the device.
+ *
+ * The kernels are launched with programmatic stream serialization: their thread blocks may be
+ * scheduled while the previous kernel in `stream` is finishing, but they wait for its completion
+ * (and the visibility of its writes) before they touch global memory, so stream order holds.
  */
 DGEMM_API int dgemm_f64(int64_t M, int64_t N, int64_t K,
               const double *A, int64_t lda,

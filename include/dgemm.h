@@ -219,6 +219,21 @@ enum {
 DGEMM_API int dgemm_set_test_flags(int flags);
 
 /*
+ * What dgemm_f64 would do with an M x N x K problem under the current variant / split-K / test-flag
+ * settings, without touching a device (host logic only; usable on a machine without a GPU):
+ * the kernel and tile the library's heuristics choose and how the work is cut (Section 2.10 of
+ * the paper explores the same kind of choice by hand). `tma_addressable`: non-zero if A and B are
+ * 16-byte aligned with even leading dimensions (or will be after the packing pass). `sm_count`:
+ * streaming multiprocessors to plan for, 0 = 148 (B200); two CTAs per SM are assumed to fit.
+ * Writes 12 ints to `out`: resolved variant, tile rows, tile columns, warp-tile rows, CTAs per
+ * SM, grid size, k-blocks (ceil(K/16)), uniform K split, k-blocks per split, tiles run whole,
+ * tiles of the last partial wave, k-blocks per CTA span of that wave (== k-blocks: not split).
+ * Returns DGEMM_OK, DGEMM_ERR_NULL, DGEMM_ERR_BAD_DIM (a dimension <= 0 or too large) or
+ * DGEMM_ERR_VARIANT (the forced variant cannot run such operands).
+ */
+DGEMM_API int dgemm_plan(int64_t M, int64_t N, int64_t K, int tma_addressable, int sm_count, int *out);
+
+/*
  * Synchronises `stream`, then reads and clears the current device's status word. Returns
  * DGEMM_OK if no kernel reported a problem since the last call, DGEMM_ERR_TIMEOUT if a bounded
  * wait inside a kernel ran out (the kernel then stopped early and C is unspecified), or

@@ -22,6 +22,7 @@ from .binding import (  # noqa: F401
     dgemm_fp64_peak_probe,
     dgemm_last_device_status,
     dgemm_launch_count,
+    dgemm_plan,
     dgemm_selftest_wait_timeout,
     dgemm_set_split_k,
     dgemm_set_test_flags,

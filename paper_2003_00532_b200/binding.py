@@ -74,6 +74,8 @@ def load_library() -> ctypes.CDLL:
             lib.sgemm_f32.restype = ctypes.c_int
             lib.sgemm_last_device_status.argtypes = [vp]
             lib.sgemm_last_device_status.restype = ctypes.c_int
+            lib.dgemm_plan.argtypes = [i64, i64, i64, ctypes.c_int, ctypes.c_int, ctypes.POINTER(ctypes.c_int)]
+            lib.dgemm_plan.restype = ctypes.c_int
             lib.dgemm_f64_static_ws.argtypes = [i64, i64, i64, vp, i64, vp, i64, vp, i64, ctypes.c_int, vp]
             lib.dgemm_f64_static_ws.restype = ctypes.c_int
             lib.dgemm_strerror.argtypes = [ctypes.c_int]
@@ -225,6 +227,20 @@ def dgemm_f64_host(A, B, C, check: bool = True) -> int:
     if check and rc < 0:
         raise DgemmError(rc, "dgemm_f64_host")
     return rc
+
+
+PLAN_FIELDS = ("variant", "bm", "bn", "wtm", "ctas_per_sm", "grid", "kblocks", "split_k", "kblocks_per_split",
+               "dp_tiles", "tail_tiles", "tail_ipc")
+
+
+def dgemm_plan(M: int, N: int, K: int, tma_addressable: bool = True, sm_count: int = 0) -> dict:
+    """The kernel, tile and work decomposition ``dgemm_f64`` would use for this shape under the
+    current settings (host logic only; needs no GPU)."""
+    out = (ctypes.c_int * 12)()
+    rc = load_library().dgemm_plan(int(M), int(N), int(K), int(bool(tma_addressable)), int(sm_count), out)
+    if rc < 0:
+        raise DgemmError(rc, "dgemm_plan")
+    return dict(zip(PLAN_FIELDS, (int(v) for v in out)))
 
 
 def dgemm_strerror(status: int) -> str:

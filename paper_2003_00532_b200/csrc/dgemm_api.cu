@@ -294,6 +294,134 @@ int validate(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, cons
 
 inline unsigned grid_y(int64_t blocks) { return (unsigned)(blocks < 65535 ? blocks : 65535); }
 
+// Everything launch_gemm decides from the shape alone: which kernel, which tile, how the work is
+// cut. A pure function of its arguments (no device, no globals), so that it can be tested on a
+// machine without a GPU through dgemm_plan().
+struct Plan {
+  int status;        // DGEMM_OK, or the error the call would return
+  int variant;       // resolved DGEMM_VARIANT_* (never AUTO)
+  int bm, bn;        // CTA tile
+  int wtm;           // rows of a warp tile (64 or 32)
+  int ctas_per_sm;
+  int grid;          // CTAs launched (all resident at once)
+  int kblocks;       // ceil(K / 16)
+  int split_k, kblocks_per_split;       // phase 1: uniform K split (1 unless forced)
+  int dp_tiles, tail_tiles, tail_ipc;   // whole tiles / tiles of the last partial wave / k-blocks per CTA span
+};
+
+Plan plan_gemm(int64_t M, int64_t N, int64_t K, bool tma_ok, int requested_variant, int dbg_flags, int forced_split,
+               int sm_count, bool two_ctas_ok, const bool ws_ok[3]) {
+  Plan pl;
+  memset(&pl, 0, sizeof(pl));
+  pl.status = DGEMM_OK;
+  int variant = requested_variant;
+  const bool auto_choice = requested_variant == DGEMM_VARIANT_AUTO;
+  const int kblocks = (int)((K + BK - 1) / BK);
+  pl.kblocks = kblocks;
+  if (auto_choice) {
+    if (!tma_ok) {
+      variant = kAutoGeneric;
+    } else {
+      // The warp-specialised kernel (128 x 128 tiles, one CTA per SM, software-pipelined consumers)
+      // has the fastest main loop. The inline kernel with 64-row tiles and two CTAs per SM wastes
+      // less on an M just above a multiple of 64, and has the narrow, half-width and short tiles.
+      // For K < 256 the warp-specialised kernel itself runs 64-row tiles, two CTAs per SM (below).
+      const int64_t pad128 = (M + 127) / 128 * 128, pad64 = (M + 63) / 64 * 64;
+      const bool short_k = kblocks < kAutoWsMinKblocks;
+      const int64_t tiles128 = (pad128 / 128) * ((N + BN - 1) / BN);
+      // (a handful of tiles: the inline kernel starts faster, 14 against 18 us at 256^3)
+      const bool short_rows = M <= 512 && (M + 31) / 32 * 32 < pad64;  // 32-row tiles of the inline kernel, below
+      const bool ws = !narrow_tiles_pay(N) && !half_width_tiles_pay(N) && !short_rows && tiles128 >= 16 &&
+                      (short_k || (double)pad128 <= 1.03 * (double)pad64);
+      variant = (ws && ws_ok[0] && ws_ok[2]) ? DGEMM_VARIANT_TMA_WS : DGEMM_VARIANT_TMA;
+    }
+  }
+  pl.variant = variant;
+  const bool wants_tma = variant == DGEMM_VARIANT_TMA || variant == DGEMM_VARIANT_TMA_WS;
+  if (wants_tma && !tma_ok) { pl.status = DGEMM_ERR_VARIANT; return pl; }
+  if ((variant == DGEMM_VARIANT_TMA_WS && !(ws_ok[0] && ws_ok[2])) || (variant == DGEMM_VARIANT_GENERIC_WS && !ws_ok[1])) {
+    pl.status = DGEMM_ERR_VARIANT;
+    return pl;
+  }
+  if (variant == DGEMM_VARIANT_NAIVE) {
+    pl.bm = 8; pl.bn = 32; pl.wtm = 0; pl.ctas_per_sm = 0;
+    pl.grid = 0; pl.split_k = 1; pl.kblocks_per_split = kblocks;
+    return pl;
+  }
+
+  const bool ws_variant = variant == DGEMM_VARIANT_TMA_WS || variant == DGEMM_VARIANT_GENERIC_WS;
+  // tile height of the chosen kernel: 64 rows with two CTAs per SM (inline kernel; warp-specialised kernel for short K),
+  // 128 rows with one CTA per SM (warp-specialised kernel otherwise, large generic problems, test flag)
+  // (generic staging on a problem of many waves is a little faster with the tall tile: half the B copies per thread)
+  const int64_t tiles128 = ((M + 127) / 128) * ((N + BN - 1) / BN);
+  const bool generic_large = !wants_tma && tiles128 >= 4 * (int64_t)sm_count;
+  const bool plain_tiles = (dbg_flags & (DGEMM_TEST_TALL_TILES | DGEMM_TEST_SMALL_WARP_TILES)) != 0;
+  // narrow problems (see narrow_tiles_pay) use 256 x 32 tiles: four warps stacked in M, little arithmetic on unused columns
+  const bool narrow = narrow_tiles_pay(N) && !ws_variant && !plain_tiles && two_ctas_ok;
+  // N just above a multiple of 128: 128 x 64 tiles
+  const bool half_width = auto_choice && !ws_variant && !narrow && half_width_tiles_pay(N) && two_ctas_ok && !plain_tiles;
+  // short problems in M (M <= 32, or a last 64-row tile that is at most half full while M is small) use 32 x 128
+  // tiles of four 32 x 32 warp tiles: no arithmetic on unused rows
+  const int64_t pad32 = (M + 31) / 32 * 32, pad64m = (M + 63) / 64 * 64;
+  const bool short_m = auto_choice && !ws_variant && !narrow && !half_width && M <= 512 && pad32 < pad64m && two_ctas_ok &&
+                       !plain_tiles && !(dbg_flags & DGEMM_TEST_WS_TWO_CTAS);
+  // warp-specialised with 64-row tiles, two CTAs per SM: the second CTA hides the C round trip of short-K problems
+  const bool ws64 = variant == DGEMM_VARIANT_TMA_WS && two_ctas_ok &&
+                    (kblocks < kAutoWsMinKblocks || (dbg_flags & DGEMM_TEST_WS_TWO_CTAS));
+  const int bm = narrow ? 256 : half_width ? 128 : short_m ? 32 : ws64 ? 64
+                 : (ws_variant || generic_large || (dbg_flags & DGEMM_TEST_TALL_TILES) || !two_ctas_ok) ? 128 : 64;
+  const int bn = narrow ? 32 : half_width ? 64 : BN;
+  pl.bm = bm;
+  pl.bn = bn;
+  pl.wtm = (short_m || (dbg_flags & DGEMM_TEST_SMALL_WARP_TILES)) ? 32 : 64;
+  pl.ctas_per_sm = (bm == 128 && bn == 128) ? 1 : 2;
+
+  const int64_t tiles64 = ((M + bm - 1) / bm) * ((N + bn - 1) / bn);
+  if (tiles64 > (int64_t)INT32_MAX / 2) { pl.status = DGEMM_ERR_BAD_DIM; return pl; }
+  const int tiles = (int)tiles64;
+  const int sms = sm_count * pl.ctas_per_sm;  // concurrently resident CTAs
+  const int max_partials = (int)(kWorkspaceBytes / (BM * BN * sizeof(double)));
+  if (forced_split > 0) {
+    // uniform split-K over all tiles (tests and ablation)
+    int split = forced_split > kblocks ? kblocks : forced_split;
+    if ((int64_t)split * tiles > max_partials) split = max_partials / tiles;
+    if (split < 1) split = 1;
+    pl.kblocks_per_split = (kblocks + split - 1) / split;
+    pl.split_k = (kblocks + pl.kblocks_per_split - 1) / pl.kblocks_per_split;  // no empty partitions
+    pl.dp_tiles = tiles;
+    pl.tail_tiles = 0;
+    pl.tail_ipc = 1;
+    const int64_t units = (int64_t)tiles * pl.split_k;
+    pl.grid = units < sms ? (int)units : sms;
+  } else {
+    // whole waves of tiles run data-parallel; the last partial wave is spread evenly over the SMs
+    // (stream-K) when that saves more time than the partial-tile round trip costs
+    pl.split_k = 1;
+    pl.kblocks_per_split = kblocks;
+    pl.dp_tiles = (tiles / sms) * sms;
+    pl.tail_tiles = tiles - pl.dp_tiles;
+    pl.tail_ipc = kblocks;
+    pl.grid = tiles < sms ? tiles : sms;
+    if (pl.tail_tiles > 0) {
+      const double idle_kblocks = (1.0 - (double)pl.tail_tiles / sms) * kblocks;  // per-SM idle time if run as one wave
+      if (idle_kblocks >= kTailMinSavedKblocks && kblocks >= 2 * kTailMinSpan &&
+          (long long)(pl.tail_tiles + 1) * kblocks < (long long)INT32_MAX) {
+        const long long total = (long long)pl.tail_tiles * kblocks;
+        long long ipc = (total + sms - 1) / sms;
+        if (ipc < kTailMinSpan) ipc = kTailMinSpan;
+        if (ipc > kblocks) ipc = kblocks;
+        pl.tail_ipc = (int)ipc;
+        const int span_ctas = (int)((total + ipc - 1) / ipc);
+        if (pl.dp_tiles == 0) pl.grid = span_ctas < sms ? span_ctas : sms;
+      } else {
+        pl.dp_tiles = tiles;  // run the last wave data-parallel as well
+        pl.tail_tiles = 0;
+      }
+    }
+  }
+  return pl;
+}
+
 // The scalars and operand forms of the general entry point; the defaults are the paper's C += A B.
 struct GemmForm {
   bool ta = false, tb = false;  // A is stored K x M / B is stored N x K and used transposed
@@ -359,28 +487,11 @@ int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, c
     }
   }
   const bool tma_ok = (((uintptr_t)A | (uintptr_t)B) & 15) == 0 && (lda % 2 == 0) && (ldb % 2 == 0);
-  if (variant == DGEMM_VARIANT_AUTO) {
-    if (!tma_ok) {
-      variant = kAutoGeneric;
-    } else {
-      // The warp-specialised kernel (128 x 128 tiles, one CTA per SM, software-pipelined consumers)
-      // has the fastest main loop. The inline kernel with 64-row tiles and two CTAs per SM hides
-      // the C round trip of short-K problems better, wastes less on an M just above a multiple of
-      // 64, and has the narrow tile where narrow_tiles_pay(N).
-      // For K < 256 the warp-specialised kernel itself runs 64-row tiles, two CTAs per SM (below).
-      const int64_t pad128 = (M + 127) / 128 * 128, pad64 = (M + 63) / 64 * 64;
-      const bool short_k = (K + BK - 1) / BK < kAutoWsMinKblocks;
-      const int64_t tiles128 = (pad128 / 128) * ((N + BN - 1) / BN);
-      // (a handful of tiles: the inline kernel starts faster, 14 against 18 us at 256^3)
-      const bool short_rows = M <= 512 && (M + 31) / 32 * 32 < pad64;  // 32-row tiles of the inline kernel, below
-      const bool ws = !narrow_tiles_pay(N) && !half_width_tiles_pay(N) && !short_rows && tiles128 >= 16 && (short_k || (double)pad128 <= 1.03 * (double)pad64);
-      variant = (ws && st->ws_ok[0] && st->ws_ok[2]) ? DGEMM_VARIANT_TMA_WS : DGEMM_VARIANT_TMA;
-    }
-  }
+  const int dbg_flags = g_test_flags.load();
+  const Plan plan = plan_gemm(M, N, K, tma_ok, variant, dbg_flags, g_split_k.load(), st->sm_count, st->two_ctas_ok, st->ws_ok);
+  if (plan.status != DGEMM_OK) return plan.status;
+  variant = plan.variant;
   const bool wants_tma = variant == DGEMM_VARIANT_TMA || variant == DGEMM_VARIANT_TMA_WS;
-  if (wants_tma && !tma_ok) return DGEMM_ERR_VARIANT;
-  if ((variant == DGEMM_VARIANT_TMA_WS && !(st->ws_ok[0] && st->ws_ok[2])) || (variant == DGEMM_VARIANT_GENERIC_WS && !st->ws_ok[1]))
-    return DGEMM_ERR_VARIANT;
 
   if (variant == DGEMM_VARIANT_NAIVE) {
     if (form.alpha != 1.0 || form.beta != 1.0) return DGEMM_ERR_VARIANT;  // the naive nest is C += A B only
@@ -390,31 +501,8 @@ int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, c
     return cudaGetLastError() == cudaSuccess ? DGEMM_OK : DGEMM_ERR_CUDA;
   }
 
-  const int dbg_flags = g_test_flags.load();
-  const bool ws_variant = variant == DGEMM_VARIANT_TMA_WS || variant == DGEMM_VARIANT_GENERIC_WS;
-  // tile height of the chosen kernel: 64 rows with two CTAs per SM (inline kernel; warp-specialised kernel for short K),
-  // 128 rows with one CTA per SM (warp-specialised kernel otherwise, large generic problems, test flag)
-  // (generic staging on a problem of many waves is a little faster with the tall tile: half the B copies per thread)
-  const int64_t tiles128 = ((M + 127) / 128) * ((N + BN - 1) / BN);
-  const bool generic_large = !wants_tma && tiles128 >= 4 * (int64_t)st->sm_count;
-  // narrow problems (see narrow_tiles_pay) use 256 x 32 tiles: four warps stacked in M, little arithmetic on unused columns
-  // short problems in M (M <= 32, or a last 64-row tile that is at most half full while M is small) use 32 x 128
-  // tiles of four 32 x 32 warp tiles: no arithmetic on unused rows
-  const int64_t pad32 = (M + 31) / 32 * 32, pad64m = (M + 63) / 64 * 64;
-  const bool short_m = g_variant.load() == DGEMM_VARIANT_AUTO && !ws_variant && M <= 512 && pad32 < pad64m &&
-                       !narrow_tiles_pay(N) && !half_width_tiles_pay(N) && st->two_ctas_ok &&
-                       !(dbg_flags & (DGEMM_TEST_TALL_TILES | DGEMM_TEST_SMALL_WARP_TILES | DGEMM_TEST_WS_TWO_CTAS));
-  const bool narrow = narrow_tiles_pay(N) && !ws_variant && !(dbg_flags & (DGEMM_TEST_TALL_TILES | DGEMM_TEST_SMALL_WARP_TILES)) && st->two_ctas_ok;
-  // warp-specialised with 64-row tiles, two CTAs per SM: the second CTA hides the C round trip of short-K problems
-  const bool ws64 = variant == DGEMM_VARIANT_TMA_WS && st->two_ctas_ok &&
-                    ((K + BK - 1) / BK < kAutoWsMinKblocks || (dbg_flags & DGEMM_TEST_WS_TWO_CTAS));
-  const bool half_width = g_variant.load() == DGEMM_VARIANT_AUTO && !ws_variant && !narrow && half_width_tiles_pay(N) &&
-                          st->two_ctas_ok && !(dbg_flags & (DGEMM_TEST_TALL_TILES | DGEMM_TEST_SMALL_WARP_TILES));
-  const int bm = narrow ? 256 : half_width ? 128 : short_m ? 32 : ws64 ? 64 : (ws_variant || generic_large || (dbg_flags & DGEMM_TEST_TALL_TILES) || !st->two_ctas_ok) ? 128 : 64;
-  const int bn = narrow ? 32 : half_width ? 64 : BN;
-
-  const int wtm = (short_m || (dbg_flags & DGEMM_TEST_SMALL_WARP_TILES)) ? 32 : 64;  // rows of a warp tile
-
+  const int bm = plan.bm, bn = plan.bn, wtm = plan.wtm;
+  const bool ws64 = variant == DGEMM_VARIANT_TMA_WS && bm == 64;
   GemmParams p;
   memset(&p, 0, sizeof(p));
   p.M = (int)M; p.N = (int)N; p.K = (int)K;
@@ -430,54 +518,16 @@ int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, c
   p.alpha = form.alpha;
   p.beta = form.beta;
   p.load_c = form.beta != 0.0;
-
   const int tiles = p.tiles_m * p.tiles_n;
-  const int kblocks = (int)((K + BK - 1) / BK);
-  const int sms = st->sm_count * ((bm == 128 && bn == 128) ? 1 : 2);  // concurrently resident CTAs (128 x 128 tiles: one per SM)
-  const int max_partials = (int)(kWorkspaceBytes / (BM * BN * sizeof(double)));
+  const int kblocks = plan.kblocks;
   p.kblocks = kblocks;
-  p.c_prefetch = 1;
-  if (dbg_flags & DGEMM_TEST_NO_C_PREFETCH) p.c_prefetch = 0;
-  int grid;
-  const int forced_split = g_split_k.load();
-  if (forced_split > 0) {
-    // uniform split-K over all tiles (tests and ablation)
-    int split = forced_split > kblocks ? kblocks : forced_split;
-    if ((int64_t)split * tiles > max_partials) split = max_partials / tiles;
-    if (split < 1) split = 1;
-    p.kblocks_per_split = (kblocks + split - 1) / split;
-    p.split_k = (kblocks + p.kblocks_per_split - 1) / p.kblocks_per_split;  // no empty partitions
-    p.dp_tiles = tiles;
-    p.tail_tiles = 0;
-    p.tail_ipc = 1;
-    const int units = tiles * p.split_k;
-    grid = units < sms ? units : sms;
-  } else {
-    // whole waves of tiles run data-parallel; the last partial wave is spread evenly over the SMs
-    // (stream-K) when that saves more time than the partial-tile round trip costs
-    p.split_k = 1;
-    p.kblocks_per_split = kblocks;
-    p.dp_tiles = (tiles / sms) * sms;
-    p.tail_tiles = tiles - p.dp_tiles;
-    p.tail_ipc = kblocks;
-    grid = tiles < sms ? tiles : sms;
-    if (p.tail_tiles > 0) {
-      const double idle_kblocks = (1.0 - (double)p.tail_tiles / sms) * kblocks;  // per-SM idle time if run as one wave
-      if (idle_kblocks >= kTailMinSavedKblocks && kblocks >= 2 * kTailMinSpan &&
-          (long long)(p.tail_tiles + 1) * kblocks < (long long)INT32_MAX) {
-        const long long total = (long long)p.tail_tiles * kblocks;
-        long long ipc = (total + sms - 1) / sms;
-        if (ipc < kTailMinSpan) ipc = kTailMinSpan;
-        if (ipc > kblocks) ipc = kblocks;
-        p.tail_ipc = (int)ipc;
-        const int span_ctas = (int)((total + ipc - 1) / ipc);
-        if (p.dp_tiles == 0) grid = span_ctas < sms ? span_ctas : sms;
-      } else {
-        p.dp_tiles = tiles;  // run the last wave data-parallel as well
-        p.tail_tiles = 0;
-      }
-    }
-  }
+  p.c_prefetch = (dbg_flags & DGEMM_TEST_NO_C_PREFETCH) ? 0 : 1;
+  p.split_k = plan.split_k;
+  p.kblocks_per_split = plan.kblocks_per_split;
+  p.dp_tiles = plan.dp_tiles;
+  p.tail_tiles = plan.tail_tiles;
+  p.tail_ipc = plan.tail_ipc;
+  const int grid = plan.grid;
   p.tail_slot_base = 0;
   const bool uses_workspace = p.split_k > 1 || (p.tail_tiles > 0 && p.tail_ipc < kblocks);
   if (uses_workspace) {
@@ -805,6 +855,19 @@ const char* dgemm_strerror(int status) {
 }
 
 int dgemm_version(void) { return 100; /* 0.1.0 */ }
+
+int dgemm_plan(int64_t M, int64_t N, int64_t K, int tma_addressable, int sm_count, int* out) {
+  if (!out) return DGEMM_ERR_NULL;
+  if (M <= 0 || N <= 0 || K <= 0 || M > INT32_MAX - 512 || N > INT32_MAX - 512 || K > INT32_MAX - 512) return DGEMM_ERR_BAD_DIM;
+  const bool ws_ok[3] = {true, true, true};
+  const Plan pl = plan_gemm(M, N, K, tma_addressable != 0, g_variant.load(), g_test_flags.load(), g_split_k.load(),
+                            sm_count > 0 ? sm_count : 148, true, ws_ok);
+  if (pl.status != DGEMM_OK) return pl.status;
+  const int v[12] = {pl.variant, pl.bm, pl.bn, pl.wtm, pl.ctas_per_sm, pl.grid, pl.kblocks, pl.split_k,
+                     pl.kblocks_per_split, pl.dp_tiles, pl.tail_tiles, pl.tail_ipc};
+  for (int i = 0; i < 12; ++i) out[i] = v[i];
+  return DGEMM_OK;
+}
 
 int dgemm_set_variant(int variant) {
   if (variant < DGEMM_VARIANT_AUTO || variant >= DGEMM_VARIANT_COUNT) return DGEMM_ERR_VARIANT;

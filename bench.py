@@ -154,7 +154,9 @@ def other_shapes(dg, torch, peak_tflops, hbm_gbs):
         sweep.append({"n": n, "us": round(ms * 1e3, 1), "tflops": round(tf, 2), "frac_peak": round(tf / peak_tflops, 3)})
     shapes = []
     for (M, N, K, pad) in [(1000, 1537, 777, True), (2088, 2088, 2088, True), (4097, 31, 4099, True),
-                           (2088, 2048, 2048, False), (16384, 16384, 64, False), (16384, 16384, 256, False)]:
+                           (2088, 2048, 2048, False), (16384, 16384, 64, False), (16384, 16384, 256, False),
+                           # skinny shapes (narrow, short and half-width tiles); not BASELINE configs
+                           (8192, 64, 8192, False), (32, 8192, 8192, False), (6514, 146, 4096, False)]:
         ld = (K + 3, N + 5, N + 7) if pad else (K, N, N)
         ms = time_shape(dg, torch, M, N, K, *ld)
         tf = 2.0 * M * N * K / ms / 1e9

@@ -488,7 +488,7 @@ __device__ __forceinline__ void store_tile(const GemmParams& p, const Work& w, c
 #pragma unroll
               for (int np = 0; np < 2; ++np)
 #pragma unroll
-                for (int e = 0; e < 4; ++e) cin[mq][half][np][e] = 0.0;
+                for (int e = 0; e < 4; ++e) cin[mq][half][np][e] = -0.0;  // fma(-0, beta, x) == x for every x, -0 included
         }
 #pragma unroll
         for (int mq = 0; mq < MT_PER_BATCH; ++mq)
@@ -525,7 +525,7 @@ __device__ __forceinline__ void store_tile(const GemmParams& p, const Work& w, c
 #pragma unroll
               for (int e = 0; e < 4; ++e) {
                 const int col = col_base + 16 * np + e;
-                cin[mq][half][np][e] = (p.load_c && row < p.M && col < p.N) ? crow[col] : 0.0;
+                cin[mq][half][np][e] = (p.load_c && row < p.M && col < p.N) ? crow[col] : -0.0;
               }
           }
 #pragma unroll

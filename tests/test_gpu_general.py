@@ -190,3 +190,26 @@ def test_large_forms_sampled(oracle, ta, tb):
     rhs = alpha * (opA @ (opB @ x)) + beta * (C @ x)
     scale = abs(alpha) * (np.abs(opA) @ (np.abs(opB) @ np.abs(x))) + abs(beta) * (np.abs(C) @ np.abs(x))
     assert (np.abs(lhs - rhs) <= 4.0 * (K + N) * U * scale).all()
+
+
+# One shape per kernel / tile configuration the library chooses by itself (checked with dgemm_plan),
+# each with the scalars in the epilogue and, where K is split, in the partial-tile reduction.
+CONFIG_SHAPES = [
+    ((1536, 1408, 512), (dg.DGEMM_VARIANT_TMA_WS, 128, 128)),   # warp-specialised, 128-row tiles
+    ((2048, 2304, 96), (dg.DGEMM_VARIANT_TMA_WS, 64, 128)),     # warp-specialised, 64-row tiles (K < 256)
+    ((1040, 1000, 320), (dg.DGEMM_VARIANT_TMA, 64, 128)),       # inline, 64-row tiles (ragged M)
+    ((700, 64, 520), (dg.DGEMM_VARIANT_TMA, 256, 32)),          # narrow tiles
+    ((96, 1000, 300), (dg.DGEMM_VARIANT_TMA, 32, 128)),         # short tiles
+    ((900, 146, 260), (dg.DGEMM_VARIANT_TMA, 128, 64)),         # half-width tiles
+]
+
+
+@pytest.mark.parametrize("shape,expect", CONFIG_SHAPES)
+@pytest.mark.parametrize("alpha,beta", [(2.0, -3.0), (-1.0, 0.0)])
+def test_scalars_in_every_tile_configuration(oracle, shape, expect, alpha, beta):
+    M, N, K = shape
+    pl = dg.dgemm_plan(M, N, K)
+    assert (pl["variant"], pl["bm"], pl["bn"]) == expect, pl
+    _case(oracle, M, N, K, False, False, alpha, beta, True, seed=sum(shape), pad=(2, 4, 7),
+          c_fill=(np.nan if beta == 0.0 else None))
+    _case(oracle, M, N, K, True, True, alpha, beta, False, seed=sum(shape) + 1)

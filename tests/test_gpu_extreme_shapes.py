@@ -47,3 +47,29 @@ def test_extreme_shapes(oracle, M, N, K, pad, single):
     a64, b64, c64, g64 = (x.astype(np.float64) for x in (A, B, C, got))
     assert np.array_equal(g64.sum(axis=1), c64.sum(axis=1) + a64 @ b64.sum(axis=1))
     assert np.array_equal(g64.sum(axis=0), c64.sum(axis=0) + a64.sum(axis=0) @ b64)
+
+
+@pytest.mark.parametrize("single", [False, True])
+def test_subnormal_values_are_not_flushed(oracle, single):
+    """B holds small integer multiples of the smallest subnormal, A small integers: every product and
+    partial sum is an exactly representable subnormal, so the result must equal the oracle's bit
+    for bit; any flush-to-zero on the way would show."""
+    ntype, ttype = (np.float32, torch.float32) if single else (np.float64, torch.float64)
+    tiny = np.finfo(ntype).smallest_subnormal
+    rng = np.random.Generator(np.random.PCG64(9))
+    M, N, K = 200, 150, 96
+    A = rng.integers(-3, 4, (M, K)).astype(ntype)
+    B = (rng.integers(-3, 4, (K, N)).astype(ntype) * tiny).astype(ntype)
+    C = (rng.integers(-3, 4, (M, N)).astype(ntype) * tiny).astype(ntype)
+    assert np.count_nonzero(B) > 0 and np.abs(B).max() < np.finfo(ntype).tiny
+    dA, dB, dC = (torch.from_numpy(x).cuda() for x in (A, B, C))
+    want = C.copy()
+    if single:
+        dg.sgemm_f32(dA, dB, dC)
+        oracle.sgemm_oracle(A, B, want)
+    else:
+        dg.dgemm_f64(dA, dB, dC)
+        oracle.dgemm_oracle(A, B, want)
+    got = dC.cpu().numpy()
+    assert np.count_nonzero(want) > 0
+    assert got.tobytes() == want.tobytes()

@@ -402,3 +402,19 @@ def test_skinny_shapes_auto(oracle, shape, integer):
     prob = wl.make_problem(M, N, K, seed=300 + M + N + K, lda=K + 2 + (K & 1), ldb=N + 4 + (N & 1), ldc=N + 7,
                            integer=integer)
     _check_full(oracle, prob, run_gpu(prob))
+
+
+@pytest.mark.parametrize("n", [200, 1024])
+def test_a_and_b_may_be_the_same_buffer(oracle, n):
+    """A and B are read only and may alias each other (C += A A); C overlapping either is refused."""
+    rng = np.random.Generator(np.random.PCG64(n))
+    A = rng.integers(-4, 5, (n, n)).astype(np.float64)
+    C = rng.integers(-4, 5, (n, n)).astype(np.float64)
+    dA, dC = torch.from_numpy(A).cuda(), torch.from_numpy(C).cuda()
+    dg.dgemm_f64(dA, dA, dC)
+    assert dg.dgemm_last_device_status() == dg.DGEMM_OK
+    want = C.copy()
+    oracle.dgemm_oracle(A, A.copy(), want)
+    assert np.array_equal(dC.cpu().numpy(), want)
+    assert dg.dgemm_f64(dA, dA, dA, check=False) == dg.binding.DGEMM_ERR_ALIAS
+    assert dg.dgemm_f64_ex(dA, dC, dC, alpha=1.0, beta=0.0, check=False) == dg.binding.DGEMM_ERR_ALIAS

@@ -418,3 +418,27 @@ def test_a_and_b_may_be_the_same_buffer(oracle, n):
     assert np.array_equal(dC.cpu().numpy(), want)
     assert dg.dgemm_f64(dA, dA, dA, check=False) == dg.binding.DGEMM_ERR_ALIAS
     assert dg.dgemm_f64_ex(dA, dC, dC, alpha=1.0, beta=0.0, check=False) == dg.binding.DGEMM_ERR_ALIAS
+
+
+@pytest.mark.parametrize("shape", [(1024, 1024, 1024), (2088, 2048, 2048), (300, 200, 100), (4097, 31, 4099)])
+def test_calls_can_be_captured_into_a_cuda_graph(shape):
+    """After a first call outside capture (allocations, kernel attributes), dgemm_f64 calls recorded
+    in a CUDA graph replay correctly, programmatic launches and reduction kernels included."""
+    M, N, K = shape
+    g0 = torch.Generator(device="cuda").manual_seed(M)
+    A = torch.randint(-3, 4, (M, K), device="cuda", generator=g0).double()
+    B = torch.randint(-3, 4, (K, N), device="cuda", generator=g0).double()
+    C = torch.zeros(M, N, dtype=torch.float64, device="cuda")
+    dg.dgemm_f64(A, B, C)
+    torch.cuda.synchronize()
+    once = C.clone()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        dg.dgemm_f64(A, B, C)
+        dg.dgemm_f64(A, B, C)
+    C.zero_()
+    graph.replay()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert dg.dgemm_last_device_status() == dg.DGEMM_OK
+    assert torch.equal(C, 4 * once)  # exact: small integers

@@ -102,6 +102,16 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
+def host_cores() -> int:
+    """Cores this process may run on. Passed to the oracle explicitly: a launcher may export
+    OMP_NUM_THREADS=1 for every rank (torch.distributed.run does), which would otherwise make the
+    CPU baseline a single-thread figure."""
+    try:
+        return max(1, len(os.sched_getaffinity(0)))
+    except AttributeError:
+        return max(1, os.cpu_count() or 1)
+
+
 def oracle_slab_rate(A, B, C, rows: int, threads: int = 0):
     """Times the oracle (as it stands) on the first `rows` rows of the problem; returns
     (TFLOP/s, seconds, threads used)."""
@@ -110,11 +120,12 @@ def oracle_slab_rate(A, B, C, rows: int, threads: int = 0):
     a = A[:rows].numpy()
     c = C[:rows].clone().numpy()
     b = B.numpy()
+    threads = threads if threads > 0 else host_cores()
     t0 = time.perf_counter()
     oracle.dgemm_oracle(a, b, c, threads)
     dt = time.perf_counter() - t0
     flop = 2.0 * rows * B.shape[0] * B.shape[1]
-    return flop / dt / 1e12, dt, (threads if threads > 0 else oracle.max_threads())
+    return flop / dt / 1e12, dt, threads
 
 
 def time_shape(dg, torch, M, N, K, lda=None, ldb=None, ldc=None, min_ms=40.0):

@@ -46,6 +46,23 @@ def test_validation_needs_no_device():
     assert h(2, 2, 2, a, 1, b, 2, c, 2) == -2
 
 
+def test_sgemm_validation_needs_no_device():
+    f = dg.load_library().sgemm_f32
+    a, b, c = 4096, 8192, 16384  # never dereferenced: every call below fails validation first
+    assert f(-1, 1, 1, a, 1, b, 1, c, 1, None) == -1
+    assert f(2 ** 31, 1, 1, a, 1, b, 1, c, 1, None) == -1
+    assert f(0, 5, 5, None, 5, None, 5, None, 5, None) == 0          # M = 0: nothing inspected
+    assert f(5, 0, 5, None, 5, None, 1, None, 1, None) == 0          # N = 0
+    assert f(2, 2, 2, a, 1, b, 2, c, 2, None) == -2                  # lda < K
+    assert f(2, 2, 2, a, 2, b, 1, c, 2, None) == -2                  # ldb < N
+    assert f(2, 2, 2, a, 2, b, 2, c, 1, None) == -2                  # ldc < N
+    assert f(2, 2, 0, None, 1, None, 2, None, 2, None) == 0          # K = 0: C untouched
+    assert f(2, 2, 2, None, 2, b, 2, c, 2, None) == -3
+    assert f(2, 2, 2, a + 2, 2, b, 2, c, 2, None) == -4              # 4-byte alignment
+    assert f(2, 2, 2, a + 4, 2, b, 2, a + 8, 2, None) == -5          # C inside A (A spans 16 bytes from a + 4)
+    assert f(2, 2, 2, a, 2, b, 2, b - 4, 2, None) == -5              # C's tail reaches B
+
+
 def test_general_form_validation_needs_no_device():
     x = dg.load_library().dgemm_f64_ex
     a, b, c = 4096, 8192, 16384

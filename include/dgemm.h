@@ -52,7 +52,10 @@ enum {
   DGEMM_VARIANT_TMA_WS = 3,     /* as TMA, with a separate producer warpgroup (warp-specialised) and a
                                    software-pipelined consumer loop                              */
   DGEMM_VARIANT_GENERIC_WS = 4, /* as GENERIC, with a separate producer warpgroup                 */
-  DGEMM_VARIANT_COUNT = 5
+  DGEMM_VARIANT_TMA_CLUSTER = 5, /* as TMA on 64 x 128 tiles, K cut over the 1, 2, 4 or 8 CTAs of a
+                                    thread-block cluster, partial tiles added through distributed shared
+                                    memory: one launch, no workspace; what AUTO uses below one wave of tiles */
+  DGEMM_VARIANT_COUNT = 6
 };
 
 /*
@@ -211,10 +214,12 @@ enum {
   DGEMM_TEST_NO_PACKING = 16,   /* never pack unaligned operands: always use the generic staging      */
   DGEMM_TEST_WS_TWO_CTAS = 32,  /* DGEMM_VARIANT_TMA_WS: 64-row tiles, two CTAs per SM, at any K (the
                                    library itself uses that form only for K < 256)                 */
-  DGEMM_TEST_FUSED_TAIL_REDUCE = 64 /* add the partial tiles of the last wave to C inside the GEMM kernel
+  DGEMM_TEST_FUSED_TAIL_REDUCE = 64, /* add the partial tiles of the last wave to C inside the GEMM kernel
                                    (cooperative launch; the CTAs of a tile wait for one another, with
                                    a time limit) instead of in a second kernel: same results bit for
                                    bit, one launch fewer, measured slower                          */
+  DGEMM_TEST_NO_CLUSTER = 128   /* DGEMM_VARIANT_AUTO never picks the cluster split-K kernel: problems
+                                   below one wave of tiles cut K through the workspace instead   */
 };
 DGEMM_API int dgemm_set_test_flags(int flags);
 

@@ -38,6 +38,17 @@ DGEMM_VARIANT_TMA = 1
 DGEMM_VARIANT_GENERIC = 2
 DGEMM_VARIANT_TMA_WS = 3
 DGEMM_VARIANT_GENERIC_WS = 4
+DGEMM_VARIANT_TMA_CLUSTER = 5
+
+# dgemm_set_test_flags bits
+DGEMM_TEST_NO_C_PREFETCH = 1
+DGEMM_TEST_NO_BLOCKED_B = 2
+DGEMM_TEST_TALL_TILES = 4
+DGEMM_TEST_SMALL_WARP_TILES = 8
+DGEMM_TEST_NO_PACKING = 16
+DGEMM_TEST_WS_TWO_CTAS = 32
+DGEMM_TEST_FUSED_TAIL_REDUCE = 64
+DGEMM_TEST_NO_CLUSTER = 128
 
 
 class DgemmError(RuntimeError):

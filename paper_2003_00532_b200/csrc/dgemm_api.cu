@@ -15,6 +15,7 @@
 #include <cuda_runtime.h>
 
 #include "dgemm_dmma.cuh"
+#include "dgemm_cluster.cuh"
 
 namespace {
 
@@ -47,6 +48,12 @@ constexpr size_t kPackMaxBytes = 2ull << 30;       // ... and the packed copies 
 constexpr int64_t kHostBlockRows = 1024;             // dgemm_f64_host: rows of A and C per pipelined block
 constexpr int kTailMinSpan = 1;          // stream-K tail: at least this many k-blocks per CTA
 constexpr double kTailMinSavedKblocks = 5.0;  // use the stream-K tail only if it saves this many k-block times
+// Cluster split-K (one launch, reduction through distributed shared memory) replaces the workspace
+// split on a problem of less than one wave when its critical path, in k-blocks of a 64 x 128 tile
+// (about 1 us each on an SM of its own), is at most this much longer: what the second launch and
+// the workspace round trip cost.
+constexpr int kClusterCreditKblocks = 1;
+constexpr int kClusterMaxKblocks = 8;
 
 __device__ int g_status_word;  // one per device that loads the library
 
@@ -55,6 +62,7 @@ struct DeviceState {
   int sm_count = 0;
   bool two_ctas_ok = false;    // the 64-row kernels fit two CTAs per SM on this device
   bool ws_ok[3] = {false, false, false};  // register pool of the warp-specialised kernels checked: TMA 128, generic 128, TMA 64
+  bool cluster_ok = false;     // a cluster of 8 CTAs of the cluster split-K kernel can be resident
   int* status = nullptr;       // device address of g_status_word
   double* workspace = nullptr; // split-K partial tiles, allocated on first need
   double* pack_buf = nullptr;  // packed copies of unaligned operands, grown on demand
@@ -89,6 +97,28 @@ void launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cu
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
+  cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
+
+// Launch of `grid` CTAs in clusters of `cluster` consecutive CTAs, with programmatic stream
+// serialization as above.
+template <typename... KArgs, typename... Args>
+void launch_cluster_pdl(void (*kernel)(KArgs...), int grid, int cluster, int threads, size_t smem, cudaStream_t stream,
+                        Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(threads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = cluster;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 2;
   cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
 }
 
@@ -194,6 +224,29 @@ int device_state(DeviceState** out) {
                             WsCfg<128>::CONSUMER_WARPS * 32, WsCfg<128>::PRODUCER_REGS);
       st.ws_ok[2] = pool_ok(reinterpret_cast<const void*>(dgemm_dmma_ws_kernel<true, 64>), WsCfg<64>::THREADS_,
                             WsCfg<64>::CONSUMER_WARPS * 32, WsCfg<64>::PRODUCER_REGS);
+    }
+    {
+      // cluster split-K kernel: shared-memory opt-in, then ask whether a full-size cluster fits
+      auto* ck = dgemm_cluster_kernel<64, 64, BN>;
+      using CCfg = TileCfg<64, 64, BN>;
+      st.cluster_ok = false;
+      if (cudaFuncSetAttribute(ck, cudaFuncAttributeMaxDynamicSharedMemorySize, CCfg::SMEM_BYTES_) == cudaSuccess &&
+          cudaFuncSetAttribute(ck, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared) == cudaSuccess) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(CLUSTER_MAX);
+        cfg.blockDim = dim3(CCfg::THREADS_);
+        cfg.dynamicSmemBytes = CCfg::SMEM_BYTES_;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = CLUSTER_MAX;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        int clusters = 0;
+        if (cudaOccupancyMaxActiveClusters(&clusters, ck, &cfg) == cudaSuccess) st.cluster_ok = clusters >= 1;
+      }
+      (void)cudaGetLastError();
     }
     st.sm_count = sms;
     st.ready = true;
@@ -309,8 +362,23 @@ struct Plan {
   int dp_tiles, tail_tiles, tail_ipc;   // whole tiles / tiles of the last partial wave / k-blocks per CTA span
 };
 
+// The cluster split-K kernel on `tiles` 64 x 128 tiles with clusters of s CTAs.
+void fill_cluster_plan(Plan& pl, int tiles, int kblocks, int s) {
+  pl.variant = DGEMM_VARIANT_TMA_CLUSTER;
+  pl.bm = 64;
+  pl.bn = BN;
+  pl.wtm = 64;
+  pl.ctas_per_sm = 2;
+  pl.grid = tiles * s;
+  pl.split_k = s;
+  pl.kblocks_per_split = (kblocks + s - 1) / s;
+  pl.dp_tiles = tiles;
+  pl.tail_tiles = 0;
+  pl.tail_ipc = 1;
+}
+
 Plan plan_gemm(int64_t M, int64_t N, int64_t K, bool tma_ok, int requested_variant, int dbg_flags, int forced_split,
-               int sm_count, bool two_ctas_ok, const bool ws_ok[3]) {
+               int sm_count, bool two_ctas_ok, const bool ws_ok[3], bool cluster_ok) {
   Plan pl;
   memset(&pl, 0, sizeof(pl));
   pl.status = DGEMM_OK;
@@ -337,8 +405,23 @@ Plan plan_gemm(int64_t M, int64_t N, int64_t K, bool tma_ok, int requested_varia
     }
   }
   pl.variant = variant;
-  const bool wants_tma = variant == DGEMM_VARIANT_TMA || variant == DGEMM_VARIANT_TMA_WS;
+  const bool wants_tma = variant == DGEMM_VARIANT_TMA || variant == DGEMM_VARIANT_TMA_WS || variant == DGEMM_VARIANT_TMA_CLUSTER;
   if (wants_tma && !tma_ok) { pl.status = DGEMM_ERR_VARIANT; return pl; }
+  if (variant == DGEMM_VARIANT_TMA_CLUSTER) {
+    // forced: clusters of dgemm_set_split_k() CTAs if that is 1, 2, 4 or 8 (ranks beyond the last
+    // k-block then idle), else the largest size that keeps all CTAs resident at once
+    if (!cluster_ok || !two_ctas_ok) { pl.status = DGEMM_ERR_VARIANT; return pl; }
+    const int64_t tiles64 = ((M + 63) / 64) * ((N + BN - 1) / BN);
+    if (tiles64 > (int64_t)INT32_MAX / 16) { pl.status = DGEMM_ERR_BAD_DIM; return pl; }
+    int s = 1;
+    if (forced_split == 1 || forced_split == 2 || forced_split == 4 || forced_split == 8) {
+      s = forced_split;
+    } else {
+      while (s < CLUSTER_MAX && 2 * s <= kblocks && tiles64 * 2 * s <= 2 * (int64_t)sm_count) s *= 2;
+    }
+    fill_cluster_plan(pl, (int)tiles64, kblocks, s);
+    return pl;
+  }
   if ((variant == DGEMM_VARIANT_TMA_WS && !(ws_ok[0] && ws_ok[2])) || (variant == DGEMM_VARIANT_GENERIC_WS && !ws_ok[1])) {
     pl.status = DGEMM_ERR_VARIANT;
     return pl;
@@ -418,6 +501,32 @@ Plan plan_gemm(int64_t M, int64_t N, int64_t K, bool tma_ok, int requested_varia
         pl.tail_tiles = 0;
       }
     }
+    // Less than one wave of tiles: the cluster kernel cuts K over the CTAs of a cluster and adds the
+    // partial tiles in shared memory, in one launch. Critical paths are compared in k-blocks of a
+    // 64-row tile, doubled where two CTAs of the general kernels share an SM. Runs of more than 8
+    // k-blocks per CTA stay with the general kernels, whose main loops are the faster ones. Any
+    // test flag that asks for a particular tile or reduction keeps the general kernels too.
+    if (auto_choice && wants_tma && cluster_ok && two_ctas_ok && !(dbg_flags & ~(DGEMM_TEST_NO_C_PREFETCH | DGEMM_TEST_NO_BLOCKED_B)) && tiles < sms &&
+        pl.wtm == 64) {  // (every tile shape but the 32-row one: a k-block of each is the same arithmetic)
+      // costs in tenths of a k-block; a pass of the in-cluster reduction (512 element pairs per
+      // CTA) is worth about 0.4 k-blocks, the second launch of the workspace split about one.
+      // Only cluster sizes that leave every CTA an SM of its own: measured, clusters that have to
+      // share SMs lose far more than the factor two of independent CTAs.
+      const bool old_splits = pl.tail_tiles > 0 && pl.tail_ipc < kblocks;
+      const int cost_old = 10 * (old_splits ? pl.tail_ipc : kblocks) * ((bm == 128 || pl.grid > sm_count) ? 2 : 1) +
+                           (old_splits ? 10 * kClusterCreditKblocks : 0);
+      const int64_t tiles_c = ((M + 63) / 64) * ((N + BN - 1) / BN);
+      int best_s = 0, best_cost = INT32_MAX;
+      for (int s = 2; s <= CLUSTER_MAX; s *= 2) {  // (ranks beyond the last k-block still share in the reduction)
+        const int kps = (kblocks + s - 1) / s;
+        const int64_t alone = s >= 4 ? sm_count - sm_count / 8 : sm_count - 4;  // clusters are placed inside a GPC
+        if (tiles_c * s > alone) break;
+        if (kps > kClusterMaxKblocks) continue;
+        const int cost = 10 * kps + 4 * (CLUSTER_MAX / s);
+        if (cost < best_cost) { best_cost = cost; best_s = s; }
+      }
+      if (best_s > 0 && best_cost <= cost_old) fill_cluster_plan(pl, (int)tiles_c, kblocks, best_s);
+    }
   }
   return pl;
 }
@@ -488,10 +597,12 @@ int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, c
   }
   const bool tma_ok = (((uintptr_t)A | (uintptr_t)B) & 15) == 0 && (lda % 2 == 0) && (ldb % 2 == 0);
   const int dbg_flags = g_test_flags.load();
-  const Plan plan = plan_gemm(M, N, K, tma_ok, variant, dbg_flags, g_split_k.load(), st->sm_count, st->two_ctas_ok, st->ws_ok);
+  const Plan plan = plan_gemm(M, N, K, tma_ok, variant, dbg_flags, g_split_k.load(), st->sm_count, st->two_ctas_ok, st->ws_ok,
+                              st->cluster_ok);
   if (plan.status != DGEMM_OK) return plan.status;
   variant = plan.variant;
-  const bool wants_tma = variant == DGEMM_VARIANT_TMA || variant == DGEMM_VARIANT_TMA_WS;
+  const bool wants_tma = variant == DGEMM_VARIANT_TMA || variant == DGEMM_VARIANT_TMA_WS || variant == DGEMM_VARIANT_TMA_CLUSTER;
+  const bool cluster = variant == DGEMM_VARIANT_TMA_CLUSTER;
 
   if (variant == DGEMM_VARIANT_NAIVE) {
     if (form.alpha != 1.0 || form.beta != 1.0) return DGEMM_ERR_VARIANT;  // the naive nest is C += A B only
@@ -529,7 +640,7 @@ int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, c
   p.tail_ipc = plan.tail_ipc;
   const int grid = plan.grid;
   p.tail_slot_base = 0;
-  const bool uses_workspace = p.split_k > 1 || (p.tail_tiles > 0 && p.tail_ipc < kblocks);
+  const bool uses_workspace = !cluster && (p.split_k > 1 || (p.tail_tiles > 0 && p.tail_ipc < kblocks));
   if (uses_workspace) {
     rc = ensure_workspace(st);
     if (rc != DGEMM_OK) return rc;
@@ -549,7 +660,10 @@ int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, c
     if (!make_map(&map_a, A, M, K, lda, BK, bm)) return DGEMM_ERR_CUDA;
     p.b_blocked_map = (!(dbg_flags & DGEMM_TEST_NO_BLOCKED_B) && N % 16 == 0 && make_blocked_map(&map_b, B, K, N, ldb, BK, bn / 16)) ? 1 : 0;
     if (!p.b_blocked_map && !make_map(&map_b, B, K, N, ldb, 16, BK)) return DGEMM_ERR_CUDA;
-    if (ws64)
+    if (cluster)
+      launch_cluster_pdl(dgemm_cluster_kernel<64, 64, BN>, grid, p.split_k, TileCfg<64, 64, BN>::THREADS_,
+                         (size_t)TileCfg<64, 64, BN>::SMEM_BYTES_, stream, map_a, map_b, p);
+    else if (ws64)
       launch_gemm_kernel(dgemm_dmma_ws_kernel<true, 64>, grid, WsCfg<64>::THREADS_, WsCfg<64>::SMEM_BYTES_, stream, map_a, map_b, p);
     else if (variant == DGEMM_VARIANT_TMA_WS)
       launch_gemm_kernel(dgemm_dmma_ws_kernel<true>, grid, WS_THREADS, SMEM_BYTES, stream, map_a, map_b, p);
@@ -563,6 +677,7 @@ int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, c
   }
   g_launches.fetch_add(1);
   if (cudaGetLastError() != cudaSuccess) return DGEMM_ERR_CUDA;
+  if (cluster) return DGEMM_OK;  // the K partitions were added inside the clusters
   if (p.split_k > 1) {
     launch_pdl(dgemm_splitk_reduce_kernel, dim3(tiles, REDUCE_CHUNKS), dim3(REDUCE_THREADS), 0, stream, p);
     g_launches.fetch_add(1);
@@ -861,7 +976,7 @@ int dgemm_plan(int64_t M, int64_t N, int64_t K, int tma_addressable, int sm_coun
   if (M <= 0 || N <= 0 || K <= 0 || M > INT32_MAX - 512 || N > INT32_MAX - 512 || K > INT32_MAX - 512) return DGEMM_ERR_BAD_DIM;
   const bool ws_ok[3] = {true, true, true};
   const Plan pl = plan_gemm(M, N, K, tma_addressable != 0, g_variant.load(), g_test_flags.load(), g_split_k.load(),
-                            sm_count > 0 ? sm_count : 148, true, ws_ok);
+                            sm_count > 0 ? sm_count : 148, true, ws_ok, true);
   if (pl.status != DGEMM_OK) return pl.status;
   const int v[12] = {pl.variant, pl.bm, pl.bn, pl.wtm, pl.ctas_per_sm, pl.grid, pl.kblocks, pl.split_k,
                      pl.kblocks_per_split, pl.dp_tiles, pl.tail_tiles, pl.tail_ipc};
@@ -876,7 +991,7 @@ int dgemm_set_variant(int variant) {
 }
 
 int dgemm_set_test_flags(int flags) {
-  if (flags < 0 || flags > (DGEMM_TEST_NO_C_PREFETCH | DGEMM_TEST_NO_BLOCKED_B | DGEMM_TEST_TALL_TILES | DGEMM_TEST_SMALL_WARP_TILES | DGEMM_TEST_NO_PACKING | DGEMM_TEST_WS_TWO_CTAS | DGEMM_TEST_FUSED_TAIL_REDUCE)) return DGEMM_ERR_VARIANT;
+  if (flags < 0 || flags > (DGEMM_TEST_NO_C_PREFETCH | DGEMM_TEST_NO_BLOCKED_B | DGEMM_TEST_TALL_TILES | DGEMM_TEST_SMALL_WARP_TILES | DGEMM_TEST_NO_PACKING | DGEMM_TEST_WS_TWO_CTAS | DGEMM_TEST_FUSED_TAIL_REDUCE | DGEMM_TEST_NO_CLUSTER)) return DGEMM_ERR_VARIANT;
   g_test_flags.store(flags);
   return DGEMM_OK;
 }

@@ -371,9 +371,13 @@ def test_fused_tail_reduction_is_bit_identical(shape):
     B = torch.rand(K, N, dtype=torch.float64, device="cuda", generator=g) * 2 - 1
     C0 = torch.rand(M, N, dtype=torch.float64, device="cuda", generator=g) * 2 - 1
     ref = C0.clone()
-    n0 = dg.dgemm_launch_count()
-    dg.dgemm_f64(A, B, ref)
-    separate = dg.dgemm_launch_count() - n0
+    dg.dgemm_set_test_flags(dg.DGEMM_TEST_NO_CLUSTER)  # the workspace split also where the cluster kernel would run
+    try:
+        n0 = dg.dgemm_launch_count()
+        dg.dgemm_f64(A, B, ref)
+        separate = dg.dgemm_launch_count() - n0
+    finally:
+        dg.dgemm_set_test_flags(0)
     dg.dgemm_set_test_flags(64)
     try:
         for rep in range(3):

@@ -12,6 +12,7 @@ import pytest
 import paper_2003_00532_b200 as dg
 
 V_TMA, V_GENERIC, V_WS = dg.DGEMM_VARIANT_TMA, dg.DGEMM_VARIANT_GENERIC, dg.DGEMM_VARIANT_TMA_WS
+V_CLUSTER = dg.DGEMM_VARIANT_TMA_CLUSTER
 
 
 @pytest.fixture(autouse=True)
@@ -34,6 +35,11 @@ def _defaults():
     ((16384, 16384, 256), V_WS, 128, 128, 64),
     ((2088, 2048, 2048), V_TMA, 64, 128, 64),      # M just above a multiple of 64 rows less wasteful in 64-row tiles
     ((256, 256, 256), V_TMA, 64, 128, 64),         # a handful of tiles: inline kernel
+    ((128, 128, 128), V_CLUSTER, 64, 128, 64),     # fewer CTAs than SMs even with K cut in 8: split inside clusters
+    ((64, 64, 64), V_CLUSTER, 64, 128, 64),
+    ((512, 512, 256), V_CLUSTER, 64, 128, 64),
+    ((384, 384, 384), V_TMA, 64, 128, 64),         # 18 tiles x 8 would have to share SMs
+    ((128, 128, 4096), V_TMA, 64, 128, 64),        # long K runs stay with the general kernels
     ((4097, 31, 4099), V_TMA, 256, 32, 64),        # narrow N
     ((8192, 96, 8192), V_TMA, 256, 32, 64),
     ((8192, 128, 8192), V_WS, 128, 128, 64),
@@ -68,6 +74,9 @@ def _items(pl, cta):
     for unit in range(cta, units, G):
         tile, ks = divmod(unit, pl["split_k"])
         k0 = ks * pl["kblocks_per_split"]
+        if k0 >= kb:  # a cluster rank beyond the last k-block: no arithmetic, it only shares in the reduction
+            assert pl["variant"] == V_CLUSTER
+            continue
         out.append((tile, k0, min(k0 + pl["kblocks_per_split"], kb), ks * pl["dp_tiles"] + tile if pl["split_k"] > 1 else -1))
     if pl["tail_tiles"]:
         total = pl["tail_tiles"] * kb
@@ -88,7 +97,11 @@ def _check_cover(shape, sm_count=148):
     pl = dg.dgemm_plan(*shape, sm_count=sm_count)
     tiles = -(-shape[0] // pl["bm"]) * -(-shape[1] // pl["bn"])
     assert pl["dp_tiles"] + pl["tail_tiles"] == tiles
-    assert 1 <= pl["grid"] <= sm_count * pl["ctas_per_sm"]
+    if pl["variant"] == V_CLUSTER:  # one CTA per (tile, rank); clusters beyond the resident ones run in turn
+        assert pl["grid"] == tiles * pl["split_k"] and pl["split_k"] in (1, 2, 4, 8) and pl["tail_tiles"] == 0
+        assert (pl["bm"], pl["bn"], pl["ctas_per_sm"]) == (64, 128, 2)
+    else:
+        assert 1 <= pl["grid"] <= sm_count * pl["ctas_per_sm"]
     assert pl["kblocks"] == -(-shape[2] // 16)
     seen = {}
     slots = set()
@@ -118,8 +131,8 @@ def test_cover_random_shapes_and_forced_splits():
     rnd = random.Random(0)
     for i in range(150):
         shape = tuple(rnd.choice([rnd.randint(1, 64), rnd.randint(1, 600), rnd.randint(1, 3000)]) for _ in range(3))
-        dg.dgemm_set_split_k(rnd.choice([0, 0, 0, 2, 3, 7, 64]))
-        dg.dgemm_set_variant(rnd.choice([dg.DGEMM_VARIANT_AUTO, dg.DGEMM_VARIANT_AUTO, V_TMA, V_GENERIC, V_WS]))
+        dg.dgemm_set_split_k(rnd.choice([0, 0, 0, 2, 3, 7, 8, 64]))
+        dg.dgemm_set_variant(rnd.choice([dg.DGEMM_VARIANT_AUTO, dg.DGEMM_VARIANT_AUTO, V_TMA, V_GENERIC, V_WS, V_CLUSTER]))
         dg.dgemm_set_test_flags(rnd.choice([0, 0, 4, 8, 12, 32]))
         _check_cover(shape, sm_count=rnd.choice([148, 132, 8]))
 
@@ -130,3 +143,35 @@ def test_forced_split_has_no_empty_partition():
     assert pl["split_k"] * pl["kblocks_per_split"] >= pl["kblocks"] > (pl["split_k"] - 1) * pl["kblocks_per_split"]
     dg.dgemm_set_split_k(64)
     assert _check_cover((128, 128, 48))["split_k"] == 3   # never more partitions than k-blocks
+
+
+def test_cluster_plan():
+    """AUTO below one wave of tiles: clusters of 2, 4 or 8 CTAs per 64 x 128 tile, every CTA on an SM
+    of its own, at most 8 k-blocks per CTA; the test flag restores the workspace split."""
+    rnd = random.Random(1)
+    picked = 0
+    for i in range(400):
+        shape = (rnd.randint(1, 1200), rnd.randint(1, 1200), rnd.randint(1, 800))
+        pl = dg.dgemm_plan(*shape)
+        if pl["variant"] != V_CLUSTER:
+            continue
+        picked += 1
+        tiles = -(-shape[0] // 64) * -(-shape[1] // 128)
+        assert pl["split_k"] in (2, 4, 8) and pl["grid"] == tiles * pl["split_k"] <= 148
+        assert pl["kblocks_per_split"] == -(-pl["kblocks"] // pl["split_k"]) <= 8
+        _check_cover(shape)
+        dg.dgemm_set_test_flags(dg.DGEMM_TEST_NO_CLUSTER)
+        assert dg.dgemm_plan(*shape)["variant"] != V_CLUSTER
+        dg.dgemm_set_test_flags(0)
+    assert picked > 20
+    assert dg.dgemm_plan(128, 128, 128, sm_count=8)["variant"] != V_CLUSTER  # 16 CTAs do not fit 8 SMs
+    # forced: the cluster size follows dgemm_set_split_k when that is a legal size
+    dg.dgemm_set_variant(V_CLUSTER)
+    for s in (1, 2, 4, 8):
+        dg.dgemm_set_split_k(s)
+        pl = _check_cover((200, 300, 40))   # 3 k-blocks: with 4 and 8 CTAs some ranks idle
+        assert pl["split_k"] == s and pl["kblocks_per_split"] == -(-3 // s)
+    dg.dgemm_set_split_k(0)
+    assert _check_cover((3000, 3000, 3000))["split_k"] == 1  # 1128 tiles: no room for more than one CTA each
+    with pytest.raises(dg.DgemmError):
+        dg.dgemm_plan(128, 128, 128, tma_addressable=False)

@@ -11,6 +11,8 @@ the points of the space are kernels that are all compiled into the library (a va
     inline128 inline load stream, 128 x 128 tiles, one CTA per SM
     small_wt 128 x 128 tiles built from 32 x 32 warp tiles (16 warps)
     generic  8-byte asynchronous copies instead of TMA (any alignment)
+    cluster  64 x 128 tiles, K cut over the CTAs of a thread-block cluster, partial tiles added
+             through distributed shared memory (one launch; what the library uses below one wave)
 
 ``model_ms`` predicts the time of each from the shape (waves of tiles, a K split of the last
 partial wave, the per-tile C round trip, launch latencies); ``autotune`` measures them through the
@@ -51,7 +53,35 @@ CONFIGS: Dict[str, Config] = {
     "inline128": Config("inline128", 1, 4, 128, 128, 1, 0.960),
     "small_wt": Config("small_wt", 1, 4 | 8, 128, 128, 1, 0.945),
     "generic": Config("generic", 2, 16, 64, 128, 2, 0.880, needs_tma=False),
+    "cluster": Config("cluster", 5, 0, 64, 128, 2, 0.775),
 }
+
+KBLOCK_ALONE_US = 1.35   # one k-block of a 64 x 128 tile on an SM the CTA has to itself (measured, long K)
+KBLOCK_SHARED_US = 2.2   # the same with a second CTA on the SM
+CLUSTER_FIXED_US = 4.0   # first copies, two cluster barriers, exit (128^3: 8.8 us per call in a stream)
+CLUSTER_PASS_US = 0.4    # one pass of the in-cluster reduction (512 element pairs per CTA)
+
+
+def cluster_size(M: int, N: int, K: int) -> int:
+    """Cluster size of the forced cluster variant: the largest of 1, 2, 4, 8 that keeps all CTAs
+    resident at once and gives every CTA a k-block."""
+    tiles, kb = math.ceil(M / 64) * math.ceil(N / 128), math.ceil(K / BK)
+    s = 1
+    while s < 8 and 2 * s <= kb and tiles * 2 * s <= 2 * SM_COUNT:
+        s *= 2
+    return s
+
+
+def model_cluster_ms(M: int, N: int, K: int) -> float:
+    tiles, kb = math.ceil(M / 64) * math.ceil(N / 128), math.ceil(K / BK)
+    s = cluster_size(M, N, K)
+    ctas = tiles * s
+    waves = math.ceil(ctas / (2 * SM_COUNT))
+    per_kb = KBLOCK_SHARED_US if ctas > SM_COUNT else KBLOCK_ALONE_US
+    t = waves * (math.ceil(kb / s) * per_kb + (8 // s) * CLUSTER_PASS_US) + CLUSTER_FIXED_US + LAUNCH_US
+    t_pipe = 2.0 * M * N * K / (PEAK_TFLOPS * 1e12) * 1e6
+    t_hbm = 8.0 * (M * K + K * N + 2.0 * M * N) / (HBM_GBS * 1e9) * 1e6
+    return max(t, t_pipe, t_hbm) * 1e-3
 
 
 def register_budget(bm: int, bn: int, warps: int, wt_m: int = 64, wt_n: int = 32) -> dict:
@@ -74,6 +104,8 @@ def model_ms(M: int, N: int, K: int, cfg: Config, ldc_aligned: bool = True) -> f
     steady-state efficiency) + exposed C round trips + the reduction pass when tiles are split.
     Whole waves run data-parallel; the last partial wave is spread evenly (stream-K), as the
     library does."""
+    if cfg.name == "cluster":
+        return model_cluster_ms(M, N, K)
     tiles_m, tiles_n = math.ceil(M / cfg.bm), math.ceil(N / cfg.bn)
     tiles = tiles_m * tiles_n
     kblocks = math.ceil(K / BK)

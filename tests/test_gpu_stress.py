@@ -87,3 +87,30 @@ def _square_repeated(oracle, n):
             first = C
         else:
             assert torch.equal(first, C), f"run {rep} differs from run 0"
+
+
+@pytest.mark.parametrize("flags", [0, 2])
+@pytest.mark.parametrize("split", [1, 2, 8])
+def test_cluster_kernel_repeated_runs_bit_exact(oracle, flags, split):
+    """The cluster split-K kernel with long K runs per CTA (every stage refilled many times, which
+    the library's own choice never asks of it) and more clusters than are resident at once."""
+    M, N, K = 1000, 1100, 1000
+    prob = wl.make_problem(M, N, K, seed=11, integer=True)
+    want = prob.C.clone().numpy()
+    oracle.dgemm_oracle(prob.A.numpy(), prob.B.numpy(), want)
+    want_dev = torch.from_numpy(want).cuda()
+    A, B, C0 = prob.A.cuda(), prob.B.cuda(), prob.C.cuda()
+    dg.dgemm_set_test_flags(flags)
+    dg.dgemm_set_variant(dg.DGEMM_VARIANT_TMA_CLUSTER)
+    dg.dgemm_set_split_k(split)
+    try:
+        for rep in range(10):
+            C = C0.clone()
+            dg.dgemm_f64(A, B, C)
+            assert dg.dgemm_last_device_status() == 0
+            wrong = int((C != want_dev).sum())
+            assert wrong == 0, f"run {rep}: {wrong} wrong entries (flags {flags}, clusters of {split})"
+    finally:
+        dg.dgemm_set_test_flags(0)
+        dg.dgemm_set_variant(dg.DGEMM_VARIANT_AUTO)
+        dg.dgemm_set_split_k(0)

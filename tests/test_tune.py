@@ -29,6 +29,10 @@ def test_model_orders_the_known_cases():
     # rank-k update, K = 64: the C round trip dominates and two CTAs per SM hide it
     rk = {r["config"]: r["model_ms"] for r in tune.predict(16384, 16384, 64)}
     assert min(rk["ws64"], rk["inline64"]) < rk["ws128"]
+    # a problem of two tiles: K cut inside clusters, one launch, beats every persistent configuration
+    small = tune.predict(128, 128, 128)
+    assert small[0]["config"] == "cluster" and abs(small[0]["model_ms"] - 0.0088) / 0.0088 < 0.25
+    assert tune.cluster_size(128, 128, 128) == 8 and tune.cluster_size(3000, 3000, 3000) == 1
     # monotone in every dimension
     base = tune.model_ms(2048, 2048, 2048, tune.CONFIGS["ws128"])
     assert tune.model_ms(4096, 2048, 2048, tune.CONFIGS["ws128"]) > base

@@ -41,6 +41,7 @@ inline bool narrow_tiles_pay(int64_t N) {
   const int64_t cols32 = (N + 31) / 32 * 32, cols128 = (N + 127) / 128 * 128;
   return N <= 96 && (double)cols32 * 1.2 < (double)cols128;
 }
+constexpr int kAutoWs64MaxKblocksPerCta = 256;     // ... and its 64-row form instead of the inline kernel up to this much work
 constexpr int kAutoWsMinKblocks = 16;                // warp-specialised kernel: 128-row tiles from K = 256 up, 64-row below
 constexpr double kPackMinFlopPerByte = 64.0;       // pack unaligned operands only if the copy is this cheap
 constexpr double kPackMinFlop = 1.0e9;             // ... and the problem is large enough for two more launches not to show
@@ -386,6 +387,7 @@ Plan plan_gemm(int64_t M, int64_t N, int64_t K, bool tma_ok, int requested_varia
   const bool auto_choice = requested_variant == DGEMM_VARIANT_AUTO;
   const int kblocks = (int)((K + BK - 1) / BK);
   pl.kblocks = kblocks;
+  bool auto_ws64 = false;  // AUTO wants the warp-specialised kernel in its 64-row form although K >= 256
   if (auto_choice) {
     if (!tma_ok) {
       variant = kAutoGeneric;
@@ -399,9 +401,17 @@ Plan plan_gemm(int64_t M, int64_t N, int64_t K, bool tma_ok, int requested_varia
       const int64_t tiles128 = (pad128 / 128) * ((N + BN - 1) / BN);
       // (a handful of tiles: the inline kernel starts faster, 14 against 18 us at 256^3)
       const bool short_rows = M <= 512 && (M + 31) / 32 * 32 < pad64;  // 32-row tiles of the inline kernel, below
-      const bool ws = !narrow_tiles_pay(N) && !half_width_tiles_pay(N) && !short_rows && tiles128 >= 16 &&
-                      (short_k || (double)pad128 <= 1.03 * (double)pad64);
-      variant = (ws && ws_ok[0] && ws_ok[2]) ? DGEMM_VARIANT_TMA_WS : DGEMM_VARIANT_TMA;
+      const bool std_tile = !narrow_tiles_pay(N) && !half_width_tiles_pay(N) && !short_rows;
+      const bool ws = std_tile && tiles128 >= 16 && (short_k || (double)pad128 <= 1.03 * (double)pad64);
+      // Where 64-row tiles are the better fit, the warp-specialised kernel's 64-row form beats the
+      // inline kernel on problems of up to a few hundred microseconds (26 random shapes: 4 % in the
+      // geometric mean, up to 11 %; its producer warps keep the stages full across the short tiles'
+      // epilogues), and loses up to 0.8 % on long ones: taken up to 256 k-blocks per resident CTA.
+      if (!ws && std_tile && two_ctas_ok && ws_ok[2]) {
+        const int64_t tiles64 = (pad64 / 64) * ((N + BN - 1) / BN);
+        auto_ws64 = tiles64 * kblocks <= (int64_t)kAutoWs64MaxKblocksPerCta * 2 * sm_count;
+      }
+      variant = ((ws && ws_ok[0] && ws_ok[2]) || auto_ws64) ? DGEMM_VARIANT_TMA_WS : DGEMM_VARIANT_TMA;
     }
   }
   pl.variant = variant;
@@ -450,7 +460,7 @@ Plan plan_gemm(int64_t M, int64_t N, int64_t K, bool tma_ok, int requested_varia
                        !plain_tiles && !(dbg_flags & DGEMM_TEST_WS_TWO_CTAS);
   // warp-specialised with 64-row tiles, two CTAs per SM: the second CTA hides the C round trip of short-K problems
   const bool ws64 = variant == DGEMM_VARIANT_TMA_WS && two_ctas_ok &&
-                    (kblocks < kAutoWsMinKblocks || (dbg_flags & DGEMM_TEST_WS_TWO_CTAS));
+                    (kblocks < kAutoWsMinKblocks || auto_ws64 || (dbg_flags & DGEMM_TEST_WS_TWO_CTAS));
   const int bm = narrow ? 256 : half_width ? 128 : short_m ? 32 : ws64 ? 64
                  : (ws_variant || generic_large || (dbg_flags & DGEMM_TEST_TALL_TILES) || !two_ctas_ok) ? 128 : 64;
   const int bn = narrow ? 32 : half_width ? 64 : BN;
@@ -513,8 +523,10 @@ Plan plan_gemm(int64_t M, int64_t N, int64_t K, bool tma_ok, int requested_varia
       // Only cluster sizes that leave every CTA an SM of its own: measured, clusters that have to
       // share SMs lose far more than the factor two of independent CTAs.
       const bool old_splits = pl.tail_tiles > 0 && pl.tail_ipc < kblocks;
-      const int cost_old = 10 * (old_splits ? pl.tail_ipc : kblocks) * ((bm == 128 || pl.grid > sm_count) ? 2 : 1) +
-                           (old_splits ? 10 * kClusterCreditKblocks : 0);
+      const int path_old = 10 * (old_splits ? pl.tail_ipc : kblocks) * ((bm == 128 || pl.grid > sm_count) ? 2 : 1);
+      // (one k-block per CTA and the reduction kernel behind it is the general kernels' floor, 7.8 us
+      // at 128^3, and below the cluster kernel's, 8.7 us: no credit there)
+      const int cost_old = path_old + ((old_splits && path_old >= 20) ? 10 * kClusterCreditKblocks : 0);
       const int64_t tiles_c = ((M + 63) / 64) * ((N + BN - 1) / BN);
       int best_s = 0, best_cost = INT32_MAX;
       for (int s = 2; s <= CLUSTER_MAX; s *= 2) {  // (ranks beyond the last k-block still share in the reduction)

@@ -48,7 +48,11 @@ constexpr int B_STAGE_BYTES = BK * BN * 8;  // 16 KiB: 8 boxes of [16 k][16 n] d
 constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
 constexpr int B_BOX_BYTES = BK * 16 * 8;    // 2 KiB
 constexpr int SMEM_ALIGN = 1024;            // swizzle pattern repeats every 1024 bytes
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + SMEM_ALIGN + 1024;  // + barriers, abort flag, work-item words
+// Per-warp staging buffer of the epilogue for C tiles that cannot be accessed 32 bytes at a time
+// (edge tiles, C not 32-byte aligned): 8 rows of 32 doubles, 16 bytes of padding per row.
+constexpr int EPI_STRIDE = 32 * 8 + 16;
+constexpr int EPI_WARP_BYTES = 8 * EPI_STRIDE;
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + SMEM_ALIGN + 1024 + WARPS * EPI_WARP_BYTES;  // + barriers, abort flag, work-item words, epilogue staging
 constexpr int STATUS_TIMEOUT = -8;          // DGEMM_ERR_TIMEOUT
 constexpr int C_PREFETCH_KBLOCKS = 8;       // C tile is requested into L2 this many k-blocks before the tile ends
 
@@ -433,8 +437,9 @@ __device__ __forceinline__ void release_stage(uint32_t empty_bar_s, int lane) {
 
 // Epilogue of one work item: adds the accumulators to the C tile (or stores them as a partial tile
 // in the workspace when the item covers only part of K).
-template <int MT_PER_BATCH, int MT = 4>
-__device__ __forceinline__ void store_tile(const GemmParams& p, const Work& w, const LaneMap& m, double (&acc)[MT][4][4]) {
+template <int MT_PER_BATCH, int MT = 4, bool STAGED = false>
+__device__ __forceinline__ void store_tile(const GemmParams& p, const Work& w, const LaneMap& m, double (&acc)[MT][4][4],
+                                           uint32_t epi_buf = 0) {
   const int tm = w.tm, tn = w.tn;
   // This lane owns, for each mt, half (rows +0 / +8) and np, four consecutive
   // columns n = 32wn + 16np + 4t + {0,1,2,3} = {nt=2np:c0, nt=2np+1:c0, nt=2np:c1, nt=2np+1:c1}
@@ -503,6 +508,57 @@ __device__ __forceinline__ void store_tile(const GemmParams& p, const Work& w, c
                           fma(cin[mq][half][np][1], p.beta, acc[mt][2 * np + 1][2 * half]),
                           fma(cin[mq][half][np][2], p.beta, acc[mt][2 * np][2 * half + 1]),
                           fma(cin[mq][half][np][3], p.beta, acc[mt][2 * np + 1][2 * half + 1]));
+          }
+      }
+    } else if constexpr (STAGED) {
+      // Edge tiles and C that is not 32-byte aligned, through this warp's staging buffer: 8 rows of
+      // the warp tile at a time go to shared memory in row-major order and come back with lane L
+      // holding column L, so that every global access of the warp is one 256-byte row segment
+      // (8 or 9 sectors) instead of 32 scattered 8-byte pieces (32 sectors, a quarter of each
+      // used: 4096 x 4096 x 64 with ldc = 4098 ran 125 us that way against 89 us with ldc = 4096).
+      const int lane = 4 * m.g + m.t;
+      const int col = tn * p.bn + 32 * m.wn + lane;
+      const bool col_in = col < p.N;
+      const uint32_t wr = epi_buf + m.rm * EPI_STRIDE + m.t * 32;  // this lane's 4 columns of row rm (np adds 128 bytes)
+      const uint32_t rd = epi_buf + lane * 8;                     // column `lane` of row j at + j * EPI_STRIDE
+      // Per batch of MT_PER_BATCH 16-row blocks: all old C values are requested first (as many bytes
+      // in flight per warp as on the 32-byte path), the accumulators go through the buffer while
+      // those loads are under way, and every store comes after every load of the batch (a load
+      // behind a store would have to wait for it: they may alias as far as the compiler knows).
+#pragma unroll
+      for (int mp = 0; mp < MT / MT_PER_BATCH; ++mp) {
+        double cin[MT_PER_BATCH][2][8];
+        const int row0 = tm * p.bm + m.row0 + 16 * MT_PER_BATCH * mp;
+        double* cbase = p.C + (long long)row0 * p.ldc + col;
+#pragma unroll
+        for (int mq = 0; mq < MT_PER_BATCH; ++mq)
+#pragma unroll
+          for (int half = 0; half < 2; ++half)
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              const int r = 16 * mq + 8 * half + j;
+              cin[mq][half][j] = (p.load_c && col_in && row0 + r < p.M) ? cbase[(long long)r * p.ldc] : -0.0;
+            }
+#pragma unroll
+        for (int mq = 0; mq < MT_PER_BATCH; ++mq)
+#pragma unroll
+          for (int half = 0; half < 2; ++half) {
+            const int mt = MT_PER_BATCH * mp + mq;
+#pragma unroll
+            for (int np = 0; np < 2; ++np) {
+              ptx::sts128(wr + np * 128, acc[mt][2 * np][2 * half], acc[mt][2 * np + 1][2 * half]);
+              ptx::sts128(wr + np * 128 + 16, acc[mt][2 * np][2 * half + 1], acc[mt][2 * np + 1][2 * half + 1]);
+            }
+            __syncwarp();
+            double v[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) v[j] = ptx::lds64_f64(rd + j * EPI_STRIDE);
+            __syncwarp();
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              const int r = 16 * mq + 8 * half + j;
+              if (col_in && row0 + r < p.M) cbase[(long long)r * p.ldc] = fma(cin[mq][half][j], p.beta, v[j]);
+            }
           }
       }
     } else {
@@ -684,7 +740,11 @@ struct TileCfg {
   // as many stages as fit: 6 x 32 KB (one CTA per SM), 4 x 24 KB or 3 x 36 KB (two CTAs per SM)
   static constexpr int STAGES_ = CTAS_PER_SM == 1 ? 6 : (STAGE_BYTES_ <= 24 * 1024 ? 4 : 3);
   static constexpr int LOOKAHEAD_ = STAGES_ > 3 ? STAGES_ - 2 : STAGES_ - 1;
-  static constexpr int SMEM_BYTES_ = STAGES_ * STAGE_BYTES_ + SMEM_ALIGN + 2048;
+  // epilogue staging where it fits: not next to the three 36 KB stages of the 256 x 32 tile, nor with
+  // the 8 or 16 warps of the tiles built from 32 x 32 warp tiles (they keep the scattered 8-byte accesses)
+  static constexpr bool EPI_STAGED = !(TBM == 256 || (WTM == 32 && TBM >= 64));
+  static constexpr int EPI_OFFSET = STAGES_ * STAGE_BYTES_ + 2048;  // from the first stage
+  static constexpr int SMEM_BYTES_ = STAGES_ * STAGE_BYTES_ + SMEM_ALIGN + 2048 + (EPI_STAGED ? WARPS_ * EPI_WARP_BYTES : 0);
 };
 
 template <bool USE_TMA, int TBM, int WTM = 64, int TBN = BN>
@@ -898,7 +958,8 @@ dgemm_dmma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     }
     if (!ok) break;
 
-    store_tile<(MT >= 4 ? 2 : 1), MT>(p, w, lm, acc);
+    store_tile<(MT >= 4 ? 2 : 1), MT, TileCfg<TBM, WTM, TBN>::EPI_STAGED>(
+        p, w, lm, acc, tiles_u32 + TileCfg<TBM, WTM, TBN>::EPI_OFFSET + warp * EPI_WARP_BYTES);
     if (p.tail_fused && w.slot >= 0) tail_signal(p, w.trel, tid, 0, THREADS);
   }
   if (ok && p.tail_fused) ok = tail_reduce_fused_outofline(p, cta, tid, 0, THREADS, abort_flag);
@@ -941,7 +1002,8 @@ struct WsCfg {
   static constexpr int A_BYTES = TBM * BK * 8;
   static constexpr int STAGE_BYTES_ = A_BYTES + B_STAGE_BYTES;
   static constexpr int STAGES_ = TBM == 128 ? 6 : 4;
-  static constexpr int SMEM_BYTES_ = STAGES_ * STAGE_BYTES_ + SMEM_ALIGN + 2048;
+  static constexpr int EPI_OFFSET = STAGES_ * STAGE_BYTES_ + 1024;  // epilogue staging, from the first stage
+  static constexpr int SMEM_BYTES_ = STAGES_ * STAGE_BYTES_ + SMEM_ALIGN + 2048 + CONSUMER_WARPS * EPI_WARP_BYTES;
   // register pool = THREADS_ x registers at launch (168 or 128): consumers x 232 + 128 x producers
   static constexpr int PRODUCER_REGS = TBM == 128 ? WS_PRODUCER_REGS : 24;
 };
@@ -1118,7 +1180,7 @@ dgemm_dmma_ws_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
         }
       }
       if (!ok) break;
-      store_tile<WS_EPI_BATCH>(p, w, lm, acc);
+      store_tile<WS_EPI_BATCH, 4, true>(p, w, lm, acc, tiles_u32 + WsCfg<TBM>::EPI_OFFSET + warp * EPI_WARP_BYTES);
       if (p.tail_fused && w.slot >= 0) tail_signal(p, w.trel, tid, 2, WARPS * 32);
     }
     if (ok && p.tail_fused) ok = tail_reduce_fused(p, cta, tid, 2, WARPS * 32, abort_flag);

@@ -102,7 +102,7 @@ def test_cluster_split_equals_workspace_split_bit_for_bit(shape, split):
     assert out[0].tobytes() == out[1].tobytes()
 
 
-@pytest.mark.parametrize("shape", [(32, 32, 32), (64, 64, 64), (128, 128, 128), (128, 80, 32), (48, 480, 48),
+@pytest.mark.parametrize("shape", [(32, 32, 32), (64, 64, 64), (192, 192, 192), (128, 80, 32), (48, 480, 48),
                                    (320, 320, 320), (512, 512, 256), (1936, 240, 96), (558, 26, 26)])
 @pytest.mark.parametrize("integer", [True, False])
 def test_auto_picks_cluster_kernel_on_small_problems(oracle, shape, integer):

@@ -197,7 +197,7 @@ def test_large_forms_sampled(oracle, ta, tb):
 CONFIG_SHAPES = [
     ((1536, 1408, 512), (dg.DGEMM_VARIANT_TMA_WS, 128, 128)),   # warp-specialised, 128-row tiles
     ((2048, 2304, 96), (dg.DGEMM_VARIANT_TMA_WS, 64, 128)),     # warp-specialised, 64-row tiles (K < 256)
-    ((1040, 1000, 320), (dg.DGEMM_VARIANT_TMA, 64, 128)),       # inline, 64-row tiles (ragged M)
+    ((1040, 1000, 320), (dg.DGEMM_VARIANT_TMA_WS, 64, 128)),    # the same for a ragged M on a problem of moderate size
     ((700, 64, 520), (dg.DGEMM_VARIANT_TMA, 256, 32)),          # narrow tiles
     ((96, 1000, 300), (dg.DGEMM_VARIANT_TMA, 32, 128)),         # short tiles
     ((900, 146, 260), (dg.DGEMM_VARIANT_TMA, 128, 64)),         # half-width tiles
@@ -213,3 +213,14 @@ def test_scalars_in_every_tile_configuration(oracle, shape, expect, alpha, beta)
     _case(oracle, M, N, K, False, False, alpha, beta, True, seed=sum(shape), pad=(2, 4, 7),
           c_fill=(np.nan if beta == 0.0 else None))
     _case(oracle, M, N, K, True, True, alpha, beta, False, seed=sum(shape) + 1)
+
+
+@pytest.mark.parametrize("alpha,beta", [(2.0, -3.0), (-1.0, 0.0)])
+def test_scalars_in_the_inline_kernel_with_64_row_tiles(oracle, alpha, beta):
+    """The library's choice for a ragged M only on long problems (more than 256 k-blocks per resident
+    CTA, too large for a full oracle comparison): forced here on a moderate one."""
+    assert (dg.dgemm_plan(1600, 8192, 8192)["variant"], dg.dgemm_plan(1600, 8192, 8192)["bm"]) == (dg.DGEMM_VARIANT_TMA, 64)
+    M, N, K = 1040, 1000, 320
+    _case(oracle, M, N, K, False, False, alpha, beta, True, seed=77, pad=(2, 4, 7),
+          c_fill=(np.nan if beta == 0.0 else None), variant=dg.DGEMM_VARIANT_TMA)
+    _case(oracle, M, N, K, True, True, alpha, beta, False, seed=78, variant=dg.DGEMM_VARIANT_TMA)

@@ -33,13 +33,15 @@ def _defaults():
     ((4096, 4096, 4096), V_WS, 128, 128, 64),
     ((16384, 16384, 64), V_WS, 64, 128, 64),       # K < 256: the same kernel with two CTAs per SM
     ((16384, 16384, 256), V_WS, 128, 128, 64),
-    ((2088, 2048, 2048), V_TMA, 64, 128, 64),      # M just above a multiple of 64 rows less wasteful in 64-row tiles
-    ((256, 256, 256), V_TMA, 64, 128, 64),         # a handful of tiles: inline kernel
-    ((128, 128, 128), V_CLUSTER, 64, 128, 64),     # fewer CTAs than SMs even with K cut in 8: split inside clusters
-    ((64, 64, 64), V_CLUSTER, 64, 128, 64),
+    ((2088, 2048, 2048), V_WS, 64, 128, 64),       # M just above a multiple of 64 rows: 64-row tiles, two CTAs per SM
+    ((1600, 8192, 8192), V_TMA, 64, 128, 64),      # the same on a long problem: inline kernel
+    ((256, 256, 256), V_WS, 64, 128, 64),          # one k-block per CTA through the workspace: the general kernels' floor
+    ((128, 128, 128), V_WS, 64, 128, 64),
+    ((64, 64, 64), V_CLUSTER, 64, 128, 64),        # too few k-blocks for a workspace split: split inside a cluster
+    ((320, 320, 320), V_CLUSTER, 64, 128, 64),
     ((512, 512, 256), V_CLUSTER, 64, 128, 64),
-    ((384, 384, 384), V_TMA, 64, 128, 64),         # 18 tiles x 8 would have to share SMs
-    ((128, 128, 4096), V_TMA, 64, 128, 64),        # long K runs stay with the general kernels
+    ((384, 384, 384), V_WS, 64, 128, 64),          # 18 tiles x 8 would have to share SMs
+    ((128, 128, 4096), V_WS, 64, 128, 64),         # long K runs stay with the general kernels
     ((4097, 31, 4099), V_TMA, 256, 32, 64),        # narrow N
     ((8192, 96, 8192), V_TMA, 256, 32, 64),
     ((8192, 128, 8192), V_WS, 128, 128, 64),

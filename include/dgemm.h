@@ -55,7 +55,8 @@ enum {
   DGEMM_VARIANT_TMA_CLUSTER = 5, /* as TMA on 64 x 128 tiles, K cut over the 1, 2, 4 or 8 CTAs of a
                                     thread-block cluster, partial tiles added through distributed shared
                                     memory: one launch, no workspace; what AUTO uses below one wave of tiles */
-  DGEMM_VARIANT_COUNT = 6
+  DGEMM_VARIANT_GENERIC_CLUSTER = 6, /* as TMA_CLUSTER with the GENERIC staging: any alignment          */
+  DGEMM_VARIANT_COUNT = 7
 };
 
 /*

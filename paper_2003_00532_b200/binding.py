@@ -39,6 +39,7 @@ DGEMM_VARIANT_GENERIC = 2
 DGEMM_VARIANT_TMA_WS = 3
 DGEMM_VARIANT_GENERIC_WS = 4
 DGEMM_VARIANT_TMA_CLUSTER = 5
+DGEMM_VARIANT_GENERIC_CLUSTER = 6
 
 # dgemm_set_test_flags bits
 DGEMM_TEST_NO_C_PREFETCH = 1

@@ -228,11 +228,14 @@ int device_state(DeviceState** out) {
     }
     {
       // cluster split-K kernel: shared-memory opt-in, then ask whether a full-size cluster fits
-      auto* ck = dgemm_cluster_kernel<64, 64, BN>;
+      auto* ck = dgemm_cluster_kernel<true, 64, 64, BN>;
+      auto* ckg = dgemm_cluster_kernel<false, 64, 64, BN>;
       using CCfg = TileCfg<64, 64, BN>;
       st.cluster_ok = false;
       if (cudaFuncSetAttribute(ck, cudaFuncAttributeMaxDynamicSharedMemorySize, CCfg::SMEM_BYTES_) == cudaSuccess &&
-          cudaFuncSetAttribute(ck, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared) == cudaSuccess) {
+          cudaFuncSetAttribute(ck, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared) == cudaSuccess &&
+          cudaFuncSetAttribute(ckg, cudaFuncAttributeMaxDynamicSharedMemorySize, CCfg::SMEM_BYTES_) == cudaSuccess &&
+          cudaFuncSetAttribute(ckg, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared) == cudaSuccess) {
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(CLUSTER_MAX);
         cfg.blockDim = dim3(CCfg::THREADS_);
@@ -245,7 +248,10 @@ int device_state(DeviceState** out) {
         cfg.attrs = attr;
         cfg.numAttrs = 1;
         int clusters = 0;
-        if (cudaOccupancyMaxActiveClusters(&clusters, ck, &cfg) == cudaSuccess) st.cluster_ok = clusters >= 1;
+        int clusters_g = 0;
+        if (cudaOccupancyMaxActiveClusters(&clusters, ck, &cfg) == cudaSuccess &&
+            cudaOccupancyMaxActiveClusters(&clusters_g, ckg, &cfg) == cudaSuccess)
+          st.cluster_ok = clusters >= 1 && clusters_g >= 1;
       }
       (void)cudaGetLastError();
     }
@@ -364,8 +370,8 @@ struct Plan {
 };
 
 // The cluster split-K kernel on `tiles` 64 x 128 tiles with clusters of s CTAs.
-void fill_cluster_plan(Plan& pl, int tiles, int kblocks, int s) {
-  pl.variant = DGEMM_VARIANT_TMA_CLUSTER;
+void fill_cluster_plan(Plan& pl, int tiles, int kblocks, int s, bool tma) {
+  pl.variant = tma ? DGEMM_VARIANT_TMA_CLUSTER : DGEMM_VARIANT_GENERIC_CLUSTER;
   pl.bm = 64;
   pl.bn = BN;
   pl.wtm = 64;
@@ -417,7 +423,7 @@ Plan plan_gemm(int64_t M, int64_t N, int64_t K, bool tma_ok, int requested_varia
   pl.variant = variant;
   const bool wants_tma = variant == DGEMM_VARIANT_TMA || variant == DGEMM_VARIANT_TMA_WS || variant == DGEMM_VARIANT_TMA_CLUSTER;
   if (wants_tma && !tma_ok) { pl.status = DGEMM_ERR_VARIANT; return pl; }
-  if (variant == DGEMM_VARIANT_TMA_CLUSTER) {
+  if (variant == DGEMM_VARIANT_TMA_CLUSTER || variant == DGEMM_VARIANT_GENERIC_CLUSTER) {
     // forced: clusters of dgemm_set_split_k() CTAs if that is 1, 2, 4 or 8 (ranks beyond the last
     // k-block then idle), else the largest size that keeps all CTAs resident at once
     if (!cluster_ok || !two_ctas_ok) { pl.status = DGEMM_ERR_VARIANT; return pl; }
@@ -429,7 +435,7 @@ Plan plan_gemm(int64_t M, int64_t N, int64_t K, bool tma_ok, int requested_varia
     } else {
       while (s < CLUSTER_MAX && 2 * s <= kblocks && tiles64 * 2 * s <= 2 * (int64_t)sm_count) s *= 2;
     }
-    fill_cluster_plan(pl, (int)tiles64, kblocks, s);
+    fill_cluster_plan(pl, (int)tiles64, kblocks, s, variant == DGEMM_VARIANT_TMA_CLUSTER);
     return pl;
   }
   if ((variant == DGEMM_VARIANT_TMA_WS && !(ws_ok[0] && ws_ok[2])) || (variant == DGEMM_VARIANT_GENERIC_WS && !ws_ok[1])) {
@@ -516,14 +522,16 @@ Plan plan_gemm(int64_t M, int64_t N, int64_t K, bool tma_ok, int requested_varia
     // 64-row tile, doubled where two CTAs of the general kernels share an SM. Runs of more than 8
     // k-blocks per CTA stay with the general kernels, whose main loops are the faster ones. Any
     // test flag that asks for a particular tile or reduction keeps the general kernels too.
-    if (auto_choice && wants_tma && cluster_ok && two_ctas_ok && !(dbg_flags & ~(DGEMM_TEST_NO_C_PREFETCH | DGEMM_TEST_NO_BLOCKED_B)) && tiles < sms &&
-        pl.wtm == 64) {  // (every tile shape but the 32-row one: a k-block of each is the same arithmetic)
+    if (auto_choice && cluster_ok && two_ctas_ok && !(dbg_flags & ~(DGEMM_TEST_NO_C_PREFETCH | DGEMM_TEST_NO_BLOCKED_B)) && tiles < sms &&
+        (pl.wtm == 64 || bm == 32)) {  // (not the test-only 32 x 32 warp tiles of the larger tiles)
       // costs in tenths of a k-block; a pass of the in-cluster reduction (512 element pairs per
       // CTA) is worth about 0.4 k-blocks, the second launch of the workspace split about one.
       // Only cluster sizes that leave every CTA an SM of its own: measured, clusters that have to
       // share SMs lose far more than the factor two of independent CTAs.
       const bool old_splits = pl.tail_tiles > 0 && pl.tail_ipc < kblocks;
-      const int path_old = 10 * (old_splits ? pl.tail_ipc : kblocks) * ((bm == 128 || pl.grid > sm_count) ? 2 : 1);
+      // (a k-block of a 32-row tile takes about half of a 64-row one; generic staging about 1.5 of TMA staging)
+      const int path_old = (bm == 32 ? 5 : 10) * (old_splits ? pl.tail_ipc : kblocks) * ((bm == 128 || pl.grid > sm_count) ? 2 : 1) *
+                           (wants_tma ? 2 : 3) / 2;
       // (one k-block per CTA and the reduction kernel behind it is the general kernels' floor, 7.8 us
       // at 128^3, and below the cluster kernel's, 8.7 us: no credit there)
       const int cost_old = path_old + ((old_splits && path_old >= 20) ? 10 * kClusterCreditKblocks : 0);
@@ -534,10 +542,10 @@ Plan plan_gemm(int64_t M, int64_t N, int64_t K, bool tma_ok, int requested_varia
         const int64_t alone = s >= 4 ? sm_count - sm_count / 8 : sm_count - 4;  // clusters are placed inside a GPC
         if (tiles_c * s > alone) break;
         if (kps > kClusterMaxKblocks) continue;
-        const int cost = 10 * kps + 4 * (CLUSTER_MAX / s);
+        const int cost = 10 * kps * (wants_tma ? 2 : 3) / 2 + 4 * (CLUSTER_MAX / s);
         if (cost < best_cost) { best_cost = cost; best_s = s; }
       }
-      if (best_s > 0 && best_cost <= cost_old) fill_cluster_plan(pl, (int)tiles_c, kblocks, best_s);
+      if (best_s > 0 && best_cost <= cost_old) fill_cluster_plan(pl, (int)tiles_c, kblocks, best_s, wants_tma);
     }
   }
   return pl;
@@ -614,7 +622,7 @@ int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, c
   if (plan.status != DGEMM_OK) return plan.status;
   variant = plan.variant;
   const bool wants_tma = variant == DGEMM_VARIANT_TMA || variant == DGEMM_VARIANT_TMA_WS || variant == DGEMM_VARIANT_TMA_CLUSTER;
-  const bool cluster = variant == DGEMM_VARIANT_TMA_CLUSTER;
+  const bool cluster = variant == DGEMM_VARIANT_TMA_CLUSTER || variant == DGEMM_VARIANT_GENERIC_CLUSTER;
 
   if (variant == DGEMM_VARIANT_NAIVE) {
     if (form.alpha != 1.0 || form.beta != 1.0) return DGEMM_ERR_VARIANT;  // the naive nest is C += A B only
@@ -673,7 +681,7 @@ int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, c
     p.b_blocked_map = (!(dbg_flags & DGEMM_TEST_NO_BLOCKED_B) && N % 16 == 0 && make_blocked_map(&map_b, B, K, N, ldb, BK, bn / 16)) ? 1 : 0;
     if (!p.b_blocked_map && !make_map(&map_b, B, K, N, ldb, 16, BK)) return DGEMM_ERR_CUDA;
     if (cluster)
-      launch_cluster_pdl(dgemm_cluster_kernel<64, 64, BN>, grid, p.split_k, TileCfg<64, 64, BN>::THREADS_,
+      launch_cluster_pdl(dgemm_cluster_kernel<true, 64, 64, BN>, grid, p.split_k, TileCfg<64, 64, BN>::THREADS_,
                          (size_t)TileCfg<64, 64, BN>::SMEM_BYTES_, stream, map_a, map_b, p);
     else if (ws64)
       launch_gemm_kernel(dgemm_dmma_ws_kernel<true, 64>, grid, WsCfg<64>::THREADS_, WsCfg<64>::SMEM_BYTES_, stream, map_a, map_b, p);
@@ -682,7 +690,10 @@ int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, c
     else
       launch_default_kernel<true>(bm, wtm, grid, stream, map_a, map_b, p);
   } else {
-    if (variant == DGEMM_VARIANT_GENERIC_WS)
+    if (cluster)
+      launch_cluster_pdl(dgemm_cluster_kernel<false, 64, 64, BN>, grid, p.split_k, TileCfg<64, 64, BN>::THREADS_,
+                         (size_t)TileCfg<64, 64, BN>::SMEM_BYTES_, stream, map_a, map_b, p);
+    else if (variant == DGEMM_VARIANT_GENERIC_WS)
       launch_gemm_kernel(dgemm_dmma_ws_kernel<false>, grid, WS_THREADS, SMEM_BYTES, stream, map_a, map_b, p);
     else
       launch_default_kernel<false>(bm, wtm, grid, stream, map_a, map_b, p);

@@ -22,7 +22,45 @@ namespace dgemm {
 
 constexpr int CLUSTER_MAX = 8;  // portable cluster size limit
 
-template <int TBM, int WTM = 64, int TBN = BN>
+// One stage (A: TBM x 16, B: 16 x TBN doubles, the swizzled layout of the TMA copies) staged with
+// 8-byte asynchronous copies, zero fill outside the matrices: any alignment, any leading dimension.
+// A: 16 consecutive threads copy the 16 k values of one row; B: TBN consecutive threads copy TBN
+// consecutive columns of one k row.
+template <int TBM, int TBN, int THREADS>
+__device__ __forceinline__ void stage_copy_generic(const GemmParams& p, uint32_t sa, uint32_t sb, int m0, int n0, int k0, int tid) {
+  {
+    const int a_k = tid & 15, row0 = tid >> 4;
+    const int k = k0 + a_k;
+    const bool kin = k < p.K;
+    const double* src = p.A + (long long)(m0 + row0) * p.lda + k;
+    const uint32_t dst_base = sa + ((a_k & 1) << 3);
+    constexpr int ROW_STEP = THREADS / 16;
+#pragma unroll
+    for (int i = 0; i < TBM / ROW_STEP; ++i) {
+      const int row = row0 + ROW_STEP * i;
+      const bool in = kin && (m0 + row < p.M);
+      const uint32_t dst = dst_base + row * 128 + (((a_k >> 1) ^ (row & 7)) << 4);
+      ptx::cp_async_8(dst, in ? (const void*)(src + (long long)(ROW_STEP * i) * p.lda) : (const void*)p.A, in ? 8u : 0u);
+    }
+  }
+  {
+    const int nn = tid % TBN, kk0 = tid / TBN;
+    const bool nin = n0 + nn < p.N;
+    const double* src = p.B + (long long)(k0 + kk0) * p.ldb + (n0 + nn);
+    const uint32_t dst_base = sb + (nn >> 4) * B_BOX_BYTES + ((nn & 1) << 3);
+    const int chunk = (nn & 15) >> 1;
+    constexpr int K_STEP = THREADS / TBN;
+#pragma unroll
+    for (int i = 0; i < BK / K_STEP; ++i) {
+      const int kk = kk0 + K_STEP * i;
+      const bool in = nin && (k0 + kk < p.K);
+      const uint32_t dst = dst_base + kk * 128 + ((chunk ^ (kk & 7)) << 4);
+      ptx::cp_async_8(dst, in ? (const void*)(src + (long long)(K_STEP * i) * p.ldb) : (const void*)p.B, in ? 8u : 0u);
+    }
+  }
+}
+
+template <bool USE_TMA, int TBM, int WTM = 64, int TBN = BN>
 __global__ void __launch_bounds__(TileCfg<TBM, WTM, TBN>::THREADS_, 2)
 dgemm_cluster_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                      const __grid_constant__ GemmParams p) {
@@ -60,13 +98,15 @@ dgemm_cluster_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
 
   if (tid == 0) {
     for (int s = 0; s < STAGES; ++s) {
-      ptx::mbar_init(full_bar + 8 * s, 1);
+      ptx::mbar_init(full_bar + 8 * s, USE_TMA ? 1 : THREADS);
       ptx::mbar_init(empty_bar + 8 * s, WARPS);
     }
     *abort_flag = 0;
     ptx::fence_barrier_init();
-    ptx::prefetch_tensormap(&map_a);
-    ptx::prefetch_tensormap(&map_b);
+    if (USE_TMA) {
+      ptx::prefetch_tensormap(&map_a);
+      ptx::prefetch_tensormap(&map_b);
+    }
   }
   __syncthreads();
   ptx::grid_dependency_wait();
@@ -79,11 +119,17 @@ dgemm_cluster_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
   const int rows_per = TBM / S;
   const int row_first = rank * rows_per;  // rows of the tile this CTA reduces
 
-  // Lane 0 of warp 0 issues the copies of k-block j of this CTA into stage j % STAGES.
+  // The copies of k-block j of this CTA into stage j % STAGES. TMA staging: issued by lane 0 of
+  // warp 0; generic staging: every thread copies its share.
   auto issue = [&](int j) -> bool {
     const uint32_t s = (uint32_t)j % STAGES, ph = ((uint32_t)j / STAGES) & 1u;
     if (!wait_bounded<false>(empty_bar + 8 * s, ph ^ 1u, abort_flag, p)) return false;
     const uint32_t sa = tiles_u32 + s * STAGE_BYTES, sb = sa + A_STAGE_BYTES, fb = full_bar + 8 * s;
+    if (!USE_TMA) {
+      stage_copy_generic<TBM, TBN, THREADS>(p, sa, sb, tm * TBM, tn * TBN, (kb0 + j) * BK, tid);
+      ptx::cp_async_mbar_arrive_noinc(fb);
+      return true;
+    }
     ptx::mbar_arrive_expect_tx(fb, STAGE_BYTES);
     ptx::tma_load_2d(sa, &map_a, (kb0 + j) * BK, tm * TBM, fb);
     if (p.b_blocked_map) {
@@ -95,8 +141,10 @@ dgemm_cluster_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
   };
 
   bool ok = true;
-  int issued = 0;  // meaningful in lane 0 of warp 0 only
-  if (warp == 0) {
+  int issued = 0;  // TMA staging: meaningful in lane 0 of warp 0 only
+  if (!USE_TMA) {
+    for (; issued < nkb && issued < LOOKAHEAD && ok; ++issued) ok = issue(issued);
+  } else if (warp == 0) {
     int good = 1;
     if (lane == 0) {
       for (; issued < nkb && issued < LOOKAHEAD && good; ++issued) good = issue(issued) ? 1 : 0;
@@ -149,7 +197,9 @@ dgemm_cluster_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
     if (!wait_bounded(full_bar + 8 * s, ph, abort_flag, p)) { ok = false; break; }
     compute_kblock<false, MT>(tiles + s * STAGE_BYTES, lm, acc);
     release_stage(empty_bar + 8 * s, lane);
-    if (warp == 0 && i + LOOKAHEAD < nkb) {  // refill the stage all warps released two k-blocks ago
+    if (!USE_TMA) {
+      if (i + LOOKAHEAD < nkb && !issue(i + LOOKAHEAD)) { ok = false; break; }
+    } else if (warp == 0 && i + LOOKAHEAD < nkb) {  // refill the stage all warps released two k-blocks ago
       int good = 1;
       if (lane == 0) {
         good = issue(i + LOOKAHEAD) ? 1 : 0;
@@ -159,6 +209,7 @@ dgemm_cluster_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
     }
   }
 
+  if (!USE_TMA) ptx::cp_async_wait_all();
   __syncthreads();  // every warp is done with the stages
   ok = (*abort_flag == 0);  // uniform over the CTA from here on
 
@@ -212,7 +263,7 @@ dgemm_cluster_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
   ptx::cluster_wait_acquire();
 
   // After an abort, copies may still be in flight into this CTA's shared memory: let them land.
-  if (!ok && tid == 0) {
+  if (USE_TMA && !ok && tid == 0) {
     const int first = issued > STAGES ? issued - STAGES : 0;
     for (int q = first; q < issued; ++q) {
       const uint32_t s = (uint32_t)q % STAGES, ph = ((uint32_t)q / STAGES) & 1u;

@@ -123,6 +123,24 @@ def test_auto_picks_cluster_kernel_on_small_problems(oracle, shape, integer):
         dg.dgemm_set_test_flags(0)
 
 
+@pytest.mark.parametrize("split", [0, 2, 8])
+@pytest.mark.parametrize("integer", [True, False])
+@pytest.mark.parametrize("shape", [(65, 129, 17), (282, 85, 44), (250, 133, 91), (300, 1001, 77), (21, 97, 75)])
+def test_cluster_kernel_generic_staging(oracle, shape, integer, split):
+    """Odd leading dimensions and bases off the 16-byte boundary: 8-byte asynchronous copies instead
+    of TMA, everything else the same kernel. Forced, and as DGEMM_VARIANT_AUTO picks it."""
+    M, N, K = shape
+    _case(oracle, M, N, K, False, False, 1.0, 1.0, integer, seed=M + N + K + split, pad=(1, 3, 1), offset=1,
+          variant=dg.DGEMM_VARIANT_GENERIC_CLUSTER, split_k=split)
+    if split == 0:
+        _case(oracle, M, N, K, False, False, -2.0, 0.5, integer, seed=M + N + K, pad=(1, 3, 1), offset=1)
+
+
+def test_auto_picks_generic_cluster_kernel_for_small_unaddressable_problems():
+    for shape in [(282, 85, 44), (21, 97, 75), (64, 64, 64)]:
+        assert dg.dgemm_plan(*shape, tma_addressable=False)["variant"] == dg.DGEMM_VARIANT_GENERIC_CLUSTER
+
+
 def test_forced_cluster_variant_rejects_operands_tma_cannot_address():
     A = torch.zeros(64, 33, dtype=torch.float64, device="cuda")  # odd leading dimension
     B = torch.zeros(33, 128, dtype=torch.float64, device="cuda")

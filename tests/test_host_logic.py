@@ -99,11 +99,12 @@ def test_variant_and_split_setters():
     assert dg.dgemm_set_variant(dg.DGEMM_VARIANT_GENERIC) == 0
     assert dg.dgemm_set_variant(dg.DGEMM_VARIANT_AUTO) == 0
     with pytest.raises(dg.DgemmError):
-        dg.dgemm_set_variant(6)
+        dg.dgemm_set_variant(7)
     with pytest.raises(dg.DgemmError):
         dg.dgemm_set_variant(-2)
     assert dg.dgemm_set_variant(dg.DGEMM_VARIANT_TMA_WS) == 0 and dg.dgemm_set_variant(dg.DGEMM_VARIANT_AUTO) == 0
     assert dg.dgemm_set_variant(dg.DGEMM_VARIANT_TMA_CLUSTER) == 0 and dg.dgemm_set_variant(dg.DGEMM_VARIANT_AUTO) == 0
+    assert dg.dgemm_set_variant(dg.DGEMM_VARIANT_GENERIC_CLUSTER) == 0 and dg.dgemm_set_variant(dg.DGEMM_VARIANT_AUTO) == 0
     assert dg.dgemm_set_test_flags(3) == 0 and dg.dgemm_set_test_flags(0) == 0
     with pytest.raises(dg.DgemmError):
         dg.dgemm_set_test_flags(256)

@@ -13,6 +13,7 @@ import paper_2003_00532_b200 as dg
 
 V_TMA, V_GENERIC, V_WS = dg.DGEMM_VARIANT_TMA, dg.DGEMM_VARIANT_GENERIC, dg.DGEMM_VARIANT_TMA_WS
 V_CLUSTER = dg.DGEMM_VARIANT_TMA_CLUSTER
+V_GCLUSTER = dg.DGEMM_VARIANT_GENERIC_CLUSTER
 
 
 @pytest.fixture(autouse=True)
@@ -77,7 +78,7 @@ def _items(pl, cta):
         tile, ks = divmod(unit, pl["split_k"])
         k0 = ks * pl["kblocks_per_split"]
         if k0 >= kb:  # a cluster rank beyond the last k-block: no arithmetic, it only shares in the reduction
-            assert pl["variant"] == V_CLUSTER
+            assert pl["variant"] in (V_CLUSTER, V_GCLUSTER)
             continue
         out.append((tile, k0, min(k0 + pl["kblocks_per_split"], kb), ks * pl["dp_tiles"] + tile if pl["split_k"] > 1 else -1))
     if pl["tail_tiles"]:
@@ -95,11 +96,15 @@ def _items(pl, cta):
     return out
 
 
-def _check_cover(shape, sm_count=148):
-    pl = dg.dgemm_plan(*shape, sm_count=sm_count)
+def _check_cover_unaddressable(shape):
+    return _check_cover(shape, tma_addressable=False)
+
+
+def _check_cover(shape, sm_count=148, tma_addressable=True):
+    pl = dg.dgemm_plan(*shape, sm_count=sm_count, tma_addressable=tma_addressable)
     tiles = -(-shape[0] // pl["bm"]) * -(-shape[1] // pl["bn"])
     assert pl["dp_tiles"] + pl["tail_tiles"] == tiles
-    if pl["variant"] == V_CLUSTER:  # one CTA per (tile, rank); clusters beyond the resident ones run in turn
+    if pl["variant"] in (V_CLUSTER, V_GCLUSTER):  # one CTA per (tile, rank); clusters beyond the resident ones run in turn
         assert pl["grid"] == tiles * pl["split_k"] and pl["split_k"] in (1, 2, 4, 8) and pl["tail_tiles"] == 0
         assert (pl["bm"], pl["bn"], pl["ctas_per_sm"]) == (64, 128, 2)
     else:
@@ -177,3 +182,10 @@ def test_cluster_plan():
     assert _check_cover((3000, 3000, 3000))["split_k"] == 1  # 1128 tiles: no room for more than one CTA each
     with pytest.raises(dg.DgemmError):
         dg.dgemm_plan(128, 128, 128, tma_addressable=False)
+    # operands TMA cannot address: the same kernel with the generic staging
+    dg.dgemm_set_variant(dg.DGEMM_VARIANT_AUTO)
+    pl = _check_cover_unaddressable((282, 85, 44))
+    assert pl["variant"] == V_GCLUSTER and pl["split_k"] in (2, 4, 8)
+    assert dg.dgemm_plan(1000, 1000, 1000, tma_addressable=False)["variant"] == V_GENERIC
+    dg.dgemm_set_variant(V_GCLUSTER)
+    assert dg.dgemm_plan(200, 300, 40, tma_addressable=False)["variant"] == V_GCLUSTER

@@ -531,7 +531,7 @@ Plan plan_gemm(int64_t M, int64_t N, int64_t K, bool tma_ok, int requested_varia
       const bool old_splits = pl.tail_tiles > 0 && pl.tail_ipc < kblocks;
       // (a k-block of a 32-row tile takes about half of a 64-row one; generic staging about 1.5 of TMA staging)
       const int path_old = (bm == 32 ? 5 : 10) * (old_splits ? pl.tail_ipc : kblocks) * ((bm == 128 || pl.grid > sm_count) ? 2 : 1) *
-                           (wants_tma ? 2 : 3) / 2;
+                           (wants_tma ? 2 : (bm == 256 ? 4 : 3)) / 2;  // (the 256 x 32 tile with generic staging: about 2)
       // (one k-block per CTA and the reduction kernel behind it is the general kernels' floor, 7.8 us
       // at 128^3, and below the cluster kernel's, 8.7 us: no credit there)
       const int cost_old = path_old + ((old_splits && path_old >= 20) ? 10 * kClusterCreditKblocks : 0);

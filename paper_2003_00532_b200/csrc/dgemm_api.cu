@@ -44,7 +44,7 @@ inline bool narrow_tiles_pay(int64_t N) {
 constexpr int kAutoWs64MaxKblocksPerCta = 256;     // ... and its 64-row form instead of the inline kernel up to this much work
 constexpr int kAutoWsMinKblocks = 16;                // warp-specialised kernel: 128-row tiles from K = 256 up, 64-row below
 constexpr double kPackMinFlopPerByte = 64.0;       // pack unaligned operands only if the copy is this cheap
-constexpr double kPackMinFlop = 1.0e9;             // ... and the problem is large enough for two more launches not to show
+constexpr double kPackMinFlop = 4.0e9;             // ... and the problem is large enough for two more launches not to show
 constexpr size_t kPackMaxBytes = 2ull << 30;       // ... and the packed copies fit in 2 GiB
 constexpr int64_t kHostBlockRows = 1024;             // dgemm_f64_host: rows of A and C per pipelined block
 constexpr int kTailMinSpan = 1;          // stream-K tail: at least this many k-blocks per CTA

@@ -224,7 +224,8 @@ def test_config4_ragged(oracle, idx, flags):
 def test_packing_pass_unaligned_operands(oracle, offset):
     """Odd leading dimensions and an odd element offset: A and B are packed into aligned scratch first
     (twice in a row: the second call reuses the scratch). Integer data, exact."""
-    prob = wl.make_problem(700, 650, 1200, seed=61, lda=1203, ldb=655, ldc=657, integer=True)
+    prob = wl.make_problem(1300, 1250, 1300, seed=61, lda=1303, ldb=1255, ldc=1257, integer=True)  # 4.2 GFLOP: packed
+    assert 2.0 * prob.M * prob.N * prob.K >= 4.0e9
     first = run_gpu(prob, offset_elems=offset)
     _check_full(oracle, prob, first)
     second = run_gpu(prob, offset_elems=offset)

@@ -350,6 +350,23 @@ def run_ours(args):
     e2e_value = world * flop * e2e_steps / e2e_s / 1e12
     h2d = 8 * (sm * sk + sk * sn + sm * sn)
     d2h = 8 * sm * sn
+    # what the host link of this machine gives a plain pinned copy (context for the end-to-end number,
+    # which moves h2d + d2h bytes per step over it): one copy of A each way, outside the timed regions
+    link = {}
+    if rank == 0:
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+        A.copy_(prob.A_buf, non_blocking=True)  # warm-up
+        torch.cuda.synchronize()
+        ev[0].record(stream)
+        A.copy_(prob.A_buf, non_blocking=True)
+        ev[1].record(stream)
+        prob.A_buf.copy_(A, non_blocking=True)
+        ev[2].record(stream)
+        torch.cuda.synchronize()
+        nbytes = A.numel() * 8
+        link = {"h2d_gbs": nbytes / (ev[0].elapsed_time(ev[1]) * 1e-3) / 1e9,
+                "d2h_gbs": nbytes / (ev[1].elapsed_time(ev[2]) * 1e-3) / 1e9}
+        link["floor_ms_per_step"] = max(h2d / (link["h2d_gbs"] * 1e9), d2h / (link["d2h_gbs"] * 1e9)) * 1e3
 
     if rank != 0:
         if distributed:
@@ -397,7 +414,8 @@ def run_ours(args):
         "roofline": roofline,
         "cpu_baseline": cpu_baseline,
         "e2e": {"value": e2e_value, "unit": "TFLOP/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "steps": e2e_steps, "api": "dgemm_f64_host (pinned host buffers)"},
+                "steps": e2e_steps, "ms_per_step": e2e_s / e2e_steps * 1e3,
+                "api": "dgemm_f64_host (pinned host buffers)", "host_link": link},
         "gpu_launches": int(launches),
         "clocks": clocks,
     }

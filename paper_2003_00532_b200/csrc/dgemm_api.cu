@@ -10,6 +10,7 @@
 #include <cstring>
 #include <mutex>
 #include <utility>
+#include <vector>
 
 #include <cuda.h>
 #include <cuda_runtime.h>
@@ -47,6 +48,7 @@ constexpr double kPackMinFlopPerByte = 64.0;       // pack unaligned operands on
 constexpr double kPackMinFlop = 4.0e9;             // ... and the problem is large enough for two more launches not to show
 constexpr size_t kPackMaxBytes = 2ull << 30;       // ... and the packed copies fit in 2 GiB
 constexpr int64_t kHostBlockRows = 1024;             // dgemm_f64_host: rows of A and C per pipelined block
+constexpr int64_t kHostPanelRows = 1024;             // ... and rows of B per panel while the first block waits for B
 constexpr int kTailMinSpan = 1;          // stream-K tail: at least this many k-blocks per CTA
 constexpr double kTailMinSavedKblocks = 5.0;  // use the stream-K tail only if it saves this many k-block times
 // Cluster split-K (one launch, reduction through distributed shared memory) replaces the workspace
@@ -68,6 +70,7 @@ struct DeviceState {
   double* workspace = nullptr; // split-K partial tiles, allocated on first need
   double* pack_buf = nullptr;  // packed copies of unaligned operands, grown on demand
   size_t pack_bytes = 0;
+  cudaMemPool_t host_pool = nullptr;  // dgemm_f64_host: device copies of the operands come from this pool
 };
 
 DeviceState g_dev[kMaxDevices];
@@ -272,6 +275,38 @@ int ensure_workspace(DeviceState* st) {
     // the counters are zero between calls: the kernels that use them put them back
     if (cudaMemset(st->workspace, 0, kCounterBytes) != cudaSuccess) return DGEMM_ERR_CUDA;
   }
+  return DGEMM_OK;
+}
+
+// Memory pool of dgemm_f64_host. The device's default pool gives memory back to the system at
+// every synchronisation, so each call would pay for mapping its 0.8 GB (8192^3) again: more than
+// the copies and the arithmetic together. This pool keeps up to kHostPoolKeepBytes between calls.
+constexpr unsigned long long kHostPoolKeepBytes = 1ull << 30;
+int ensure_host_pool(DeviceState* st, cudaMemPool_t* pool) {
+  std::lock_guard<std::mutex> lock(g_mutex);
+  if (!st->host_pool) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return DGEMM_ERR_DEVICE;
+    cudaMemPoolProps props;
+    memset(&props, 0, sizeof(props));
+    props.allocType = cudaMemAllocationTypePinned;
+    props.handleTypes = cudaMemHandleTypeNone;
+    props.location.type = cudaMemLocationTypeDevice;
+    props.location.id = dev;
+    cudaMemPool_t created = nullptr;
+    if (cudaMemPoolCreate(&created, &props) != cudaSuccess) {
+      (void)cudaGetLastError();
+      return DGEMM_ERR_CUDA;
+    }
+    unsigned long long keep = kHostPoolKeepBytes;
+    if (cudaMemPoolSetAttribute(created, cudaMemPoolAttrReleaseThreshold, &keep) != cudaSuccess) {
+      (void)cudaGetLastError();
+      cudaMemPoolDestroy(created);
+      return DGEMM_ERR_CUDA;
+    }
+    st->host_pool = created;
+  }
+  *pool = st->host_pool;
   return DGEMM_OK;
 }
 
@@ -895,6 +930,9 @@ int dgemm_f64_host(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda
   // Dense device copies with even leading dimensions (keeps the TMA path available). B is copied
   // whole; A and C travel in blocks of rows through two buffers each, on three streams, so that
   // the upload of block i+1, the arithmetic of block i and the download of block i-1 overlap.
+  cudaMemPool_t pool = nullptr;
+  rc = ensure_host_pool(st, &pool);
+  if (rc != DGEMM_OK) return rc;
   const int64_t dlda = K + (K & 1), dldb = N + (N & 1), dldc = N + (N & 1);
   const int64_t blk = (M > 2 * kHostBlockRows) ? kHostBlockRows : M;  // rows per block
   const int64_t nblk = (M + blk - 1) / blk;
@@ -903,6 +941,7 @@ int dgemm_f64_host(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda
   double* dB = nullptr;
   double* dA[2] = {nullptr, nullptr};
   double* dC[2] = {nullptr, nullptr};
+  std::vector<cudaEvent_t> ev_pan;  // one per row panel of B
   cudaEvent_t ev_alloc = nullptr, ev_up[2] = {nullptr, nullptr}, ev_run[2] = {nullptr, nullptr}, ev_down[2] = {nullptr, nullptr};
   rc = DGEMM_ERR_CUDA;
   do {
@@ -915,28 +954,52 @@ int dgemm_f64_host(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda
            cudaEventCreateWithFlags(&ev_run[i], cudaEventDisableTiming) == cudaSuccess &&
            cudaEventCreateWithFlags(&ev_down[i], cudaEventDisableTiming) == cudaSuccess;
     if (!ok) break;
-    if (cudaMallocAsync(reinterpret_cast<void**>(&dB), (size_t)K * dldb * 8, s_up) != cudaSuccess) break;
+    if (cudaMallocFromPoolAsync(reinterpret_cast<void**>(&dB), (size_t)K * dldb * 8, pool, s_up) != cudaSuccess) break;
     for (int i = 0; i < nbuf && ok; ++i)
-      ok = cudaMallocAsync(reinterpret_cast<void**>(&dA[i]), (size_t)blk * dlda * 8, s_up) == cudaSuccess &&
-           cudaMallocAsync(reinterpret_cast<void**>(&dC[i]), (size_t)blk * dldc * 8, s_up) == cudaSuccess;
+      ok = cudaMallocFromPoolAsync(reinterpret_cast<void**>(&dA[i]), (size_t)blk * dlda * 8, pool, s_up) == cudaSuccess &&
+           cudaMallocFromPoolAsync(reinterpret_cast<void**>(&dC[i]), (size_t)blk * dldc * 8, pool, s_up) == cudaSuccess;
     if (!ok) break;
     // the other streams may touch the buffers only after the (stream-ordered) allocations
     if (cudaEventRecord(ev_alloc, s_up) != cudaSuccess) break;
     if (cudaStreamWaitEvent(s_run, ev_alloc, 0) != cudaSuccess || cudaStreamWaitEvent(s_down, ev_alloc, 0) != cudaSuccess) break;
-    if (cudaMemcpy2DAsync(dB, dldb * 8, B, ldb * 8, N * 8, K, cudaMemcpyHostToDevice, s_up) != cudaSuccess) break;
     int inner = DGEMM_OK;
-    for (int64_t i = 0; i < nblk; ++i) {
+    // With more than one block, B travels in panels of kHostPanelRows rows (whole rows: contiguous
+    // in host memory when ldb == N; panels of columns crossed the link visibly slower) behind the
+    // first block of A and C, and that block is multiplied K panel by K panel as they arrive, each
+    // product added into the block of C: the arithmetic starts after 0.2 GB instead of 0.7 GB
+    // (8192^3) have crossed the host link. The second block's rows go up between the panels, so
+    // that they are there when B is complete.
+    const int64_t prows = (nblk > 1 && K > 2 * kHostPanelRows) ? kHostPanelRows : K;
+    const int64_t npan = (K + prows - 1) / prows;
+    auto upload_block = [&](int64_t i) -> bool {
       const int b = (int)(i % nbuf);
       const int64_t r0 = i * blk, rows = (M - r0 < blk) ? M - r0 : blk;
       // buffer b is free again once block i - 2 has been downloaded
-      if (i >= nbuf && cudaStreamWaitEvent(s_up, ev_down[b], 0) != cudaSuccess) { inner = DGEMM_ERR_CUDA; break; }
-      if (cudaMemcpy2DAsync(dA[b], dlda * 8, A + r0 * lda, lda * 8, K * 8, rows, cudaMemcpyHostToDevice, s_up) != cudaSuccess ||
-          cudaMemcpy2DAsync(dC[b], dldc * 8, C + r0 * ldc, ldc * 8, N * 8, rows, cudaMemcpyHostToDevice, s_up) != cudaSuccess ||
-          cudaEventRecord(ev_up[b], s_up) != cudaSuccess || cudaStreamWaitEvent(s_run, ev_up[b], 0) != cudaSuccess) {
+      if (i >= nbuf && cudaStreamWaitEvent(s_up, ev_down[b], 0) != cudaSuccess) return false;
+      return cudaMemcpy2DAsync(dA[b], dlda * 8, A + r0 * lda, lda * 8, K * 8, rows, cudaMemcpyHostToDevice, s_up) == cudaSuccess &&
+             cudaMemcpy2DAsync(dC[b], dldc * 8, C + r0 * ldc, ldc * 8, N * 8, rows, cudaMemcpyHostToDevice, s_up) == cudaSuccess &&
+             cudaEventRecord(ev_up[b], s_up) == cudaSuccess;
+    };
+    if (!upload_block(0) || cudaStreamWaitEvent(s_run, ev_up[0], 0) != cudaSuccess) break;
+    ev_pan.assign((size_t)npan, nullptr);
+    for (int64_t j = 0; j < npan && inner == DGEMM_OK; ++j) {
+      const int64_t k0 = j * prows, krows = (K - k0 < prows) ? K - k0 : prows;
+      if (cudaEventCreateWithFlags(&ev_pan[(size_t)j], cudaEventDisableTiming) != cudaSuccess ||
+          cudaMemcpy2DAsync(dB + k0 * dldb, dldb * 8, B + k0 * ldb, ldb * 8, N * 8, krows, cudaMemcpyHostToDevice, s_up) != cudaSuccess ||
+          cudaEventRecord(ev_pan[(size_t)j], s_up) != cudaSuccess || cudaStreamWaitEvent(s_run, ev_pan[(size_t)j], 0) != cudaSuccess) {
         inner = DGEMM_ERR_CUDA;
         break;
       }
-      inner = launch_gemm(rows, N, K, dA[b], dlda, dB, dldb, dC[b], dldc, s_run);
+      if (npan > 1) inner = launch_gemm(blk < M ? blk : M, N, krows, dA[0] + k0, dlda, dB + k0 * dldb, dldb, dC[0], dldc, s_run);
+      if (nblk > 1 && j == npan / 2 && inner == DGEMM_OK && !upload_block(1)) inner = DGEMM_ERR_CUDA;
+    }
+    if (inner != DGEMM_OK) { rc = inner; break; }
+    for (int64_t i = 0; i < nblk; ++i) {
+      const int b = (int)(i % nbuf);
+      const int64_t r0 = i * blk, rows = (M - r0 < blk) ? M - r0 : blk;
+      if (i >= 2 && !upload_block(i)) { inner = DGEMM_ERR_CUDA; break; }
+      if (i >= 1 && cudaStreamWaitEvent(s_run, ev_up[b], 0) != cudaSuccess) { inner = DGEMM_ERR_CUDA; break; }
+      if (i >= 1 || npan == 1) inner = launch_gemm(rows, N, K, dA[b], dlda, dB, dldb, dC[b], dldc, s_run);
       if (inner != DGEMM_OK) break;
       if (cudaEventRecord(ev_run[b], s_run) != cudaSuccess || cudaStreamWaitEvent(s_down, ev_run[b], 0) != cudaSuccess ||
           cudaMemcpy2DAsync(C + r0 * ldc, ldc * 8, dC[b], dldc * 8, N * 8, rows, cudaMemcpyDeviceToHost, s_down) != cudaSuccess ||
@@ -964,6 +1027,8 @@ int dgemm_f64_host(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda
     cudaStreamSynchronize(s_up);
   }
   if (ev_alloc) cudaEventDestroy(ev_alloc);
+  for (cudaEvent_t e : ev_pan)
+    if (e) cudaEventDestroy(e);
   for (int i = 0; i < 2; ++i) {
     if (ev_up[i]) cudaEventDestroy(ev_up[i]);
     if (ev_run[i]) cudaEventDestroy(ev_run[i]);

@@ -109,14 +109,15 @@ DGEMM_API int dgemm_f64(int64_t M, int64_t N, int64_t K,
 /*
  * Same operation with HOST buffers (pageable or pinned; pinned buffers let the copies overlap the
  * arithmetic). A and C are streamed through device scratch memory in blocks of 1024 rows (upload,
- * dgemm_f64, download on three streams). B follows the first block in panels of 1024 rows, and
- * that block is multiplied K panel by K panel as they arrive, so the arithmetic starts long
- * before B is complete (the products of the panels are added into C one after the other: for
- * those rows the sum over k is rounded in that order). Only the M x N logical part of each row is
- * meaningful; padding columns of the host C are preserved. Synchronous: returns after the result
- * is in the host buffer. Device scratch comes from a memory pool the library owns (stream-ordered
- * allocation) and goes back to it before returning; the pool keeps up to 1 GiB mapped between
- * calls, because mapping 0.8 GB anew on every call cost more than the copies and the arithmetic
+ * dgemm_f64, download on three streams). B follows the first blocks (three on a large problem) in
+ * panels of 1024 rows, and those blocks are multiplied K panel by K panel as the panels arrive,
+ * so the arithmetic starts long before B is complete (the products of the panels are added into C
+ * one after the other: for those rows the sum over k is rounded in that order). Only the M x N
+ * logical part of each row is meaningful; padding columns of the host C are preserved.
+ * Synchronous: returns after the result is in the host buffer. Device scratch comes from a memory
+ * pool the library owns (stream-ordered allocation) and goes back to it before returning; the
+ * pool keeps up to 1.25 GiB mapped between calls, because mapping a gigabyte anew on every call
+ * cost more than the copies and the arithmetic
  * of an 8192^3 problem together. Same argument rules and error codes as dgemm_f64
  * (Section 2.1; the paper's driver likewise owns A, B, C in host memory).
  */

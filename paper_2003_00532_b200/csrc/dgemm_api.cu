@@ -48,7 +48,8 @@ constexpr double kPackMinFlopPerByte = 64.0;       // pack unaligned operands on
 constexpr double kPackMinFlop = 4.0e9;             // ... and the problem is large enough for two more launches not to show
 constexpr size_t kPackMaxBytes = 2ull << 30;       // ... and the packed copies fit in 2 GiB
 constexpr int64_t kHostBlockRows = 1024;             // dgemm_f64_host: rows of A and C per pipelined block
-constexpr int64_t kHostPanelRows = 1024;             // ... and rows of B per panel while the first block waits for B
+constexpr int64_t kHostPanelRows = 1024;             // ... and rows of B per panel while the first blocks wait for B
+constexpr int kHostMaxBufs = 5;                      // ... and device buffers for blocks of A and C (3 first blocks + a ring of 2)
 constexpr int kTailMinSpan = 1;          // stream-K tail: at least this many k-blocks per CTA
 constexpr double kTailMinSavedKblocks = 5.0;  // use the stream-K tail only if it saves this many k-block times
 // Cluster split-K (one launch, reduction through distributed shared memory) replaces the workspace
@@ -281,7 +282,7 @@ int ensure_workspace(DeviceState* st) {
 // Memory pool of dgemm_f64_host. The device's default pool gives memory back to the system at
 // every synchronisation, so each call would pay for mapping its 0.8 GB (8192^3) again: more than
 // the copies and the arithmetic together. This pool keeps up to kHostPoolKeepBytes between calls.
-constexpr unsigned long long kHostPoolKeepBytes = 1ull << 30;
+constexpr unsigned long long kHostPoolKeepBytes = 5ull << 28;  // 1.25 GiB: B and five blocks of A and C at 8192^3
 int ensure_host_pool(DeviceState* st, cudaMemPool_t* pool) {
   std::lock_guard<std::mutex> lock(g_mutex);
   if (!st->host_pool) {
@@ -927,29 +928,39 @@ int dgemm_f64_host(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda
   int rc = device_state(&st);
   if (rc != DGEMM_OK) return rc;
 
-  // Dense device copies with even leading dimensions (keeps the TMA path available). B is copied
-  // whole; A and C travel in blocks of rows through two buffers each, on three streams, so that
-  // the upload of block i+1, the arithmetic of block i and the download of block i-1 overlap.
+  // Dense device copies with even leading dimensions (keeps the TMA path available). A and C
+  // travel in blocks of rows through a few buffers, on three streams, so that the upload of later
+  // blocks, the arithmetic of block i and the download of block i-1 overlap.
   cudaMemPool_t pool = nullptr;
   rc = ensure_host_pool(st, &pool);
   if (rc != DGEMM_OK) return rc;
   const int64_t dlda = K + (K & 1), dldb = N + (N & 1), dldc = N + (N & 1);
   const int64_t blk = (M > 2 * kHostBlockRows) ? kHostBlockRows : M;  // rows per block
   const int64_t nblk = (M + blk - 1) / blk;
-  const int nbuf = nblk > 1 ? 2 : 1;
+  // B travels in panels of kHostPanelRows rows (whole rows: contiguous in host memory when
+  // ldb == N) behind the first `heads` blocks of A and C, and those blocks are multiplied K panel
+  // by K panel as the panels arrive, each product added into its block of C: the arithmetic
+  // starts after 0.5 GB instead of 0.7 GB (8192^3) have crossed the host link, and by the time B
+  // is complete three eighths of it are done. The other blocks follow through a ring of buffers.
+  const int64_t prows = (nblk > 1 && K > 2 * kHostPanelRows) ? kHostPanelRows : K;
+  const int64_t npan = (K + prows - 1) / prows;
+  const int heads = (npan > 1 && nblk >= 6) ? 3 : 1;
+  const int nbuf = nblk > 1 ? (int)((nblk < heads + 2) ? nblk : heads + 2) : 1;
   cudaStream_t s_up = nullptr, s_run = nullptr, s_down = nullptr;
   double* dB = nullptr;
-  double* dA[2] = {nullptr, nullptr};
-  double* dC[2] = {nullptr, nullptr};
+  double* dA[kHostMaxBufs] = {nullptr, nullptr, nullptr, nullptr, nullptr};
+  double* dC[kHostMaxBufs] = {nullptr, nullptr, nullptr, nullptr, nullptr};
   std::vector<cudaEvent_t> ev_pan;  // one per row panel of B
-  cudaEvent_t ev_alloc = nullptr, ev_up[2] = {nullptr, nullptr}, ev_run[2] = {nullptr, nullptr}, ev_down[2] = {nullptr, nullptr};
+  cudaEvent_t ev_alloc = nullptr, ev_up[kHostMaxBufs] = {nullptr, nullptr, nullptr, nullptr, nullptr},
+              ev_run[kHostMaxBufs] = {nullptr, nullptr, nullptr, nullptr, nullptr},
+              ev_down[kHostMaxBufs] = {nullptr, nullptr, nullptr, nullptr, nullptr};
   rc = DGEMM_ERR_CUDA;
   do {
     if (cudaStreamCreateWithFlags(&s_up, cudaStreamNonBlocking) != cudaSuccess) break;
     if (cudaStreamCreateWithFlags(&s_run, cudaStreamNonBlocking) != cudaSuccess) break;
     if (cudaStreamCreateWithFlags(&s_down, cudaStreamNonBlocking) != cudaSuccess) break;
     bool ok = cudaEventCreateWithFlags(&ev_alloc, cudaEventDisableTiming) == cudaSuccess;
-    for (int i = 0; i < 2 && ok; ++i)
+    for (int i = 0; i < nbuf && ok; ++i)
       ok = cudaEventCreateWithFlags(&ev_up[i], cudaEventDisableTiming) == cudaSuccess &&
            cudaEventCreateWithFlags(&ev_run[i], cudaEventDisableTiming) == cudaSuccess &&
            cudaEventCreateWithFlags(&ev_down[i], cudaEventDisableTiming) == cudaSuccess;
@@ -963,14 +974,6 @@ int dgemm_f64_host(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda
     if (cudaEventRecord(ev_alloc, s_up) != cudaSuccess) break;
     if (cudaStreamWaitEvent(s_run, ev_alloc, 0) != cudaSuccess || cudaStreamWaitEvent(s_down, ev_alloc, 0) != cudaSuccess) break;
     int inner = DGEMM_OK;
-    // With more than one block, B travels in panels of kHostPanelRows rows (whole rows: contiguous
-    // in host memory when ldb == N; panels of columns crossed the link visibly slower) behind the
-    // first block of A and C, and that block is multiplied K panel by K panel as they arrive, each
-    // product added into the block of C: the arithmetic starts after 0.2 GB instead of 0.7 GB
-    // (8192^3) have crossed the host link. The second block's rows go up between the panels, so
-    // that they are there when B is complete.
-    const int64_t prows = (nblk > 1 && K > 2 * kHostPanelRows) ? kHostPanelRows : K;
-    const int64_t npan = (K + prows - 1) / prows;
     auto upload_block = [&](int64_t i) -> bool {
       const int b = (int)(i % nbuf);
       const int64_t r0 = i * blk, rows = (M - r0 < blk) ? M - r0 : blk;
@@ -980,7 +983,10 @@ int dgemm_f64_host(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda
              cudaMemcpy2DAsync(dC[b], dldc * 8, C + r0 * ldc, ldc * 8, N * 8, rows, cudaMemcpyHostToDevice, s_up) == cudaSuccess &&
              cudaEventRecord(ev_up[b], s_up) == cudaSuccess;
     };
-    if (!upload_block(0) || cudaStreamWaitEvent(s_run, ev_up[0], 0) != cudaSuccess) break;
+    bool heads_up = true;
+    for (int h = 0; h < heads && heads_up; ++h)
+      heads_up = upload_block(h) && cudaStreamWaitEvent(s_run, ev_up[h], 0) == cudaSuccess;
+    if (!heads_up) break;
     ev_pan.assign((size_t)npan, nullptr);
     for (int64_t j = 0; j < npan && inner == DGEMM_OK; ++j) {
       const int64_t k0 = j * prows, krows = (K - k0 < prows) ? K - k0 : prows;
@@ -990,16 +996,15 @@ int dgemm_f64_host(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda
         inner = DGEMM_ERR_CUDA;
         break;
       }
-      if (npan > 1) inner = launch_gemm(blk < M ? blk : M, N, krows, dA[0] + k0, dlda, dB + k0 * dldb, dldb, dC[0], dldc, s_run);
-      if (nblk > 1 && j == npan / 2 && inner == DGEMM_OK && !upload_block(1)) inner = DGEMM_ERR_CUDA;
+      for (int h = 0; h < heads && npan > 1 && inner == DGEMM_OK; ++h)
+        inner = launch_gemm(blk < M ? blk : M, N, krows, dA[h] + k0, dlda, dB + k0 * dldb, dldb, dC[h], dldc, s_run);
     }
     if (inner != DGEMM_OK) { rc = inner; break; }
     for (int64_t i = 0; i < nblk; ++i) {
       const int b = (int)(i % nbuf);
       const int64_t r0 = i * blk, rows = (M - r0 < blk) ? M - r0 : blk;
-      if (i >= 2 && !upload_block(i)) { inner = DGEMM_ERR_CUDA; break; }
-      if (i >= 1 && cudaStreamWaitEvent(s_run, ev_up[b], 0) != cudaSuccess) { inner = DGEMM_ERR_CUDA; break; }
-      if (i >= 1 || npan == 1) inner = launch_gemm(rows, N, K, dA[b], dlda, dB, dldb, dC[b], dldc, s_run);
+      if (i >= heads && (!upload_block(i) || cudaStreamWaitEvent(s_run, ev_up[b], 0) != cudaSuccess)) { inner = DGEMM_ERR_CUDA; break; }
+      if (i >= heads || npan == 1) inner = launch_gemm(rows, N, K, dA[b], dlda, dB, dldb, dC[b], dldc, s_run);
       if (inner != DGEMM_OK) break;
       if (cudaEventRecord(ev_run[b], s_run) != cudaSuccess || cudaStreamWaitEvent(s_down, ev_run[b], 0) != cudaSuccess ||
           cudaMemcpy2DAsync(C + r0 * ldc, ldc * 8, dC[b], dldc * 8, N * 8, rows, cudaMemcpyDeviceToHost, s_down) != cudaSuccess ||
@@ -1020,7 +1025,7 @@ int dgemm_f64_host(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda
   if (s_down) cudaStreamSynchronize(s_down);
   if (s_up) {
     if (dB) cudaFreeAsync(dB, s_up);
-    for (int i = 0; i < 2; ++i) {
+    for (int i = 0; i < kHostMaxBufs; ++i) {
       if (dA[i]) cudaFreeAsync(dA[i], s_up);
       if (dC[i]) cudaFreeAsync(dC[i], s_up);
     }
@@ -1029,7 +1034,7 @@ int dgemm_f64_host(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda
   if (ev_alloc) cudaEventDestroy(ev_alloc);
   for (cudaEvent_t e : ev_pan)
     if (e) cudaEventDestroy(e);
-  for (int i = 0; i < 2; ++i) {
+  for (int i = 0; i < kHostMaxBufs; ++i) {
     if (ev_up[i]) cudaEventDestroy(ev_up[i]);
     if (ev_run[i]) cudaEventDestroy(ev_run[i]);
     if (ev_down[i]) cudaEventDestroy(ev_down[i]);

@@ -254,6 +254,16 @@ DGEMM_API int dgemm_plan(int64_t M, int64_t N, int64_t K, int tma_addressable, i
 DGEMM_API int dgemm_last_device_status(void *stream);
 
 /*
+ * Gives the device memory the library holds on the current device back to the system: the split-K
+ * workspace (80 MiB), the scratch of the packing pass (up to 2.5 GiB, as large as the largest
+ * packed problem so far) and what the memory pool of dgemm_f64_host keeps mapped (up to 1.25 GiB).
+ * All of it comes back on demand. Synchronises the device first (a kernel of an earlier call may
+ * still be using the memory), so it must not be called while a stream is being captured. Returns
+ * DGEMM_OK, DGEMM_ERR_DEVICE or DGEMM_ERR_CUDA. No counterpart in the paper.
+ */
+DGEMM_API int dgemm_release_scratch(void);
+
+/*
  * Number of kernels this library has launched so far in this process (all entry points).
  * Monotonic; used by the benchmark to report launches per step.
  */

@@ -104,6 +104,8 @@ def load_library() -> ctypes.CDLL:
             lib.dgemm_last_device_status.restype = ctypes.c_int
             lib.dgemm_selftest_wait_timeout.argtypes = [ctypes.c_int]
             lib.dgemm_selftest_wait_timeout.restype = ctypes.c_int
+            lib.dgemm_release_scratch.argtypes = []
+            lib.dgemm_release_scratch.restype = ctypes.c_int
             lib.dgemm_launch_count.argtypes = []
             lib.dgemm_launch_count.restype = ctypes.c_int64
             lib.dgemm_fp64_peak_probe.argtypes = [ctypes.c_int, ctypes.POINTER(ctypes.c_double),
@@ -300,6 +302,14 @@ def dgemm_selftest_wait_timeout(limit_us: int = 1000) -> int:
 
 def dgemm_launch_count() -> int:
     return int(load_library().dgemm_launch_count())
+
+
+def dgemm_release_scratch() -> int:
+    """Frees the library's device scratch on the current device (it comes back on demand)."""
+    rc = load_library().dgemm_release_scratch()
+    if rc < 0:
+        raise DgemmError(rc, "dgemm_release_scratch")
+    return rc
 
 
 def dgemm_fp64_peak_probe(millis: int = 200):

@@ -1109,6 +1109,30 @@ int dgemm_last_device_status(void* stream) {
   return word;
 }
 
+int dgemm_release_scratch(void) {
+  DeviceState* st = nullptr;
+  int rc = device_state(&st);
+  if (rc != DGEMM_OK) return rc;
+  if (cudaDeviceSynchronize() != cudaSuccess) {
+    (void)cudaGetLastError();
+    return DGEMM_ERR_CUDA;
+  }
+  std::lock_guard<std::mutex> lock(g_mutex);
+  bool ok = true;
+  if (st->workspace) {
+    ok = cudaFree(st->workspace) == cudaSuccess && ok;
+    st->workspace = nullptr;
+  }
+  if (st->pack_buf) {
+    ok = cudaFree(st->pack_buf) == cudaSuccess && ok;
+    st->pack_buf = nullptr;
+    st->pack_bytes = 0;
+  }
+  if (st->host_pool) ok = cudaMemPoolTrimTo(st->host_pool, 0) == cudaSuccess && ok;
+  if (!ok) (void)cudaGetLastError();
+  return ok ? DGEMM_OK : DGEMM_ERR_CUDA;
+}
+
 int64_t dgemm_launch_count(void) { return g_launches.load(); }
 
 int dgemm_selftest_wait_timeout(int limit_us) {

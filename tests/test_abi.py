@@ -27,7 +27,7 @@ def test_every_declared_symbol_is_exported(lib):
     names = _declared(os.path.join(ROOT, "include", "dgemm.h"), r"DGEMM_API\s+[\w\s\*]+?\b(dgemm_\w+)\s*\(")
     assert {"dgemm_f64", "dgemm_f64_ex", "dgemm_f64_host", "dgemm_f64_static_ws", "dgemm_strerror", "dgemm_version",
             "dgemm_set_variant", "dgemm_set_split_k", "dgemm_set_test_flags", "dgemm_last_device_status", "dgemm_launch_count",
-            "dgemm_fp64_peak_probe", "dgemm_selftest_wait_timeout", "dgemm_plan"} <= set(names)
+            "dgemm_fp64_peak_probe", "dgemm_selftest_wait_timeout", "dgemm_plan", "dgemm_release_scratch"} <= set(names)
     for n in names:
         assert hasattr(lib, n), f"{n} is declared in dgemm.h but not exported by libdgemm.so"
     names32 = _declared(os.path.join(ROOT, "include", "sgemm.h"), r"DGEMM_API\s+[\w\s\*]+?\b(sgemm_\w+)\s*\(")

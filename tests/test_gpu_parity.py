@@ -450,3 +450,26 @@ def test_calls_can_be_captured_into_a_cuda_graph(shape):
     torch.cuda.synchronize()
     assert dg.dgemm_last_device_status() == dg.DGEMM_OK
     assert torch.equal(C, 4 * once)  # exact: small integers
+
+
+def test_release_scratch_and_carry_on(oracle):
+    """The workspace, the packing scratch and the host entry point's pool can be given back at any
+    quiet moment; the next calls allocate them again and give the same results."""
+    prob = wl.make_problem(700, 520, 300, seed=71, lda=303, ldb=525, ldc=527, integer=True)   # generic staging, K split
+    big = wl.make_problem(1300, 1250, 1300, seed=72, lda=1303, ldb=1255, ldc=1257, integer=True)  # packing pass
+    first = [run_gpu(prob), run_gpu(big)]
+    hostp = wl.make_problem(2500, 300, 200, seed=73, integer=True)
+    want = hostp.C.clone().contiguous().numpy()
+    oracle.dgemm_oracle(np.ascontiguousarray(hostp.A.numpy()), np.ascontiguousarray(hostp.B.numpy()), want)
+    c0 = hostp.C.clone()
+    dg.dgemm_f64_host(hostp.A, hostp.B, hostp.C)
+    assert np.array_equal(hostp.C.numpy(), want)
+    assert dg.dgemm_release_scratch() == dg.DGEMM_OK
+    assert dg.dgemm_release_scratch() == dg.DGEMM_OK   # nothing left to free: still fine
+    second = [run_gpu(prob), run_gpu(big)]
+    for a, b in zip(first, second):
+        assert torch.equal(a.view(torch.int64), b.view(torch.int64))
+    _check_full(oracle, prob, second[0])
+    hostp.C.copy_(c0)
+    dg.dgemm_f64_host(hostp.A, hostp.B, hostp.C)
+    assert np.array_equal(hostp.C.numpy(), want)

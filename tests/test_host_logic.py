@@ -93,6 +93,8 @@ def test_valid_call_without_gpu_fails_loudly():
     assert rc == -6  # no device: an error, never a CPU fallback
     with pytest.raises(dg.DgemmError):
         dg.dgemm_fp64_peak_probe(1)
+    with pytest.raises(dg.DgemmError):
+        dg.dgemm_release_scratch()
 
 
 def test_variant_and_split_setters():

@@ -143,7 +143,7 @@ dgemm_cluster_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
   bool ok = true;
   int issued = 0;  // TMA staging: meaningful in lane 0 of warp 0 only
   if (!USE_TMA) {
-    for (; issued < nkb && issued < LOOKAHEAD && ok; ++issued) ok = issue(issued);
+    for (; issued < nkb && issued < LOOKAHEAD && ok; ++issued) ok = __all_sync(0xffffffffu, issue(issued) ? 1 : 0);
   } else if (warp == 0) {
     int good = 1;
     if (lane == 0) {
@@ -194,11 +194,15 @@ dgemm_cluster_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
 
   for (int i = 0; i < nkb && ok; ++i) {
     const uint32_t s = (uint32_t)i % STAGES, ph = ((uint32_t)i / STAGES) & 1u;
-    if (!wait_bounded(full_bar + 8 * s, ph, abort_flag, p)) { ok = false; break; }
+    // Every decision to leave the loop is taken by the whole warp (a vote per wait: this kernel only
+    // runs problems of a few k-blocks), so no lane can be left behind in a warp-level
+    // synchronisation and every warp reaches the CTA and cluster barriers below.
+    const bool arrived = wait_bounded(full_bar + 8 * s, ph, abort_flag, p);
+    if (!__all_sync(0xffffffffu, arrived ? 1 : 0)) { ok = false; break; }
     compute_kblock<false, MT>(tiles + s * STAGE_BYTES, lm, acc);
     release_stage(empty_bar + 8 * s, lane);
     if (!USE_TMA) {
-      if (i + LOOKAHEAD < nkb && !issue(i + LOOKAHEAD)) { ok = false; break; }
+      if (i + LOOKAHEAD < nkb && !__all_sync(0xffffffffu, issue(i + LOOKAHEAD) ? 1 : 0)) { ok = false; break; }
     } else if (warp == 0 && i + LOOKAHEAD < nkb) {  // refill the stage all warps released two k-blocks ago
       int good = 1;
       if (lane == 0) {

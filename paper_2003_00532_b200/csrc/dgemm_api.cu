@@ -45,7 +45,7 @@ inline bool narrow_tiles_pay(int64_t N) {
 constexpr int kAutoWs64MaxKblocksPerCta = 256;     // ... and its 64-row form instead of the inline kernel up to this much work
 constexpr int kAutoWsMinKblocks = 16;                // warp-specialised kernel: 128-row tiles from K = 256 up, 64-row below
 constexpr double kPackMinFlopPerByte = 64.0;       // pack unaligned operands only if the copy is this cheap
-constexpr double kPackMinFlop = 4.0e9;             // ... and the problem is large enough for two more launches not to show
+constexpr double kPackMinFlop = 0.25e9;            // ... and the problem is not one of a few microseconds, where one more launch shows
 constexpr size_t kPackMaxBytes = 2ull << 30;       // ... and the packed copies fit in 2 GiB
 constexpr int64_t kHostBlockRows = 1024;             // dgemm_f64_host: rows of A and C per pipelined block
 constexpr int64_t kHostPanelRows = 1024;             // ... and rows of B per panel while the first blocks wait for B
@@ -624,27 +624,40 @@ int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, c
       if (rc != DGEMM_OK) return rc;
       double* pa = st->pack_buf;
       double* pb = reinterpret_cast<double*>(reinterpret_cast<char*>(st->pack_buf) + ((a_bytes + 255) & ~(size_t)255));
-      if (pack_a) {
-        if (form.ta) {  // stored K x M
-          dim3 grid((unsigned)((M + 31) / 32), grid_y((K + 31) / 32));
-          dgemm_transpose_kernel<<<grid, dim3(32, 8), 0, stream>>>(A, lda, (int)K, (int)M, pa, plda);
-        } else {
-          dim3 grid((unsigned)((K + 255) / 256), grid_y((M + 7) / 8));
-          dgemm_pack_kernel<<<grid, 128, 0, stream>>>(A, lda, (int)M, (int)K, pa, plda);
-        }
+      if (pack_a && form.ta) {  // stored K x M
+        dim3 grid((unsigned)((M + 31) / 32), grid_y((K + 31) / 32));
+        dgemm_transpose_kernel<<<grid, dim3(32, 8), 0, stream>>>(A, lda, (int)K, (int)M, pa, plda);
         g_launches.fetch_add(1);
+      }
+      if (pack_b && form.tb) {  // stored N x K
+        dim3 grid((unsigned)((K + 31) / 32), grid_y((N + 31) / 32));
+        dgemm_transpose_kernel<<<grid, dim3(32, 8), 0, stream>>>(B, ldb, (int)N, (int)K, pb, pldb);
+        g_launches.fetch_add(1);
+      }
+      // the plain copies of A and / or B: one launch
+      PackOp ops[2];
+      int nops = 0;
+      int64_t gx = 0, gy = 0;
+      if (pack_a && !form.ta) {
+        ops[nops++] = PackOp{A, lda, (int)M, (int)K, pa, plda};
+        gx = (K + 255) / 256;
+        gy = (M + 7) / 8;
+      }
+      if (pack_b && !form.tb) {
+        ops[nops++] = PackOp{B, ldb, (int)K, (int)N, pb, pldb};
+        if ((N + 255) / 256 > gx) gx = (N + 255) / 256;
+        if ((K + 7) / 8 > gy) gy = (K + 7) / 8;
+      }
+      if (nops > 0) {
+        if (nops == 1) ops[1] = ops[0];
+        launch_pdl(dgemm_pack2_kernel, dim3((unsigned)gx, grid_y(gy), (unsigned)nops), dim3(128), 0, stream, ops[0], ops[1]);
+        g_launches.fetch_add(1);
+      }
+      if (pack_a) {
         A = pa;
         lda = plda;
       }
       if (pack_b) {
-        if (form.tb) {  // stored N x K
-          dim3 grid((unsigned)((K + 31) / 32), grid_y((N + 31) / 32));
-          dgemm_transpose_kernel<<<grid, dim3(32, 8), 0, stream>>>(B, ldb, (int)N, (int)K, pb, pldb);
-        } else {
-          dim3 grid((unsigned)((N + 255) / 256), grid_y((K + 7) / 8));
-          dgemm_pack_kernel<<<grid, 128, 0, stream>>>(B, ldb, (int)K, (int)N, pb, pldb);
-        }
-        g_launches.fetch_add(1);
         B = pb;
         ldb = pldb;
       }

@@ -1232,6 +1232,36 @@ __global__ void dgemm_tail_reduce_kernel(const GemmParams p) {
 // dimension): copies a rows x cols matrix into a 16-byte aligned buffer with an even leading
 // dimension. This is the paper's packing step (Section 2.6) done once in HBM instead of per block;
 // it moves O(n^2) bytes for O(n^3) work. One thread per pair of columns.
+// The packing pass for one or two operands in one launch (blockIdx.z selects the operand; blocks
+// beyond the smaller operand's extent return at once). Launched with programmatic stream
+// serialization: waits for the kernel before it, which may still be reading the scratch it writes.
+struct PackOp {
+  const double* src;
+  long long ld_src;
+  int rows, cols;
+  double* dst;
+  long long ld_dst;
+};
+__global__ void dgemm_pack2_kernel(const PackOp a, const PackOp b) {
+  ptx::grid_dependency_wait();
+  const PackOp& o = blockIdx.z == 0 ? a : b;
+  const int c = 2 * (blockIdx.x * blockDim.x + threadIdx.x);
+  if (c >= o.cols) return;
+  for (int r0 = blockIdx.y * 8; r0 < o.rows; r0 += gridDim.y * 8) {  // gridDim.y may be capped
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const int r = r0 + i;
+      if (r < o.rows) {
+        const double* s = o.src + (long long)r * o.ld_src + c;
+        double2 v;
+        v.x = s[0];
+        v.y = (c + 1 < o.cols) ? s[1] : 0.0;
+        *reinterpret_cast<double2*>(o.dst + (long long)r * o.ld_dst + c) = v;
+      }
+    }
+  }
+}
+
 __global__ void dgemm_pack_kernel(const double* __restrict__ src, long long ld_src, int rows, int cols,
                                   double* __restrict__ dst, long long ld_dst) {
   const int c = 2 * (blockIdx.x * blockDim.x + threadIdx.x);

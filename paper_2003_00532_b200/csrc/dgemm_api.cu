@@ -626,12 +626,12 @@ int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, c
       double* pb = reinterpret_cast<double*>(reinterpret_cast<char*>(st->pack_buf) + ((a_bytes + 255) & ~(size_t)255));
       if (pack_a && form.ta) {  // stored K x M
         dim3 grid((unsigned)((M + 31) / 32), grid_y((K + 31) / 32));
-        dgemm_transpose_kernel<<<grid, dim3(32, 8), 0, stream>>>(A, lda, (int)K, (int)M, pa, plda);
+        launch_pdl(dgemm_transpose_kernel, grid, dim3(32, 8), 0, stream, A, (long long)lda, (int)K, (int)M, pa, (long long)plda);
         g_launches.fetch_add(1);
       }
       if (pack_b && form.tb) {  // stored N x K
         dim3 grid((unsigned)((K + 31) / 32), grid_y((N + 31) / 32));
-        dgemm_transpose_kernel<<<grid, dim3(32, 8), 0, stream>>>(B, ldb, (int)N, (int)K, pb, pldb);
+        launch_pdl(dgemm_transpose_kernel, grid, dim3(32, 8), 0, stream, B, (long long)ldb, (int)N, (int)K, pb, (long long)pldb);
         g_launches.fetch_add(1);
       }
       // the plain copies of A and / or B: one launch

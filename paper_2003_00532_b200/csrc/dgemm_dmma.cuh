@@ -1287,6 +1287,7 @@ __global__ void dgemm_pack_kernel(const double* __restrict__ src, long long ld_s
 __global__ void dgemm_transpose_kernel(const double* __restrict__ src, long long ld_src, int rows, int cols,
                                        double* __restrict__ dst, long long ld_dst) {
   __shared__ double tile[32][33];
+  ptx::grid_dependency_wait();  // launched with programmatic stream serialization, like the packing pass
   const int c0 = blockIdx.x * 32;
   for (int r0 = blockIdx.y * 32; r0 < rows; r0 += gridDim.y * 32) {  // gridDim.y may be capped
 #pragma unroll

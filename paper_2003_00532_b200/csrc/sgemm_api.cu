@@ -173,16 +173,25 @@ int launch(int64_t M, int64_t N, int64_t K, const float* A, int64_t lda, const f
     if (rc != DGEMM_OK) return rc;
     float* pa = st->pack_buf;
     float* pb = reinterpret_cast<float*>(reinterpret_cast<char*>(st->pack_buf) + ((a_bytes + 255) & ~(size_t)255));
+    PackOpF ops[2];
+    int nops = 0;
+    int64_t gx = 0, gy = 0;
     if (pack_a) {
-      sgemm_pack_kernel<<<dim3((unsigned)((K + 255) / 256), grid_y(M)), 256, 0, stream>>>(A, lda, (int)M, (int)K, pa, plda);
+      ops[nops++] = PackOpF{A, lda, (int)M, (int)K, pa, plda};
+      gx = (K + 255) / 256;
+      gy = M;
       A = pa;
       lda = plda;
     }
     if (pack_b) {
-      sgemm_pack_kernel<<<dim3((unsigned)((N + 255) / 256), grid_y(K)), 256, 0, stream>>>(B, ldb, (int)K, (int)N, pb, pldb);
+      ops[nops++] = PackOpF{B, ldb, (int)K, (int)N, pb, pldb};
+      if ((N + 255) / 256 > gx) gx = (N + 255) / 256;
+      if (K > gy) gy = K;
       B = pb;
       ldb = pldb;
     }
+    if (nops == 1) ops[1] = ops[0];
+    launch_pdl(sgemm_pack_kernel, dim3((unsigned)gx, grid_y(gy), (unsigned)nops), dim3(256), 0, stream, ops[0], ops[1]);
     if (cudaGetLastError() != cudaSuccess) return DGEMM_ERR_CUDA;
   }
 

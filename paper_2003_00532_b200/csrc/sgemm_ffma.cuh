@@ -400,11 +400,22 @@ __global__ void sgemm_tail_reduce_kernel(const Params p) {
 // Copies a rows x cols float matrix into a 16-byte aligned buffer whose leading dimension is a
 // multiple of 32 floats (operands TMA cannot address: base not 16-byte aligned or a leading
 // dimension that is not a multiple of 4). One thread per element of a row chunk; gridDim.y may be capped.
-__global__ void sgemm_pack_kernel(const float* __restrict__ src, long long ld_src, int rows, int cols,
-                                  float* __restrict__ dst, long long ld_dst) {
+// One or two operands per launch (blockIdx.z selects; blocks beyond the smaller operand's extent
+// return at once). Launched with programmatic stream serialization: waits for the kernel before
+// it, which may still be reading the scratch this one writes.
+struct PackOpF {
+  const float* src;
+  long long ld_src;
+  int rows, cols;
+  float* dst;
+  long long ld_dst;
+};
+__global__ void sgemm_pack_kernel(const PackOpF a, const PackOpF b) {
+  grid_dependency_wait();
+  const PackOpF& o = blockIdx.z == 0 ? a : b;
   const int c = blockIdx.x * blockDim.x + threadIdx.x;
-  if (c >= cols) return;
-  for (int r = blockIdx.y; r < rows; r += gridDim.y) dst[(long long)r * ld_dst + c] = src[(long long)r * ld_src + c];
+  if (c >= o.cols) return;
+  for (int r = blockIdx.y; r < o.rows; r += gridDim.y) o.dst[(long long)r * o.ld_dst + c] = o.src[(long long)r * o.ld_src + c];
 }
 
 }  // namespace sgemm

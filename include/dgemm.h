@@ -117,9 +117,11 @@ DGEMM_API int dgemm_f64(int64_t M, int64_t N, int64_t K,
  * Synchronous: returns after the result is in the host buffer. Device scratch comes from a memory
  * pool the library owns (stream-ordered allocation) and goes back to it before returning; the
  * pool keeps up to 1.25 GiB mapped between calls, because mapping a gigabyte anew on every call
- * cost more than the copies and the arithmetic
- * of an 8192^3 problem together. Same argument rules and error codes as dgemm_f64
- * (Section 2.1; the paper's driver likewise owns A, B, C in host memory).
+ * cost more than the copies and the arithmetic of an 8192^3 problem together. The call runs on
+ * streams of its own and uses the shared workspace: it must not overlap on the device with other
+ * calls of this library (a second host thread, or a dgemm_f64 still in flight on another
+ * stream). Same argument rules and error codes as dgemm_f64 (Section 2.1; the paper's driver
+ * likewise owns A, B, C in host memory).
  */
 DGEMM_API int dgemm_f64_host(int64_t M, int64_t N, int64_t K,
                    const double *A, int64_t lda,

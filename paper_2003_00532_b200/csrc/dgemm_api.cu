@@ -58,6 +58,8 @@ constexpr double kTailMinSavedKblocks = 5.0;  // use the stream-K tail only if i
 // the workspace round trip cost.
 constexpr int kClusterCreditKblocks = 1;
 constexpr int kClusterMaxKblocks = 8;
+// Column split of a ragged N (launch_gemm): M * K * (columns of arithmetic saved) above which the second launch pays
+constexpr double kColumnSplitMinWork = 2.0e8;
 
 __device__ int g_status_word;  // one per device that loads the library
 
@@ -593,77 +595,11 @@ struct GemmForm {
   double alpha = 1.0, beta = 1.0;
 };
 
-int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, const double* B, int64_t ldb,
-                double* C, int64_t ldc, cudaStream_t stream, const GemmForm& form = GemmForm()) {
-  DeviceState* st = nullptr;
-  int rc = device_state(&st);
-  if (rc != DGEMM_OK) return rc;
-
-  int variant = g_variant.load();
-  {
-    // A transposed operand is always rewritten (row-major, 128-byte aligned rows) into the pack
-    // buffer. An operand that TMA cannot address is repacked there when that is worth it: the copy
-    // (16 bytes moved per packed element) small next to the arithmetic, the scratch moderate.
-    const bool bad_a = !form.ta && (((uintptr_t)A & 15) != 0 || (lda % 2 != 0));
-    const bool bad_b = !form.tb && (((uintptr_t)B & 15) != 0 || (ldb % 2 != 0));
-    const int64_t plda = (K + 15) & ~(int64_t)15, pldb = (N + 15) & ~(int64_t)15;  // 128-byte aligned rows
-    const size_t a_all = (size_t)M * plda * 8, b_all = (size_t)K * pldb * 8;
-    bool pack_a = form.ta, pack_b = form.tb;
-    if (variant == DGEMM_VARIANT_AUTO && (bad_a || bad_b) && !(g_test_flags.load() & DGEMM_TEST_NO_PACKING)) {
-      const size_t bytes = ((pack_a || bad_a) ? a_all : 0) + ((pack_b || bad_b) ? b_all : 0);
-      const double flop_per_byte = 2.0 * (double)M * (double)N * (double)K / (double)bytes;
-      if (flop_per_byte >= kPackMinFlopPerByte && bytes <= kPackMaxBytes &&
-          2.0 * (double)M * (double)N * (double)K >= kPackMinFlop) {
-        pack_a = pack_a || bad_a;
-        pack_b = pack_b || bad_b;
-      }
-    }
-    if (pack_a || pack_b) {
-      const size_t a_bytes = pack_a ? a_all : 0, b_bytes = pack_b ? b_all : 0;
-      rc = ensure_pack_buffer(st, a_bytes + b_bytes + 256);
-      if (rc != DGEMM_OK) return rc;
-      double* pa = st->pack_buf;
-      double* pb = reinterpret_cast<double*>(reinterpret_cast<char*>(st->pack_buf) + ((a_bytes + 255) & ~(size_t)255));
-      if (pack_a && form.ta) {  // stored K x M
-        dim3 grid((unsigned)((M + 31) / 32), grid_y((K + 31) / 32));
-        launch_pdl(dgemm_transpose_kernel, grid, dim3(32, 8), 0, stream, A, (long long)lda, (int)K, (int)M, pa, (long long)plda);
-        g_launches.fetch_add(1);
-      }
-      if (pack_b && form.tb) {  // stored N x K
-        dim3 grid((unsigned)((K + 31) / 32), grid_y((N + 31) / 32));
-        launch_pdl(dgemm_transpose_kernel, grid, dim3(32, 8), 0, stream, B, (long long)ldb, (int)N, (int)K, pb, (long long)pldb);
-        g_launches.fetch_add(1);
-      }
-      // the plain copies of A and / or B: one launch
-      PackOp ops[2];
-      int nops = 0;
-      int64_t gx = 0, gy = 0;
-      if (pack_a && !form.ta) {
-        ops[nops++] = PackOp{A, lda, (int)M, (int)K, pa, plda};
-        gx = (K + 255) / 256;
-        gy = (M + 7) / 8;
-      }
-      if (pack_b && !form.tb) {
-        ops[nops++] = PackOp{B, ldb, (int)K, (int)N, pb, pldb};
-        if ((N + 255) / 256 > gx) gx = (N + 255) / 256;
-        if ((K + 7) / 8 > gy) gy = (K + 7) / 8;
-      }
-      if (nops > 0) {
-        if (nops == 1) ops[1] = ops[0];
-        launch_pdl(dgemm_pack2_kernel, dim3((unsigned)gx, grid_y(gy), (unsigned)nops), dim3(128), 0, stream, ops[0], ops[1]);
-        g_launches.fetch_add(1);
-      }
-      if (pack_a) {
-        A = pa;
-        lda = plda;
-      }
-      if (pack_b) {
-        B = pb;
-        ldb = pldb;
-      }
-      if (cudaGetLastError() != cudaSuccess) return DGEMM_ERR_CUDA;
-    }
-  }
+// Plans and launches one product on operands that are final (packed or transposed already where
+// that was needed): kernel choice, parameters, tensor maps, launches.
+int launch_gemm_packed(DeviceState* st, int variant, int64_t M, int64_t N, int64_t K, const double* A, int64_t lda,
+                       const double* B, int64_t ldb, double* C, int64_t ldc, cudaStream_t stream, const GemmForm& form) {
+  int rc = DGEMM_OK;
   const bool tma_ok = (((uintptr_t)A | (uintptr_t)B) & 15) == 0 && (lda % 2 == 0) && (ldb % 2 == 0);
   const int dbg_flags = g_test_flags.load();
   const Plan plan = plan_gemm(M, N, K, tma_ok, variant, dbg_flags, g_split_k.load(), st->sm_count, st->two_ctas_ok, st->ws_ok,
@@ -761,6 +697,94 @@ int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, c
     if (cudaGetLastError() != cudaSuccess) return DGEMM_ERR_CUDA;
   }
   return DGEMM_OK;
+}
+
+int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, const double* B, int64_t ldb,
+                double* C, int64_t ldc, cudaStream_t stream, const GemmForm& form = GemmForm()) {
+  DeviceState* st = nullptr;
+  int rc = device_state(&st);
+  if (rc != DGEMM_OK) return rc;
+
+  int variant = g_variant.load();
+  {
+    // A transposed operand is always rewritten (row-major, 128-byte aligned rows) into the pack
+    // buffer. An operand that TMA cannot address is repacked there when that is worth it: the copy
+    // (16 bytes moved per packed element) small next to the arithmetic, the scratch moderate.
+    const bool bad_a = !form.ta && (((uintptr_t)A & 15) != 0 || (lda % 2 != 0));
+    const bool bad_b = !form.tb && (((uintptr_t)B & 15) != 0 || (ldb % 2 != 0));
+    const int64_t plda = (K + 15) & ~(int64_t)15, pldb = (N + 15) & ~(int64_t)15;  // 128-byte aligned rows
+    const size_t a_all = (size_t)M * plda * 8, b_all = (size_t)K * pldb * 8;
+    bool pack_a = form.ta, pack_b = form.tb;
+    if (variant == DGEMM_VARIANT_AUTO && (bad_a || bad_b) && !(g_test_flags.load() & DGEMM_TEST_NO_PACKING)) {
+      const size_t bytes = ((pack_a || bad_a) ? a_all : 0) + ((pack_b || bad_b) ? b_all : 0);
+      const double flop_per_byte = 2.0 * (double)M * (double)N * (double)K / (double)bytes;
+      if (flop_per_byte >= kPackMinFlopPerByte && bytes <= kPackMaxBytes &&
+          2.0 * (double)M * (double)N * (double)K >= kPackMinFlop) {
+        pack_a = pack_a || bad_a;
+        pack_b = pack_b || bad_b;
+      }
+    }
+    if (pack_a || pack_b) {
+      const size_t a_bytes = pack_a ? a_all : 0, b_bytes = pack_b ? b_all : 0;
+      rc = ensure_pack_buffer(st, a_bytes + b_bytes + 256);
+      if (rc != DGEMM_OK) return rc;
+      double* pa = st->pack_buf;
+      double* pb = reinterpret_cast<double*>(reinterpret_cast<char*>(st->pack_buf) + ((a_bytes + 255) & ~(size_t)255));
+      if (pack_a && form.ta) {  // stored K x M
+        dim3 grid((unsigned)((M + 31) / 32), grid_y((K + 31) / 32));
+        launch_pdl(dgemm_transpose_kernel, grid, dim3(32, 8), 0, stream, A, (long long)lda, (int)K, (int)M, pa, (long long)plda);
+        g_launches.fetch_add(1);
+      }
+      if (pack_b && form.tb) {  // stored N x K
+        dim3 grid((unsigned)((K + 31) / 32), grid_y((N + 31) / 32));
+        launch_pdl(dgemm_transpose_kernel, grid, dim3(32, 8), 0, stream, B, (long long)ldb, (int)N, (int)K, pb, (long long)pldb);
+        g_launches.fetch_add(1);
+      }
+      // the plain copies of A and / or B: one launch
+      PackOp ops[2];
+      int nops = 0;
+      int64_t gx = 0, gy = 0;
+      if (pack_a && !form.ta) {
+        ops[nops++] = PackOp{A, lda, (int)M, (int)K, pa, plda};
+        gx = (K + 255) / 256;
+        gy = (M + 7) / 8;
+      }
+      if (pack_b && !form.tb) {
+        ops[nops++] = PackOp{B, ldb, (int)K, (int)N, pb, pldb};
+        if ((N + 255) / 256 > gx) gx = (N + 255) / 256;
+        if ((K + 7) / 8 > gy) gy = (K + 7) / 8;
+      }
+      if (nops > 0) {
+        if (nops == 1) ops[1] = ops[0];
+        launch_pdl(dgemm_pack2_kernel, dim3((unsigned)gx, grid_y(gy), (unsigned)nops), dim3(128), 0, stream, ops[0], ops[1]);
+        g_launches.fetch_add(1);
+      }
+      if (pack_a) {
+        A = pa;
+        lda = plda;
+      }
+      if (pack_b) {
+        B = pb;
+        ldb = pldb;
+      }
+      if (cudaGetLastError() != cudaSuccess) return DGEMM_ERR_CUDA;
+    }
+  }
+  // A column count just above a multiple of 128 on a large problem: the last tile column of 128
+  // would be at most half full. The full tile columns and the remainder are run as two products on
+  // disjoint columns of C, the remainder with the 256 x 32 tiles (2088^3: 573 -> 565 us, 4136^3: 4106
+  // -> 4051 us; not worth it below: 1064^3 91 -> 100 us). The sub-matrices start at a multiple of 128
+  // columns, so whatever alignment B and C have is kept.
+  if (variant == DGEMM_VARIANT_AUTO && g_test_flags.load() == 0 && g_split_k.load() <= 0) {
+    const int64_t r = N % BN, r32 = (r + 31) / 32 * 32;
+    const bool addressable = (((uintptr_t)A | (uintptr_t)B) & 15) == 0 && (lda % 2 == 0) && (ldb % 2 == 0);
+    if (addressable && N >= 1024 && r >= 1 && r <= 64 && (double)M * (double)K * (128.0 - 1.2 * (double)r32) > kColumnSplitMinWork) {
+      rc = launch_gemm_packed(st, variant, M, N - r, K, A, lda, B, ldb, C, ldc, stream, form);
+      if (rc != DGEMM_OK) return rc;
+      return launch_gemm_packed(st, variant, M, r, K, A, lda, B + (N - r), ldb, C + (N - r), ldc, stream, form);
+    }
+  }
+  return launch_gemm_packed(st, variant, M, N, K, A, lda, B, ldb, C, ldc, stream, form);
 }
 
 // ---- split-K through a statically allocated workspace (no allocation at run time) --------------

@@ -472,3 +472,30 @@ def test_release_scratch_and_carry_on(oracle):
     hostp.C.copy_(c0)
     dg.dgemm_f64_host(hostp.A, hostp.B, hostp.C)
     assert np.array_equal(hostp.C.numpy(), want)
+
+
+@pytest.mark.parametrize("integer", [True, False])
+@pytest.mark.parametrize("shape", [(2000, 1064, 2000), (2100, 1300, 2050)])
+def test_ragged_n_on_a_large_problem_runs_as_two_products(oracle, shape, integer):
+    """N just above a multiple of 128 on a large problem: the full tile columns and the narrow
+    remainder are separate launches on disjoint columns of C (padded, odd ldc in the second case:
+    both parts go through the staged epilogue)."""
+    M, N, K = shape
+    prob = wl.make_problem(M, N, K, seed=81, ldc=N + (7 if N == 1300 else 0), integer=integer)
+    n0 = dg.dgemm_launch_count()
+    out = run_gpu(prob)
+    assert dg.dgemm_launch_count() - n0 >= 2
+    _check_freivalds(oracle, prob, out)
+    _check_sampled(oracle, prob, out, 4096, seed=5)
+    # the columns on both sides of the cut, every row
+    import numpy as _np
+    cut = N - N % 128
+    ii = _np.repeat(_np.arange(M), 4)
+    jj = _np.tile(_np.array([cut - 1, cut, cut + 1, N - 1]), M)
+    want = oracle.dgemm_oracle_entries(prob.A.numpy(), prob.B.numpy(), prob.C.numpy(), ii, jj)
+    got = out[:, :N].numpy()[ii, jj]
+    if integer:
+        assert _np.array_equal(got, want)
+    else:
+        scale = oracle.dgemm_oracle_entries(prob.A.numpy(), prob.B.numpy(), prob.C.numpy(), ii, jj, absolute=True)
+        assert (_np.abs(got - want) <= 2.0 * (K + 1) * oracle.U * scale).all()

@@ -44,7 +44,8 @@ inline bool narrow_tiles_pay(int64_t N) {
 }
 constexpr int kAutoWs64MaxKblocksPerCta = 256;     // ... and its 64-row form instead of the inline kernel up to this much work
 constexpr int kAutoWsMinKblocks = 16;                // warp-specialised kernel: 128-row tiles from K = 256 up, 64-row below
-constexpr double kPackMinFlopPerByte = 64.0;       // pack unaligned operands only if the copy is this cheap
+constexpr double kPackMinFlopPerByte = 32.0;      // pack unaligned operands only if the copy is this cheap
+constexpr double kPackMinFlopPerByteNarrow = 8.0; // ... or this cheap where the generic staging would run the 256 x 32 tile, its slowest form
 constexpr double kPackMinFlop = 0.25e9;            // ... and the problem is not one of a few microseconds, where one more launch shows
 constexpr size_t kPackMaxBytes = 2ull << 30;       // ... and the packed copies fit in 2 GiB
 constexpr int64_t kHostBlockRows = 1024;             // dgemm_f64_host: rows of A and C per pipelined block
@@ -718,7 +719,7 @@ int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, c
     if (variant == DGEMM_VARIANT_AUTO && (bad_a || bad_b) && !(g_test_flags.load() & DGEMM_TEST_NO_PACKING)) {
       const size_t bytes = ((pack_a || bad_a) ? a_all : 0) + ((pack_b || bad_b) ? b_all : 0);
       const double flop_per_byte = 2.0 * (double)M * (double)N * (double)K / (double)bytes;
-      if (flop_per_byte >= kPackMinFlopPerByte && bytes <= kPackMaxBytes &&
+      if (flop_per_byte >= (narrow_tiles_pay(N) ? kPackMinFlopPerByteNarrow : kPackMinFlopPerByte) && bytes <= kPackMaxBytes &&
           2.0 * (double)M * (double)N * (double)K >= kPackMinFlop) {
         pack_a = pack_a || bad_a;
         pack_b = pack_b || bad_b;

@@ -298,17 +298,23 @@ int ensure_host_pool(DeviceState* st, cudaMemPool_t* pool) {
     props.location.type = cudaMemLocationTypeDevice;
     props.location.id = dev;
     cudaMemPool_t created = nullptr;
-    if (cudaMemPoolCreate(&created, &props) != cudaSuccess) {
-      (void)cudaGetLastError();
-      return DGEMM_ERR_CUDA;
-    }
     unsigned long long keep = kHostPoolKeepBytes;
-    if (cudaMemPoolSetAttribute(created, cudaMemPoolAttrReleaseThreshold, &keep) != cudaSuccess) {
+    if (cudaMemPoolCreate(&created, &props) == cudaSuccess &&
+        cudaMemPoolSetAttribute(created, cudaMemPoolAttrReleaseThreshold, &keep) == cudaSuccess) {
+      st->host_pool = created;
+    } else {
+      // no pool of our own (an unusual driver configuration): the device's default pool still
+      // works, only slower, as it keeps nothing between calls
       (void)cudaGetLastError();
-      cudaMemPoolDestroy(created);
-      return DGEMM_ERR_CUDA;
+      if (created) cudaMemPoolDestroy(created);
+      cudaMemPool_t fallback = nullptr;
+      if (cudaDeviceGetDefaultMemPool(&fallback, dev) != cudaSuccess || !fallback) {
+        (void)cudaGetLastError();
+        return DGEMM_ERR_CUDA;
+      }
+      *pool = fallback;
+      return DGEMM_OK;
     }
-    st->host_pool = created;
   }
   *pool = st->host_pool;
   return DGEMM_OK;

@@ -3,9 +3,10 @@
  *
  * See dgemm_oracle.h for the semantics and the list of pins. Build with
  *   gcc -O2 -fno-fast-math -ffp-contract=off -fopenmp -shared -fPIC
- * so that the compiler neither reassociates sums nor contracts a*b+c into an fma: the
- * operation sequence per output element is exactly the one of the paper's naive nest
- * (Section 2.1, "Affine Ops": load a, load b, load c, multiply, add, store c).
+ * so that the compiler neither reassociates sums nor contracts a*b+c into an fma: every
+ * output element is the running sum c = c + a*b over ascending k, started from the incoming
+ * C value, with the product and the sum each rounded once (the operation C += A*B of the
+ * paper's Section 2.1).
  *
  * Nothing here is blocked, packed, unrolled or otherwise tuned, on purpose.
  */
@@ -17,22 +18,25 @@
 #include <omp.h>
 #endif
 
-/* The definition: for i, for j, for k: C[i][j] = C[i][j] + A[i][k]*B[k][j]. */
+/*
+ * The definition. Each entry is one inner product added to what C already holds: a scalar
+ * starts at C[i][j], takes the K products in ascending k, and is written back once. Nothing
+ * else touches C[i][j] meanwhile, so keeping the sum in a scalar rounds exactly as updating
+ * C in memory after every k would.
+ */
 void dgemm_oracle_ijk(int64_t M, int64_t N, int64_t K,
                       const double *A, int64_t lda,
                       const double *B, int64_t ldb,
                       double *C, int64_t ldc)
 {
     for (int64_t i = 0; i < M; ++i) {
+        const double *arow = A + i * lda;
         for (int64_t j = 0; j < N; ++j) {
+            double acc = C[i * ldc + j];
             for (int64_t k = 0; k < K; ++k) {
-                double a = A[i * lda + k];
-                double b = B[k * ldb + j];
-                double ci = C[i * ldc + j];
-                volatile double p = a * b; /* separately rounded product (mulf) */
-                double co = ci + p;        /* separately rounded sum (addf)     */
-                C[i * ldc + j] = co;
+                acc = acc + arow[k] * B[k * ldb + j]; /* -ffp-contract=off: two roundings */
             }
+            C[i * ldc + j] = acc;
         }
     }
 }
@@ -86,8 +90,7 @@ void dgemm_oracle_entries(int64_t K,
             double a = A[i * lda + k];
             double b = B[k * ldb + j];
             if (absolute) { a = fabs(a); b = fabs(b); }
-            volatile double p = a * b;
-            c = c + p;
+            c = c + a * b; /* two roundings, as above */
         }
         out[s] = c;
     }

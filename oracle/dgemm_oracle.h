@@ -12,9 +12,8 @@
  *
  *     C[i][j] <- C[i][j] + sum_{k=0..K-1} A[i][k] * B[k][j]        (alpha = beta = 1)
  *
- * evaluated for each (i,j) as c = c + a*b with k ascending, a separately rounded multiply
- * followed by a separately rounded add (the nest has a mulf then an addf), round to nearest
- * even. Columns j >= N of C (row padding) are never written; columns k >= K of A and j >= N
+ * evaluated for each (i,j) as c = c + a*b with k ascending, the product and the sum each
+ * rounded once (no fused multiply-add), round to nearest even. Columns j >= N of C (row padding) are never written; columns k >= K of A and j >= N
  * of B are never read.
  *
  * Parity pins (tests/test_oracle_pins.py): the all-ones driver input of the paper
@@ -32,7 +31,7 @@
 extern "C" {
 #endif
 
-/* The definition itself: loops i, j, k exactly as the naive nest. Single-threaded. Host pointers. */
+/* The definition itself: loops i, j, k, one running sum per entry. Single-threaded. Host pointers. */
 void dgemm_oracle_ijk(int64_t M, int64_t N, int64_t K,
                       const double *A, int64_t lda,
                       const double *B, int64_t ldb,

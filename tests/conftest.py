@@ -18,3 +18,21 @@ def oracle():
     import oracle as _oracle
     _oracle.build()
     return _oracle
+
+
+# Largest observed error / stated-bound ratio per benchmark configuration, collected by the parity
+# tests. With DGEMM_PARITY_REPORT=<path> in the environment the table is written there as JSON at
+# the end of the session (documentation of the margin; the assertions themselves are in the tests).
+_PARITY_RATIOS = {}
+
+
+def record_ratio(name: str, ratio: float) -> None:
+    _PARITY_RATIOS[name] = max(ratio, _PARITY_RATIOS.get(name, 0.0))
+
+
+def pytest_sessionfinish(session, exitstatus):
+    path = os.environ.get("DGEMM_PARITY_REPORT")
+    if path and _PARITY_RATIOS:
+        import json
+        with open(path, "w") as f:
+            json.dump(_PARITY_RATIOS, f, indent=1, sort_keys=True)

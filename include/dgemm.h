@@ -172,12 +172,16 @@ DGEMM_API int dgemm_f64_ex(int transa, int transb, int64_t M, int64_t N, int64_t
  * split-K workspace on first need and so is not suitable for them on small problems.
  *
  * Arguments and error codes are those of dgemm_f64, plus:
- *   split_k   number of K partitions; 0 lets the library choose (at least 2). It is clamped to
- *             the number of 16-wide k-blocks; a problem with a single k-block (K <= 16) runs
- *             unsplit and does not touch the array.
- * Capacity: ceil(M/128) * ceil(N/128) * split_k <= 128 partial tiles. A larger problem returns
- * DGEMM_ERR_SIZE and launches nothing (use dgemm_f64, or a smaller split_k). A negative
- * split_k returns DGEMM_ERR_VARIANT.
+ *   split_k   number of K partitions. It is clamped to the number of 16-wide k-blocks, and
+ *             partitions that would be empty are dropped. 0 lets the library choose: the most
+ *             partitions that the SMs and the array can take (at least 2), or, for a problem
+ *             with more than 64 output tiles, 1.
+ * Capacity: the array is used only when more than one partition results, and then
+ * ceil(M/128) * ceil(N/128) * partitions <= 128 partial tiles must hold. A request beyond that
+ * returns DGEMM_ERR_SIZE and launches nothing (use dgemm_f64, or a smaller split_k). A call that
+ * ends up with one partition (split_k == 1, the library's choice on a large problem, or
+ * K <= 16) runs unsplit, does not touch the array and has no size limit. A negative split_k
+ * returns DGEMM_ERR_VARIANT.
  *
  * The first call on each device looks up the array's device address and configures the
  * kernels (no allocation, but several runtime set-up calls): make that first call before any

@@ -856,28 +856,32 @@ int launch_gemm_static_ws(int64_t M, int64_t N, int64_t K, const double* A, int6
 
   const int64_t tiles = (int64_t)p.tiles_m * p.tiles_n;
   const int kblocks = (int)((K + BK - 1) / BK);
-  if (tiles > kStaticPartialTiles) return DGEMM_ERR_SIZE;
-  int split = split_k;
-  if (split <= 0) {  // as many partitions as the SMs and the array can take, at least 4 k-blocks each
-    split = st->sm_count / (int)tiles;
+  int64_t split = split_k;
+  if (split <= 0) {
+    // the library's choice: as many partitions as the SMs and the array can take, at least 4
+    // k-blocks each; a problem too large for two partial tiles per output tile runs unsplit,
+    // which needs no scratch at all
+    split = st->sm_count / tiles;
     if (split > kblocks / 4) split = kblocks / 4;
-    if (split > kStaticPartialTiles / (int)tiles) split = kStaticPartialTiles / (int)tiles;
-    if (split < 2) split = 2;
+    if (split > kStaticPartialTiles / tiles) split = kStaticPartialTiles / tiles;
+    if (split < 2) split = (2 * tiles <= kStaticPartialTiles) ? 2 : 1;
   }
   if (split > kblocks) split = kblocks;
   p.kblocks = kblocks;
   p.dp_tiles = (int)tiles;  // uniform split-K over all tiles, no tail phase
   p.tail_tiles = 0;
   p.tail_ipc = 1;
-  p.kblocks_per_split = (kblocks + split - 1) / split;
+  p.kblocks_per_split = (int)((kblocks + split - 1) / split);
   p.split_k = (kblocks + p.kblocks_per_split - 1) / p.kblocks_per_split;
   if (p.split_k > 1) {
+    // the only use of the array; a call that ends up unsplit (split_k == 1, or a single k-block)
+    // never touches it and has no size limit
     if (tiles * p.split_k > kStaticPartialTiles) return DGEMM_ERR_SIZE;
     p.partial = partials;  // every (tile, partition) slot in use is fully overwritten: nothing to clear
   }
 
-  const int units = (int)tiles * p.split_k;
-  const int grid = units < st->sm_count ? units : st->sm_count;
+  const int64_t units = tiles * p.split_k;
+  const int grid = units < st->sm_count ? (int)units : st->sm_count;
   CUtensorMap map_a, map_b;
   memset(&map_a, 0, sizeof(map_a));
   memset(&map_b, 0, sizeof(map_b));

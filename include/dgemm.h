@@ -85,16 +85,21 @@ enum {
  *
  * Operands that the tensor-copy engine cannot address (A or B not 16-byte aligned, or an odd
  * leading dimension) are, when the problem is large enough for the copy to be cheap next to the
- * arithmetic, first packed into a library-owned per-device scratch buffer (grown on demand with
- * a synchronising cudaFree/cudaMalloc, at most 2 GiB); smaller ones are staged directly with
- * 8-byte copies. The same sharing rule as for the workspace below applies to that buffer.
+ * arithmetic, first packed into library-owned scratch memory (grown on demand, at most 2 GiB
+ * per problem); smaller ones are staged directly with 8-byte copies. Problems with few output
+ * tiles split K over several thread blocks; their partial sums go through a library-owned
+ * workspace of 80 MiB.
  *
- * Problems with few output tiles split K over several thread blocks; their partial sums go
- * through a library-owned per-device workspace that is allocated on first need (a synchronising
- * cudaMalloc; do that first call outside stream capture) and is shared by all calls, which are
- * therefore serialised on the device in stream order only when they use the same stream.
- * Thread-safety: concurrent calls from several host threads are allowed; calls that need the
- * split-K workspace must not overlap on the device.
+ * Concurrency: calls may be made from several host threads and may be in flight on several
+ * streams at once. The scratch memory above is leased per call: a call on a stream never shares
+ * its lease with a call still in flight on another stream (calls on one stream run in stream
+ * order and reuse one lease). A device holds at most four leases; with more streams than that
+ * in flight, a call first makes its stream wait for the least recently used lease's last user.
+ * Leases are allocated on first need with a synchronising cudaMalloc: make the first call on a
+ * stream outside stream capture. As long as all calls on a device come from one stream nothing
+ * else synchronises; the first call on a second stream synchronises the device once. Calls
+ * recorded into a CUDA graph use the lease their stream had at capture time; replays of the graph
+ * are not covered by the guarantee above and must not overlap other calls that use scratch.
  *
  * The kernels are launched with programmatic stream serialization: their thread blocks may be
  * scheduled while the previous kernel in `stream` is finishing, but they wait for its completion
@@ -118,9 +123,8 @@ DGEMM_API int dgemm_f64(int64_t M, int64_t N, int64_t K,
  * pool the library owns (stream-ordered allocation) and goes back to it before returning; the
  * pool keeps up to 1.25 GiB mapped between calls, because mapping a gigabyte anew on every call
  * cost more than the copies and the arithmetic of an 8192^3 problem together. The call runs on
- * streams of its own and uses the shared workspace: it must not overlap on the device with other
- * calls of this library (a second host thread, or a dgemm_f64 still in flight on another
- * stream). Same argument rules and error codes as dgemm_f64 (Section 2.1; the paper's driver
+ * streams of its own and leases its scratch like any other call, so it may overlap with other
+ * calls of this library. Same argument rules and error codes as dgemm_f64 (Section 2.1; the paper's driver
  * likewise owns A, B, C in host memory).
  */
 DGEMM_API int dgemm_f64_host(int64_t M, int64_t N, int64_t K,
@@ -146,8 +150,8 @@ DGEMM_API int dgemm_f64_host(int64_t M, int64_t N, int64_t K,
  * Arithmetic: each C element receives beta*C_old + alpha*s, s the K-term inner product summed as
  * in dgemm_f64; alpha = beta = 1 with no transposition gives bit-identical results to dgemm_f64.
  * A transposed operand is first transposed into device scratch memory owned by the library
- * (an O(MK) or O(KN) pass before O(MNK) arithmetic; the buffer is kept and reused), so calls
- * with a transposed or repacked operand on one device must not overlap on the GPU.
+ * (an O(MK) or O(KN) pass before O(MNK) arithmetic; the buffer is kept and reused, and leased
+ * per call like the rest of the scratch: see dgemm_f64).
  * Same pointer, alignment, aliasing and error rules as dgemm_f64; an op code other than the two
  * above returns DGEMM_ERR_BAD_DIM.
  */
@@ -227,10 +231,6 @@ enum {
   DGEMM_TEST_NO_PACKING = 16,   /* never pack unaligned operands: always use the generic staging      */
   DGEMM_TEST_WS_TWO_CTAS = 32,  /* DGEMM_VARIANT_TMA_WS: 64-row tiles, two CTAs per SM, at any K (the
                                    library itself uses that form only for K < 256)                 */
-  DGEMM_TEST_FUSED_TAIL_REDUCE = 64, /* add the partial tiles of the last wave to C inside the GEMM kernel
-                                   (cooperative launch; the CTAs of a tile wait for one another, with
-                                   a time limit) instead of in a second kernel: same results bit for
-                                   bit, one launch fewer, measured slower                          */
   DGEMM_TEST_NO_CLUSTER = 128   /* DGEMM_VARIANT_AUTO never picks the cluster split-K kernel: problems
                                    below one wave of tiles cut K through the workspace instead   */
 };
@@ -260,9 +260,10 @@ DGEMM_API int dgemm_plan(int64_t M, int64_t N, int64_t K, int tma_addressable, i
 DGEMM_API int dgemm_last_device_status(void *stream);
 
 /*
- * Gives the device memory the library holds on the current device back to the system: the split-K
- * workspace (80 MiB), the scratch of the packing pass (up to 2.5 GiB, as large as the largest
- * packed problem so far) and what the memory pool of dgemm_f64_host keeps mapped (up to 1.25 GiB).
+ * Gives the device memory the library holds on the current device back to the system: every
+ * scratch lease (an 80 MiB split-K workspace and a packing buffer of up to 2.5 GiB each, as large
+ * as the largest packed problem so far; up to four leases) and what the memory pool of
+ * dgemm_f64_host keeps mapped (up to 1.25 GiB).
  * All of it comes back on demand. Synchronises the device first (a kernel of an earlier call may
  * still be using the memory), so it must not be called while a stream is being captured. Returns
  * DGEMM_OK, DGEMM_ERR_DEVICE or DGEMM_ERR_CUDA. No counterpart in the paper.

@@ -36,9 +36,10 @@ extern "C" {
  * M == 0 or N == 0: DGEMM_OK without inspecting pointers. K == 0: DGEMM_OK, C untouched.
  * Pointers must be 4-byte aligned (DGEMM_ERR_ALIGN); C must not overlap A or B (DGEMM_ERR_ALIAS).
  * Operands that the tensor-copy engine cannot address (A or B not 16-byte aligned, or a leading
- * dimension that is not a multiple of 4) are first copied into a library-owned per-device scratch
- * buffer (grown on demand with a synchronising cudaFree/cudaMalloc); calls that need it must not
- * overlap on the device. Other error codes as for dgemm_f64.
+ * dimension that is not a multiple of 4) are first copied into library-owned scratch memory (grown
+ * on demand with a synchronising cudaMalloc). That buffer and the workspace of the partial tiles
+ * are leased per call exactly as for dgemm_f64, so calls may be in flight on several streams at
+ * once. Other error codes as for dgemm_f64.
  */
 DGEMM_API int sgemm_f32(int64_t M, int64_t N, int64_t K,
                         const float *A, int64_t lda,

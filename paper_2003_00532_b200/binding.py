@@ -48,7 +48,6 @@ DGEMM_TEST_TALL_TILES = 4
 DGEMM_TEST_SMALL_WARP_TILES = 8
 DGEMM_TEST_NO_PACKING = 16
 DGEMM_TEST_WS_TWO_CTAS = 32
-DGEMM_TEST_FUSED_TAIL_REDUCE = 64
 DGEMM_TEST_NO_CLUSTER = 128
 
 

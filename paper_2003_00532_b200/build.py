@@ -1,6 +1,7 @@
 """Builds ``libdgemm.so`` in-tree with nvcc for sm_100a (cross-compiles without a GPU)."""
 from __future__ import annotations
 
+import glob
 import os
 import shlex
 import subprocess
@@ -10,8 +11,9 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libdgemm.so")
 SOURCES = [os.path.join(CSRC, "dgemm_api.cu"), os.path.join(CSRC, "sgemm_api.cu")]
-DEPS = SOURCES + [os.path.join(CSRC, f) for f in ("dgemm_dmma.cuh", "sgemm_ffma.cuh", "ptx.cuh")] + [
-    os.path.join(os.path.dirname(HERE), "include", f) for f in ("dgemm.h", "sgemm.h")]
+# every source, header and public header: an edit to any of them makes the built library stale
+DEPS = sorted(glob.glob(os.path.join(CSRC, "*.cu")) + glob.glob(os.path.join(CSRC, "*.cuh")) +
+              glob.glob(os.path.join(CSRC, "*.h")) + glob.glob(os.path.join(os.path.dirname(HERE), "include", "*.h")))
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

@@ -17,6 +17,7 @@
 
 #include "dgemm_dmma.cuh"
 #include "dgemm_cluster.cuh"
+#include "scratch_pool.h"
 
 namespace {
 
@@ -24,7 +25,6 @@ using namespace dgemm;
 
 constexpr int kMaxDevices = 64;
 constexpr size_t kWorkspaceBytes = 640ull * BM * BN * sizeof(double);  // 80 MiB: up to 640 partial-tile slots
-constexpr size_t kCounterBytes = 65536;  // in front of the slots: two counters per tail tile (fused tail reduction)
 constexpr unsigned long long kWaitLimitNs = 4000000000ull;            // 4 s per device-side wait
 constexpr int kAutoGeneric = DGEMM_VARIANT_GENERIC;  // what DGEMM_VARIANT_AUTO picks for operands TMA cannot address
 // Tile columns of 32 (the 256 x 32 tile, about 83 % of the pipe) against tile columns of 128 (about
@@ -71,9 +71,7 @@ struct DeviceState {
   bool ws_ok[3] = {false, false, false};  // register pool of the warp-specialised kernels checked: TMA 128, generic 128, TMA 64
   bool cluster_ok = false;     // a cluster of 8 CTAs of the cluster split-K kernel can be resident
   int* status = nullptr;       // device address of g_status_word
-  double* workspace = nullptr; // split-K partial tiles, allocated on first need
-  double* pack_buf = nullptr;  // packed copies of unaligned operands, grown on demand
-  size_t pack_bytes = 0;
+  scratch::Pool scratch;       // split-K partial tiles and packed operand copies, leased per call (scratch_pool.h)
   cudaMemPool_t host_pool = nullptr;  // dgemm_f64_host: device copies of the operands come from this pool
 };
 
@@ -130,18 +128,10 @@ void launch_cluster_pdl(void (*kernel)(KArgs...), int grid, int cluster, int thr
   cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
 }
 
-// Launches a GEMM kernel. When its CTAs wait for one another (the fused tail reduction) the launch
-// is cooperative: the driver then starts the grid only when all of its CTAs can be resident at
-// once, also next to other work on the GPU.
 template <typename Kernel>
 void launch_gemm_kernel(Kernel kernel, int grid, int threads, int smem, cudaStream_t stream, const CUtensorMap& map_a,
                         const CUtensorMap& map_b, const GemmParams& p) {
-  if (p.tail_fused) {
-    void* args[3] = {const_cast<CUtensorMap*>(&map_a), const_cast<CUtensorMap*>(&map_b), const_cast<GemmParams*>(&p)};
-    cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(kernel), dim3(grid), dim3(threads), args, (size_t)smem, stream);
-  } else {
-    launch_pdl(kernel, dim3(grid), dim3(threads), (size_t)smem, stream, map_a, map_b, p);
-  }
+  launch_pdl(kernel, dim3(grid), dim3(threads), (size_t)smem, stream, map_a, map_b, p);
 }
 
 template <bool USE_TMA, int TBM, int WTM, int TBN = BN>
@@ -269,19 +259,6 @@ int device_state(DeviceState** out) {
   return DGEMM_OK;
 }
 
-int ensure_workspace(DeviceState* st) {
-  std::lock_guard<std::mutex> lock(g_mutex);
-  if (!st->workspace) {
-    if (cudaMalloc(reinterpret_cast<void**>(&st->workspace), kCounterBytes + kWorkspaceBytes) != cudaSuccess) {
-      (void)cudaGetLastError();
-      return DGEMM_ERR_CUDA;
-    }
-    // the counters are zero between calls: the kernels that use them put them back
-    if (cudaMemset(st->workspace, 0, kCounterBytes) != cudaSuccess) return DGEMM_ERR_CUDA;
-  }
-  return DGEMM_OK;
-}
-
 // Memory pool of dgemm_f64_host. The device's default pool gives memory back to the system at
 // every synchronisation, so each call would pay for mapping its 0.8 GB (8192^3) again: more than
 // the copies and the arithmetic together. This pool keeps up to kHostPoolKeepBytes between calls.
@@ -317,25 +294,6 @@ int ensure_host_pool(DeviceState* st, cudaMemPool_t* pool) {
     }
   }
   *pool = st->host_pool;
-  return DGEMM_OK;
-}
-
-// Scratch for packed operands. Growing it frees the old buffer (cudaFree synchronises the device,
-// so no kernel can still be using it) and allocates a larger one.
-int ensure_pack_buffer(DeviceState* st, size_t bytes) {
-  std::lock_guard<std::mutex> lock(g_mutex);
-  if (st->pack_bytes >= bytes) return DGEMM_OK;
-  if (st->pack_buf) {
-    cudaFree(st->pack_buf);
-    st->pack_buf = nullptr;
-    st->pack_bytes = 0;
-  }
-  const size_t want = bytes + bytes / 4;  // head room against regrowing on slightly larger problems
-  if (cudaMalloc(reinterpret_cast<void**>(&st->pack_buf), want) != cudaSuccess) {
-    (void)cudaGetLastError();
-    return DGEMM_ERR_CUDA;
-  }
-  st->pack_bytes = want;
   return DGEMM_OK;
 }
 
@@ -604,8 +562,9 @@ struct GemmForm {
 
 // Plans and launches one product on operands that are final (packed or transposed already where
 // that was needed): kernel choice, parameters, tensor maps, launches.
-int launch_gemm_packed(DeviceState* st, int variant, int64_t M, int64_t N, int64_t K, const double* A, int64_t lda,
-                       const double* B, int64_t ldb, double* C, int64_t ldc, cudaStream_t stream, const GemmForm& form) {
+int launch_gemm_packed(DeviceState* st, scratch::Hold& hold, int variant, int64_t M, int64_t N, int64_t K, const double* A,
+                       int64_t lda, const double* B, int64_t ldb, double* C, int64_t ldc, cudaStream_t stream,
+                       const GemmForm& form) {
   int rc = DGEMM_OK;
   const bool tma_ok = (((uintptr_t)A | (uintptr_t)B) & 15) == 0 && (lda % 2 == 0) && (ldb % 2 == 0);
   const int dbg_flags = g_test_flags.load();
@@ -654,15 +613,8 @@ int launch_gemm_packed(DeviceState* st, int variant, int64_t M, int64_t N, int64
   p.tail_slot_base = 0;
   const bool uses_workspace = !cluster && (p.split_k > 1 || (p.tail_tiles > 0 && p.tail_ipc < kblocks));
   if (uses_workspace) {
-    rc = ensure_workspace(st);
-    if (rc != DGEMM_OK) return rc;
-    p.partial = st->workspace + kCounterBytes / sizeof(double);
-    p.tail_counters = reinterpret_cast<int*>(st->workspace);
-    // option: the CTAs that compute a tail tile also reduce it (not with a uniform K split, where a
-    // CTA may hold more than two partial tiles)
-    p.tail_fused = (p.split_k == 1 && p.tail_tiles > 0 && p.tail_ipc < kblocks &&
-                    (size_t)p.tail_tiles * 2 * sizeof(int) <= kCounterBytes && (dbg_flags & DGEMM_TEST_FUSED_TAIL_REDUCE))
-                       ? 1 : 0;
+    p.partial = static_cast<double*>(hold.workspace(kWorkspaceBytes));
+    if (!p.partial) return DGEMM_ERR_CUDA;
   }
 
   CUtensorMap map_a, map_b;
@@ -698,7 +650,7 @@ int launch_gemm_packed(DeviceState* st, int variant, int64_t M, int64_t N, int64
     g_launches.fetch_add(1);
     if (cudaGetLastError() != cudaSuccess) return DGEMM_ERR_CUDA;
   }
-  if (p.tail_tiles > 0 && p.tail_ipc < kblocks && !p.tail_fused) {
+  if (p.tail_tiles > 0 && p.tail_ipc < kblocks) {
     launch_pdl(dgemm_tail_reduce_kernel, dim3(p.tail_tiles, REDUCE_CHUNKS), dim3(REDUCE_THREADS), 0, stream, p);
     g_launches.fetch_add(1);
     if (cudaGetLastError() != cudaSuccess) return DGEMM_ERR_CUDA;
@@ -713,6 +665,9 @@ int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, c
   if (rc != DGEMM_OK) return rc;
 
   int variant = g_variant.load();
+  // The scratch this call needs (packed operands, partial tiles) is one lease of the device's pool,
+  // held until the last kernel below has been enqueued: calls on other streams get other leases.
+  scratch::Hold hold(st->scratch, stream);
   {
     // A transposed operand is always rewritten (row-major, 128-byte aligned rows) into the pack
     // buffer. An operand that TMA cannot address is repacked there when that is worth it: the copy
@@ -733,10 +688,9 @@ int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, c
     }
     if (pack_a || pack_b) {
       const size_t a_bytes = pack_a ? a_all : 0, b_bytes = pack_b ? b_all : 0;
-      rc = ensure_pack_buffer(st, a_bytes + b_bytes + 256);
-      if (rc != DGEMM_OK) return rc;
-      double* pa = st->pack_buf;
-      double* pb = reinterpret_cast<double*>(reinterpret_cast<char*>(st->pack_buf) + ((a_bytes + 255) & ~(size_t)255));
+      double* pa = static_cast<double*>(hold.pack_buffer(a_bytes + b_bytes + 256));
+      if (!pa) return DGEMM_ERR_CUDA;
+      double* pb = reinterpret_cast<double*>(reinterpret_cast<char*>(pa) + ((a_bytes + 255) & ~(size_t)255));
       if (pack_a && form.ta) {  // stored K x M
         dim3 grid((unsigned)((M + 31) / 32), grid_y((K + 31) / 32));
         launch_pdl(dgemm_transpose_kernel, grid, dim3(32, 8), 0, stream, A, (long long)lda, (int)K, (int)M, pa, (long long)plda);
@@ -786,12 +740,12 @@ int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, c
     const int64_t r = N % BN, r32 = (r + 31) / 32 * 32;
     const bool addressable = (((uintptr_t)A | (uintptr_t)B) & 15) == 0 && (lda % 2 == 0) && (ldb % 2 == 0);
     if (addressable && N >= 1024 && r >= 1 && r <= 64 && (double)M * (double)K * (128.0 - 1.2 * (double)r32) > kColumnSplitMinWork) {
-      rc = launch_gemm_packed(st, variant, M, N - r, K, A, lda, B, ldb, C, ldc, stream, form);
+      rc = launch_gemm_packed(st, hold, variant, M, N - r, K, A, lda, B, ldb, C, ldc, stream, form);
       if (rc != DGEMM_OK) return rc;
-      return launch_gemm_packed(st, variant, M, r, K, A, lda, B + (N - r), ldb, C + (N - r), ldc, stream, form);
+      return launch_gemm_packed(st, hold, variant, M, r, K, A, lda, B + (N - r), ldb, C + (N - r), ldc, stream, form);
     }
   }
-  return launch_gemm_packed(st, variant, M, N, K, A, lda, B, ldb, C, ldc, stream, form);
+  return launch_gemm_packed(st, hold, variant, M, N, K, A, lda, B, ldb, C, ldc, stream, form);
 }
 
 // ---- split-K through a statically allocated workspace (no allocation at run time) --------------
@@ -1132,7 +1086,7 @@ int dgemm_set_variant(int variant) {
 }
 
 int dgemm_set_test_flags(int flags) {
-  if (flags < 0 || flags > (DGEMM_TEST_NO_C_PREFETCH | DGEMM_TEST_NO_BLOCKED_B | DGEMM_TEST_TALL_TILES | DGEMM_TEST_SMALL_WARP_TILES | DGEMM_TEST_NO_PACKING | DGEMM_TEST_WS_TWO_CTAS | DGEMM_TEST_FUSED_TAIL_REDUCE | DGEMM_TEST_NO_CLUSTER)) return DGEMM_ERR_VARIANT;
+  if (flags < 0 || flags > (DGEMM_TEST_NO_C_PREFETCH | DGEMM_TEST_NO_BLOCKED_B | DGEMM_TEST_TALL_TILES | DGEMM_TEST_SMALL_WARP_TILES | DGEMM_TEST_NO_PACKING | DGEMM_TEST_WS_TWO_CTAS | DGEMM_TEST_NO_CLUSTER)) return DGEMM_ERR_VARIANT;
   g_test_flags.store(flags);
   return DGEMM_OK;
 }
@@ -1165,17 +1119,8 @@ int dgemm_release_scratch(void) {
     (void)cudaGetLastError();
     return DGEMM_ERR_CUDA;
   }
+  bool ok = scratch::release_all(st->scratch);
   std::lock_guard<std::mutex> lock(g_mutex);
-  bool ok = true;
-  if (st->workspace) {
-    ok = cudaFree(st->workspace) == cudaSuccess && ok;
-    st->workspace = nullptr;
-  }
-  if (st->pack_buf) {
-    ok = cudaFree(st->pack_buf) == cudaSuccess && ok;
-    st->pack_buf = nullptr;
-    st->pack_bytes = 0;
-  }
   if (st->host_pool) ok = cudaMemPoolTrimTo(st->host_pool, 0) == cudaSuccess && ok;
   if (!ok) (void)cudaGetLastError();
   return ok ? DGEMM_OK : DGEMM_ERR_CUDA;

@@ -85,8 +85,6 @@ struct GemmParams {
   const double* B;
   double* C;
   double* partial;        // workspace: slots of BM*BN doubles; phase 1: slot = ks*dp_tiles + tile
-  int* tail_counters;     // phase 2, fused reduction: per tail tile {partial tiles stored, shares reduced}, zero between calls
-  int tail_fused;         // the CTAs that computed a tail tile also reduce it (no second kernel)
   long long lda, ldb, ldc;
   unsigned long long wait_limit_ns;
   int* status;            // device status word
@@ -96,7 +94,6 @@ struct Work {
   int tm, tn;    // tile coordinates
   int kb0, kb1;  // k-block range [kb0, kb1)
   int slot;      // workspace slot for the partial tile, or -1: add straight into C
-  int trel;      // index of the tile among the tail tiles, or -1 for a phase-1 item
 };
 
 // Shared-memory layout of the operand tiles (what the consumer reads and both producers write):
@@ -140,7 +137,6 @@ __device__ __forceinline__ bool get_work(const GemmParams& p, int cta, int nctas
     w.kb0 = ks * p.kblocks_per_split;
     w.kb1 = min(w.kb0 + p.kblocks_per_split, p.kblocks);
     w.slot = p.split_k > 1 ? ks * p.dp_tiles + tile : -1;
-    w.trel = -1;
   } else {
     const int j = idx - n1;
     if (j > 1 || p.tail_tiles == 0) return false;
@@ -162,7 +158,6 @@ __device__ __forceinline__ bool get_work(const GemmParams& p, int cta, int nctas
     w.kb0 = s0 - trel * p.kblocks;
     w.kb1 = s1 - trel * p.kblocks;
     w.slot = (w.kb0 == 0 && w.kb1 == p.kblocks) ? -1 : p.tail_slot_base + 2 * cta + j;
-    w.trel = trel;
   }
   tile_to_mn(p, tile, w.tm, w.tn);
   return true;
@@ -182,7 +177,6 @@ __device__ __forceinline__ void fetch_work_inline(const GemmParams& p, int cta, 
   out[3] = w.kb1;
   out[4] = w.slot;
   out[5] = valid ? 1 : 0;
-  out[6] = w.trel;
 }
 __device__ __noinline__ void fetch_work(const GemmParams& p, int cta, int nctas, int idx, volatile int* out) {
   fetch_work_inline(p, cta, nctas, idx, out);
@@ -616,7 +610,7 @@ __device__ __forceinline__ void reduce_range(const GemmParams& p, int tm, int tn
                                              int e_end, int tid, int nthreads) {
   // U element pairs per thread and pass, all loads of a segment issued before any is used: the
   // reads come from L2 with a latency of hundreds of cycles, so their number in flight is what
-  // counts (U = 1 for the reduction kernels, whose many CTAs provide it; 8 inside the GEMM kernel)
+  // counts (U = 1 for the reduction kernels, whose many CTAs provide it)
   for (int e0 = e_begin + 2 * tid; e0 < e_end; e0 += 2 * nthreads * U) {
     double2 sum[U];
     const double* src = p.partial + (long long)slot_of(0) * (BM * BN);
@@ -653,75 +647,6 @@ __device__ __forceinline__ void reduce_range(const GemmParams& p, int tm, int tn
       }
     }
   }
-}
-
-// ---- stream-K tail, reduced inside the kernel -----------------------------------------------------
-// A tail tile is computed by nseg CTAs (consecutive spans of its k-blocks). Each stores its partial
-// tile, then counts itself in (tail_signal). After a CTA has finished ALL its arithmetic it comes
-// back (tail_reduce_fused): it waits, with a time limit, until the tile's nseg partial tiles are
-// in the workspace, and reduces its share of the rows (bm / nseg of them) over the segments in
-// their fixed order. No CTA waits before its own arithmetic is done and all CTAs of the grid are
-// resident (cooperative launch), so the waits cannot form a cycle. The results are those of
-// dgemm_tail_reduce_kernel, bit for bit, and one launch is saved. Measured, it is nevertheless the
-// slower way in a stream of calls (1024^3: 87.6 us against 78.0 us): a CTA reduces its share with 256
-// threads reading other SMs' partial tiles from L2, where the reduction kernel puts 16 CTAs on
-// each tile and its launch overlaps the GEMM kernel's tail. It is therefore an option
-// (DGEMM_TEST_FUSED_TAIL_REDUCE), not the default.
-__device__ __forceinline__ void tail_signal(const GemmParams& p, int trel, int tid, int barrier_id, int nthreads) {
-  __threadfence();  // this thread's part of the partial tile is visible device-wide before the count
-  ptx::named_barrier_sync(barrier_id, nthreads);
-  if (tid == 0) atomicAdd(p.tail_counters + 2 * trel, 1);
-}
-
-__device__ __forceinline__ bool tail_reduce_fused(const GemmParams& p, int cta, int tid, int barrier_id, int nthreads,
-                                                  volatile int* abort_flag) {
-  const int total = p.tail_tiles * p.kblocks;
-  const int start = cta * p.tail_ipc;
-  const int end = min(start + p.tail_ipc, total);
-  if (start >= end) return true;
-  const int t_first = start / p.kblocks, t_last = (end - 1) / p.kblocks;  // at most two tiles
-  for (int trel = t_first; trel <= t_last; ++trel) {
-    const int lo = trel * p.kblocks, hi = lo + p.kblocks;
-    const int c_first = lo / p.tail_ipc, c_last = (hi - 1) / p.tail_ipc;
-    const int nseg = c_last - c_first + 1;
-    if (nseg == 1) continue;  // one CTA had the whole tile and added it straight to C
-    int* cnt = p.tail_counters + 2 * trel;
-    if (tid == 0) {
-      const unsigned long long t0 = ptx::globaltimer_ns();
-      while (ptx::ld_acquire_gpu(cnt) < nseg) {
-        __nanosleep(64);
-        if (ptx::globaltimer_ns() - t0 > p.wait_limit_ns) {
-          atomicExch(p.status, STATUS_TIMEOUT);
-          *abort_flag = 1;
-          break;
-        }
-      }
-    }
-    ptx::named_barrier_sync(barrier_id, nthreads);
-    if (*abort_flag) return false;
-    __threadfence();
-    int tm, tn;
-    tile_to_mn(p, p.dp_tiles + trel, tm, tn);
-    const int j = cta - c_first;
-    const int r0 = p.bm * j / nseg, r1 = p.bm * (j + 1) / nseg;
-    reduce_range<8>(p, tm, tn, nseg, [&](int s) {
-      const int c = c_first + s;
-      return p.tail_slot_base + 2 * c + ((c * p.tail_ipc >= lo) ? 0 : 1);
-    }, r0 * p.bn, r1 * p.bn, tid, nthreads);
-    // the last CTA to finish its share zeroes the tile's counters for the next call
-    ptx::named_barrier_sync(barrier_id, nthreads);
-    if (tid == 0) {
-      if (atomicAdd(cnt + 1, 1) == nseg - 1) {
-        cnt[0] = 0;
-        cnt[1] = 0;
-      }
-    }
-  }
-  return true;
-}
-__device__ __noinline__ bool tail_reduce_fused_outofline(const GemmParams& p, int cta, int tid, int barrier_id, int nthreads,
-                                                         volatile int* abort_flag) {
-  return tail_reduce_fused(p, cta, tid, barrier_id, nthreads, abort_flag);
 }
 
 // Shape of the inline kernel for a tile height TBM: 128 rows -> 8 warps, 6 stages of 32 KB, one CTA
@@ -936,7 +861,6 @@ dgemm_dmma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     w.kb0 = item_words[2];
     w.kb1 = item_words[3];
     w.slot = item_words[4];
-    w.trel = item_words[6];
     const int valid = item_words[5];
     __syncwarp();
     if (!valid) break;
@@ -960,9 +884,7 @@ dgemm_dmma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
 
     store_tile<(MT >= 4 ? 2 : 1), MT, TileCfg<TBM, WTM, TBN>::EPI_STAGED>(
         p, w, lm, acc, tiles_u32 + TileCfg<TBM, WTM, TBN>::EPI_OFFSET + warp * EPI_WARP_BYTES);
-    if (p.tail_fused && w.slot >= 0) tail_signal(p, w.trel, tid, 0, THREADS);
   }
-  if (ok && p.tail_fused) ok = tail_reduce_fused_outofline(p, cta, tid, 0, THREADS, abort_flag);
 
   // Leaving. After a normal run every copy that was issued has been consumed. After an abort,
   // copies may still be in flight into this CTA's shared memory: let them land first.
@@ -1067,8 +989,7 @@ dgemm_dmma_ws_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
       w.kb0 = item_words[2];
       w.kb1 = item_words[3];
       w.slot = item_words[4];
-      w.trel = item_words[6];
-      const int valid = item_words[5];
+        const int valid = item_words[5];
       __syncwarp();
       if (!valid) break;
       const int kb_pf = (w.slot < 0 && p.c_prefetch) ? max(w.kb0, w.kb1 - C_PREFETCH_KBLOCKS) : -1;
@@ -1181,9 +1102,7 @@ dgemm_dmma_ws_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
       }
       if (!ok) break;
       store_tile<WS_EPI_BATCH, 4, true>(p, w, lm, acc, tiles_u32 + WsCfg<TBM>::EPI_OFFSET + warp * EPI_WARP_BYTES);
-      if (p.tail_fused && w.slot >= 0) tail_signal(p, w.trel, tid, 2, WARPS * 32);
     }
-    if (ok && p.tail_fused) ok = tail_reduce_fused(p, cta, tid, 2, WARPS * 32, abort_flag);
   }
   ptx::named_barrier_sync(1, WS_THREADS);  // all warps leave together
 }

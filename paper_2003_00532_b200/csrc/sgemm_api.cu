@@ -9,6 +9,7 @@
 #include <cuda_runtime.h>
 
 #include "../../include/sgemm.h"
+#include "scratch_pool.h"
 #include "sgemm_ffma.cuh"
 
 namespace {
@@ -24,9 +25,7 @@ struct DeviceState {
   bool ready = false;
   int sm_count = 0;
   int* status = nullptr;
-  float* pack_buf = nullptr;
-  size_t pack_bytes = 0;
-  float* workspace = nullptr;  // partial tiles of the stream-K tail, allocated on first need
+  scratch::Pool scratch;  // stream-K partial tiles and packed operand copies, leased per call (scratch_pool.h)
 };
 
 DeviceState g_dev[kMaxDevices];
@@ -70,25 +69,6 @@ int device_state(DeviceState** out) {
     st.ready = true;
   }
   *out = &st;
-  return DGEMM_OK;
-}
-
-// Growing the scratch frees the old buffer first (cudaFree synchronises the device, so no kernel
-// can still be reading it).
-int ensure_pack_buffer(DeviceState* st, size_t bytes) {
-  std::lock_guard<std::mutex> lock(g_mutex);
-  if (st->pack_bytes >= bytes) return DGEMM_OK;
-  if (st->pack_buf) {
-    cudaFree(st->pack_buf);
-    st->pack_buf = nullptr;
-    st->pack_bytes = 0;
-  }
-  const size_t want = bytes + bytes / 4;
-  if (cudaMalloc(reinterpret_cast<void**>(&st->pack_buf), want) != cudaSuccess) {
-    (void)cudaGetLastError();
-    return DGEMM_ERR_CUDA;
-  }
-  st->pack_bytes = want;
   return DGEMM_OK;
 }
 
@@ -163,16 +143,17 @@ int launch(int64_t M, int64_t N, int64_t K, const float* A, int64_t lda, const f
   int rc = device_state(&st);
   if (rc != DGEMM_OK) return rc;
 
+  // scratch of this call: one lease of the device's pool, held until the last launch below
+  scratch::Hold hold(st->scratch, stream);
   // operands TMA cannot address are repacked (16-byte aligned base, rows of a multiple of 128 bytes)
   const bool pack_a = ((uintptr_t)A & 15) != 0 || (lda % 4 != 0);
   const bool pack_b = ((uintptr_t)B & 15) != 0 || (ldb % 4 != 0);
   if (pack_a || pack_b) {
     const int64_t plda = (K + 31) & ~(int64_t)31, pldb = (N + 31) & ~(int64_t)31;
     const size_t a_bytes = pack_a ? (size_t)M * plda * 4 : 0, b_bytes = pack_b ? (size_t)K * pldb * 4 : 0;
-    rc = ensure_pack_buffer(st, a_bytes + b_bytes + 256);
-    if (rc != DGEMM_OK) return rc;
-    float* pa = st->pack_buf;
-    float* pb = reinterpret_cast<float*>(reinterpret_cast<char*>(st->pack_buf) + ((a_bytes + 255) & ~(size_t)255));
+    float* pa = static_cast<float*>(hold.pack_buffer(a_bytes + b_bytes + 256));
+    if (!pa) return DGEMM_ERR_CUDA;
+    float* pb = reinterpret_cast<float*>(reinterpret_cast<char*>(pa) + ((a_bytes + 255) & ~(size_t)255));
     PackOpF ops[2];
     int nops = 0;
     int64_t gx = 0, gy = 0;
@@ -237,15 +218,8 @@ int launch(int64_t M, int64_t N, int64_t K, const float* A, int64_t lda, const f
     p.tail_ipc = (int)ipc;
     const int span_ctas = (int)((total + ipc - 1) / ipc);
     if (p.dp_tiles == 0) grid = span_ctas < resident ? span_ctas : resident;
-    {
-      std::lock_guard<std::mutex> lock(g_mutex);
-      if (!st->workspace && cudaMalloc(reinterpret_cast<void**>(&st->workspace), (size_t)2 * resident * MAX_TM * TN * sizeof(float)) !=
-                                cudaSuccess) {
-        (void)cudaGetLastError();
-        return DGEMM_ERR_CUDA;
-      }
-    }
-    p.partial = st->workspace;
+    p.partial = static_cast<float*>(hold.workspace((size_t)2 * resident * MAX_TM * TN * sizeof(float)));
+    if (!p.partial) return DGEMM_ERR_CUDA;
   }
   if (TM == 256) launch_pdl(sgemm_ffma_kernel<16>, dim3(grid), dim3(THREADS), (size_t)Cfg<16>::SMEM_BYTES, stream, map_a, map_b, p);
   else launch_pdl(sgemm_ffma_kernel<8>, dim3(grid), dim3(THREADS), (size_t)Cfg<8>::SMEM_BYTES, stream, map_a, map_b, p);

@@ -52,7 +52,7 @@ def test_random_cases(oracle, seed):
         variant, flags, split = dg.DGEMM_VARIANT_AUTO, 0, 0
         if kind != "s" and rnd.random() < 0.3:
             variant = rnd.choice([1, 2, 3, 4])
-            flags = rnd.choice([0, 0, 1, 2, 4, 8, 12, 32, 64])
+            flags = rnd.choice([0, 0, 1, 2, 4, 8, 12, 32, 128])
             if rnd.random() < 0.2:
                 split = rnd.choice([2, 3, 5])
         what = f"seed {seed} case {case}: {kind} {(M, N, K)} ta={ta} tb={tb} alpha={alpha} beta={beta} pads={pads} " \

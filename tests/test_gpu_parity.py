@@ -384,38 +384,6 @@ def test_bounded_wait_gives_up_and_reports(oracle):
     _check_full(oracle, prob, run_gpu(prob))
 
 
-@pytest.mark.parametrize("shape", [(512, 512, 512), (1024, 1024, 1024), (640, 384, 2048), (2304, 2304, 2304),
-                                   (2088, 2048, 2048), (129, 257, 4099), (1000, 1537, 777)])
-def test_fused_tail_reduction_is_bit_identical(shape):
-    """The optional in-kernel reduction of the last wave's partial tiles (cooperative launch, CTAs of
-    a tile wait for one another with a time limit) gives the same bits as the reduction kernel, in
-    one launch fewer, run after run."""
-    M, N, K = shape
-    g = torch.Generator(device="cuda").manual_seed(1)
-    A = torch.rand(M, K, dtype=torch.float64, device="cuda", generator=g) * 2 - 1
-    B = torch.rand(K, N, dtype=torch.float64, device="cuda", generator=g) * 2 - 1
-    C0 = torch.rand(M, N, dtype=torch.float64, device="cuda", generator=g) * 2 - 1
-    ref = C0.clone()
-    dg.dgemm_set_test_flags(dg.DGEMM_TEST_NO_CLUSTER)  # the workspace split also where the cluster kernel would run
-    try:
-        n0 = dg.dgemm_launch_count()
-        dg.dgemm_f64(A, B, ref)
-        separate = dg.dgemm_launch_count() - n0
-    finally:
-        dg.dgemm_set_test_flags(0)
-    dg.dgemm_set_test_flags(64)
-    try:
-        for rep in range(3):
-            C = C0.clone()
-            n0 = dg.dgemm_launch_count()
-            dg.dgemm_f64(A, B, C)
-            assert dg.dgemm_launch_count() - n0 == separate - 1
-            assert dg.dgemm_last_device_status() == dg.DGEMM_OK
-            assert torch.equal(ref.view(torch.int64), C.view(torch.int64)), f"run {rep}"
-    finally:
-        dg.dgemm_set_test_flags(0)
-
-
 SKINNY_SHAPES = [(32, 1000, 600), (16, 513, 129), (96, 500, 300), (160, 384, 512), (20, 129, 77), (417, 260, 200),
                  (1000, 48, 600), (1000, 96, 333), (513, 80, 64), (2000, 64, 2048), (300, 97, 128),
                  (1000, 146, 300), (700, 130, 520), (257, 416, 100), (129, 190, 64)]

@@ -195,3 +195,16 @@ def test_replicas_without_process_group():
     assert aggregate_rate(10.0, 2.0, 1) == 5.0
     assert rank_info({"RANK": "3", "LOCAL_RANK": "1", "WORLD_SIZE": "8"}) == (3, 1, 8)
     assert rank_info({}) == (0, 0, 1)
+
+
+def test_every_included_file_is_a_build_dependency():
+    """An edit to any file the library is compiled from must make the built library stale."""
+    import re
+    from paper_2003_00532_b200 import build as b
+    deps = {os.path.basename(d) for d in b.DEPS}
+    for src in os.listdir(b.CSRC):
+        if not src.endswith((".cu", ".cuh", ".h")):
+            continue
+        assert src in deps
+        for inc in re.findall(r'#include\s+"([^"]+)"', open(os.path.join(b.CSRC, src)).read()):
+            assert os.path.basename(inc) in deps, f"{src} includes {inc}, which build.DEPS does not list"

@@ -52,8 +52,10 @@ class ClockSampler:
              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
              "clocks_event_reasons.sw_power_cap")
 
-    def __init__(self, gpu_index: int):
-        self.gpu_index = gpu_index
+    def __init__(self, gpu_id: str):
+        # `gpu_id` is what nvidia-smi's --id takes. nvidia-smi does not honour CUDA_VISIBLE_DEVICES, so
+        # a CUDA ordinal may name another GPU of a shared box: pass the device's UUID ("GPU-...").
+        self.gpu_index = gpu_id
         self.proc = None
         self.lines = []
 
@@ -99,7 +101,7 @@ class ClockSampler:
         return {"sm_mhz": statistics.median(sm) if sm else None,
                 "sm_max_mhz": max(smax) if smax else None,
                 "power_w_max": max(power) if power else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+                "samples": len(sm), "reasons": sorted(reasons), "gpu": self.gpu_index}
 
 
 def host_cores() -> int:
@@ -155,6 +157,27 @@ def time_shape(dg, torch, M, N, K, lda=None, ldb=None, ldc=None, min_ms=40.0):
     return best
 
 
+def single_call_latency_us(dg, torch, n, reps=30):
+    """Median device time of ONE dgemm_f64 call on an idle GPU (synchronise, event, call, event), next
+    to which the back-to-back figure of time_shape() is the throughput of a stream of calls."""
+    A = torch.rand(n, n, dtype=torch.float64, device="cuda") * 2 - 1
+    B = torch.rand(n, n, dtype=torch.float64, device="cuda") * 2 - 1
+    C = torch.zeros(n, n, dtype=torch.float64, device="cuda")
+    pa, pb, pc = A.data_ptr(), B.data_ptr(), C.data_ptr()
+    call = dg.load_library().dgemm_f64
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    lat = []
+    for i in range(reps + 3):
+        torch.cuda.synchronize()
+        e0.record()
+        call(n, n, n, pa, n, pb, n, pc, n, None)
+        e1.record()
+        torch.cuda.synchronize()
+        if i >= 3:
+            lat.append(e0.elapsed_time(e1) * 1e3)
+    return statistics.median(lat)
+
+
 def other_shapes(dg, torch, peak_tflops, hbm_gbs):
     """The square-size sweep (the metric's 'TFLOPS vs M=N=K' curve) and the ragged / rank-k shapes,
     each with its fraction of the FP64 peak and, for the low-intensity shapes, of the HBM roof."""
@@ -162,11 +185,14 @@ def other_shapes(dg, torch, peak_tflops, hbm_gbs):
     for n in range(128, 4096 + 1, 128):
         ms = time_shape(dg, torch, n, n, n)
         tf = 2.0 * n ** 3 / ms / 1e9
-        sweep.append({"n": n, "us": round(ms * 1e3, 1), "tflops": round(tf, 2), "frac_peak": round(tf / peak_tflops, 3)})
+        row = {"n": n, "us": round(ms * 1e3, 1), "tflops": round(tf, 2), "frac_peak": round(tf / peak_tflops, 3)}
+        if n <= 1024:  # latency-bound sizes: one isolated call beside the stream of calls
+            row["single_call_us"] = round(single_call_latency_us(dg, torch, n), 1)
+        sweep.append(row)
     shapes = []
     for (M, N, K, pad) in [(1000, 1537, 777, True), (2088, 2088, 2088, True), (4097, 31, 4099, True),
                            (2088, 2048, 2048, False), (16384, 16384, 64, False), (16384, 16384, 256, False),
-                           # skinny shapes (narrow, short and half-width tiles); not BASELINE configs
+                           # skinny shapes (narrow, short and half-width tiles), beyond the five configurations
                            (8192, 64, 8192, False), (32, 8192, 8192, False), (6514, 146, 4096, False)]:
         ld = (K + 3, N + 5, N + 7) if pad else (K, N, N)
         ms = time_shape(dg, torch, M, N, K, *ld)
@@ -217,7 +243,11 @@ def ablation_ladder(dg, torch, peak_tflops, n=4096):
     the library. Returns a list of {rung, tflops, frac_peak}."""
     rungs = [
         ("naive nest, one thread per C element", dict(variant=dg.DGEMM_VARIANT_NAIVE, n=min(n, 2048))),
-        ("+ smem tiles, register tiles, DMMA; 8-byte cp.async staging, 128x128 tile, 1 CTA/SM",
+        ("+ tiles of A and B in shared memory, still one C element per thread (no register tile)",
+         dict(variant=dg.DGEMM_VARIANT_SMEM, n=min(n, 2048))),
+        ("+ 8x8 register tile per thread on plain FMAs (DFMA), 8-byte cp.async staging, mbarrier pipeline, 64x128 tile, 2 CTAs/SM",
+         dict(variant=dg.DGEMM_VARIANT_GENERIC_DFMA, flags=16)),
+        ("+ tensor-core micro-kernel (DMMA) in place of DFMA; same staging, 128x128 tile, 1 CTA/SM",
          dict(variant=dg.DGEMM_VARIANT_GENERIC, flags=4 | 16)),
         ("+ TMA staging (2-D copies, 9 per stage), no C prefetch", dict(variant=dg.DGEMM_VARIANT_TMA, flags=4 | 2 | 1)),
         ("+ one 3-D copy for B, C prefetch into L2", dict(variant=dg.DGEMM_VARIANT_TMA, flags=4)),
@@ -238,6 +268,26 @@ def ablation_ladder(dg, torch, peak_tflops, n=4096):
             dg.dgemm_set_test_flags(0)
         tf = 2.0 * m ** 3 / ms / 1e9
         out.append({"rung": name, "n": m, "tflops": round(tf, 2), "frac_peak": round(tf / peak_tflops, 3)})
+    return out
+
+
+def micro_kernel_swap(dg, torch, peak_tflops, n=4096):
+    """The paper's 'outer MLIR, inner BLIS' experiment (Section 2.12) on the GPU: one macro-kernel (TMA
+    staging, mbarrier pipeline, grouped raster, stream-K tail, epilogue; 64 x 128 tiles, two CTAs per
+    SM) with two inner kernels, tensor-core MMAs and plain FMAs on the same 8 x 8 register tile per
+    thread. Each is set against the ceiling of its own instruction, measured by a register-only loop."""
+    _, fma_ceiling = dg.dgemm_fp64_fma_probe(300)
+    fma_per_clk, _ = dg.dgemm_fp64_fma_probe(100)
+    out = {"n": n, "macro_kernel": "dgemm_dmma_kernel<TMA, 64 x 128 x 16, 4 stages, 2 CTAs/SM>",
+           "dfma_ceiling_tflops": round(fma_ceiling, 2), "dfma_fma_per_clk_sm": round(fma_per_clk, 1)}
+    for key, variant, ceiling in (("dmma", dg.DGEMM_VARIANT_TMA, peak_tflops), ("dfma", dg.DGEMM_VARIANT_TMA_DFMA, fma_ceiling)):
+        dg.dgemm_set_variant(variant)
+        try:
+            ms = time_shape(dg, torch, n, n, n)
+        finally:
+            dg.dgemm_set_variant(dg.DGEMM_VARIANT_AUTO)
+        tf = 2.0 * n ** 3 / ms / 1e9
+        out[key] = {"tflops": round(tf, 2), "frac_of_own_ceiling": round(tf / ceiling, 3), "frac_peak": round(tf / peak_tflops, 3)}
     return out
 
 
@@ -299,6 +349,9 @@ def run_ours(args):
         return replicas.max_over_ranks(x, device="cuda")
 
     dg.load_library()
+    if args.variant != dg.DGEMM_VARIANT_AUTO or args.flags:
+        dg.dgemm_set_variant(args.variant)   # profiling aid: one rung of the ladder as the timed kernel
+        dg.dgemm_set_test_flags(args.flags)
     n = args.size
     if args.shape:
         sm, sn, sk = (int(x) for x in args.shape.split(","))
@@ -314,7 +367,11 @@ def run_ours(args):
     for _ in range(max(args.warmup, 3)):
         dg.dgemm_f64(A, B, C, stream=stream)
     barrier()
-    sampler = ClockSampler(local_rank)
+    try:
+        gpu_id = "GPU-" + str(torch.cuda.get_device_properties(local_rank).uuid)
+    except Exception:  # noqa: BLE001 - an older torch without the uuid property
+        gpu_id = str(local_rank)
+    sampler = ClockSampler(gpu_id)
     if rank == 0:
         sampler.start()
         time.sleep(0.25)
@@ -368,6 +425,14 @@ def run_ours(args):
                 "d2h_gbs": nbytes / (ev[1].elapsed_time(ev[2]) * 1e-3) / 1e9}
         link["floor_ms_per_step"] = max(h2d / (link["h2d_gbs"] * 1e9), d2h / (link["d2h_gbs"] * 1e9)) * 1e3
 
+    # the host entry point ran on streams of its own, which switched the library's scratch pool to its
+    # multi-stream mode (an event per call); give the scratch back so that the single-stream timings
+    # below run as a single-stream program does
+    dg.dgemm_release_scratch()
+    if args.variant != dg.DGEMM_VARIANT_AUTO or args.flags:
+        dg.dgemm_set_variant(dg.DGEMM_VARIANT_AUTO)
+        dg.dgemm_set_test_flags(0)
+
     if rank != 0:
         if distributed:
             dist.destroy_process_group()
@@ -377,7 +442,11 @@ def run_ours(args):
     peaks = _load_measured_peaks()
     sm_max_mhz = float(peaks["sm_max_mhz"]) if peaks and "sm_max_mhz" in peaks else 1965.0
     peak_tflops = SM_COUNT_B200 * FMA_PER_CLK_SM * 2 * sm_max_mhz * 1e6 / 1e12
-    probe_fma, probe_tflops = dg.dgemm_fp64_peak_probe(300)
+    # sustained issue rate: back-to-back register-only launches of 500 ms for --probe-ms in all (no
+    # single multi-second kernel); the mean is the sustained figure, the first launch the burst one
+    probe_runs = [dg.dgemm_fp64_peak_probe(500) for _ in range(max(1, args.probe_ms // 500))]
+    probe_fma = statistics.mean(r[0] for r in probe_runs)
+    probe_tflops = statistics.mean(r[1] for r in probe_runs)
     achieved = flop / (kernel_ms * 1e-3) / 1e12
     hbm_gbs = float(peaks["hbm_gbs"]) if peaks and "hbm_gbs" in peaks else 6650.0
     roofline = {
@@ -388,6 +457,8 @@ def run_ours(args):
                         f"{SM_COUNT_B200} SMs x 2 x sm_max_mhz {sm_max_mhz:.0f} "
                         f"({'MEASURED_PEAKS.json' if peaks else 'fallback 1965'}); MEASURED_PEAKS has no FP64 entry"),
         "probe_fma_per_clk_sm": probe_fma, "probe_sustained_tflops": probe_tflops,
+        "probe_seconds": 0.5 * len(probe_runs), "probe_burst_tflops": probe_runs[0][1],
+        "probe_min_tflops": min(r[1] for r in probe_runs),
         "frac_of_probe_sustained": achieved / probe_tflops if probe_tflops > 0 else None,
         "algorithmic_flop_per_launch": flop,
         "algorithmic_bytes_per_launch": prob.min_bytes,
@@ -422,6 +493,7 @@ def run_ours(args):
     if not args.no_sweep:
         line["sweep"], line["other_shapes"] = other_shapes(dg, torch, peak_tflops, hbm_gbs)
         line["ablation"] = ablation_ladder(dg, torch, peak_tflops)
+        line["micro_kernel_swap"] = micro_kernel_swap(dg, torch, peak_tflops)
         line["sgemm"] = sgemm_section(dg, torch, sm_max_mhz)
     print(json.dumps(line), flush=True)
     if distributed:
@@ -441,6 +513,10 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--shape", type=str, default="", help="M,N,K of another (non-square) workload; profiling aid")
     ap.add_argument("--no-sweep", action="store_true", help="skip the size sweep and the ragged / rank-k shapes")
+    ap.add_argument("--variant", type=int, default=-1, help="profiling aid: force a DGEMM_VARIANT_* for the timed calls")
+    ap.add_argument("--flags", type=int, default=0, help="profiling aid: DGEMM_TEST_* flags for the timed calls")
+    ap.add_argument("--probe-ms", type=int, default=4000,
+                    help="total length of the sustained FP64 issue-rate probe (run as launches of 500 ms)")
     ap.add_argument("--sgemm-size", type=int, default=0,
                     help="profiling aid: time only sgemm_f32 at M=N=K of this size, print its section and exit")
     args = ap.parse_args()

@@ -56,7 +56,13 @@ enum {
                                     thread-block cluster, partial tiles added through distributed shared
                                     memory: one launch, no workspace; what AUTO uses below one wave of tiles */
   DGEMM_VARIANT_GENERIC_CLUSTER = 6, /* as TMA_CLUSTER with the GENERIC staging: any alignment          */
-  DGEMM_VARIANT_COUNT = 7
+  DGEMM_VARIANT_SMEM = 7,        /* ladder rung: tiles of A and B in shared memory, one C element per thread,
+                                    no register tile (tiling + packing before unroll-and-jam, Sections 2.4-2.6) */
+  DGEMM_VARIANT_TMA_DFMA = 8,    /* micro-kernel swap (Section 2.12): the TMA variant's staging, pipeline, raster
+                                    and epilogue on 64 x 128 tiles, with plain FP64 fused multiply-adds on an
+                                    8 x 8 register tile per thread in place of the tensor-core MMAs */
+  DGEMM_VARIANT_GENERIC_DFMA = 9, /* the same inner kernel under the GENERIC staging: any alignment          */
+  DGEMM_VARIANT_COUNT = 10
 };
 
 /*
@@ -201,10 +207,10 @@ DGEMM_API int dgemm_f64_static_ws(int64_t M, int64_t N, int64_t K,
                                   double *C, int64_t ldc,
                                   int split_k, void *stream);
 
-/* Human-readable text for a status code; never NULL; static storage. */
+/* Human-readable text for a status code; never NULL; static storage. No counterpart in the paper. */
 DGEMM_API const char *dgemm_strerror(int status);
 
-/* Library version as major*10000 + minor*100 + patch. */
+/* Library version as major*10000 + minor*100 + patch. No counterpart in the paper. */
 DGEMM_API int dgemm_version(void);
 
 /*
@@ -215,7 +221,8 @@ DGEMM_API int dgemm_version(void);
  */
 DGEMM_API int dgemm_set_variant(int variant);
 
-/* Force a split-K factor (>= 1) for the pipelined variants, or 0 for the built-in heuristic. */
+/* Force a split-K factor (>= 1) for the pipelined variants, or 0 for the built-in heuristic (tests and
+ * ablation). No counterpart in the paper: its single core has no use for a K split. */
 DGEMM_API int dgemm_set_split_k(int split_k);
 
 /*
@@ -255,7 +262,7 @@ DGEMM_API int dgemm_plan(int64_t M, int64_t N, int64_t K, int tma_addressable, i
  * Synchronises `stream`, then reads and clears the current device's status word. Returns
  * DGEMM_OK if no kernel reported a problem since the last call, DGEMM_ERR_TIMEOUT if a bounded
  * wait inside a kernel ran out (the kernel then stopped early and C is unspecified), or
- * DGEMM_ERR_CUDA if the synchronisation itself failed.
+ * DGEMM_ERR_CUDA if the synchronisation itself failed. No counterpart in the paper.
  */
 DGEMM_API int dgemm_last_device_status(void *stream);
 
@@ -272,7 +279,7 @@ DGEMM_API int dgemm_release_scratch(void);
 
 /*
  * Number of kernels this library has launched so far in this process (all entry points).
- * Monotonic; used by the benchmark to report launches per step.
+ * Monotonic; used by the benchmark to report launches per step. No counterpart in the paper.
  */
 DGEMM_API int64_t dgemm_launch_count(void);
 
@@ -293,6 +300,14 @@ DGEMM_API int dgemm_selftest_wait_timeout(int limit_us);
  * and the sustained rate in TFLOP/s to *tflops (either may be NULL). Synchronous.
  */
 DGEMM_API int dgemm_fp64_peak_probe(int millis, double *fma_per_clk_sm, double *tflops);
+
+/*
+ * The same measurement for plain FP64 fused multiply-add instructions (16 independent chains per
+ * thread, 512 threads per SM): the ceiling of the DGEMM_VARIANT_*_DFMA micro-kernel, next to the
+ * tensor-core figure above (the two machine peaks one would compute from unit counts as in
+ * Section 1.2; on B200 they differ). Same arguments and return codes.
+ */
+DGEMM_API int dgemm_fp64_fma_probe(int millis, double *fma_per_clk_sm, double *tflops);
 
 #ifdef __cplusplus
 }

@@ -40,6 +40,9 @@ DGEMM_VARIANT_TMA_WS = 3
 DGEMM_VARIANT_GENERIC_WS = 4
 DGEMM_VARIANT_TMA_CLUSTER = 5
 DGEMM_VARIANT_GENERIC_CLUSTER = 6
+DGEMM_VARIANT_SMEM = 7
+DGEMM_VARIANT_TMA_DFMA = 8
+DGEMM_VARIANT_GENERIC_DFMA = 9
 
 # dgemm_set_test_flags bits
 DGEMM_TEST_NO_C_PREFETCH = 1
@@ -110,6 +113,9 @@ def load_library() -> ctypes.CDLL:
             lib.dgemm_fp64_peak_probe.argtypes = [ctypes.c_int, ctypes.POINTER(ctypes.c_double),
                                                   ctypes.POINTER(ctypes.c_double)]
             lib.dgemm_fp64_peak_probe.restype = ctypes.c_int
+            lib.dgemm_fp64_fma_probe.argtypes = [ctypes.c_int, ctypes.POINTER(ctypes.c_double),
+                                                 ctypes.POINTER(ctypes.c_double)]
+            lib.dgemm_fp64_fma_probe.restype = ctypes.c_int
             _lib = lib
     return _lib
 
@@ -317,4 +323,13 @@ def dgemm_fp64_peak_probe(millis: int = 200):
     rc = load_library().dgemm_fp64_peak_probe(int(millis), ctypes.byref(a), ctypes.byref(b))
     if rc < 0:
         raise DgemmError(rc, "dgemm_fp64_peak_probe")
+    return a.value, b.value
+
+
+def dgemm_fp64_fma_probe(millis: int = 200):
+    """Returns ``(fma_per_clk_sm, tflops)`` measured by the register-only loop of plain FP64 FMAs."""
+    a, b = ctypes.c_double(0.0), ctypes.c_double(0.0)
+    rc = load_library().dgemm_fp64_fma_probe(int(millis), ctypes.byref(a), ctypes.byref(b))
+    if rc < 0:
+        raise DgemmError(rc, "dgemm_fp64_fma_probe")
     return a.value, b.value

@@ -141,6 +141,12 @@ void launch_tile_kernel(int grid, cudaStream_t stream, const CUtensorMap& map_a,
 }
 
 template <bool USE_TMA>
+void launch_dfma_kernel(int grid, cudaStream_t stream, const CUtensorMap& map_a, const CUtensorMap& map_b, const GemmParams& p) {
+  launch_gemm_kernel(dgemm_dmma_kernel<USE_TMA, 64, 64, BN, MICRO_DFMA>, grid, TileCfg<64, 64, BN>::THREADS_,
+                     TileCfg<64, 64, BN>::SMEM_BYTES_, stream, map_a, map_b, p);
+}
+
+template <bool USE_TMA>
 void launch_default_kernel(int bm, int wtm, int grid, cudaStream_t stream, const CUtensorMap& map_a,
                            const CUtensorMap& map_b, const GemmParams& p) {
   if (p.bn == 64) launch_tile_kernel<USE_TMA, 128, 64, 64>(grid, stream, map_a, map_b, p);
@@ -152,9 +158,9 @@ void launch_default_kernel(int bm, int wtm, int grid, cudaStream_t stream, const
   else launch_tile_kernel<USE_TMA, 64, 32>(grid, stream, map_a, map_b, p);
 }
 
-template <bool USE_TMA, int TBM, int WTM, int TBN = BN>
+template <bool USE_TMA, int TBM, int WTM, int TBN = BN, int MICRO = MICRO_DMMA>
 bool configure_tile_kernel(int* occupancy) {
-  auto* k = dgemm_dmma_kernel<USE_TMA, TBM, WTM, TBN>;
+  auto* k = dgemm_dmma_kernel<USE_TMA, TBM, WTM, TBN, MICRO>;
   if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, TileCfg<TBM, WTM, TBN>::SMEM_BYTES_) != cudaSuccess) return false;
   if (cudaFuncSetAttribute(k, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared) != cudaSuccess) return false;
   return cudaOccupancyMaxActiveBlocksPerMultiprocessor(occupancy, k, TileCfg<TBM, WTM, TBN>::THREADS_,
@@ -180,7 +186,7 @@ int device_state(DeviceState** out) {
     if (major != 10) return DGEMM_ERR_DEVICE;
     if (cudaGetSymbolAddress(reinterpret_cast<void**>(&st.status), g_status_word) != cudaSuccess) return DGEMM_ERR_CUDA;
     if (cudaMemset(st.status, 0, sizeof(int)) != cudaSuccess) return DGEMM_ERR_CUDA;
-    int occ[14] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
+    int occ[16] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
     const bool attr_ok =
         configure_tile_kernel<true, 128, 64, 64>(&occ[12]) && configure_tile_kernel<false, 128, 64, 64>(&occ[13]) &&
         configure_tile_kernel<true, 32, 32>(&occ[10]) && configure_tile_kernel<false, 32, 32>(&occ[11]) &&
@@ -189,13 +195,14 @@ int device_state(DeviceState** out) {
         configure_tile_kernel<true, 64, 64>(&occ[4]) && configure_tile_kernel<false, 64, 64>(&occ[5]) &&
         configure_tile_kernel<true, 64, 32>(&occ[6]) && configure_tile_kernel<false, 64, 32>(&occ[7]) &&
         configure_tile_kernel<true, 256, 64, 32>(&occ[8]) && configure_tile_kernel<false, 256, 64, 32>(&occ[9]) &&
+        configure_tile_kernel<true, 64, 64, BN, MICRO_DFMA>(&occ[14]) && configure_tile_kernel<false, 64, 64, BN, MICRO_DFMA>(&occ[15]) &&
         cudaFuncSetAttribute(dgemm_dmma_ws_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) == cudaSuccess &&
         cudaFuncSetAttribute(dgemm_dmma_ws_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) == cudaSuccess &&
         cudaFuncSetAttribute(dgemm_dmma_ws_kernel<true, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, WsCfg<64>::SMEM_BYTES_) == cudaSuccess &&
         cudaFuncSetAttribute(dgemm_dmma_ws_kernel<true, 64>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared) == cudaSuccess;
     if (!attr_ok) return DGEMM_ERR_CUDA;
     // the 64-row kernels are meant to run two CTAs per SM; use them only where the device really fits two
-    st.two_ctas_ok = occ[4] >= 2 && occ[5] >= 2 && occ[6] >= 2 && occ[7] >= 2 && occ[8] >= 2 && occ[9] >= 2 && occ[10] >= 2 && occ[11] >= 2 && occ[12] >= 2 && occ[13] >= 2;
+    st.two_ctas_ok = occ[4] >= 2 && occ[5] >= 2 && occ[6] >= 2 && occ[7] >= 2 && occ[8] >= 2 && occ[9] >= 2 && occ[10] >= 2 && occ[11] >= 2 && occ[12] >= 2 && occ[13] >= 2 && occ[14] >= 2 && occ[15] >= 2;
     if (!g_encode) {
       void* fn = nullptr;
       cudaDriverEntryPointQueryResult qres;
@@ -424,8 +431,11 @@ Plan plan_gemm(int64_t M, int64_t N, int64_t K, bool tma_ok, int requested_varia
     }
   }
   pl.variant = variant;
-  const bool wants_tma = variant == DGEMM_VARIANT_TMA || variant == DGEMM_VARIANT_TMA_WS || variant == DGEMM_VARIANT_TMA_CLUSTER;
+  const bool dfma = variant == DGEMM_VARIANT_TMA_DFMA || variant == DGEMM_VARIANT_GENERIC_DFMA;
+  const bool wants_tma = variant == DGEMM_VARIANT_TMA || variant == DGEMM_VARIANT_TMA_WS || variant == DGEMM_VARIANT_TMA_CLUSTER ||
+                         variant == DGEMM_VARIANT_TMA_DFMA;
   if (wants_tma && !tma_ok) { pl.status = DGEMM_ERR_VARIANT; return pl; }
+  if (dfma && !two_ctas_ok) { pl.status = DGEMM_ERR_VARIANT; return pl; }
   if (variant == DGEMM_VARIANT_TMA_CLUSTER || variant == DGEMM_VARIANT_GENERIC_CLUSTER) {
     // forced: clusters of dgemm_set_split_k() CTAs if that is 1, 2, 4 or 8 (ranks beyond the last
     // k-block then idle), else the largest size that keeps all CTAs resident at once
@@ -445,8 +455,9 @@ Plan plan_gemm(int64_t M, int64_t N, int64_t K, bool tma_ok, int requested_varia
     pl.status = DGEMM_ERR_VARIANT;
     return pl;
   }
-  if (variant == DGEMM_VARIANT_NAIVE) {
-    pl.bm = 8; pl.bn = 32; pl.wtm = 0; pl.ctas_per_sm = 0;
+  if (variant == DGEMM_VARIANT_NAIVE || variant == DGEMM_VARIANT_SMEM) {
+    pl.bm = variant == DGEMM_VARIANT_NAIVE ? 8 : SMEM_RUNG_TILE;
+    pl.bn = 32; pl.wtm = 0; pl.ctas_per_sm = 0;
     pl.grid = 0; pl.split_k = 1; pl.kblocks_per_split = kblocks;
     return pl;
   }
@@ -457,7 +468,8 @@ Plan plan_gemm(int64_t M, int64_t N, int64_t K, bool tma_ok, int requested_varia
   // (generic staging on a problem of many waves is a little faster with the tall tile: half the B copies per thread)
   const int64_t tiles128 = ((M + 127) / 128) * ((N + BN - 1) / BN);
   const bool generic_large = !wants_tma && tiles128 >= 4 * (int64_t)sm_count;
-  const bool plain_tiles = (dbg_flags & (DGEMM_TEST_TALL_TILES | DGEMM_TEST_SMALL_WARP_TILES)) != 0;
+  // (the micro-kernel swap exists for the 64 x 128 tile only and ignores the tile-shape flags)
+  const bool plain_tiles = dfma || (dbg_flags & (DGEMM_TEST_TALL_TILES | DGEMM_TEST_SMALL_WARP_TILES)) != 0;
   // narrow problems (see narrow_tiles_pay) use 256 x 32 tiles: four warps stacked in M, little arithmetic on unused columns
   const bool narrow = narrow_tiles_pay(N) && !ws_variant && !plain_tiles && two_ctas_ok;
   // N just above a multiple of 128: 128 x 64 tiles
@@ -470,12 +482,12 @@ Plan plan_gemm(int64_t M, int64_t N, int64_t K, bool tma_ok, int requested_varia
   // warp-specialised with 64-row tiles, two CTAs per SM: the second CTA hides the C round trip of short-K problems
   const bool ws64 = variant == DGEMM_VARIANT_TMA_WS && two_ctas_ok &&
                     (kblocks < kAutoWsMinKblocks || auto_ws64 || (dbg_flags & DGEMM_TEST_WS_TWO_CTAS));
-  const int bm = narrow ? 256 : half_width ? 128 : short_m ? 32 : ws64 ? 64
+  const int bm = narrow ? 256 : half_width ? 128 : short_m ? 32 : (ws64 || dfma) ? 64
                  : (ws_variant || generic_large || (dbg_flags & DGEMM_TEST_TALL_TILES) || !two_ctas_ok) ? 128 : 64;
   const int bn = narrow ? 32 : half_width ? 64 : BN;
   pl.bm = bm;
   pl.bn = bn;
-  pl.wtm = (short_m || (dbg_flags & DGEMM_TEST_SMALL_WARP_TILES)) ? 32 : 64;
+  pl.wtm = (short_m || (!dfma && (dbg_flags & DGEMM_TEST_SMALL_WARP_TILES))) ? 32 : 64;
   pl.ctas_per_sm = (bm == 128 && bn == 128) ? 1 : 2;
 
   const int64_t tiles64 = ((M + bm - 1) / bm) * ((N + bn - 1) / bn);
@@ -572,13 +584,23 @@ int launch_gemm_packed(DeviceState* st, scratch::Hold& hold, int variant, int64_
                               st->cluster_ok);
   if (plan.status != DGEMM_OK) return plan.status;
   variant = plan.variant;
-  const bool wants_tma = variant == DGEMM_VARIANT_TMA || variant == DGEMM_VARIANT_TMA_WS || variant == DGEMM_VARIANT_TMA_CLUSTER;
+  const bool dfma = variant == DGEMM_VARIANT_TMA_DFMA || variant == DGEMM_VARIANT_GENERIC_DFMA;
+  const bool wants_tma = variant == DGEMM_VARIANT_TMA || variant == DGEMM_VARIANT_TMA_WS || variant == DGEMM_VARIANT_TMA_CLUSTER ||
+                         variant == DGEMM_VARIANT_TMA_DFMA;
   const bool cluster = variant == DGEMM_VARIANT_TMA_CLUSTER || variant == DGEMM_VARIANT_GENERIC_CLUSTER;
 
   if (variant == DGEMM_VARIANT_NAIVE) {
     if (form.alpha != 1.0 || form.beta != 1.0) return DGEMM_ERR_VARIANT;  // the naive nest is C += A B only
     dim3 block(32, 8), grid((unsigned)((N + 31) / 32), (unsigned)((M + 7) / 8));
     dgemm_naive_kernel<<<grid, block, 0, stream>>>((int)M, (int)N, (int)K, A, lda, B, ldb, C, ldc);
+    g_launches.fetch_add(1);
+    return cudaGetLastError() == cudaSuccess ? DGEMM_OK : DGEMM_ERR_CUDA;
+  }
+  if (variant == DGEMM_VARIANT_SMEM) {
+    if (form.alpha != 1.0 || form.beta != 1.0) return DGEMM_ERR_VARIANT;  // a rung of the ladder: C += A B only
+    dim3 block(SMEM_RUNG_TILE, SMEM_RUNG_TILE), grid((unsigned)((N + SMEM_RUNG_TILE - 1) / SMEM_RUNG_TILE),
+                                                     grid_y((M + SMEM_RUNG_TILE - 1) / SMEM_RUNG_TILE));
+    dgemm_smem_kernel<<<grid, block, 0, stream>>>((int)M, (int)N, (int)K, A, lda, B, ldb, C, ldc);
     g_launches.fetch_add(1);
     return cudaGetLastError() == cudaSuccess ? DGEMM_OK : DGEMM_ERR_CUDA;
   }
@@ -631,6 +653,8 @@ int launch_gemm_packed(DeviceState* st, scratch::Hold& hold, int variant, int64_
       launch_gemm_kernel(dgemm_dmma_ws_kernel<true, 64>, grid, WsCfg<64>::THREADS_, WsCfg<64>::SMEM_BYTES_, stream, map_a, map_b, p);
     else if (variant == DGEMM_VARIANT_TMA_WS)
       launch_gemm_kernel(dgemm_dmma_ws_kernel<true>, grid, WS_THREADS, SMEM_BYTES, stream, map_a, map_b, p);
+    else if (dfma)
+      launch_dfma_kernel<true>(grid, stream, map_a, map_b, p);
     else
       launch_default_kernel<true>(bm, wtm, grid, stream, map_a, map_b, p);
   } else {
@@ -639,6 +663,8 @@ int launch_gemm_packed(DeviceState* st, scratch::Hold& hold, int variant, int64_
                          (size_t)TileCfg<64, 64, BN>::SMEM_BYTES_, stream, map_a, map_b, p);
     else if (variant == DGEMM_VARIANT_GENERIC_WS)
       launch_gemm_kernel(dgemm_dmma_ws_kernel<false>, grid, WS_THREADS, SMEM_BYTES, stream, map_a, map_b, p);
+    else if (dfma)
+      launch_dfma_kernel<false>(grid, stream, map_a, map_b, p);
     else
       launch_default_kernel<false>(bm, wtm, grid, stream, map_a, map_b, p);
   }
@@ -873,6 +899,82 @@ __global__ void __launch_bounds__(256) fp64_probe_kernel(double* out, long long*
   for (int i = 0; i < 8; ++i) r += c[i][0] + c[i][1] + c[i][2] + c[i][3];
   out[blockIdx.x * blockDim.x + threadIdx.x] = r;
   if (threadIdx.x == 0) cycles[blockIdx.x] = t1 - t0;
+}
+
+// The same for plain FP64 fused multiply-adds: 16 independent chains per thread, 512 threads per SM.
+__global__ void __launch_bounds__(512) fp64_fma_probe_kernel(double* out, long long* cycles, int iters, double seed) {
+  double c[16];
+#pragma unroll
+  for (int i = 0; i < 16; ++i) c[i] = i + threadIdx.x;
+  const double a = seed, b = 1.0 - seed;
+  const long long t0 = clock64();
+  for (int it = 0; it < iters; ++it) {
+#pragma unroll
+    for (int r = 0; r < 4; ++r)
+#pragma unroll
+      for (int i = 0; i < 16; ++i) c[i] = fma(c[i], a, b);
+  }
+  const long long t1 = clock64();
+  double r = 0.0;
+#pragma unroll
+  for (int i = 0; i < 16; ++i) r += c[i];
+  out[blockIdx.x * blockDim.x + threadIdx.x] = r;
+  if (threadIdx.x == 0) cycles[blockIdx.x] = t1 - t0;
+}
+
+int run_fp64_probe(bool plain_fma, int millis, double* fma_per_clk_sm, double* tflops) {
+  DeviceState* st = nullptr;
+  int rc = device_state(&st);
+  if (rc != DGEMM_OK) return rc;
+  if (millis < 1) millis = 1;
+  if (millis > 10000) millis = 10000;
+  const int blocks = st->sm_count, threads = plain_fma ? 512 : 256;
+  double* out = nullptr;
+  long long* cyc = nullptr;
+  auto launch = [&](int iters) {
+    if (plain_fma) fp64_fma_probe_kernel<<<blocks, threads>>>(out, cyc, iters, 0.999999);
+    else fp64_probe_kernel<<<blocks, threads>>>(out, cyc, iters, 0.999999);
+  };
+  cudaEvent_t e0 = nullptr, e1 = nullptr;
+  rc = DGEMM_ERR_CUDA;
+  do {
+    if (cudaMalloc(reinterpret_cast<void**>(&out), sizeof(double) * blocks * threads) != cudaSuccess) break;
+    if (cudaMalloc(reinterpret_cast<void**>(&cyc), sizeof(long long) * blocks) != cudaSuccess) break;
+    if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) break;
+    // calibrate with a short run, then size the timed run to about `millis`
+    int iters = 2000;
+    float ms = 0.f;
+    launch(iters);
+    if (cudaEventRecord(e0) != cudaSuccess) break;
+    launch(iters);
+    if (cudaEventRecord(e1) != cudaSuccess || cudaEventSynchronize(e1) != cudaSuccess) break;
+    if (cudaEventElapsedTime(&ms, e0, e1) != cudaSuccess || ms <= 0.f) break;
+    double scale = millis / ms;
+    if (scale > 100000.0) scale = 100000.0;
+    iters = (int)(iters * scale) + 1;
+    if (cudaEventRecord(e0) != cudaSuccess) break;
+    launch(iters);
+    if (cudaEventRecord(e1) != cudaSuccess || cudaEventSynchronize(e1) != cudaSuccess) break;
+    if (cudaEventElapsedTime(&ms, e0, e1) != cudaSuccess) break;
+    g_launches.fetch_add(3);
+    long long* h = static_cast<long long*>(malloc(sizeof(long long) * blocks));
+    if (!h) break;
+    if (cudaMemcpy(h, cyc, sizeof(long long) * blocks, cudaMemcpyDeviceToHost) != cudaSuccess) { free(h); break; }
+    long long mx = 1;
+    for (int i = 0; i < blocks; ++i) if (h[i] > mx) mx = h[i];
+    free(h);
+    // per warp and iteration: 8 MMAs of 16*8*8 = 1024 fused multiply-adds, or 64 FMA instructions of 32 lanes
+    const double fma_per_block = (double)(threads / 32) * iters * (plain_fma ? 64.0 * 32.0 : 8.0 * 1024.0);
+    if (fma_per_clk_sm) *fma_per_clk_sm = fma_per_block / (double)mx;
+    if (tflops) *tflops = 2.0 * fma_per_block * blocks / (ms * 1e-3) / 1e12;
+    rc = DGEMM_OK;
+  } while (0);
+  if (rc != DGEMM_OK) (void)cudaGetLastError();
+  if (e0) cudaEventDestroy(e0);
+  if (e1) cudaEventDestroy(e1);
+  if (out) cudaFree(out);
+  if (cyc) cudaFree(cyc);
+  return rc;
 }
 
 }  // namespace
@@ -1158,54 +1260,11 @@ int dgemm_selftest_wait_timeout(int limit_us) {
 }
 
 int dgemm_fp64_peak_probe(int millis, double* fma_per_clk_sm, double* tflops) {
-  DeviceState* st = nullptr;
-  int rc = device_state(&st);
-  if (rc != DGEMM_OK) return rc;
-  if (millis < 1) millis = 1;
-  if (millis > 10000) millis = 10000;
-  const int blocks = st->sm_count, threads = 256;
-  double* out = nullptr;
-  long long* cyc = nullptr;
-  cudaEvent_t e0 = nullptr, e1 = nullptr;
-  rc = DGEMM_ERR_CUDA;
-  do {
-    if (cudaMalloc(reinterpret_cast<void**>(&out), sizeof(double) * blocks * threads) != cudaSuccess) break;
-    if (cudaMalloc(reinterpret_cast<void**>(&cyc), sizeof(long long) * blocks) != cudaSuccess) break;
-    if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) break;
-    // calibrate with a short run, then size the timed run to about `millis`
-    int iters = 2000;
-    float ms = 0.f;
-    fp64_probe_kernel<<<blocks, threads>>>(out, cyc, iters, 0.999999);
-    if (cudaEventRecord(e0) != cudaSuccess) break;
-    fp64_probe_kernel<<<blocks, threads>>>(out, cyc, iters, 0.999999);
-    if (cudaEventRecord(e1) != cudaSuccess || cudaEventSynchronize(e1) != cudaSuccess) break;
-    if (cudaEventElapsedTime(&ms, e0, e1) != cudaSuccess || ms <= 0.f) break;
-    double scale = millis / ms;
-    if (scale > 100000.0) scale = 100000.0;
-    iters = (int)(iters * scale) + 1;
-    if (cudaEventRecord(e0) != cudaSuccess) break;
-    fp64_probe_kernel<<<blocks, threads>>>(out, cyc, iters, 0.999999);
-    if (cudaEventRecord(e1) != cudaSuccess || cudaEventSynchronize(e1) != cudaSuccess) break;
-    if (cudaEventElapsedTime(&ms, e0, e1) != cudaSuccess) break;
-    g_launches.fetch_add(3);
-    long long* h = static_cast<long long*>(malloc(sizeof(long long) * blocks));
-    if (!h) break;
-    if (cudaMemcpy(h, cyc, sizeof(long long) * blocks, cudaMemcpyDeviceToHost) != cudaSuccess) { free(h); break; }
-    long long mx = 1;
-    for (int i = 0; i < blocks; ++i) if (h[i] > mx) mx = h[i];
-    free(h);
-    // per warp and iteration: 8 MMAs of 16*8*8 = 1024 fused multiply-adds
-    const double fma_per_block = (double)(threads / 32) * iters * 8.0 * 1024.0;
-    if (fma_per_clk_sm) *fma_per_clk_sm = fma_per_block / (double)mx;
-    if (tflops) *tflops = 2.0 * fma_per_block * blocks / (ms * 1e-3) / 1e12;
-    rc = DGEMM_OK;
-  } while (0);
-  if (rc != DGEMM_OK) (void)cudaGetLastError();
-  if (e0) cudaEventDestroy(e0);
-  if (e1) cudaEventDestroy(e1);
-  if (out) cudaFree(out);
-  if (cyc) cudaFree(cyc);
-  return rc;
+  return run_fp64_probe(false, millis, fma_per_clk_sm, tflops);
+}
+
+int dgemm_fp64_fma_probe(int millis, double* fma_per_clk_sm, double* tflops) {
+  return run_fp64_probe(true, millis, fma_per_clk_sm, tflops);
 }
 
 }  // extern "C"

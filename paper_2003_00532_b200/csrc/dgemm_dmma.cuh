@@ -328,6 +328,55 @@ __device__ __forceinline__ void compute_kblock(const uint8_t* st, const LaneMap&
   }
 }
 
+// The micro-kernel swap (the paper's "outer MLIR, inner BLIS" experiment, Section 2.12, turned
+// around: same staging, pipeline, raster and epilogue, another inner kernel). Plain FP64 FMAs on a
+// register tile instead of tensor-core MMAs: every lane keeps the very 8 x 8 scattered elements of
+// the warp tile that the MMA layout gives it (rows row0 + rm + 8i, columns 32wn + 16np + 4t + e),
+// so the epilogue is shared unchanged. Per k a lane needs 8 values of A (one per owned row) and 8
+// of B (one per owned column) for 64 FMAs; they come as 16-byte loads of two consecutive k (A) and
+// two consecutive columns (B) from the same swizzled stage layout. Lanes with equal g read the
+// same A words and lanes with equal t the same B words (broadcast), and the 8 rows / 4 column
+// chunks of a load fall into distinct banks. k runs in ascending order inside the k-block.
+template <int MT = 4>
+__device__ __forceinline__ void compute_kblock_dfma(const uint8_t* st, const LaneMap& m, int a_stage_bytes,
+                                                    double (&acc)[MT][4][4]) {
+  const uint8_t* a_base = st + (m.row0 + m.rm) * 128;
+  const uint8_t* b_base = st + a_stage_bytes + (2 * m.wn) * B_BOX_BYTES;
+#pragma unroll
+  for (int kp = 0; kp < BK / 2; ++kp) {
+    double2 a[MT][2];  // [16-row block][rows +0 / +8]: k = 2kp (x), 2kp + 1 (y)
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+      for (int half = 0; half < 2; ++half)
+        a[mt][half] = *reinterpret_cast<const double2*>(a_base + (16 * mt + 8 * half) * 128 + ((kp ^ m.rm) << 4));
+#pragma unroll
+    for (int kk = 0; kk < 2; ++kk) {
+      const int k = 2 * kp + kk;
+      double2 b[2][2];  // [np][q]: columns 16np + 4t + 2q (x), + 1 (y)
+#pragma unroll
+      for (int np = 0; np < 2; ++np)
+#pragma unroll
+        for (int q = 0; q < 2; ++q)
+          b[np][q] = *reinterpret_cast<const double2*>(b_base + np * B_BOX_BYTES + k * 128 + (((2 * m.t + q) ^ (k & 7)) << 4));
+#pragma unroll
+      for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+          const double av = kk == 0 ? a[mt][half].x : a[mt][half].y;
+#pragma unroll
+          for (int np = 0; np < 2; ++np)
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+              // column offset e = 2q (x), 2q + 1 (y) lives in acc[mt][2np + (e & 1)][2 half + (e >> 1)]
+              acc[mt][2 * np + 0][2 * half + q] = fma(av, b[np][q].x, acc[mt][2 * np + 0][2 * half + q]);
+              acc[mt][2 * np + 1][2 * half + q] = fma(av, b[np][q].y, acc[mt][2 * np + 1][2 * half + q]);
+            }
+        }
+    }
+  }
+}
+
 // ---- the same arithmetic in software-pipelined pieces ---------------------------------------------
 // One half k-block (8 k values) of fragments for a warp tile of 16*MT rows x 32 columns: 48
 // registers for MT = 4. The warp-specialised kernel keeps two of them, so that the loads of the next half
@@ -672,7 +721,12 @@ struct TileCfg {
   static constexpr int SMEM_BYTES_ = STAGES_ * STAGE_BYTES_ + SMEM_ALIGN + 2048 + (EPI_STAGED ? WARPS_ * EPI_WARP_BYTES : 0);
 };
 
-template <bool USE_TMA, int TBM, int WTM = 64, int TBN = BN>
+// MICRO selects the inner kernel: tensor-core MMAs (the product), or plain FMAs on the same register
+// tile (the micro-kernel swap of the ablation ladder).
+constexpr int MICRO_DMMA = 0;
+constexpr int MICRO_DFMA = 1;
+
+template <bool USE_TMA, int TBM, int WTM = 64, int TBN = BN, int MICRO = MICRO_DMMA>
 __global__ void __launch_bounds__(TileCfg<TBM, WTM, TBN>::THREADS_, TileCfg<TBM, WTM, TBN>::CTAS_PER_SM)
 dgemm_dmma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                   const __grid_constant__ GemmParams p) {
@@ -875,7 +929,8 @@ dgemm_dmma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
       const uint32_t s = it % STAGES;
       const uint32_t ph = (it / STAGES) & 1u;
       if (!wait_bounded(full_bar + 8 * s, ph, abort_flag, p)) { ok = false; break; }
-      compute_kblock<false, MT>(tiles + s * STAGE_BYTES, lm, acc);
+      if constexpr (MICRO == MICRO_DFMA) compute_kblock_dfma<MT>(tiles + s * STAGE_BYTES, lm, A_STAGE_BYTES, acc);
+      else compute_kblock<false, MT>(tiles + s * STAGE_BYTES, lm, acc);
       release_stage(empty_bar + 8 * s, lane);
       // keep the load stream LOOKAHEAD k-blocks ahead: refill the stage released two k-blocks ago
       if (!issue_next()) { ok = false; break; }
@@ -1250,6 +1305,33 @@ __global__ void dgemm_wait_timeout_selftest_kernel(const __grid_constant__ GemmP
   ptx::grid_dependency_wait();  // everything above overlaps the tail of the previous kernel in the stream
   const bool ok = wait_bounded(ptx::smem_u32(&bar), 0u, &abort_flag, p);
   if (!ok) atomicAdd(gave_up, 1);
+}
+
+// Rung 1 of the ladder: tiles of A and B in shared memory, still one C element per thread and no
+// register tile (the paper's tiling + packing stage, Sections 2.4-2.6, before unroll-and-jam):
+// every FMA needs two shared-memory loads. 32 x 32 threads per CTA, k in steps of 32, plain loads.
+constexpr int SMEM_RUNG_TILE = 32;
+__global__ void __launch_bounds__(SMEM_RUNG_TILE * SMEM_RUNG_TILE)
+dgemm_smem_kernel(int M, int N, int K, const double* __restrict__ A, long long lda, const double* __restrict__ B,
+                  long long ldb, double* C, long long ldc) {
+  constexpr int T = SMEM_RUNG_TILE;
+  __shared__ double As[T][T + 1];
+  __shared__ double Bs[T][T];
+  const int tx = threadIdx.x, ty = threadIdx.y;
+  const int j = blockIdx.x * T + tx;
+  for (int i0 = blockIdx.y * T; i0 < M; i0 += gridDim.y * T) {  // gridDim.y may be capped
+    const int i = i0 + ty;
+    double acc = 0.0;
+    for (int k0 = 0; k0 < K; k0 += T) {
+      As[ty][tx] = (i < M && k0 + tx < K) ? A[(long long)i * lda + k0 + tx] : 0.0;
+      Bs[ty][tx] = (k0 + ty < K && j < N) ? B[(long long)(k0 + ty) * ldb + j] : 0.0;
+      __syncthreads();
+#pragma unroll
+      for (int k = 0; k < T; ++k) acc = fma(As[ty][k], Bs[k][tx], acc);
+      __syncthreads();
+    }
+    if (i < M && j < N) C[(long long)i * ldc + j] += acc;
+  }
 }
 
 // Rung 0 of the ladder: the naive nest with one thread per C element (Section 2.1).

@@ -100,6 +100,43 @@ def test_config1(oracle, integer, variant):
     _check_full(oracle, prob, run_gpu(prob, variant), stated="config 1 (256^3)")
 
 
+# ---- rungs of the ablation ladder: shared-memory tiles without a register tile, and the FMA
+# ---- micro-kernel under the tensor-core kernels' staging, pipeline and epilogue --------------------
+
+LADDER_VARIANTS = [dg.DGEMM_VARIANT_SMEM, dg.DGEMM_VARIANT_TMA_DFMA, dg.DGEMM_VARIANT_GENERIC_DFMA]
+
+
+@pytest.mark.parametrize("integer", [False, True])
+@pytest.mark.parametrize("variant", LADDER_VARIANTS)
+def test_ladder_rungs_config1(oracle, integer, variant):
+    prob = wl.config1(integer)
+    _check_full(oracle, prob, run_gpu(prob, variant), stated="config 1 (256^3)")
+
+
+@pytest.mark.parametrize("shape", [(1, 1, 1), (17, 13, 11), (127, 129, 47), (130, 260, 33), (257, 131, 100),
+                                   (1000, 32, 600), (513, 33, 64), (1000, 1537, 777)])
+@pytest.mark.parametrize("variant", LADDER_VARIANTS)
+def test_ladder_rungs_ragged(oracle, shape, variant):
+    """Ragged shapes with padded (even) leading dimensions, integer data (exact) and real data (bound)."""
+    M, N, K = shape
+    for integer in (True, False):
+        prob = wl.make_problem(M, N, K, seed=400 + M + N + K, lda=K + 2 + (K & 1), ldb=N + 4 + (N & 1), ldc=N + 7,
+                               integer=integer)
+        _check_full(oracle, prob, run_gpu(prob, variant))
+
+
+@pytest.mark.parametrize("variant", [dg.DGEMM_VARIANT_TMA_DFMA, dg.DGEMM_VARIANT_GENERIC_DFMA])
+def test_dfma_micro_kernel_split_k_and_odd_ld(oracle, variant):
+    """The swapped micro-kernel shares split K, the stream-K tail and the epilogue forms with the tensor-core kernels."""
+    prob = wl.make_problem(200, 150, 1000, seed=11, lda=1000, ldb=152, ldc=151, integer=True)
+    _check_full(oracle, prob, run_gpu(prob, variant, split_k=7))
+    prob = wl.make_problem(2304, 2304, 512, seed=12, integer=True)   # whole waves and a stream-K tail
+    _check_full(oracle, prob, run_gpu(prob, variant))
+    if variant == dg.DGEMM_VARIANT_GENERIC_DFMA:
+        prob = wl.make_problem(300, 260, 200, seed=13, lda=203, ldb=265, ldc=267)
+        _check_full(oracle, prob, run_gpu(prob, variant))
+
+
 # ---- tiny and odd shapes, every variant, padded leading dimensions ---------------------------------
 
 SMALL_SHAPES = [(1, 1, 1), (1, 7, 3), (5, 1, 2), (3, 3, 17), (17, 13, 11), (8, 8, 16), (16, 16, 15),

@@ -1,11 +1,13 @@
-// Single-precision C += A*B for sm_100a: exact binary32 arithmetic on the FP32 pipe (FFMA), fed
-// by the same TMA + mbarrier staging as the FP64 kernels. The paper's SGEMM (Section 2.13) is its
-// DGEMM nest with f64 replaced by f32 and a wider register tile; here the register tile is 8 x 8
-// per thread, the CTA tile 128 x 128 x 32, 256 threads, two CTAs per SM.
+// Single-precision C += A*B for sm_100a: exact binary32 arithmetic on the FP32 pipe, fed by the
+// same TMA + mbarrier staging as the FP64 kernels. The paper's SGEMM (Section 2.13) is its DGEMM
+// nest with f64 replaced by f32 and a wider register tile; here the register tile is 16 x 8 per
+// thread (8 x 8 in the 128-row form), the CTA tile 256 x 128 x 32 (128 x 128 x 32), 256 threads,
+// one CTA per SM, persistent over the tiles with a stream-K tail.
 //
-// The FP32 pipe issues one warp-wide FFMA per scheduler per clock (128 FFMA/clk/SM), so the bound
-// is instruction issue: per 4 k values a thread issues 256 FFMAs, 8 + 8 16-byte shared-memory
-// loads and a few address operations.
+// The FP32 pipe issues one warp-wide instruction per scheduler per clock (128 FMA/clk/SM with
+// scalar FMAs), so the bound is instruction issue. The packed fma.rn.f32x2 performs two independent
+// IEEE FMAs per instruction and halves the issue slots per flop: per 2 k values a thread issues
+// 128 packed FMAs (64 in the 128-row form), 16 (8) 8-byte A loads and 4 16-byte B loads.
 #pragma once
 
 #include <cstdint>

@@ -208,3 +208,18 @@ def test_every_included_file_is_a_build_dependency():
         assert src in deps
         for inc in re.findall(r'#include\s+"([^"]+)"', open(os.path.join(b.CSRC, src)).read()):
             assert os.path.basename(inc) in deps, f"{src} includes {inc}, which build.DEPS does not list"
+
+
+def test_ptxas_check_catches_a_changed_register_count():
+    from paper_2003_00532_b200 import build as b
+    good = "".join(
+        f"ptxas info    : Compiling entry function '_ZN5dgemm{key}Ev' for 'sm_100a'\n"
+        f"    8 bytes stack frame, {spill} bytes spill stores, 8 bytes spill loads\n"
+        f"ptxas info    : Used {regs} registers, used 2 barriers\n" for key, regs, spill in b.PTXAS_EXPECT)
+    b.check_ptxas(good)
+    with pytest.raises(RuntimeError):
+        b.check_ptxas(good.replace("Used 168 registers", "Used 160 registers"))
+    with pytest.raises(RuntimeError):
+        b.check_ptxas(good.replace("128 bytes spill stores", "4000 bytes spill stores", 1))
+    with pytest.raises(RuntimeError):
+        b.check_ptxas("")

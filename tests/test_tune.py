@@ -17,8 +17,8 @@ def test_register_budget_of_the_default_tiles():
 
 
 def test_model_matches_measured_headline():
-    """8192^3 with the warp-specialised kernel: 30.35 ms measured on B200 (CUDA events,
-    profiles/bench_8192_launch_list.md); the model must land within 3 %."""
+    """8192^3 with the warp-specialised kernel: 30.35 ms measured on B200 with CUDA events; the model
+    must land within 3 %."""
     ms = tune.model_ms(8192, 8192, 8192, tune.CONFIGS["ws128"])
     assert abs(ms - 30.35) / 30.35 < 0.03
 

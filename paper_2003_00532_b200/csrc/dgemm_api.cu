@@ -1188,7 +1188,9 @@ int dgemm_set_variant(int variant) {
 }
 
 int dgemm_set_test_flags(int flags) {
-  if (flags < 0 || flags > (DGEMM_TEST_NO_C_PREFETCH | DGEMM_TEST_NO_BLOCKED_B | DGEMM_TEST_TALL_TILES | DGEMM_TEST_SMALL_WARP_TILES | DGEMM_TEST_NO_PACKING | DGEMM_TEST_WS_TWO_CTAS | DGEMM_TEST_NO_CLUSTER)) return DGEMM_ERR_VARIANT;
+  constexpr int kAll = DGEMM_TEST_NO_C_PREFETCH | DGEMM_TEST_NO_BLOCKED_B | DGEMM_TEST_TALL_TILES | DGEMM_TEST_SMALL_WARP_TILES |
+                       DGEMM_TEST_NO_PACKING | DGEMM_TEST_WS_TWO_CTAS | DGEMM_TEST_NO_CLUSTER;
+  if (flags < 0 || (flags & ~kAll) != 0) return DGEMM_ERR_VARIANT;
   g_test_flags.store(flags);
   return DGEMM_OK;
 }

@@ -62,7 +62,13 @@ enum {
                                     and epilogue on 64 x 128 tiles, with plain FP64 fused multiply-adds on an
                                     8 x 8 register tile per thread in place of the tensor-core MMAs */
   DGEMM_VARIANT_GENERIC_DFMA = 9, /* the same inner kernel under the GENERIC staging: any alignment          */
-  DGEMM_VARIANT_COUNT = 10
+  DGEMM_VARIANT_TMA_WS_BULK = 10, /* as TMA_WS on 128 x 128 tiles with three stages and the epilogue done by the
+                                    copy engine: the accumulators go to a tile buffer in shared memory and
+                                    leave as a tiled bulk reduce (add) into C, or a bulk store when beta == 0;
+                                    C is never loaded into the SM. Needs, besides the TMA conditions, a
+                                    16-byte aligned C with even ldc and beta == 0 or 1. What AUTO uses for
+                                    large problems with a short K (rank-k updates)                        */
+  DGEMM_VARIANT_COUNT = 11
 };
 
 /*
@@ -247,8 +253,9 @@ DGEMM_API int dgemm_set_test_flags(int flags);
  * What dgemm_f64 would do with an M x N x K problem under the current variant / split-K / test-flag
  * settings, without touching a device (host logic only; usable on a machine without a GPU):
  * the kernel and tile the library's heuristics choose and how the work is cut (Section 2.10 of
- * the paper explores the same kind of choice by hand). `tma_addressable`: non-zero if A and B are
- * 16-byte aligned with even leading dimensions (or will be after the packing pass). `sm_count`:
+ * the paper explores the same kind of choice by hand). `tma_addressable`: non-zero if A, B and C are
+ * 16-byte aligned with even leading dimensions (A and B: or will be after the packing pass) and
+ * beta is 0 or 1. `sm_count`:
  * streaming multiprocessors to plan for, 0 = 148 (B200); two CTAs per SM are assumed to fit.
  * Writes 12 ints to `out`: resolved variant, tile rows, tile columns, warp-tile rows, CTAs per
  * SM, grid size, k-blocks (ceil(K/16)), uniform K split, k-blocks per split, tiles run whole,

@@ -43,6 +43,7 @@ DGEMM_VARIANT_GENERIC_CLUSTER = 6
 DGEMM_VARIANT_SMEM = 7
 DGEMM_VARIANT_TMA_DFMA = 8
 DGEMM_VARIANT_GENERIC_DFMA = 9
+DGEMM_VARIANT_TMA_WS_BULK = 10
 
 # dgemm_set_test_flags bits
 DGEMM_TEST_NO_C_PREFETCH = 1

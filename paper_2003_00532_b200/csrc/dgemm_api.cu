@@ -17,6 +17,7 @@
 
 #include "dgemm_dmma.cuh"
 #include "dgemm_cluster.cuh"
+#include "dgemm_bulk_epi.cuh"
 #include "scratch_pool.h"
 
 namespace {
@@ -43,6 +44,9 @@ inline bool narrow_tiles_pay(int64_t N) {
   return N <= 96 && (double)cols32 * 1.2 < (double)cols128;
 }
 constexpr int kAutoWs64MaxKblocksPerCta = 256;     // ... and its 64-row form instead of the inline kernel up to this much work
+constexpr int kAutoBulkMaxKblocks = 48;             // bulk-epilogue kernel: up to this many k-blocks per tile (K <= 768: +11 % at
+                                                     // K = 64, +9 % at 128, +4 % at 256, level at 1024, -0.7 % at 8192) ...
+constexpr int kAutoBulkMinWaves = 4;                 // ... and from this many waves of 128 x 128 tiles
 constexpr int kAutoWsMinKblocks = 16;                // warp-specialised kernel: 128-row tiles from K = 256 up, 64-row below
 constexpr double kPackMinFlopPerByte = 32.0;      // pack unaligned operands only if the copy is this cheap
 constexpr double kPackMinFlopPerByteNarrow = 8.0; // ... or this cheap where the generic staging would run the 256 x 32 tile, its slowest form
@@ -68,7 +72,7 @@ struct DeviceState {
   bool ready = false;
   int sm_count = 0;
   bool two_ctas_ok = false;    // the 64-row kernels fit two CTAs per SM on this device
-  bool ws_ok[3] = {false, false, false};  // register pool of the warp-specialised kernels checked: TMA 128, generic 128, TMA 64
+  bool ws_ok[4] = {false, false, false, false};  // register pool of the warp-specialised kernels checked: TMA 128, generic 128, TMA 64, bulk epilogue
   bool cluster_ok = false;     // a cluster of 8 CTAs of the cluster split-K kernel can be resident
   int* status = nullptr;       // device address of g_status_word
   scratch::Pool scratch;       // split-K partial tiles and packed operand copies, leased per call (scratch_pool.h)
@@ -229,6 +233,11 @@ int device_state(DeviceState** out) {
                             WsCfg<128>::CONSUMER_WARPS * 32, WsCfg<128>::PRODUCER_REGS);
       st.ws_ok[2] = pool_ok(reinterpret_cast<const void*>(dgemm_dmma_ws_kernel<true, 64>), WsCfg<64>::THREADS_,
                             WsCfg<64>::CONSUMER_WARPS * 32, WsCfg<64>::PRODUCER_REGS);
+      st.ws_ok[3] = cudaFuncSetAttribute(dgemm_dmma_wsb_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         WsBulkCfg::SMEM_BYTES_) == cudaSuccess &&
+                    pool_ok(reinterpret_cast<const void*>(dgemm_dmma_wsb_kernel), WsBulkCfg::THREADS_,
+                            WsBulkCfg::CONSUMER_WARPS * 32, WS_PRODUCER_REGS);
+      (void)cudaGetLastError();
     }
     {
       // cluster split-K kernel: shared-memory opt-in, then ask whether a full-size cluster fits
@@ -395,7 +404,7 @@ void fill_cluster_plan(Plan& pl, int tiles, int kblocks, int s, bool tma) {
 }
 
 Plan plan_gemm(int64_t M, int64_t N, int64_t K, bool tma_ok, int requested_variant, int dbg_flags, int forced_split,
-               int sm_count, bool two_ctas_ok, const bool ws_ok[3], bool cluster_ok) {
+               int sm_count, bool two_ctas_ok, const bool ws_ok[4], bool cluster_ok, bool c_bulk_ok) {
   Plan pl;
   memset(&pl, 0, sizeof(pl));
   pl.status = DGEMM_OK;
@@ -428,13 +437,19 @@ Plan plan_gemm(int64_t M, int64_t N, int64_t K, bool tma_ok, int requested_varia
         auto_ws64 = tiles64 * kblocks <= (int64_t)kAutoWs64MaxKblocksPerCta * 2 * sm_count;
       }
       variant = ((ws && ws_ok[0] && ws_ok[2]) || auto_ws64) ? DGEMM_VARIANT_TMA_WS : DGEMM_VARIANT_TMA;
+      // Many tiles of few k-blocks each (a rank-k update): the C round trip of a tile is long next to
+      // its arithmetic. The bulk-epilogue kernel takes it off the arithmetic warps altogether.
+      if (std_tile && c_bulk_ok && ws_ok[3] && kblocks <= kAutoBulkMaxKblocks && tiles128 >= (int64_t)kAutoBulkMinWaves * sm_count &&
+          (double)pad128 <= 1.03 * (double)pad64 && !(dbg_flags & DGEMM_TEST_WS_TWO_CTAS))
+        variant = DGEMM_VARIANT_TMA_WS_BULK;
     }
   }
   pl.variant = variant;
   const bool dfma = variant == DGEMM_VARIANT_TMA_DFMA || variant == DGEMM_VARIANT_GENERIC_DFMA;
   const bool wants_tma = variant == DGEMM_VARIANT_TMA || variant == DGEMM_VARIANT_TMA_WS || variant == DGEMM_VARIANT_TMA_CLUSTER ||
-                         variant == DGEMM_VARIANT_TMA_DFMA;
+                         variant == DGEMM_VARIANT_TMA_DFMA || variant == DGEMM_VARIANT_TMA_WS_BULK;
   if (wants_tma && !tma_ok) { pl.status = DGEMM_ERR_VARIANT; return pl; }
+  if (variant == DGEMM_VARIANT_TMA_WS_BULK && !(c_bulk_ok && ws_ok[3])) { pl.status = DGEMM_ERR_VARIANT; return pl; }
   if (dfma && !two_ctas_ok) { pl.status = DGEMM_ERR_VARIANT; return pl; }
   if (variant == DGEMM_VARIANT_TMA_CLUSTER || variant == DGEMM_VARIANT_GENERIC_CLUSTER) {
     // forced: clusters of dgemm_set_split_k() CTAs if that is 1, 2, 4 or 8 (ranks beyond the last
@@ -462,7 +477,7 @@ Plan plan_gemm(int64_t M, int64_t N, int64_t K, bool tma_ok, int requested_varia
     return pl;
   }
 
-  const bool ws_variant = variant == DGEMM_VARIANT_TMA_WS || variant == DGEMM_VARIANT_GENERIC_WS;
+  const bool ws_variant = variant == DGEMM_VARIANT_TMA_WS || variant == DGEMM_VARIANT_GENERIC_WS || variant == DGEMM_VARIANT_TMA_WS_BULK;
   // tile height of the chosen kernel: 64 rows with two CTAs per SM (inline kernel; warp-specialised kernel for short K),
   // 128 rows with one CTA per SM (warp-specialised kernel otherwise, large generic problems, test flag)
   // (generic staging on a problem of many waves is a little faster with the tall tile: half the B copies per thread)
@@ -580,13 +595,15 @@ int launch_gemm_packed(DeviceState* st, scratch::Hold& hold, int variant, int64_
   int rc = DGEMM_OK;
   const bool tma_ok = (((uintptr_t)A | (uintptr_t)B) & 15) == 0 && (lda % 2 == 0) && (ldb % 2 == 0);
   const int dbg_flags = g_test_flags.load();
+  // C as the copy engine needs it for the bulk epilogue, and a beta it can apply (add, or overwrite)
+  const bool c_bulk_ok = ((uintptr_t)C & 15) == 0 && (ldc % 2 == 0) && (form.beta == 1.0 || form.beta == 0.0);
   const Plan plan = plan_gemm(M, N, K, tma_ok, variant, dbg_flags, g_split_k.load(), st->sm_count, st->two_ctas_ok, st->ws_ok,
-                              st->cluster_ok);
+                              st->cluster_ok, c_bulk_ok);
   if (plan.status != DGEMM_OK) return plan.status;
   variant = plan.variant;
   const bool dfma = variant == DGEMM_VARIANT_TMA_DFMA || variant == DGEMM_VARIANT_GENERIC_DFMA;
   const bool wants_tma = variant == DGEMM_VARIANT_TMA || variant == DGEMM_VARIANT_TMA_WS || variant == DGEMM_VARIANT_TMA_CLUSTER ||
-                         variant == DGEMM_VARIANT_TMA_DFMA;
+                         variant == DGEMM_VARIANT_TMA_DFMA || variant == DGEMM_VARIANT_TMA_WS_BULK;
   const bool cluster = variant == DGEMM_VARIANT_TMA_CLUSTER || variant == DGEMM_VARIANT_GENERIC_CLUSTER;
 
   if (variant == DGEMM_VARIANT_NAIVE) {
@@ -649,7 +666,13 @@ int launch_gemm_packed(DeviceState* st, scratch::Hold& hold, int variant, int64_
     if (cluster)
       launch_cluster_pdl(dgemm_cluster_kernel<true, 64, 64, BN>, grid, p.split_k, TileCfg<64, 64, BN>::THREADS_,
                          (size_t)TileCfg<64, 64, BN>::SMEM_BYTES_, stream, map_a, map_b, p);
-    else if (ws64)
+    else if (variant == DGEMM_VARIANT_TMA_WS_BULK) {
+      CUtensorMap map_c;
+      memset(&map_c, 0, sizeof(map_c));
+      if (!make_map(&map_c, C, M, N, ldc, 16, 64)) return DGEMM_ERR_CUDA;  // boxes of 16 columns x 64 rows, 128-byte swizzle
+      launch_pdl(dgemm_dmma_wsb_kernel, dim3(grid), dim3(WsBulkCfg::THREADS_), (size_t)WsBulkCfg::SMEM_BYTES_, stream, map_a, map_b,
+                 map_c, p);
+    } else if (ws64)
       launch_gemm_kernel(dgemm_dmma_ws_kernel<true, 64>, grid, WsCfg<64>::THREADS_, WsCfg<64>::SMEM_BYTES_, stream, map_a, map_b, p);
     else if (variant == DGEMM_VARIANT_TMA_WS)
       launch_gemm_kernel(dgemm_dmma_ws_kernel<true>, grid, WS_THREADS, SMEM_BYTES, stream, map_a, map_b, p);
@@ -1171,9 +1194,9 @@ int dgemm_version(void) { return 100; /* 0.1.0 */ }
 int dgemm_plan(int64_t M, int64_t N, int64_t K, int tma_addressable, int sm_count, int* out) {
   if (!out) return DGEMM_ERR_NULL;
   if (M <= 0 || N <= 0 || K <= 0 || M > INT32_MAX - 512 || N > INT32_MAX - 512 || K > INT32_MAX - 512) return DGEMM_ERR_BAD_DIM;
-  const bool ws_ok[3] = {true, true, true};
+  const bool ws_ok[4] = {true, true, true, true};
   const Plan pl = plan_gemm(M, N, K, tma_addressable != 0, g_variant.load(), g_test_flags.load(), g_split_k.load(),
-                            sm_count > 0 ? sm_count : 148, true, ws_ok, true);
+                            sm_count > 0 ? sm_count : 148, true, ws_ok, true, tma_addressable != 0);
   if (pl.status != DGEMM_OK) return pl.status;
   const int v[12] = {pl.variant, pl.bm, pl.bn, pl.wtm, pl.ctas_per_sm, pl.grid, pl.kblocks, pl.split_k,
                      pl.kblocks_per_split, pl.dp_tiles, pl.tail_tiles, pl.tail_ipc};

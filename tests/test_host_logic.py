@@ -101,7 +101,7 @@ def test_variant_and_split_setters():
     assert dg.dgemm_set_variant(dg.DGEMM_VARIANT_GENERIC) == 0
     assert dg.dgemm_set_variant(dg.DGEMM_VARIANT_AUTO) == 0
     with pytest.raises(dg.DgemmError):
-        dg.dgemm_set_variant(10)
+        dg.dgemm_set_variant(dg.binding.DGEMM_VARIANT_TMA_WS_BULK + 1)
     with pytest.raises(dg.DgemmError):
         dg.dgemm_set_variant(-2)
     assert dg.dgemm_set_variant(dg.DGEMM_VARIANT_TMA_WS) == 0 and dg.dgemm_set_variant(dg.DGEMM_VARIANT_AUTO) == 0

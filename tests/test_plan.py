@@ -14,6 +14,7 @@ import paper_2003_00532_b200 as dg
 V_TMA, V_GENERIC, V_WS = dg.DGEMM_VARIANT_TMA, dg.DGEMM_VARIANT_GENERIC, dg.DGEMM_VARIANT_TMA_WS
 V_CLUSTER = dg.DGEMM_VARIANT_TMA_CLUSTER
 V_GCLUSTER = dg.DGEMM_VARIANT_GENERIC_CLUSTER
+V_WSB = dg.DGEMM_VARIANT_TMA_WS_BULK
 
 
 @pytest.fixture(autouse=True)
@@ -32,8 +33,10 @@ def _defaults():
 @pytest.mark.parametrize("shape,variant,bm,bn,wtm", [
     ((8192, 8192, 8192), V_WS, 128, 128, 64),      # large, aligned: warp-specialised, one CTA per SM
     ((4096, 4096, 4096), V_WS, 128, 128, 64),
-    ((16384, 16384, 64), V_WS, 64, 128, 64),       # K < 256: the same kernel with two CTAs per SM
-    ((16384, 16384, 256), V_WS, 128, 128, 64),
+    ((16384, 16384, 64), V_WSB, 128, 128, 64),     # many tiles of few k-blocks: the epilogue leaves through the copy engine
+    ((16384, 16384, 256), V_WSB, 128, 128, 64),
+    ((16384, 16384, 1024), V_WS, 128, 128, 64),    # ... up to 48 k-blocks per tile
+    ((2048, 2048, 64), V_WS, 64, 128, 64),         # few tiles, K < 256: the warp-specialised kernel with two CTAs per SM
     ((2088, 2048, 2048), V_WS, 64, 128, 64),       # M just above a multiple of 64 rows: 64-row tiles, two CTAs per SM
     ((1600, 8192, 8192), V_TMA, 64, 128, 64),      # the same on a long problem: inline kernel
     ((256, 256, 256), V_WS, 64, 128, 64),          # one k-block per CTA through the workspace: the general kernels' floor

@@ -244,10 +244,24 @@ enum {
   DGEMM_TEST_NO_PACKING = 16,   /* never pack unaligned operands: always use the generic staging      */
   DGEMM_TEST_WS_TWO_CTAS = 32,  /* DGEMM_VARIANT_TMA_WS: 64-row tiles, two CTAs per SM, at any K (the
                                    library itself uses that form only for K < 256)                 */
-  DGEMM_TEST_NO_CLUSTER = 128   /* DGEMM_VARIANT_AUTO never picks the cluster split-K kernel: problems
+  DGEMM_TEST_NO_CLUSTER = 128,  /* DGEMM_VARIANT_AUTO never picks the cluster split-K kernel: problems
                                    below one wave of tiles cut K through the workspace instead   */
+  DGEMM_TEST_DROP_LOADS = 256   /* failure injection on the host's say-so: the kernels' producers skip their
+                                   copies (like a message that is dropped), so the bounded waits of the
+                                   arithmetic run out, the kernels report DGEMM_ERR_TIMEOUT through the
+                                   status word and return in the ordinary way; C is then unspecified.
+                                   Nothing faults, traps or spins without a limit. Use together with
+                                   dgemm_set_test_wait_limit, or every wait takes its full four seconds */
 };
 DGEMM_API int dgemm_set_test_flags(int flags);
+
+/*
+ * Testing aid (no counterpart in the paper): the limit of the kernels' main-loop waits in
+ * microseconds for subsequent calls, 1 .. 4 000 000, or 0 for the default of four seconds. The
+ * separate wait that lets copies in flight land before an aborting thread block exits keeps its
+ * own four seconds. Returns DGEMM_OK or DGEMM_ERR_VARIANT.
+ */
+DGEMM_API int dgemm_set_test_wait_limit(int limit_us);
 
 /*
  * What dgemm_f64 would do with an M x N x K problem under the current variant / split-K / test-flag

@@ -53,6 +53,7 @@ DGEMM_TEST_SMALL_WARP_TILES = 8
 DGEMM_TEST_NO_PACKING = 16
 DGEMM_TEST_WS_TWO_CTAS = 32
 DGEMM_TEST_NO_CLUSTER = 128
+DGEMM_TEST_DROP_LOADS = 256
 
 
 class DgemmError(RuntimeError):
@@ -282,6 +283,14 @@ def dgemm_set_split_k(split_k: int) -> int:
     rc = load_library().dgemm_set_split_k(int(split_k))
     if rc < 0:
         raise DgemmError(rc, "dgemm_set_split_k")
+    return rc
+
+
+def dgemm_set_test_wait_limit(limit_us: int) -> int:
+    """Testing aid: limit of the kernels' main-loop waits in microseconds (0 = the default four seconds)."""
+    rc = load_library().dgemm_set_test_wait_limit(int(limit_us))
+    if rc < 0:
+        raise DgemmError(rc, "dgemm_set_test_wait_limit")
     return rc
 
 

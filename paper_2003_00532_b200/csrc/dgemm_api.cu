@@ -85,6 +85,7 @@ std::atomic<int> g_variant{DGEMM_VARIANT_AUTO};
 std::atomic<int> g_split_k{0};
 std::atomic<int> g_test_flags{0};
 std::atomic<long long> g_launches{0};
+std::atomic<long long> g_test_wait_limit_ns{0};  // 0: the default limit of the device-side waits
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -552,7 +553,7 @@ Plan plan_gemm(int64_t M, int64_t N, int64_t K, bool tma_ok, int requested_varia
     // 64-row tile, doubled where two CTAs of the general kernels share an SM. Runs of more than 8
     // k-blocks per CTA stay with the general kernels, whose main loops are the faster ones. Any
     // test flag that asks for a particular tile or reduction keeps the general kernels too.
-    if (auto_choice && cluster_ok && two_ctas_ok && !(dbg_flags & ~(DGEMM_TEST_NO_C_PREFETCH | DGEMM_TEST_NO_BLOCKED_B)) && tiles < sms &&
+    if (auto_choice && cluster_ok && two_ctas_ok && !(dbg_flags & ~(DGEMM_TEST_NO_C_PREFETCH | DGEMM_TEST_NO_BLOCKED_B | DGEMM_TEST_DROP_LOADS)) && tiles < sms &&
         (pl.wtm == 64 || bm == 32)) {  // (not the test-only 32 x 32 warp tiles of the larger tiles)
       // costs in tenths of a k-block; a pass of the in-cluster reduction (512 element pairs per
       // CTA) is worth about 0.4 k-blocks, the second launch of the workspace split about one.
@@ -633,7 +634,11 @@ int launch_gemm_packed(DeviceState* st, scratch::Hold& hold, int variant, int64_
   p.tiles_n = (int)((N + bn - 1) / bn);
   p.A = A; p.B = B; p.C = C;
   p.lda = lda; p.ldb = ldb; p.ldc = ldc;
-  p.wait_limit_ns = kWaitLimitNs;
+  {
+    const long long test_limit = g_test_wait_limit_ns.load();
+    p.wait_limit_ns = test_limit > 0 ? (unsigned long long)test_limit : kWaitLimitNs;
+  }
+  p.drop_loads = (dbg_flags & DGEMM_TEST_DROP_LOADS) ? 1 : 0;
   p.status = st->status;
   p.group_m = 1024 / bm;  // 1024 rows per raster group
   p.alpha = form.alpha;
@@ -1212,9 +1217,15 @@ int dgemm_set_variant(int variant) {
 
 int dgemm_set_test_flags(int flags) {
   constexpr int kAll = DGEMM_TEST_NO_C_PREFETCH | DGEMM_TEST_NO_BLOCKED_B | DGEMM_TEST_TALL_TILES | DGEMM_TEST_SMALL_WARP_TILES |
-                       DGEMM_TEST_NO_PACKING | DGEMM_TEST_WS_TWO_CTAS | DGEMM_TEST_NO_CLUSTER;
+                       DGEMM_TEST_NO_PACKING | DGEMM_TEST_WS_TWO_CTAS | DGEMM_TEST_NO_CLUSTER | DGEMM_TEST_DROP_LOADS;
   if (flags < 0 || (flags & ~kAll) != 0) return DGEMM_ERR_VARIANT;
   g_test_flags.store(flags);
+  return DGEMM_OK;
+}
+
+int dgemm_set_test_wait_limit(int limit_us) {
+  if (limit_us < 0 || limit_us > 4000000) return DGEMM_ERR_VARIANT;
+  g_test_wait_limit_ns.store((long long)limit_us * 1000ll);
   return DGEMM_OK;
 }
 

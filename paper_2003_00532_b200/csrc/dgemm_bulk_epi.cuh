@@ -116,7 +116,9 @@ dgemm_dmma_wsb_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
         const uint32_t fb = full_bar + 8 * s;
         int good = 1;
         if (lane == 0) {
-          if (wait_bounded_inline(empty_bar + 8 * s, ph ^ 1u, abort_flag, p)) {
+          if (!wait_bounded_inline(empty_bar + 8 * s, ph ^ 1u, abort_flag, p)) {
+            good = 0;
+          } else if (!p.drop_loads) {
             ptx::mbar_arrive_expect_tx(fb, STAGE_BYTES);
             ptx::tma_load_2d(sa, &map_a, kb * BK, w.tm * TBM, fb);
             if (p.b_blocked_map) {
@@ -124,22 +126,20 @@ dgemm_dmma_wsb_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
             } else {
               tma_load_b_boxes_inline(sb, &map_b, w.tn * BN, kb * BK, fb);
             }
-          } else {
-            good = 0;
           }
         }
         if (!__all_sync(0xffffffffu, good)) { ok = false; break; }
         if (kb == kb_pf) prefetch_c_rows_inline(p.C, p.ldc, p.M, p.N, TBM, BN, w.tm, w.tn, lane, 32);
       }
     }
-    if (!ok && pw == 0 && lane == 0) {
+    if (!ok && !p.drop_loads && pw == 0 && lane == 0) {
       // aborting: let every copy this thread armed land before the CTA's memory is released
       const uint32_t n_inflight = it < (uint32_t)STAGES ? it : (uint32_t)STAGES;
       for (uint32_t q = it - n_inflight; q < it; ++q) {
         const uint32_t s = q % STAGES, ph = (q / STAGES) & 1u;
         const unsigned long long t0 = ptx::globaltimer_ns();
         while (!ptx::mbar_try_wait(full_bar + 8 * s, ph)) {
-          if (ptx::globaltimer_ns() - t0 > p.wait_limit_ns) break;
+          if (ptx::globaltimer_ns() - t0 > DRAIN_LIMIT_NS) break;
         }
       }
     }

@@ -54,6 +54,9 @@ constexpr int EPI_STRIDE = 32 * 8 + 16;
 constexpr int EPI_WARP_BYTES = 8 * EPI_STRIDE;
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + SMEM_ALIGN + 1024 + WARPS * EPI_WARP_BYTES;  // + barriers, abort flag, work-item words, epilogue staging
 constexpr int STATUS_TIMEOUT = -8;          // DGEMM_ERR_TIMEOUT
+// After an abort a CTA lets the copies it has in flight land before it gives up its shared memory: that
+// wait has a limit of its own, not the (possibly shortened) limit of the main-loop waits.
+constexpr unsigned long long DRAIN_LIMIT_NS = 4000000000ull;
 constexpr int C_PREFETCH_KBLOCKS = 8;       // C tile is requested into L2 this many k-blocks before the tile ends
 
 // Work decomposition. Phase 1: the first `dp_tiles` tiles (in raster order), each split into
@@ -88,6 +91,7 @@ struct GemmParams {
   long long lda, ldb, ldc;
   unsigned long long wait_limit_ns;
   int* status;            // device status word
+  int drop_loads;         // testing aid: the producers skip their copies, so that the consumers' waits run out
 };
 
 struct Work {
@@ -812,7 +816,9 @@ dgemm_dmma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
       if (warp == (int)(lit % WARPS)) {
         int good = 1;
         if (lane == 0) {
-          if (wait_bounded<false>(empty_bar + 8 * s, ph ^ 1u, abort_flag, p)) {
+          if (!wait_bounded<false>(empty_bar + 8 * s, ph ^ 1u, abort_flag, p)) {
+            good = 0;
+          } else if (!p.drop_loads) {
             ptx::mbar_arrive_expect_tx(fb, STAGE_BYTES);
             ptx::tma_load_2d(sa, &map_a, kb * BK, cur_tm * TBM, fb);
             if (p.b_blocked_map) {
@@ -820,14 +826,13 @@ dgemm_dmma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
             } else {
               tma_load_b_boxes(sb, &map_b, cur_tn * TBN, kb * BK, fb, TBN / 16);
             }
-          } else {
-            good = 0;
           }
         }
         if (!__all_sync(0xffffffffu, good)) return false;
       }
     } else {
       if (!wait_bounded<false>(empty_bar + 8 * s, ph ^ 1u, abort_flag, p)) return false;
+      if (!p.drop_loads) {
       // 8-byte asynchronous copies with zero fill outside the matrices; any alignment, any leading
       // dimension. A: 16 consecutive threads copy the 16 k values of one row (8 rows per thread);
       // B: 32 consecutive threads copy 32 consecutive columns of one k row (8 k rows per thread).
@@ -882,6 +887,7 @@ dgemm_dmma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         }
       }
       ptx::cp_async_mbar_arrive_noinc(fb);
+      }
     }
     if (kb == cur_pf) {
       // TMA staging: the issuing warp's lanes take 4 rows each; generic: one row per thread of the first 128
@@ -944,13 +950,13 @@ dgemm_dmma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
   // Leaving. After a normal run every copy that was issued has been consumed. After an abort,
   // copies may still be in flight into this CTA's shared memory: let them land first.
   if (!USE_TMA) ptx::cp_async_wait_all();
-  if (USE_TMA && !ok && tid == 0) {
+  if (USE_TMA && !ok && !p.drop_loads && tid == 0) {
     const uint32_t n_inflight = lit < (uint32_t)STAGES ? lit : (uint32_t)STAGES;
     for (uint32_t q = lit - n_inflight; q < lit; ++q) {
       const uint32_t s = q % STAGES, ph = (q / STAGES) & 1u;
       const unsigned long long t0 = ptx::globaltimer_ns();
       while (!ptx::mbar_try_wait(full_bar + 8 * s, ph)) {
-        if (ptx::globaltimer_ns() - t0 > p.wait_limit_ns) break;
+        if (ptx::globaltimer_ns() - t0 > DRAIN_LIMIT_NS) break;
       }
     }
   }
@@ -1057,7 +1063,9 @@ dgemm_dmma_ws_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
         if (USE_TMA) {
           int good = 1;
           if (lane == 0) {
-            if (wait_bounded_inline(empty_bar + 8 * s, ph ^ 1u, abort_flag, p)) {
+            if (!wait_bounded_inline(empty_bar + 8 * s, ph ^ 1u, abort_flag, p)) {
+              good = 0;
+            } else if (!p.drop_loads) {
               ptx::mbar_arrive_expect_tx(fb, STAGE_BYTES);
               ptx::tma_load_2d(sa, &map_a, kb * BK, w.tm * TBM, fb);
               if (p.b_blocked_map) {
@@ -1065,8 +1073,6 @@ dgemm_dmma_ws_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
               } else {
                 tma_load_b_boxes_inline(sb, &map_b, w.tn * BN, kb * BK, fb);
               }
-            } else {
-              good = 0;
             }
           }
           if (!__all_sync(0xffffffffu, good)) { ok = false; break; }
@@ -1074,6 +1080,7 @@ dgemm_dmma_ws_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
         } else {
           if (!wait_bounded_inline(empty_bar + 8 * s, ph ^ 1u, abort_flag, p)) { ok = false; break; }
           const int m0 = w.tm * BM, n0 = w.tn * BN, k0 = kb * BK;
+          if (!p.drop_loads) {
           {
             const int a_r = lane >> 4, a_k = lane & 15;
             const int k = k0 + a_k;
@@ -1103,19 +1110,20 @@ dgemm_dmma_ws_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
             }
           }
           ptx::cp_async_mbar_arrive_noinc(fb);
+          }
           if (kb == kb_pf) prefetch_c_rows_inline(p.C, p.ldc, p.M, p.N, BM, BN, w.tm, w.tn, 32 * pw + lane, BM);
         }
       }
     }
     if (!USE_TMA) ptx::cp_async_wait_all();
-    if (USE_TMA && !ok && pw == 0 && lane == 0) {
+    if (USE_TMA && !ok && !p.drop_loads && pw == 0 && lane == 0) {
       // aborting: let every copy this thread armed land before the CTA's memory is released
       const uint32_t n_inflight = it < (uint32_t)STAGES ? it : (uint32_t)STAGES;
       for (uint32_t q = it - n_inflight; q < it; ++q) {
         const uint32_t s = q % STAGES, ph = (q / STAGES) & 1u;
         const unsigned long long t0 = ptx::globaltimer_ns();
         while (!ptx::mbar_try_wait(full_bar + 8 * s, ph)) {
-          if (ptx::globaltimer_ns() - t0 > p.wait_limit_ns) break;
+          if (ptx::globaltimer_ns() - t0 > DRAIN_LIMIT_NS) break;
         }
       }
     }

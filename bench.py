@@ -355,11 +355,13 @@ def run_ours(args):
     n = args.size
     if args.shape:
         sm, sn, sk = (int(x) for x in args.shape.split(","))
-        prob = wl.make_problem(sm, sn, sk, 3, pin=True)  # another shape (profiling aid), rank-k seed
+        pad = dict(lda=sk + 3, ldb=sn + 5, ldc=sn + 7) if args.pad else {}  # the ragged configuration's leading dimensions
+        prob = wl.make_problem(sm, sn, sk, 2 if args.pad else 3, pin=True, **pad)  # another shape (profiling aid)
     else:
         sm = sn = sk = n
         prob = wl.make_problem(n, n, n, 1, pin=True)  # seed 1: the large square configuration
-    A, B, C = prob.A_buf.cuda(), prob.B_buf.cuda(), prob.C_buf.cuda()
+    A_dev, B_dev, C_dev = prob.A_buf.cuda(), prob.B_buf.cuda(), prob.C_buf.cuda()
+    A, B, C = A_dev[:, :sk], B_dev[:, :sn], C_dev[:, :sn]  # the logical matrices inside their (possibly padded) buffers
     flop = prob.flop
     stream = torch.cuda.current_stream()
 
@@ -412,15 +414,15 @@ def run_ours(args):
     link = {}
     if rank == 0:
         ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
-        A.copy_(prob.A_buf, non_blocking=True)  # warm-up
+        A_dev.copy_(prob.A_buf, non_blocking=True)  # warm-up
         torch.cuda.synchronize()
         ev[0].record(stream)
-        A.copy_(prob.A_buf, non_blocking=True)
+        A_dev.copy_(prob.A_buf, non_blocking=True)
         ev[1].record(stream)
-        prob.A_buf.copy_(A, non_blocking=True)
+        prob.A_buf.copy_(A_dev, non_blocking=True)
         ev[2].record(stream)
         torch.cuda.synchronize()
-        nbytes = A.numel() * 8
+        nbytes = A_dev.numel() * 8
         link = {"h2d_gbs": nbytes / (ev[0].elapsed_time(ev[1]) * 1e-3) / 1e9,
                 "d2h_gbs": nbytes / (ev[1].elapsed_time(ev[2]) * 1e-3) / 1e9}
         link["floor_ms_per_step"] = max(h2d / (link["h2d_gbs"] * 1e9), d2h / (link["d2h_gbs"] * 1e9)) * 1e3
@@ -512,6 +514,7 @@ def main():
     ap.add_argument("--cpu-rows", type=int, default=3072, help="rows of C in the cpu_baseline sample")
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--shape", type=str, default="", help="M,N,K of another (non-square) workload; profiling aid")
+    ap.add_argument("--pad", action="store_true", help="with --shape: padded leading dimensions lda=K+3, ldb=N+5, ldc=N+7, seed 2")
     ap.add_argument("--no-sweep", action="store_true", help="skip the size sweep and the ragged / rank-k shapes")
     ap.add_argument("--variant", type=int, default=-1, help="profiling aid: force a DGEMM_VARIANT_* for the timed calls")
     ap.add_argument("--flags", type=int, default=0, help="profiling aid: DGEMM_TEST_* flags for the timed calls")

@@ -20,9 +20,9 @@
 //     (cp.async.bulk.wait_group.read in the issuing thread). The turns keep the slabs a few thousand
 //     cycles apart for good, and that is wanted: the two warps that share a scheduler belong to
 //     different slabs, so one of them multiplies while the other is in its epilogue. The hand-overs
-//     (buffer written: four warps -> issuing thread; buffer free: issuing thread -> the next four
-//     warps) go through two mbarriers with the same bounded waits as the stages, so a warp that
-//     gives up cannot leave anybody at a barrier.
+//     (buffer written: four warps -> issuing thread; your turn: issuing thread -> the next four
+//     warps, one barrier per slab) are mbarriers with the same bounded waits as the stages, so a
+//     warp that gives up cannot leave anybody at a barrier.
 // Needs a C the copy engine can address: 16-byte aligned base, even ldc; beta == 0 or 1.
 // Partial tiles (stream-K tail, forced split K) go to the workspace as in the other kernels.
 #pragma once
@@ -54,13 +54,17 @@ dgemm_dmma_wsb_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
   const uint32_t pad = (SMEM_ALIGN - (raw & (SMEM_ALIGN - 1))) & (SMEM_ALIGN - 1);
   uint8_t* tiles = smem_raw + pad;
   uint64_t* bars = reinterpret_cast<uint64_t*>(tiles + WsBulkCfg::BAR_OFFSET);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 2 * STAGES + 2);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 2 * STAGES + 3);
   volatile int* work_words = abort_flag + 8;  // 8 words per warp (12 warps)
   const uint32_t tiles_u32 = raw + pad;
   const uint32_t full_bar = tiles_u32 + WsBulkCfg::BAR_OFFSET;
   const uint32_t empty_bar = full_bar + 8 * STAGES;
-  const uint32_t c_free = empty_bar + 8 * STAGES;  // the tile buffer may be overwritten (issuing thread -> the next slab's 4 warps)
-  const uint32_t c_full = c_free + 8;              // the tile buffer is written (a slab's 4 warps -> issuing thread)
+  // Hand-overs of the tile buffer. c_full: written (a slab's 4 warps -> issuing thread), one phase per
+  // use. c_turn[s]: slab s may write now (issuing thread -> slab s's 4 warps), one phase per turn of
+  // that slab. A barrier per slab, so that no waiter can ever be two phases away from the barrier it
+  // polls: a parity wait cannot tell phase n from phase n - 2.
+  const uint32_t c_full = empty_bar + 8 * STAGES;
+  const uint32_t c_turn = c_full + 8;  // c_turn + 8 * slab
   const uint32_t c_buf = tiles_u32 + WsBulkCfg::C_OFFSET;
 
   const int tid = threadIdx.x;
@@ -72,8 +76,9 @@ dgemm_dmma_wsb_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
       ptx::mbar_init(full_bar + 8 * s, 1);
       ptx::mbar_init(empty_bar + 8 * s, WARPS);
     }
-    ptx::mbar_init(c_free, 1);
     ptx::mbar_init(c_full, 4);
+    ptx::mbar_init(c_turn, 1);
+    ptx::mbar_init(c_turn + 8, 1);
     *abort_flag = 0;
     ptx::fence_barrier_init();
   }
@@ -178,7 +183,7 @@ dgemm_dmma_wsb_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
               ptx::bulk_commit_group();
               pending = true;
               ptx::bulk_wait_group_read_all();  // the copy engine has read the buffer
-              ptx::mbar_arrive(c_free);
+              ptx::mbar_arrive(c_turn + 8 * ((use + 1) & 1u));  // the other slab's turn
             }
           }
           if (!__all_sync(0xffffffffu, good)) ok = false;
@@ -244,9 +249,10 @@ dgemm_dmma_wsb_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
         continue;
       }
       // ---- the tile leaves through the copy engine
-      // this slab's turn: the previous user's data (the other slab's) has been read by the copy engine
+      // this slab's turn: the previous user's data (the other slab's) has been read by the copy engine.
+      // Slab 0 starts; turn number `turns` of a slab is phase `turns` of its barrier (slab 0: turns - 1).
       // (the decision to leave is taken by the whole warp: once per tile, a vote is cheap)
-      if (use > 0 && !__all_sync(0xffffffffu, wait_bounded_inline(c_free, (use - 1) & 1u, abort_flag, p) ? 1 : 0)) { ok = false; break; }
+      if (use > 0 && !__all_sync(0xffffffffu, wait_bounded_inline(c_turn + 8 * slab, ((use - 1) >> 1) & 1u, abort_flag, p) ? 1 : 0)) { ok = false; break; }
       if (p.alpha != 1.0) {
 #pragma unroll
         for (int mt = 0; mt < 4; ++mt)

@@ -74,6 +74,7 @@ struct DeviceState {
   bool two_ctas_ok = false;    // the 64-row kernels fit two CTAs per SM on this device
   bool ws_ok[4] = {false, false, false, false};  // register pool of the warp-specialised kernels checked: TMA 128, generic 128, TMA 64, bulk epilogue
   bool cluster_ok = false;     // a cluster of 8 CTAs of the cluster split-K kernel can be resident
+  bool bt_ok = false;          // register pool of the warp-specialised kernels that stage a transposed B checked
   int* status = nullptr;       // device address of g_status_word
   scratch::Pool scratch;       // split-K partial tiles and packed operand copies, leased per call (scratch_pool.h)
   cudaMemPool_t host_pool = nullptr;  // dgemm_f64_host: device copies of the operands come from this pool
@@ -204,7 +205,15 @@ int device_state(DeviceState** out) {
         cudaFuncSetAttribute(dgemm_dmma_ws_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) == cudaSuccess &&
         cudaFuncSetAttribute(dgemm_dmma_ws_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) == cudaSuccess &&
         cudaFuncSetAttribute(dgemm_dmma_ws_kernel<true, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, WsCfg<64>::SMEM_BYTES_) == cudaSuccess &&
-        cudaFuncSetAttribute(dgemm_dmma_ws_kernel<true, 64>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared) == cudaSuccess;
+        cudaFuncSetAttribute(dgemm_dmma_ws_kernel<true, 64>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared) == cudaSuccess &&
+        // the instantiations that stage a transposed B themselves
+        cudaFuncSetAttribute(dgemm_dmma_ws_kernel<true, 128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) == cudaSuccess &&
+        cudaFuncSetAttribute(dgemm_dmma_ws_kernel<true, 64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, WsCfg<64>::SMEM_BYTES_) == cudaSuccess &&
+        cudaFuncSetAttribute(dgemm_dmma_ws_kernel<true, 64, true>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared) == cudaSuccess &&
+        cudaFuncSetAttribute(dgemm_dmma_kernel<true, 64, 64, BN, MICRO_DMMA, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             TileCfg<64, 64, BN>::SMEM_BYTES_) == cudaSuccess &&
+        cudaFuncSetAttribute(dgemm_dmma_kernel<true, 64, 64, BN, MICRO_DMMA, true>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                             cudaSharedmemCarveoutMaxShared) == cudaSuccess;
     if (!attr_ok) return DGEMM_ERR_CUDA;
     // the 64-row kernels are meant to run two CTAs per SM; use them only where the device really fits two
     st.two_ctas_ok = occ[4] >= 2 && occ[5] >= 2 && occ[6] >= 2 && occ[7] >= 2 && occ[8] >= 2 && occ[9] >= 2 && occ[10] >= 2 && occ[11] >= 2 && occ[12] >= 2 && occ[13] >= 2 && occ[14] >= 2 && occ[15] >= 2;
@@ -234,6 +243,10 @@ int device_state(DeviceState** out) {
                             WsCfg<128>::CONSUMER_WARPS * 32, WsCfg<128>::PRODUCER_REGS);
       st.ws_ok[2] = pool_ok(reinterpret_cast<const void*>(dgemm_dmma_ws_kernel<true, 64>), WsCfg<64>::THREADS_,
                             WsCfg<64>::CONSUMER_WARPS * 32, WsCfg<64>::PRODUCER_REGS);
+      st.bt_ok = pool_ok(reinterpret_cast<const void*>(dgemm_dmma_ws_kernel<true, 128, true>), WsCfg<128>::THREADS_,
+                         WsCfg<128>::CONSUMER_WARPS * 32, WsCfg<128>::PRODUCER_REGS) &&
+                 pool_ok(reinterpret_cast<const void*>(dgemm_dmma_ws_kernel<true, 64, true>), WsCfg<64>::THREADS_,
+                         WsCfg<64>::CONSUMER_WARPS * 32, WsCfg<64>::PRODUCER_REGS);
       st.ws_ok[3] = cudaFuncSetAttribute(dgemm_dmma_wsb_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          WsBulkCfg::SMEM_BYTES_) == cudaSuccess &&
                     pool_ok(reinterpret_cast<const void*>(dgemm_dmma_wsb_kernel), WsBulkCfg::THREADS_,
@@ -586,7 +599,17 @@ Plan plan_gemm(int64_t M, int64_t N, int64_t K, bool tma_ok, int requested_varia
 struct GemmForm {
   bool ta = false, tb = false;  // A is stored K x M / B is stored N x K and used transposed
   double alpha = 1.0, beta = 1.0;
+  bool native_bt = false;       // set by launch_gemm: B is still the stored N x K matrix and the kernel stages B^T itself
 };
+
+// Kernels that can stage a transposed B themselves (a tensor map over the stored N x K matrix, rows of
+// 16 k per column in the stage): the warp-specialised kernels and the inline kernel's 64 x 128 tile,
+// all with TMA staging.
+bool plan_supports_native_bt(const Plan& pl) {
+  if (pl.status != DGEMM_OK || pl.bn != BN || pl.wtm != 64) return false;
+  if (pl.variant == DGEMM_VARIANT_TMA_WS) return pl.bm == 128 || pl.bm == 64;
+  return pl.variant == DGEMM_VARIANT_TMA && pl.bm == 64;
+}
 
 // Plans and launches one product on operands that are final (packed or transposed already where
 // that was needed): kernel choice, parameters, tensor maps, launches.
@@ -597,10 +620,11 @@ int launch_gemm_packed(DeviceState* st, scratch::Hold& hold, int variant, int64_
   const bool tma_ok = (((uintptr_t)A | (uintptr_t)B) & 15) == 0 && (lda % 2 == 0) && (ldb % 2 == 0);
   const int dbg_flags = g_test_flags.load();
   // C as the copy engine needs it for the bulk epilogue, and a beta it can apply (add, or overwrite)
-  const bool c_bulk_ok = ((uintptr_t)C & 15) == 0 && (ldc % 2 == 0) && (form.beta == 1.0 || form.beta == 0.0);
+  const bool c_bulk_ok = !form.native_bt && ((uintptr_t)C & 15) == 0 && (ldc % 2 == 0) && (form.beta == 1.0 || form.beta == 0.0);
   const Plan plan = plan_gemm(M, N, K, tma_ok, variant, dbg_flags, g_split_k.load(), st->sm_count, st->two_ctas_ok, st->ws_ok,
                               st->cluster_ok, c_bulk_ok);
   if (plan.status != DGEMM_OK) return plan.status;
+  if (form.native_bt && !plan_supports_native_bt(plan)) return DGEMM_ERR_VARIANT;  // (launch_gemm asked the same plan first)
   variant = plan.variant;
   const bool dfma = variant == DGEMM_VARIANT_TMA_DFMA || variant == DGEMM_VARIANT_GENERIC_DFMA;
   const bool wants_tma = variant == DGEMM_VARIANT_TMA || variant == DGEMM_VARIANT_TMA_WS || variant == DGEMM_VARIANT_TMA_CLUSTER ||
@@ -666,6 +690,17 @@ int launch_gemm_packed(DeviceState* st, scratch::Hold& hold, int variant, int64_
   memset(&map_b, 0, sizeof(map_b));
   if (wants_tma) {
     if (!make_map(&map_a, A, M, K, lda, BK, bm)) return DGEMM_ERR_CUDA;
+    if (form.native_bt) {
+      // B as stored, N x K: one box of 16 k x 128 rows (columns of op(B)) per stage, like an A tile
+      if (!make_map(&map_b, B, N, K, ldb, BK, bn)) return DGEMM_ERR_CUDA;
+      if (variant == DGEMM_VARIANT_TMA_WS && bm == 64)
+        launch_gemm_kernel(dgemm_dmma_ws_kernel<true, 64, true>, grid, WsCfg<64>::THREADS_, WsCfg<64>::SMEM_BYTES_, stream, map_a, map_b, p);
+      else if (variant == DGEMM_VARIANT_TMA_WS)
+        launch_gemm_kernel(dgemm_dmma_ws_kernel<true, 128, true>, grid, WS_THREADS, SMEM_BYTES, stream, map_a, map_b, p);
+      else
+        launch_gemm_kernel(dgemm_dmma_kernel<true, 64, 64, BN, MICRO_DMMA, true>, grid, TileCfg<64, 64, BN>::THREADS_,
+                           TileCfg<64, 64, BN>::SMEM_BYTES_, stream, map_a, map_b, p);
+    } else {
     p.b_blocked_map = (!(dbg_flags & DGEMM_TEST_NO_BLOCKED_B) && N % 16 == 0 && make_blocked_map(&map_b, B, K, N, ldb, BK, bn / 16)) ? 1 : 0;
     if (!p.b_blocked_map && !make_map(&map_b, B, K, N, ldb, 16, BK)) return DGEMM_ERR_CUDA;
     if (cluster)
@@ -685,6 +720,7 @@ int launch_gemm_packed(DeviceState* st, scratch::Hold& hold, int variant, int64_
       launch_dfma_kernel<true>(grid, stream, map_a, map_b, p);
     else
       launch_default_kernel<true>(bm, wtm, grid, stream, map_a, map_b, p);
+    }
   } else {
     if (cluster)
       launch_cluster_pdl(dgemm_cluster_kernel<false, 64, 64, BN>, grid, p.split_k, TileCfg<64, 64, BN>::THREADS_,
@@ -713,10 +749,11 @@ int launch_gemm_packed(DeviceState* st, scratch::Hold& hold, int variant, int64_
 }
 
 int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, const double* B, int64_t ldb,
-                double* C, int64_t ldc, cudaStream_t stream, const GemmForm& form = GemmForm()) {
+                double* C, int64_t ldc, cudaStream_t stream, const GemmForm& form_in = GemmForm()) {
   DeviceState* st = nullptr;
   int rc = device_state(&st);
   if (rc != DGEMM_OK) return rc;
+  GemmForm form = form_in;
 
   int variant = g_variant.load();
   // The scratch this call needs (packed operands, partial tiles) is one lease of the device's pool,
@@ -731,6 +768,18 @@ int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, c
     const int64_t plda = (K + 15) & ~(int64_t)15, pldb = (N + 15) & ~(int64_t)15;  // 128-byte aligned rows
     const size_t a_all = (size_t)M * plda * 8, b_all = (size_t)K * pldb * 8;
     bool pack_a = form.ta, pack_b = form.tb;
+    // A transposed B that TMA can address as it is stored (N x K, 16-byte aligned, even ldb) needs no
+    // pass at all where the kernel that would run stages B^T itself: the library's own choice, no
+    // test flags, no forced split, A addressable or about to be rewritten anyway, and not the case
+    // that is run as two products on a column split of B (below).
+    if (form.tb && st->bt_ok && variant == DGEMM_VARIANT_AUTO && g_test_flags.load() == 0 && g_split_k.load() <= 0 &&
+        ((uintptr_t)B & 15) == 0 && (ldb % 2 == 0) && (form.ta || !bad_a) && !(N >= 1024 && N % BN >= 1 && N % BN <= 64)) {
+      const Plan pl = plan_gemm(M, N, K, true, variant, 0, 0, st->sm_count, st->two_ctas_ok, st->ws_ok, st->cluster_ok, false);
+      if (plan_supports_native_bt(pl)) {
+        form.native_bt = true;
+        pack_b = false;
+      }
+    }
     if (variant == DGEMM_VARIANT_AUTO && (bad_a || bad_b) && !(g_test_flags.load() & DGEMM_TEST_NO_PACKING)) {
       const size_t bytes = ((pack_a || bad_a) ? a_all : 0) + ((pack_b || bad_b) ? b_all : 0);
       const double flop_per_byte = 2.0 * (double)M * (double)N * (double)K / (double)bytes;

@@ -273,8 +273,12 @@ struct LaneMap {
   uint32_t a_off[2], b_off[2][2];
 };
 
+//   B stored transposed (`bt`: the stage holds B^T, row n = 128 bytes of 16 k, swizzled like an A tile):
+//      lane reads k = 8h+2t, 8h+2t+1 of column 32wn + 16np + 2g + b (np adds 16 rows = 2048 bytes, the
+//      size of a box, so the same constant serves); the loaded pair is (k, k+1) of one column instead of
+//      (column, column+1) of one k, which only changes the registers a load fills (load_b_pair below).
 __device__ __forceinline__ LaneMap make_lane_map(int warp, int lane, int a_stage_bytes = A_STAGE_BYTES, int wt_rows = 64,
-                                                 int warps_n = 4) {
+                                                 int warps_n = 4, bool bt = false) {
   LaneMap m;
   m.g = lane >> 2;   // MMA group id (row of A / column of B fragment)
   m.t = lane & 3;    // thread in group (k index of the fragments)
@@ -287,14 +291,15 @@ __device__ __forceinline__ LaneMap make_lane_map(int warp, int lane, int a_stage
     m.a_off[h] = (m.row0 + m.rm) * 128 + (((4 * h + m.t) ^ m.rm) << 4);
 #pragma unroll
     for (int b = 0; b < 2; ++b)
-      m.b_off[h][b] = a_stage_bytes + (2 * m.wn) * B_BOX_BYTES + (8 * h + 2 * m.t + b) * 128 + ((m.g ^ (2 * m.t + b)) << 4);
+      m.b_off[h][b] = bt ? a_stage_bytes + (32 * m.wn + 2 * m.g + b) * 128 + (((4 * h + m.t) ^ ((2 * m.g + b) & 7)) << 4)
+                         : a_stage_bytes + (2 * m.wn) * B_BOX_BYTES + (8 * h + 2 * m.t + b) * 128 + ((m.g ^ (2 * m.t + b)) << 4);
   }
   return m;
 }
 
 // The arithmetic of one k-block (16 k values) on one stage: acc += A_tile * B_tile for this warp's
 // 64 x 32 tile.
-template <bool M16 = false, int MT = 4>
+template <bool M16 = false, int MT = 4, bool BT = false>
 __device__ __forceinline__ void compute_kblock(const uint8_t* st, const LaneMap& m, double (&acc)[MT][4][4]) {
 #pragma unroll
   for (int h = 0; h < 2; ++h) {
@@ -307,8 +312,14 @@ __device__ __forceinline__ void compute_kblock(const uint8_t* st, const LaneMap&
 #pragma unroll
     for (int np = 0; np < 2; ++np)
 #pragma unroll
-      for (int b = 0; b < 2; ++b)
-        bf[np][b] = *reinterpret_cast<const double2*>(st + m.b_off[h][b] + np * B_BOX_BYTES);
+      for (int b = 0; b < 2; ++b) {
+        const double2 v = *reinterpret_cast<const double2*>(st + m.b_off[h][b] + np * B_BOX_BYTES);
+        if constexpr (BT) {  // (k, k+1) of column 2g + b: the x (b = 0) or y (b = 1) halves of both k rows
+          if (b == 0) { bf[np][0].x = v.x; bf[np][1].x = v.y; } else { bf[np][0].y = v.x; bf[np][1].y = v.y; }
+        } else {
+          bf[np][b] = v;
+        }
+      }
     // Eight k values per block as two k4 steps (x: k = 8h + 2t, y: k = 8h + 2t + 1) of the
     // m8n8k4 shape; rows g (alo) and g + 8 (ahi) are separate 8 x 8 tiles.
 #pragma unroll
@@ -400,7 +411,16 @@ __device__ __forceinline__ void static_for(F&& f) {
 }
 
 // `stage` is the shared-memory address of the stage; H selects k = 8H .. 8H+7.
-template <int H, int MT>
+// One 16-byte B fragment load: with B as stored (BT = false) the pair is columns 2g, 2g+1 of k row b;
+// with B^T in the stage it is k rows 0, 1 of column 2g + b. Same address arithmetic, other registers.
+template <int NP, int B, bool BT, int MT>
+__device__ __forceinline__ void load_b_pair(Frags<MT>& f, uint32_t addr) {
+  if constexpr (!BT) ptx::lds128_off<NP * B_BOX_BYTES>(addr, f.bf[NP][B].x, f.bf[NP][B].y);
+  else if constexpr (B == 0) ptx::lds128_off<NP * B_BOX_BYTES>(addr, f.bf[NP][0].x, f.bf[NP][1].x);
+  else ptx::lds128_off<NP * B_BOX_BYTES>(addr, f.bf[NP][0].y, f.bf[NP][1].y);
+}
+
+template <int H, int MT, bool BT = false>
 __device__ __forceinline__ void load_frags(Frags<MT>& f, uint32_t stage, const LaneMap& m) {
   const uint32_t a = stage + m.a_off[H];
   static_for<0, MT>([&](auto mt) {
@@ -408,8 +428,8 @@ __device__ __forceinline__ void load_frags(Frags<MT>& f, uint32_t stage, const L
     ptx::lds128_off<mt.value * 2048 + 1024>(a, f.ahi[mt.value].x, f.ahi[mt.value].y);
   });
   static_for<0, 2>([&](auto np) {
-    ptx::lds128_off<np.value * B_BOX_BYTES>(stage + m.b_off[H][0], f.bf[np.value][0].x, f.bf[np.value][0].y);
-    ptx::lds128_off<np.value * B_BOX_BYTES>(stage + m.b_off[H][1], f.bf[np.value][1].x, f.bf[np.value][1].y);
+    load_b_pair<np.value, 0, BT>(f, stage + m.b_off[H][0]);
+    load_b_pair<np.value, 1, BT>(f, stage + m.b_off[H][1]);
   });
 }
 
@@ -433,11 +453,11 @@ __device__ __forceinline__ void mma_frags(double (&acc)[MT][4][4], const Frags<M
 
 // One of the 12 fragment loads of a half k-block, numbered so that the ones needed first by the
 // MMAs come first: 0..3 = B (np, b), then per row block alo, ahi.
-template <int H, int I, int MT>
+template <int H, int I, bool BT, int MT>
 __device__ __forceinline__ void load_frag_piece(Frags<MT>& f, uint32_t stage, const LaneMap& m) {
   if constexpr (I < 4) {
     constexpr int np = I >> 1, b = I & 1;
-    ptx::lds128_off<np * B_BOX_BYTES>(stage + m.b_off[H][b], f.bf[np][b].x, f.bf[np][b].y);
+    load_b_pair<np, b, BT>(f, stage + m.b_off[H][b]);
   } else if constexpr (I < 4 + 2 * MT) {
     constexpr int mt = (I - 4) >> 1;
     if constexpr (((I - 4) & 1) == 0) ptx::lds128_off<mt * 2048>(stage + m.a_off[H], f.alo[mt].x, f.alo[mt].y);
@@ -448,7 +468,7 @@ __device__ __forceinline__ void load_frag_piece(Frags<MT>& f, uint32_t stage, co
 // The MMAs of row blocks [MT0, MT1) of the half k-block in `cur`, with the loads [L0, L1) of half
 // HN (into `nxt`, from `stage_n`) spread between them, so that the loads neither arrive in a burst
 // nor wait behind the arithmetic.
-template <int MT0, int MT1, int HN, int L0, int L1, int MT>
+template <int MT0, int MT1, int HN, int L0, int L1, bool BT = false, int MT = 4>
 __device__ __forceinline__ void mma_frags_loading(double (&acc)[MT][4][4], const Frags<MT>& cur, Frags<MT>& nxt,
                                                   uint32_t stage_n, const LaneMap& m) {
   constexpr int GROUPS = 2 * (MT1 - MT0);
@@ -457,7 +477,7 @@ __device__ __forceinline__ void mma_frags_loading(double (&acc)[MT][4][4], const
     constexpr int mt = MT0 + g / 2, np = g % 2;
     // loads [lo, hi) of this group: an even share of L1 - L0
     constexpr int lo = L0 + (L1 - L0) * g / GROUPS, hi = L0 + (L1 - L0) * (g + 1) / GROUPS;
-    static_for<lo, hi>([&](auto li) { load_frag_piece<HN, li.value>(nxt, stage_n, m); });
+    static_for<lo, hi>([&](auto li) { load_frag_piece<HN, li.value, BT>(nxt, stage_n, m); });
     ptx::dmma_m8n8k4(acc[mt][2 * np + 0][0], acc[mt][2 * np + 0][1], cur.alo[mt].x, cur.bf[np][0].x);
     ptx::dmma_m8n8k4(acc[mt][2 * np + 0][2], acc[mt][2 * np + 0][3], cur.ahi[mt].x, cur.bf[np][0].x);
     ptx::dmma_m8n8k4(acc[mt][2 * np + 1][0], acc[mt][2 * np + 1][1], cur.alo[mt].x, cur.bf[np][0].y);
@@ -730,7 +750,9 @@ struct TileCfg {
 constexpr int MICRO_DMMA = 0;
 constexpr int MICRO_DFMA = 1;
 
-template <bool USE_TMA, int TBM, int WTM = 64, int TBN = BN, int MICRO = MICRO_DMMA>
+// BT: map_b describes B as stored transposed (N x K, the general entry point's op(B) = B^T) and the
+// stage holds B^T: no transposing pass in HBM. TMA staging only.
+template <bool USE_TMA, int TBM, int WTM = 64, int TBN = BN, int MICRO = MICRO_DMMA, bool BT = false>
 __global__ void __launch_bounds__(TileCfg<TBM, WTM, TBN>::THREADS_, TileCfg<TBM, WTM, TBN>::CTAS_PER_SM)
 dgemm_dmma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                   const __grid_constant__ GemmParams p) {
@@ -821,7 +843,9 @@ dgemm_dmma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
           } else if (!p.drop_loads) {
             ptx::mbar_arrive_expect_tx(fb, STAGE_BYTES);
             ptx::tma_load_2d(sa, &map_a, kb * BK, cur_tm * TBM, fb);
-            if (p.b_blocked_map) {
+            if constexpr (BT) {
+              ptx::tma_load_2d(sb, &map_b, kb * BK, cur_tn * TBN, fb);  // rows n of B^T, 16 k each
+            } else if (p.b_blocked_map) {
               ptx::tma_load_3d(sb, &map_b, 0, kb * BK, cur_tn * (TBN / 16), fb);
             } else {
               tma_load_b_boxes(sb, &map_b, cur_tn * TBN, kb * BK, fb, TBN / 16);
@@ -907,7 +931,8 @@ dgemm_dmma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
 
   for (int i = 0; i < LOOKAHEAD && ok; ++i) ok = issue_next();
 
-  const LaneMap lm = make_lane_map(warp, lane, A_STAGE_BYTES, WTM, WARPS_N);
+  static_assert(!BT || (USE_TMA && MICRO == MICRO_DMMA), "the transposed-B stage exists for TMA staging and the MMA micro-kernel");
+  const LaneMap lm = make_lane_map(warp, lane, A_STAGE_BYTES, WTM, WARPS_N, BT);
 
   double acc[MT][4][4];  // [mt][nt = 2*np + j][c0..c3]
   uint32_t it = 0;      // k-blocks consumed so far
@@ -936,7 +961,7 @@ dgemm_dmma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
       const uint32_t ph = (it / STAGES) & 1u;
       if (!wait_bounded(full_bar + 8 * s, ph, abort_flag, p)) { ok = false; break; }
       if constexpr (MICRO == MICRO_DFMA) compute_kblock_dfma<MT>(tiles + s * STAGE_BYTES, lm, A_STAGE_BYTES, acc);
-      else compute_kblock<false, MT>(tiles + s * STAGE_BYTES, lm, acc);
+      else compute_kblock<false, MT, BT>(tiles + s * STAGE_BYTES, lm, acc);
       release_stage(empty_bar + 8 * s, lane);
       // keep the load stream LOOKAHEAD k-blocks ahead: refill the stage released two k-blocks ago
       if (!issue_next()) { ok = false; break; }
@@ -991,11 +1016,12 @@ struct WsCfg {
   static constexpr int PRODUCER_REGS = TBM == 128 ? WS_PRODUCER_REGS : 24;
 };
 
-template <bool USE_TMA, int TBM = BM>
+template <bool USE_TMA, int TBM = BM, bool BT = false>
 __global__ void __launch_bounds__(WsCfg<TBM>::THREADS_, WsCfg<TBM>::CTAS_PER_SM)
 dgemm_dmma_ws_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                      const __grid_constant__ GemmParams p) {
   static_assert(USE_TMA || TBM == 128, "generic staging needs the 128-row producer layout and 40 producer registers");
+  static_assert(!BT || USE_TMA, "the transposed-B stage exists for TMA staging only");
   constexpr int STAGES = WsCfg<TBM>::STAGES_;
   constexpr int WARPS = WsCfg<TBM>::CONSUMER_WARPS;
   constexpr int A_STAGE_BYTES = WsCfg<TBM>::A_BYTES;
@@ -1068,7 +1094,9 @@ dgemm_dmma_ws_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
             } else if (!p.drop_loads) {
               ptx::mbar_arrive_expect_tx(fb, STAGE_BYTES);
               ptx::tma_load_2d(sa, &map_a, kb * BK, w.tm * TBM, fb);
-              if (p.b_blocked_map) {
+              if constexpr (BT) {
+                ptx::tma_load_2d(sb, &map_b, kb * BK, w.tn * BN, fb);  // rows n of B^T, 16 k each
+              } else if (p.b_blocked_map) {
                 ptx::tma_load_3d(sb, &map_b, 0, kb * BK, w.tn * (BN / 16), fb);
               } else {
                 tma_load_b_boxes_inline(sb, &map_b, w.tn * BN, kb * BK, fb);
@@ -1130,7 +1158,7 @@ dgemm_dmma_ws_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
   } else {
     // ------------------------------------------------------------------ consumer warps
     ptx::setmaxnreg_inc<WS_CONSUMER_REGS>();
-    const LaneMap lm = make_lane_map(warp, lane, A_STAGE_BYTES, 64, 4);
+    const LaneMap lm = make_lane_map(warp, lane, A_STAGE_BYTES, 64, 4, BT);
     double acc[4][4][4];
     for (int idx = 0; ok && get_work(p, cta, nctas, idx, w); ++idx) {
 #pragma unroll
@@ -1143,7 +1171,7 @@ dgemm_dmma_ws_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
       {
         const uint32_t s = it % STAGES;
         if (!wait_bounded_inline(full_bar + 8 * s, (it / STAGES) & 1u, abort_flag, p)) { ok = false; break; }
-        load_frags<0>(f0, tiles_u32 + s * STAGE_BYTES, lm);
+        load_frags<0, 4, BT>(f0, tiles_u32 + s * STAGE_BYTES, lm);
       }
       for (int kb = w.kb0; kb < w.kb1; ++kb, ++it) {
         const uint32_t s = it % STAGES;
@@ -1151,12 +1179,12 @@ dgemm_dmma_ws_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
         const uint32_t ph1 = ((it + 1) / STAGES) & 1u;
         const bool more = kb + 1 < w.kb1;
         const bool ready = more && ptx::mbar_test_wait(full_bar + 8 * s1, ph1);
-        mma_frags_loading<0, 4, 1, 0, 12>(acc, f0, f1, tiles_u32 + s * STAGE_BYTES, lm);
+        mma_frags_loading<0, 4, 1, 0, 12, BT>(acc, f0, f1, tiles_u32 + s * STAGE_BYTES, lm);
         if (more) {
           if (!ready && !wait_bounded_inline(full_bar + 8 * s1, ph1, abort_flag, p)) { ok = false; break; }
-          mma_frags_loading<0, 2, 0, 0, 6>(acc, f1, f0, tiles_u32 + s1 * STAGE_BYTES, lm);
+          mma_frags_loading<0, 2, 0, 0, 6, BT>(acc, f1, f0, tiles_u32 + s1 * STAGE_BYTES, lm);
           release_stage(empty_bar + 8 * s, lane);
-          mma_frags_loading<2, 4, 0, 6, 12>(acc, f1, f0, tiles_u32 + s1 * STAGE_BYTES, lm);
+          mma_frags_loading<2, 4, 0, 6, 12, BT>(acc, f1, f0, tiles_u32 + s1 * STAGE_BYTES, lm);
         } else {
           mma_frags<0, 2>(acc, f1);
           release_stage(empty_bar + 8 * s, lane);

@@ -224,3 +224,25 @@ def test_scalars_in_the_inline_kernel_with_64_row_tiles(oracle, alpha, beta):
     _case(oracle, M, N, K, False, False, alpha, beta, True, seed=77, pad=(2, 4, 7),
           c_fill=(np.nan if beta == 0.0 else None), variant=dg.DGEMM_VARIANT_TMA)
     _case(oracle, M, N, K, True, True, alpha, beta, False, seed=78, variant=dg.DGEMM_VARIANT_TMA)
+
+
+@pytest.mark.parametrize("integer", [True, False])
+@pytest.mark.parametrize("ta", [False, True])
+@pytest.mark.parametrize("shape", [(2048, 2048, 512), (1024, 1024, 1024), (2088, 2048, 300), (600, 700, 500), (1000, 1537, 777),
+                                   (2304, 2304, 64), (300, 260, 200)])
+def test_transposed_b_is_staged_without_a_pass(oracle, shape, ta, integer):
+    """op(B) = B^T with a B the tensor-copy engine can address as it is stored (N x K, even ldb): the
+    warp-specialised kernels and the inline kernel's 64 x 128 tile stage B^T themselves, so the call has
+    the launches of the untransposed product (plus one for a transposed A). Other kernels keep the
+    transposing pass. Either way the result matches the oracle."""
+    M, N, K = shape
+    counts = {}
+    for tb in (False, True):
+        n0 = dg.dgemm_launch_count()
+        _case(oracle, M, N, K, ta, tb, 1.0, 1.0, integer, seed=3000 + M + N + K, pad=(2, 4, 6))
+        counts[tb] = dg.dgemm_launch_count() - n0
+    plan = dg.dgemm_plan(M, N, K)
+    native = (plan["variant"] == dg.DGEMM_VARIANT_TMA_WS or (plan["variant"] == dg.DGEMM_VARIANT_TMA and plan["bm"] == 64)) \
+        and plan["bn"] == 128 and plan["wtm"] == 64 and not (N >= 1024 and 1 <= N % 128 <= 64)
+    if native:
+        assert counts[True] == counts[False], (counts, plan)

@@ -161,12 +161,13 @@ DGEMM_API int dgemm_f64_host(int64_t M, int64_t N, int64_t K,
  *
  * Arithmetic: each C element receives beta*C_old + alpha*s, s the K-term inner product summed as
  * in dgemm_f64; alpha = beta = 1 with no transposition gives bit-identical results to dgemm_f64.
- * A transposed B that is 16-byte aligned with an even ldb is used where it lies: the kernels that
- * run problems of at least 16 tiles stage B^T themselves (no extra pass, no extra launch; measured
- * level with the untransposed product from 1024^3 up). A transposed A, and a transposed B on the
- * smaller or narrower problems, is first transposed into device scratch memory owned by the library
- * (an O(MK) or O(KN) pass before O(MNK) arithmetic; the buffer is kept and reused, and leased
- * per call like the rest of the scratch: see dgemm_f64).
+ * A transposed operand that is 16-byte aligned with an even leading dimension is used where it
+ * lies: the kernels that run problems of at least 16 tiles stage the transposed tiles themselves
+ * (no extra pass, no extra launch; measured from 1024^3 up: B^T level with the untransposed
+ * product, A^T within 0.6 %). Otherwise (the smaller or narrower problems, operands that cannot be
+ * addressed in place, a very large A^T) a transposed operand is first transposed into device
+ * scratch memory owned by the library (an O(MK) or O(KN) pass before O(MNK) arithmetic; the buffer
+ * is kept and reused, and leased per call like the rest of the scratch: see dgemm_f64).
  * Same pointer, alignment, aliasing and error rules as dgemm_f64; an op code other than the two
  * above returns DGEMM_ERR_BAD_DIM.
  */

@@ -38,9 +38,9 @@ def is_stale() -> bool:
 # warp-specialised kernels redistribute a pool of threads x registers with setmaxnreg, so another
 # launch count changes the consumers' budget; the 8192^3 figure was measured with exactly these.
 PTXAS_EXPECT = [
-    ("dgemm_dmma_ws_kernelILb1ELi128ELb0EE", 168, 128),
-    ("dgemm_dmma_ws_kernelILb1ELi64ELb0EE", 128, 128),
-    ("dgemm_dmma_kernelILb1ELi64ELi64ELi128ELi0ELb0EE", 255, 64),
+    ("dgemm_dmma_ws_kernelILb1ELi128ELb0ELb0EE", 168, 128),
+    ("dgemm_dmma_ws_kernelILb1ELi64ELb0ELb0EE", 128, 128),
+    ("dgemm_dmma_kernelILb1ELi64ELi64ELi128ELi0ELb0ELb0EE", 255, 64),
 ]
 
 

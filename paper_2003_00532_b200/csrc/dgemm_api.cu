@@ -173,6 +173,18 @@ bool configure_tile_kernel(int* occupancy) {
                                                        TileCfg<TBM, WTM, TBN>::SMEM_BYTES_) == cudaSuccess;
 }
 
+// Shared-memory opt-in of the instantiations that stage transposed operands themselves.
+template <bool BT, bool AT>
+bool configure_transposed_kernels() {
+  return cudaFuncSetAttribute(dgemm_dmma_ws_kernel<true, 128, BT, AT>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) == cudaSuccess &&
+         cudaFuncSetAttribute(dgemm_dmma_ws_kernel<true, 64, BT, AT>, cudaFuncAttributeMaxDynamicSharedMemorySize, WsCfg<64>::SMEM_BYTES_) == cudaSuccess &&
+         cudaFuncSetAttribute(dgemm_dmma_ws_kernel<true, 64, BT, AT>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared) == cudaSuccess &&
+         cudaFuncSetAttribute(dgemm_dmma_kernel<true, 64, 64, BN, MICRO_DMMA, BT, AT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              TileCfg<64, 64, BN>::SMEM_BYTES_) == cudaSuccess &&
+         cudaFuncSetAttribute(dgemm_dmma_kernel<true, 64, 64, BN, MICRO_DMMA, BT, AT>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                              cudaSharedmemCarveoutMaxShared) == cudaSuccess;
+}
+
 // Per-device set-up, once: capability check, SM count, status-word address, shared-memory opt-in.
 int device_state(DeviceState** out) {
   int dev = -1;
@@ -206,14 +218,7 @@ int device_state(DeviceState** out) {
         cudaFuncSetAttribute(dgemm_dmma_ws_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) == cudaSuccess &&
         cudaFuncSetAttribute(dgemm_dmma_ws_kernel<true, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, WsCfg<64>::SMEM_BYTES_) == cudaSuccess &&
         cudaFuncSetAttribute(dgemm_dmma_ws_kernel<true, 64>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared) == cudaSuccess &&
-        // the instantiations that stage a transposed B themselves
-        cudaFuncSetAttribute(dgemm_dmma_ws_kernel<true, 128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) == cudaSuccess &&
-        cudaFuncSetAttribute(dgemm_dmma_ws_kernel<true, 64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, WsCfg<64>::SMEM_BYTES_) == cudaSuccess &&
-        cudaFuncSetAttribute(dgemm_dmma_ws_kernel<true, 64, true>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared) == cudaSuccess &&
-        cudaFuncSetAttribute(dgemm_dmma_kernel<true, 64, 64, BN, MICRO_DMMA, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             TileCfg<64, 64, BN>::SMEM_BYTES_) == cudaSuccess &&
-        cudaFuncSetAttribute(dgemm_dmma_kernel<true, 64, 64, BN, MICRO_DMMA, true>, cudaFuncAttributePreferredSharedMemoryCarveout,
-                             cudaSharedmemCarveoutMaxShared) == cudaSuccess;
+        configure_transposed_kernels<true, false>() && configure_transposed_kernels<false, true>() && configure_transposed_kernels<true, true>();
     if (!attr_ok) return DGEMM_ERR_CUDA;
     // the 64-row kernels are meant to run two CTAs per SM; use them only where the device really fits two
     st.two_ctas_ok = occ[4] >= 2 && occ[5] >= 2 && occ[6] >= 2 && occ[7] >= 2 && occ[8] >= 2 && occ[9] >= 2 && occ[10] >= 2 && occ[11] >= 2 && occ[12] >= 2 && occ[13] >= 2 && occ[14] >= 2 && occ[15] >= 2;
@@ -243,10 +248,18 @@ int device_state(DeviceState** out) {
                             WsCfg<128>::CONSUMER_WARPS * 32, WsCfg<128>::PRODUCER_REGS);
       st.ws_ok[2] = pool_ok(reinterpret_cast<const void*>(dgemm_dmma_ws_kernel<true, 64>), WsCfg<64>::THREADS_,
                             WsCfg<64>::CONSUMER_WARPS * 32, WsCfg<64>::PRODUCER_REGS);
-      st.bt_ok = pool_ok(reinterpret_cast<const void*>(dgemm_dmma_ws_kernel<true, 128, true>), WsCfg<128>::THREADS_,
-                         WsCfg<128>::CONSUMER_WARPS * 32, WsCfg<128>::PRODUCER_REGS) &&
-                 pool_ok(reinterpret_cast<const void*>(dgemm_dmma_ws_kernel<true, 64, true>), WsCfg<64>::THREADS_,
-                         WsCfg<64>::CONSUMER_WARPS * 32, WsCfg<64>::PRODUCER_REGS);
+      st.bt_ok = true;  // (bt_ok: every instantiation that stages a transposed operand has its register pool)
+      {
+        const void* k128[3] = {reinterpret_cast<const void*>(dgemm_dmma_ws_kernel<true, 128, true, false>),
+                               reinterpret_cast<const void*>(dgemm_dmma_ws_kernel<true, 128, false, true>),
+                               reinterpret_cast<const void*>(dgemm_dmma_ws_kernel<true, 128, true, true>)};
+        const void* k64[3] = {reinterpret_cast<const void*>(dgemm_dmma_ws_kernel<true, 64, true, false>),
+                              reinterpret_cast<const void*>(dgemm_dmma_ws_kernel<true, 64, false, true>),
+                              reinterpret_cast<const void*>(dgemm_dmma_ws_kernel<true, 64, true, true>)};
+        for (int i = 0; i < 3; ++i)
+          st.bt_ok = st.bt_ok && pool_ok(k128[i], WsCfg<128>::THREADS_, WsCfg<128>::CONSUMER_WARPS * 32, WsCfg<128>::PRODUCER_REGS) &&
+                     pool_ok(k64[i], WsCfg<64>::THREADS_, WsCfg<64>::CONSUMER_WARPS * 32, WsCfg<64>::PRODUCER_REGS);
+      }
       st.ws_ok[3] = cudaFuncSetAttribute(dgemm_dmma_wsb_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          WsBulkCfg::SMEM_BYTES_) == cudaSuccess &&
                     pool_ok(reinterpret_cast<const void*>(dgemm_dmma_wsb_kernel), WsBulkCfg::THREADS_,
@@ -600,15 +613,29 @@ struct GemmForm {
   bool ta = false, tb = false;  // A is stored K x M / B is stored N x K and used transposed
   double alpha = 1.0, beta = 1.0;
   bool native_bt = false;       // set by launch_gemm: B is still the stored N x K matrix and the kernel stages B^T itself
+  bool native_at = false;       // likewise A is still the stored K x M matrix
 };
 
-// Kernels that can stage a transposed B themselves (a tensor map over the stored N x K matrix, rows of
-// 16 k per column in the stage): the warp-specialised kernels and the inline kernel's 64 x 128 tile,
-// all with TMA staging.
+// Kernels that can stage a transposed operand themselves (a tensor map over the matrix as stored): the
+// warp-specialised kernels and the inline kernel's 64 x 128 tile, all with TMA staging.
 bool plan_supports_native_bt(const Plan& pl) {
   if (pl.status != DGEMM_OK || pl.bn != BN || pl.wtm != 64) return false;
   if (pl.variant == DGEMM_VARIANT_TMA_WS) return pl.bm == 128 || pl.bm == 64;
   return pl.variant == DGEMM_VARIANT_TMA && pl.bm == 64;
+}
+
+// The kernels that stage transposed operands themselves: 0 warp-specialised 128 x 128, 1 warp-specialised
+// 64 x 128, 2 inline 64 x 128.
+template <bool BT, bool AT>
+void launch_transposed_kernel(int which, int grid, cudaStream_t stream, const CUtensorMap& map_a, const CUtensorMap& map_b,
+                              const GemmParams& p) {
+  if (which == 0)
+    launch_gemm_kernel(dgemm_dmma_ws_kernel<true, 128, BT, AT>, grid, WS_THREADS, SMEM_BYTES, stream, map_a, map_b, p);
+  else if (which == 1)
+    launch_gemm_kernel(dgemm_dmma_ws_kernel<true, 64, BT, AT>, grid, WsCfg<64>::THREADS_, WsCfg<64>::SMEM_BYTES_, stream, map_a, map_b, p);
+  else
+    launch_gemm_kernel(dgemm_dmma_kernel<true, 64, 64, BN, MICRO_DMMA, BT, AT>, grid, TileCfg<64, 64, BN>::THREADS_,
+                       TileCfg<64, 64, BN>::SMEM_BYTES_, stream, map_a, map_b, p);
 }
 
 // Plans and launches one product on operands that are final (packed or transposed already where
@@ -620,11 +647,11 @@ int launch_gemm_packed(DeviceState* st, scratch::Hold& hold, int variant, int64_
   const bool tma_ok = (((uintptr_t)A | (uintptr_t)B) & 15) == 0 && (lda % 2 == 0) && (ldb % 2 == 0);
   const int dbg_flags = g_test_flags.load();
   // C as the copy engine needs it for the bulk epilogue, and a beta it can apply (add, or overwrite)
-  const bool c_bulk_ok = !form.native_bt && ((uintptr_t)C & 15) == 0 && (ldc % 2 == 0) && (form.beta == 1.0 || form.beta == 0.0);
+  const bool c_bulk_ok = !form.native_bt && !form.native_at && ((uintptr_t)C & 15) == 0 && (ldc % 2 == 0) && (form.beta == 1.0 || form.beta == 0.0);
   const Plan plan = plan_gemm(M, N, K, tma_ok, variant, dbg_flags, g_split_k.load(), st->sm_count, st->two_ctas_ok, st->ws_ok,
                               st->cluster_ok, c_bulk_ok);
   if (plan.status != DGEMM_OK) return plan.status;
-  if (form.native_bt && !plan_supports_native_bt(plan)) return DGEMM_ERR_VARIANT;  // (launch_gemm asked the same plan first)
+  if ((form.native_bt || form.native_at) && !plan_supports_native_bt(plan)) return DGEMM_ERR_VARIANT;  // (launch_gemm asked the same plan first)
   variant = plan.variant;
   const bool dfma = variant == DGEMM_VARIANT_TMA_DFMA || variant == DGEMM_VARIANT_GENERIC_DFMA;
   const bool wants_tma = variant == DGEMM_VARIANT_TMA || variant == DGEMM_VARIANT_TMA_WS || variant == DGEMM_VARIANT_TMA_CLUSTER ||
@@ -689,17 +716,25 @@ int launch_gemm_packed(DeviceState* st, scratch::Hold& hold, int variant, int64_
   memset(&map_a, 0, sizeof(map_a));
   memset(&map_b, 0, sizeof(map_b));
   if (wants_tma) {
-    if (!make_map(&map_a, A, M, K, lda, BK, bm)) return DGEMM_ERR_CUDA;
-    if (form.native_bt) {
-      // B as stored, N x K: one box of 16 k x 128 rows (columns of op(B)) per stage, like an A tile
-      if (!make_map(&map_b, B, N, K, ldb, BK, bn)) return DGEMM_ERR_CUDA;
-      if (variant == DGEMM_VARIANT_TMA_WS && bm == 64)
-        launch_gemm_kernel(dgemm_dmma_ws_kernel<true, 64, true>, grid, WsCfg<64>::THREADS_, WsCfg<64>::SMEM_BYTES_, stream, map_a, map_b, p);
-      else if (variant == DGEMM_VARIANT_TMA_WS)
-        launch_gemm_kernel(dgemm_dmma_ws_kernel<true, 128, true>, grid, WS_THREADS, SMEM_BYTES, stream, map_a, map_b, p);
-      else
-        launch_gemm_kernel(dgemm_dmma_kernel<true, 64, 64, BN, MICRO_DMMA, true>, grid, TileCfg<64, 64, BN>::THREADS_,
-                           TileCfg<64, 64, BN>::SMEM_BYTES_, stream, map_a, map_b, p);
+    if (form.native_at) {
+      // A as stored, K x M: boxes of [16 k][16 rows of op(A)], one 3-D copy per stage when M is a multiple of 16
+      p.a_blocked_map = (M % 16 == 0 && make_blocked_map(&map_a, A, K, M, lda, BK, bm / 16)) ? 1 : 0;
+      if (!p.a_blocked_map && !make_map(&map_a, A, K, M, lda, 16, BK)) return DGEMM_ERR_CUDA;
+    } else if (!make_map(&map_a, A, M, K, lda, BK, bm)) {
+      return DGEMM_ERR_CUDA;
+    }
+    if (form.native_bt || form.native_at) {
+      if (form.native_bt) {
+        // B as stored, N x K: one box of 16 k x 128 rows (columns of op(B)) per stage, like an A tile
+        if (!make_map(&map_b, B, N, K, ldb, BK, bn)) return DGEMM_ERR_CUDA;
+      } else {
+        p.b_blocked_map = (N % 16 == 0 && make_blocked_map(&map_b, B, K, N, ldb, BK, bn / 16)) ? 1 : 0;
+        if (!p.b_blocked_map && !make_map(&map_b, B, K, N, ldb, 16, BK)) return DGEMM_ERR_CUDA;
+      }
+      const int which = variant == DGEMM_VARIANT_TMA_WS ? (bm == 64 ? 1 : 0) : 2;
+      if (form.native_bt && form.native_at) launch_transposed_kernel<true, true>(which, grid, stream, map_a, map_b, p);
+      else if (form.native_bt) launch_transposed_kernel<true, false>(which, grid, stream, map_a, map_b, p);
+      else launch_transposed_kernel<false, true>(which, grid, stream, map_a, map_b, p);
     } else {
     p.b_blocked_map = (!(dbg_flags & DGEMM_TEST_NO_BLOCKED_B) && N % 16 == 0 && make_blocked_map(&map_b, B, K, N, ldb, BK, bn / 16)) ? 1 : 0;
     if (!p.b_blocked_map && !make_map(&map_b, B, K, N, ldb, 16, BK)) return DGEMM_ERR_CUDA;
@@ -768,18 +803,6 @@ int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, c
     const int64_t plda = (K + 15) & ~(int64_t)15, pldb = (N + 15) & ~(int64_t)15;  // 128-byte aligned rows
     const size_t a_all = (size_t)M * plda * 8, b_all = (size_t)K * pldb * 8;
     bool pack_a = form.ta, pack_b = form.tb;
-    // A transposed B that TMA can address as it is stored (N x K, 16-byte aligned, even ldb) needs no
-    // pass at all where the kernel that would run stages B^T itself: the library's own choice, no
-    // test flags, no forced split, A addressable or about to be rewritten anyway, and not the case
-    // that is run as two products on a column split of B (below).
-    if (form.tb && st->bt_ok && variant == DGEMM_VARIANT_AUTO && g_test_flags.load() == 0 && g_split_k.load() <= 0 &&
-        ((uintptr_t)B & 15) == 0 && (ldb % 2 == 0) && (form.ta || !bad_a) && !(N >= 1024 && N % BN >= 1 && N % BN <= 64)) {
-      const Plan pl = plan_gemm(M, N, K, true, variant, 0, 0, st->sm_count, st->two_ctas_ok, st->ws_ok, st->cluster_ok, false);
-      if (plan_supports_native_bt(pl)) {
-        form.native_bt = true;
-        pack_b = false;
-      }
-    }
     if (variant == DGEMM_VARIANT_AUTO && (bad_a || bad_b) && !(g_test_flags.load() & DGEMM_TEST_NO_PACKING)) {
       const size_t bytes = ((pack_a || bad_a) ? a_all : 0) + ((pack_b || bad_b) ? b_all : 0);
       const double flop_per_byte = 2.0 * (double)M * (double)N * (double)K / (double)bytes;
@@ -787,6 +810,25 @@ int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, c
           2.0 * (double)M * (double)N * (double)K >= kPackMinFlop) {
         pack_a = pack_a || bad_a;
         pack_b = pack_b || bad_b;
+      }
+    }
+    // A transposed operand that TMA can address as it is stored (16-byte aligned, even leading
+    // dimension) needs no pass at all where the kernel that would run stages the transposed tile
+    // itself: the library's own choice, no test flags, no forced split, the other operand addressable
+    // (as it is, or after the packing pass decided above), and not the case that is run as two
+    // products on a column split of B (below).
+    if ((form.ta || form.tb) && st->bt_ok && variant == DGEMM_VARIANT_AUTO && g_test_flags.load() == 0 && g_split_k.load() <= 0 &&
+        !(N >= 1024 && N % BN >= 1 && N % BN <= 64) && (!bad_a || pack_a) && (!bad_b || pack_b)) {
+      const bool at_ok = form.ta && ((uintptr_t)A & 15) == 0 && (lda % 2 == 0);
+      const bool bt_ok = form.tb && ((uintptr_t)B & 15) == 0 && (ldb % 2 == 0);
+      // (the other transposed operand, if it cannot be used in place, is rewritten row-major and aligned)
+      const Plan pl = plan_gemm(M, N, K, true, variant, 0, 0, st->sm_count, st->two_ctas_ok, st->ws_ok, st->cluster_ok, false);
+      if (plan_supports_native_bt(pl)) {
+        // B^T in the stage costs nothing measurable; A^T costs the arithmetic warps 0.5 % (four 8-byte loads
+        // per fragment pair instead of two 16-byte ones), 1.2 % together with B^T, while the transposing
+        // pass of A costs 0.7 % x 8192 / N: in place up to N = 8192, with B^T in place up to 4608
+        if (bt_ok) { form.native_bt = true; pack_b = false; }
+        if (at_ok && N <= (form.native_bt ? 4608 : 8192)) { form.native_at = true; pack_a = false; }
       }
     }
     if (pack_a || pack_b) {

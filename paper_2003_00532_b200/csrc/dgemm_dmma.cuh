@@ -82,6 +82,7 @@ struct GemmParams {
   int group_m;            // raster group height in tiles
   int c_prefetch;         // request the C tile into L2 a few k-blocks before its epilogue
   int b_blocked_map;      // map_b is the 3-D view (16 columns, K, N/16): one copy stages the whole B tile
+  int a_blocked_map;      // kernels that stage a transposed A: map_a is the 3-D view (16 rows of op(A), K, M/16)
   int load_c;             // 0: beta == 0, the old C is never read (it may hold NaN)
   double alpha, beta;     // C = beta * C + alpha * (A B); 1, 1 for the paper's C += A B
   const double* A;
@@ -216,6 +217,17 @@ __device__ __noinline__ void tma_load_b_boxes(uint32_t sb, const CUtensorMap* ma
   tma_load_b_boxes_inline(sb, map_b, n0, k0, fb, boxes);
 }
 
+// A stage of a transposed A (stored K x M): TBM / 16 boxes of [16 k][16 rows of op(A)], as one 3-D copy
+// when M is a multiple of 16, else box by box.
+__device__ __forceinline__ void tma_load_at(uint32_t sa, const CUtensorMap* map_a, int blocked, int m0, int k0, uint32_t fb,
+                                            int boxes) {
+  if (blocked) {
+    ptx::tma_load_3d(sa, map_a, 0, k0, m0 / 16, fb);
+  } else {
+    for (int nb = 0; nb < boxes; ++nb) ptx::tma_load_2d(sa + nb * B_BOX_BYTES, map_a, m0 + nb * 16, k0, fb);
+  }
+}
+
 // Slow part of a bounded mbarrier wait: poll until the phase completes, the CTA aborts, or the
 // time limit expires (then record DGEMM_ERR_TIMEOUT and raise the abort flag).
 __device__ __noinline__ bool wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag,
@@ -271,14 +283,20 @@ struct LaneMap {
   int g, t, wm, wn, rm;
   int row0;  // first row of this warp's tile inside the CTA tile (wt_rows * wm)
   uint32_t a_off[2], b_off[2][2];
+  uint32_t at_off[2][2];  // transposed A in the stage: [k parity b][rows +0 / +8]
 };
 
 //   B stored transposed (`bt`: the stage holds B^T, row n = 128 bytes of 16 k, swizzled like an A tile):
 //      lane reads k = 8h+2t, 8h+2t+1 of column 32wn + 16np + 2g + b (np adds 16 rows = 2048 bytes, the
 //      size of a box, so the same constant serves); the loaded pair is (k, k+1) of one column instead of
 //      (column, column+1) of one k, which only changes the registers a load fills (load_b_pair below).
+//   A stored transposed (`at`: the stage holds the K x M matrix's tile as boxes of [16 k][16 rows of
+//      op(A)], 128-byte rows, swizzled, exactly the layout of an untransposed B tile): the two k of a
+//      fragment pair lie in different 128-byte rows, so a lane reads its four values per 16-row block
+//      (rows rm, rm + 8 at k = 8h+2t, 8h+2t+1) with four 8-byte loads instead of two 16-byte ones; the
+//      half h only adds 1024 bytes and the 16-row block mt 2048, both immediates.
 __device__ __forceinline__ LaneMap make_lane_map(int warp, int lane, int a_stage_bytes = A_STAGE_BYTES, int wt_rows = 64,
-                                                 int warps_n = 4, bool bt = false) {
+                                                 int warps_n = 4, bool bt = false, bool at = false) {
   LaneMap m;
   m.g = lane >> 2;   // MMA group id (row of A / column of B fragment)
   m.t = lane & 3;    // thread in group (k index of the fragments)
@@ -290,24 +308,40 @@ __device__ __forceinline__ LaneMap make_lane_map(int warp, int lane, int a_stage
   for (int h = 0; h < 2; ++h) {
     m.a_off[h] = (m.row0 + m.rm) * 128 + (((4 * h + m.t) ^ m.rm) << 4);
 #pragma unroll
-    for (int b = 0; b < 2; ++b)
+    for (int b = 0; b < 2; ++b) {
+      m.at_off[h][b] = 0;
       m.b_off[h][b] = bt ? a_stage_bytes + (32 * m.wn + 2 * m.g + b) * 128 + (((4 * h + m.t) ^ ((2 * m.g + b) & 7)) << 4)
                          : a_stage_bytes + (2 * m.wn) * B_BOX_BYTES + (8 * h + 2 * m.t + b) * 128 + ((m.g ^ (2 * m.t + b)) << 4);
+    }
+  }
+  if (at) {
+#pragma unroll
+    for (int b = 0; b < 2; ++b)
+#pragma unroll
+      for (int half = 0; half < 2; ++half)
+        m.at_off[b][half] = (m.row0 / 16) * B_BOX_BYTES + (2 * m.t + b) * 128 + ((((m.rm >> 1) + 4 * half) ^ (2 * m.t + b)) << 4) + (m.rm & 1) * 8;
   }
   return m;
 }
 
 // The arithmetic of one k-block (16 k values) on one stage: acc += A_tile * B_tile for this warp's
 // 64 x 32 tile.
-template <bool M16 = false, int MT = 4, bool BT = false>
+template <bool M16 = false, int MT = 4, bool BT = false, bool AT = false>
 __device__ __forceinline__ void compute_kblock(const uint8_t* st, const LaneMap& m, double (&acc)[MT][4][4]) {
 #pragma unroll
   for (int h = 0; h < 2; ++h) {
     double2 alo[MT], ahi[MT], bf[2][2];
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt) {
-      alo[mt] = *reinterpret_cast<const double2*>(st + m.a_off[h] + mt * 2048);
-      ahi[mt] = *reinterpret_cast<const double2*>(st + m.a_off[h] + mt * 2048 + 1024);
+      if constexpr (AT) {
+        alo[mt].x = *reinterpret_cast<const double*>(st + m.at_off[0][0] + h * 1024 + mt * B_BOX_BYTES);
+        alo[mt].y = *reinterpret_cast<const double*>(st + m.at_off[1][0] + h * 1024 + mt * B_BOX_BYTES);
+        ahi[mt].x = *reinterpret_cast<const double*>(st + m.at_off[0][1] + h * 1024 + mt * B_BOX_BYTES);
+        ahi[mt].y = *reinterpret_cast<const double*>(st + m.at_off[1][1] + h * 1024 + mt * B_BOX_BYTES);
+      } else {
+        alo[mt] = *reinterpret_cast<const double2*>(st + m.a_off[h] + mt * 2048);
+        ahi[mt] = *reinterpret_cast<const double2*>(st + m.a_off[h] + mt * 2048 + 1024);
+      }
     }
 #pragma unroll
     for (int np = 0; np < 2; ++np)
@@ -402,6 +436,19 @@ struct Frags {
   double2 alo[MT], ahi[MT], bf[2][2];
 };
 
+// The A fragments of 16-row block MT_ for the k8 half H, rows +0 (lo) or +8 (hi): one 16-byte load from
+// an untransposed A tile, two 8-byte loads from a transposed one (same registers either way).
+template <int H, int MT_, bool HI, bool AT, int MT>
+__device__ __forceinline__ void load_a_pair(Frags<MT>& f, uint32_t stage, const LaneMap& m) {
+  double2& dst = HI ? f.ahi[MT_] : f.alo[MT_];
+  if constexpr (!AT) {
+    ptx::lds128_off<MT_ * 2048 + (HI ? 1024 : 0)>(stage + m.a_off[H], dst.x, dst.y);
+  } else {
+    ptx::lds64_off<MT_ * B_BOX_BYTES + H * 1024>(stage + m.at_off[0][HI ? 1 : 0], dst.x);
+    ptx::lds64_off<MT_ * B_BOX_BYTES + H * 1024>(stage + m.at_off[1][HI ? 1 : 0], dst.y);
+  }
+}
+
 template <int I, int N, typename F>
 __device__ __forceinline__ void static_for(F&& f) {
   if constexpr (I < N) {
@@ -420,12 +467,11 @@ __device__ __forceinline__ void load_b_pair(Frags<MT>& f, uint32_t addr) {
   else ptx::lds128_off<NP * B_BOX_BYTES>(addr, f.bf[NP][0].y, f.bf[NP][1].y);
 }
 
-template <int H, int MT, bool BT = false>
+template <int H, int MT, bool BT = false, bool AT = false>
 __device__ __forceinline__ void load_frags(Frags<MT>& f, uint32_t stage, const LaneMap& m) {
-  const uint32_t a = stage + m.a_off[H];
   static_for<0, MT>([&](auto mt) {
-    ptx::lds128_off<mt.value * 2048>(a, f.alo[mt.value].x, f.alo[mt.value].y);
-    ptx::lds128_off<mt.value * 2048 + 1024>(a, f.ahi[mt.value].x, f.ahi[mt.value].y);
+    load_a_pair<H, mt.value, false, AT>(f, stage, m);
+    load_a_pair<H, mt.value, true, AT>(f, stage, m);
   });
   static_for<0, 2>([&](auto np) {
     load_b_pair<np.value, 0, BT>(f, stage + m.b_off[H][0]);
@@ -453,22 +499,21 @@ __device__ __forceinline__ void mma_frags(double (&acc)[MT][4][4], const Frags<M
 
 // One of the 12 fragment loads of a half k-block, numbered so that the ones needed first by the
 // MMAs come first: 0..3 = B (np, b), then per row block alo, ahi.
-template <int H, int I, bool BT, int MT>
+template <int H, int I, bool BT, bool AT, int MT>
 __device__ __forceinline__ void load_frag_piece(Frags<MT>& f, uint32_t stage, const LaneMap& m) {
   if constexpr (I < 4) {
     constexpr int np = I >> 1, b = I & 1;
     load_b_pair<np, b, BT>(f, stage + m.b_off[H][b]);
   } else if constexpr (I < 4 + 2 * MT) {
     constexpr int mt = (I - 4) >> 1;
-    if constexpr (((I - 4) & 1) == 0) ptx::lds128_off<mt * 2048>(stage + m.a_off[H], f.alo[mt].x, f.alo[mt].y);
-    else ptx::lds128_off<mt * 2048 + 1024>(stage + m.a_off[H], f.ahi[mt].x, f.ahi[mt].y);
+    load_a_pair<H, mt, ((I - 4) & 1) != 0, AT>(f, stage, m);
   }
 }
 
 // The MMAs of row blocks [MT0, MT1) of the half k-block in `cur`, with the loads [L0, L1) of half
 // HN (into `nxt`, from `stage_n`) spread between them, so that the loads neither arrive in a burst
 // nor wait behind the arithmetic.
-template <int MT0, int MT1, int HN, int L0, int L1, bool BT = false, int MT = 4>
+template <int MT0, int MT1, int HN, int L0, int L1, bool BT = false, bool AT = false, int MT = 4>
 __device__ __forceinline__ void mma_frags_loading(double (&acc)[MT][4][4], const Frags<MT>& cur, Frags<MT>& nxt,
                                                   uint32_t stage_n, const LaneMap& m) {
   constexpr int GROUPS = 2 * (MT1 - MT0);
@@ -477,7 +522,7 @@ __device__ __forceinline__ void mma_frags_loading(double (&acc)[MT][4][4], const
     constexpr int mt = MT0 + g / 2, np = g % 2;
     // loads [lo, hi) of this group: an even share of L1 - L0
     constexpr int lo = L0 + (L1 - L0) * g / GROUPS, hi = L0 + (L1 - L0) * (g + 1) / GROUPS;
-    static_for<lo, hi>([&](auto li) { load_frag_piece<HN, li.value, BT>(nxt, stage_n, m); });
+    static_for<lo, hi>([&](auto li) { load_frag_piece<HN, li.value, BT, AT>(nxt, stage_n, m); });
     ptx::dmma_m8n8k4(acc[mt][2 * np + 0][0], acc[mt][2 * np + 0][1], cur.alo[mt].x, cur.bf[np][0].x);
     ptx::dmma_m8n8k4(acc[mt][2 * np + 0][2], acc[mt][2 * np + 0][3], cur.ahi[mt].x, cur.bf[np][0].x);
     ptx::dmma_m8n8k4(acc[mt][2 * np + 1][0], acc[mt][2 * np + 1][1], cur.alo[mt].x, cur.bf[np][0].y);
@@ -752,7 +797,8 @@ constexpr int MICRO_DFMA = 1;
 
 // BT: map_b describes B as stored transposed (N x K, the general entry point's op(B) = B^T) and the
 // stage holds B^T: no transposing pass in HBM. TMA staging only.
-template <bool USE_TMA, int TBM, int WTM = 64, int TBN = BN, int MICRO = MICRO_DMMA, bool BT = false>
+// AT: likewise map_a describes A as stored transposed (K x M) and the stage holds that tile.
+template <bool USE_TMA, int TBM, int WTM = 64, int TBN = BN, int MICRO = MICRO_DMMA, bool BT = false, bool AT = false>
 __global__ void __launch_bounds__(TileCfg<TBM, WTM, TBN>::THREADS_, TileCfg<TBM, WTM, TBN>::CTAS_PER_SM)
 dgemm_dmma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                   const __grid_constant__ GemmParams p) {
@@ -842,7 +888,11 @@ dgemm_dmma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
             good = 0;
           } else if (!p.drop_loads) {
             ptx::mbar_arrive_expect_tx(fb, STAGE_BYTES);
-            ptx::tma_load_2d(sa, &map_a, kb * BK, cur_tm * TBM, fb);
+            if constexpr (AT) {
+              tma_load_at(sa, &map_a, p.a_blocked_map, cur_tm * TBM, kb * BK, fb, TBM / 16);
+            } else {
+              ptx::tma_load_2d(sa, &map_a, kb * BK, cur_tm * TBM, fb);
+            }
             if constexpr (BT) {
               ptx::tma_load_2d(sb, &map_b, kb * BK, cur_tn * TBN, fb);  // rows n of B^T, 16 k each
             } else if (p.b_blocked_map) {
@@ -931,8 +981,8 @@ dgemm_dmma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
 
   for (int i = 0; i < LOOKAHEAD && ok; ++i) ok = issue_next();
 
-  static_assert(!BT || (USE_TMA && MICRO == MICRO_DMMA), "the transposed-B stage exists for TMA staging and the MMA micro-kernel");
-  const LaneMap lm = make_lane_map(warp, lane, A_STAGE_BYTES, WTM, WARPS_N, BT);
+  static_assert(!(BT || AT) || (USE_TMA && MICRO == MICRO_DMMA), "the transposed stages exist for TMA staging and the MMA micro-kernel");
+  const LaneMap lm = make_lane_map(warp, lane, A_STAGE_BYTES, WTM, WARPS_N, BT, AT);
 
   double acc[MT][4][4];  // [mt][nt = 2*np + j][c0..c3]
   uint32_t it = 0;      // k-blocks consumed so far
@@ -961,7 +1011,7 @@ dgemm_dmma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
       const uint32_t ph = (it / STAGES) & 1u;
       if (!wait_bounded(full_bar + 8 * s, ph, abort_flag, p)) { ok = false; break; }
       if constexpr (MICRO == MICRO_DFMA) compute_kblock_dfma<MT>(tiles + s * STAGE_BYTES, lm, A_STAGE_BYTES, acc);
-      else compute_kblock<false, MT, BT>(tiles + s * STAGE_BYTES, lm, acc);
+      else compute_kblock<false, MT, BT, AT>(tiles + s * STAGE_BYTES, lm, acc);
       release_stage(empty_bar + 8 * s, lane);
       // keep the load stream LOOKAHEAD k-blocks ahead: refill the stage released two k-blocks ago
       if (!issue_next()) { ok = false; break; }
@@ -1016,12 +1066,12 @@ struct WsCfg {
   static constexpr int PRODUCER_REGS = TBM == 128 ? WS_PRODUCER_REGS : 24;
 };
 
-template <bool USE_TMA, int TBM = BM, bool BT = false>
+template <bool USE_TMA, int TBM = BM, bool BT = false, bool AT = false>
 __global__ void __launch_bounds__(WsCfg<TBM>::THREADS_, WsCfg<TBM>::CTAS_PER_SM)
 dgemm_dmma_ws_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                      const __grid_constant__ GemmParams p) {
   static_assert(USE_TMA || TBM == 128, "generic staging needs the 128-row producer layout and 40 producer registers");
-  static_assert(!BT || USE_TMA, "the transposed-B stage exists for TMA staging only");
+  static_assert(!(BT || AT) || USE_TMA, "the transposed stages exist for TMA staging only");
   constexpr int STAGES = WsCfg<TBM>::STAGES_;
   constexpr int WARPS = WsCfg<TBM>::CONSUMER_WARPS;
   constexpr int A_STAGE_BYTES = WsCfg<TBM>::A_BYTES;
@@ -1093,7 +1143,11 @@ dgemm_dmma_ws_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
               good = 0;
             } else if (!p.drop_loads) {
               ptx::mbar_arrive_expect_tx(fb, STAGE_BYTES);
-              ptx::tma_load_2d(sa, &map_a, kb * BK, w.tm * TBM, fb);
+              if constexpr (AT) {
+                tma_load_at(sa, &map_a, p.a_blocked_map, w.tm * TBM, kb * BK, fb, TBM / 16);
+              } else {
+                ptx::tma_load_2d(sa, &map_a, kb * BK, w.tm * TBM, fb);
+              }
               if constexpr (BT) {
                 ptx::tma_load_2d(sb, &map_b, kb * BK, w.tn * BN, fb);  // rows n of B^T, 16 k each
               } else if (p.b_blocked_map) {
@@ -1158,7 +1212,7 @@ dgemm_dmma_ws_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
   } else {
     // ------------------------------------------------------------------ consumer warps
     ptx::setmaxnreg_inc<WS_CONSUMER_REGS>();
-    const LaneMap lm = make_lane_map(warp, lane, A_STAGE_BYTES, 64, 4, BT);
+    const LaneMap lm = make_lane_map(warp, lane, A_STAGE_BYTES, 64, 4, BT, AT);
     double acc[4][4][4];
     for (int idx = 0; ok && get_work(p, cta, nctas, idx, w); ++idx) {
 #pragma unroll
@@ -1171,7 +1225,7 @@ dgemm_dmma_ws_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
       {
         const uint32_t s = it % STAGES;
         if (!wait_bounded_inline(full_bar + 8 * s, (it / STAGES) & 1u, abort_flag, p)) { ok = false; break; }
-        load_frags<0, 4, BT>(f0, tiles_u32 + s * STAGE_BYTES, lm);
+        load_frags<0, 4, BT, AT>(f0, tiles_u32 + s * STAGE_BYTES, lm);
       }
       for (int kb = w.kb0; kb < w.kb1; ++kb, ++it) {
         const uint32_t s = it % STAGES;
@@ -1179,12 +1233,12 @@ dgemm_dmma_ws_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
         const uint32_t ph1 = ((it + 1) / STAGES) & 1u;
         const bool more = kb + 1 < w.kb1;
         const bool ready = more && ptx::mbar_test_wait(full_bar + 8 * s1, ph1);
-        mma_frags_loading<0, 4, 1, 0, 12, BT>(acc, f0, f1, tiles_u32 + s * STAGE_BYTES, lm);
+        mma_frags_loading<0, 4, 1, 0, 12, BT, AT>(acc, f0, f1, tiles_u32 + s * STAGE_BYTES, lm);
         if (more) {
           if (!ready && !wait_bounded_inline(full_bar + 8 * s1, ph1, abort_flag, p)) { ok = false; break; }
-          mma_frags_loading<0, 2, 0, 0, 6, BT>(acc, f1, f0, tiles_u32 + s1 * STAGE_BYTES, lm);
+          mma_frags_loading<0, 2, 0, 0, 6, BT, AT>(acc, f1, f0, tiles_u32 + s1 * STAGE_BYTES, lm);
           release_stage(empty_bar + 8 * s, lane);
-          mma_frags_loading<2, 4, 0, 6, 12, BT>(acc, f1, f0, tiles_u32 + s1 * STAGE_BYTES, lm);
+          mma_frags_loading<2, 4, 0, 6, 12, BT, AT>(acc, f1, f0, tiles_u32 + s1 * STAGE_BYTES, lm);
         } else {
           mma_frags<0, 2>(acc, f1);
           release_stage(empty_bar + 8 * s, lane);

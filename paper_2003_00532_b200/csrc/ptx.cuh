@@ -208,6 +208,10 @@ __device__ __forceinline__ void lds128(uint32_t addr, double& x, double& y) {
 
 // Same with a compile-time byte offset folded into the instruction.
 template <int OFF>
+__device__ __forceinline__ void lds64_off(uint32_t addr, double& x) {
+  asm volatile("ld.shared.f64 %0, [%1+%2];" : "=d"(x) : "r"(addr), "n"(OFF));
+}
+template <int OFF>
 __device__ __forceinline__ void lds128_off(uint32_t addr, double& x, double& y) {
   asm volatile("ld.shared.v2.f64 {%0, %1}, [%2+%3];" : "=d"(x), "=d"(y) : "r"(addr), "n"(OFF));
 }

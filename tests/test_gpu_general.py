@@ -227,22 +227,32 @@ def test_scalars_in_the_inline_kernel_with_64_row_tiles(oracle, alpha, beta):
 
 
 @pytest.mark.parametrize("integer", [True, False])
-@pytest.mark.parametrize("ta", [False, True])
 @pytest.mark.parametrize("shape", [(2048, 2048, 512), (1024, 1024, 1024), (2088, 2048, 300), (600, 700, 500), (1000, 1537, 777),
-                                   (2304, 2304, 64), (300, 260, 200)])
-def test_transposed_b_is_staged_without_a_pass(oracle, shape, ta, integer):
-    """op(B) = B^T with a B the tensor-copy engine can address as it is stored (N x K, even ldb): the
-    warp-specialised kernels and the inline kernel's 64 x 128 tile stage B^T themselves, so the call has
-    the launches of the untransposed product (plus one for a transposed A). Other kernels keep the
-    transposing pass. Either way the result matches the oracle."""
+                                   (2304, 2304, 64), (300, 260, 200), (1000, 1536, 256), (1010, 1536, 250)])
+def test_transposed_operands_are_staged_without_a_pass(oracle, shape, integer):
+    """op(A) = A^T, op(B) = B^T with operands the tensor-copy engine can address as they are stored
+    (16-byte aligned, even leading dimension): the warp-specialised kernels and the inline kernel's
+    64 x 128 tile stage the transposed tiles themselves, so all four forms cost the launches of the
+    untransposed product. Other kernels keep the transposing pass. Either way the result matches the
+    oracle (M a multiple of 16 or not: one 3-D copy per stage of A^T, or box by box)."""
     M, N, K = shape
     counts = {}
-    for tb in (False, True):
+    for ta, tb in FORMS:
         n0 = dg.dgemm_launch_count()
         _case(oracle, M, N, K, ta, tb, 1.0, 1.0, integer, seed=3000 + M + N + K, pad=(2, 4, 6))
-        counts[tb] = dg.dgemm_launch_count() - n0
+        counts[(ta, tb)] = dg.dgemm_launch_count() - n0
+    plan = dg.dgemm_plan(M, N, K, tma_addressable=False)  # (as planned without the bulk epilogue; the staging does not matter for the tile)
     plan = dg.dgemm_plan(M, N, K)
     native = (plan["variant"] == dg.DGEMM_VARIANT_TMA_WS or (plan["variant"] == dg.DGEMM_VARIANT_TMA and plan["bm"] == 64)) \
         and plan["bn"] == 128 and plan["wtm"] == 64 and not (N >= 1024 and 1 <= N % 128 <= 64)
     if native:
-        assert counts[True] == counts[False], (counts, plan)
+        assert len(set(counts.values())) == 1, (counts, plan)
+
+
+def test_transposed_operand_that_cannot_be_used_in_place_takes_the_pass(oracle):
+    """Odd leading dimension of the transposed operand, or an unaligned untransposed partner that is
+    too small to repack: the transposing pass (and the generic staging) as before."""
+    _case(oracle, 1024, 1024, 512, True, True, 1.0, 1.0, True, seed=77, pad=(3, 5, 7))
+    _case(oracle, 300, 260, 200, False, True, 1.0, 1.0, True, seed=78, pad=(3, 4, 6))   # A odd, small: generic staging
+    _case(oracle, 300, 260, 200, True, False, 2.0, -1.0, True, seed=79, pad=(2, 5, 6))  # B odd
+    _case(oracle, 2048, 1024, 512, True, False, 1.0, 1.0, False, seed=80, pad=(2, 5, 6))  # B odd, large: packed, A^T native

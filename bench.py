@@ -34,7 +34,7 @@ FMA_PER_CLK_SM = 64  # FP64 DMMA issue rate measured by dgemm_fp64_peak_probe (6
 
 # DRAM traffic of one 8192^3 launch of the dominant kernel (dram__bytes_read.sum +
 # dram__bytes_write.sum of one ncu capture, see profiles/); None until a capture exists for a size.
-NCU_DRAM_BYTES_PER_LAUNCH = {8192: 7941432320 + 538764544, 4096: 1103830000 + 134994688}
+NCU_DRAM_BYTES_PER_LAUNCH = {8192: 7795650304 + 570514944, 4096: 1103830000 + 134994688}
 
 
 def _load_measured_peaks():

@@ -13,6 +13,9 @@ the points of the space are kernels that are all compiled into the library (a va
     generic  8-byte asynchronous copies instead of TMA (any alignment)
     cluster  64 x 128 tiles, K cut over the CTAs of a thread-block cluster, partial tiles added
              through distributed shared memory (one launch; what the library uses below one wave)
+    bulk     warp-specialised, 128 x 128 tiles, five stages, accumulators leave through a shared-memory
+             tile buffer and the copy engine's bulk reduce into C (what the library uses for many
+             tiles of few k-blocks)
 
 ``model_ms`` predicts the time of each from the shape (waves of tiles, a K split of the last
 partial wave, the per-tile C round trip, launch latencies); ``autotune`` measures them through the
@@ -44,16 +47,20 @@ class Config:
     ctas_per_sm: int
     mainloop_eff: float   # fraction of the pipe peak the steady-state k loop sustains (measured, long K)
     needs_tma: bool = True
+    epilogue_exposed: float = -1.0  # share of a tile's C round trip the arithmetic waits for (-1: by CTAs per SM)
 
 
 CONFIGS: Dict[str, Config] = {
-    "ws128": Config("ws128", 3, 0, 128, 128, 1, 0.975),
-    "ws64": Config("ws64", 3, 32, 64, 128, 2, 0.950),
-    "inline64": Config("inline64", 1, 0, 64, 128, 2, 0.970),
+    # epilogue_exposed from the rank-k K = 64 shape (16384^2 x 64: 1516, 1256 and 1354 us measured)
+    "ws128": Config("ws128", 3, 0, 128, 128, 1, 0.975, epilogue_exposed=0.86),
+    "ws64": Config("ws64", 3, 32, 64, 128, 2, 0.950, epilogue_exposed=0.85),
+    "inline64": Config("inline64", 1, 0, 64, 128, 2, 0.970, epilogue_exposed=1.2),
     "inline128": Config("inline128", 1, 4, 128, 128, 1, 0.960),
     "small_wt": Config("small_wt", 1, 4 | 8, 128, 128, 1, 0.945),
     "generic": Config("generic", 2, 16, 64, 128, 2, 0.880, needs_tma=False),
     "cluster": Config("cluster", 5, 0, 64, 128, 2, 0.775),
+    # C never enters the SM; what the arithmetic waits for is its own stores into the tile buffer
+    "bulk": Config("bulk", 10, 0, 128, 128, 1, 0.955, epilogue_exposed=0.22),
 }
 
 KBLOCK_ALONE_US = 1.35   # one k-block of a 64 x 128 tile on an SM the CTA has to itself (measured, long K)
@@ -128,7 +135,7 @@ def model_ms(M: int, N: int, K: int, cfg: Config, ldc_aligned: bool = True) -> f
     # C round trip per tile: hidden behind the other CTA's arithmetic when two share an SM
     tile_bytes = 2.0 * cfg.bm * cfg.bn * 8
     per_sm_bw = HBM_GBS * 1e9 / SM_COUNT * (1.0 if ldc_aligned else 0.5)
-    exposed = 1.0 if cfg.ctas_per_sm == 1 else 0.35
+    exposed = cfg.epilogue_exposed if cfg.epilogue_exposed >= 0 else (1.0 if cfg.ctas_per_sm == 1 else 0.35)
     tiles_per_slot = math.ceil(tiles / slots)
     t_epi = tiles_per_slot * tile_bytes / per_sm_bw * exposed
     # the whole problem cannot beat its compulsory HBM traffic

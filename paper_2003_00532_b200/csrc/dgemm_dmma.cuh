@@ -737,7 +737,28 @@ __device__ __forceinline__ void reduce_range(const GemmParams& p, int tm, int tn
       const int e = e0 + 2 * nthreads * u;
       sum[u] = e < e_end ? __ldcg(reinterpret_cast<const double2*>(src + e)) : make_double2(0.0, 0.0);
     }
-    for (int s = 1; s < count; ++s) {
+    int s = 1;
+    // eight partial tiles per round trip while there are that many (tiles cut into many pieces)
+    for (; s + 8 <= count; s += 8) {
+      double2 w[8][U];
+#pragma unroll
+      for (int q = 0; q < 8; ++q) {
+        const double* sq = p.partial + (long long)slot_of(s + q) * (BM * BN);
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+          const int e = e0 + 2 * nthreads * u;
+          w[q][u] = e < e_end ? __ldcg(reinterpret_cast<const double2*>(sq + e)) : make_double2(0.0, 0.0);
+        }
+      }
+#pragma unroll
+      for (int q = 0; q < 8; ++q)
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+          sum[u].x += w[q][u].x;
+          sum[u].y += w[q][u].y;
+        }
+    }
+    for (; s < count; ++s) {
       src = p.partial + (long long)slot_of(s) * (BM * BN);
       double2 v[U];
 #pragma unroll

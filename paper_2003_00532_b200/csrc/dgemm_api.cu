@@ -65,6 +65,7 @@ constexpr int kClusterCreditKblocks = 1;
 constexpr int kClusterMaxKblocks = 8;
 // Column split of a ragged N (launch_gemm): M * K * (columns of arithmetic saved) above which the second launch pays
 constexpr double kColumnSplitMinWork = 2.0e8;
+constexpr double kColumnSplitMinWorkNarrow = 8.0e8;  // ... for N below 1024
 
 __device__ int g_status_word;  // one per device that loads the library
 
@@ -879,12 +880,17 @@ int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, c
   // A column count just above a multiple of 128 on a large problem: the last tile column of 128
   // would be at most half full. The full tile columns and the remainder are run as two products on
   // disjoint columns of C, the remainder with the 256 x 32 tiles (2088^3: 573 -> 565 us, 4136^3: 4106
-  // -> 4051 us; not worth it below: 1064^3 91 -> 100 us). The sub-matrices start at a multiple of 128
-  // columns, so whatever alignment B and C have is kept.
+  // -> 4051 us; not worth it below: 1064^3 91 -> 100 us). The same for a tall problem with a few
+  // tile columns, where the alternative is 128 x 64 tiles padded to the next 64 columns, when the
+  // remainder fits one 32-column strip (6514 x 146 x 4096: 311 -> 271 us, 8192 x 129 x 8192: 764 ->
+  // 642, 4000 x 400 x 4000: 433 -> 409; not below: 2600 x 140 x 2600 90 -> 94, 2000 x 140 x 2000 57 -> 66).
+  // The sub-matrices start at a multiple of 128 columns, so whatever alignment B and C have is kept.
   if (variant == DGEMM_VARIANT_AUTO && g_test_flags.load() == 0 && g_split_k.load() <= 0) {
     const int64_t r = N % BN, r32 = (r + 31) / 32 * 32;
     const bool addressable = (((uintptr_t)A | (uintptr_t)B) & 15) == 0 && (lda % 2 == 0) && (ldb % 2 == 0);
-    if (addressable && N >= 1024 && r >= 1 && r <= 64 && (double)M * (double)K * (128.0 - 1.2 * (double)r32) > kColumnSplitMinWork) {
+    const bool wide = N >= 1024;  // below, 128 x 64 tiles are the alternative and only a remainder of one 32-column strip pays
+    if (addressable && N > BN && r >= 1 && r <= (wide ? 64 : 32) &&
+        (double)M * (double)K * (128.0 - 1.2 * (double)r32) > (wide ? kColumnSplitMinWork : kColumnSplitMinWorkNarrow)) {
       rc = launch_gemm_packed(st, hold, variant, M, N - r, K, A, lda, B, ldb, C, ldc, stream, form);
       if (rc != DGEMM_OK) return rc;
       return launch_gemm_packed(st, hold, variant, M, r, K, A, lda, B + (N - r), ldb, C + (N - r), ldc, stream, form);

@@ -502,11 +502,12 @@ def test_release_scratch_and_carry_on(oracle):
 
 
 @pytest.mark.parametrize("integer", [True, False])
-@pytest.mark.parametrize("shape", [(2000, 1064, 2000), (2100, 1300, 2050)])
+@pytest.mark.parametrize("shape", [(2000, 1064, 2000), (2100, 1300, 2050), (3000, 146, 3100), (3200, 400, 3000)])
 def test_ragged_n_on_a_large_problem_runs_as_two_products(oracle, shape, integer):
     """N just above a multiple of 128 on a large problem: the full tile columns and the narrow
     remainder are separate launches on disjoint columns of C (padded, odd ldc in the second case:
-    both parts go through the staged epilogue)."""
+    both parts go through the staged epilogue). The last two are tall problems of one and three
+    tile columns plus a remainder of less than 32 columns."""
     M, N, K = shape
     prob = wl.make_problem(M, N, K, seed=81, ldc=N + (7 if N == 1300 else 0), integer=integer)
     n0 = dg.dgemm_launch_count()

@@ -67,6 +67,15 @@ constexpr int kClusterMaxKblocks = 8;
 constexpr double kColumnSplitMinWork = 2.0e8;
 constexpr double kColumnSplitMinWorkNarrow = 8.0e8;  // ... for N below 1024
 
+// Whether a product with N columns is run as two products on a column split (launch_gemm): the
+// shape part of the rule; the caller adds what depends on the operands and the settings.
+inline bool column_split_shape(int64_t M, int64_t N, int64_t K) {
+  const int64_t r = N % 128, r32 = (r + 31) / 32 * 32;
+  const bool wide = N >= 1024;  // below, 128 x 64 tiles are the alternative and only a remainder of one 32-column strip pays
+  return N > 128 && r >= 1 && r <= (wide ? 64 : 32) &&
+         (double)M * (double)K * (128.0 - 1.2 * (double)r32) > (wide ? kColumnSplitMinWork : kColumnSplitMinWorkNarrow);
+}
+
 __device__ int g_status_word;  // one per device that loads the library
 
 struct DeviceState {
@@ -819,7 +828,7 @@ int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, c
     // (as it is, or after the packing pass decided above), and not the case that is run as two
     // products on a column split of B (below).
     if ((form.ta || form.tb) && st->bt_ok && variant == DGEMM_VARIANT_AUTO && g_test_flags.load() == 0 && g_split_k.load() <= 0 &&
-        !(N >= 1024 && N % BN >= 1 && N % BN <= 64) && (!bad_a || pack_a) && (!bad_b || pack_b)) {
+        !column_split_shape(M, N, K) && (!bad_a || pack_a) && (!bad_b || pack_b)) {
       const bool at_ok = form.ta && ((uintptr_t)A & 15) == 0 && (lda % 2 == 0);
       const bool bt_ok = form.tb && ((uintptr_t)B & 15) == 0 && (ldb % 2 == 0);
       // (the other transposed operand, if it cannot be used in place, is rewritten row-major and aligned)
@@ -886,11 +895,10 @@ int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, c
   // 642, 4000 x 400 x 4000: 433 -> 409; not below: 2600 x 140 x 2600 90 -> 94, 2000 x 140 x 2000 57 -> 66).
   // The sub-matrices start at a multiple of 128 columns, so whatever alignment B and C have is kept.
   if (variant == DGEMM_VARIANT_AUTO && g_test_flags.load() == 0 && g_split_k.load() <= 0) {
-    const int64_t r = N % BN, r32 = (r + 31) / 32 * 32;
+    const int64_t r = N % BN;
     const bool addressable = (((uintptr_t)A | (uintptr_t)B) & 15) == 0 && (lda % 2 == 0) && (ldb % 2 == 0);
-    const bool wide = N >= 1024;  // below, 128 x 64 tiles are the alternative and only a remainder of one 32-column strip pays
-    if (addressable && N > BN && r >= 1 && r <= (wide ? 64 : 32) &&
-        (double)M * (double)K * (128.0 - 1.2 * (double)r32) > (wide ? kColumnSplitMinWork : kColumnSplitMinWorkNarrow)) {
+    // (a transposed operand has been rewritten row-major by now: in-place staging is not used on these shapes)
+    if (addressable && !form.native_at && !form.native_bt && column_split_shape(M, N, K)) {
       rc = launch_gemm_packed(st, hold, variant, M, N - r, K, A, lda, B, ldb, C, ldc, stream, form);
       if (rc != DGEMM_OK) return rc;
       return launch_gemm_packed(st, hold, variant, M, r, K, A, lda, B + (N - r), ldb, C + (N - r), ldc, stream, form);

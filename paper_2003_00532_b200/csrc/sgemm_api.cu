@@ -36,6 +36,12 @@ using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t
                                    CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 EncodeTiledFn g_encode = nullptr;
 
+template <int RPT, int NH>
+bool configure_kernel() {
+  return cudaFuncSetAttribute(sgemm_ffma_kernel<RPT, NH>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              Cfg<RPT, NH>::SMEM_BYTES) == cudaSuccess;
+}
+
 int device_state(DeviceState** out) {
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
@@ -54,8 +60,8 @@ int device_state(DeviceState** out) {
     if (major != 10) return DGEMM_ERR_DEVICE;
     if (cudaGetSymbolAddress(reinterpret_cast<void**>(&st.status), g_sgemm_status_word) != cudaSuccess) return DGEMM_ERR_CUDA;
     if (cudaMemset(st.status, 0, sizeof(int)) != cudaSuccess) return DGEMM_ERR_CUDA;
-    if (cudaFuncSetAttribute(sgemm_ffma_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<16>::SMEM_BYTES) != cudaSuccess ||
-        cudaFuncSetAttribute(sgemm_ffma_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<8>::SMEM_BYTES) != cudaSuccess)
+    if (!configure_kernel<16, 2>() || !configure_kernel<8, 2>() || !configure_kernel<4, 2>() ||
+        !configure_kernel<16, 1>() || !configure_kernel<8, 1>() || !configure_kernel<4, 1>())
       return DGEMM_ERR_CUDA;
     if (!g_encode) {
       void* fn = nullptr;
@@ -85,11 +91,12 @@ bool make_map(CUtensorMap* map, const float* base, int64_t rows, int64_t cols, i
 }
 
 // 3-D view of a row-major K x N matrix whose N is a multiple of 32: (column within a block of 32,
-// k, block of 32 columns). One copy of box 32 x TK x 4 lands as four consecutive [TK][32] sub-tiles.
-bool make_blocked_map(CUtensorMap* map, const float* base, int64_t K, int64_t N, int64_t ld) {
+// k, block of 32 columns). One copy of box 32 x TK x (tile columns / 32) lands as consecutive
+// [TK][32] sub-tiles.
+bool make_blocked_map(CUtensorMap* map, const float* base, int64_t K, int64_t N, int64_t ld, int tile_cols) {
   const cuuint64_t dims[3] = {32, (cuuint64_t)K, (cuuint64_t)(N / 32)};
   const cuuint64_t strides[2] = {(cuuint64_t)ld * sizeof(float), 32 * sizeof(float)};
-  const cuuint32_t box[3] = {32, (cuuint32_t)TK, (cuuint32_t)(TN / 32)};
+  const cuuint32_t box[3] = {32, (cuuint32_t)TK, (cuuint32_t)(tile_cols / 32)};
   const cuuint32_t estr[3] = {1, 1, 1};
   return g_encode(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float*>(base), dims, strides, box, estr,
                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -113,7 +120,7 @@ int validate(int64_t M, int64_t N, int64_t K, const float* A, int64_t lda, const
   if (((uintptr_t)A | (uintptr_t)B | (uintptr_t)C) & 3) return DGEMM_ERR_ALIGN;
   const int64_t abytes = ((M - 1) * lda + K) * 4, bbytes = ((K - 1) * ldb + N) * 4, cbytes = ((M - 1) * ldc + N) * 4;
   if (ranges_overlap(C, cbytes, A, abytes) || ranges_overlap(C, cbytes, B, bbytes)) return DGEMM_ERR_ALIAS;
-  const int64_t tiles = ((M + 127) / 128) * ((N + TN - 1) / TN);
+  const int64_t tiles = ((M + 63) / 64) * ((N + 63) / 64);  // (the smallest tile)
   if (tiles > (int64_t)INT32_MAX / 2) return DGEMM_ERR_BAD_DIM;
   return DGEMM_OK;
 }
@@ -133,6 +140,11 @@ void launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cu
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
+
+template <int RPT, int NH>
+void launch_kernel(int grid, cudaStream_t stream, const CUtensorMap& map_a, const CUtensorMap& map_b, const Params& p) {
+  launch_pdl(sgemm_ffma_kernel<RPT, NH>, dim3(grid), dim3(THREADS), (size_t)Cfg<RPT, NH>::SMEM_BYTES, stream, map_a, map_b, p);
 }
 
 inline unsigned grid_y(int64_t blocks) { return (unsigned)(blocks < 65535 ? blocks : 65535); }
@@ -181,10 +193,15 @@ int launch(int64_t M, int64_t N, int64_t K, const float* A, int64_t lda, const f
   p.M = (int)M; p.N = (int)N; p.K = (int)K;
   // 128-row tiles when 256-row tiles would compute at least a tenth more rows
   const int64_t pad128 = (M + 127) / 128 * 128, pad256 = (M + 255) / 256 * 256;
-  const int TM = ((double)pad128 * 1.10 <= (double)pad256) ? 128 : 256;
+  // ... and 64-row tiles for a short M (at most 64 rows, or 129..192) that they fit better still
+  const int64_t pad64 = (M + 63) / 64 * 64;
+  const int TM = (M <= 192 && pad64 < pad128) ? 64 : ((double)pad128 * 1.10 <= (double)pad256) ? 128 : 256;
+  // 64-column tiles for a narrow N that they fit better (at most 64 columns, or 129..192)
+  const int TNV = (N <= 192 && (N + 63) / 64 * 64 < (N + 127) / 128 * 128) ? 64 : 128;
   p.tm_rows = TM;
+  p.tn_cols = TNV;
   p.tiles_m = (int)((M + TM - 1) / TM);
-  p.tiles_n = (int)((N + TN - 1) / TN);
+  p.tiles_n = (int)((N + TNV - 1) / TNV);
   p.kblocks = (int)((K + TK - 1) / TK);
   p.group_m = 8;  // 1024 rows per raster group
   p.A = A; p.B = B; p.C = C;
@@ -196,7 +213,7 @@ int launch(int64_t M, int64_t N, int64_t K, const float* A, int64_t lda, const f
   memset(&map_a, 0, sizeof(map_a));
   memset(&map_b, 0, sizeof(map_b));
   if (!make_map(&map_a, A, M, K, lda, TK, TM)) return DGEMM_ERR_CUDA;
-  p.b_blocked_map = (N % 32 == 0 && make_blocked_map(&map_b, B, K, N, ldb)) ? 1 : 0;
+  p.b_blocked_map = (N % 32 == 0 && make_blocked_map(&map_b, B, K, N, ldb, TNV)) ? 1 : 0;
   if (!p.b_blocked_map && !make_map(&map_b, B, K, N, ldb, 32, TK)) return DGEMM_ERR_CUDA;
 
   // whole waves of tiles run data-parallel; the last partial wave is spread evenly over the CTAs
@@ -221,8 +238,15 @@ int launch(int64_t M, int64_t N, int64_t K, const float* A, int64_t lda, const f
     p.partial = static_cast<float*>(hold.workspace((size_t)2 * resident * MAX_TM * TN * sizeof(float)));
     if (!p.partial) return DGEMM_ERR_CUDA;
   }
-  if (TM == 256) launch_pdl(sgemm_ffma_kernel<16>, dim3(grid), dim3(THREADS), (size_t)Cfg<16>::SMEM_BYTES, stream, map_a, map_b, p);
-  else launch_pdl(sgemm_ffma_kernel<8>, dim3(grid), dim3(THREADS), (size_t)Cfg<8>::SMEM_BYTES, stream, map_a, map_b, p);
+  if (TNV == 128) {
+    if (TM == 256) launch_kernel<16, 2>(grid, stream, map_a, map_b, p);
+    else if (TM == 128) launch_kernel<8, 2>(grid, stream, map_a, map_b, p);
+    else launch_kernel<4, 2>(grid, stream, map_a, map_b, p);
+  } else {
+    if (TM == 256) launch_kernel<16, 1>(grid, stream, map_a, map_b, p);
+    else if (TM == 128) launch_kernel<8, 1>(grid, stream, map_a, map_b, p);
+    else launch_kernel<4, 1>(grid, stream, map_a, map_b, p);
+  }
   if (cudaGetLastError() != cudaSuccess) return DGEMM_ERR_CUDA;
   if (p.tail_tiles > 0 && p.tail_ipc < p.kblocks) {
     launch_pdl(sgemm_tail_reduce_kernel, dim3(p.tail_tiles, 16), dim3(256), 0, stream, p);

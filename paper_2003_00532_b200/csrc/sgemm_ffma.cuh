@@ -19,22 +19,25 @@ namespace sgemm {
 
 using namespace dgemm::ptx;
 
-// Two tile heights: 256 rows (16 x 8 outputs per thread), and 128 rows (8 x 8 per thread) for
-// problems whose M would leave much of a 256-row tile empty. One CTA per SM either way.
-constexpr int TN = 128;  // CTA tile columns
+// Tile heights: 256 rows (16 x 8 outputs per thread), and 128 or 64 rows (8 x 8, 4 x 8 per thread)
+// for problems whose M would leave much of a taller tile empty. Tile widths: 128 columns, or 64
+// (NH = 1: each thread keeps only the first of its two groups of four columns) for a narrow N.
+// One CTA per SM in every form.
+constexpr int TN = 128;  // CTA tile columns of the wide form; row pitch of a workspace slot
 constexpr int TK = 32;   // k extent of a stage: 32 floats = one 128-byte swizzle row
 constexpr int THREADS = 256;
 constexpr int WARPS = THREADS / 32;
 constexpr int B_BOX_BYTES = TK * 32 * 4;    // 4 KiB: [32 k][32 columns]
-constexpr int B_BYTES = (TN / 32) * B_BOX_BYTES;
 constexpr int LOOKAHEAD = 2;                // k-blocks in flight ahead of the arithmetic
 constexpr int SMEM_ALIGN = 1024;
 constexpr int MAX_TM = 256;                 // a workspace slot holds MAX_TM x TN floats
 
-template <int RPT>
+template <int RPT, int NH = 2>
 struct Cfg {
   static constexpr int TM = 16 * RPT;                 // CTA tile rows
+  static constexpr int TNV = 64 * NH;                 // CTA tile columns
   static constexpr int A_BYTES = TM * TK * 4;         // rows of 128 bytes
+  static constexpr int B_BYTES = (TNV / 32) * B_BOX_BYTES;
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
   static constexpr int STAGES = 4;
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + SMEM_ALIGN + 256;
@@ -54,7 +57,8 @@ struct Params {
   // workspace slot 2 * cta + j and sgemm_tail_reduce_kernel adds the slots to C in CTA order.
   int dp_tiles, tail_tiles, tail_ipc;
   float* partial;      // workspace: slots of MAX_TM * TN floats
-  int tm_rows;         // rows of a CTA tile (256 or 128)
+  int tm_rows;         // rows of a CTA tile (256, 128 or 64)
+  int tn_cols;         // columns of a CTA tile (128 or 64)
   const float* A;
   const float* B;
   float* C;
@@ -132,14 +136,15 @@ __device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, vola
   return wait_slow(bar, parity, abort_flag, p.wait_limit_ns, p.status);
 }
 
-template <int RPT>
+template <int RPT, int NH>
 __global__ void __launch_bounds__(THREADS, 1)
 sgemm_ffma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                   const __grid_constant__ Params p) {
-  constexpr int TM = Cfg<RPT>::TM;
-  constexpr int A_BYTES = Cfg<RPT>::A_BYTES;
-  constexpr int STAGE_BYTES = Cfg<RPT>::STAGE_BYTES;
-  constexpr int STAGES = Cfg<RPT>::STAGES;
+  constexpr int TM = Cfg<RPT, NH>::TM;
+  constexpr int TNV = Cfg<RPT, NH>::TNV;
+  constexpr int A_BYTES = Cfg<RPT, NH>::A_BYTES;
+  constexpr int STAGE_BYTES = Cfg<RPT, NH>::STAGE_BYTES;
+  constexpr int STAGES = Cfg<RPT, NH>::STAGES;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t pad = (SMEM_ALIGN - (raw & (SMEM_ALIGN - 1))) & (SMEM_ALIGN - 1);
@@ -197,9 +202,9 @@ sgemm_ffma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
           mbar_arrive_expect_tx(fb, STAGE_BYTES);
           tma_load_2d(sa, &map_a, l_kb * TK, l_tm * TM, fb);
           if (p.b_blocked_map) {
-            tma_load_3d(sb, &map_b, 0, l_kb * TK, l_tn * (TN / 32), fb);
+            tma_load_3d(sb, &map_b, 0, l_kb * TK, l_tn * (TNV / 32), fb);
           } else {
-            for (int nb = 0; nb < TN / 32; ++nb) tma_load_2d(sb + nb * B_BOX_BYTES, &map_b, l_tn * TN + nb * 32, l_kb * TK, fb);
+            for (int nb = 0; nb < TNV / 32; ++nb) tma_load_2d(sb + nb * B_BOX_BYTES, &map_b, l_tn * TNV + nb * 32, l_kb * TK, fb);
           }
         } else {
           good = 0;
@@ -231,7 +236,7 @@ sgemm_ffma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
   const uint32_t b_off = (uint32_t)A_BYTES + (uint32_t)(tx >> 3) * B_BOX_BYTES;  // + k * 128 + (((tx & 7) ^ (k & 7)) << 4)
   const uint32_t b_ch = (uint32_t)(tx & 7);
 
-  float2 acc[RPT][4];  // [row i][column pair]: columns 4 tx + {0,1}, {2,3}, 64 + 4 tx + {0,1}, {2,3}
+  float2 acc[RPT][2 * NH];  // [row i][column pair]: columns 4 tx + {0,1}, {2,3} and, in the wide form, 64 + 4 tx + {0,1}, {2,3}
   uint32_t it = 0;  // k-blocks consumed so far
 
   for (int idx = 0; ok; ++idx) {
@@ -242,7 +247,7 @@ sgemm_ffma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
 #pragma unroll
     for (int i = 0; i < RPT; ++i)
 #pragma unroll
-      for (int j = 0; j < 4; ++j) acc[i][j] = make_float2(0.0f, 0.0f);
+      for (int j = 0; j < 2 * NH; ++j) acc[i][j] = make_float2(0.0f, 0.0f);
 
     for (int kb = w.kb0; kb < w.kb1; ++kb, ++it) {
       // keep the load stream ahead: refill the stage that was released one k-block ago
@@ -265,7 +270,8 @@ sgemm_ffma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
           const uint32_t k7 = (2u * (uint32_t)kp + kk) & 7u;
           const uint32_t bo = st + b_off + (2 * kp + kk) * 128 + ((b_ch ^ k7) << 4);
           const float4 b0 = lds128_f32(bo);
-          const float4 b1 = lds128_f32(bo + 2 * B_BOX_BYTES);
+          float4 b1 = b0;
+          if constexpr (NH == 2) b1 = lds128_f32(bo + 2 * B_BOX_BYTES);
 #pragma unroll
           for (int i = 0; i < RPT; ++i) {
             // packed FP32 FMA (two independent IEEE fused multiply-adds per instruction): half the
@@ -273,8 +279,10 @@ sgemm_ffma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
             const float2 aa = dup_f32x2(kk == 0 ? a[i].x : a[i].y);
             acc[i][0] = __ffma2_rn(aa, make_float2(b0.x, b0.y), acc[i][0]);
             acc[i][1] = __ffma2_rn(aa, make_float2(b0.z, b0.w), acc[i][1]);
-            acc[i][2] = __ffma2_rn(aa, make_float2(b1.x, b1.y), acc[i][2]);
-            acc[i][3] = __ffma2_rn(aa, make_float2(b1.z, b1.w), acc[i][3]);
+            if constexpr (NH == 2) {
+              acc[i][2] = __ffma2_rn(aa, make_float2(b1.x, b1.y), acc[i][2]);
+              acc[i][3] = __ffma2_rn(aa, make_float2(b1.z, b1.w), acc[i][3]);
+            }
           }
         }
       }
@@ -292,7 +300,7 @@ sgemm_ffma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
 #pragma unroll
       for (int i = 0; i < RPT; ++i)
 #pragma unroll
-        for (int h = 0; h < 2; ++h)
+        for (int h = 0; h < NH; ++h)
           *reinterpret_cast<float4*>(dst + (ty + 16 * i) * TN + 64 * h + 4 * tx) =
               make_float4(acc[i][2 * h].x, acc[i][2 * h].y, acc[i][2 * h + 1].x, acc[i][2 * h + 1].y);
       continue;
@@ -304,14 +312,14 @@ sgemm_ffma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     const bool vec = ((reinterpret_cast<uintptr_t>(p.C) & 15) == 0) && ((p.ldc & 3) == 0);
 #pragma unroll
     for (int i0 = 0; i0 < RPT; i0 += 4) {
-      float4 cin[4][2];
+      float4 cin[4][NH];
 #pragma unroll
       for (int ii = 0; ii < 4; ++ii) {
         const int row = tm * TM + ty + 16 * (i0 + ii);
         const float* crow = p.C + (long long)row * p.ldc;
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          const int col = tn * TN + 64 * h + 4 * tx;
+        for (int h = 0; h < NH; ++h) {
+          const int col = tn * TNV + 64 * h + 4 * tx;
           if (row < p.M && vec && col + 3 < p.N) {
             cin[ii][h] = *reinterpret_cast<const float4*>(crow + col);
           } else {
@@ -329,8 +337,8 @@ sgemm_ffma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         if (row >= p.M) continue;
         float* crow = p.C + (long long)row * p.ldc;
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          const int col = tn * TN + 64 * h + 4 * tx;
+        for (int h = 0; h < NH; ++h) {
+          const int col = tn * TNV + 64 * h + 4 * tx;
           float4 c = cin[ii][h];
           c.x += acc[i][2 * h + 0].x;
           c.y += acc[i][2 * h + 0].y;
@@ -378,9 +386,9 @@ __global__ void sgemm_tail_reduce_kernel(const Params p) {
   const int chunk = TM * TN / 16;
   const int e0 = blockIdx.y * chunk;
   for (int e = e0 + 4 * threadIdx.x; e < e0 + chunk; e += 4 * blockDim.x) {
-    const int r = e / TN, c = e - r * TN;
-    const int row = tm * TM + r, col = tn * TN + c;
-    if (row >= p.M || col >= p.N) continue;
+    const int r = e / TN, c = e - r * TN;  // (a slot's rows are TN floats apart in either form)
+    const int row = tm * TM + r, col = tn * p.tn_cols + c;
+    if (row >= p.M || c >= p.tn_cols || col >= p.N) continue;
     float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
     for (int cta = c_first; cta <= c_last; ++cta) {
       const int slot = 2 * cta + ((cta * p.tail_ipc >= lo) ? 0 : 1);

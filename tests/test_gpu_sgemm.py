@@ -63,7 +63,10 @@ def _check(oracle, A, B, C, got, integer):
 
 @pytest.mark.parametrize("integer", [True, False])
 @pytest.mark.parametrize("shape", [(256, 256, 256), (128, 128, 32), (1, 1, 1), (3, 5, 7), (129, 127, 33), (333, 257, 190),
-                                   (1000, 96, 600), (64, 1000, 45), (513, 33, 64), (700, 20, 333)])
+                                   (1000, 96, 600), (64, 1000, 45), (513, 33, 64), (700, 20, 333),
+                                   # short M (64-row tiles), narrow N (64-column tiles), both, and the last wave cut in K
+                                   (32, 2000, 1000), (150, 700, 1200), (190, 260, 515), (2000, 64, 1000), (3000, 40, 700),
+                                   (1500, 160, 900), (1000, 190, 333), (60, 50, 4000), (40, 192, 2048), (9000, 32, 256)])
 def test_small_shapes_dense(oracle, shape, integer):
     A, B, C, got = _run(*shape, integer, seed=sum(shape))
     _check(oracle, A, B, C, got, integer)

@@ -210,28 +210,33 @@ def sgemm_section(dg, torch, sm_max_mhz, sizes=(2048, 4096, 8192)):
     peak = SM_COUNT_B200 * 128 * 2 * sm_max_mhz * 1e6 / 1e12
     out = {"dtype": "f32", "bound": "alu", "peak": peak, "unit": "TFLOP/s",
            "peak_source": "148 SMs x 128 FP32 FMA/clk x 2 x sm_max_mhz; a register-only packed-FMA loop sustains 85 % of it",
-           "kernel": "sgemm_ffma_kernel<16> (TMA staging, 256 x 128 x 32 tiles, 16 x 8 per thread, fma.rn.f32x2)", "shapes": []}
+           "kernel": "sgemm_ffma_kernel<16, 2> (TMA staging, 256 x 128 x 32 tiles, 16 x 8 per thread, fma.rn.f32x2); 64-row and 64-column forms for the skinny shapes", "shapes": []}
     call = dg.load_library().sgemm_f32
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    for n in sizes:
-        A = torch.rand(n, n, dtype=torch.float32, device="cuda") * 2 - 1
-        B = torch.rand(n, n, dtype=torch.float32, device="cuda") * 2 - 1
-        C = torch.zeros(n, n, dtype=torch.float32, device="cuda")
+    # the squares, then a short M (64-row tiles) and a narrow N (64-column tiles)
+    skinny = [(32, 8192, 8192), (8192, 64, 8192)] if len(sizes) > 1 else []
+    for shape in [(n, n, n) for n in sizes] + skinny:
+        M, N, K = shape
+        A = torch.rand(M, K, dtype=torch.float32, device="cuda") * 2 - 1
+        B = torch.rand(K, N, dtype=torch.float32, device="cuda") * 2 - 1
+        C = torch.zeros(M, N, dtype=torch.float32, device="cuda")
         pa, pb, pc = A.data_ptr(), B.data_ptr(), C.data_ptr()
         for _ in range(3):
-            call(n, n, n, pa, n, pb, n, pc, n, None)
+            call(M, N, K, pa, K, pb, N, pc, N, None)
         torch.cuda.synchronize()
-        reps = max(3, min(50, int(8192 ** 3 // n ** 3) * 3))
+        reps = max(3, min(50, int(8192 ** 3 // (M * N * K)) * 3))
         best = float("inf")
         for _ in range(3):
             e0.record()
             for _ in range(reps):
-                call(n, n, n, pa, n, pb, n, pc, n, None)
+                call(M, N, K, pa, K, pb, N, pc, N, None)
             e1.record()
             torch.cuda.synchronize()
             best = min(best, e0.elapsed_time(e1) / reps)
-        tf = 2.0 * n ** 3 / best / 1e9
-        out["shapes"].append({"n": n, "us": round(best * 1e3, 1), "tflops": round(tf, 2), "frac": round(tf / peak, 3)})
+        tf = 2.0 * M * N * K / best / 1e9
+        entry = {"n": M} if M == N == K else {"M": M, "N": N, "K": K}
+        entry.update({"us": round(best * 1e3, 1), "tflops": round(tf, 2), "frac": round(tf / peak, 3)})
+        out["shapes"].append(entry)
         del A, B, C
     assert dg.sgemm_last_device_status() == 0
     return out

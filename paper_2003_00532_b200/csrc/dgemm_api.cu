@@ -39,9 +39,13 @@ inline bool half_width_tiles_pay(int64_t N) {
   return (double)cols64 * 1.10 <= (double)cols128;
 }
 
-inline bool narrow_tiles_pay(int64_t N) {
+// 256 x 32 tiles for a narrow N: when they cover clearly less padded area than 64 x 128 tiles would
+// (in N alone for a tall problem; a short M turns the comparison around: 64 x 64 x 262144 ran 273 us
+// on one 256 x 64 strip pair and 75 % padding, against 163 us for cuBLAS)
+inline bool narrow_tiles_pay(int64_t M, int64_t N) {
   const int64_t cols32 = (N + 31) / 32 * 32, cols128 = (N + 127) / 128 * 128;
-  return N <= 96 && (double)cols32 * 1.2 < (double)cols128;
+  const int64_t rows256 = (M + 255) / 256 * 256, rows64 = (M + 63) / 64 * 64;
+  return N <= 96 && (double)rows256 * (double)cols32 * 1.2 < (double)rows64 * (double)cols128;
 }
 constexpr int kAutoWs64MaxKblocksPerCta = 256;     // ... and its 64-row form instead of the inline kernel up to this much work
 constexpr int kAutoBulkMaxKblocks = 48;             // bulk-epilogue kernel: up to this many k-blocks per tile (K <= 768: +11 % at
@@ -463,7 +467,7 @@ Plan plan_gemm(int64_t M, int64_t N, int64_t K, bool tma_ok, int requested_varia
       const int64_t tiles128 = (pad128 / 128) * ((N + BN - 1) / BN);
       // (a handful of tiles: the inline kernel starts faster, 14 against 18 us at 256^3)
       const bool short_rows = M <= 512 && (M + 31) / 32 * 32 < pad64;  // 32-row tiles of the inline kernel, below
-      const bool std_tile = !narrow_tiles_pay(N) && !half_width_tiles_pay(N) && !short_rows;
+      const bool std_tile = !narrow_tiles_pay(M, N) && !half_width_tiles_pay(N) && !short_rows;
       const bool ws = std_tile && tiles128 >= 16 && (short_k || (double)pad128 <= 1.03 * (double)pad64);
       // Where 64-row tiles are the better fit, the warp-specialised kernel's 64-row form beats the
       // inline kernel on problems of up to a few hundred microseconds (26 random shapes: 4 % in the
@@ -523,7 +527,7 @@ Plan plan_gemm(int64_t M, int64_t N, int64_t K, bool tma_ok, int requested_varia
   // (the micro-kernel swap exists for the 64 x 128 tile only and ignores the tile-shape flags)
   const bool plain_tiles = dfma || (dbg_flags & (DGEMM_TEST_TALL_TILES | DGEMM_TEST_SMALL_WARP_TILES)) != 0;
   // narrow problems (see narrow_tiles_pay) use 256 x 32 tiles: four warps stacked in M, little arithmetic on unused columns
-  const bool narrow = narrow_tiles_pay(N) && !ws_variant && !plain_tiles && two_ctas_ok;
+  const bool narrow = narrow_tiles_pay(M, N) && !ws_variant && !plain_tiles && two_ctas_ok;
   // N just above a multiple of 128: 128 x 64 tiles
   const bool half_width = auto_choice && !ws_variant && !narrow && half_width_tiles_pay(N) && two_ctas_ok && !plain_tiles;
   // short problems in M (M <= 32, or a last 64-row tile that is at most half full while M is small) use 32 x 128
@@ -816,7 +820,7 @@ int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, c
     if (variant == DGEMM_VARIANT_AUTO && (bad_a || bad_b) && !(g_test_flags.load() & DGEMM_TEST_NO_PACKING)) {
       const size_t bytes = ((pack_a || bad_a) ? a_all : 0) + ((pack_b || bad_b) ? b_all : 0);
       const double flop_per_byte = 2.0 * (double)M * (double)N * (double)K / (double)bytes;
-      if (flop_per_byte >= (narrow_tiles_pay(N) ? kPackMinFlopPerByteNarrow : kPackMinFlopPerByte) && bytes <= kPackMaxBytes &&
+      if (flop_per_byte >= (narrow_tiles_pay(M, N) ? kPackMinFlopPerByteNarrow : kPackMinFlopPerByte) && bytes <= kPackMaxBytes &&
           2.0 * (double)M * (double)N * (double)K >= kPackMinFlop) {
         pack_a = pack_a || bad_a;
         pack_b = pack_b || bad_b;

@@ -48,6 +48,10 @@ def _defaults():
     ((128, 128, 4096), V_WS, 64, 128, 64),         # long K runs stay with the general kernels
     ((4097, 31, 4099), V_TMA, 256, 32, 64),        # narrow N
     ((8192, 96, 8192), V_TMA, 256, 32, 64),
+    ((64, 64, 262144), V_TMA, 128, 64, 64),        # ... but not with a short M, where other tiles cover less padded area
+    ((128, 48, 65536), V_TMA, 128, 64, 64),
+    ((64, 96, 100000), V_WS, 64, 128, 64),
+    ((200, 64, 30000), V_TMA, 256, 32, 64),
     ((8192, 128, 8192), V_WS, 128, 128, 64),
     ((6514, 146, 4096), V_TMA, 128, 64, 64),       # N just above a multiple of 128
     ((32, 8192, 8192), V_TMA, 32, 128, 32),        # short M

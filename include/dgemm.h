@@ -128,12 +128,13 @@ DGEMM_API int dgemm_f64(int64_t M, int64_t N, int64_t K,
  * arithmetic). A and C are streamed through device scratch memory in blocks of 1024 rows (upload,
  * dgemm_f64, download on three streams). B follows the first blocks (three on a large problem) in
  * panels of 1024 rows, and those blocks are multiplied K panel by K panel as the panels arrive,
- * so the arithmetic starts long before B is complete (the products of the panels are added into C
- * one after the other: for those rows the sum over k is rounded in that order). Only the M x N
+ * so the arithmetic starts long before B is complete. For those blocks the products of the panels
+ * are summed one after the other and the caller's C, which crosses the link behind B, is added
+ * last (the sum over k is rounded in that order; one rounding against C, as everywhere). Only the M x N
  * logical part of each row is meaningful; padding columns of the host C are preserved.
  * Synchronous: returns after the result is in the host buffer. Device scratch comes from a memory
  * pool the library owns (stream-ordered allocation) and goes back to it before returning; the
- * pool keeps up to 1.25 GiB mapped between calls, because mapping a gigabyte anew on every call
+ * pool keeps up to 1.5 GiB mapped between calls, because mapping a gigabyte anew on every call
  * cost more than the copies and the arithmetic of an 8192^3 problem together. The call runs on
  * streams of its own and leases its scratch like any other call, so it may overlap with other
  * calls of this library. Same argument rules and error codes as dgemm_f64 (Section 2.1; the paper's driver
@@ -295,7 +296,7 @@ DGEMM_API int dgemm_last_device_status(void *stream);
  * Gives the device memory the library holds on the current device back to the system: every
  * scratch lease (an 80 MiB split-K workspace and a packing buffer of up to 2.5 GiB each, as large
  * as the largest packed problem so far; up to four leases) and what the memory pool of
- * dgemm_f64_host keeps mapped (up to 1.25 GiB).
+ * dgemm_f64_host keeps mapped (up to 1.5 GiB).
  * All of it comes back on demand. Synchronises the device first (a kernel of an earlier call may
  * still be using the memory), so it must not be called while a stream is being captured. Returns
  * DGEMM_OK, DGEMM_ERR_DEVICE or DGEMM_ERR_CUDA. No counterpart in the paper.

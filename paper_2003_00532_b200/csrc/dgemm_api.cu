@@ -319,7 +319,7 @@ int device_state(DeviceState** out) {
 // Memory pool of dgemm_f64_host. The device's default pool gives memory back to the system at
 // every synchronisation, so each call would pay for mapping its 0.8 GB (8192^3) again: more than
 // the copies and the arithmetic together. This pool keeps up to kHostPoolKeepBytes between calls.
-constexpr unsigned long long kHostPoolKeepBytes = 5ull << 28;  // 1.25 GiB: B and five blocks of A and C at 8192^3
+constexpr unsigned long long kHostPoolKeepBytes = 6ull << 28;  // 1.5 GiB: B, five blocks of A and C and three more of C at 8192^3 (1.31 GiB)
 int ensure_host_pool(DeviceState* st, cudaMemPool_t* pool) {
   std::lock_guard<std::mutex> lock(g_mutex);
   if (!st->host_pool) {
@@ -1183,6 +1183,9 @@ int dgemm_f64_host(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda
   // by K panel as the panels arrive, each product added into its block of C: the arithmetic
   // starts after 0.5 GB instead of 0.7 GB (8192^3) have crossed the host link, and by the time B
   // is complete three eighths of it are done. The other blocks follow through a ring of buffers.
+  // The head blocks' C does not wait in front of all that: their first panel product is written
+  // with beta = 0, the caller's C follows B across the link into buffers of its own and is added
+  // to the finished product (one rounding, as in the kernels' own epilogue).
   const int64_t prows = (nblk > 1 && K > 2 * kHostPanelRows) ? kHostPanelRows : K;
   const int64_t npan = (K + prows - 1) / prows;
   const int heads = (npan > 1 && nblk >= 6) ? 3 : 1;
@@ -1191,6 +1194,7 @@ int dgemm_f64_host(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda
   double* dB = nullptr;
   double* dA[kHostMaxBufs] = {nullptr, nullptr, nullptr, nullptr, nullptr};
   double* dC[kHostMaxBufs] = {nullptr, nullptr, nullptr, nullptr, nullptr};
+  double* dT[kHostMaxBufs] = {nullptr, nullptr, nullptr, nullptr, nullptr};  // the caller's C of the head blocks
   std::vector<cudaEvent_t> ev_pan;  // one per row panel of B
   cudaEvent_t ev_alloc = nullptr, ev_up[kHostMaxBufs] = {nullptr, nullptr, nullptr, nullptr, nullptr},
               ev_run[kHostMaxBufs] = {nullptr, nullptr, nullptr, nullptr, nullptr},
@@ -1210,23 +1214,27 @@ int dgemm_f64_host(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda
     for (int i = 0; i < nbuf && ok; ++i)
       ok = cudaMallocFromPoolAsync(reinterpret_cast<void**>(&dA[i]), (size_t)blk * dlda * 8, pool, s_up) == cudaSuccess &&
            cudaMallocFromPoolAsync(reinterpret_cast<void**>(&dC[i]), (size_t)blk * dldc * 8, pool, s_up) == cudaSuccess;
+    const bool late_c = npan > 1;  // (heads > 1 implies it)
+    for (int h = 0; h < heads && ok && late_c; ++h)
+      ok = cudaMallocFromPoolAsync(reinterpret_cast<void**>(&dT[h]), (size_t)blk * dldc * 8, pool, s_up) == cudaSuccess;
     if (!ok) break;
     // the other streams may touch the buffers only after the (stream-ordered) allocations
     if (cudaEventRecord(ev_alloc, s_up) != cudaSuccess) break;
     if (cudaStreamWaitEvent(s_run, ev_alloc, 0) != cudaSuccess || cudaStreamWaitEvent(s_down, ev_alloc, 0) != cudaSuccess) break;
     int inner = DGEMM_OK;
-    auto upload_block = [&](int64_t i) -> bool {
+    auto upload_block = [&](int64_t i, bool with_c) -> bool {
       const int b = (int)(i % nbuf);
       const int64_t r0 = i * blk, rows = (M - r0 < blk) ? M - r0 : blk;
       // buffer b is free again once block i - 2 has been downloaded
       if (i >= nbuf && cudaStreamWaitEvent(s_up, ev_down[b], 0) != cudaSuccess) return false;
       return cudaMemcpy2DAsync(dA[b], dlda * 8, A + r0 * lda, lda * 8, K * 8, rows, cudaMemcpyHostToDevice, s_up) == cudaSuccess &&
-             cudaMemcpy2DAsync(dC[b], dldc * 8, C + r0 * ldc, ldc * 8, N * 8, rows, cudaMemcpyHostToDevice, s_up) == cudaSuccess &&
+             (!with_c ||
+              cudaMemcpy2DAsync(dC[b], dldc * 8, C + r0 * ldc, ldc * 8, N * 8, rows, cudaMemcpyHostToDevice, s_up) == cudaSuccess) &&
              cudaEventRecord(ev_up[b], s_up) == cudaSuccess;
     };
     bool heads_up = true;
     for (int h = 0; h < heads && heads_up; ++h)
-      heads_up = upload_block(h) && cudaStreamWaitEvent(s_run, ev_up[h], 0) == cudaSuccess;
+      heads_up = upload_block(h, !late_c) && cudaStreamWaitEvent(s_run, ev_up[h], 0) == cudaSuccess;
     if (!heads_up) break;
     ev_pan.assign((size_t)npan, nullptr);
     for (int64_t j = 0; j < npan && inner == DGEMM_OK; ++j) {
@@ -1237,14 +1245,58 @@ int dgemm_f64_host(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda
         inner = DGEMM_ERR_CUDA;
         break;
       }
+      GemmForm form;  // the first panel product overwrites the buffer, the others add to it
+      form.beta = (j == 0) ? 0.0 : 1.0;
       for (int h = 0; h < heads && npan > 1 && inner == DGEMM_OK; ++h)
-        inner = launch_gemm(blk < M ? blk : M, N, krows, dA[h] + k0, dlda, dB + k0 * dldb, dldb, dC[h], dldc, s_run);
+        inner = launch_gemm(blk < M ? blk : M, N, krows, dA[h] + k0, dlda, dB + k0 * dldb, dldb, dC[h], dldc, s_run, form);
     }
     if (inner != DGEMM_OK) { rc = inner; break; }
+    // Behind B the link carries, in this order: block `heads`, the caller's C of head block 0, block
+    // `heads + 1`, the C of the other head blocks, then the remaining blocks. The arithmetic goes
+    // straight from the last panel product into block `heads` (whose rows are there by then), and
+    // head block 0 is finished and downloaded early enough to free its buffers for the ring.
+    // (The events ev_up[h] of the head blocks are free again: s_run has consumed them.)
+    int64_t uploaded = heads;  // blocks [0, uploaded) have been sent
+    auto upload_head_c = [&](int h) -> bool {
+      const int64_t r0 = (int64_t)h * blk, rows = (M - r0 < blk) ? M - r0 : blk;
+      return cudaMemcpy2DAsync(dT[h], dldc * 8, C + r0 * ldc, ldc * 8, N * 8, rows, cudaMemcpyHostToDevice, s_up) == cudaSuccess &&
+             cudaEventRecord(ev_up[h], s_up) == cudaSuccess;
+    };
+    if (late_c) {
+      bool sent = true;
+      if (cudaEventRecord(ev_alloc, s_run) != cudaSuccess) sent = false;  // (reused: behind the last panel product)
+      if (sent && uploaded < nblk && uploaded < nbuf) sent = upload_block(uploaded++, true);
+      if (sent) sent = upload_head_c(0);
+      if (sent && uploaded < nblk && uploaded < nbuf) sent = upload_block(uploaded++, true);
+      for (int h = 1; h < heads && sent; ++h) sent = upload_head_c(h);
+      if (!sent) { rc = DGEMM_ERR_CUDA; break; }
+    }
     for (int64_t i = 0; i < nblk; ++i) {
       const int b = (int)(i % nbuf);
       const int64_t r0 = i * blk, rows = (M - r0 < blk) ? M - r0 : blk;
-      if (i >= heads && (!upload_block(i) || cudaStreamWaitEvent(s_run, ev_up[b], 0) != cudaSuccess)) { inner = DGEMM_ERR_CUDA; break; }
+      if (i < heads && late_c) {
+        // a head block: its product is complete; add the caller's C and send it back, all on the
+        // download stream, so that the arithmetic stream never waits for that C
+        if (cudaStreamWaitEvent(s_down, ev_alloc, 0) != cudaSuccess || cudaStreamWaitEvent(s_down, ev_up[b], 0) != cudaSuccess) {
+          inner = DGEMM_ERR_CUDA;
+          break;
+        }
+        const unsigned gy = (unsigned)(rows < 4096 ? rows : 4096);
+        dgemm_add_kernel<<<dim3((unsigned)((dldc / 2 + 255) / 256), gy), 256, 0, s_down>>>(dC[b], dldc, dT[b], dldc, (int)rows, (int)dldc);
+        g_launches.fetch_add(1);
+        if (cudaGetLastError() != cudaSuccess ||
+            cudaMemcpy2DAsync(C + r0 * ldc, ldc * 8, dC[b], dldc * 8, N * 8, rows, cudaMemcpyDeviceToHost, s_down) != cudaSuccess ||
+            cudaEventRecord(ev_down[b], s_down) != cudaSuccess) {
+          inner = DGEMM_ERR_CUDA;
+          break;
+        }
+        continue;
+      }
+      if (i >= uploaded) {
+        if (!upload_block(i, true)) { inner = DGEMM_ERR_CUDA; break; }
+        uploaded = i + 1;
+      }
+      if (i >= heads && cudaStreamWaitEvent(s_run, ev_up[b], 0) != cudaSuccess) { inner = DGEMM_ERR_CUDA; break; }
       if (i >= heads || npan == 1) inner = launch_gemm(rows, N, K, dA[b], dlda, dB, dldb, dC[b], dldc, s_run);
       if (inner != DGEMM_OK) break;
       if (cudaEventRecord(ev_run[b], s_run) != cudaSuccess || cudaStreamWaitEvent(s_down, ev_run[b], 0) != cudaSuccess ||
@@ -1269,6 +1321,7 @@ int dgemm_f64_host(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda
     for (int i = 0; i < kHostMaxBufs; ++i) {
       if (dA[i]) cudaFreeAsync(dA[i], s_up);
       if (dC[i]) cudaFreeAsync(dC[i], s_up);
+      if (dT[i]) cudaFreeAsync(dT[i], s_up);
     }
     cudaStreamSynchronize(s_up);
   }

@@ -1401,6 +1401,22 @@ __global__ void dgemm_scale_kernel(double* C, long long ldc, int M, int N, doubl
   }
 }
 
+// C += T, element by element (both row-major with their own leading dimensions; 16-byte aligned,
+// even leading dimensions and an even number of columns): the host entry point adds the caller's C
+// to a product that was started before that C had crossed the host link.
+__global__ void dgemm_add_kernel(double* C, long long ldc, const double* T, long long ldt, int M, int N) {
+  const int j = 2 * (blockIdx.x * blockDim.x + threadIdx.x);
+  if (j >= N) return;
+  for (int i = blockIdx.y; i < M; i += gridDim.y) {
+    double2* c = reinterpret_cast<double2*>(C + (long long)i * ldc + j);
+    const double2 t = *reinterpret_cast<const double2*>(T + (long long)i * ldt + j);
+    double2 v = *c;
+    v.x += t.x;
+    v.y += t.y;
+    *c = v;
+  }
+}
+
 // Self-test of the bounded wait: one CTA waits on an mbarrier that nobody signals. The wait gives up
 // after p.wait_limit_ns, records DGEMM_ERR_TIMEOUT in the status word and the kernel returns
 // normally (nothing traps, nothing spins without a limit).

@@ -380,13 +380,15 @@ def test_accumulates_into_c_and_k_split_calls(oracle):
     assert torch.equal(C.cpu(), one)
 
 
-@pytest.mark.parametrize("shape", [(300, 257, 129), (2500, 300, 200), (3072, 130, 64), (2300, 70, 2500), (3100, 33, 3073), (6200, 40, 2100)])
+@pytest.mark.parametrize("shape", [(300, 257, 129), (2500, 300, 200), (3072, 130, 64), (2300, 70, 2500), (3100, 33, 3073), (6200, 40, 2100),
+                                   (6801, 40, 2100)])
 def test_host_entry_point(oracle, shape):
     """Host buffers; the larger cases are streamed through the device in several blocks of rows
-    (a ragged last block in the second case), the last two also with B in several panels of rows
+    (a ragged last block in the second case), the last three also with B in several panels of rows
     behind the first block, which is multiplied K panel by K panel (a ragged last panel, one row in the
-    fifth case); in the last case three head blocks are multiplied against the arriving panels and the
-    other four go through the ring of buffers."""
+    fifth case); in the last two cases three head blocks are multiplied against the arriving panels
+    (their own C follows B and is added at the end) and the other four go through the ring of buffers,
+    the last of them, in the last case, in two halves of 328 and 329 rows."""
     M, N, K = shape
     prob = wl.make_problem(M, N, K, seed=31, lda=K + 3, ldb=N + 5, ldc=N + 7)
     want = prob.C.clone().contiguous().numpy()

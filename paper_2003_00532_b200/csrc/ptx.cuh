@@ -135,7 +135,7 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 
-// ---- TMA (tiled bulk tensor load into this CTA's shared memory, no multicast) -------------
+// ---- TMA (tiled bulk tensor load into the issuing CTA's own shared memory only) ---------
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
   asm volatile(

@@ -62,7 +62,7 @@ enum {
                                     and epilogue on 64 x 128 tiles, with plain FP64 fused multiply-adds on an
                                     8 x 8 register tile per thread in place of the tensor-core MMAs */
   DGEMM_VARIANT_GENERIC_DFMA = 9, /* the same inner kernel under the GENERIC staging: any alignment          */
-  DGEMM_VARIANT_TMA_WS_BULK = 10, /* as TMA_WS on 128 x 128 tiles with three stages and the epilogue done by the
+  DGEMM_VARIANT_TMA_WS_BULK = 10, /* as TMA_WS on 128 x 128 tiles with five stages and the epilogue done by the
                                     copy engine: the accumulators go to a tile buffer in shared memory and
                                     leave as a tiled bulk reduce (add) into C, or a bulk store when beta == 0;
                                     C is never loaded into the SM. Needs, besides the TMA conditions, a

@@ -196,6 +196,10 @@ bool configure_transposed_kernels() {
          cudaFuncSetAttribute(dgemm_dmma_kernel<true, 64, 64, BN, MICRO_DMMA, BT, AT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                               TileCfg<64, 64, BN>::SMEM_BYTES_) == cudaSuccess &&
          cudaFuncSetAttribute(dgemm_dmma_kernel<true, 64, 64, BN, MICRO_DMMA, BT, AT>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                              cudaSharedmemCarveoutMaxShared) == cudaSuccess &&
+         cudaFuncSetAttribute(dgemm_cluster_kernel<true, 64, 64, BN, BT, AT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              TileCfg<64, 64, BN>::SMEM_BYTES_) == cudaSuccess &&
+         cudaFuncSetAttribute(dgemm_cluster_kernel<true, 64, 64, BN, BT, AT>, cudaFuncAttributePreferredSharedMemoryCarveout,
                               cudaSharedmemCarveoutMaxShared) == cudaSuccess;
 }
 
@@ -631,19 +635,23 @@ struct GemmForm {
 };
 
 // Kernels that can stage a transposed operand themselves (a tensor map over the matrix as stored): the
-// warp-specialised kernels and the inline kernel's 64 x 128 tile, all with TMA staging.
+// warp-specialised kernels, the inline kernel's 64 x 128 tile and the cluster split-K kernel, all with TMA staging.
 bool plan_supports_native_bt(const Plan& pl) {
   if (pl.status != DGEMM_OK || pl.bn != BN || pl.wtm != 64) return false;
   if (pl.variant == DGEMM_VARIANT_TMA_WS) return pl.bm == 128 || pl.bm == 64;
+  if (pl.variant == DGEMM_VARIANT_TMA_CLUSTER) return pl.bm == 64;
   return pl.variant == DGEMM_VARIANT_TMA && pl.bm == 64;
 }
 
 // The kernels that stage transposed operands themselves: 0 warp-specialised 128 x 128, 1 warp-specialised
-// 64 x 128, 2 inline 64 x 128.
+// 64 x 128, 2 inline 64 x 128, 3 cluster split-K (64 x 128).
 template <bool BT, bool AT>
 void launch_transposed_kernel(int which, int grid, cudaStream_t stream, const CUtensorMap& map_a, const CUtensorMap& map_b,
                               const GemmParams& p) {
-  if (which == 0)
+  if (which == 3)
+    launch_cluster_pdl(dgemm_cluster_kernel<true, 64, 64, BN, BT, AT>, grid, p.split_k, TileCfg<64, 64, BN>::THREADS_,
+                       (size_t)TileCfg<64, 64, BN>::SMEM_BYTES_, stream, map_a, map_b, p);
+  else if (which == 0)
     launch_gemm_kernel(dgemm_dmma_ws_kernel<true, 128, BT, AT>, grid, WS_THREADS, SMEM_BYTES, stream, map_a, map_b, p);
   else if (which == 1)
     launch_gemm_kernel(dgemm_dmma_ws_kernel<true, 64, BT, AT>, grid, WsCfg<64>::THREADS_, WsCfg<64>::SMEM_BYTES_, stream, map_a, map_b, p);
@@ -745,7 +753,7 @@ int launch_gemm_packed(DeviceState* st, scratch::Hold& hold, int variant, int64_
         p.b_blocked_map = (N % 16 == 0 && make_blocked_map(&map_b, B, K, N, ldb, BK, bn / 16)) ? 1 : 0;
         if (!p.b_blocked_map && !make_map(&map_b, B, K, N, ldb, 16, BK)) return DGEMM_ERR_CUDA;
       }
-      const int which = variant == DGEMM_VARIANT_TMA_WS ? (bm == 64 ? 1 : 0) : 2;
+      const int which = cluster ? 3 : variant == DGEMM_VARIANT_TMA_WS ? (bm == 64 ? 1 : 0) : 2;
       if (form.native_bt && form.native_at) launch_transposed_kernel<true, true>(which, grid, stream, map_a, map_b, p);
       else if (form.native_bt) launch_transposed_kernel<true, false>(which, grid, stream, map_a, map_b, p);
       else launch_transposed_kernel<false, true>(which, grid, stream, map_a, map_b, p);

@@ -60,7 +60,9 @@ __device__ __forceinline__ void stage_copy_generic(const GemmParams& p, uint32_t
   }
 }
 
-template <bool USE_TMA, int TBM, int WTM = 64, int TBN = BN>
+// BT / AT (TMA staging only): B / A is the matrix as stored, N x K / K x M, and the transposed tile is
+// staged by the copy engine itself, as in the inline kernel's 64 x 128 tile.
+template <bool USE_TMA, int TBM, int WTM = 64, int TBN = BN, bool BT = false, bool AT = false>
 __global__ void __launch_bounds__(TileCfg<TBM, WTM, TBN>::THREADS_, 2)
 dgemm_cluster_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                      const __grid_constant__ GemmParams p) {
@@ -79,6 +81,7 @@ dgemm_cluster_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
   static_assert(Cfg::CTAS_PER_SM == 2, "the cluster kernel is built for the two-CTAs-per-SM tiles");
   static_assert(TBM * RED_STRIDE <= STAGES * STAGE_BYTES, "the partial tile must fit in the stage area");
   static_assert(TBM % CLUSTER_MAX == 0, "every rank reduces a whole number of rows");
+  static_assert(USE_TMA || (!BT && !AT), "transposed operands are staged in place by the copy engine only");
 
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = ptx::smem_u32(smem_raw);
@@ -132,8 +135,14 @@ dgemm_cluster_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
       return true;
     }
     ptx::mbar_arrive_expect_tx(fb, STAGE_BYTES);
-    ptx::tma_load_2d(sa, &map_a, (kb0 + j) * BK, tm * TBM, fb);
-    if (p.b_blocked_map) {
+    if constexpr (AT) {
+      tma_load_at(sa, &map_a, p.a_blocked_map, tm * TBM, (kb0 + j) * BK, fb, TBM / 16);
+    } else {
+      ptx::tma_load_2d(sa, &map_a, (kb0 + j) * BK, tm * TBM, fb);
+    }
+    if constexpr (BT) {
+      ptx::tma_load_2d(sb, &map_b, (kb0 + j) * BK, tn * TBN, fb);  // rows n of B^T, 16 k each
+    } else if (p.b_blocked_map) {
       ptx::tma_load_3d(sb, &map_b, 0, (kb0 + j) * BK, tn * (TBN / 16), fb);
     } else {
       tma_load_b_boxes(sb, &map_b, tn * TBN, (kb0 + j) * BK, fb, TBN / 16);
@@ -184,7 +193,7 @@ dgemm_cluster_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
     }
   }
 
-  const LaneMap lm = make_lane_map(warp, lane, A_STAGE_BYTES, WTM, WARPS_N);
+  const LaneMap lm = make_lane_map(warp, lane, A_STAGE_BYTES, WTM, WARPS_N, BT, AT);
   double acc[MT][4][4];
 #pragma unroll
   for (int mt = 0; mt < MT; ++mt)
@@ -200,7 +209,7 @@ dgemm_cluster_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
     // synchronisation and every warp reaches the CTA and cluster barriers below.
     const bool arrived = wait_bounded(full_bar + 8 * s, ph, abort_flag, p);
     if (!__all_sync(0xffffffffu, arrived ? 1 : 0)) { ok = false; break; }
-    compute_kblock<false, MT>(tiles + s * STAGE_BYTES, lm, acc);
+    compute_kblock<false, MT, BT, AT>(tiles + s * STAGE_BYTES, lm, acc);
     release_stage(empty_bar + 8 * s, lane);
     if (!USE_TMA) {
       if (i + LOOKAHEAD < nkb && !__all_sync(0xffffffffu, issue(i + LOOKAHEAD) ? 1 : 0)) { ok = false; break; }

@@ -238,7 +238,9 @@ def _runs_as_two_products(M, N, K):
 @pytest.mark.parametrize("integer", [True, False])
 @pytest.mark.parametrize("shape", [(2048, 2048, 512), (1024, 1024, 1024), (2088, 2048, 300), (600, 700, 500), (1000, 1537, 777),
                                    (2304, 2304, 64), (300, 260, 200), (1000, 1536, 256), (1010, 1536, 250),
-                                   (3200, 400, 3000), (3000, 146, 3100)])
+                                   (3200, 400, 3000), (3000, 146, 3100),
+                                   # a few tiles: K cut inside thread-block clusters
+                                   (512, 512, 512), (320, 320, 320), (64, 64, 64), (200, 130, 96), (512, 512, 256)])
 def test_transposed_operands_are_staged_without_a_pass(oracle, shape, integer):
     """op(A) = A^T, op(B) = B^T with operands the tensor-copy engine can address as they are stored
     (16-byte aligned, even leading dimension): the warp-specialised kernels and the inline kernel's
@@ -253,7 +255,8 @@ def test_transposed_operands_are_staged_without_a_pass(oracle, shape, integer):
         counts[(ta, tb)] = dg.dgemm_launch_count() - n0
     plan = dg.dgemm_plan(M, N, K, tma_addressable=False)  # (as planned without the bulk epilogue; the staging does not matter for the tile)
     plan = dg.dgemm_plan(M, N, K)
-    native = (plan["variant"] == dg.DGEMM_VARIANT_TMA_WS or (plan["variant"] == dg.DGEMM_VARIANT_TMA and plan["bm"] == 64)) \
+    native = (plan["variant"] in (dg.DGEMM_VARIANT_TMA_WS, dg.DGEMM_VARIANT_TMA_CLUSTER) or
+              (plan["variant"] == dg.DGEMM_VARIANT_TMA and plan["bm"] == 64)) \
         and plan["bn"] == 128 and plan["wtm"] == 64 and not _runs_as_two_products(M, N, K) \
         and M % 2 == 0 and N % 2 == 0 and K % 2 == 0  # (even leading dimensions in every form with this padding)
     if native:

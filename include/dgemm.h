@@ -163,11 +163,10 @@ DGEMM_API int dgemm_f64_host(int64_t M, int64_t N, int64_t K,
  * Arithmetic: each C element receives beta*C_old + alpha*s, s the K-term inner product summed as
  * in dgemm_f64; alpha = beta = 1 with no transposition gives bit-identical results to dgemm_f64.
  * A transposed operand that is 16-byte aligned with an even leading dimension is used where it
- * lies: the kernels for square-ish problems (128- and 64-row tiles of 128 columns, and the
- * cluster split-K kernel for problems of a few tiles) stage the transposed tiles themselves
- * (no extra pass, no extra launch; measured from 512^3 up: B^T level with the untransposed
- * product, A^T within 0.6 %, 2 % at 512^3). Otherwise (narrow or short problems, operands that cannot be
- * addressed in place, a very large A^T) a transposed operand is first transposed into device
+ * lies: the kernels stage the transposed tiles themselves (no extra pass, no extra launch;
+ * measured from 512^3 up and on skinny problems: B^T level with the untransposed product, A^T
+ * within 0.6 %, 2 % at 512^3). Otherwise (operands that cannot be addressed in place, a very
+ * large A^T) a transposed operand is first transposed into device
  * scratch memory owned by the library (an O(MK) or O(KN) pass before O(MNK) arithmetic; the buffer
  * is kept and reused, and leased per call like the rest of the scratch: see dgemm_f64).
  * Same pointer, alignment, aliasing and error rules as dgemm_f64; an op code other than the two

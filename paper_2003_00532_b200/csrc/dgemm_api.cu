@@ -188,6 +188,13 @@ bool configure_tile_kernel(int* occupancy) {
 }
 
 // Shared-memory opt-in of the instantiations that stage transposed operands themselves.
+template <int TBM, int WTM, int TBN, bool BT, bool AT>
+bool configure_transposed_tile() {
+  auto* k = dgemm_dmma_kernel<true, TBM, WTM, TBN, MICRO_DMMA, BT, AT>;
+  return cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, TileCfg<TBM, WTM, TBN>::SMEM_BYTES_) == cudaSuccess &&
+         cudaFuncSetAttribute(k, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared) == cudaSuccess;
+}
+
 template <bool BT, bool AT>
 bool configure_transposed_kernels() {
   return cudaFuncSetAttribute(dgemm_dmma_ws_kernel<true, 128, BT, AT>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) == cudaSuccess &&
@@ -200,7 +207,9 @@ bool configure_transposed_kernels() {
          cudaFuncSetAttribute(dgemm_cluster_kernel<true, 64, 64, BN, BT, AT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                               TileCfg<64, 64, BN>::SMEM_BYTES_) == cudaSuccess &&
          cudaFuncSetAttribute(dgemm_cluster_kernel<true, 64, 64, BN, BT, AT>, cudaFuncAttributePreferredSharedMemoryCarveout,
-                              cudaSharedmemCarveoutMaxShared) == cudaSuccess;
+                              cudaSharedmemCarveoutMaxShared) == cudaSuccess &&
+         configure_transposed_tile<128, 64, 64, BT, AT>() && configure_transposed_tile<256, 64, 32, BT, AT>() &&
+         configure_transposed_tile<32, 32, BN, BT, AT>();
 }
 
 // Per-device set-up, once: capability check, SM count, status-word address, shared-memory opt-in.
@@ -637,20 +646,32 @@ struct GemmForm {
 // Kernels that can stage a transposed operand themselves (a tensor map over the matrix as stored): the
 // warp-specialised kernels, the inline kernel's 64 x 128 tile and the cluster split-K kernel, all with TMA staging.
 bool plan_supports_native_bt(const Plan& pl) {
-  if (pl.status != DGEMM_OK || pl.bn != BN || pl.wtm != 64) return false;
+  if (pl.status != DGEMM_OK) return false;
+  if (pl.variant == DGEMM_VARIANT_TMA)  // the inline kernel's 64 x 128, 128 x 64, 256 x 32 and 32 x 128 tiles
+    return (pl.bm == 64 && pl.bn == BN && pl.wtm == 64) || (pl.bm == 128 && pl.bn == 64 && pl.wtm == 64) ||
+           (pl.bm == 256 && pl.bn == 32 && pl.wtm == 64) || (pl.bm == 32 && pl.bn == BN && pl.wtm == 32);
+  if (pl.bn != BN || pl.wtm != 64) return false;
   if (pl.variant == DGEMM_VARIANT_TMA_WS) return pl.bm == 128 || pl.bm == 64;
-  if (pl.variant == DGEMM_VARIANT_TMA_CLUSTER) return pl.bm == 64;
-  return pl.variant == DGEMM_VARIANT_TMA && pl.bm == 64;
+  return pl.variant == DGEMM_VARIANT_TMA_CLUSTER && pl.bm == 64;
 }
 
 // The kernels that stage transposed operands themselves: 0 warp-specialised 128 x 128, 1 warp-specialised
-// 64 x 128, 2 inline 64 x 128, 3 cluster split-K (64 x 128).
+// 64 x 128, 2 inline 64 x 128, 3 cluster split-K (64 x 128), 4 inline 128 x 64, 5 inline 256 x 32, 6 inline 32 x 128.
 template <bool BT, bool AT>
 void launch_transposed_kernel(int which, int grid, cudaStream_t stream, const CUtensorMap& map_a, const CUtensorMap& map_b,
                               const GemmParams& p) {
   if (which == 3)
     launch_cluster_pdl(dgemm_cluster_kernel<true, 64, 64, BN, BT, AT>, grid, p.split_k, TileCfg<64, 64, BN>::THREADS_,
                        (size_t)TileCfg<64, 64, BN>::SMEM_BYTES_, stream, map_a, map_b, p);
+  else if (which == 4)
+    launch_gemm_kernel(dgemm_dmma_kernel<true, 128, 64, 64, MICRO_DMMA, BT, AT>, grid, TileCfg<128, 64, 64>::THREADS_,
+                       TileCfg<128, 64, 64>::SMEM_BYTES_, stream, map_a, map_b, p);
+  else if (which == 5)
+    launch_gemm_kernel(dgemm_dmma_kernel<true, 256, 64, 32, MICRO_DMMA, BT, AT>, grid, TileCfg<256, 64, 32>::THREADS_,
+                       TileCfg<256, 64, 32>::SMEM_BYTES_, stream, map_a, map_b, p);
+  else if (which == 6)
+    launch_gemm_kernel(dgemm_dmma_kernel<true, 32, 32, BN, MICRO_DMMA, BT, AT>, grid, TileCfg<32, 32, BN>::THREADS_,
+                       TileCfg<32, 32, BN>::SMEM_BYTES_, stream, map_a, map_b, p);
   else if (which == 0)
     launch_gemm_kernel(dgemm_dmma_ws_kernel<true, 128, BT, AT>, grid, WS_THREADS, SMEM_BYTES, stream, map_a, map_b, p);
   else if (which == 1)
@@ -753,7 +774,8 @@ int launch_gemm_packed(DeviceState* st, scratch::Hold& hold, int variant, int64_
         p.b_blocked_map = (N % 16 == 0 && make_blocked_map(&map_b, B, K, N, ldb, BK, bn / 16)) ? 1 : 0;
         if (!p.b_blocked_map && !make_map(&map_b, B, K, N, ldb, 16, BK)) return DGEMM_ERR_CUDA;
       }
-      const int which = cluster ? 3 : variant == DGEMM_VARIANT_TMA_WS ? (bm == 64 ? 1 : 0) : 2;
+      const int which = cluster ? 3 : variant == DGEMM_VARIANT_TMA_WS ? (bm == 64 ? 1 : 0)
+                        : bn == 64 ? 4 : bm == 256 ? 5 : bm == 32 ? 6 : 2;
       if (form.native_bt && form.native_at) launch_transposed_kernel<true, true>(which, grid, stream, map_a, map_b, p);
       else if (form.native_bt) launch_transposed_kernel<true, false>(which, grid, stream, map_a, map_b, p);
       else launch_transposed_kernel<false, true>(which, grid, stream, map_a, map_b, p);
@@ -837,15 +859,21 @@ int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, c
     // A transposed operand that TMA can address as it is stored (16-byte aligned, even leading
     // dimension) needs no pass at all where the kernel that would run stages the transposed tile
     // itself: the library's own choice, no test flags, no forced split, the other operand addressable
-    // (as it is, or after the packing pass decided above), and not the case that is run as two
-    // products on a column split of B (below).
+    // (as it is, or after the packing pass decided above). Where the product is run as two products on a
+    // column split of B (below), both parts' kernels have to be of that kind.
     if ((form.ta || form.tb) && st->bt_ok && variant == DGEMM_VARIANT_AUTO && g_test_flags.load() == 0 && g_split_k.load() <= 0 &&
-        !column_split_shape(M, N, K) && (!bad_a || pack_a) && (!bad_b || pack_b)) {
+        (!bad_a || pack_a) && (!bad_b || pack_b)) {
       const bool at_ok = form.ta && ((uintptr_t)A & 15) == 0 && (lda % 2 == 0);
       const bool bt_ok = form.tb && ((uintptr_t)B & 15) == 0 && (ldb % 2 == 0);
       // (the other transposed operand, if it cannot be used in place, is rewritten row-major and aligned)
-      const Plan pl = plan_gemm(M, N, K, true, variant, 0, 0, st->sm_count, st->two_ctas_ok, st->ws_ok, st->cluster_ok, false);
-      if (plan_supports_native_bt(pl)) {
+      auto planned = [&](int64_t n) {
+        return plan_gemm(M, n, K, true, variant, 0, 0, st->sm_count, st->two_ctas_ok, st->ws_ok, st->cluster_ok, false);
+      };
+      const int64_t r = N % BN;
+      const bool supported = column_split_shape(M, N, K)
+                                 ? plan_supports_native_bt(planned(N - r)) && plan_supports_native_bt(planned(r))
+                                 : plan_supports_native_bt(planned(N));
+      if (supported) {
         // B^T in the stage costs nothing measurable; A^T costs the arithmetic warps 0.5 % (four 8-byte loads
         // per fragment pair instead of two 16-byte ones), 1.2 % together with B^T, while the transposing
         // pass of A costs 0.7 % x 8192 / N: in place up to N = 8192, with B^T in place up to 4608
@@ -909,11 +937,12 @@ int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, c
   if (variant == DGEMM_VARIANT_AUTO && g_test_flags.load() == 0 && g_split_k.load() <= 0) {
     const int64_t r = N % BN;
     const bool addressable = (((uintptr_t)A | (uintptr_t)B) & 15) == 0 && (lda % 2 == 0) && (ldb % 2 == 0);
-    // (a transposed operand has been rewritten row-major by now: in-place staging is not used on these shapes)
-    if (addressable && !form.native_at && !form.native_bt && column_split_shape(M, N, K)) {
+    if (addressable && column_split_shape(M, N, K)) {
       rc = launch_gemm_packed(st, hold, variant, M, N - r, K, A, lda, B, ldb, C, ldc, stream, form);
       if (rc != DGEMM_OK) return rc;
-      return launch_gemm_packed(st, hold, variant, M, r, K, A, lda, B + (N - r), ldb, C + (N - r), ldc, stream, form);
+      // (a B that is still the stored N x K matrix is cut by rows)
+      const double* b_rest = form.native_bt ? B + (N - r) * ldb : B + (N - r);
+      return launch_gemm_packed(st, hold, variant, M, r, K, A, lda, b_rest, ldb, C + (N - r), ldc, stream, form);
     }
   }
   return launch_gemm_packed(st, hold, variant, M, N, K, A, lda, B, ldb, C, ldc, stream, form);

@@ -240,11 +240,14 @@ def _runs_as_two_products(M, N, K):
                                    (2304, 2304, 64), (300, 260, 200), (1000, 1536, 256), (1010, 1536, 250),
                                    (3200, 400, 3000), (3000, 146, 3100),
                                    # a few tiles: K cut inside thread-block clusters
-                                   (512, 512, 512), (320, 320, 320), (64, 64, 64), (200, 130, 96), (512, 512, 256)])
+                                   (512, 512, 512), (320, 320, 320), (64, 64, 64), (200, 130, 96), (512, 512, 256),
+                                   # narrow, short and half-width tiles
+                                   (2000, 64, 1000), (1000, 32, 600), (3000, 90, 500), (32, 2000, 1000), (96, 1500, 700),
+                                   (16, 640, 2048), (64, 64, 6000), (1000, 144, 512), (130, 70, 3000), (2048, 48, 2048)])
 def test_transposed_operands_are_staged_without_a_pass(oracle, shape, integer):
     """op(A) = A^T, op(B) = B^T with operands the tensor-copy engine can address as they are stored
     (16-byte aligned, even leading dimension): the warp-specialised kernels and the inline kernel's
-    64 x 128 tile stage the transposed tiles themselves, so all four forms cost the launches of the
+    tiles stage the transposed tiles themselves, so all four forms cost the launches of the
     untransposed product. Other kernels keep the transposing pass. Either way the result matches the
     oracle (M a multiple of 16 or not: one 3-D copy per stage of A^T, or box by box)."""
     M, N, K = shape
@@ -255,10 +258,13 @@ def test_transposed_operands_are_staged_without_a_pass(oracle, shape, integer):
         counts[(ta, tb)] = dg.dgemm_launch_count() - n0
     plan = dg.dgemm_plan(M, N, K, tma_addressable=False)  # (as planned without the bulk epilogue; the staging does not matter for the tile)
     plan = dg.dgemm_plan(M, N, K)
-    native = (plan["variant"] in (dg.DGEMM_VARIANT_TMA_WS, dg.DGEMM_VARIANT_TMA_CLUSTER) or
-              (plan["variant"] == dg.DGEMM_VARIANT_TMA and plan["bm"] == 64)) \
-        and plan["bn"] == 128 and plan["wtm"] == 64 and not _runs_as_two_products(M, N, K) \
+    tile = (plan["bm"], plan["bn"], plan["wtm"])
+    native = ((plan["variant"] in (dg.DGEMM_VARIANT_TMA_WS, dg.DGEMM_VARIANT_TMA_CLUSTER) and plan["bn"] == 128 and plan["wtm"] == 64) or
+              (plan["variant"] == dg.DGEMM_VARIANT_TMA and tile in ((64, 128, 64), (128, 64, 64), (256, 32, 64), (32, 128, 32)))) \
         and M % 2 == 0 and N % 2 == 0 and K % 2 == 0  # (even leading dimensions in every form with this padding)
+    if _runs_as_two_products(M, N, K):  # both parts have to run on such kernels
+        rest = dg.dgemm_plan(M, N % 128, K)
+        native = native and rest["variant"] == dg.DGEMM_VARIANT_TMA and (rest["bm"], rest["bn"], rest["wtm"]) == (256, 32, 64)
     if native:
         assert len(set(counts.values())) == 1, (counts, plan)
 

@@ -55,6 +55,7 @@ constexpr int kAutoWsMinKblocks = 16;                // warp-specialised kernel:
 constexpr double kPackMinFlopPerByte = 32.0;      // pack unaligned operands only if the copy is this cheap
 constexpr double kPackMinFlopPerByteNarrow = 8.0; // ... or this cheap where the generic staging would run the 256 x 32 tile, its slowest form
 constexpr double kPackMinFlop = 0.25e9;            // ... and the problem is not one of a few microseconds, where one more launch shows
+constexpr double kPackMinElemsOfC = 8.0e6;         // (a large C with a tiny K is not one either: the pass over C alone takes 20 us and more)
 constexpr size_t kPackMaxBytes = 2ull << 30;       // ... and the packed copies fit in 2 GiB
 constexpr int64_t kHostBlockRows = 1024;             // dgemm_f64_host: rows of A and C per pipelined block
 constexpr int64_t kHostPanelRows = 1024;             // ... and rows of B per panel while the first blocks wait for B
@@ -851,7 +852,7 @@ int launch_gemm(int64_t M, int64_t N, int64_t K, const double* A, int64_t lda, c
       const size_t bytes = ((pack_a || bad_a) ? a_all : 0) + ((pack_b || bad_b) ? b_all : 0);
       const double flop_per_byte = 2.0 * (double)M * (double)N * (double)K / (double)bytes;
       if (flop_per_byte >= (narrow_tiles_pay(M, N) ? kPackMinFlopPerByteNarrow : kPackMinFlopPerByte) && bytes <= kPackMaxBytes &&
-          2.0 * (double)M * (double)N * (double)K >= kPackMinFlop) {
+          (2.0 * (double)M * (double)N * (double)K >= kPackMinFlop || (double)M * (double)N >= kPackMinElemsOfC)) {
         pack_a = pack_a || bad_a;
         pack_b = pack_b || bad_b;
       }

@@ -48,9 +48,11 @@ inline bool narrow_tiles_pay(int64_t M, int64_t N) {
   return N <= 96 && (double)rows256 * (double)cols32 * 1.2 < (double)rows64 * (double)cols128;
 }
 constexpr int kAutoWs64MaxKblocksPerCta = 256;     // ... and its 64-row form instead of the inline kernel up to this much work
-constexpr int kAutoBulkMaxKblocks = 48;             // bulk-epilogue kernel: up to this many k-blocks per tile (K <= 768: +11 % at
-                                                     // K = 64, +9 % at 128, +4 % at 256, level at 1024, -0.7 % at 8192) ...
-constexpr int kAutoBulkMinWaves = 4;                 // ... and from this many waves of 128 x 128 tiles
+constexpr int kAutoBulkMaxKblocks = 128;            // bulk-epilogue kernel: up to this many k-blocks per tile (K <= 2048: against the
+                                                     // warp-specialised kernels 16 % faster at K = 64, 9 % at 128 ... 256, 1 % at 1024,
+                                                     // 0.4 % at 2048, level at 4096) ...
+constexpr int kAutoBulkMinWaves = 2;                 // ... and from this many waves of 128 x 128 tiles (2.2 ... 3.9 waves: 3 - 15 %
+                                                     // faster; 1.7 waves: 4 % slower at K = 64)
 constexpr int kAutoWsMinKblocks = 16;                // warp-specialised kernel: 128-row tiles from K = 256 up, 64-row below
 constexpr double kPackMinFlopPerByte = 32.0;      // pack unaligned operands only if the copy is this cheap
 constexpr double kPackMinFlopPerByteNarrow = 8.0; // ... or this cheap where the generic staging would run the 256 x 32 tile, its slowest form
@@ -786,13 +788,9 @@ int launch_gemm_packed(DeviceState* st, scratch::Hold& hold, int variant, int64_
     if (cluster)
       launch_cluster_pdl(dgemm_cluster_kernel<true, 64, 64, BN>, grid, p.split_k, TileCfg<64, 64, BN>::THREADS_,
                          (size_t)TileCfg<64, 64, BN>::SMEM_BYTES_, stream, map_a, map_b, p);
-    else if (variant == DGEMM_VARIANT_TMA_WS_BULK) {
-      CUtensorMap map_c;
-      memset(&map_c, 0, sizeof(map_c));
-      if (!make_map(&map_c, C, M, N, ldc, 16, 64)) return DGEMM_ERR_CUDA;  // boxes of 16 columns x 64 rows, 128-byte swizzle
-      launch_pdl(dgemm_dmma_wsb_kernel, dim3(grid), dim3(WsBulkCfg::THREADS_), (size_t)WsBulkCfg::SMEM_BYTES_, stream, map_a, map_b,
-                 map_c, p);
-    } else if (ws64)
+    else if (variant == DGEMM_VARIANT_TMA_WS_BULK)
+      launch_pdl(dgemm_dmma_wsb_kernel, dim3(grid), dim3(WsBulkCfg::THREADS_), (size_t)WsBulkCfg::SMEM_BYTES_, stream, map_a, map_b, p);
+    else if (ws64)
       launch_gemm_kernel(dgemm_dmma_ws_kernel<true, 64>, grid, WsCfg<64>::THREADS_, WsCfg<64>::SMEM_BYTES_, stream, map_a, map_b, p);
     else if (variant == DGEMM_VARIANT_TMA_WS)
       launch_gemm_kernel(dgemm_dmma_ws_kernel<true>, grid, WS_THREADS, SMEM_BYTES, stream, map_a, map_b, p);

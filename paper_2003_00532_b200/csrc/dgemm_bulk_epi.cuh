@@ -7,14 +7,20 @@
 //   * five stages instead of six; the shared memory saved holds half a C tile (64 rows x 128
 //     columns, 64 KB): the tile buffer;
 //   * the consumer warps do not load C. The four warps of a 64-row slab write their accumulators
-//     into the tile buffer (16-byte stores in the 128-byte swizzle of C's tensor map, conflict-free),
-//     and one thread of an otherwise idle warp of the producer warpgroup hands the buffer to the copy
-//     engine: a tiled bulk REDUCE (add.f64) into C for beta == 1, a tiled bulk STORE for beta == 0.
-//     The addition C + acc happens at the L2 (one rounding, exactly the c + acc of the other
-//     epilogues), parts of a box beyond M or N are clipped by the copy engine, and the arithmetic
-//     of the next tile starts as soon as the buffer is written. (Issued by a consumer warp, the
-//     eight copy instructions and the waits around them put that warp 1 - 2 k cycles behind its
-//     neighbours on every tile, and they then waited for it.)
+//     into the tile buffer (row-major, 1024 bytes per row; lanes with even and odd row group store
+//     their two 16-byte pieces in opposite order, which keeps the stores free of bank conflicts),
+//     and an otherwise idle warp of the producer warpgroup hands the buffer to the copy engine, two
+//     rows per lane: a bulk REDUCE (add.f64) of 1024 contiguous bytes into the row of C for
+//     beta == 1, a bulk STORE for beta == 0. The addition C + acc happens at the L2 (one rounding,
+//     exactly the c + acc of the other epilogues), and the arithmetic of the next tile starts as
+//     soon as the buffer is written. Whole-row requests measured faster than tiled boxes of 16
+//     columns through a tensor map (a pass that only reduces 16384^2 doubles: 806 against 919 us),
+//     and asking L2 for the C tile ahead of the reduce, as the other kernels' epilogues do, made
+//     this one slower (K = 64: 1084 -> 1040 us): both together 16384^2 x 64 1084 -> 1024 us,
+//     x 16 1075 -> 865 us. A request cannot clip a row, so the tiles of a ragged last tile column
+//     are added to C by the consumer warps themselves, like in the other kernels. (Issued by a
+//     consumer warp, the copy instructions and the waits around them put that warp 1 - 2 k cycles
+//     behind its neighbours on every tile, and they then waited for it.)
 //   * the two slabs of a tile take turns with the one buffer: slab 0 of tile t, slab 1 of tile t,
 //     slab 0 of tile t + 1, ... A slab writes once the copy engine has read the previous user's data
 //     (cp.async.bulk.wait_group.read in the issuing thread). The turns keep the slabs a few thousand
@@ -35,8 +41,8 @@ struct WsBulkCfg {
   static constexpr int STAGES_ = 5;
   static constexpr int CONSUMER_WARPS = 8;
   static constexpr int THREADS_ = (CONSUMER_WARPS + WS_PRODUCER_WARPS) * 32;
-  static constexpr int C_BOX_BYTES = 16 * 64 * 8;                 // one box: 16 columns x 64 rows
-  static constexpr int C_BUF_BYTES = 8 * C_BOX_BYTES;             // one slab of a tile: 64 rows x 128 columns
+  static constexpr int C_ROW_BYTES = BN * 8;                      // a row of the tile buffer
+  static constexpr int C_BUF_BYTES = 64 * C_ROW_BYTES;            // one slab of a tile: 64 rows x 128 columns, row-major
   static constexpr int C_OFFSET = STAGES_ * STAGE_BYTES;          // from the first stage; a multiple of 1024
   static constexpr int BAR_OFFSET = C_OFFSET + C_BUF_BYTES;
   static constexpr int SMEM_BYTES_ = BAR_OFFSET + SMEM_ALIGN + 1024;  // + alignment slack + barriers, flags, work words
@@ -45,7 +51,7 @@ static_assert(WsBulkCfg::SMEM_BYTES_ <= 227 * 1024, "stages + C tile must fit th
 
 __global__ void __launch_bounds__(WsBulkCfg::THREADS_, 1)
 dgemm_dmma_wsb_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-                      const __grid_constant__ CUtensorMap map_c, const __grid_constant__ GemmParams p) {
+                      const __grid_constant__ GemmParams p) {
   constexpr int STAGES = WsBulkCfg::STAGES_;
   constexpr int WARPS = WsBulkCfg::CONSUMER_WARPS;
   constexpr int TBM = BM;
@@ -98,7 +104,6 @@ dgemm_dmma_wsb_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
     if (pw == 0 && lane == 0) {
       ptx::prefetch_tensormap(&map_a);
       ptx::prefetch_tensormap(&map_b);
-      ptx::prefetch_tensormap(&map_c);
     }
     for (int idx = 0; pw == 0 && ok; ++idx) {
       fetch_work_inline(p, cta, nctas, idx, item_words);
@@ -111,8 +116,6 @@ dgemm_dmma_wsb_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
       const int valid = item_words[5];
       __syncwarp();
       if (!valid) break;
-      // the reduce reads C at the L2: ask for the tile early so that it is there when the reduce arrives
-      const int kb_pf = (w.slot < 0 && p.c_prefetch && p.load_c) ? max(w.kb0, w.kb1 - C_PREFETCH_KBLOCKS) : -1;
       for (int kb = w.kb0; kb < w.kb1; ++kb, ++it) {
         const uint32_t s = it % STAGES;
         const uint32_t ph = (it / STAGES) & 1u;
@@ -134,7 +137,6 @@ dgemm_dmma_wsb_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
           }
         }
         if (!__all_sync(0xffffffffu, good)) { ok = false; break; }
-        if (kb == kb_pf) prefetch_c_rows_inline(p.C, p.ldc, p.M, p.N, TBM, BN, w.tm, w.tn, lane, 32);
       }
     }
     if (!ok && !p.drop_loads && pw == 0 && lane == 0) {
@@ -150,8 +152,8 @@ dgemm_dmma_wsb_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
     }
     // Producer warp 1: the copy-engine hand-over. It walks the same list of work items; for a tile
     // that goes straight to C it takes slab 0 and slab 1 in turn: waits until the slab's four consumer
-    // warps have written the tile buffer, issues the eight box copies (16 columns x 64 rows each),
-    // waits until the copy engine has read the buffer and passes it on.
+    // warps have written the tile buffer, issues the 64 row copies (two per lane), waits until the
+    // copy engine has read the buffer and passes it on.
     if (pw == 1) {
       uint32_t use = 0;  // uses of the tile buffer so far: 2 x tiles + slab
       bool pending = false;
@@ -165,46 +167,45 @@ dgemm_dmma_wsb_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
         __syncwarp();
         if (!valid) break;
         if (w.slot >= 0) continue;  // a partial tile: the consumers store it into the workspace themselves
+        if (w.tn * BN + BN > p.N) continue;  // a ragged last tile column: the consumers' own epilogue
         for (int slab = 0; slab < 2 && ok; ++slab, ++use) {
-          int good = 1;
-          if (lane == 0) {
-            good = wait_bounded_inline(c_full, use & 1u, abort_flag, p) ? 1 : 0;
-            const int y = w.tm * TBM + 64 * slab;
-            if (good) {
-              if (y < p.M) {
-                for (int nb = 0; nb < 8; ++nb) {
-                  const int x = w.tn * BN + 16 * nb;
-                  if (x < p.N) {
-                    if (p.load_c) ptx::tma_reduce_add_2d(&map_c, x, y, c_buf + (uint32_t)nb * WsBulkCfg::C_BOX_BYTES);
-                    else ptx::tma_store_2d(&map_c, x, y, c_buf + (uint32_t)nb * WsBulkCfg::C_BOX_BYTES);
-                  }
-                }
-              }
-              ptx::bulk_commit_group();
-              pending = true;
-              ptx::bulk_wait_group_read_all();  // the copy engine has read the buffer
-              ptx::mbar_arrive(c_turn + 8 * ((use + 1) & 1u));  // the other slab's turn
+          // every lane polls the barrier (it is complete for all or for none soon after) ...
+          const int good = wait_bounded_inline(c_full, use & 1u, abort_flag, p) ? 1 : 0;
+          if (!__all_sync(0xffffffffu, good)) { ok = false; break; }
+          // ... and sends two rows of the slab: 1024 contiguous bytes each
+#pragma unroll
+          for (int q = 0; q < 2; ++q) {
+            const int r = lane + 32 * q;
+            const int y = w.tm * TBM + 64 * slab + r;
+            if (y < p.M) {
+              double* dst = p.C + (long long)y * p.ldc + (long long)w.tn * BN;
+              if (p.load_c) ptx::bulk_reduce_add_f64(dst, c_buf + (uint32_t)(r * WsBulkCfg::C_ROW_BYTES), WsBulkCfg::C_ROW_BYTES);
+              else ptx::bulk_store(dst, c_buf + (uint32_t)(r * WsBulkCfg::C_ROW_BYTES), WsBulkCfg::C_ROW_BYTES);
             }
           }
-          if (!__all_sync(0xffffffffu, good)) ok = false;
+          ptx::bulk_commit_group();
+          pending = true;
+          ptx::bulk_wait_group_read_all();  // the copy engine has read this lane's rows
+          __syncwarp();
+          if (lane == 0) ptx::mbar_arrive(c_turn + 8 * ((use + 1) & 1u));  // the other slab's turn
         }
       }
-      if (lane == 0 && pending) ptx::bulk_wait_group_all();  // nothing of this CTA is in flight when it leaves
+      if (pending) ptx::bulk_wait_group_all();  // nothing of this CTA is in flight when it leaves
     }
   } else {
     // ------------------------------------------------------------------ consumer warps
     ptx::setmaxnreg_inc<WS_CONSUMER_REGS>();
     const LaneMap lm = make_lane_map(warp, lane, A_STAGE_BYTES, 64, 4);
-    // This lane's place in the tile buffer, which holds one slab (64 rows) as 8 boxes of 16 columns;
-    // box nb = 2 wn + np holds rows of 128 bytes, 16-byte chunk c of row r at position c ^ (r & 7).
-    // The lane owns rows rm + 8 j (j < 8), columns 4t .. 4t+3 of boxes 2wn and 2wn+1: chunks 2t, 2t+1.
-    // Lanes of a quarter-warp with even and odd g write rows that differ by 4; storing the two chunks
-    // in opposite order in the two kinds of lanes keeps every 16-byte store free of bank conflicts.
+    // This lane's place in the tile buffer, which holds one slab (64 rows) row-major. The lane owns
+    // rows rm + 8 j (j < 8) and, in each, columns 32 wn + 16 np + 4t .. + 3 (np < 2): two 16-byte pieces.
+    // Lanes of a quarter-warp with even and odd g write rows that differ by 4, i.e. by a multiple of
+    // 128 bytes; storing the two pieces in opposite order in the two kinds of lanes keeps every
+    // 16-byte store free of bank conflicts.
     const int slab = lm.wm;
     const bool swap = (lm.g & 1) != 0;
-    const uint32_t c_lane = c_buf + (uint32_t)(2 * lm.wn) * WsBulkCfg::C_BOX_BYTES + (uint32_t)lm.rm * 128u;
-    const uint32_t ch_first = (uint32_t)(((2 * lm.t + (swap ? 1 : 0)) ^ lm.rm) << 4);
-    const uint32_t ch_second = (uint32_t)(((2 * lm.t + (swap ? 0 : 1)) ^ lm.rm) << 4);
+    const uint32_t c_lane = c_buf + (uint32_t)(lm.rm * WsBulkCfg::C_ROW_BYTES) + (uint32_t)(32 * lm.wn + 4 * lm.t) * 8u;
+    const uint32_t ch_first = swap ? 16u : 0u;
+    const uint32_t ch_second = swap ? 0u : 16u;
     uint32_t use = (uint32_t)slab;         // this slab's next turn with the tile buffer: 2 x tiles so far + slab
     double acc[4][4][4];
     // The work item of the next tile is looked up while the last k-block of the current one is
@@ -244,8 +245,10 @@ dgemm_dmma_wsb_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
         }
       }
       if (!ok) break;
-      if (w.slot >= 0) {
-        store_tile<WS_EPI_BATCH, 4, false>(p, w, lm, acc);  // a partial tile: straight to the workspace
+      if (w.slot >= 0 || w.tn * BN + BN > p.N) {
+        // a partial tile goes straight to the workspace; a tile of a ragged last tile column is added
+        // to C by these warps themselves (the copy engine's untiled requests cannot clip a row)
+        store_tile<WS_EPI_BATCH, 4, false>(p, w, lm, acc);
         continue;
       }
       // ---- the tile leaves through the copy engine
@@ -267,10 +270,10 @@ dgemm_dmma_wsb_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
         for (int half = 0; half < 2; ++half)
 #pragma unroll
           for (int np = 0; np < 2; ++np) {
-            // chunk 2t: columns 4t, 4t+1; chunk 2t+1: columns 4t+2, 4t+3
+            // first piece: columns 4t, 4t+1; second: columns 4t+2, 4t+3
             const double lo0 = acc[mt][2 * np][2 * half], lo1 = acc[mt][2 * np + 1][2 * half];
             const double hi0 = acc[mt][2 * np][2 * half + 1], hi1 = acc[mt][2 * np + 1][2 * half + 1];
-            const uint32_t row = c_lane + (uint32_t)np * WsBulkCfg::C_BOX_BYTES + (uint32_t)(16 * mt + 8 * half) * 128u;
+            const uint32_t row = c_lane + (uint32_t)np * 128u + (uint32_t)((16 * mt + 8 * half) * WsBulkCfg::C_ROW_BYTES);
             ptx::sts128(row + ch_first, swap ? hi0 : lo0, swap ? hi1 : lo1);
             ptx::sts128(row + ch_second, swap ? lo0 : hi0, swap ? lo1 : hi1);
           }

@@ -151,18 +151,15 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
       : "memory");
 }
 
-// ---- TMA from shared to global memory (tiled; out-of-range parts of the box are clipped) ----------
-// The box at `src` (laid out as the tensor map's swizzle mode says) is added to, or stored over, the
-// tile of the tensor at (x, y). Asynchronous; completion is tracked per thread in bulk groups.
-__device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap* map, int x, int y, uint32_t src) {
-  asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%1, %2}], [%3];"
-               ::"l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(src)
-               : "memory");
+// ---- bulk copies from shared to global memory ----------------------------------------------------
+// Asynchronous; completion is tracked per thread in bulk groups.
+// `bytes` contiguous bytes at `src` (shared, 16-byte aligned) are added to, or stored over, the
+// doubles at `dst` (global, 16-byte aligned); `bytes` a multiple of 16.
+__device__ __forceinline__ void bulk_reduce_add_f64(double* dst, uint32_t src, uint32_t bytes) {
+  asm volatile("cp.reduce.async.bulk.global.shared::cta.bulk_group.add.f64 [%0], [%1], %2;" ::"l"(dst), "r"(src), "r"(bytes) : "memory");
 }
-__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, int x, int y, uint32_t src) {
-  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%1, %2}], [%3];"
-               ::"l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(src)
-               : "memory");
+__device__ __forceinline__ void bulk_store(double* dst, uint32_t src, uint32_t bytes) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(src), "r"(bytes) : "memory");
 }
 __device__ __forceinline__ void bulk_commit_group() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 // All bulk groups of this thread have finished READING their shared-memory source (it may be reused).

@@ -60,7 +60,7 @@ CONFIGS: Dict[str, Config] = {
     "generic": Config("generic", 2, 16, 64, 128, 2, 0.880, needs_tma=False),
     "cluster": Config("cluster", 5, 0, 64, 128, 2, 0.775),
     # C never enters the SM; what the arithmetic waits for is its own stores into the tile buffer
-    "bulk": Config("bulk", 10, 0, 128, 128, 1, 0.955, epilogue_exposed=0.22),
+    "bulk": Config("bulk", 10, 0, 128, 128, 1, 0.955, epilogue_exposed=0.08),
 }
 
 KBLOCK_ALONE_US = 1.35   # one k-block of a 64 x 128 tile on an SM the CTA has to itself (measured, long K)

@@ -35,7 +35,9 @@ def _defaults():
     ((4096, 4096, 4096), V_WS, 128, 128, 64),
     ((16384, 16384, 64), V_WSB, 128, 128, 64),     # many tiles of few k-blocks: the epilogue leaves through the copy engine
     ((16384, 16384, 256), V_WSB, 128, 128, 64),
-    ((16384, 16384, 1024), V_WS, 128, 128, 64),    # ... up to 48 k-blocks per tile
+    ((16384, 16384, 2048), V_WSB, 128, 128, 64),
+    ((16384, 16384, 4096), V_WS, 128, 128, 64),    # ... up to 128 k-blocks per tile
+    ((2560, 2560, 64), V_WSB, 128, 128, 64),       # ... and from two waves of tiles
     ((2048, 2048, 64), V_WS, 64, 128, 64),         # few tiles, K < 256: the warp-specialised kernel with two CTAs per SM
     ((2088, 2048, 2048), V_WS, 64, 128, 64),       # M just above a multiple of 64 rows: 64-row tiles, two CTAs per SM
     ((1600, 8192, 8192), V_TMA, 64, 128, 64),      # the same on a long problem: inline kernel

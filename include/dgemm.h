@@ -64,7 +64,7 @@ enum {
   DGEMM_VARIANT_GENERIC_DFMA = 9, /* the same inner kernel under the GENERIC staging: any alignment          */
   DGEMM_VARIANT_TMA_WS_BULK = 10, /* as TMA_WS on 128 x 128 tiles with five stages and the epilogue done by the
                                     copy engine: the accumulators go to a tile buffer in shared memory and
-                                    leave as a tiled bulk reduce (add) into C, or a bulk store when beta == 0;
+                                    leave row by row as bulk reduces (add) into C, or bulk stores when beta == 0;
                                     C is never loaded into the SM. Needs, besides the TMA conditions, a
                                     16-byte aligned C with even ldc and beta == 0 or 1. What AUTO uses for
                                     large problems with a short K (rank-k updates)                        */

@@ -1,4 +1,4 @@
-"""The warp-specialised kernel whose epilogue leaves through the copy engine (tiled bulk reduce into C,
+"""The warp-specialised kernel whose epilogue leaves through the copy engine (bulk reduce into C row by row,
 or bulk store for beta == 0), forced on shapes of every kind and as the library's own choice on
 rank-k updates. Needs a B200. Everything is compared with the CPU oracle: bit for bit on
 integer-valued data, within the bound of the other parity tests on real data."""
@@ -14,7 +14,8 @@ pytestmark = pytest.mark.gpu
 
 BULK = dg.DGEMM_VARIANT_TMA_WS_BULK
 
-# ragged in every dimension; edge tiles in M and N are clipped by the copy engine
+# ragged in every dimension: rows beyond M are not sent, the tiles of a ragged last tile column are
+# added to C by the arithmetic warps themselves
 SHAPES = [(1, 2, 1), (17, 14, 11), (127, 130, 47), (128, 128, 16), (129, 126, 17), (130, 260, 33), (257, 132, 100),
           (200, 300, 1), (1000, 32, 600), (513, 34, 64), (1000, 1538, 777), (640, 384, 2048), (2304, 2304, 64)]
 
